@@ -1,0 +1,411 @@
+/*
+ * CPU oracle for GPU-thread-driven demand paging (GPUVM, arXiv 2411.05309).
+ *
+ * TEST INFRASTRUCTURE ONLY.  Plain, slow, single-threaded C that shares no code
+ * with the CUDA path.  Only the test-suite, the smoke check and the benchmark's
+ * CPU-baseline leg may call it; the product never does.
+ *
+ * Two parts.
+ *
+ *  (R) Results.  The paging runtime is a cache in front of host memory
+ *      (Section 3.1, Fig. 2: a thread computes page number and offset, consults
+ *      the page table, and reads or writes the data in the frame), so what a
+ *      workload computes through it equals what the same workload computes
+ *      directly on the host arrays.  The *_direct functions are those plain
+ *      definitions.
+ *
+ *  (P) Paging replay.  A sequential model of the runtime's bookkeeping that
+ *      takes one access at a time, in program order: address split and
+ *      page-table lookup (Fig. 2 steps 1-2), frame ring with a single head
+ *      cursor (Section 3.3 "Eviction scheme", Fig. 4), eviction of the frame
+ *      under the cursor, write-back of the victim, fetch of the new page.  Two
+ *      policies: FIFO, which is the ring of the paper, and clock/second chance,
+ *      which adds one reference bit per frame.  A dirty bit per frame decides
+ *      whether a victim is copied back.  With move_bytes on, the replay owns a
+ *      private frame buffer and every load and store of the paged workloads goes
+ *      through it, so lost write-backs show up as wrong host contents.
+ *
+ * Readings where the paper is silent: a write miss fetches the page first; the
+ * newly installed page has its reference bit set; the cursor moves past a frame
+ * when that frame is filled; a hit sets the reference bit and, for a write, the
+ * dirty bit.
+ *
+ * Pins (see tests): textbook reference strings with known FIFO and OPT fault
+ * counts, a queue-formulated second-chance model, Belady lower bound, compulsory
+ * misses, capacity, byte-exact host contents after flush, library BFS.
+ */
+#include <stdint.h>
+#include <stddef.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------ (R) -- */
+
+/* Streaming read-reduce: S = sum of a[i] as 64-bit integers. */
+int64_t orc_stream_sum_i32_direct(const int32_t *a, uint64_t n)
+{
+    int64_t s = 0;
+    for (uint64_t i = 0; i < n; ++i) s += (int64_t)a[i];
+    return s;
+}
+
+/*
+ * Random gather, one sum per block of `block` consecutive indices.
+ *   fsum[b] = binary32( sum over the block, accumulated in binary64, index order )
+ *   bsum[b] = sum over the block of the raw 32-bit patterns of the gathered
+ *             values, taken as unsigned, accumulated in int64 (an exact,
+ *             order-free fingerprint of WHICH elements were gathered).
+ */
+void orc_gather_block_sums_direct(const float *x, const int64_t *idx, uint64_t n_idx,
+                                  uint64_t block, float *fsum, int64_t *bsum)
+{
+    uint64_t nb = (n_idx + block - 1) / block;
+    for (uint64_t b = 0; b < nb; ++b) {
+        double acc = 0.0;
+        int64_t bits = 0;
+        uint64_t end = (b + 1) * block < n_idx ? (b + 1) * block : n_idx;
+        for (uint64_t k = b * block; k < end; ++k) {
+            float v = x[idx[k]];
+            uint32_t u;
+            memcpy(&u, &v, 4);
+            acc += (double)v;
+            bits += (int64_t)u;
+        }
+        fsum[b] = (float)acc;
+        bsum[b] = bits;
+    }
+}
+
+/* Hop distance from `source` over a directed CSR graph; -1 when unreachable. */
+void orc_bfs_levels_direct(const int64_t *row_off, const int32_t *col, uint64_t nv,
+                           uint64_t source, int32_t *level)
+{
+    for (uint64_t v = 0; v < nv; ++v) level[v] = -1;
+    if (source >= nv) return;
+    uint64_t *queue = (uint64_t *)malloc(nv * sizeof(uint64_t));
+    uint64_t head = 0, tail = 0;
+    level[source] = 0;
+    queue[tail++] = source;
+    while (head < tail) {
+        uint64_t u = queue[head++];
+        for (int64_t e = row_off[u]; e < row_off[u + 1]; ++e) {
+            int32_t v = col[e];
+            if (level[v] < 0) {
+                level[v] = level[u] + 1;
+                queue[tail++] = (uint64_t)v;
+            }
+        }
+    }
+    free(queue);
+}
+
+/* c[i] = a[i] + b[i], one correctly rounded binary32 addition per element. */
+void orc_vadd_f32_direct(const float *a, const float *b, float *c, uint64_t n)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        volatile float s = a[i] + b[i];
+        c[i] = s;
+    }
+}
+
+/*
+ * Embedding bag: out[g][d] = ((0 + t[r0][d]) + t[r1][d]) + ... in binary32, rows
+ * of bag g taken in list order (rows[g*bag .. g*bag+bag-1]).
+ */
+void orc_embag_f32_direct(const float *table, uint64_t dims, const int64_t *rows,
+                          uint64_t n_bags, uint64_t bag, float *out)
+{
+    for (uint64_t g = 0; g < n_bags; ++g)
+        for (uint64_t d = 0; d < dims; ++d) {
+            volatile float acc = 0.0f;
+            for (uint64_t k = 0; k < bag; ++k)
+                acc = acc + table[(uint64_t)rows[g * bag + k] * dims + d];
+            out[g * dims + d] = acc;
+        }
+}
+
+/* ------------------------------------------------------------------ (P) -- */
+
+enum { ORC_FIFO = 0, ORC_CLOCK = 1 };
+#define ORC_NONE UINT64_MAX
+
+typedef struct {
+    uint8_t *host;            /* backing store: holds every page (Fig. 4, left)   */
+    uint64_t bytes;
+    uint64_t page_bytes;
+    uint64_t n_pages;         /* ceil(bytes / page_bytes)                          */
+    uint64_t n_frames;
+    int policy;
+    int move_bytes;
+    uint64_t *map;            /* page table: page -> frame or ORC_NONE             */
+    uint64_t *frame_page;     /* page map of the ring: frame -> page or ORC_NONE   */
+    uint8_t *frame_dirty;
+    uint8_t *frame_ref;
+    uint8_t *frames;          /* private frame buffer (move_bytes only)            */
+    uint64_t hand;            /* the ring's head cursor                            */
+    /* counters */
+    uint64_t accesses, hits, faults, evictions, writebacks;
+    uint64_t bytes_in, bytes_out, resident, max_resident, hand_steps;
+} orc_pager;
+
+static uint64_t page_len(const orc_pager *p, uint64_t vpn)
+{
+    uint64_t start = vpn * p->page_bytes;
+    uint64_t left = p->bytes - start;
+    return left < p->page_bytes ? left : p->page_bytes;
+}
+
+orc_pager *orc_pager_create(void *host, uint64_t bytes, uint64_t page_bytes,
+                            uint64_t n_frames, int policy, int move_bytes)
+{
+    if (!host || !bytes || !page_bytes || !n_frames) return NULL;
+    orc_pager *p = (orc_pager *)calloc(1, sizeof(orc_pager));
+    p->host = (uint8_t *)host;
+    p->bytes = bytes;
+    p->page_bytes = page_bytes;
+    p->n_pages = (bytes + page_bytes - 1) / page_bytes;
+    p->n_frames = n_frames;
+    p->policy = policy;
+    p->move_bytes = move_bytes;
+    p->map = (uint64_t *)malloc(p->n_pages * sizeof(uint64_t));
+    p->frame_page = (uint64_t *)malloc(n_frames * sizeof(uint64_t));
+    p->frame_dirty = (uint8_t *)calloc(n_frames, 1);
+    p->frame_ref = (uint8_t *)calloc(n_frames, 1);
+    for (uint64_t i = 0; i < p->n_pages; ++i) p->map[i] = ORC_NONE;
+    for (uint64_t i = 0; i < n_frames; ++i) p->frame_page[i] = ORC_NONE;
+    if (move_bytes) p->frames = (uint8_t *)malloc(n_frames * page_bytes);
+    return p;
+}
+
+void orc_pager_destroy(orc_pager *p)
+{
+    if (!p) return;
+    free(p->map); free(p->frame_page); free(p->frame_dirty); free(p->frame_ref);
+    free(p->frames); free(p);
+}
+
+/* Copy a victim back to the host if it was written, then drop its mapping. */
+static void evict_frame(orc_pager *p, uint64_t f)
+{
+    uint64_t q = p->frame_page[f];
+    if (p->frame_dirty[f]) {
+        p->writebacks++;
+        p->bytes_out += page_len(p, q);
+        if (p->move_bytes)
+            memcpy(p->host + q * p->page_bytes, p->frames + f * p->page_bytes, page_len(p, q));
+    }
+    p->evictions++;
+    p->map[q] = ORC_NONE;
+    p->frame_page[f] = ORC_NONE;
+    p->frame_dirty[f] = 0;
+    p->frame_ref[f] = 0;
+    p->resident--;
+}
+
+/* One access in program order.  Returns the frame that now holds the page. */
+uint64_t orc_pager_access(orc_pager *p, uint64_t vpn, int is_write)
+{
+    p->accesses++;
+    uint64_t f = p->map[vpn];
+    if (f != ORC_NONE) {                      /* Fig. 2 step 2: resident */
+        p->hits++;
+        p->frame_ref[f] = 1;
+        if (is_write) p->frame_dirty[f] = 1;
+        return f;
+    }
+    p->faults++;
+    for (;;) {                                /* take the next ring slot */
+        f = p->hand;
+        p->hand = (p->hand + 1) % p->n_frames;
+        p->hand_steps++;
+        if (p->frame_page[f] == ORC_NONE) break;
+        if (p->policy == ORC_CLOCK && p->frame_ref[f]) {
+            p->frame_ref[f] = 0;              /* second chance */
+            continue;
+        }
+        evict_frame(p, f);
+        break;
+    }
+    p->bytes_in += page_len(p, vpn);
+    if (p->move_bytes)
+        memcpy(p->frames + f * p->page_bytes, p->host + vpn * p->page_bytes, page_len(p, vpn));
+    p->map[vpn] = f;
+    p->frame_page[f] = vpn;
+    p->frame_ref[f] = 1;
+    p->frame_dirty[f] = is_write ? 1 : 0;
+    p->resident++;
+    if (p->resident > p->max_resident) p->max_resident = p->resident;
+    return f;
+}
+
+/* Replay a trace of (page, is_write) records. */
+void orc_pager_replay(orc_pager *p, const uint64_t *vpn, const uint8_t *is_write, uint64_t n)
+{
+    for (uint64_t i = 0; i < n; ++i) orc_pager_access(p, vpn[i], is_write ? is_write[i] : 0);
+}
+
+/* Write every dirty frame back; mappings stay. */
+void orc_pager_flush(orc_pager *p)
+{
+    for (uint64_t f = 0; f < p->n_frames; ++f)
+        if (p->frame_page[f] != ORC_NONE && p->frame_dirty[f]) {
+            uint64_t q = p->frame_page[f];
+            p->writebacks++;
+            p->bytes_out += page_len(p, q);
+            if (p->move_bytes)
+                memcpy(p->host + q * p->page_bytes, p->frames + f * p->page_bytes, page_len(p, q));
+            p->frame_dirty[f] = 0;
+        }
+}
+
+/* counters out: accesses, hits, faults, evictions, writebacks, bytes_in,
+ * bytes_out, resident, max_resident, hand_steps */
+void orc_pager_counters(const orc_pager *p, uint64_t out[10])
+{
+    out[0] = p->accesses; out[1] = p->hits; out[2] = p->faults; out[3] = p->evictions;
+    out[4] = p->writebacks; out[5] = p->bytes_in; out[6] = p->bytes_out;
+    out[7] = p->resident; out[8] = p->max_resident; out[9] = p->hand_steps;
+}
+
+/* Structural invariants of the replay's tables; 0 when they hold. */
+int orc_pager_check(const orc_pager *p)
+{
+    uint64_t mapped = 0, used = 0;
+    for (uint64_t v = 0; v < p->n_pages; ++v)
+        if (p->map[v] != ORC_NONE) {
+            mapped++;
+            if (p->map[v] >= p->n_frames) return 1;
+            if (p->frame_page[p->map[v]] != v) return 2;
+        }
+    for (uint64_t f = 0; f < p->n_frames; ++f)
+        if (p->frame_page[f] != ORC_NONE) {
+            used++;
+            if (p->frame_page[f] >= p->n_pages) return 3;
+            if (p->map[p->frame_page[f]] != f) return 4;
+        }
+    if (mapped != used || mapped != p->resident || mapped > p->n_frames) return 5;
+    return 0;
+}
+
+/* Element accessors through the pager.  An element never straddles a page
+ * because page sizes are multiples of the element size and arrays start on page
+ * boundaries.  Without move_bytes the data is read/written in place. */
+static void paged_load(orc_pager *p, uint64_t byte_off, void *dst, uint64_t n)
+{
+    uint64_t vpn = byte_off / p->page_bytes, off = byte_off % p->page_bytes;
+    uint64_t f = orc_pager_access(p, vpn, 0);
+    if (p->move_bytes) memcpy(dst, p->frames + f * p->page_bytes + off, n);
+    else memcpy(dst, p->host + byte_off, n);
+}
+
+static void paged_store(orc_pager *p, uint64_t byte_off, const void *src, uint64_t n)
+{
+    uint64_t vpn = byte_off / p->page_bytes, off = byte_off % p->page_bytes;
+    uint64_t f = orc_pager_access(p, vpn, 1);
+    if (p->move_bytes) memcpy(p->frames + f * p->page_bytes + off, src, n);
+    else memcpy(p->host + byte_off, src, n);
+}
+
+/* The five workloads, element by element in canonical program order, every
+ * paged operand going through the pager.  Offsets are byte offsets of the arrays
+ * inside the backing store. */
+
+int64_t orc_stream_sum_i32_paged(orc_pager *p, uint64_t a_off, uint64_t n)
+{
+    int64_t s = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        int32_t v;
+        paged_load(p, a_off + 4 * i, &v, 4);
+        s += (int64_t)v;
+    }
+    return s;
+}
+
+void orc_gather_block_sums_paged(orc_pager *p, uint64_t x_off, const int64_t *idx,
+                                 uint64_t n_idx, uint64_t block, float *fsum, int64_t *bsum)
+{
+    uint64_t nb = (n_idx + block - 1) / block;
+    for (uint64_t b = 0; b < nb; ++b) {
+        double acc = 0.0;
+        int64_t bits = 0;
+        uint64_t end = (b + 1) * block < n_idx ? (b + 1) * block : n_idx;
+        for (uint64_t k = b * block; k < end; ++k) {
+            float v;
+            uint32_t u;
+            paged_load(p, x_off + 4 * (uint64_t)idx[k], &v, 4);
+            memcpy(&u, &v, 4);
+            acc += (double)v;
+            bits += (int64_t)u;
+        }
+        fsum[b] = (float)acc;
+        bsum[b] = bits;
+    }
+}
+
+/* Level-synchronous BFS: level by level, vertices ascending inside a level; per
+ * vertex row_off[v], row_off[v+1], then its edge range ascending.  The level
+ * array is ordinary (unpaged) memory. */
+void orc_bfs_levels_paged(orc_pager *p, uint64_t off_off, uint64_t col_off, uint64_t nv,
+                          uint64_t source, int32_t *level)
+{
+    for (uint64_t v = 0; v < nv; ++v) level[v] = -1;
+    if (source >= nv) return;
+    level[source] = 0;
+    for (int32_t cur = 0;; ++cur) {
+        int found = 0;
+        for (uint64_t u = 0; u < nv; ++u) {
+            if (level[u] != cur) continue;
+            int64_t lo, hi;
+            paged_load(p, off_off + 8 * u, &lo, 8);
+            paged_load(p, off_off + 8 * (u + 1), &hi, 8);
+            for (int64_t e = lo; e < hi; ++e) {
+                int32_t v;
+                paged_load(p, col_off + 4 * (uint64_t)e, &v, 4);
+                if (level[v] < 0) { level[v] = cur + 1; found = 1; }
+            }
+        }
+        if (!found) break;
+    }
+}
+
+void orc_vadd_f32_paged(orc_pager *p, uint64_t a_off, uint64_t b_off, uint64_t c_off, uint64_t n)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        float a, b;
+        paged_load(p, a_off + 4 * i, &a, 4);
+        paged_load(p, b_off + 4 * i, &b, 4);
+        volatile float s = a + b;
+        float c = s;
+        paged_store(p, c_off + 4 * i, &c, 4);
+    }
+}
+
+void orc_embag_f32_paged(orc_pager *p, uint64_t t_off, uint64_t dims, const int64_t *rows,
+                         uint64_t n_bags, uint64_t bag, float *out)
+{
+    for (uint64_t g = 0; g < n_bags; ++g) {
+        for (uint64_t d = 0; d < dims; ++d) out[g * dims + d] = 0.0f;
+        for (uint64_t k = 0; k < bag; ++k) {
+            uint64_t r = (uint64_t)rows[g * bag + k];
+            for (uint64_t d = 0; d < dims; ++d) {
+                float v;
+                paged_load(p, t_off + 4 * (r * dims + d), &v, 4);
+                volatile float s = out[g * dims + d] + v;
+                out[g * dims + d] = s;
+            }
+        }
+    }
+}
+
+/* Oversubscription level, Eq. 1: workload size / available GPU memory - 1. */
+double orc_oversubscription_level(double workload_bytes, double gpu_bytes)
+{
+    return workload_bytes / gpu_bytes - 1.0;
+}
+
+/* Queue depth by Little's law as used in Section 3.2: latency x throughput /
+ * request size, all in binary units. */
+double orc_queue_depth(double latency_s, double bytes_per_s, double request_bytes)
+{
+    return latency_s * bytes_per_s / request_bytes;
+}
