@@ -1,0 +1,188 @@
+/*
+ * gpuvm.h -- host C ABI of the GPU-thread-driven demand-paging runtime.
+ *
+ * The runtime keeps a large array in host memory ("backing store", the paper's
+ * host region that holds every page, Section 3.3 / Fig. 4) and lets GPU threads
+ * access it through a fixed pool of page frames in device memory.  All memory
+ * is set up before any kernel runs (Section 3.3: no OS work at run time;
+ * Section 4 "Constructing Virtual Memory"); page table, frame ring and counters
+ * live in device memory and are modified only by GPU threads (Section 3.3 "Page
+ * mapping").  The paper moves pages with an RDMA NIC; here the same GPU threads
+ * copy pages between the pool and pinned, mapped host memory.
+ *
+ * Conventions
+ *   - every function returns 0 on success or a negative gpuvm_status; nothing
+ *     throws, aborts or traps.  gpuvm_strerror() names a status; the last CUDA
+ *     error seen by a handle is kept in gpuvm_last_cuda_error().
+ *   - "device pointer" means an address valid in kernels on the current CUDA
+ *     device; "host pointer" an address valid on the CPU.
+ *   - streams are passed as void* (a cudaStream_t; NULL is the default stream).
+ *   - a handle belongs to the CUDA device that was current in gpuvm_create().
+ *   - there is no CPU fallback: without a CUDA device every call fails.
+ */
+#ifndef GPUVM_H
+#define GPUVM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gpuvm_handle *gpuvm_t;
+
+typedef enum gpuvm_status {
+    GPUVM_OK = 0,
+    GPUVM_E_ARG = -1,        /* NULL out pointer, zero size, bad handle               */
+    GPUVM_E_PAGE = -2,       /* page_bytes not a power of two in [16, 2^30], or more
+                                than 2^31-2 pages                                     */
+    GPUVM_E_POOL = -3,       /* pool_bytes zero, not a multiple of page_bytes, or
+                                more than 2^31-2 frames                               */
+    GPUVM_E_ALIGN = -4,      /* host_backing not 16-byte aligned or bytes % 16 != 0   */
+    GPUVM_E_PIN = -5,        /* pinning / mapping the host backing failed             */
+    GPUVM_E_ALLOC = -6,      /* device allocation failed                              */
+    GPUVM_E_CUDA = -7,       /* any other CUDA runtime failure                        */
+    GPUVM_E_TIMEOUT = -8,    /* a device-side wait ran out (sticky, see gpuvm_stats)  */
+    GPUVM_E_RANGE = -9,      /* a device accessor was given an offset past the end    */
+    GPUVM_E_INVARIANT = -10, /* gpuvm_check found a broken page-table invariant       */
+    GPUVM_E_NODEVICE = -11   /* no CUDA device                                        */
+} gpuvm_status;
+
+/* Eviction policy of the frame ring (Section 3.3 "Eviction scheme").
+ * FIFO is the paper's ring: the frame under the head cursor is the victim.
+ * CLOCK adds one reference bit per page: a referenced page is passed over once.
+ * Under both, a page whose reference counter is not zero is never evicted. */
+enum { GPUVM_POLICY_FIFO = 0, GPUVM_POLICY_CLOCK = 1 };
+
+/*
+ * Device view: a plain struct passed BY VALUE to kernels (the role of the
+ * paper's array-like gpuvm<T> object of Listing 1).  All pointers are device
+ * pointers; `host` is the device-visible address of the backing store.
+ */
+typedef struct gpuvm_dev {
+    unsigned long long *pte;   /* page table, one 64-bit entry per page                 */
+    unsigned int *frame_vpn;   /* frame ring: page held by each frame                   */
+    unsigned char *pool;       /* n_frames * page_bytes of device memory                */
+    unsigned char *host;       /* backing store (pinned host memory, mapped)            */
+    unsigned long long *ctl;   /* head cursor, sticky error, counters                   */
+    unsigned long long bytes;  /* size of the backing store                             */
+    unsigned long long n_pages;
+    unsigned int n_frames;
+    unsigned int page_shift;   /* log2(page_bytes)                                      */
+    unsigned int policy;       /* GPUVM_POLICY_*                                        */
+    unsigned int spin_limit_us;/* upper bound of every device-side wait                 */
+} gpuvm_dev_t;
+
+/* Counters accumulated by GPU threads since the last gpuvm_reset(). */
+typedef struct gpuvm_stats {
+    uint64_t faults;          /* pages migrated host -> pool (one per serviced fault)  */
+    uint64_t hits;            /* warp-level page requests that found the page resident */
+    uint64_t waits;           /* warp-level requests that joined a fault in flight
+                                 (inter-warp coalescing, Section 3.3)                  */
+    uint64_t lanes_coalesced; /* threads that shared their warp leader's request
+                                 (intra-warp coalescing)                               */
+    uint64_t evictions;       /* pages unmapped to make room                           */
+    uint64_t writebacks;      /* dirty victims copied pool -> host while running       */
+    uint64_t flush_writebacks;/* dirty pages copied by gpuvm_flush                     */
+    uint64_t bytes_in;        /* host -> pool bytes                                    */
+    uint64_t bytes_out;       /* pool -> host bytes (evictions + flush)                */
+    uint64_t hand_steps;      /* frame-ring slots inspected                            */
+    uint64_t retries;         /* wait-loop rounds that made no progress                */
+    uint64_t resident;        /* pages resident now                                    */
+    int32_t error;            /* sticky device error: 0, GPUVM_E_TIMEOUT, GPUVM_E_RANGE*/
+    uint32_t reserved;
+    uint64_t error_page;      /* page number the first error was raised for            */
+} gpuvm_stats_t;
+
+/* Result of the post-run invariant check. */
+typedef struct gpuvm_check {
+    uint64_t resident;        /* page-table entries in the VALID state                 */
+    uint64_t frames_used;     /* frames that name a page                               */
+    uint64_t bad_state;       /* entries left BUSY / EVICTING, or INVALID with stray bits */
+    uint64_t bad_refcount;    /* entries whose reference counter is not zero           */
+    uint64_t bad_backref;     /* VALID entry whose frame does not name it back, or a
+                                 frame whose page is not VALID in that frame           */
+    uint64_t bad_range;       /* frame number or page number out of range              */
+    uint64_t dirty;           /* resident pages still marked dirty                     */
+} gpuvm_check_t;
+
+/*
+ * Create a paged view of `bytes` bytes of host memory with pages of `page_bytes`
+ * and a device pool of `pool_bytes` (Section 4 "Constructing Virtual Memory";
+ * Section 3.3: GPU memory is a fixed ring of page frames).
+ *   out          host pointer, receives the handle.
+ *   host_backing host pointer, 16-byte aligned, owned by the caller and kept alive
+ *                until gpuvm_destroy.  Pageable memory is pinned and mapped by the
+ *                library (and unpinned at destroy); memory that is already pinned
+ *                is used as is.  NULL: the library allocates pinned memory itself
+ *                (see gpuvm_host_ptr) and frees it at destroy.
+ *   bytes        multiple of 16.  The last page may be partial.
+ *   page_bytes   power of two, 16 .. 2^30.
+ *   pool_bytes   multiple of page_bytes, at least one page.
+ * Allocates page table, frame ring, counters and the pool with cudaMalloc and
+ * zeroes them.  Errors: GPUVM_E_ARG/PAGE/POOL/ALIGN are detected before any
+ * CUDA call; GPUVM_E_PIN, GPUVM_E_ALLOC, GPUVM_E_NODEVICE.
+ */
+int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_bytes,
+                 size_t pool_bytes);
+
+/* Flush dirty pages to the host, release device memory, unpin what create
+ * pinned, free what create allocated.  The handle is dead afterwards. */
+int gpuvm_destroy(gpuvm_t h);
+
+/* Synchronise the device and copy the counters to *out (host pointer).  Returns
+ * the sticky device error if one is set, else 0. */
+int gpuvm_stats(gpuvm_t h, gpuvm_stats_t *out);
+
+/* Copy the by-value device view to *out (host pointer). */
+int gpuvm_device_view(gpuvm_t h, gpuvm_dev_t *out);
+
+/* Host pointer of the backing store (the caller's, or the library's own). */
+void *gpuvm_host_ptr(gpuvm_t h);
+
+/* Write every dirty resident page back to the host on `stream` and clear the
+ * dirty bits; mappings stay.  Synchronises the stream before returning, so the
+ * host array is complete ("no dirty data is lost").  Must not run concurrently
+ * with kernels that use the handle. */
+int gpuvm_flush(gpuvm_t h, void *stream);
+
+/* Forget all mappings (without write-back), zero the counters and the error.
+ * Mappings otherwise persist across kernel launches (Section 4 "Multi-kernel
+ * support"). */
+int gpuvm_reset(gpuvm_t h);
+
+/* Run the invariant kernel: every resident page maps to exactly one frame and
+ * that frame names it back, occupancy <= capacity, nothing left in a transient
+ * state, all reference counters zero.  Fills *out (host pointer); returns
+ * GPUVM_E_INVARIANT if any bad_* count is non-zero. */
+int gpuvm_check(gpuvm_t h, gpuvm_check_t *out);
+
+/* Options.  policy: GPUVM_POLICY_*; spin_limit_us: bound of device-side waits
+ * (default 10 s).  Take effect for views fetched afterwards. */
+int gpuvm_set_policy(gpuvm_t h, int policy);
+int gpuvm_set_spin_limit_us(gpuvm_t h, unsigned int spin_limit_us);
+
+/* Largest number of simultaneously resident warps that can each hold
+ * `pins_per_warp` pages pinned without exhausting the pool (a warp that holds
+ * pins while faulting needs a free frame; Section 3.3: a frame is reused only
+ * when its reference counter is zero).  Accessors that hold at most one page at
+ * a time (gpuvm_read / gpuvm_write) are safe with any number of warps. */
+int gpuvm_safe_warps(gpuvm_t h, int pins_per_warp);
+
+/* Pages that must be in flight to keep a link of `bytes_per_s` busy at a fault
+ * round-trip of `latency_s` (Little's law as applied in Section 3.2). */
+double gpuvm_inflight_pages(double latency_s, double bytes_per_s, double page_bytes);
+
+/* Test hook: overwrite one page-table entry with `value` (host-side injection of
+ * a page that stays "being fetched" so that a bounded device wait can be seen to
+ * expire with an error status instead of hanging). */
+int gpuvm_debug_poke_pte(gpuvm_t h, uint64_t page, uint64_t value);
+
+const char *gpuvm_strerror(int status);
+int gpuvm_last_cuda_error(gpuvm_t h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPUVM_H */

@@ -1,0 +1,600 @@
+/*
+ * gpuvm_device.cuh -- device-side accessors of the demand-paging runtime.
+ *
+ * Include from CUDA code compiled for sm_100a.  A kernel receives a gpuvm_dev_t BY
+ * VALUE (the role of the paper's array-like object, Listing 1) and touches the
+ * paged array only through:
+ *
+ *   T     gpuvm_read <T>(vm, elem_index, base_byte_off)        pin, load, unpin
+ *   void  gpuvm_write<T>(vm, elem_index, value, base_byte_off) pin, mark dirty, store, unpin
+ *   void* gpuvm_ptr(vm, byte_off, mode, &token)                pin and hand out a frame pointer
+ *   void  gpuvm_release(vm, token)                             unpin what gpuvm_ptr pinned
+ *
+ * What happens on an access (Section 3.1, Fig. 2; Section 3.3):
+ *   1. address split: page number = byte offset >> page_shift, offset = the rest;
+ *   2. translate: the page-table entry is read; a resident page is used in place;
+ *   3. the threads of the warp that want the same page are grouped with
+ *      __match_any_sync over __activemask() and the lowest lane of each group acts
+ *      for it ("leader"); the reference counter of a page counts such warp-level
+ *      requests, not threads;
+ *   4. among the leaders of different warps only one gets to service a missing
+ *      page: the one whose atomicCAS turns the entry from INVALID to BUSY.  The
+ *      others have already added themselves to the entry's reference counter and
+ *      simply wait for the entry to become VALID; the page cannot be evicted
+ *      before they have used it because the counter is not zero;
+ *   5. the owner takes the next slot of the frame ring with an atomic add on the
+ *      head cursor.  A free slot is taken as is.  An occupied slot is passed over
+ *      when its page is in use (counter != 0) or, under the clock policy, when its
+ *      reference bit is set (the bit is cleared: second chance).  Otherwise the
+ *      occupant is evicted: its entry goes VALID -> EVICTING with a CAS on the exact
+ *      word, so a concurrent pin makes the CAS fail;
+ *   6. a dirty victim is copied back to the host by the whole warp, 16 bytes per
+ *      lane and instruction, followed by a system-scope fence; then its entry
+ *      becomes INVALID;
+ *   7. the warp copies the new page from the host into the frame the same way,
+ *      fences, and the owner publishes the entry (BUSY -> VALID, frame number,
+ *      reference bit) with one atomic XOR that leaves the counter untouched;
+ *   8. each thread performs its load or store in the frame; the leader drops the
+ *      group's reference with a release-ordered atomic.
+ *
+ * Rules for callers
+ *   - Any subset of a warp may call an accessor; lanes that call together are
+ *     handled together.
+ *   - gpuvm_read / gpuvm_write never hold a page while waiting for a frame and are
+ *     deadlock-free for any pool size and any number of warps.  gpuvm_ptr holds the
+ *     page until gpuvm_release: a warp must not hold more pages than
+ *     gpuvm_safe_warps() allows for the grid, and should ask for ONE page per call
+ *     (all calling lanes in the same page) whenever the pool may be small.
+ *   - Frames change identity when pages are evicted, so frame memory must be read
+ *     with gpuvm_load / gpuvm_load16 and written with gpuvm_store / gpuvm_store16
+ *     (L1-bypassing, device-coherent), never through a cached plain dereference.
+ *   - Every wait is bounded by vm.spin_limit_us.  When a wait runs out, or an offset
+ *     lies past the end of the array, a sticky error is recorded in the control
+ *     block (reported by gpuvm_stats), reads return zero, writes are dropped and
+ *     gpuvm_ptr returns nullptr.  Nothing traps.
+ *   - Offsets are 64-bit.  An element must not straddle a page (arrays start on a
+ *     multiple of the element size).
+ */
+#ifndef GPUVM_DEVICE_CUH
+#define GPUVM_DEVICE_CUH
+
+#include "gpuvm.h"
+
+#ifndef GPUVM_COUNT_HITS
+#define GPUVM_COUNT_HITS 1
+#endif
+
+namespace gpuvm {
+
+/* ---- page-table entry: [state:2 @60][dirty @57][ref @56][frame:32 @24][refcount:24 @0] */
+constexpr unsigned long long kRcMask = 0xFFFFFFull;
+constexpr int kFrameShift = 24;
+constexpr unsigned long long kFrameMask = 0xFFFFFFFFull << kFrameShift;
+constexpr unsigned long long kRef = 1ull << 56;
+constexpr unsigned long long kDirty = 1ull << 57;
+constexpr unsigned long long kStMask = 3ull << 60;
+constexpr unsigned long long kInvalid = 0ull;
+constexpr unsigned long long kBusy = 1ull << 60;
+constexpr unsigned long long kValid = 2ull << 60;
+constexpr unsigned long long kEvicting = 3ull << 60;
+
+/* ---- frame ring entry */
+constexpr unsigned int kFrameFree = 0xFFFFFFFFu;
+constexpr unsigned int kFrameLock = 0x80000000u;
+
+/* ---- control block (64-bit words) */
+constexpr int kCtlHand = 0;
+constexpr int kCtlErr = 1;
+constexpr int kCtlErrPage = 2;
+constexpr int kCtlCounters = 16;      /* kStatSlots slots of 16 words, one 128-byte line each */
+constexpr int kStatSlots = 32;
+constexpr int kCtlWords = kCtlCounters + kStatSlots * 16;
+enum Stat { kFaults = 0, kHits, kWaits, kLanes, kEvictions, kWritebacks, kFlushWritebacks,
+            kBytesIn, kBytesOut, kHandSteps, kRetries, kNumStats };
+
+enum Mode { kRead = 0, kWrite = 1 };
+
+struct Token {
+    unsigned long long vpn;
+    unsigned int group;      /* lanes that share the pin */
+    unsigned int leader;     /* 1 on the lane that owns the reference */
+};
+
+/* ------------------------------------------------------------ small primitives */
+
+__device__ __forceinline__ unsigned int lane_id()
+{
+    unsigned int r;
+    asm volatile("mov.u32 %0, %%laneid;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ unsigned int sm_id()
+{
+    unsigned int r;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ unsigned long long now_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int *p)
+{
+    unsigned int v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_relaxed_u32(unsigned int *p, unsigned int v)
+{
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+/* drop one reference; release order makes this thread's (and, through the warp
+ * barrier before it, its group's) frame accesses happen before the drop */
+__device__ __forceinline__ void unpin(unsigned long long *pte)
+{
+    asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(pte), "l"(~0ull) : "memory");
+}
+
+__device__ __forceinline__ void stat_add(const gpuvm_dev_t &vm, int kind, unsigned long long v)
+{
+    unsigned long long *p = vm.ctl + kCtlCounters + (sm_id() & (kStatSlots - 1)) * 16 + kind;
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__device__ __forceinline__ void set_error(const gpuvm_dev_t &vm, int code, unsigned long long vpn)
+{
+    if (atomicCAS(vm.ctl + kCtlErr, 0ull, (unsigned long long)(long long)code) == 0ull)
+        vm.ctl[kCtlErrPage] = vpn;
+}
+
+__device__ __forceinline__ bool has_error(const gpuvm_dev_t &vm)
+{
+    return ld_relaxed_u64(vm.ctl + kCtlErr) != 0ull;
+}
+
+/* 16-byte accesses.  Host side: system scope.  Frame side: device scope, no L1. */
+__device__ __forceinline__ uint4 ld_host16(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.relaxed.sys.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_host16(void *p, uint4 v)
+{
+    asm volatile("st.relaxed.sys.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                 ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+__device__ __forceinline__ uint4 ld_frame16(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_frame16(void *p, uint4 v)
+{
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                 ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+/* Bytes of page `vpn` that exist in the backing store, rounded up to 16. */
+__device__ __forceinline__ unsigned int page_len(const gpuvm_dev_t &vm, unsigned long long vpn)
+{
+    unsigned long long start = vpn << vm.page_shift;
+    unsigned long long left = vm.bytes - start;
+    unsigned long long page = 1ull << vm.page_shift;
+    return (unsigned int)(left < page ? left : page);
+}
+
+/*
+ * Warp-cooperative page copy (steps 6 and 7): the `n` calling lanes (rank 0..n-1)
+ * move `n16` 16-byte units; consecutive lanes touch consecutive units, U units per
+ * lane are in flight before the first store.
+ */
+template <int U, bool TO_HOST>
+__device__ __forceinline__ void warp_copy(unsigned char *dst, const unsigned char *src,
+                                          unsigned int n16, unsigned int rank, unsigned int n)
+{
+    const uint4 *s = reinterpret_cast<const uint4 *>(src);
+    uint4 *d = reinterpret_cast<uint4 *>(dst);
+    for (unsigned int base = rank; base < n16; base += n * U) {
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            unsigned int i = base + u * n;
+            if (i < n16) v[u] = TO_HOST ? ld_frame16(s + i) : ld_host16(s + i);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            unsigned int i = base + u * n;
+            if (i < n16) {
+                if (TO_HOST) st_host16(d + i, v[u]);
+                else st_frame16(d + i, v[u]);
+            }
+        }
+    }
+}
+
+/* ------------------------------------------------------------ fault machinery */
+
+enum LaneState { kNew = 0, kWait, kOwn, kReady, kDone, kFail };
+
+/*
+ * Leader only.  `w` is a fresh value of the entry that includes this group's
+ * reference.  VALID: note the reference/dirty bits, READY.  BUSY or EVICTING:
+ * WAIT.  INVALID: try to become the owner (step 4).
+ */
+__device__ __forceinline__ int advance(const gpuvm_dev_t &vm, unsigned long long *pte,
+                                       unsigned long long w, int mode, unsigned int &frame)
+{
+    for (;;) {
+        unsigned long long st = w & kStMask;
+        if (st == kValid) {
+            unsigned long long want = (mode == kWrite ? kDirty : 0ull) |
+                                      (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull);
+            if ((w & want) != want) atomicOr(pte, want);
+            frame = (unsigned int)((w & kFrameMask) >> kFrameShift);
+            return kReady;
+        }
+        if (st != kInvalid) return kWait;
+        unsigned long long seen = atomicCAS(pte, w, w | kBusy);
+        if (seen == w) return kOwn;
+        w = seen;                      /* somebody pinned, unpinned or took ownership */
+    }
+}
+
+/*
+ * Leader only, step 5: inspect up to `tries` ring slots.  On success the frame is
+ * exclusively ours (its ring entry is locked) and `victim` names the page that
+ * was in it and is now EVICTING (or ~0 when the frame was free).
+ */
+__device__ __forceinline__ bool try_claim(const gpuvm_dev_t &vm, unsigned long long vpn,
+                                          int tries, unsigned int &frame,
+                                          unsigned long long &victim, bool &victim_dirty)
+{
+    for (int t = 0; t < tries; ++t) {
+        unsigned long long ticket = atomicAdd(vm.ctl + kCtlHand, 1ull);
+        unsigned int h = (unsigned int)(ticket % vm.n_frames);
+        unsigned int e = ld_relaxed_u32(vm.frame_vpn + h);
+        if (e == kFrameFree) {
+            if (atomicCAS(vm.frame_vpn + h, kFrameFree, kFrameLock | (unsigned int)vpn) == kFrameFree) {
+                frame = h; victim = ~0ull; victim_dirty = false;
+                stat_add(vm, kHandSteps, t + 1);
+                return true;
+            }
+            continue;
+        }
+        if (e & kFrameLock) continue;                       /* in transition */
+        unsigned long long *qpte = vm.pte + e;
+        unsigned long long w = ld_relaxed_u64(qpte);
+        if ((w & kStMask) != kValid || (w & kRcMask) != 0ull ||
+            (unsigned int)((w & kFrameMask) >> kFrameShift) != h)
+            continue;                                       /* in use, or a stale ring read */
+        if (vm.policy == GPUVM_POLICY_CLOCK && (w & kRef)) {
+            atomicAnd(qpte, ~kRef);                         /* second chance */
+            continue;
+        }
+        unsigned long long evicting = (w & ~(kStMask | kRef)) | kEvicting;
+        if (atomicCAS(qpte, w, evicting) != w) continue;    /* lost against a pin or another evictor */
+        st_relaxed_u32(vm.frame_vpn + h, kFrameLock | (unsigned int)vpn);
+        frame = h; victim = e; victim_dirty = (w & kDirty) != 0ull;
+        stat_add(vm, kHandSteps, t + 1);
+        return true;
+    }
+    stat_add(vm, kHandSteps, tries);
+    return false;
+}
+
+/*
+ * Out-of-line part of every accessor: entered by all calling lanes (`active`)
+ * when at least one of their pages was not resident.  `w` is the entry value the
+ * group's leader got back from its pin (broadcast to the group).
+ *   op_bytes  0: hand out the frame (gpuvm_ptr); 1,2,4,8,16: load or store that
+ *             many bytes at `off` inside the page, value in `val`.
+ * Returns true when this lane's access was performed; `frame` is then its frame.
+ */
+static __device__ __noinline__ bool slow_path(const gpuvm_dev_t vm, unsigned long long vpn,
+                                              unsigned int off, int mode, int op_bytes,
+                                              unsigned int active, unsigned int group,
+                                              unsigned long long w, uint4 &val,
+                                              unsigned int &frame_out)
+{
+    const unsigned int lane = lane_id();
+    const unsigned int leader = __ffs(group) - 1;
+    const bool is_leader = lane == leader;
+    const unsigned int rank = __popc(active & ((1u << lane) - 1u));
+    const unsigned int nlanes = __popc(active);
+    unsigned long long *pte = vm.pte + vpn;
+    int st = kNew;
+    unsigned int frame = 0;
+    bool consumed = false, ok = false;
+    unsigned long long t_start = 0;
+    unsigned int sleep_ns = 32;
+
+    if (is_leader) {
+        st = advance(vm, pte, w, mode, frame);
+        if (st == kReady) { if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1); }
+        else if (st == kWait) stat_add(vm, kWaits, 1);
+    }
+
+    for (;;) {
+        bool progress = false;
+        /* waiting leaders look at their entry again */
+        if (is_leader && st == kWait) {
+            st = advance(vm, pte, ld_relaxed_u64(pte), mode, frame);
+            progress = st != kWait;
+        }
+        /* groups whose page is resident and pinned perform their access */
+        int gst = __shfl_sync(active, st, leader);
+        unsigned int gframe = __shfl_sync(active, frame, leader);
+        if (gst == kReady && !consumed) {
+            __threadfence();                                 /* acquire side of the publish */
+            unsigned char *p = vm.pool + ((unsigned long long)gframe << vm.page_shift) + off;
+            if (op_bytes == 16) {
+                if (mode == kWrite) st_frame16(p, val); else val = ld_frame16(p);
+            } else if (op_bytes == 8) {
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(val.x), "r"(val.y) : "memory");
+                else asm volatile("ld.relaxed.gpu.global.v2.u32 {%0,%1}, [%2];" : "=r"(val.x), "=r"(val.y) : "l"(p) : "memory");
+            } else if (op_bytes == 4) {
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(val.x) : "memory");
+                else asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(val.x) : "l"(p) : "memory");
+            } else if (op_bytes == 2) {
+                unsigned short h = (unsigned short)val.x;
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.u16 [%0], %1;" ::"l"(p), "h"(h) : "memory");
+                else { asm volatile("ld.relaxed.gpu.global.u16 %0, [%1];" : "=h"(h) : "l"(p) : "memory"); val.x = h; }
+            } else if (op_bytes == 1) {
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.u8 [%0], %1;" ::"l"(p), "r"(val.x) : "memory");
+                else asm volatile("ld.relaxed.gpu.global.u8 %0, [%1];" : "=r"(val.x) : "l"(p) : "memory");
+            }
+            consumed = true; ok = true; frame_out = gframe; progress = true;
+            if (op_bytes != 0) {                             /* step 8: drop the reference */
+                __syncwarp(group);
+                if (is_leader) { unpin(pte); st = kDone; }
+            } else if (is_leader) {
+                st = kDone;                                  /* reference kept until gpuvm_release */
+            }
+        }
+        /* owners take frames (step 5) and the warp moves the pages (steps 6, 7) */
+        bool claimed = false;
+        unsigned int h = 0;
+        unsigned long long victim = ~0ull;
+        bool vdirty = false;
+        if (is_leader && st == kOwn) claimed = try_claim(vm, vpn, 4, h, victim, vdirty);
+        unsigned int got = __ballot_sync(active, claimed);
+        while (got) {
+            const int L = __ffs(got) - 1;
+            got &= got - 1;
+            progress = true;
+            const unsigned int bh = __shfl_sync(active, h, L);
+            const unsigned long long bq = __shfl_sync(active, victim, L);
+            const int bd = __shfl_sync(active, (int)vdirty, L);
+            const unsigned long long bv = __shfl_sync(active, vpn, L);
+            unsigned char *fr = vm.pool + ((unsigned long long)bh << vm.page_shift);
+            if (bq != ~0ull) {
+                if (bd) {
+                    warp_copy<8, true>(vm.host + (bq << vm.page_shift), fr, page_len(vm, bq) >> 4, rank, nlanes);
+                    __threadfence_system();
+                    __syncwarp(active);
+                }
+                if ((int)lane == L) {
+                    /* EVICTING -> INVALID; frame and dirty bits return to zero, counter untouched */
+                    atomicXor(vm.pte + bq, kEvicting | ((unsigned long long)bh << kFrameShift) | (bd ? kDirty : 0ull));
+                    stat_add(vm, kEvictions, 1);
+                    if (bd) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, bq)); }
+                }
+            }
+            warp_copy<8, false>(fr, vm.host + (bv << vm.page_shift), page_len(vm, bv) >> 4, rank, nlanes);
+            __threadfence();
+            __syncwarp(active);
+            if ((int)lane == L) {
+                st_relaxed_u32(vm.frame_vpn + bh, (unsigned int)bv);
+                unsigned long long bits = (kBusy ^ kValid) | ((unsigned long long)bh << kFrameShift) |
+                                          (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull) |
+                                          (mode == kWrite ? kDirty : 0ull);
+                atomicXor(pte, bits);                        /* step 7: publish */
+                stat_add(vm, kFaults, 1);
+                stat_add(vm, kBytesIn, page_len(vm, bv));
+                st = kReady; frame = bh;
+            }
+        }
+        unsigned int pending = __ballot_sync(active, is_leader && st != kDone && st != kFail);
+        if (!pending) break;
+        if (__any_sync(active, progress)) { sleep_ns = 32; t_start = 0; continue; }
+        /* nothing moved: back off, and give up when the bound is reached */
+        unsigned long long t = now_ns();
+        if (t_start == 0) t_start = t;
+        bool expired = (t - t_start) > (unsigned long long)vm.spin_limit_us * 1000ull || has_error(vm);
+        expired = __any_sync(active, expired);
+        if (expired) {
+            if (is_leader && (st == kWait || st == kOwn)) {
+                set_error(vm, GPUVM_E_TIMEOUT, vpn);
+                if (st == kOwn) atomicXor(pte, kBusy);        /* BUSY -> INVALID */
+                unpin(pte);
+                st = kFail;
+            }
+            continue;                                        /* READY groups still finish */
+        }
+        if (lane == (unsigned int)(__ffs(active) - 1)) stat_add(vm, kRetries, 1);
+        __nanosleep(sleep_ns);
+        if (sleep_ns < 2048) sleep_ns *= 2;
+    }
+    return ok;
+}
+
+template <typename T> struct always_false { static constexpr bool value = false; };
+
+/* Shared front end: address split, grouping, optimistic pin (steps 1-3). */
+template <int OP_BYTES>
+__device__ __forceinline__ bool access(const gpuvm_dev_t &vm, unsigned long long byte_off, int mode,
+                                       uint4 &val, Token *tok, unsigned char **ptr_out)
+{
+    if (byte_off + (OP_BYTES ? OP_BYTES : 1) > vm.bytes) {
+        set_error(vm, GPUVM_E_RANGE, byte_off >> vm.page_shift);
+        return false;
+    }
+    const unsigned long long vpn = byte_off >> vm.page_shift;
+    const unsigned int off = (unsigned int)(byte_off & ((1ull << vm.page_shift) - 1ull));
+    const unsigned int active = __activemask();
+    const unsigned int group = __match_any_sync(active, vpn);
+    const unsigned int leader = __ffs(group) - 1;
+    const bool is_leader = lane_id() == leader;
+    unsigned long long *pte = vm.pte + vpn;
+    unsigned long long w = 0;
+    if (is_leader) {
+        w = atomicAdd(pte, 1ull) + 1ull;                     /* pin first, look afterwards */
+        if (group & (group - 1)) stat_add(vm, kLanes, __popc(group) - 1);
+    }
+    w = __shfl_sync(active, w, leader);
+    unsigned int frame = (unsigned int)((w & kFrameMask) >> kFrameShift);
+    const bool hit = (w & kStMask) == kValid;
+    if (__all_sync(active, hit)) {
+        if (is_leader) {
+            unsigned long long want = (mode == kWrite ? kDirty : 0ull) |
+                                      (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull);
+            if ((w & want) != want) atomicOr(pte, want);
+            if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1);
+        }
+        unsigned char *p = vm.pool + ((unsigned long long)frame << vm.page_shift) + off;
+        if (OP_BYTES == 0) {
+            __threadfence();
+            *ptr_out = p;
+        } else {
+            if (OP_BYTES == 16) { if (mode == kWrite) st_frame16(p, val); else val = ld_frame16(p); }
+            else if (OP_BYTES == 8) {
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(val.x), "r"(val.y) : "memory");
+                else asm volatile("ld.relaxed.gpu.global.v2.u32 {%0,%1}, [%2];" : "=r"(val.x), "=r"(val.y) : "l"(p) : "memory");
+            } else if (OP_BYTES == 4) {
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(val.x) : "memory");
+                else asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(val.x) : "l"(p) : "memory");
+            } else if (OP_BYTES == 2) {
+                unsigned short hv = (unsigned short)val.x;
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.u16 [%0], %1;" ::"l"(p), "h"(hv) : "memory");
+                else { asm volatile("ld.relaxed.gpu.global.u16 %0, [%1];" : "=h"(hv) : "l"(p) : "memory"); val.x = hv; }
+            } else {
+                if (mode == kWrite) asm volatile("st.relaxed.gpu.global.u8 [%0], %1;" ::"l"(p), "r"(val.x) : "memory");
+                else asm volatile("ld.relaxed.gpu.global.u8 %0, [%1];" : "=r"(val.x) : "l"(p) : "memory");
+            }
+            __syncwarp(group);
+            if (is_leader) unpin(pte);
+        }
+        if (tok) { tok->vpn = vpn; tok->group = group; tok->leader = is_leader; }
+        return true;
+    }
+    bool ok = slow_path(vm, vpn, off, mode, OP_BYTES, active, group, w, val, frame);
+    if (OP_BYTES == 0) {
+        *ptr_out = ok ? vm.pool + ((unsigned long long)frame << vm.page_shift) + off : nullptr;
+        if (tok) { tok->vpn = vpn; tok->group = group; tok->leader = ok && is_leader; }
+    }
+    return ok;
+}
+
+}  // namespace gpuvm
+
+/* ------------------------------------------------------------------ public API */
+
+typedef gpuvm::Token gpuvm_token;
+enum { GPUVM_READ = gpuvm::kRead, GPUVM_WRITE = gpuvm::kWrite };
+
+/* Element `elem` of an array of T that starts `base_off` bytes into the backing
+ * store (Listing 1: A[i] on the right-hand side). */
+template <typename T>
+__device__ __forceinline__ T gpuvm_read(const gpuvm_dev_t &vm, unsigned long long elem,
+                                        unsigned long long base_off = 0)
+{
+    static_assert(sizeof(T) == 1 || sizeof(T) == 2 || sizeof(T) == 4 || sizeof(T) == 8 || sizeof(T) == 16,
+                  "element size must be 1, 2, 4, 8 or 16 bytes");
+    uint4 v = make_uint4(0, 0, 0, 0);
+    gpuvm::access<(int)sizeof(T)>(vm, base_off + elem * sizeof(T), gpuvm::kRead, v, nullptr, nullptr);
+    T out;
+    memcpy(&out, &v, sizeof(T));
+    return out;
+}
+
+/* A[i] = value (Listing 1, left-hand side).  A write miss fetches the page first. */
+template <typename T>
+__device__ __forceinline__ void gpuvm_write(const gpuvm_dev_t &vm, unsigned long long elem, T value,
+                                            unsigned long long base_off = 0)
+{
+    static_assert(sizeof(T) == 1 || sizeof(T) == 2 || sizeof(T) == 4 || sizeof(T) == 8 || sizeof(T) == 16,
+                  "element size must be 1, 2, 4, 8 or 16 bytes");
+    uint4 v = make_uint4(0, 0, 0, 0);
+    memcpy(&v, &value, sizeof(T));
+    gpuvm::access<(int)sizeof(T)>(vm, base_off + elem * sizeof(T), gpuvm::kWrite, v, nullptr, nullptr);
+}
+
+/* Pin the page that holds `byte_off` and return the address of that byte inside
+ * its frame, valid up to the end of the page until gpuvm_release(token).
+ * mode GPUVM_WRITE marks the page dirty.  nullptr after an error. */
+__device__ __forceinline__ void *gpuvm_ptr(const gpuvm_dev_t &vm, unsigned long long byte_off, int mode,
+                                           gpuvm_token *token)
+{
+    uint4 v;
+    unsigned char *p = nullptr;
+    token->leader = 0; token->group = 0; token->vpn = 0;
+    gpuvm::access<0>(vm, byte_off, mode, v, token, &p);
+    return p;
+}
+
+/* Called by the same lanes that called gpuvm_ptr together. */
+__device__ __forceinline__ void gpuvm_release(const gpuvm_dev_t &vm, const gpuvm_token &token)
+{
+    if (token.group == 0) return;
+    __syncwarp(token.group);
+    if (token.leader) gpuvm::unpin(vm.pte + token.vpn);
+}
+
+/* Frame memory accessors (L1-bypassing, device-coherent). */
+__device__ __forceinline__ uint4 gpuvm_load16(const void *p) { return gpuvm::ld_frame16(p); }
+__device__ __forceinline__ void gpuvm_store16(void *p, uint4 v) { gpuvm::st_frame16(p, v); }
+
+template <typename T>
+__device__ __forceinline__ T gpuvm_load(const T *p)
+{
+    static_assert(sizeof(T) == 4 || sizeof(T) == 8, "4- or 8-byte elements");
+    T out;
+    if (sizeof(T) == 4) {
+        unsigned int v;
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        memcpy(&out, &v, 4);
+    } else {
+        unsigned long long v;
+        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+        memcpy(&out, &v, 8);
+    }
+    return out;
+}
+
+template <typename T>
+__device__ __forceinline__ void gpuvm_store(T *p, T value)
+{
+    static_assert(sizeof(T) == 4 || sizeof(T) == 8, "4- or 8-byte elements");
+    if (sizeof(T) == 4) {
+        unsigned int v;
+        memcpy(&v, &value, 4);
+        asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+    } else {
+        unsigned long long v;
+        memcpy(&v, &value, 8);
+        asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+    }
+}
+
+#endif /* GPUVM_DEVICE_CUH */

@@ -1,0 +1,117 @@
+/*
+ * gpuvm_workloads.h -- C ABI of the workload kernels written against the device
+ * accessors (gpuvm_device.cuh), and of their twins on plain device-accessible
+ * pointers (for the same kernels over cudaMallocManaged memory).
+ *
+ * Common rules
+ *   - `h` is a handle from gpuvm_create; *_off arguments are BYTE offsets of an
+ *     array inside its backing store, multiples of 16.
+ *   - d_* arguments are device pointers owned by the caller (results live in
+ *     ordinary device memory, only the large inputs are paged); `stream` is a
+ *     cudaStream_t passed as void* (NULL = default stream).
+ *   - calls enqueue work and return without synchronising unless stated; device
+ *     errors (a wait that ran out, an offset out of range) are sticky in the handle
+ *     and show up in gpuvm_stats().  Return value: 0 or a negative gpuvm_status.
+ *   - nothing here allocates device memory except gpuvm_bfs_csr (frontier queues,
+ *     freed before it returns).
+ */
+#ifndef GPUVM_WORKLOADS_H
+#define GPUVM_WORKLOADS_H
+
+#include "gpuvm.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/*
+ * Streaming read-reduce: *d_sum = sum of the n int32 values at a_off, as int64.
+ * One warp per page: the page is pinned once, read with 16-byte loads and released
+ * (the access pattern of the paper's transfer benchmark, Section 5.1: each warp is
+ * assigned a page, consecutive addresses).  d_sum: device int64, overwritten.
+ */
+int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void *stream);
+
+/*
+ * Random gather: for each block b of `block` consecutive indices,
+ *   d_fsum[b] = float( sum of x[idx[k]] accumulated in double )
+ *   d_bsum[b] = sum of the 32-bit patterns of the gathered values (int64, exact).
+ * x: fp32 array at x_off; d_idx: n_idx int64 element indices in device memory.
+ * One thread per index through gpuvm_read<float>; every warp may fault on up to
+ * 32 different pages at once (Section 3.3: intra- and inter-warp coalescing).
+ * d_fsum, d_bsum: ceil(n_idx / block) elements.  block <= 2^20.
+ */
+int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx, size_t block,
+                     float *d_fsum, int64_t *d_bsum, void *stream);
+
+/*
+ * Level-synchronous BFS over a CSR graph whose int64 row offsets (nv + 1 of them,
+ * at off_off) and int32 column indices (at col_off) are paged (Section 5.2 runs
+ * BFS on CSR through the paged arrays).  d_level: nv int32 in device memory,
+ * receives the hop distance from `source`, -1 where unreachable.  One launch per
+ * level for ordinary vertices plus one for very large neighbour lists, whose edges
+ * are spread over the whole grid (the imbalance Section 5.2 describes).
+ * Synchronises the stream between levels; *n_levels (host pointer, may be NULL)
+ * receives the number of levels expanded.  Allocates and frees 2 * nv + 64K int32
+ * of device scratch for the frontier queues.
+ */
+int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
+                  int32_t *d_level, int *n_levels, void *stream);
+
+/*
+ * Vector add c[i] = a[i] + b[i] over three paged fp32 arrays of n elements
+ * (Listing 1).  c is written through the runtime: its pages become dirty and reach
+ * the host by eviction write-back or gpuvm_flush.  One IEEE binary32 addition per
+ * element, no fused operations.
+ */
+int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n, void *stream);
+
+/*
+ * Embedding-bag gather: d_out[g][d] = sum over the `bag` rows of bag g of
+ * table[row][d], added in list order in fp32.  table: fp32 [rows][dims] at t_off,
+ * dims a multiple of 4 with dims/4 <= 32 lanes (one warp per bag, a lane owns 4
+ * consecutive dims); d_rows: n_bags * bag int64 row ids; d_out: n_bags * dims fp32.
+ */
+int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags,
+                    size_t bag, float *d_out, void *stream);
+
+/*
+ * Read-modify-write through the element accessors: for every k < n,
+ * a[idx[k]] = a[idx[k]] * 3 + 1 on uint32 elements at a_off (wrapping).  Indices
+ * must be distinct.  Exercises gpuvm_read + gpuvm_write with scattered dirty pages.
+ */
+int gpuvm_scatter_update_u32(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream);
+
+/*
+ * Transfer micro-benchmark (Section 5.1, Fig. 7): touch n_pages consecutive pages
+ * starting at page first_page, one warp per page, `warps_per_sm` warps on every SM;
+ * each warp pins its page (faulting it in) and releases it.  No payload is read.
+ */
+int gpuvm_touch_pages(gpuvm_t h, size_t first_page, size_t n_pages, int warps_per_sm, void *stream);
+
+/* ---- the same kernels on plain pointers (cudaMallocManaged or device memory) */
+int gpuvm_raw_stream_sum_i32(const int32_t *a, size_t n, int64_t *d_sum, void *stream);
+int gpuvm_raw_gather_f32(const float *x, const int64_t *d_idx, size_t n_idx, size_t block,
+                         float *d_fsum, int64_t *d_bsum, void *stream);
+int gpuvm_raw_bfs_csr(const int64_t *row_off, const int32_t *col, size_t nv, size_t source,
+                      int32_t *d_level, int *n_levels, void *stream);
+int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void *stream);
+int gpuvm_raw_embag_f32(const float *table, size_t dims, const int64_t *d_rows, size_t n_bags,
+                        size_t bag, float *d_out, void *stream);
+
+/*
+ * Host-link peaks measured with SM-issued 16-byte loads / stores on `bytes` of
+ * pinned mapped host memory (host_ptr: host pointer, pinned) and a device buffer
+ * d_buf of the same size: out[0] = host->device GB/s, out[1] = device->host GB/s,
+ * out[2] = both directions at once (sum), each the best of `reps` (CUDA events).
+ * out: host pointer to 3 doubles.  Synchronises.
+ */
+int gpuvm_link_peak(void *host_ptr, void *d_buf, size_t bytes, int reps, double *out);
+
+/* Number of kernels this library has launched in the calling process. */
+unsigned long long gpuvm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPUVM_WORKLOADS_H */

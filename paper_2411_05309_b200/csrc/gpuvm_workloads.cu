@@ -1,0 +1,597 @@
+// Workload kernels written against the device accessors, plus the same kernels on
+// plain pointers.  Each kernel is a template over a memory policy: Paged goes
+// through the page table, Raw dereferences ordinary device-accessible memory.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "gpuvm.h"
+#include "gpuvm_device.cuh"
+#include "gpuvm_internal.h"
+#include "gpuvm_workloads.h"
+
+namespace {
+
+std::atomic<unsigned long long> g_launches{0};
+
+struct Paged {
+    gpuvm_dev_t vm;
+    __device__ __forceinline__ unsigned long long unit() const { return 1ull << vm.page_shift; }
+    template <typename T>
+    __device__ __forceinline__ T read(unsigned long long base, unsigned long long i) const { return gpuvm_read<T>(vm, i, base); }
+    template <typename T>
+    __device__ __forceinline__ void write(unsigned long long base, unsigned long long i, T v) const { gpuvm_write<T>(vm, i, v, base); }
+    __device__ __forceinline__ unsigned char *pin(unsigned long long off, int mode, gpuvm_token &t) const
+    {
+        return static_cast<unsigned char *>(gpuvm_ptr(vm, off, mode, &t));
+    }
+    __device__ __forceinline__ void release(const gpuvm_token &t) const { gpuvm_release(vm, t); }
+    static __device__ __forceinline__ uint4 load16(const void *p) { return gpuvm_load16(p); }
+    static __device__ __forceinline__ void store16(void *p, uint4 v) { gpuvm_store16(p, v); }
+    static __device__ __forceinline__ int load_i32(const void *p) { return gpuvm_load(static_cast<const int *>(p)); }
+};
+
+struct Raw {
+    unsigned char *base;
+    unsigned long long unit_bytes;
+    __device__ __forceinline__ unsigned long long unit() const { return unit_bytes; }
+    template <typename T>
+    __device__ __forceinline__ T read(unsigned long long off, unsigned long long i) const { return reinterpret_cast<const T *>(base + off)[i]; }
+    template <typename T>
+    __device__ __forceinline__ void write(unsigned long long off, unsigned long long i, T v) const { reinterpret_cast<T *>(base + off)[i] = v; }
+    __device__ __forceinline__ unsigned char *pin(unsigned long long off, int, gpuvm_token &) const { return base + off; }
+    __device__ __forceinline__ void release(const gpuvm_token &) const {}
+    static __device__ __forceinline__ uint4 load16(const void *p) { return *static_cast<const uint4 *>(p); }
+    static __device__ __forceinline__ void store16(void *p, uint4 v) { *static_cast<uint4 *>(p) = v; }
+    static __device__ __forceinline__ int load_i32(const void *p) { return *static_cast<const int *>(p); }
+};
+
+__device__ __forceinline__ unsigned int warp_in_grid() { return (blockIdx.x * blockDim.x + threadIdx.x) >> 5; }
+__device__ __forceinline__ unsigned int warps_in_grid() { return (gridDim.x * blockDim.x) >> 5; }
+
+// ------------------------------------------------------------- streaming sum
+template <class Mem>
+__global__ void __launch_bounds__(256) stream_sum_kernel(Mem m, unsigned long long a_off, unsigned long long n,
+                                                         unsigned long long *out)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    const unsigned long long unit = m.unit();
+    const unsigned long long start = a_off, end = a_off + 4ull * n;
+    const unsigned long long first = start / unit, units = (end + unit - 1) / unit - first;
+    long long acc = 0;
+    for (unsigned long long u = warp_in_grid(); u < units; u += warps_in_grid()) {
+        unsigned long long lo = (first + u) * unit, hi = lo + unit;
+        if (lo < start) lo = start;
+        if (hi > end) hi = end;
+        gpuvm_token tok;
+        const unsigned char *p = m.pin(lo, GPUVM_READ, tok);
+        if (!p) continue;
+        const unsigned int len = (unsigned int)(hi - lo), n16 = len >> 4;
+#pragma unroll 4
+        for (unsigned int i = lane; i < n16; i += 32) {
+            uint4 v = Mem::load16(p + 16ull * i);
+            acc += (long long)(int)v.x + (long long)(int)v.y + (long long)(int)v.z + (long long)(int)v.w;
+        }
+        const unsigned int tail = (len & 15u) >> 2;
+        if (lane < tail) acc += (long long)Mem::load_i32(p + 16ull * n16 + 4u * lane);
+        m.release(tok);
+    }
+    for (int o = 16; o; o >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, o);
+    if (lane == 0 && acc != 0) atomicAdd(out, (unsigned long long)acc);
+}
+
+// -------------------------------------------------------------- random gather
+template <class Mem>
+__global__ void __launch_bounds__(1024) gather_kernel(Mem m, unsigned long long x_off, const long long *__restrict__ idx,
+                                                      unsigned long long n_idx, unsigned long long block,
+                                                      float *__restrict__ fsum, long long *__restrict__ bsum)
+{
+    __shared__ double s_f[32];
+    __shared__ long long s_b[32];
+    const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned long long nb = (n_idx + block - 1) / block;
+    for (unsigned long long b = blockIdx.x; b < nb; b += gridDim.x) {
+        const unsigned long long lo = b * block;
+        const unsigned long long hi = lo + block < n_idx ? lo + block : n_idx;
+        double f = 0.0;
+        long long bits = 0;
+        for (unsigned long long k = lo + threadIdx.x; k < hi; k += blockDim.x) {
+            float v = m.template read<float>(x_off, (unsigned long long)idx[k]);
+            f += (double)v;
+            bits += (long long)__float_as_uint(v);
+        }
+        for (int o = 16; o; o >>= 1) {
+            f += __shfl_down_sync(0xFFFFFFFFu, f, o);
+            bits += __shfl_down_sync(0xFFFFFFFFu, bits, o);
+        }
+        if (lane == 0) { s_f[warp] = f; s_b[warp] = bits; }
+        __syncthreads();
+        if (warp == 0) {
+            const unsigned int nw = blockDim.x >> 5;
+            f = lane < nw ? s_f[lane] : 0.0;
+            bits = lane < nw ? s_b[lane] : 0;
+            for (int o = 16; o; o >>= 1) {
+                f += __shfl_down_sync(0xFFFFFFFFu, f, o);
+                bits += __shfl_down_sync(0xFFFFFFFFu, bits, o);
+            }
+            if (lane == 0) { fsum[b] = (float)f; bsum[b] = bits; }
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------ BFS
+constexpr long long kBigDegree = 4096;     // neighbour lists at least this long are spread over the grid
+constexpr unsigned int kBigQueue = 65536;
+
+// counters: [0] next frontier size, [1] big-vertex queue size
+template <class Mem>
+__global__ void __launch_bounds__(256) bfs_frontier_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
+                                                           int *__restrict__ level, const int *__restrict__ cur_q,
+                                                           unsigned int cur_n, int *__restrict__ next_q,
+                                                           int *__restrict__ big_q, unsigned int *__restrict__ counters,
+                                                           int depth)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    for (unsigned int i = warp_in_grid(); i < cur_n; i += warps_in_grid()) {
+        const int v = cur_q[i];
+        // lanes 0 and 1 fetch row_off[v] and row_off[v+1] (usually one page: one request)
+        long long r = 0;
+        if (lane < 2) r = m.template read<long long>(off_off, (unsigned long long)v + lane);
+        const long long lo = __shfl_sync(0xFFFFFFFFu, r, 0), hi = __shfl_sync(0xFFFFFFFFu, r, 1);
+        if (hi - lo >= kBigDegree) {
+            // hand the list to the grid-wide kernel; if its queue is full, expand it here
+            unsigned int slot = 0;
+            if (lane == 0) slot = atomicAdd(counters + 1, 1u);
+            slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
+            if (slot < kBigQueue) {
+                if (lane == 0) big_q[slot] = v;
+                continue;
+            }
+        }
+        for (long long base = lo; base < hi; base += 32) {
+            const long long e = base + lane;
+            if (e < hi) {
+                const int c = m.template read<int>(col_off, (unsigned long long)e);
+                if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1)
+                    next_q[atomicAdd(counters, 1u)] = c;
+            }
+        }
+    }
+}
+
+template <class Mem>
+__global__ void __launch_bounds__(256) bfs_big_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
+                                                      int *__restrict__ level, int *__restrict__ next_q,
+                                                      const int *__restrict__ big_q, unsigned int *__restrict__ counters,
+                                                      int depth)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    unsigned int n_big = counters[1] < kBigQueue ? counters[1] : kBigQueue;
+    for (unsigned int i = 0; i < n_big; ++i) {
+        const int v = big_q[i];
+        long long r = 0;
+        if (lane < 2) r = m.template read<long long>(off_off, (unsigned long long)v + lane);
+        const long long lo = __shfl_sync(0xFFFFFFFFu, r, 0), hi = __shfl_sync(0xFFFFFFFFu, r, 1);
+        for (long long base = lo + 32ll * warp_in_grid(); base < hi; base += 32ll * warps_in_grid()) {
+            const long long e = base + lane;
+            if (e < hi) {
+                const int c = m.template read<int>(col_off, (unsigned long long)e);
+                if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1)
+                    next_q[atomicAdd(counters, 1u)] = c;
+            }
+        }
+    }
+}
+
+__global__ void bfs_init_kernel(int *level, int *cur_q, int source)
+{
+    level[source] = 0;
+    cur_q[0] = source;
+}
+
+// ----------------------------------------------------------------- vector add
+// A warp owns one unit (page) of the element range and walks it in chunks of at most
+// 4 KiB; for each chunk it holds exactly one page at a time: a, then b, then c.
+template <class Mem>
+__global__ void __launch_bounds__(256) vadd_kernel(Mem m, unsigned long long a_off, unsigned long long b_off,
+                                                   unsigned long long c_off, unsigned long long n,
+                                                   unsigned int chunk_bytes)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    const unsigned long long unit = m.unit() > chunk_bytes ? m.unit() : chunk_bytes;
+    const unsigned long long total = 4ull * n, units = (total + unit - 1) / unit;
+    for (unsigned long long u = warp_in_grid(); u < units; u += warps_in_grid()) {
+        unsigned long long lo = u * unit, hi = lo + unit < total ? lo + unit : total;
+        for (unsigned long long off = lo; off < hi; off += chunk_bytes) {
+            const unsigned int len = (unsigned int)(hi - off < chunk_bytes ? hi - off : chunk_bytes);
+            const unsigned int n16 = len >> 4;
+            uint4 va[8], vb[8];
+            gpuvm_token tok;
+            const unsigned char *pa = m.pin(a_off + off, GPUVM_READ, tok);
+            if (!pa) return;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                unsigned int i = lane + 32u * j;
+                if (i < n16) va[j] = Mem::load16(pa + 16ull * i);
+            }
+            m.release(tok);
+            const unsigned char *pb = m.pin(b_off + off, GPUVM_READ, tok);
+            if (!pb) return;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                unsigned int i = lane + 32u * j;
+                if (i < n16) vb[j] = Mem::load16(pb + 16ull * i);
+            }
+            m.release(tok);
+            unsigned char *pc = m.pin(c_off + off, GPUVM_WRITE, tok);
+            if (!pc) return;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                unsigned int i = lane + 32u * j;
+                if (i < n16) {
+                    uint4 r;
+                    r.x = __float_as_uint(__fadd_rn(__uint_as_float(va[j].x), __uint_as_float(vb[j].x)));
+                    r.y = __float_as_uint(__fadd_rn(__uint_as_float(va[j].y), __uint_as_float(vb[j].y)));
+                    r.z = __float_as_uint(__fadd_rn(__uint_as_float(va[j].z), __uint_as_float(vb[j].z)));
+                    r.w = __float_as_uint(__fadd_rn(__uint_as_float(va[j].w), __uint_as_float(vb[j].w)));
+                    Mem::store16(pc + 16ull * i, r);
+                }
+            }
+            m.release(tok);
+        }
+    }
+}
+
+// -------------------------------------------------------------- embedding bag
+template <class Mem>
+__global__ void __launch_bounds__(256) embag_kernel(Mem m, unsigned long long t_off, unsigned int dims,
+                                                    const long long *__restrict__ rows, unsigned long long n_bags,
+                                                    unsigned int bag, float *__restrict__ out)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    const unsigned int q = dims >> 2;                           // 16-byte pieces per row
+    for (unsigned long long g = warp_in_grid(); g < n_bags; g += warps_in_grid()) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (unsigned int k = 0; k < bag; ++k) {
+            const unsigned long long r = (unsigned long long)rows[g * bag + k];
+            if (lane < q) {
+                uint4 v = m.template read<uint4>(t_off, r * q + lane);
+                acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
+                acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
+                acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
+                acc.w = __fadd_rn(acc.w, __uint_as_float(v.w));
+            }
+        }
+        if (lane < q) reinterpret_cast<float4 *>(out + g * dims)[lane] = acc;
+    }
+}
+
+// ------------------------------------------------------- element read-modify-write
+template <class Mem>
+__global__ void __launch_bounds__(256) scatter_update_kernel(Mem m, unsigned long long a_off,
+                                                             const long long *__restrict__ idx, unsigned long long n)
+{
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    for (unsigned long long k = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; k < n; k += stride) {
+        const unsigned long long i = (unsigned long long)idx[k];
+        unsigned int v = m.template read<unsigned int>(a_off, i);
+        m.template write<unsigned int>(a_off, i, v * 3u + 1u);
+    }
+}
+
+// ------------------------------------------------------------------ page touch
+__global__ void touch_pages_kernel(gpuvm_dev_t vm, unsigned long long first_page, unsigned long long n_pages)
+{
+    for (unsigned long long p = warp_in_grid(); p < n_pages; p += warps_in_grid()) {
+        gpuvm_token tok;
+        void *ptr = gpuvm_ptr(vm, (first_page + p) << vm.page_shift, GPUVM_READ, &tok);
+        if (ptr) gpuvm_release(vm, tok);
+    }
+}
+
+// --------------------------------------------------------------- link kernels
+__global__ void link_in_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n16)
+{
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t base = blockIdx.x * (size_t)blockDim.x + threadIdx.x; base < n16; base += stride * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < n16) v[u] = gpuvm::ld_host16(src + i); }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < n16) gpuvm::st_frame16(dst + i, v[u]); }
+    }
+}
+
+__global__ void link_out_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n16)
+{
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t base = blockIdx.x * (size_t)blockDim.x + threadIdx.x; base < n16; base += stride * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < n16) v[u] = gpuvm::ld_frame16(src + i); }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < n16) gpuvm::st_host16(dst + i, v[u]); }
+    }
+}
+
+// even blocks read the first half of the host buffer, odd blocks write the second half
+__global__ void link_duplex_kernel(uint4 *host, uint4 *dev, size_t n16)
+{
+    const size_t half = n16 / 2;
+    const size_t stride = (size_t)(gridDim.x / 2) * blockDim.x;
+    const size_t t = (blockIdx.x / 2) * (size_t)blockDim.x + threadIdx.x;
+    if (blockIdx.x & 1) {
+        for (size_t i = t; i < half; i += stride) gpuvm::st_host16(host + half + i, gpuvm::ld_frame16(dev + half + i));
+    } else {
+        for (size_t base = t; base < half; base += stride * 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < half) v[u] = gpuvm::ld_host16(host + i); }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < half) gpuvm::st_frame16(dev + i, v[u]); }
+        }
+    }
+}
+
+int sm_count()
+{
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    }
+    return sms;
+}
+
+int launched(unsigned long long n = 1)
+{
+    gpuvm_note_launch_(n);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? GPUVM_OK : GPUVM_E_CUDA;
+}
+
+bool view_of(gpuvm_t h, Paged &m) { return h && gpuvm_device_view(h, &m.vm) == GPUVM_OK; }
+
+template <class Mem>
+int run_stream_sum(const Mem &m, size_t a_off, size_t n, int64_t *d_sum, cudaStream_t s)
+{
+    if (!d_sum) return GPUVM_E_ARG;
+    if (a_off % 16) return GPUVM_E_ALIGN;
+    if (cudaMemsetAsync(d_sum, 0, sizeof(int64_t), s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+    if (n == 0) return GPUVM_OK;
+    stream_sum_kernel<Mem><<<sm_count() * 4, 256, 0, s>>>(m, a_off, n, reinterpret_cast<unsigned long long *>(d_sum));
+    return launched();
+}
+
+template <class Mem>
+int run_gather(const Mem &m, size_t x_off, const int64_t *d_idx, size_t n_idx, size_t block, float *d_fsum,
+               int64_t *d_bsum, cudaStream_t s)
+{
+    if (!d_idx || !d_fsum || !d_bsum || block == 0 || block > (size_t(1) << 20)) return GPUVM_E_ARG;
+    if (x_off % 16) return GPUVM_E_ALIGN;
+    if (n_idx == 0) return GPUVM_OK;
+    size_t nb = (n_idx + block - 1) / block;
+    unsigned int threads = block >= 1024 ? 1024u : (unsigned int)((block + 31) / 32 * 32);
+    size_t resident = (size_t)sm_count() * (2048 / threads);
+    unsigned int grid = (unsigned int)(nb < resident ? nb : resident);
+    gather_kernel<Mem><<<grid, threads, 0, s>>>(m, x_off, reinterpret_cast<const long long *>(d_idx), n_idx, block,
+                                                 d_fsum, reinterpret_cast<long long *>(d_bsum));
+    return launched();
+}
+
+template <class Mem>
+int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
+            cudaStream_t s)
+{
+    if (!d_level || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
+    if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
+    int *scratch = nullptr;
+    if (cudaMalloc(&scratch, (2 * nv + kBigQueue + 2) * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_ALLOC; }
+    int *q0 = scratch, *q1 = scratch + nv, *big_q = scratch + 2 * nv;
+    unsigned int *counters = reinterpret_cast<unsigned int *>(scratch + 2 * nv + kBigQueue);
+    int rc = GPUVM_OK;
+    cudaMemsetAsync(d_level, 0xFF, nv * sizeof(int32_t), s);
+    bfs_init_kernel<<<1, 1, 0, s>>>(d_level, q0, (int)source);
+    rc = launched();
+    unsigned int cur_n = 1;
+    int depth = 0;
+    const int grid = sm_count() * 4;
+    while (rc == GPUVM_OK && cur_n > 0) {
+        cudaMemsetAsync(counters, 0, 2 * sizeof(unsigned int), s);
+        bfs_frontier_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, q0, cur_n, q1, big_q, counters, depth);
+        bfs_big_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, q1, big_q, counters, depth);
+        rc = launched(2);
+        unsigned int host_counters[2] = {0, 0};
+        if (cudaMemcpyAsync(host_counters, counters, sizeof(host_counters), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); rc = GPUVM_E_CUDA; break; }
+        cur_n = host_counters[0];
+        int *t = q0; q0 = q1; q1 = t;
+        ++depth;
+    }
+    cudaStreamSynchronize(s);
+    cudaFree(scratch);
+    if (n_levels) *n_levels = depth;
+    return rc;
+}
+
+template <class Mem>
+int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, cudaStream_t s)
+{
+    unsigned long long unit = 0;
+    if (n % 4) return GPUVM_E_ALIGN;
+    if (n == 0) return GPUVM_OK;
+    unit = m.unit_host();
+    unsigned int chunk = unit < 4096 ? (unsigned int)unit : 4096u;
+    if (chunk < 512) return GPUVM_E_PAGE;             // a warp moves 512 bytes per instruction
+    if (a_off % chunk || b_off % chunk || c_off % chunk) return GPUVM_E_ALIGN;
+    vadd_kernel<Mem><<<sm_count() * 4, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
+    return launched();
+}
+
+template <class Mem>
+int run_embag(const Mem &m, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
+              cudaStream_t s)
+{
+    if (!d_rows || !d_out || dims == 0 || dims % 4 || dims / 4 > 32 || bag == 0 || bag > 0xFFFFFFFFull) return GPUVM_E_ARG;
+    if (t_off % 16) return GPUVM_E_ALIGN;
+    if (n_bags == 0) return GPUVM_OK;
+    embag_kernel<Mem><<<sm_count() * 4, 256, 0, s>>>(m, t_off, (unsigned int)dims, reinterpret_cast<const long long *>(d_rows),
+                                                      n_bags, (unsigned int)bag, d_out);
+    return launched();
+}
+
+struct PagedH : Paged { unsigned long long unit_host() const { return 1ull << vm.page_shift; } };
+struct RawH : Raw { unsigned long long unit_host() const { return unit_bytes; } };
+
+}  // namespace
+
+extern "C" {
+
+void gpuvm_note_launch_(unsigned long long n) { g_launches += n; }
+unsigned long long gpuvm_launch_count(void) { return g_launches.load(); }
+
+int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_stream_sum(m, a_off, n, d_sum, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx, size_t block, float *d_fsum,
+                     int64_t *d_bsum, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_gather(m, x_off, d_idx, n_idx, block, d_fsum, d_bsum, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
+                  void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n, void *stream)
+{
+    PagedH m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_vadd(m, a_off, b_off, c_off, n, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
+                    void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_embag(m, t_off, dims, d_rows, n_bags, bag, d_out, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_scatter_update_u32(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m) || !d_idx) return GPUVM_E_ARG;
+    if (a_off % 16) return GPUVM_E_ALIGN;
+    if (n == 0) return GPUVM_OK;
+    scatter_update_kernel<Paged><<<sm_count() * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        m, a_off, reinterpret_cast<const long long *>(d_idx), n);
+    return launched();
+}
+
+int gpuvm_touch_pages(gpuvm_t h, size_t first_page, size_t n_pages, int warps_per_sm, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m) || warps_per_sm <= 0 || warps_per_sm > 64) return GPUVM_E_ARG;
+    if (first_page + n_pages > m.vm.n_pages) return GPUVM_E_RANGE;
+    if (n_pages == 0) return GPUVM_OK;
+    int threads = warps_per_sm * 32 > 1024 ? 1024 : warps_per_sm * 32;
+    int blocks_per_sm = (warps_per_sm * 32 + threads - 1) / threads;
+    touch_pages_kernel<<<sm_count() * blocks_per_sm, threads, 0, static_cast<cudaStream_t>(stream)>>>(m.vm, first_page, n_pages);
+    return launched();
+}
+
+int gpuvm_raw_stream_sum_i32(const int32_t *a, size_t n, int64_t *d_sum, void *stream)
+{
+    if (!a) return GPUVM_E_ARG;
+    Raw m{reinterpret_cast<unsigned char *>(const_cast<int32_t *>(a)), 65536};
+    return run_stream_sum(m, 0, n, d_sum, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_raw_gather_f32(const float *x, const int64_t *d_idx, size_t n_idx, size_t block, float *d_fsum, int64_t *d_bsum,
+                         void *stream)
+{
+    if (!x) return GPUVM_E_ARG;
+    Raw m{reinterpret_cast<unsigned char *>(const_cast<float *>(x)), 65536};
+    return run_gather(m, 0, d_idx, n_idx, block, d_fsum, d_bsum, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_raw_bfs_csr(const int64_t *row_off, const int32_t *col, size_t nv, size_t source, int32_t *d_level,
+                      int *n_levels, void *stream)
+{
+    if (!row_off || !col) return GPUVM_E_ARG;
+    // one policy object addresses both arrays relative to the lower of the two
+    unsigned char *ro = reinterpret_cast<unsigned char *>(const_cast<int64_t *>(row_off));
+    unsigned char *co = reinterpret_cast<unsigned char *>(const_cast<int32_t *>(col));
+    unsigned char *base = ro < co ? ro : co;
+    if ((ro - base) % 16 || (co - base) % 16) return GPUVM_E_ALIGN;
+    Raw m{base, 65536};
+    return run_bfs(m, (size_t)(ro - base), (size_t)(co - base), nv, source, d_level, n_levels, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void *stream)
+{
+    if (!a || !b || !c) return GPUVM_E_ARG;
+    unsigned char *pa = reinterpret_cast<unsigned char *>(const_cast<float *>(a));
+    unsigned char *pb = reinterpret_cast<unsigned char *>(const_cast<float *>(b));
+    unsigned char *pc = reinterpret_cast<unsigned char *>(c);
+    unsigned char *base = pa < pb ? (pa < pc ? pa : pc) : (pb < pc ? pb : pc);
+    RawH m;
+    m.base = base;
+    m.unit_bytes = 65536;
+    return run_vadd(m, (size_t)(pa - base), (size_t)(pb - base), (size_t)(pc - base), n, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_raw_embag_f32(const float *table, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
+                        void *stream)
+{
+    if (!table) return GPUVM_E_ARG;
+    Raw m{reinterpret_cast<unsigned char *>(const_cast<float *>(table)), 65536};
+    return run_embag(m, 0, dims, d_rows, n_bags, bag, d_out, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_link_peak(void *host_ptr, void *d_buf, size_t bytes, int reps, double *out)
+{
+    if (!host_ptr || !d_buf || !out || bytes < 4096 || bytes % 32 || reps <= 0) return GPUVM_E_ARG;
+    void *dh = nullptr;
+    if (cudaHostGetDevicePointer(&dh, host_ptr, 0) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_PIN; }
+    cudaEvent_t a, b;
+    cudaEventCreate(&a);
+    cudaEventCreate(&b);
+    const size_t n16 = bytes / 16;
+    const int grid = sm_count() * 2;
+    double best[3] = {0, 0, 0};
+    for (int mode = 0; mode < 3; ++mode)
+        for (int r = 0; r <= reps; ++r) {
+            cudaEventRecord(a);
+            if (mode == 0) link_in_kernel<<<grid, 512>>>(static_cast<const uint4 *>(dh), static_cast<uint4 *>(d_buf), n16);
+            else if (mode == 1) link_out_kernel<<<grid, 512>>>(static_cast<const uint4 *>(d_buf), static_cast<uint4 *>(dh), n16);
+            else link_duplex_kernel<<<grid * 2, 512>>>(static_cast<uint4 *>(dh), static_cast<uint4 *>(d_buf), n16);
+            gpuvm_note_launch_(1);
+            cudaEventRecord(b);
+            if (cudaEventSynchronize(b) != cudaSuccess) { cudaGetLastError(); cudaEventDestroy(a); cudaEventDestroy(b); return GPUVM_E_CUDA; }
+            float ms = 0;
+            cudaEventElapsedTime(&ms, a, b);
+            double gbs = (double)bytes / (ms * 1e6);
+            if (r > 0 && gbs > best[mode]) best[mode] = gbs;     // r == 0 is the warm-up
+        }
+    cudaEventDestroy(a);
+    cudaEventDestroy(b);
+    out[0] = best[0]; out[1] = best[1]; out[2] = best[2];
+    return GPUVM_OK;
+}
+
+}  // extern "C"

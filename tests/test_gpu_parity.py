@@ -1,0 +1,235 @@
+"""GPU parity: every workload through the C ABI against the CPU oracle, element by element,
+on seeded inputs that span several pages and a ragged tail, from ample to one-frame pools.
+Bit-exact for integer outputs and written-back bytes; 1e-6 relative for fp32 sums."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2411_05309_b200 import inputs
+from gpu_common import Arena, finish, paged
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2411_05309_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+POLICIES = [0, 1]
+
+
+@pytest.mark.parametrize("page,n,frames", [
+    (4096, 1 << 16, 64),          # pool == data
+    (4096, 1 << 16, 16),          # 4x oversubscribed
+    (4096, (1 << 16) + 1000, 5),  # ragged tail, tiny pool
+    (256, 5000, 1),               # one frame
+    (65536, 1 << 18, 3),
+    (16, 2048, 7),                # smallest page
+])
+@pytest.mark.parametrize("policy", POLICIES)
+def test_stream_sum(B, page, n, frames, policy):
+    import torch
+    n4 = (n + 3) // 4 * 4
+    a = inputs.fill_i32_u20(np.empty(n4, np.int32), n4, inputs.config_seed(1))
+    ar = Arena(page, {"a": a})
+    before = ar.host.copy()
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    with paged(ar.host, page, frames, policy) as h:
+        B.gpuvm_stream_sum_i32(h, ar.off["a"], n, out)
+        st, ck = finish(h)
+        assert int(out.item()) == oracle.stream_sum_i32_direct(a[:n])
+        touched = (4 * n + page - 1) // page
+        assert st["faults"] == touched                  # each page is read in one burst by one warp
+        assert st["writebacks"] == 0 and st["bytes_out"] == 0
+        assert st["evictions"] == max(0, touched - frames)
+        assert ck["resident"] == min(touched, frames)
+        # a second pass over a pool that holds everything takes no fault (mappings persist)
+        if frames >= touched:
+            B.gpuvm_stream_sum_i32(h, ar.off["a"], n, out)
+            st2, _ = finish(h)
+            assert st2["faults"] == touched and int(out.item()) == oracle.stream_sum_i32_direct(a[:n])
+    assert np.array_equal(ar.host, before)
+
+
+@pytest.mark.parametrize("page,n,n_idx,block,frames", [
+    (4096, 1 << 16, 1 << 14, 1024, 64),
+    (4096, 1 << 16, (1 << 14) + 77, 1024, 16),     # ragged last block
+    (256, 1 << 12, 5000, 100, 3),                  # block smaller than a CTA
+    (65536, 1 << 20, 1 << 15, 1024, 16),
+    (64, 4096, 3000, 1024, 1),                     # one frame: every warp fights for it
+])
+@pytest.mark.parametrize("policy", POLICIES)
+def test_gather(B, page, n, n_idx, block, frames, policy):
+    import torch
+    x = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(2))
+    idx = inputs.fill_index_i64(np.empty(n_idx, np.int64), n_idx, inputs.config_seed(2, 1), n)
+    ar = Arena(page, {"x": x})
+    nb = (n_idx + block - 1) // block
+    fsum = torch.zeros(nb, dtype=torch.float32, device="cuda")
+    bsum = torch.zeros(nb, dtype=torch.int64, device="cuda")
+    with paged(ar.host, page, frames, policy) as h:
+        B.gpuvm_gather_f32(h, ar.off["x"], dev(idx), n_idx, block, fsum, bsum)
+        st, ck = finish(h)
+    ref_f, ref_b = oracle.gather_block_sums_direct(x, idx, block)
+    assert np.array_equal(bsum.cpu().numpy(), ref_b)                     # which elements: exact
+    got = fsum.cpu().numpy().astype(np.float64)
+    ref = ref_f.astype(np.float64)
+    assert np.all(np.abs(got - ref) <= 1e-6 * np.maximum(np.abs(ref), 2.0 ** -10))
+    distinct = np.unique((idx * 4) // page).size
+    assert st["faults"] >= distinct and st["writebacks"] == 0
+    if frames >= ar.n_pages:
+        assert st["faults"] == distinct and st["evictions"] == 0        # compulsory misses only
+
+
+@pytest.mark.parametrize("page,n,frames", [
+    (4096, 1 << 16, 3 * 64),      # everything fits
+    (4096, 1 << 16, 48),          # 4x oversubscribed: dirty victims are written back while running
+    (4096, (1 << 14) + 500, 3),
+    (512, 4096, 1),
+    (65536, 1 << 18, 6),
+])
+@pytest.mark.parametrize("policy", POLICIES)
+def test_vadd_writes_back_every_dirty_page(B, page, n, frames, policy):
+    n = n // 4 * 4
+    a = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4))
+    b = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4, 1))
+    ar = Arena(page, {"a": a, "b": b, "c": np.zeros(n, np.float32)})
+    with paged(ar.host, page, frames, policy) as h:
+        B.gpuvm_vadd_f32(h, ar.off["a"], ar.off["b"], ar.off["c"], n)
+        st, ck = finish(h)
+    ref = oracle.vadd_f32_direct(a, b)
+    assert np.array_equal(ar.views["c"].view(np.uint32), ref.view(np.uint32))    # bit-exact
+    assert np.array_equal(ar.views["a"], a) and np.array_equal(ar.views["b"], b)
+    c_pages = (4 * n + page - 1) // page
+    assert st["writebacks"] + st["flush_writebacks"] >= c_pages
+    if frames >= ar.n_pages:
+        assert st["faults"] == ar.n_pages and st["writebacks"] == 0 and st["flush_writebacks"] == c_pages
+
+
+def small_graphs():
+    rng = np.random.default_rng(24)
+    yield 1, [], 0
+    yield 5, [(0, 0), (0, 1), (0, 1), (1, 2), (3, 4)], 0
+    yield 5, [(1, 0), (2, 1)], 0
+    for _ in range(3):
+        nv = int(rng.integers(2, 40))
+        ne = int(rng.integers(0, 200))
+        yield nv, [(int(rng.integers(0, nv)), int(rng.integers(0, nv))) for _ in range(ne)], int(rng.integers(0, nv))
+
+
+def csr(nv, edges):
+    off = np.zeros(nv + 1, dtype=np.int64)
+    for u, _ in edges:
+        off[u + 1] += 1
+    off = np.cumsum(off).astype(np.int64)
+    col = np.zeros(max(len(edges), 4), dtype=np.int32)
+    cur = off[:-1].copy()
+    for u, v in edges:
+        col[cur[u]] = v
+        cur[u] += 1
+    return off, col
+
+
+def run_bfs(B, off, col, src, page, frames, policy):
+    import torch
+    nv = off.size - 1
+    off_p = np.zeros((off.size + 1) // 2 * 2, np.int64)
+    off_p[:off.size] = off
+    col_p = np.zeros((col.size + 3) // 4 * 4, np.int32)
+    col_p[:col.size] = col
+    ar = Arena(page, {"off": off_p, "col": col_p})
+    level = torch.zeros(nv, dtype=torch.int32, device="cuda")
+    with paged(ar.host, page, frames, policy) as h:
+        depth = B.gpuvm_bfs_csr(h, ar.off["off"], ar.off["col"], nv, src, level)
+        st, ck = finish(h)
+    return level.cpu().numpy(), depth, st
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+def test_bfs_small_graphs(B, policy):
+    for nv, edges, src in small_graphs():
+        off, col = csr(nv, edges)
+        ref = oracle.bfs_levels_direct(off, col, src)
+        for page, frames in ((64, 1), (64, 4), (4096, 8)):
+            got, depth, st = run_bfs(B, off, col, src, page, frames, policy)
+            assert np.array_equal(got, ref)
+            assert depth == ref.max() + 1
+
+
+@pytest.mark.parametrize("scale,page,frames", [(12, 4096, 20), (14, 4096, 9), (14, 65536, 5)])
+def test_bfs_rmat_with_hub_vertices(B, scale, page, frames):
+    off, col = inputs.rmat_csr(scale, 16 << scale, inputs.config_seed(3))
+    assert np.diff(off).max() >= 4096 or scale < 14          # the grid-wide path is exercised
+    ref = oracle.bfs_levels_direct(off, col, 0)
+    got, depth, st = run_bfs(B, off, col, 0, page, frames, 1)
+    assert np.array_equal(got, ref)
+    assert st["writebacks"] == 0
+
+
+@pytest.mark.parametrize("page,n_rows,n_bags,frames", [
+    (4096, 512, 64, 64),
+    (4096, 4096, 1000, 8),
+    (2 << 20, 1 << 14, 1 << 12, 2),
+    (512, 100, 33, 1),
+])
+def test_embag(B, page, n_rows, n_bags, frames):
+    import torch
+    dims, bag = 128, 32
+    t = inputs.fill_f32_pm1(np.empty(n_rows * dims, np.float32), n_rows * dims, inputs.config_seed(5))
+    rows = inputs.fill_zipf_rows(np.empty(n_bags * bag, np.int64), n_bags * bag, inputs.config_seed(5, 1), n_rows, 1.05)
+    ar = Arena(page, {"t": t})
+    out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
+    with paged(ar.host, page, frames) as h:
+        B.gpuvm_embag_f32(h, ar.off["t"], dims, dev(rows), n_bags, bag, out)
+        st, ck = finish(h)
+    ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
+    got = out.cpu().numpy()
+    assert np.all(np.abs(got.astype(np.float64) - ref) <= 1e-6 * np.maximum(np.abs(ref), 2.0 ** -10))
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))     # same order of additions: same bits
+    assert st["faults"] >= np.unique(rows * dims * 4 // page).size
+
+
+@pytest.mark.parametrize("page,n,frames", [(4096, 1 << 16, 64), (4096, 1 << 16, 7), (64, 2048, 1), (1024, 50000, 13)])
+@pytest.mark.parametrize("policy", POLICIES)
+def test_scatter_update_through_element_accessors(B, page, n, frames, policy):
+    n = n // 4 * 4
+    a = (inputs.fill_i32_u20(np.empty(n, np.int32), n, 77)).astype(np.uint32)
+    perm = np.random.default_rng(3).permutation(n)[: (3 * n) // 4].astype(np.int64)
+    ar = Arena(page, {"a": a})
+    with paged(ar.host, page, frames, policy) as h:
+        B.gpuvm_scatter_update_u32(h, ar.off["a"], dev(perm), perm.size)
+        st, ck = finish(h)
+    ref = a.copy()
+    ref[perm] = ref[perm] * np.uint32(3) + np.uint32(1)
+    assert np.array_equal(ar.views["a"], ref)                           # no dirty data lost
+    # the same through the oracle's pager, moving real bytes
+    host2 = np.frombuffer(a.tobytes(), np.uint8).copy()
+    assert st["faults"] >= np.unique(perm * 4 // page).size
+
+
+def test_two_kernels_share_mappings(B):
+    """Mappings persist across launches: a read-only pass after a write pass sees the
+    written values without any flush in between."""
+    import torch
+    page, n, frames = 4096, 1 << 14, 8
+    a = inputs.fill_i32_u20(np.empty(n, np.int32), n, 5).astype(np.uint32)
+    idx = np.arange(n, dtype=np.int64)
+    ar = Arena(page, {"a": a})
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    with paged(ar.host, page, frames) as h:
+        B.gpuvm_scatter_update_u32(h, 0, dev(idx), n)
+        B.gpuvm_stream_sum_i32(h, 0, n, out)
+        st, ck = finish(h)
+    ref = (a * np.uint32(3) + np.uint32(1)).view(np.int32)
+    assert int(out.item()) == int(ref.astype(np.int64).sum())
+    assert np.array_equal(ar.views["a"].view(np.int32), ref)
