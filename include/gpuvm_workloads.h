@@ -12,7 +12,7 @@
  *   - calls enqueue work and return without synchronising unless stated; device
  *     errors (a wait that ran out, an offset out of range) are sticky in the handle
  *     and show up in gpuvm_stats().  Return value: 0 or a negative gpuvm_status.
- *   - nothing here allocates device memory except gpuvm_bfs_csr (frontier queues,
+ *   - nothing here allocates device memory except gpuvm_bfs_csr (256 KiB of scratch,
  *     freed before it returns).
  */
 #ifndef GPUVM_WORKLOADS_H
@@ -48,12 +48,14 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
  * Level-synchronous BFS over a CSR graph whose int64 row offsets (nv + 1 of them,
  * at off_off) and int32 column indices (at col_off) are paged (Section 5.2 runs
  * BFS on CSR through the paged arrays).  d_level: nv int32 in device memory,
- * receives the hop distance from `source`, -1 where unreachable.  One launch per
- * level for ordinary vertices plus one for very large neighbour lists, whose edges
- * are spread over the whole grid (the imbalance Section 5.2 describes).
- * Synchronises the stream between levels; *n_levels (host pointer, may be NULL)
- * receives the number of levels expanded.  Allocates and frees 2 * nv + 64K int32
- * of device scratch for the frontier queues.
+ * receives the hop distance from `source`, -1 where unreachable.  Per level one
+ * sweep over the vertices in ascending order (warps draw chunks of 32 consecutive
+ * vertices from a ticket counter, so the grid moves through the arrays in address
+ * order) plus one launch for very large neighbour lists, whose edges are spread
+ * over the whole grid (the imbalance Section 5.2 describes).  Synchronises the
+ * stream between levels; *n_levels (host pointer, may be NULL) receives the number
+ * of levels expanded, counting the last one that discovers nothing.  Allocates and
+ * frees 256 KiB of device scratch (queue of large vertices, counters).
  */
 int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
                   int32_t *d_level, int *n_levels, void *stream);

@@ -1,0 +1,247 @@
+"""The five oversubscribed workload configurations and their runners.
+
+Each configuration places its paged arrays at page-aligned offsets of ONE backing store
+(one handle, one frame pool), fills them with the seeded generators, keeps small
+operands (indices, row ids, outputs) in ordinary device memory, and runs the workload
+through the C ABI.  ``shrink`` divides every size by 2**shrink (page size kept) so that
+the same code serves small parity cases.
+
+Effective bytes (numerator of "effective application GB/s"): streaming sum = bytes of the
+array; gather = 4 bytes per index; BFS = 16 bytes of offsets per expanded vertex + 4 bytes
+per traversed edge; vector add = bytes of a, b and c; embedding bag = bytes of the rows
+looked up.
+"""
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import time
+
+import numpy as np
+
+from . import binding as B
+from . import inputs
+
+KiB, MiB, GiB = 1 << 10, 1 << 20, 1 << 30
+
+
+def _pad(nbytes: int, page: int) -> int:
+    return (nbytes + page - 1) // page * page
+
+
+def _host_view(ptr: int, nbytes: int) -> np.ndarray:
+    return np.ctypeslib.as_array((ctypes.c_uint8 * nbytes).from_address(ptr))
+
+
+@dataclasses.dataclass
+class RunResult:
+    seconds: float            # CUDA-event time: workload kernel(s) + flush, cold pool
+    kernel_seconds: float     # workload kernel(s) only
+    stats: dict
+    check: dict
+    effective_bytes: int
+    extra: dict
+
+
+class Workload:
+    """Base: owns the handle, the host arena and the device-side operands."""
+
+    name = "?"
+    cfg = 0
+    page_bytes = 0
+    kernels_per_run = 1
+
+    def __init__(self, shrink: int = 0):
+        self.shrink = shrink
+        self.h = None
+        self.off = {}
+        self.host = None
+
+    # -- layout -------------------------------------------------------------
+    def _create(self, arrays: dict, pool_bytes: int):
+        """arrays: name -> nbytes.  The library allocates the pinned backing store."""
+        total = 0
+        for name, nbytes in arrays.items():
+            self.off[name] = total
+            total += _pad(nbytes, self.page_bytes)
+        self.nbytes = total
+        if callable(pool_bytes):
+            pool_bytes = pool_bytes(total)
+        self.pool_bytes = max(self.page_bytes, pool_bytes // self.page_bytes * self.page_bytes)
+        self.h = B.gpuvm_create(None, total, self.page_bytes, self.pool_bytes)
+        self.host = _host_view(B.gpuvm_host_ptr(self.h), total)
+        self.n_pages = total // self.page_bytes
+        self.n_frames = self.pool_bytes // self.page_bytes
+
+    def view(self, name: str, dtype, count: int) -> np.ndarray:
+        o = self.off[name]
+        return self.host[o:o + count * np.dtype(dtype).itemsize].view(dtype)
+
+    def close(self):
+        if self.h:
+            B.gpuvm_destroy(self.h)
+            self.h = None
+            self.host = None
+
+    # -- to be provided -----------------------------------------------------
+    def setup(self):
+        raise NotImplementedError
+
+    def launch(self, stream):
+        raise NotImplementedError
+
+    def effective_bytes(self) -> int:
+        raise NotImplementedError
+
+    def describe(self) -> dict:
+        return {"workload": self.name, "cfg": self.cfg, "shrink": self.shrink, "page_bytes": self.page_bytes,
+                "pool_bytes": self.pool_bytes, "paged_bytes": self.nbytes, "pages": self.n_pages,
+                "frames": self.n_frames, "oversubscription_level": self.nbytes / self.pool_bytes - 1}
+
+    # -- one cold run ---------------------------------------------------------
+    def run(self, check: bool = True) -> RunResult:
+        import torch
+        stream = torch.cuda.current_stream()
+        B.gpuvm_reset(self.h)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record(stream)
+        extra = self.launch(stream) or {}
+        e1.record(stream)
+        B.gpuvm_flush(self.h, stream)
+        e2.record(stream)
+        e2.synchronize()
+        stats = B.gpuvm_stats(self.h)
+        ck = B.gpuvm_check(self.h) if check else {}
+        return RunResult(e0.elapsed_time(e2) / 1e3, e0.elapsed_time(e1) / 1e3, stats, ck,
+                         self.effective_bytes(), extra)
+
+
+class StreamSum(Workload):
+    """Streaming read-reduce: int64 sum over an int32 array, 4 KiB pages, pool = 1/4 of the data."""
+    name, cfg, page_bytes = "stream_sum_i32", 1, 4 * KiB
+
+    def setup(self):
+        import torch
+        self.n = (1 << 24) >> self.shrink
+        self._create({"a": 4 * self.n}, (16 * MiB) >> self.shrink)
+        inputs.fill_i32_u20(B.gpuvm_host_ptr(self.h) + self.off["a"], self.n, inputs.config_seed(1))
+        self.d_sum = torch.zeros(1, dtype=torch.int64, device="cuda")
+        return self
+
+    def launch(self, stream):
+        B.gpuvm_stream_sum_i32(self.h, self.off["a"], self.n, self.d_sum, stream)
+
+    def effective_bytes(self):
+        return 4 * self.n
+
+
+class Gather(Workload):
+    """Random gather: fp32 array, uniform int64 indices, one sum per 1024 indices, 64 KiB pages, pool 1/4."""
+    name, cfg, page_bytes = "random_gather_f32", 2, 64 * KiB
+    block = 1024
+
+    def setup(self):
+        import torch
+        self.n = (1 << 28) >> self.shrink
+        self.n_idx = (1 << 26) >> self.shrink
+        self._create({"x": 4 * self.n}, (256 * MiB) >> self.shrink)
+        inputs.fill_f32_pm1(B.gpuvm_host_ptr(self.h) + self.off["x"], self.n, inputs.config_seed(2))
+        self.idx_host = torch.empty(self.n_idx, dtype=torch.int64).pin_memory()
+        inputs.fill_index_i64(self.idx_host.data_ptr(), self.n_idx, inputs.config_seed(2, 1), self.n)
+        self.d_idx = self.idx_host.cuda()
+        nb = (self.n_idx + self.block - 1) // self.block
+        self.d_fsum = torch.zeros(nb, dtype=torch.float32, device="cuda")
+        self.d_bsum = torch.zeros(nb, dtype=torch.int64, device="cuda")
+        return self
+
+    def launch(self, stream):
+        B.gpuvm_gather_f32(self.h, self.off["x"], self.d_idx, self.n_idx, self.block, self.d_fsum, self.d_bsum, stream)
+
+    def effective_bytes(self):
+        return 4 * self.n_idx
+
+
+class Bfs(Workload):
+    """BFS from vertex 0 on an RMAT graph; row offsets and column indices paged at 64 KiB, pool = half."""
+    name, cfg, page_bytes = "bfs_rmat_csr", 3, 64 * KiB
+    kernels_per_run = None        # 1 + 2 per level
+
+    def setup(self):
+        import torch
+        self.scale = 24 - self.shrink
+        self.nv = 1 << self.scale
+        self.ne = 16 << self.scale
+        off_bytes = _pad(8 * (self.nv + 1), 16)
+        self._create({"off": off_bytes, "col": 4 * self.ne}, lambda total: total // 2)   # pool = half their size
+        base = B.gpuvm_host_ptr(self.h)
+        inputs.rmat_csr(self.scale, self.ne, inputs.config_seed(3), base + self.off["off"], base + self.off["col"])
+        self.d_level = torch.zeros(self.nv, dtype=torch.int32, device="cuda")
+        self.levels = 0
+        return self
+
+    def launch(self, stream):
+        self.levels = B.gpuvm_bfs_csr(self.h, self.off["off"], self.off["col"], self.nv, 0, self.d_level, stream)
+        return {"levels": self.levels}
+
+    def effective_bytes(self):
+        lvl = self.d_level.cpu().numpy()
+        off = self.view("off", np.int64, self.nv + 1)
+        deg = np.diff(off)
+        visited = lvl >= 0
+        self.traversed_edges = int(deg[visited].sum())
+        return int(16 * visited.sum() + 4 * self.traversed_edges)
+
+
+class VAdd(Workload):
+    """c = a + b over three fp32 arrays, 64 KiB pages, pool = one array (3x oversubscribed)."""
+    name, cfg, page_bytes = "vector_add_f32", 4, 64 * KiB
+
+    def setup(self):
+        self.n = (1 << 30) >> self.shrink
+        self._create({"a": 4 * self.n, "b": 4 * self.n, "c": 4 * self.n}, (4 * GiB) >> self.shrink)
+        base = B.gpuvm_host_ptr(self.h)
+        inputs.fill_f32_pm1(base + self.off["a"], self.n, inputs.config_seed(4))
+        inputs.fill_f32_pm1(base + self.off["b"], self.n, inputs.config_seed(4, 1))
+        self.view("c", np.float32, self.n)[...] = 0
+        return self
+
+    def launch(self, stream):
+        B.gpuvm_vadd_f32(self.h, self.off["a"], self.off["b"], self.off["c"], self.n, stream)
+
+    def effective_bytes(self):
+        return 12 * self.n
+
+
+class EmbeddingBag(Workload):
+    """Zipf-skewed embedding gather: rows x 128 fp32 table, bags of 32 rows, 2 MiB pages, pool 1/4."""
+    name, cfg, page_bytes = "zipf_embedding_bag_f32", 5, 2 * MiB
+    dims, bag, s = 128, 32, 1.05
+
+    def setup(self):
+        import torch
+        self.n_rows = (1 << 27) >> self.shrink
+        self.n_lookups = (1 << 24) >> self.shrink
+        self.n_bags = self.n_lookups // self.bag
+        self._create({"t": 4 * self.dims * self.n_rows}, (16 * GiB) >> self.shrink)
+        inputs.fill_f32_pm1(B.gpuvm_host_ptr(self.h) + self.off["t"], self.dims * self.n_rows, inputs.config_seed(5))
+        self.rows_host = torch.empty(self.n_lookups, dtype=torch.int64).pin_memory()
+        inputs.fill_zipf_rows(self.rows_host.data_ptr(), self.n_lookups, inputs.config_seed(5, 1), self.n_rows, self.s)
+        self.d_rows = self.rows_host.cuda()
+        self.d_out = torch.zeros(self.n_bags * self.dims, dtype=torch.float32, device="cuda")
+        return self
+
+    def launch(self, stream):
+        B.gpuvm_embag_f32(self.h, self.off["t"], self.dims, self.d_rows, self.n_bags, self.bag, self.d_out, stream)
+
+    def effective_bytes(self):
+        return 4 * self.dims * self.n_lookups
+
+
+WORKLOADS = {1: StreamSum, 2: Gather, 3: Bfs, 4: VAdd, 5: EmbeddingBag}
+
+
+def make(cfg: int, shrink: int = 0) -> Workload:
+    t0 = time.time()
+    w = WORKLOADS[cfg](shrink).setup()
+    w.setup_seconds = time.time() - t0
+    return w

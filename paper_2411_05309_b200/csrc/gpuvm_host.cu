@@ -9,6 +9,7 @@
 
 #include "gpuvm.h"
 #include "gpuvm_device.cuh"
+#include "gpuvm_internal.h"
 
 struct gpuvm_handle {
     gpuvm_dev_t dev;
@@ -209,6 +210,7 @@ int gpuvm_flush(gpuvm_t h, void *stream)
     unsigned int warps = h->dev.n_frames < 148u * 32u ? h->dev.n_frames : 148u * 32u;
     unsigned int blocks = (warps + 7) / 8;
     flush_kernel<<<blocks, 256, 0, s>>>(h->dev);
+    gpuvm_note_launch_(1);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     return e == cudaSuccess ? GPUVM_OK : fail(h, e, GPUVM_E_CUDA);
@@ -233,6 +235,7 @@ int gpuvm_check(gpuvm_t h, gpuvm_check_t *out)
     cudaError_t e = cudaMemset(h->check_buf, 0, 8 * sizeof(unsigned long long));
     if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
     check_kernel<<<148, 256>>>(h->dev, h->check_buf);
+    gpuvm_note_launch_(1);
     unsigned long long c[8];
     e = cudaMemcpy(c, h->check_buf, sizeof(c), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);

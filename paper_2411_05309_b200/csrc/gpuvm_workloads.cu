@@ -125,50 +125,70 @@ __global__ void __launch_bounds__(1024) gather_kernel(Mem m, unsigned long long 
 constexpr long long kBigDegree = 4096;     // neighbour lists at least this long are spread over the grid
 constexpr unsigned int kBigQueue = 65536;
 
-// counters: [0] next frontier size, [1] big-vertex queue size
+// counters: [0] vertices discovered in this level, [1] big-vertex queue size, [2] chunk ticket
+//
+// One level = one sweep over the vertices in ascending order: a warp draws the next chunk
+// of 32 consecutive vertices from a ticket counter, so at any moment the whole grid works
+// inside a narrow window of the row-offset and column arrays and a level touches every page
+// at most about once, in address order.
 template <class Mem>
-__global__ void __launch_bounds__(256) bfs_frontier_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
-                                                           int *__restrict__ level, const int *__restrict__ cur_q,
-                                                           unsigned int cur_n, int *__restrict__ next_q,
-                                                           int *__restrict__ big_q, unsigned int *__restrict__ counters,
-                                                           int depth)
+__global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
+                                                        int *__restrict__ level, unsigned int nv,
+                                                        int *__restrict__ big_q, unsigned int *__restrict__ counters,
+                                                        int depth)
 {
     const unsigned int lane = threadIdx.x & 31;
-    for (unsigned int i = warp_in_grid(); i < cur_n; i += warps_in_grid()) {
-        const int v = cur_q[i];
-        // lanes 0 and 1 fetch row_off[v] and row_off[v+1] (usually one page: one request)
-        long long r = 0;
-        if (lane < 2) r = m.template read<long long>(off_off, (unsigned long long)v + lane);
-        const long long lo = __shfl_sync(0xFFFFFFFFu, r, 0), hi = __shfl_sync(0xFFFFFFFFu, r, 1);
-        if (hi - lo >= kBigDegree) {
-            // hand the list to the grid-wide kernel; if its queue is full, expand it here
-            unsigned int slot = 0;
-            if (lane == 0) slot = atomicAdd(counters + 1, 1u);
-            slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
-            if (slot < kBigQueue) {
-                if (lane == 0) big_q[slot] = v;
-                continue;
-            }
+    unsigned int found = 0;
+    for (;;) {
+        unsigned int chunk = 0;
+        if (lane == 0) chunk = atomicAdd(counters + 2, 1u);
+        chunk = __shfl_sync(0xFFFFFFFFu, chunk, 0);
+        const unsigned long long v0 = 32ull * chunk;
+        if (v0 >= nv) break;
+        const unsigned long long v = v0 + lane;
+        const bool active = v < nv && level[v] == depth;
+        unsigned int mask = __ballot_sync(0xFFFFFFFFu, active);
+        if (!mask) continue;
+        long long lo = 0, hi = 0;
+        if (active) {
+            lo = m.template read<long long>(off_off, v);
+            hi = m.template read<long long>(off_off, v + 1);
         }
-        for (long long base = lo; base < hi; base += 32) {
-            const long long e = base + lane;
-            if (e < hi) {
-                const int c = m.template read<int>(col_off, (unsigned long long)e);
-                if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1)
-                    next_q[atomicAdd(counters, 1u)] = c;
+        while (mask) {
+            const int L = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
+            if (bhi - blo >= kBigDegree) {
+                // hand the list to the grid-wide kernel; if its queue is full, expand it here
+                unsigned int slot = 0;
+                if (lane == 0) slot = atomicAdd(counters + 1, 1u);
+                slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
+                if (slot < kBigQueue) {
+                    if (lane == 0) big_q[slot] = (int)(v0 + L);
+                    continue;
+                }
+            }
+            for (long long base = blo; base < bhi; base += 32) {
+                const long long e = base + lane;
+                if (e < bhi) {
+                    const int c = m.template read<int>(col_off, (unsigned long long)e);
+                    if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1) ++found;
+                }
             }
         }
     }
+    for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
+    if (lane == 0 && found) atomicAdd(counters, found);
 }
 
 template <class Mem>
 __global__ void __launch_bounds__(256) bfs_big_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
-                                                      int *__restrict__ level, int *__restrict__ next_q,
-                                                      const int *__restrict__ big_q, unsigned int *__restrict__ counters,
-                                                      int depth)
+                                                      int *__restrict__ level, const int *__restrict__ big_q,
+                                                      unsigned int *__restrict__ counters, int depth)
 {
     const unsigned int lane = threadIdx.x & 31;
-    unsigned int n_big = counters[1] < kBigQueue ? counters[1] : kBigQueue;
+    const unsigned int n_big = counters[1] < kBigQueue ? counters[1] : kBigQueue;
+    unsigned int found = 0;
     for (unsigned int i = 0; i < n_big; ++i) {
         const int v = big_q[i];
         long long r = 0;
@@ -178,18 +198,15 @@ __global__ void __launch_bounds__(256) bfs_big_kernel(Mem m, unsigned long long 
             const long long e = base + lane;
             if (e < hi) {
                 const int c = m.template read<int>(col_off, (unsigned long long)e);
-                if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1)
-                    next_q[atomicAdd(counters, 1u)] = c;
+                if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1) ++found;
             }
         }
     }
+    for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
+    if (lane == 0 && found) atomicAdd(counters, found);
 }
 
-__global__ void bfs_init_kernel(int *level, int *cur_q, int source)
-{
-    level[source] = 0;
-    cur_q[0] = source;
-}
+__global__ void bfs_init_kernel(int *level, int source) { level[source] = 0; }
 
 // ----------------------------------------------------------------- vector add
 // A warp owns one unit (page) of the element range and walks it in chunks of at most
@@ -388,27 +405,25 @@ int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t sour
 {
     if (!d_level || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
-    int *scratch = nullptr;
-    if (cudaMalloc(&scratch, (2 * nv + kBigQueue + 2) * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_ALLOC; }
-    int *q0 = scratch, *q1 = scratch + nv, *big_q = scratch + 2 * nv;
-    unsigned int *counters = reinterpret_cast<unsigned int *>(scratch + 2 * nv + kBigQueue);
-    int rc = GPUVM_OK;
+    int *scratch = nullptr;                       // big-vertex queue + 4 counters
+    if (cudaMalloc(&scratch, (kBigQueue + 4) * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_ALLOC; }
+    int *big_q = scratch;
+    unsigned int *counters = reinterpret_cast<unsigned int *>(scratch + kBigQueue);
     cudaMemsetAsync(d_level, 0xFF, nv * sizeof(int32_t), s);
-    bfs_init_kernel<<<1, 1, 0, s>>>(d_level, q0, (int)source);
-    rc = launched();
-    unsigned int cur_n = 1;
+    bfs_init_kernel<<<1, 1, 0, s>>>(d_level, (int)source);
+    int rc = launched();
     int depth = 0;
     const int grid = sm_count() * 4;
-    while (rc == GPUVM_OK && cur_n > 0) {
-        cudaMemsetAsync(counters, 0, 2 * sizeof(unsigned int), s);
-        bfs_frontier_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, q0, cur_n, q1, big_q, counters, depth);
-        bfs_big_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, q1, big_q, counters, depth);
+    unsigned int found = 1;
+    while (rc == GPUVM_OK && found > 0) {
+        cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
+        bfs_sweep_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, (unsigned int)nv, big_q, counters, depth);
+        bfs_big_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, big_q, counters, depth);
         rc = launched(2);
         unsigned int host_counters[2] = {0, 0};
         if (cudaMemcpyAsync(host_counters, counters, sizeof(host_counters), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
             cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); rc = GPUVM_E_CUDA; break; }
-        cur_n = host_counters[0];
-        int *t = q0; q0 = q1; q1 = t;
+        found = host_counters[0];
         ++depth;
     }
     cudaStreamSynchronize(s);
