@@ -12,7 +12,7 @@
  *   - calls enqueue work and return without synchronising unless stated; device
  *     errors (a wait that ran out, an offset out of range) are sticky in the handle
  *     and show up in gpuvm_stats().  Return value: 0 or a negative gpuvm_status.
- *   - nothing here allocates device memory except gpuvm_bfs_csr (256 KiB of scratch,
+ *   - nothing here allocates device memory except gpuvm_bfs_csr (1 MiB of scratch,
  *     freed before it returns).
  */
 #ifndef GPUVM_WORKLOADS_H
@@ -51,11 +51,12 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
  * receives the hop distance from `source`, -1 where unreachable.  Per level one
  * sweep over the vertices in ascending order (warps draw chunks of 32 consecutive
  * vertices from a ticket counter, so the grid moves through the arrays in address
- * order) plus one launch for very large neighbour lists, whose edges are spread
- * over the whole grid (the imbalance Section 5.2 describes).  Synchronises the
+ * order; per chunk the column pages its edges span are pinned one at a time) plus
+ * one launch for very long neighbour lists, which are cut at page boundaries and
+ * spread over the whole grid (the imbalance Section 5.2 describes).  Synchronises the
  * stream between levels; *n_levels (host pointer, may be NULL) receives the number
  * of levels expanded, counting the last one that discovers nothing.  Allocates and
- * frees 256 KiB of device scratch (queue of large vertices, counters).
+ * frees 1 MiB of device scratch (queue of neighbour-list pieces, counters).
  */
 int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
                   int32_t *d_level, int *n_levels, void *stream);

@@ -123,21 +123,38 @@ __global__ void __launch_bounds__(1024) gather_kernel(Mem m, unsigned long long 
 
 // ------------------------------------------------------------------------ BFS
 constexpr long long kBigDegree = 4096;     // neighbour lists at least this long are spread over the grid
-constexpr unsigned int kBigQueue = 65536;
+constexpr unsigned int kBigQueue = 65536;  // entries of the span queue (two int64 each)
 
-// counters: [0] vertices discovered in this level, [1] big-vertex queue size, [2] chunk ticket
-//
+// counters: [0] vertices discovered in this level, [1] span queue size, [2] chunk ticket, [3] span ticket
+
+// Visit the edges [elo, ehi) that lie inside the pinned unit starting at edge `first`.
+template <class Mem>
+__device__ __forceinline__ unsigned int bfs_visit(const unsigned char *unit_ptr, long long first, long long elo,
+                                                  long long ehi, unsigned int lane, int *__restrict__ level, int depth)
+{
+    unsigned int found = 0;
+    for (long long e = elo + lane; e < ehi; e += 32) {
+        const int c = Mem::load_i32(unit_ptr + 4 * (e - first));
+        if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1) ++found;
+    }
+    return found;
+}
+
 // One level = one sweep over the vertices in ascending order: a warp draws the next chunk
 // of 32 consecutive vertices from a ticket counter, so at any moment the whole grid works
 // inside a narrow window of the row-offset and column arrays and a level touches every page
-// at most about once, in address order.
+// at most about once, in address order.  Per chunk the warp reads the 33 row offsets with
+// two accessor calls and then walks the column pages that the chunk's edges span, holding
+// one page at a time: one pin per page and chunk instead of one per neighbour list, which
+// keeps the atomic traffic on the entries of the few pages under the window low.
 template <class Mem>
 __global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
                                                         int *__restrict__ level, unsigned int nv,
-                                                        int *__restrict__ big_q, unsigned int *__restrict__ counters,
+                                                        long long *__restrict__ span_q, unsigned int *__restrict__ counters,
                                                         int depth)
 {
     const unsigned int lane = threadIdx.x & 31;
+    const unsigned long long unit = m.unit();
     unsigned int found = 0;
     for (;;) {
         unsigned int chunk = 0;
@@ -147,60 +164,90 @@ __global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long lon
         if (v0 >= nv) break;
         const unsigned long long v = v0 + lane;
         const bool active = v < nv && level[v] == depth;
-        unsigned int mask = __ballot_sync(0xFFFFFFFFu, active);
-        if (!mask) continue;
-        long long lo = 0, hi = 0;
-        if (active) {
-            lo = m.template read<long long>(off_off, v);
-            hi = m.template read<long long>(off_off, v + 1);
-        }
-        while (mask) {
-            const int L = __ffs(mask) - 1;
-            mask &= mask - 1;
+        if (!__any_sync(0xFFFFFFFFu, active)) continue;
+        // row offsets of the chunk: off[v0 .. v0+32], clamped to the nv + 1 entries that exist
+        long long lo = m.template read<long long>(off_off, v < nv ? v : nv);
+        long long hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+        if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
+        if (!active) { lo = 0; hi = 0; }
+        // long neighbour lists: cut them at unit boundaries and queue the pieces for the grid
+        unsigned int bigs = __ballot_sync(0xFFFFFFFFu, hi - lo >= kBigDegree);
+        while (bigs) {
+            const int L = __ffs(bigs) - 1;
+            bigs &= bigs - 1;
             const long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
-            if (bhi - blo >= kBigDegree) {
-                // hand the list to the grid-wide kernel; if its queue is full, expand it here
-                unsigned int slot = 0;
-                if (lane == 0) slot = atomicAdd(counters + 1, 1u);
-                slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
-                if (slot < kBigQueue) {
-                    if (lane == 0) big_q[slot] = (int)(v0 + L);
-                    continue;
-                }
+            const unsigned long long b0 = (col_off + 4ull * blo) / unit, b1 = (col_off + 4ull * bhi - 1) / unit;
+            const unsigned int pieces = (unsigned int)(b1 - b0 + 1);
+            unsigned int slot = 0;
+            if (lane == 0) slot = atomicAdd(counters + 1, pieces);
+            slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
+            if (slot + pieces > kBigQueue) {                       // queue full: expand the list here
+                for (unsigned int k = slot + lane; k < kBigQueue; k += 32) { span_q[2 * k] = 0; span_q[2 * k + 1] = 0; }
+                continue;
             }
-            for (long long base = blo; base < bhi; base += 32) {
-                const long long e = base + lane;
-                if (e < bhi) {
-                    const int c = m.template read<int>(col_off, (unsigned long long)e);
-                    if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1) ++found;
-                }
+            for (unsigned int k = lane; k < pieces; k += 32) {
+                const long long s = (long long)(((b0 + k) * unit - col_off + 3) / 4);
+                const long long t = (long long)(((b0 + k + 1) * unit - col_off) / 4);
+                span_q[2 * (slot + k)] = k == 0 ? blo : s;
+                span_q[2 * (slot + k) + 1] = t < bhi ? t : bhi;
             }
+            if ((int)lane == L) { lo = 0; hi = 0; }
+        }
+        // the edges of this chunk, unit by unit
+        long long rlo = hi > lo ? lo : 0x7FFFFFFFFFFFFFFFll, rhi = hi > lo ? hi : 0;
+        for (int o = 16; o; o >>= 1) {
+            const long long a = __shfl_xor_sync(0xFFFFFFFFu, rlo, o), b = __shfl_xor_sync(0xFFFFFFFFu, rhi, o);
+            rlo = a < rlo ? a : rlo;
+            rhi = b > rhi ? b : rhi;
+        }
+        long long first = rlo;
+        while (first < rhi) {
+            const unsigned long long byte = col_off + 4ull * first;
+            long long last = (long long)(((byte / unit + 1) * unit - col_off) / 4);   // first edge of the next unit
+            if (last > rhi) last = rhi;
+            unsigned int touch = __ballot_sync(0xFFFFFFFFu, lo < last && hi > first);
+            if (touch) {
+                gpuvm_token tok;
+                const unsigned char *p = m.pin(byte, GPUVM_READ, tok);
+                if (!p) return;
+                while (touch) {
+                    const int L = __ffs(touch) - 1;
+                    touch &= touch - 1;
+                    long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
+                    if (blo < first) blo = first;
+                    if (bhi > last) bhi = last;
+                    found += bfs_visit<Mem>(p, first, blo, bhi, lane, level, depth);
+                }
+                m.release(tok);
+            }
+            first = last;
         }
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
     if (lane == 0 && found) atomicAdd(counters, found);
 }
 
+// Pieces of long neighbour lists, one warp per piece (a piece never crosses a unit).
 template <class Mem>
-__global__ void __launch_bounds__(256) bfs_big_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
-                                                      int *__restrict__ level, const int *__restrict__ big_q,
-                                                      unsigned int *__restrict__ counters, int depth)
+__global__ void __launch_bounds__(256) bfs_span_kernel(Mem m, unsigned long long col_off, int *__restrict__ level,
+                                                       const long long *__restrict__ span_q,
+                                                       unsigned int *__restrict__ counters, int depth)
 {
     const unsigned int lane = threadIdx.x & 31;
-    const unsigned int n_big = counters[1] < kBigQueue ? counters[1] : kBigQueue;
+    const unsigned int n = counters[1] < kBigQueue ? counters[1] : kBigQueue;
     unsigned int found = 0;
-    for (unsigned int i = 0; i < n_big; ++i) {
-        const int v = big_q[i];
-        long long r = 0;
-        if (lane < 2) r = m.template read<long long>(off_off, (unsigned long long)v + lane);
-        const long long lo = __shfl_sync(0xFFFFFFFFu, r, 0), hi = __shfl_sync(0xFFFFFFFFu, r, 1);
-        for (long long base = lo + 32ll * warp_in_grid(); base < hi; base += 32ll * warps_in_grid()) {
-            const long long e = base + lane;
-            if (e < hi) {
-                const int c = m.template read<int>(col_off, (unsigned long long)e);
-                if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1) ++found;
-            }
-        }
+    for (;;) {
+        unsigned int i = 0;
+        if (lane == 0) i = atomicAdd(counters + 3, 1u);
+        i = __shfl_sync(0xFFFFFFFFu, i, 0);
+        if (i >= n) break;
+        const long long elo = span_q[2 * i], ehi = span_q[2 * i + 1];
+        if (ehi <= elo) continue;
+        gpuvm_token tok;
+        const unsigned char *p = m.pin(col_off + 4ull * elo, GPUVM_READ, tok);
+        if (!p) return;
+        found += bfs_visit<Mem>(p, elo, elo, ehi, lane, level, depth);
+        m.release(tok);
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
     if (lane == 0 && found) atomicAdd(counters, found);
@@ -399,26 +446,25 @@ int run_gather(const Mem &m, size_t x_off, const int64_t *d_idx, size_t n_idx, s
     return launched();
 }
 
+constexpr size_t kBfsScratchBytes = 2 * kBigQueue * sizeof(long long) + 4 * sizeof(unsigned int);
+
+// One BFS on caller-provided scratch (kBfsScratchBytes, 16-byte aligned).
 template <class Mem>
-int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
-            cudaStream_t s)
+int bfs_levels(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
+               void *scratch, cudaStream_t s)
 {
-    if (!d_level || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
-    if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
-    int *scratch = nullptr;                       // big-vertex queue + 4 counters
-    if (cudaMalloc(&scratch, (kBigQueue + 4) * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_ALLOC; }
-    int *big_q = scratch;
-    unsigned int *counters = reinterpret_cast<unsigned int *>(scratch + kBigQueue);
+    long long *span_q = static_cast<long long *>(scratch);
+    unsigned int *counters = reinterpret_cast<unsigned int *>(span_q + 2 * kBigQueue);
     cudaMemsetAsync(d_level, 0xFF, nv * sizeof(int32_t), s);
     bfs_init_kernel<<<1, 1, 0, s>>>(d_level, (int)source);
     int rc = launched();
     int depth = 0;
-    const int grid = sm_count() * 4;
+    const int grid = sm_count() * 2;
     unsigned int found = 1;
     while (rc == GPUVM_OK && found > 0) {
         cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
-        bfs_sweep_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, (unsigned int)nv, big_q, counters, depth);
-        bfs_big_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, big_q, counters, depth);
+        bfs_sweep_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, (unsigned int)nv, span_q, counters, depth);
+        bfs_span_kernel<Mem><<<grid, 256, 0, s>>>(m, col_off, d_level, span_q, counters, depth);
         rc = launched(2);
         unsigned int host_counters[2] = {0, 0};
         if (cudaMemcpyAsync(host_counters, counters, sizeof(host_counters), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
@@ -426,9 +472,21 @@ int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t sour
         found = host_counters[0];
         ++depth;
     }
+    if (n_levels) *n_levels = depth;
+    return rc;
+}
+
+template <class Mem>
+int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
+            cudaStream_t s)
+{
+    if (!d_level || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
+    if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
+    void *scratch = nullptr;                       // span queue + 4 counters
+    if (cudaMalloc(&scratch, kBfsScratchBytes) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_ALLOC; }
+    int rc = bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, s);
     cudaStreamSynchronize(s);
     cudaFree(scratch);
-    if (n_levels) *n_levels = depth;
     return rc;
 }
 
