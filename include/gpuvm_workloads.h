@@ -62,6 +62,39 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
                   int32_t *d_level, int *n_levels, void *stream);
 
 /*
+ * gpuvm_bfs_csr for callers that must not allocate.  (The paper has no counterpart:
+ * this entry point exists for the sake of such callers only.)
+ *
+ * Some callers cannot afford a cudaMalloc / cudaFree pair in the middle of their
+ * work: code that runs between the phases of a latency-sensitive pipeline (device
+ * allocation synchronises the whole device and may take a driver lock), plug-ins
+ * whose host forbids allocation after start-up, and processes that have handed
+ * all free device memory to their own pool, where cudaMalloc would simply fail.
+ * For them this variant does exactly what gpuvm_bfs_csr does, same kernels, same
+ * arguments, same results, but takes its scratch (the queue of neighbour-list
+ * pieces and the level counters, 1 MiB + 16 bytes) from an array that is part of
+ * the library's device image.  It calls no cudaMalloc, cudaFree or other
+ * allocating routine.
+ *
+ *   - Limit: nv <= GPUVM_BFS_NOALLOC_MAX_VERTICES, the graph size the fixed queue
+ *     is sized for; anything larger returns GPUVM_E_RANGE and runs nothing.
+ *   - Cost: every device that loads the library holds the 1 MiB array until the
+ *     process exits, whether or not this function is ever called.
+ *   - The first call on a device looks up the array's device address (once per
+ *     device, with that device current).  Make that first call during set-up,
+ *     before any stream capture is started.
+ *   - All calls on one device share the array.  Two calls whose kernels overlap
+ *     on the GPU (different streams, different threads) race on it and give wrong
+ *     levels; issue them one after the other.  Nothing needs clearing between
+ *     calls: each level re-zeroes the counters, and queue entries are written
+ *     before they are read.
+ * d_level, n_levels, stream, return value: as for gpuvm_bfs_csr.
+ */
+#define GPUVM_BFS_NOALLOC_MAX_VERTICES ((size_t)1 << 26)
+int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
+                          int32_t *d_level, int *n_levels, void *stream);
+
+/*
  * Vector add c[i] = a[i] + b[i] over three paged fp32 arrays of n elements
  * (Listing 1).  c is written through the runtime: its pages become dirty and reach
  * the host by eviction write-back or gpuvm_flush.  One IEEE binary32 addition per

@@ -71,6 +71,7 @@ SYMBOLS = {
     "gpuvm_stream_sum_i32": (_i, [_vp, _sz, _sz, _vp, _vp]),
     "gpuvm_gather_f32": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp, _vp]),
     "gpuvm_bfs_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
+    "gpuvm_bfs_csr_noalloc": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_vadd_f32": (_i, [_vp, _sz, _sz, _sz, _sz, _vp]),
     "gpuvm_embag_f32": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_scatter_update_u32": (_i, [_vp, _sz, _vp, _sz, _vp]),
@@ -224,6 +225,18 @@ def gpuvm_bfs_csr(h, off_off: int, col_off: int, nv: int, source: int, d_level, 
     levels = _i(0)
     _check(lib().gpuvm_bfs_csr(h, off_off, col_off, nv, source, _ptr(d_level), ctypes.byref(levels), _stream(stream)),
            "gpuvm_bfs_csr")
+    return levels.value
+
+
+BFS_NOALLOC_MAX_VERTICES = 1 << 26
+
+
+def gpuvm_bfs_csr_noalloc(h, off_off: int, col_off: int, nv: int, source: int, d_level, stream=None) -> int:
+    """gpuvm_bfs_csr on the library's built-in scratch array: no device allocation is made.
+    Calls on one device must not overlap; the first call per device belongs in set-up."""
+    levels = _i(0)
+    _check(lib().gpuvm_bfs_csr_noalloc(h, off_off, col_off, nv, source, _ptr(d_level), ctypes.byref(levels),
+                                       _stream(stream)), "gpuvm_bfs_csr_noalloc")
     return levels.value
 
 

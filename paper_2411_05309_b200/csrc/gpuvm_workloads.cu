@@ -516,6 +516,31 @@ int run_embag(const Mem &m, size_t t_off, size_t dims, const int64_t *d_rows, si
     return launched();
 }
 
+
+// ---- scratch for gpuvm_bfs_csr_noalloc: lives in the module image of every device that loads
+// this library, from load until exit.  Host code must never pass `g_bfs_static_scratch` itself
+// to a kernel: in host code that name is only a stand-in for the symbol, not a device
+// address.  The real address comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_bfs_static_scratch[kBfsScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::atomic<void *> g_bfs_static_ptr[kMaxDevices];
+
+// Device address of the static scratch on the current device (looked up on first use).
+int bfs_static_scratch(void **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return GPUVM_E_NODEVICE; }
+    void *p = g_bfs_static_ptr[dev].load();
+    if (!p) {
+        cudaError_t e = cudaGetSymbolAddress(&p, g_bfs_static_scratch);
+        if (e != cudaSuccess || !p) { cudaGetLastError(); return GPUVM_E_CUDA; }
+        g_bfs_static_ptr[dev].store(p);
+    }
+    *out = p;
+    return GPUVM_OK;
+}
+
 struct PagedH : Paged { unsigned long long unit_host() const { return 1ull << vm.page_shift; } };
 struct RawH : Raw { unsigned long long unit_host() const { return unit_bytes; } };
 
@@ -547,6 +572,22 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
     return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level,
+                          int *n_levels, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    if (!d_level || nv == 0 || source >= nv) return GPUVM_E_ARG;
+    if (nv > GPUVM_BFS_NOALLOC_MAX_VERTICES) return GPUVM_E_RANGE;     // beyond what the fixed scratch is sized for
+    if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
+    void *scratch = nullptr;
+    int rc = bfs_static_scratch(&scratch);
+    if (rc != GPUVM_OK) return rc;
+    // bfs_levels zeroes the counters at the start of every level and writes each queue entry
+    // before reading it, so whatever the previous call left in the array does not matter
+    return bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n, void *stream)
