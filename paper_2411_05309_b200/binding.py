@@ -50,7 +50,7 @@ class Check(ctypes.Structure):
         return {n: getattr(self, n) for n, _ in self._fields_}
 
 
-# name -> (restype, argtypes): every symbol declared in include/gpuvm.h and gpuvm_workloads.h
+# name -> (restype, argtypes): every symbol declared in include/*.h
 _vp, _sz, _i, _u64 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64
 SYMBOLS = {
     "gpuvm_create": (_i, [ctypes.POINTER(_vp), _vp, _sz, _sz, _sz]),
@@ -83,6 +83,13 @@ SYMBOLS = {
     "gpuvm_raw_embag_f32": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_link_peak": (_i, [_vp, _vp, _sz, _i, ctypes.POINTER(ctypes.c_double)]),
     "gpuvm_launch_count": (ctypes.c_ulonglong, []),
+    "gpuvm_uvm_alloc": (_i, [ctypes.POINTER(_vp), _sz]),
+    "gpuvm_uvm_free": (_i, [_vp]),
+    "gpuvm_uvm_advise_read_mostly": (_i, [_vp, _sz, _i]),
+    "gpuvm_uvm_evict_to_host": (_i, [_vp, _sz]),
+    "gpuvm_mem_info": (_i, [ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
+    "gpuvm_balloon_alloc": (_i, [ctypes.POINTER(_vp), _sz]),
+    "gpuvm_balloon_free": (_i, [_vp]),
 }
 
 _lib = None
@@ -286,3 +293,39 @@ def gpuvm_link_peak(host_ptr, d_buf, nbytes: int, reps: int = 3):
     out = (ctypes.c_double * 3)()
     _check(lib().gpuvm_link_peak(_ptr(host_ptr), _ptr(d_buf), nbytes, reps, out), "gpuvm_link_peak")
     return {"h2d_gbs": out[0], "d2h_gbs": out[1], "duplex_gbs": out[2]}
+
+
+# ------------------------------------------------------------ managed-memory helpers
+
+def gpuvm_uvm_alloc(nbytes: int) -> int:
+    p = _vp()
+    _check(lib().gpuvm_uvm_alloc(ctypes.byref(p), nbytes), "gpuvm_uvm_alloc")
+    return p.value
+
+
+def gpuvm_uvm_free(p: int):
+    _check(lib().gpuvm_uvm_free(p), "gpuvm_uvm_free")
+
+
+def gpuvm_uvm_advise_read_mostly(p: int, nbytes: int, on: bool):
+    _check(lib().gpuvm_uvm_advise_read_mostly(p, nbytes, int(on)), "gpuvm_uvm_advise_read_mostly")
+
+
+def gpuvm_uvm_evict_to_host(p: int, nbytes: int):
+    _check(lib().gpuvm_uvm_evict_to_host(p, nbytes), "gpuvm_uvm_evict_to_host")
+
+
+def gpuvm_mem_info():
+    f, t = _sz(0), _sz(0)
+    _check(lib().gpuvm_mem_info(ctypes.byref(f), ctypes.byref(t)), "gpuvm_mem_info")
+    return f.value, t.value
+
+
+def gpuvm_balloon_alloc(leave_free: int) -> int:
+    p = _vp()
+    _check(lib().gpuvm_balloon_alloc(ctypes.byref(p), leave_free), "gpuvm_balloon_alloc")
+    return p.value or 0
+
+
+def gpuvm_balloon_free(p: int):
+    _check(lib().gpuvm_balloon_free(p), "gpuvm_balloon_free")

@@ -15,7 +15,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libgpuvm.so")
-SOURCES = ["gpuvm_host.cu", "gpuvm_workloads.cu"]
+SOURCES = ["gpuvm_host.cu", "gpuvm_workloads.cu", "gpuvm_uvm.cu"]
 
 
 def _nvcc() -> str:

@@ -1,0 +1,131 @@
+"""The same workload kernels over cudaMallocManaged memory (the paper's UVM baseline).
+
+The paged arrays of a prepared workload are copied into one managed allocation, device
+memory is limited with a balloon allocation so that only about ``pool_bytes`` remain for
+managed pages (the paper "artificially limits the GPU memory", Section 5.4), all pages are
+sent back to the host for a cold start, and the ``gpuvm_raw_*`` twin of the workload kernel
+is timed with CUDA events.  Read-only workloads are run a second time with
+cudaMemAdviseSetReadMostly; the time of the advise call is reported separately, as the paper
+does (Section 5.2).
+
+A kernel that thrashes under UVM cannot be stopped from the host, so the random-access
+workloads (gather, embedding bag) are run on a growing prefix of their index list: the
+prefix is quadrupled while a run stays under ``budget_s / 8`` seconds, and the figure
+reported is that of the largest prefix, labelled with its size.
+"""
+from __future__ import annotations
+
+import ctypes
+import time
+
+import numpy as np
+
+from . import binding as B
+
+SLACK = 64 << 20          # device memory left to the driver on top of the pool
+
+
+def _timed(torch, fn):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    fn()
+    e1.record()
+    e1.synchronize()
+    return e0.elapsed_time(e1) / 1e3
+
+
+def run_twin(w, cfg: int, timeout_s: float = 120.0) -> dict:
+    import torch
+    out = {"leave_free_bytes": w.pool_bytes + SLACK, "runs": []}
+    p = B.gpuvm_uvm_alloc(w.nbytes)
+    balloon = 0
+    try:
+        ctypes.memmove(p, B.gpuvm_host_ptr(w.h), w.nbytes)          # first touch on the CPU
+        bufs = _outputs(torch, w, cfg)                               # before the balloon takes the rest
+        torch.cuda.empty_cache()
+        balloon = B.gpuvm_balloon_alloc(w.pool_bytes + SLACK)
+        free_b, total_b = B.gpuvm_mem_info()
+        out["free_bytes_under_balloon"] = free_b
+        read_only = cfg != 4
+        for advise in ([False, True] if read_only else [False]):
+            rec = {"read_mostly": advise}
+            if advise:
+                t0 = time.perf_counter()
+                B.gpuvm_uvm_advise_read_mostly(p, w.nbytes, True)
+                torch.cuda.synchronize()
+                rec["advise_seconds"] = time.perf_counter() - t0
+            rec.update(_one(torch, w, cfg, p, timeout_s / (2 if read_only else 1), bufs))
+            if advise:
+                B.gpuvm_uvm_advise_read_mostly(p, w.nbytes, False)
+            out["runs"].append(rec)
+    finally:
+        if balloon:
+            B.gpuvm_balloon_free(balloon)
+        B.gpuvm_uvm_free(p)
+    return out
+
+
+def _outputs(torch, w, cfg: int) -> dict:
+    if cfg == 1:
+        return {"sum": torch.zeros(1, dtype=torch.int64, device="cuda")}
+    if cfg == 2:
+        nb = (w.n_idx + w.block - 1) // w.block
+        return {"fs": torch.zeros(nb, dtype=torch.float32, device="cuda"),
+                "bs": torch.zeros(nb, dtype=torch.int64, device="cuda")}
+    if cfg == 3:
+        return {"lvl": torch.zeros(w.nv, dtype=torch.int32, device="cuda")}
+    if cfg == 5:
+        return {"out": torch.zeros(w.n_bags * w.dims, dtype=torch.float32, device="cuda")}
+    return {}
+
+
+def _one(torch, w, cfg: int, p: int, budget_s: float, bufs: dict) -> dict:
+    def cold():
+        B.gpuvm_uvm_evict_to_host(p, w.nbytes)
+
+    if cfg == 1:
+        got = bufs["sum"]
+        cold()
+        t = _timed(torch, lambda: B.gpuvm_raw_stream_sum_i32(p + w.off["a"], w.n, got))
+        return {"seconds": t, "effective_gbs": 4 * w.n / t / 1e9, "matches_paged_result": bool(got.item() == w.d_sum.item()),
+                "scaled": False}
+    if cfg == 3:
+        lvl = bufs["lvl"]
+        cold()
+        t = _timed(torch, lambda: B.gpuvm_raw_bfs_csr(p + w.off["off"], p + w.off["col"], w.nv, 0, lvl))
+        return {"seconds": t, "effective_gbs": w.effective_bytes() / t / 1e9,
+                "matches_paged_result": bool(torch.equal(lvl, w.d_level)), "scaled": False}
+    if cfg == 4:
+        cold()
+        t = _timed(torch, lambda: B.gpuvm_raw_vadd_f32(p + w.off["a"], p + w.off["b"], p + w.off["c"], w.n))
+        c = np.ctypeslib.as_array((ctypes.c_uint32 * w.n).from_address(p + w.off["c"]))
+        ref = w.view("c", np.uint32, w.n)
+        step = 1 << 24
+        same = all(np.array_equal(c[i:i + step], ref[i:i + step]) for i in range(0, w.n, step * 16))
+        return {"seconds": t, "effective_gbs": 12 * w.n / t / 1e9, "matches_paged_result": bool(same), "scaled": False}
+    # random-access workloads: growing prefix of the index list
+    if cfg == 2:
+        total, unit_bytes, per = w.n_idx, 4, w.block
+    else:
+        total, unit_bytes, per = w.n_bags, 4 * w.dims * w.bag, 1
+    n = min(total, (1 << 14) if cfg == 2 else (1 << 9))
+    best = None
+    spent = 0.0
+    while True:
+        n = n // per * per if per > 1 else n
+        cold()
+        if cfg == 2:
+            nb = (n + w.block - 1) // w.block
+            fs, bs = bufs["fs"][:nb], bufs["bs"][:nb]
+            t = _timed(torch, lambda: B.gpuvm_raw_gather_f32(p + w.off["x"], w.d_idx, n, w.block, fs, bs))
+            same = bool(torch.equal(bs, w.d_bsum[:nb]))
+        else:
+            o = bufs["out"][:n * w.dims]
+            t = _timed(torch, lambda: B.gpuvm_raw_embag_f32(p + w.off["t"], w.dims, w.d_rows, n, w.bag, o))
+            same = bool(torch.equal(o, w.d_out[:n * w.dims]))
+        spent += t
+        best = {"seconds": t, "effective_gbs": n * unit_bytes / t / 1e9, "matches_paged_result": same,
+                "scaled": n < total, "units_run": n, "units_total": total}
+        if n >= total or t > budget_s / 8 or spent + 4 * t > budget_s:
+            return best
+        n = min(total, n * 4)

@@ -12,7 +12,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def declared_functions():
     names = []
-    for hdr in ("gpuvm.h", "gpuvm_workloads.h"):
+    for hdr in ("gpuvm.h", "gpuvm_workloads.h", "gpuvm_uvm.h"):
         text = open(os.path.join(ROOT, "include", hdr)).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
         names += re.findall(r"\b(gpuvm_[a-z0-9_]+)\s*\(", text)
