@@ -207,6 +207,23 @@ NAMES = {1: "cfg1 streaming read-reduce: int64 sum over 64 MiB int32, 4 KiB page
 DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32"}
 
 
+# ---------------------------------------------------------------------- rank plumbing
+
+def max_over_ranks(dist, values, device="cpu"):
+    """Element-wise maximum of `values` over all ranks (the slowest rank sets the time)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return list(values)
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def replica_throughput(world: int, units_per_rank: float, slowest_seconds: float) -> float:
+    """Whole-job throughput of `world` independent replicas: all units over the slowest time."""
+    return world * units_per_rank / slowest_seconds
+
+
 # ------------------------------------------------------------------------------- ours
 
 def e2e_step(torch, B, w, cfg: int):
@@ -272,10 +289,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     step_s = sum(r.seconds for r in results) / len(results)
     kern_s = sum(r.kernel_seconds for r in results) / len(results)
-    if dist is not None:
-        t = torch.tensor([step_s, kern_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_s, kern_s = t.tolist()
+    e2e_s = sum(t for t, _, _ in e2e) / len(e2e)
+    step_s, kern_s, e2e_s = max_over_ranks(dist, [step_s, kern_s, e2e_s], "cuda")
     eff_bytes = results[-1].effective_bytes
     st = results[-1].stats
     ck = results[-1].check
@@ -286,7 +301,6 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     hbm_peak = peaks.get("hbm_gbs", 6650.0)
     link_peak = link["ce_h2d_gbs"] if bytes_out == 0 else link["ce_h2d_gbs"] + link["ce_d2h_gbs"]
     moved = bytes_in + bytes_out
-    e2e_s = sum(t for t, _, _ in e2e) / len(e2e)
 
     if rank != 0:
         if dist is not None:
@@ -295,7 +309,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         return
 
     line = {
-        "metric": METRIC, "value": world * eff_bytes / step_s / 1e9, "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": replica_throughput(world, eff_bytes, step_s) / 1e9, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": DTYPES[args.workload], "data": "synthetic",
         "config": {**w.describe(), "workload": NAMES[args.workload], "replicas": world,
@@ -321,7 +335,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                     "peak_source": "MEASURED_PEAKS.json" if peaks else "fallback"},
             "kernel_ms": kern_s * 1e3,
         },
-        "e2e": {"value": world * eff_bytes / e2e_s / 1e9, "unit": UNIT, "h2d_bytes_per_step": e2e[-1][1],
+        "e2e": {"value": replica_throughput(world, eff_bytes, e2e_s) / 1e9, "unit": UNIT, "h2d_bytes_per_step": e2e[-1][1],
                 "d2h_bytes_per_step": e2e[-1][2], "ms_per_step": e2e_s * 1e3},
         "gpu_launches": launches, "clocks": clocks, "wall_s": wall,
     }
@@ -331,7 +345,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                                 "sample": sample, "seconds": dt}
     if args.uvm:
         from paper_2411_05309_b200 import uvm
-        line["uvm"] = uvm.run_twin(w, args.workload, timeout_s=args.uvm_timeout)
+        w.close()
+        line["uvm"] = uvm.run_twin(args.workload, args.shrink, timeout_s=args.uvm_timeout)
     w.close()
     if dist is not None:
         dist.destroy_process_group()
