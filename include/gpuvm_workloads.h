@@ -37,12 +37,19 @@ int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void
  *   d_fsum[b] = float( sum of x[idx[k]] accumulated in double )
  *   d_bsum[b] = sum of the 32-bit patterns of the gathered values (int64, exact).
  * x: fp32 array at x_off; d_idx: n_idx int64 element indices in device memory.
- * One thread per index through gpuvm_read<float>; every warp may fault on up to
- * 32 different pages at once (Section 3.3: intra- and inter-warp coalescing).
  * d_fsum, d_bsum: ceil(n_idx / block) elements.  block <= 2^20.
+ *
+ * gpuvm_gather_f32: one warp per block; the warp stages up to 1024 page ids in shared
+ * memory and keeps all of them registered in the page table at once (gpuvm_batch.cuh),
+ * so that one migrated page serves many waiting requests (Section 3.3: inter-warp
+ * coalescing).  Uses 128 KiB of dynamic shared memory per thread block.
+ * gpuvm_gather_f32_unbatched: one thread per index through gpuvm_read<float>, one
+ * thread block per index block; at most 32 requests per warp are in flight.
  */
 int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx, size_t block,
                      float *d_fsum, int64_t *d_bsum, void *stream);
+int gpuvm_gather_f32_unbatched(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx, size_t block,
+                               float *d_fsum, int64_t *d_bsum, void *stream);
 
 /*
  * Level-synchronous BFS over a CSR graph whose int64 row offsets (nv + 1 of them,

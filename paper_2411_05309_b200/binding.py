@@ -70,6 +70,7 @@ SYMBOLS = {
     "gpuvm_last_cuda_error": (_i, [_vp]),
     "gpuvm_stream_sum_i32": (_i, [_vp, _sz, _sz, _vp, _vp]),
     "gpuvm_gather_f32": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp, _vp]),
+    "gpuvm_gather_f32_unbatched": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp, _vp]),
     "gpuvm_bfs_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_bfs_csr_noalloc": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_vadd_f32": (_i, [_vp, _sz, _sz, _sz, _sz, _vp]),
@@ -226,6 +227,11 @@ def gpuvm_stream_sum_i32(h, a_off: int, n: int, d_sum, stream=None):
 def gpuvm_gather_f32(h, x_off: int, d_idx, n_idx: int, block: int, d_fsum, d_bsum, stream=None):
     _check(lib().gpuvm_gather_f32(h, x_off, _ptr(d_idx), n_idx, block, _ptr(d_fsum), _ptr(d_bsum), _stream(stream)),
            "gpuvm_gather_f32")
+
+
+def gpuvm_gather_f32_unbatched(h, x_off: int, d_idx, n_idx: int, block: int, d_fsum, d_bsum, stream=None):
+    _check(lib().gpuvm_gather_f32_unbatched(h, x_off, _ptr(d_idx), n_idx, block, _ptr(d_fsum), _ptr(d_bsum),
+                                            _stream(stream)), "gpuvm_gather_f32_unbatched")
 
 
 def gpuvm_bfs_csr(h, off_off: int, col_off: int, nv: int, source: int, d_level, stream=None) -> int:

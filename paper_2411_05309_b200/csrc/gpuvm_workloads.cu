@@ -5,8 +5,10 @@
 
 #include <atomic>
 #include <cstdint>
+#include <cstdlib>
 
 #include "gpuvm.h"
+#include "gpuvm_batch.cuh"
 #include "gpuvm_device.cuh"
 #include "gpuvm_internal.h"
 #include "gpuvm_workloads.h"
@@ -119,6 +121,90 @@ __global__ void __launch_bounds__(1024) gather_kernel(Mem m, unsigned long long 
         }
         __syncthreads();
     }
+}
+
+// A requester warp takes a run of consecutive indices (whole index blocks when they fit),
+// stages their page requests in its slice of shared memory, registers them all in the page
+// table, and as the pages arrive replaces each request by the value it asked for
+// (gpuvm_batch.cuh); then it adds the values up block by block.  The faults it owns go to
+// the thread block's ring of page ids, which the block's migrator warps serve.  No
+// block-wide barrier after start-up: warps never wait for one another.
+constexpr int kGatherRequesters = 24;
+constexpr int kGatherMigrators = 4;
+constexpr int kGatherMaxWarps = 32;
+constexpr unsigned int kGatherBatch = 1024;       // requests per requester warp
+
+__global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(gpuvm_dev_t vm, unsigned long long x_off,
+                                                                            const long long *__restrict__ idx,
+                                                                            unsigned long long n_idx, unsigned long long block,
+                                                                            float *__restrict__ fsum, long long *__restrict__ bsum,
+                                                                            int requesters, unsigned int batch)
+{
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    gpuvm_fault_queue *queue = reinterpret_cast<gpuvm_fault_queue *>(s_raw);
+    gpuvm_batch_entry *tables = reinterpret_cast<gpuvm_batch_entry *>(s_raw + sizeof(gpuvm_fault_queue));
+    const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
+        reinterpret_cast<unsigned int *>(queue)[k] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) queue->requesters = (unsigned int)requesters;
+    __syncthreads();
+    if ((int)warp >= requesters) {
+        gpuvm_migrator_loop(vm, queue);
+        return;
+    }
+    gpuvm_batch_entry *table = tables + (size_t)warp * batch;
+    const unsigned long long nb = (n_idx + block - 1) / block;
+    const unsigned long long per = block <= batch ? batch / block : 1;      // index blocks per work item
+    const unsigned long long items = (nb + per - 1) / per;
+    const unsigned long long stride = (unsigned long long)gridDim.x * requesters;
+    for (unsigned long long t = (unsigned long long)blockIdx.x * requesters + warp; t < items; t += stride) {
+        const unsigned long long lo = t * per * block;
+        const unsigned long long hi = (t + 1) * per * block < n_idx ? (t + 1) * per * block : n_idx;
+        double carry_f = 0.0;               // a block longer than one batch is summed piece by piece
+        long long carry_b = 0;
+        for (unsigned long long base = lo; base < hi; base += batch) {
+            const unsigned int n = (unsigned int)(hi - base < batch ? hi - base : batch);
+            for (unsigned int k = lane; k < n; k += 32)
+                gpuvm_batch_set(vm, table, k, x_off + 4ull * (unsigned long long)idx[base + k]);
+            __syncwarp();
+            gpuvm_batch_access(vm, table, n, GPUVM_READ, [table](unsigned int i, const unsigned char *p) {
+                table[i].vpn = gpuvm_load(reinterpret_cast<const unsigned int *>(p));
+                table[i].offl = 1u;                              // served
+            }, queue);
+            __syncwarp();
+            // sum the values of this piece, index block by index block
+            unsigned long long pos = base;
+            while (pos < base + n) {
+                const unsigned long long b = pos / block;
+                unsigned long long end = (b + 1) * block;
+                if (end > base + n) end = base + n;
+                double f = 0.0;
+                long long bits = 0;
+                for (unsigned long long k = pos + lane; k < end; k += 32) {
+                    const gpuvm_batch_entry e = table[k - base];
+                    if (e.offl == 1u) {
+                        f += (double)__uint_as_float(e.vpn);
+                        bits += (long long)e.vpn;
+                    }
+                }
+                for (int o = 16; o; o >>= 1) {
+                    f += __shfl_down_sync(0xFFFFFFFFu, f, o);
+                    bits += __shfl_down_sync(0xFFFFFFFFu, bits, o);
+                }
+                carry_f += f;
+                carry_b += bits;
+                if (end == (b + 1) * block || end == n_idx) {    // the index block is complete
+                    if (lane == 0) { fsum[b] = (float)carry_f; bsum[b] = carry_b; }
+                    carry_f = 0.0;
+                    carry_b = 0;
+                }
+                pos = end;
+            }
+            __syncwarp();
+        }
+    }
+    if (lane == 0) gpuvm_requester_done(queue);
 }
 
 // ------------------------------------------------------------------------ BFS
@@ -560,6 +646,40 @@ int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void
 
 int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx, size_t block, float *d_fsum,
                      int64_t *d_bsum, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    if (!d_idx || !d_fsum || !d_bsum || block == 0 || block > (size_t(1) << 20)) return GPUVM_E_ARG;
+    if (x_off % 16) return GPUVM_E_ALIGN;
+    if (n_idx == 0) return GPUVM_OK;
+    static bool configured = false;
+    int requesters = getenv("GPUVM_TUNE_REQUESTERS") ? atoi(getenv("GPUVM_TUNE_REQUESTERS")) : kGatherRequesters;
+    int migrators = getenv("GPUVM_TUNE_MIGRATORS") ? atoi(getenv("GPUVM_TUNE_MIGRATORS")) : kGatherMigrators;
+    unsigned int batch = getenv("GPUVM_TUNE_BATCH") ? (unsigned int)atoi(getenv("GPUVM_TUNE_BATCH")) : kGatherBatch;
+    if (requesters < 1 || migrators < 1 || requesters + migrators > kGatherMaxWarps) return GPUVM_E_ARG;
+    if (batch < 32 || batch > GPUVM_BATCH_MAX || batch % 32) return GPUVM_E_ARG;
+    const size_t smem = sizeof(gpuvm_fault_queue) + (size_t)requesters * batch * sizeof(gpuvm_batch_entry);
+    if (smem > 227 * 1024) return GPUVM_E_ARG;
+    if (!configured) {
+        if (cudaFuncSetAttribute(gather_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
+            cudaGetLastError();
+            return GPUVM_E_CUDA;
+        }
+        configured = true;
+    }
+    const size_t nb = (n_idx + block - 1) / block;
+    const size_t per = block <= batch ? batch / block : 1;
+    const size_t items = (nb + per - 1) / per;
+    const size_t blocks_needed = (items + requesters - 1) / requesters;
+    const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
+    gather_batch_kernel<<<grid, (requesters + migrators) * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+        m.vm, x_off, reinterpret_cast<const long long *>(d_idx), n_idx, block, d_fsum, reinterpret_cast<long long *>(d_bsum),
+        requesters, batch);
+    return launched();
+}
+
+int gpuvm_gather_f32_unbatched(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx, size_t block, float *d_fsum,
+                               int64_t *d_bsum, void *stream)
 {
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;

@@ -67,9 +67,11 @@ def test_stream_sum(B, page, n, frames, policy):
     (256, 1 << 12, 5000, 100, 3),                  # block smaller than a CTA
     (65536, 1 << 20, 1 << 15, 1024, 16),
     (64, 4096, 3000, 1024, 1),                     # one frame: every warp fights for it
+    (4096, 1 << 16, 9000, 3000, 5),                # blocks longer than one batch of 1024
 ])
 @pytest.mark.parametrize("policy", POLICIES)
-def test_gather(B, page, n, n_idx, block, frames, policy):
+@pytest.mark.parametrize("batched", [True, False])
+def test_gather(B, page, n, n_idx, block, frames, policy, batched):
     import torch
     x = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(2))
     idx = inputs.fill_index_i64(np.empty(n_idx, np.int64), n_idx, inputs.config_seed(2, 1), n)
@@ -78,7 +80,8 @@ def test_gather(B, page, n, n_idx, block, frames, policy):
     fsum = torch.zeros(nb, dtype=torch.float32, device="cuda")
     bsum = torch.zeros(nb, dtype=torch.int64, device="cuda")
     with paged(ar.host, page, frames, policy) as h:
-        B.gpuvm_gather_f32(h, ar.off["x"], dev(idx), n_idx, block, fsum, bsum)
+        run = B.gpuvm_gather_f32 if batched else B.gpuvm_gather_f32_unbatched
+        run(h, ar.off["x"], dev(idx), n_idx, block, fsum, bsum)
         st, ck = finish(h)
     ref_f, ref_b = oracle.gather_block_sums_direct(x, idx, block)
     assert np.array_equal(bsum.cpu().numpy(), ref_b)                     # which elements: exact
