@@ -13,7 +13,8 @@
  *     errors (a wait that ran out, an offset out of range) are sticky in the handle
  *     and show up in gpuvm_stats().  Return value: 0 or a negative gpuvm_status.
  *   - nothing here allocates device memory except gpuvm_bfs_csr (1 MiB of scratch,
- *     freed before it returns).
+ *     freed before it returns) and the first gpuvm_gather_f32 on a handle (request
+ *     tables, kept by the handle).
  */
 #ifndef GPUVM_WORKLOADS_H
 #define GPUVM_WORKLOADS_H
@@ -39,10 +40,13 @@ int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void
  * x: fp32 array at x_off; d_idx: n_idx int64 element indices in device memory.
  * d_fsum, d_bsum: ceil(n_idx / block) elements.  block <= 2^20.
  *
- * gpuvm_gather_f32: one warp per block; the warp stages up to 1024 page ids in shared
- * memory and keeps all of them registered in the page table at once (gpuvm_batch.cuh),
- * so that one migrated page serves many waiting requests (Section 3.3: inter-warp
- * coalescing).  Uses 128 KiB of dynamic shared memory per thread block.
+ * gpuvm_gather_f32: a requester warp stages 2048 page requests at a time and keeps all
+ * of them registered in the page table at once (gpuvm_batch.cuh), so that one migrated
+ * page serves many waiting requests (Section 3.3: inter-warp coalescing); the faults
+ * go through a ring of page ids in shared memory to the thread block's migrator warps.
+ * The request tables (16 KiB per requester warp, 68 MiB for a full grid on 148 SMs) are
+ * device scratch owned by the handle: allocated at the first call, freed by
+ * gpuvm_destroy.
  * gpuvm_gather_f32_unbatched: one thread per index through gpuvm_read<float>, one
  * thread block per index block; at most 32 requests per warp are in flight.
  */

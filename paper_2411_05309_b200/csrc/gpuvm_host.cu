@@ -19,6 +19,8 @@ struct gpuvm_handle {
     int device;
     int last_cuda;
     unsigned long long *check_buf;   // device, 8 words
+    void *scratch;                   // device scratch for workload kernels (request tables)
+    size_t scratch_bytes;
 };
 
 namespace {
@@ -221,7 +223,7 @@ int gpuvm_destroy(gpuvm_t h)
     if (!h) return GPUVM_E_ARG;
     int rc = gpuvm_flush(h, nullptr);
     cudaFree(h->dev.pte); cudaFree(h->dev.frame_vpn); cudaFree(h->dev.ctl);
-    cudaFree(h->check_buf); cudaFree(h->dev.pool);
+    cudaFree(h->check_buf); cudaFree(h->dev.pool); cudaFree(h->scratch);
     if (h->host_registered) cudaHostUnregister(h->host_user);
     if (h->host_allocated) cudaFreeHost(h->host_user);
     cudaGetLastError();
@@ -265,6 +267,19 @@ int gpuvm_stats(gpuvm_t h, gpuvm_stats_t *out)
     out->error = (int32_t)(long long)local[kCtlErr];
     out->error_page = local[kCtlErrPage];
     return out->error;
+}
+
+void *gpuvm_scratch_(gpuvm_handle *h, size_t bytes)
+{
+    if (!h) return nullptr;
+    if (bytes <= h->scratch_bytes) return h->scratch;
+    cudaDeviceSynchronize();
+    cudaFree(h->scratch);
+    h->scratch = nullptr;
+    h->scratch_bytes = 0;
+    if (cudaMalloc(&h->scratch, bytes) != cudaSuccess) { h->last_cuda = (int)cudaGetLastError(); h->scratch = nullptr; return nullptr; }
+    h->scratch_bytes = bytes;
+    return h->scratch;
 }
 
 int gpuvm_device_view(gpuvm_t h, gpuvm_dev_t *out)

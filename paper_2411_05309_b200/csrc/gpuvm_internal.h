@@ -1,10 +1,17 @@
-// Shared by the translation units of libgpuvm: launch accounting only.
+// Shared by the translation units of libgpuvm: launch accounting and handle-owned scratch.
 #ifndef GPUVM_INTERNAL_H
 #define GPUVM_INTERNAL_H
+#include <stddef.h>
 #ifdef __cplusplus
 extern "C" {
 #endif
 void gpuvm_note_launch_(unsigned long long n);
+
+/* Device scratch owned by the handle: at least `bytes` long, 256-byte aligned, contents
+ * undefined.  Grown (never shrunk) on demand, freed by gpuvm_destroy.  NULL if the
+ * allocation fails.  Growing synchronises the device. */
+struct gpuvm_handle;
+void *gpuvm_scratch_(struct gpuvm_handle *h, size_t bytes);
 #ifdef __cplusplus
 }
 #endif

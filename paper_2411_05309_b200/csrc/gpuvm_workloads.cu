@@ -5,7 +5,6 @@
 
 #include <atomic>
 #include <cstdint>
-#include <cstdlib>
 
 #include "gpuvm.h"
 #include "gpuvm_batch.cuh"
@@ -124,25 +123,27 @@ __global__ void __launch_bounds__(1024) gather_kernel(Mem m, unsigned long long 
 }
 
 // A requester warp takes a run of consecutive indices (whole index blocks when they fit),
-// stages their page requests in its slice of shared memory, registers them all in the page
-// table, and as the pages arrive replaces each request by the value it asked for
-// (gpuvm_batch.cuh); then it adds the values up block by block.  The faults it owns go to
-// the thread block's ring of page ids, which the block's migrator warps serve.  No
-// block-wide barrier after start-up: warps never wait for one another.
-constexpr int kGatherRequesters = 24;
+// stages their page requests in its request table (handle-owned device scratch: it stays in
+// L2), registers them all in the page table, and as the pages arrive replaces each request by
+// the value it asked for (gpuvm_batch.cuh); then it adds the values up block by block.  The
+// faults it owns go to the thread block's ring of page ids in shared memory, which the
+// block's migrator warps serve.  No block-wide barrier after start-up: warps never wait for
+// one another.
+constexpr int kGatherRequesters = 28;
 constexpr int kGatherMigrators = 4;
 constexpr int kGatherMaxWarps = 32;
-constexpr unsigned int kGatherBatch = 1024;       // requests per requester warp
+constexpr unsigned int kGatherBatch = GPUVM_BATCH_MAX;   // requests per requester warp
 
 __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(gpuvm_dev_t vm, unsigned long long x_off,
                                                                             const long long *__restrict__ idx,
                                                                             unsigned long long n_idx, unsigned long long block,
                                                                             float *__restrict__ fsum, long long *__restrict__ bsum,
-                                                                            int requesters, unsigned int batch)
+                                                                            int requesters, unsigned int batch,
+                                                                            gpuvm_batch_entry *g_tables)
 {
     extern __shared__ __align__(16) unsigned char s_raw[];
     gpuvm_fault_queue *queue = reinterpret_cast<gpuvm_fault_queue *>(s_raw);
-    gpuvm_batch_entry *tables = reinterpret_cast<gpuvm_batch_entry *>(s_raw + sizeof(gpuvm_fault_queue));
+    gpuvm_batch_entry *tables = g_tables + (size_t)blockIdx.x * requesters * batch;
     const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
         reinterpret_cast<unsigned int *>(queue)[k] = 0;
@@ -652,29 +653,19 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     if (!d_idx || !d_fsum || !d_bsum || block == 0 || block > (size_t(1) << 20)) return GPUVM_E_ARG;
     if (x_off % 16) return GPUVM_E_ALIGN;
     if (n_idx == 0) return GPUVM_OK;
-    static bool configured = false;
-    int requesters = getenv("GPUVM_TUNE_REQUESTERS") ? atoi(getenv("GPUVM_TUNE_REQUESTERS")) : kGatherRequesters;
-    int migrators = getenv("GPUVM_TUNE_MIGRATORS") ? atoi(getenv("GPUVM_TUNE_MIGRATORS")) : kGatherMigrators;
-    unsigned int batch = getenv("GPUVM_TUNE_BATCH") ? (unsigned int)atoi(getenv("GPUVM_TUNE_BATCH")) : kGatherBatch;
-    if (requesters < 1 || migrators < 1 || requesters + migrators > kGatherMaxWarps) return GPUVM_E_ARG;
-    if (batch < 32 || batch > GPUVM_BATCH_MAX || batch % 32) return GPUVM_E_ARG;
-    const size_t smem = sizeof(gpuvm_fault_queue) + (size_t)requesters * batch * sizeof(gpuvm_batch_entry);
-    if (smem > 227 * 1024) return GPUVM_E_ARG;
-    if (!configured) {
-        if (cudaFuncSetAttribute(gather_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
-            cudaGetLastError();
-            return GPUVM_E_CUDA;
-        }
-        configured = true;
-    }
+    const int requesters = kGatherRequesters, migrators = kGatherMigrators;
+    const unsigned int batch = kGatherBatch;
     const size_t nb = (n_idx + block - 1) / block;
     const size_t per = block <= batch ? batch / block : 1;
     const size_t items = (nb + per - 1) / per;
     const size_t blocks_needed = (items + requesters - 1) / requesters;
     const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
-    gather_batch_kernel<<<grid, (requesters + migrators) * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+    gpuvm_batch_entry *tables = static_cast<gpuvm_batch_entry *>(
+        gpuvm_scratch_(h, (size_t)grid * requesters * batch * sizeof(gpuvm_batch_entry)));
+    if (!tables) return GPUVM_E_ALLOC;
+    gather_batch_kernel<<<grid, (requesters + migrators) * 32, sizeof(gpuvm_fault_queue), static_cast<cudaStream_t>(stream)>>>(
         m.vm, x_off, reinterpret_cast<const long long *>(d_idx), n_idx, block, d_fsum, reinterpret_cast<long long *>(d_bsum),
-        requesters, batch);
+        requesters, batch, tables);
     return launched();
 }
 
