@@ -65,6 +65,8 @@ class Workload:
             self.off[name] = total
             total += _pad(nbytes, self.page_bytes)
         self.nbytes = total
+        if getattr(self, "pool_override", None):
+            pool_bytes = self.pool_override
         if callable(pool_bytes):
             pool_bytes = pool_bytes(total)
         self.pool_bytes = max(self.page_bytes, pool_bytes // self.page_bytes * self.page_bytes)

@@ -1,0 +1,102 @@
+"""Parameter sweeps of the paged path (the paper's transfer benchmark and its
+oversubscription analysis), printed as JSON lines.
+
+    python -m paper_2411_05309_b200.sweeps pages   [--gib 4] [--warps-per-sm 16]
+    python -m paper_2411_05309_b200.sweeps oversub [--workload 1|2|3|4] [--shrink S]
+
+pages   -- Section 5.1 / Fig. 7: move a fixed amount of host memory into the pool with one
+           warp per page, consecutive pages, for page sizes from 4 KiB to 2 MiB; reports the
+           migration bandwidth against the pinned-copy peak measured in the same run.
+oversub -- Section 5.4 / Fig. 14 with Eq. 1: run a workload with the pool shrunk step by step,
+           level = paged bytes / pool bytes - 1, under the clock policy and under FIFO (the
+           paper's ring), reporting time relative to level 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+
+
+def _time(torch, fn):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    fn()
+    e1.record()
+    e1.synchronize()
+    return e0.elapsed_time(e1) / 1e3
+
+
+def sweep_pages(gib: float, warps_per_sm: int):
+    import torch
+    from . import binding as B
+    nbytes = int(gib * (1 << 30))
+    host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    devb = torch.empty(min(nbytes, 1 << 30), dtype=torch.uint8, device="cuda")
+    best = 0.0
+    for r in range(4):
+        t = _time(torch, lambda: devb.copy_(host[:devb.numel()], non_blocking=True))
+        if r:
+            best = max(best, devb.numel() / t / 1e9)
+    del devb
+    torch.cuda.empty_cache()
+    for shift in range(12, 22):
+        page = 1 << shift
+        h = B.gpuvm_create(host.data_ptr(), nbytes, page, nbytes)          # pool holds everything: no eviction
+        try:
+            times = []
+            for r in range(3):
+                B.gpuvm_reset(h)
+                times.append(_time(torch, lambda: B.gpuvm_touch_pages(h, 0, nbytes // page, warps_per_sm)))
+            st = B.gpuvm_stats(h)
+            assert st["faults"] == nbytes // page and B.gpuvm_check(h)["resident"] == nbytes // page
+            t = min(times[1:])
+            print(json.dumps({"sweep": "pages", "page_bytes": page, "bytes": nbytes, "warps_per_sm": warps_per_sm,
+                              "seconds": t, "migration_gbs": nbytes / t / 1e9, "faults_per_s": nbytes / page / t,
+                              "pinned_copy_gbs": best, "frac_of_pinned_copy": nbytes / t / 1e9 / best}), flush=True)
+        finally:
+            B.gpuvm_destroy(h)
+
+
+def sweep_oversub(cfg: int, shrink: int):
+    from . import binding as B
+    from . import configs
+    levels = [0, 0.5, 1, 2, 3, 5, 7, 11]
+    base = {}
+    for policy, pname in ((B.POLICY_CLOCK, "clock"), (B.POLICY_FIFO, "fifo")):
+        for level in levels:
+            w = configs.WORKLOADS[cfg](shrink)
+            w.pool_override = lambda total, level=level: int(total / (level + 1))
+            w.setup()
+            try:
+                B.gpuvm_set_policy(w.h, policy)
+                w.run(check=False)
+                res = w.run()
+                if level == 0:
+                    base[pname] = res.seconds
+                print(json.dumps({"sweep": "oversub", "workload": w.name, "policy": pname, "level": level,
+                                  "level_actual": w.nbytes / w.pool_bytes - 1, "pool_bytes": w.pool_bytes,
+                                  "seconds": res.seconds, "slowdown_vs_level0": res.seconds / base[pname],
+                                  "faults": res.stats["faults"], "bytes_in": res.stats["bytes_in"],
+                                  "bytes_out": res.stats["bytes_out"],
+                                  "io_amplification": res.stats["bytes_in"] / max(1, res.effective_bytes)}), flush=True)
+            finally:
+                w.close()
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("which", choices=["pages", "oversub"])
+    ap.add_argument("--gib", type=float, default=4.0)
+    ap.add_argument("--warps-per-sm", type=int, default=16)
+    ap.add_argument("--workload", type=int, default=1)
+    ap.add_argument("--shrink", type=int, default=0)
+    a = ap.parse_args(argv)
+    if a.which == "pages":
+        sweep_pages(a.gib, a.warps_per_sm)
+    else:
+        sweep_oversub(a.workload, a.shrink)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
