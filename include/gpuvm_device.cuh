@@ -9,6 +9,7 @@
  *   void  gpuvm_write<T>(vm, elem_index, value, base_byte_off) pin, mark dirty, store, unpin
  *   void* gpuvm_ptr(vm, byte_off, mode, &token)                pin and hand out a frame pointer
  *   void  gpuvm_release(vm, token)                             unpin what gpuvm_ptr pinned
+ *   void  gpuvm_clean(vm, token, p)                            write a pinned page back now (eager write-back)
  *
  * What happens on an access (Section 3.1, Fig. 2; Section 3.3):
  *   1. address split: page number = byte offset >> page_shift, offset = the rest;
@@ -92,7 +93,7 @@ constexpr int kCtlWords = kCtlCounters + kStatSlots * 16;
 enum Stat { kFaults = 0, kHits, kWaits, kLanes, kEvictions, kWritebacks, kFlushWritebacks,
             kBytesIn, kBytesOut, kHandSteps, kRetries, kNumStats };
 
-enum Mode { kRead = 0, kWrite = 1 };
+enum Mode { kRead = 0, kWrite = 1, kWriteAll = 2 };
 
 struct Token {
     unsigned long long vpn;
@@ -248,7 +249,7 @@ __device__ __forceinline__ int advance(const gpuvm_dev_t &vm, unsigned long long
     for (;;) {
         unsigned long long st = w & kStMask;
         if (st == kValid) {
-            unsigned long long want = (mode == kWrite ? kDirty : 0ull) |
+            unsigned long long want = (mode != kRead ? kDirty : 0ull) |
                                       (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull);
             if ((w & want) != want) atomicOr(pte, want);
             frame = (unsigned int)((w & kFrameMask) >> kFrameShift);
@@ -387,6 +388,7 @@ static __device__ __noinline__ bool slow_path(const gpuvm_dev_t vm, unsigned lon
             const unsigned long long bq = __shfl_sync(active, victim, L);
             const int bd = __shfl_sync(active, (int)vdirty, L);
             const unsigned long long bv = __shfl_sync(active, vpn, L);
+            const int bmode = __shfl_sync(active, mode, L);
             unsigned char *fr = vm.pool + ((unsigned long long)bh << vm.page_shift);
             if (bq != ~0ull) {
                 if (bd) {
@@ -401,17 +403,19 @@ static __device__ __noinline__ bool slow_path(const gpuvm_dev_t vm, unsigned lon
                     if (bd) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, bq)); }
                 }
             }
-            warp_copy<8, false>(fr, vm.host + (bv << vm.page_shift), page_len(vm, bv) >> 4, rank, nlanes);
-            __threadfence();
+            if (bmode != kWriteAll) {                        /* a page that will be overwritten entirely is not fetched */
+                warp_copy<8, false>(fr, vm.host + (bv << vm.page_shift), page_len(vm, bv) >> 4, rank, nlanes);
+                __threadfence();
+            }
             __syncwarp(active);
             if ((int)lane == L) {
                 st_relaxed_u32(vm.frame_vpn + bh, (unsigned int)bv);
                 unsigned long long bits = (kBusy ^ kValid) | ((unsigned long long)bh << kFrameShift) |
                                           (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull) |
-                                          (mode == kWrite ? kDirty : 0ull);
+                                          (mode != kRead ? kDirty : 0ull);
                 atomicXor(pte, bits);                        /* step 7: publish */
                 stat_add(vm, kFaults, 1);
-                stat_add(vm, kBytesIn, page_len(vm, bv));
+                if (mode != kWriteAll) stat_add(vm, kBytesIn, page_len(vm, bv));
                 st = kReady; frame = bh;
             }
         }
@@ -467,7 +471,7 @@ __device__ __forceinline__ bool access(const gpuvm_dev_t &vm, unsigned long long
     const bool hit = (w & kStMask) == kValid;
     if (__all_sync(active, hit)) {
         if (is_leader) {
-            unsigned long long want = (mode == kWrite ? kDirty : 0ull) |
+            unsigned long long want = (mode != kRead ? kDirty : 0ull) |
                                       (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull);
             if ((w & want) != want) atomicOr(pte, want);
             if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1);
@@ -511,7 +515,7 @@ __device__ __forceinline__ bool access(const gpuvm_dev_t &vm, unsigned long long
 /* ------------------------------------------------------------------ public API */
 
 typedef gpuvm::Token gpuvm_token;
-enum { GPUVM_READ = gpuvm::kRead, GPUVM_WRITE = gpuvm::kWrite };
+enum { GPUVM_READ = gpuvm::kRead, GPUVM_WRITE = gpuvm::kWrite, GPUVM_WRITE_ALL = gpuvm::kWriteAll };
 
 /* Element `elem` of an array of T that starts `base_off` bytes into the backing
  * store (Listing 1: A[i] on the right-hand side). */
@@ -542,7 +546,12 @@ __device__ __forceinline__ void gpuvm_write(const gpuvm_dev_t &vm, unsigned long
 
 /* Pin the page that holds `byte_off` and return the address of that byte inside
  * its frame, valid up to the end of the page until gpuvm_release(token).
- * mode GPUVM_WRITE marks the page dirty.  nullptr after an error. */
+ * mode GPUVM_WRITE marks the page dirty.  GPUVM_WRITE_ALL is a promise that the caller
+ * overwrites every byte of the page that lies inside the backing store before it releases
+ * the page: a missing page is then given a frame without being fetched from the host (its
+ * old contents would be overwritten anyway).  The page must stay pinned from this call to
+ * gpuvm_release for the whole overwrite; whoever reads it meanwhile sees unspecified bytes.
+ * nullptr after an error. */
 __device__ __forceinline__ void *gpuvm_ptr(const gpuvm_dev_t &vm, unsigned long long byte_off, int mode,
                                            gpuvm_token *token)
 {
@@ -559,6 +568,37 @@ __device__ __forceinline__ void gpuvm_release(const gpuvm_dev_t &vm, const gpuvm
     if (token.group == 0) return;
     __syncwarp(token.group);
     if (token.leader) gpuvm::unpin(vm.pte + token.vpn);
+}
+
+/*
+ * Eager write-back: copy the page pinned by `token` to the host now and mark it clean, so
+ * that its later eviction costs nothing and no fault has to wait for a write-back (the
+ * paper names synchronous write-back on the fault path as its weak spot, Section 5.3).
+ * Called by the lanes that pinned the page together (token.group), converged, before
+ * gpuvm_release; `p` is any address inside the page's frame.  The dirty bit is cleared
+ * before the copy starts: a store that lands during or after the copy sets it again and
+ * the page is written back once more later, so nothing is lost.
+ */
+__device__ __forceinline__ void gpuvm_clean(const gpuvm_dev_t &vm, const gpuvm_token &token, const void *p)
+{
+    if (token.group == 0 || p == nullptr) return;
+    const unsigned int lane = gpuvm::lane_id();
+    const unsigned int rank = __popc(token.group & ((1u << lane) - 1u)), n = __popc(token.group);
+    unsigned long long *pte = vm.pte + token.vpn;
+    __syncwarp(token.group);                                   /* the group's stores to the frame are done */
+    bool dirty = false;
+    if (token.leader) dirty = (atomicAnd(pte, ~gpuvm::kDirty) & gpuvm::kDirty) != 0ull;
+    dirty = __shfl_sync(token.group, (int)dirty, __ffs(token.group) - 1);
+    if (!dirty) return;
+    const unsigned long long frame = (unsigned long long)(static_cast<const unsigned char *>(p) - vm.pool) >> vm.page_shift;
+    const unsigned int len = gpuvm::page_len(vm, token.vpn);
+    gpuvm::warp_copy<8, true>(vm.host + (token.vpn << vm.page_shift), vm.pool + (frame << vm.page_shift), len >> 4, rank, n);
+    __threadfence_system();
+    __syncwarp(token.group);
+    if (token.leader) {
+        gpuvm::stat_add(vm, gpuvm::kWritebacks, 1);
+        gpuvm::stat_add(vm, gpuvm::kBytesOut, len);
+    }
 }
 
 /* Frame memory accessors (L1-bypassing, device-coherent). */

@@ -109,7 +109,12 @@ int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, 
  * Vector add c[i] = a[i] + b[i] over three paged fp32 arrays of n elements
  * (Listing 1).  c is written through the runtime: its pages become dirty and reach
  * the host by eviction write-back or gpuvm_flush.  One IEEE binary32 addition per
- * element, no fused operations.
+ * element, no fused operations.  A warp processes one page of the element range at a
+ * time.  When the pool has at least two frames for every warp of the grid and c starts
+ * on a page boundary, the page of c is kept pinned while its chunks are produced and,
+ * being overwritten entirely, is not fetched from the host first (GPUVM_WRITE_ALL);
+ * otherwise every chunk pins a, b and c one after the other and c is fetched like any
+ * page that is written to.
  */
 int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n, void *stream);
 

@@ -28,6 +28,7 @@ struct Paged {
         return static_cast<unsigned char *>(gpuvm_ptr(vm, off, mode, &t));
     }
     __device__ __forceinline__ void release(const gpuvm_token &t) const { gpuvm_release(vm, t); }
+    __device__ __forceinline__ void clean(const gpuvm_token &t, const void *p) const { gpuvm_clean(vm, t, p); }
     static __device__ __forceinline__ uint4 load16(const void *p) { return gpuvm_load16(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { gpuvm_store16(p, v); }
     static __device__ __forceinline__ int load_i32(const void *p) { return gpuvm_load(static_cast<const int *>(p)); }
@@ -43,6 +44,7 @@ struct Raw {
     __device__ __forceinline__ void write(unsigned long long off, unsigned long long i, T v) const { reinterpret_cast<T *>(base + off)[i] = v; }
     __device__ __forceinline__ unsigned char *pin(unsigned long long off, int, gpuvm_token &) const { return base + off; }
     __device__ __forceinline__ void release(const gpuvm_token &) const {}
+    __device__ __forceinline__ void clean(const gpuvm_token &, const void *) const {}
     static __device__ __forceinline__ uint4 load16(const void *p) { return *static_cast<const uint4 *>(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { *static_cast<uint4 *>(p) = v; }
     static __device__ __forceinline__ int load_i32(const void *p) { return *static_cast<const int *>(p); }
@@ -343,9 +345,16 @@ __global__ void __launch_bounds__(256) bfs_span_kernel(Mem m, unsigned long long
 __global__ void bfs_init_kernel(int *level, int source) { level[source] = 0; }
 
 // ----------------------------------------------------------------- vector add
-// A warp owns one unit (page) of the element range and walks it in chunks of at most
-// 4 KiB; for each chunk it holds exactly one page at a time: a, then b, then c.
-template <class Mem>
+// A warp owns one unit (page) of the element range and walks it in chunks of at most 4 KiB.
+// HOLD_C = false: it holds exactly one page at a time (a, then b, then c, per chunk), which
+// cannot deadlock whatever the pool size.  HOLD_C = true (chosen by the host when the pool has
+// at least two frames per warp of the grid and c starts on a page boundary): the page of c
+// stays pinned for the whole unit and, when the unit covers the whole page, is requested with
+// GPUVM_WRITE_ALL, so it is not fetched from the host before being overwritten; when the
+// unit is finished the warp writes the page back at once (gpuvm_clean), which keeps
+// write-backs off the fault path and uses the outbound half of the link while the inbound
+// half carries a and b.
+template <class Mem, bool HOLD_C>
 __global__ void __launch_bounds__(256) vadd_kernel(Mem m, unsigned long long a_off, unsigned long long b_off,
                                                    unsigned long long c_off, unsigned long long n,
                                                    unsigned int chunk_bytes)
@@ -355,13 +364,19 @@ __global__ void __launch_bounds__(256) vadd_kernel(Mem m, unsigned long long a_o
     const unsigned long long total = 4ull * n, units = (total + unit - 1) / unit;
     for (unsigned long long u = warp_in_grid(); u < units; u += warps_in_grid()) {
         unsigned long long lo = u * unit, hi = lo + unit < total ? lo + unit : total;
+        gpuvm_token tok_c;
+        unsigned char *page_c = nullptr;
+        if (HOLD_C) {
+            page_c = m.pin(c_off + lo, hi - lo == unit ? GPUVM_WRITE_ALL : GPUVM_WRITE, tok_c);
+            if (!page_c) return;
+        }
         for (unsigned long long off = lo; off < hi; off += chunk_bytes) {
             const unsigned int len = (unsigned int)(hi - off < chunk_bytes ? hi - off : chunk_bytes);
             const unsigned int n16 = len >> 4;
             uint4 va[8], vb[8];
             gpuvm_token tok;
             const unsigned char *pa = m.pin(a_off + off, GPUVM_READ, tok);
-            if (!pa) return;
+            if (!pa) break;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 unsigned int i = lane + 32u * j;
@@ -369,15 +384,15 @@ __global__ void __launch_bounds__(256) vadd_kernel(Mem m, unsigned long long a_o
             }
             m.release(tok);
             const unsigned char *pb = m.pin(b_off + off, GPUVM_READ, tok);
-            if (!pb) return;
+            if (!pb) break;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 unsigned int i = lane + 32u * j;
                 if (i < n16) vb[j] = Mem::load16(pb + 16ull * i);
             }
             m.release(tok);
-            unsigned char *pc = m.pin(c_off + off, GPUVM_WRITE, tok);
-            if (!pc) return;
+            unsigned char *pc = HOLD_C ? page_c + (off - lo) : m.pin(c_off + off, GPUVM_WRITE, tok);
+            if (!pc) break;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 unsigned int i = lane + 32u * j;
@@ -390,7 +405,11 @@ __global__ void __launch_bounds__(256) vadd_kernel(Mem m, unsigned long long a_o
                     Mem::store16(pc + 16ull * i, r);
                 }
             }
-            m.release(tok);
+            if (!HOLD_C) m.release(tok);
+        }
+        if (HOLD_C) {
+            m.clean(tok_c, page_c);          // the finished page goes to the host at once: evicting it later is free
+            m.release(tok_c);
         }
     }
 }
@@ -533,6 +552,7 @@ int run_gather(const Mem &m, size_t x_off, const int64_t *d_idx, size_t n_idx, s
     return launched();
 }
 
+constexpr int kVaddBlocksPerSm = 4;
 constexpr size_t kBfsScratchBytes = 2 * kBigQueue * sizeof(long long) + 4 * sizeof(unsigned int);
 
 // One BFS on caller-provided scratch (kBfsScratchBytes, 16-byte aligned).
@@ -578,7 +598,7 @@ int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t sour
 }
 
 template <class Mem>
-int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, cudaStream_t s)
+int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, bool hold_c, cudaStream_t s)
 {
     unsigned long long unit = 0;
     if (n % 4) return GPUVM_E_ALIGN;
@@ -587,7 +607,10 @@ int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, c
     unsigned int chunk = unit < 4096 ? (unsigned int)unit : 4096u;
     if (chunk < 512) return GPUVM_E_PAGE;             // a warp moves 512 bytes per instruction
     if (a_off % chunk || b_off % chunk || c_off % chunk) return GPUVM_E_ALIGN;
-    vadd_kernel<Mem><<<sm_count() * 4, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
+    if (hold_c && c_off % unit == 0)
+        vadd_kernel<Mem, true><<<sm_count() * kVaddBlocksPerSm, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
+    else
+        vadd_kernel<Mem, false><<<sm_count() * kVaddBlocksPerSm, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
     return launched();
 }
 
@@ -705,7 +728,9 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
 {
     PagedH m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
-    return run_vadd(m, a_off, b_off, c_off, n, static_cast<cudaStream_t>(stream));
+    // two pages per warp are held at once on the no-fetch path: only when the pool can take it
+    const bool hold_c = gpuvm_safe_warps(h, 2) >= sm_count() * kVaddBlocksPerSm * 8;
+    return run_vadd(m, a_off, b_off, c_off, n, hold_c, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
@@ -777,7 +802,7 @@ int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void 
     RawH m;
     m.base = base;
     m.unit_bytes = 65536;
-    return run_vadd(m, (size_t)(pa - base), (size_t)(pb - base), (size_t)(pc - base), n, static_cast<cudaStream_t>(stream));
+    return run_vadd(m, (size_t)(pa - base), (size_t)(pb - base), (size_t)(pc - base), n, false, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_raw_embag_f32(const float *table, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,

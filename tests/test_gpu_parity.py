@@ -119,6 +119,34 @@ def test_vadd_writes_back_every_dirty_page(B, page, n, frames, policy):
         assert st["faults"] == ar.n_pages and st["writebacks"] == 0 and st["flush_writebacks"] == c_pages
 
 
+@pytest.mark.parametrize("page,n,frames", [
+    (512, 1 << 20, 10000),         # 24576 pages through 10000 frames
+    (4096, (1 << 22) + 4096 + 512, 9600),   # last page of c is partial: fetched, not WRITE_ALL
+    (512, 1 << 18, 20000),         # everything fits
+])
+def test_vadd_no_fetch_path_with_eager_write_back(B, page, n, frames):
+    """With at least two frames per warp of the grid the kernel keeps the page of c pinned,
+    does not fetch it (it is overwritten entirely) and writes it back as soon as it is done."""
+    import torch
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert frames >= 2 * sms * 4 * 8
+    a = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4))
+    b = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4, 1))
+    ar = Arena(page, {"a": a, "b": b, "c": np.full(n, 7.0, np.float32)})
+    with paged(ar.host, page, frames) as h:
+        B.gpuvm_vadd_f32(h, ar.off["a"], ar.off["b"], ar.off["c"], n)
+        st, ck = finish(h)
+    assert np.array_equal(ar.views["c"].view(np.uint32), oracle.vadd_f32_direct(a, b).view(np.uint32))
+    assert np.array_equal(ar.views["a"], a) and np.array_equal(ar.views["b"], b)
+    c_pages = (4 * n + page - 1) // page
+    full_c_pages = (4 * n) // page
+    assert st["writebacks"] == c_pages and st["flush_writebacks"] == 0       # every page of c left eagerly
+    fetched_pages = st["bytes_in"] // page if 4 * n % page == 0 else None
+    if fetched_pages is not None:
+        assert fetched_pages == 2 * c_pages                                   # a and b only: c was not fetched
+    assert st["faults"] >= 3 * full_c_pages
+
+
 def small_graphs():
     rng = np.random.default_rng(24)
     yield 1, [], 0
