@@ -244,13 +244,16 @@ __global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long lon
 {
     const unsigned int lane = threadIdx.x & 31;
     const unsigned long long unit = m.unit();
+    const unsigned int n_chunks = (nv + 31) / 32;
     unsigned int found = 0;
     for (;;) {
         unsigned int chunk = 0;
         if (lane == 0) chunk = atomicAdd(counters + 2, 1u);
         chunk = __shfl_sync(0xFFFFFFFFu, chunk, 0);
-        const unsigned long long v0 = 32ull * chunk;
-        if (v0 >= nv) break;
+        if (chunk >= n_chunks) break;
+        // odd levels sweep downwards: the pages a sweep used last are still resident when the
+        // next sweep starts with them (a one-directional cyclic sweep defeats any LRU-like policy)
+        const unsigned long long v0 = 32ull * ((depth & 1) ? n_chunks - 1 - chunk : chunk);
         const unsigned long long v = v0 + lane;
         const bool active = v < nv && level[v] == depth;
         if (!__any_sync(0xFFFFFFFFu, active)) continue;
