@@ -33,7 +33,10 @@
  *     gpuvm_batch_access(vm, table, n, GPUVM_READ or GPUVM_WRITE, consume, queue);
  * `consume(i, p)` is called exactly once per served request, by lane i % 32, with p
  * pointing at the requested byte inside its frame (use gpuvm_load / gpuvm_store on it);
- * it may overwrite table[i] (for instance with the value it read).  Requests that fail
+ * it may overwrite table[i] (for instance with the value it read).  With WARP_CONSUME the
+ * call is made by all 32 lanes together, one served request after the other, with the same
+ * i and p in every lane: the shape for requests whose payload is a row that the warp reads
+ * with coalesced 16-byte loads.  gpuvm_batch_skip(table, i) marks slot i as unused.  Requests that fail
  * (offset out of range, wait ran out) are not consumed; the sticky error is set as for the
  * other accessors.  Returns the number of requests served for the calling lane.
  * Pages must not be larger than 128 MiB (the in-page offset shares a word with the
@@ -198,7 +201,13 @@ __device__ __forceinline__ void gpuvm_batch_set(const gpuvm_dev_t &vm, gpuvm_bat
     table[i] = e;
 }
 
-template <class Consume>
+__device__ __forceinline__ void gpuvm_batch_skip(gpuvm_batch_entry *table, unsigned int i)
+{
+    table[i].vpn = gpuvm::kRejected;
+    table[i].offl = 0;
+}
+
+template <bool WARP_CONSUME = false, class Consume>
 static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t vm, gpuvm_batch_entry *table,
                                                                unsigned int n, int mode, Consume consume,
                                                                gpuvm_fault_queue *queue = nullptr)
@@ -246,13 +255,16 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
             const unsigned int rowmask = __ballot_sync(0xFFFFFFFFu, mine);
             if (!rowmask) continue;
             any_rows = true;
+            unsigned int frame = kNotReady, off = 0;
+            unsigned long long *pte = nullptr;
+            bool is_leader = false;
+            const unsigned int i = j * 32 + lane;
             if (mine) {
-                const unsigned int i = j * 32 + lane;
                 const gpuvm_batch_entry e = table[i];
                 const unsigned int leader = e.offl >> 27;
-                unsigned long long *pte = vm.pte + e.vpn;
-                unsigned int frame = kNotReady;
-                const bool is_leader = (lead >> j) & 1ull;
+                off = e.offl & kOffMask;
+                pte = vm.pte + e.vpn;
+                is_leader = (lead >> j) & 1ull;
                 if (is_leader) {
                     if ((failed >> j) & 1ull) {
                         frame = kFailed;
@@ -264,17 +276,31 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
                     }
                 }
                 frame = __shfl_sync(rowmask, frame, leader);
-                if (frame == kFailed) {
-                    todo &= ~(1ull << j);
-                } else if (frame != kNotReady) {
-                    __threadfence();
-                    consume(i, vm.pool + ((unsigned long long)frame << vm.page_shift) + (e.offl & kOffMask));
-                    todo &= ~(1ull << j);
-                    ++served;
-                    progress = true;
+                if (frame == kFailed) todo &= ~(1ull << j);
+            }
+            const bool ready = mine && frame < kFailed;
+            if (WARP_CONSUME) {
+                unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
+                if (ready_lanes) __threadfence();
+                while (ready_lanes) {
+                    const unsigned int L = __ffs(ready_lanes) - 1;
+                    ready_lanes &= ready_lanes - 1;
+                    const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame, L), o = __shfl_sync(0xFFFFFFFFu, off, L);
+                    consume(j * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o);
                 }
-                __syncwarp(rowmask);                            /* the whole group has used the frame */
-                if (is_leader && frame < kFailed) unpin(pte);   /* step 8 */
+                __syncwarp();                                   /* every group has used its frame */
+            } else {
+                if (ready) {
+                    __threadfence();
+                    consume(i, vm.pool + ((unsigned long long)frame << vm.page_shift) + off);
+                }
+                if (mine) __syncwarp(rowmask);                  /* the whole group has used the frame */
+            }
+            if (ready) {
+                todo &= ~(1ull << j);
+                ++served;
+                progress = true;
+                if (is_leader) unpin(pte);                      /* step 8 */
             }
         }
         if (!any_rows) break;

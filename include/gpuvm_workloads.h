@@ -13,8 +13,8 @@
  *     errors (a wait that ran out, an offset out of range) are sticky in the handle
  *     and show up in gpuvm_stats().  Return value: 0 or a negative gpuvm_status.
  *   - nothing here allocates device memory except gpuvm_bfs_csr (1 MiB of scratch,
- *     freed before it returns) and the first gpuvm_gather_f32 on a handle (request
- *     tables, kept by the handle).
+ *     freed before it returns) and the first gpuvm_gather_f32 / gpuvm_embag_f32 on
+ *     a handle (request tables and row staging, kept by the handle).
  */
 #ifndef GPUVM_WORKLOADS_H
 #define GPUVM_WORKLOADS_H
@@ -121,11 +121,22 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
 /*
  * Embedding-bag gather: d_out[g][d] = sum over the `bag` rows of bag g of
  * table[row][d], added in list order in fp32.  table: fp32 [rows][dims] at t_off,
- * dims a multiple of 4 with dims/4 <= 32 lanes (one warp per bag, a lane owns 4
- * consecutive dims); d_rows: n_bags * bag int64 row ids; d_out: n_bags * dims fp32.
+ * dims a multiple of 4 with dims/4 <= 32 lanes (a lane owns 4 consecutive dims);
+ * d_rows: n_bags * bag int64 row ids; d_out: n_bags * dims fp32.
+ *
+ * gpuvm_embag_f32: a requester warp registers the rows of 32 bags (up to 32 lookups
+ * each, 1024 page requests) at once (gpuvm_batch.cuh); rows that arrive are staged in
+ * device scratch and added per bag in list order once the batch is complete, so the
+ * result has the bits of a sequential fp32 sum.  Scratch owned by the handle: 8 KiB +
+ * 1024 rows per requester warp (2.1 GiB for dims = 128 on a full grid of 148 SMs),
+ * allocated at the first call, freed by gpuvm_destroy.  Pages up to 128 MiB.
+ * gpuvm_embag_f32_unbatched: one warp per bag, one row request at a time through
+ * gpuvm_read; no scratch.
  */
 int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags,
                     size_t bag, float *d_out, void *stream);
+int gpuvm_embag_f32_unbatched(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags,
+                              size_t bag, float *d_out, void *stream);
 
 /*
  * Read-modify-write through the element accessors: for every k < n,

@@ -75,6 +75,7 @@ SYMBOLS = {
     "gpuvm_bfs_csr_noalloc": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_vadd_f32": (_i, [_vp, _sz, _sz, _sz, _sz, _vp]),
     "gpuvm_embag_f32": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
+    "gpuvm_embag_f32_unbatched": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_scatter_update_u32": (_i, [_vp, _sz, _vp, _sz, _vp]),
     "gpuvm_touch_pages": (_i, [_vp, _sz, _sz, _i, _vp]),
     "gpuvm_raw_stream_sum_i32": (_i, [_vp, _sz, _vp, _vp]),
@@ -260,6 +261,11 @@ def gpuvm_vadd_f32(h, a_off: int, b_off: int, c_off: int, n: int, stream=None):
 def gpuvm_embag_f32(h, t_off: int, dims: int, d_rows, n_bags: int, bag: int, d_out, stream=None):
     _check(lib().gpuvm_embag_f32(h, t_off, dims, _ptr(d_rows), n_bags, bag, _ptr(d_out), _stream(stream)),
            "gpuvm_embag_f32")
+
+
+def gpuvm_embag_f32_unbatched(h, t_off: int, dims: int, d_rows, n_bags: int, bag: int, d_out, stream=None):
+    _check(lib().gpuvm_embag_f32_unbatched(h, t_off, dims, _ptr(d_rows), n_bags, bag, _ptr(d_out), _stream(stream)),
+           "gpuvm_embag_f32_unbatched")
 
 
 def gpuvm_scatter_update_u32(h, a_off: int, d_idx, n: int, stream=None):

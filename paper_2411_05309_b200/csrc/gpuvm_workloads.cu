@@ -441,6 +441,80 @@ __global__ void __launch_bounds__(256) embag_kernel(Mem m, unsigned long long t_
     }
 }
 
+// Batched embedding bag.  A requester warp takes 32 bags at a time (bag b of the item belongs
+// to lane b) and up to 32 lookups of each: 1024 row requests registered in the page table at
+// once.  Rows arrive in any order, so each served row is first copied, by the whole warp with
+// coalesced 16-byte accesses, into the warp's staging area (device scratch); when the batch
+// is complete the rows of each bag are added up in list order, which keeps the fp32 result
+// bit-identical to a sequential sum.  Faults go to the block's migrator warps.
+constexpr int kEmbagRequesters = 28;
+constexpr int kEmbagMigrators = 4;
+constexpr unsigned int kEmbagLookups = 32;                 // lookups of a bag per batch (table rows)
+
+__global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
+                                                              const long long *__restrict__ rows, unsigned long long n_bags,
+                                                              unsigned int bag, float *__restrict__ out, int requesters,
+                                                              gpuvm_batch_entry *g_tables, unsigned char *g_staging)
+{
+    __shared__ gpuvm_fault_queue queue_s;
+    gpuvm_fault_queue *queue = &queue_s;
+    const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
+        reinterpret_cast<unsigned int *>(queue)[k] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) queue->requesters = (unsigned int)requesters;
+    __syncthreads();
+    if ((int)warp >= requesters) {
+        gpuvm_migrator_loop(vm, queue);
+        return;
+    }
+    const unsigned int q = dims >> 2;                            // 16-byte pieces per row
+    const unsigned long long row_bytes = 4ull * dims;
+    const size_t slot = (size_t)blockIdx.x * requesters + warp;
+    gpuvm_batch_entry *table = g_tables + slot * (32 * kEmbagLookups);
+    uint4 *staging = reinterpret_cast<uint4 *>(g_staging + slot * (32 * kEmbagLookups) * row_bytes);
+    const unsigned long long items = (n_bags + 31) / 32;
+    const unsigned long long stride = (unsigned long long)gridDim.x * requesters;
+    for (unsigned long long t = slot; t < items; t += stride) {
+        const unsigned long long g0 = 32 * t;
+        for (unsigned int k0 = 0; k0 < bag; k0 += kEmbagLookups) {
+            const unsigned int nk = bag - k0 < kEmbagLookups ? bag - k0 : kEmbagLookups;
+            // request (k, b): lookup k0 + k of bag g0 + b
+            for (unsigned int k = 0; k < nk; ++k) {
+                const unsigned long long g = g0 + lane;
+                if (g < n_bags)
+                    gpuvm_batch_set(vm, table, k * 32 + lane,
+                                    t_off + (unsigned long long)rows[g * bag + k0 + k] * row_bytes);
+                else
+                    gpuvm_batch_skip(table, k * 32 + lane);
+            }
+            __syncwarp();
+            gpuvm_batch_access<true>(vm, table, nk * 32, GPUVM_READ, [=](unsigned int i, const unsigned char *p) {
+                if (lane < q) staging[(size_t)i * q + lane] = gpuvm_load16(p + 16u * lane);
+            }, queue);
+            __syncwarp();
+            // add the staged rows of each bag in list order
+            for (unsigned int b = 0; b < 32 && g0 + b < n_bags; ++b) {
+                if (lane < q) {
+                    float4 *dst = reinterpret_cast<float4 *>(out + (g0 + b) * dims) + lane;
+                    float4 acc = k0 == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *dst;
+#pragma unroll 8
+                    for (unsigned int k = 0; k < nk; ++k) {
+                        const uint4 v = staging[(size_t)(k * 32 + b) * q + lane];
+                        acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
+                        acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
+                        acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
+                        acc.w = __fadd_rn(acc.w, __uint_as_float(v.w));
+                    }
+                    *dst = acc;
+                }
+            }
+            __syncwarp();
+        }
+    }
+    if (lane == 0) gpuvm_requester_done(queue);
+}
+
 // ------------------------------------------------------- element read-modify-write
 template <class Mem>
 __global__ void __launch_bounds__(256) scatter_update_kernel(Mem m, unsigned long long a_off,
@@ -738,6 +812,30 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
 
 int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
                     void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    if (!d_rows || !d_out || dims == 0 || dims % 4 || dims / 4 > 32 || bag == 0 || bag > 0xFFFFFFFFull) return GPUVM_E_ARG;
+    if (t_off % 16) return GPUVM_E_ALIGN;
+    if (n_bags == 0) return GPUVM_OK;
+    if (m.vm.page_shift > 27) return GPUVM_E_PAGE;
+    const int requesters = kEmbagRequesters, migrators = kEmbagMigrators;
+    const size_t items = (n_bags + 31) / 32;
+    const size_t blocks_needed = (items + requesters - 1) / requesters;
+    const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
+    const size_t per_warp = 32 * kEmbagLookups;
+    const size_t table_bytes = ((size_t)grid * requesters * per_warp * sizeof(gpuvm_batch_entry) + 255) & ~size_t(255);
+    const size_t staging_bytes = (size_t)grid * requesters * per_warp * 4 * dims;
+    unsigned char *scratch = static_cast<unsigned char *>(gpuvm_scratch_(h, table_bytes + staging_bytes));
+    if (!scratch) return GPUVM_E_ALLOC;
+    embag_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        m.vm, t_off, (unsigned int)dims, reinterpret_cast<const long long *>(d_rows), n_bags, (unsigned int)bag, d_out,
+        requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes);
+    return launched();
+}
+
+int gpuvm_embag_f32_unbatched(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag,
+                              float *d_out, void *stream)
 {
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;

@@ -94,8 +94,9 @@ def test_cfg5_zipf_embedding_bag_64GiB():
             assert np.array_equal(ref.view(np.uint32), out[start:start + 256].view(np.uint32)), start
         st = res.stats
         distinct = np.unique(rows >> 12).size                   # 4096 rows per 2 MiB page
-        assert st["faults"] >= distinct
-        # characteristic-time estimate of an LRU-like cache on this Zipf stream: about 1.06e6 faults
-        assert 0.7 * 1.06e6 <= st["faults"] <= 1.3 * 1.06e6
+        # never fewer than one fault per page touched; a one-request-at-a-time LRU-like cache on
+        # this Zipf stream takes about 1.06e6 (characteristic-time estimate), and requests that
+        # are registered together share faults, so the batched kernel stays well below that
+        assert distinct <= st["faults"] <= 1.3 * 1.06e6
     finally:
         w.close()

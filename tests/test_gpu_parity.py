@@ -207,21 +207,24 @@ def test_bfs_rmat_with_hub_vertices(B, scale, page, frames):
     assert st["writebacks"] == 0
 
 
-@pytest.mark.parametrize("page,n_rows,n_bags,frames", [
-    (4096, 512, 64, 64),
-    (4096, 4096, 1000, 8),
-    (2 << 20, 1 << 14, 1 << 12, 2),
-    (512, 100, 33, 1),
+@pytest.mark.parametrize("page,n_rows,n_bags,frames,dims,bag", [
+    (4096, 512, 64, 64, 128, 32),
+    (4096, 4096, 1000, 8, 128, 32),
+    (2 << 20, 1 << 14, 1 << 12, 2, 128, 32),
+    (512, 100, 33, 1, 128, 32),
+    (4096, 2000, 70, 16, 128, 40),                 # bags longer than one batch of 32 lookups
+    (4096, 2000, 70, 16, 64, 5),                   # narrow rows, short bags
 ])
-def test_embag(B, page, n_rows, n_bags, frames):
+@pytest.mark.parametrize("batched", [True, False])
+def test_embag(B, page, n_rows, n_bags, frames, dims, bag, batched):
     import torch
-    dims, bag = 128, 32
     t = inputs.fill_f32_pm1(np.empty(n_rows * dims, np.float32), n_rows * dims, inputs.config_seed(5))
     rows = inputs.fill_zipf_rows(np.empty(n_bags * bag, np.int64), n_bags * bag, inputs.config_seed(5, 1), n_rows, 1.05)
     ar = Arena(page, {"t": t})
     out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
     with paged(ar.host, page, frames) as h:
-        B.gpuvm_embag_f32(h, ar.off["t"], dims, dev(rows), n_bags, bag, out)
+        run = B.gpuvm_embag_f32 if batched else B.gpuvm_embag_f32_unbatched
+        run(h, ar.off["t"], dims, dev(rows), n_bags, bag, out)
         st, ck = finish(h)
     ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
     got = out.cpu().numpy()
