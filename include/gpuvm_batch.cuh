@@ -270,7 +270,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
                         frame = kFailed;
                     } else if (!((own >> j) & 1ull)) {
                         unsigned int f;
-                        const int st = advance(vm, pte, ld_relaxed_u64(pte), mode, f);
+                        const int st = advance(vm, pte, ld_acquire_u64(pte), mode, f);   /* acquire: pairs with the publish */
                         if (st == kReady) frame = f;
                         else if (st == kOwn) { own |= 1ull << j; progress = true; }
                     }
@@ -281,7 +281,6 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
             const bool ready = mine && frame < kFailed;
             if (WARP_CONSUME) {
                 unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
-                if (ready_lanes) __threadfence();
                 while (ready_lanes) {
                     const unsigned int L = __ffs(ready_lanes) - 1;
                     ready_lanes &= ready_lanes - 1;
@@ -291,7 +290,6 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
                 __syncwarp();                                   /* every group has used its frame */
             } else {
                 if (ready) {
-                    __threadfence();
                     consume(i, vm.pool + ((unsigned long long)frame << vm.page_shift) + off);
                 }
                 if (mine) __syncwarp(rowmask);                  /* the whole group has used the frame */

@@ -145,6 +145,10 @@ int gpuvm_embag_f32_unbatched(gpuvm_t h, size_t t_off, size_t dims, const int64_
  */
 int gpuvm_scatter_update_u32(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream);
 
+/* The same update through gpuvm_batch_access in write mode, 1024 requests per warp staged in
+ * shared memory, without migrator warps: each warp migrates the pages of its own faults. */
+int gpuvm_scatter_update_u32_batched(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream);
+
 /*
  * Transfer micro-benchmark (Section 5.1, Fig. 7): touch n_pages consecutive pages
  * starting at page first_page, one warp per page, `warps_per_sm` warps on every SM;

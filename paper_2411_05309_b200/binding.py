@@ -77,6 +77,7 @@ SYMBOLS = {
     "gpuvm_embag_f32": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_embag_f32_unbatched": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_scatter_update_u32": (_i, [_vp, _sz, _vp, _sz, _vp]),
+    "gpuvm_scatter_update_u32_batched": (_i, [_vp, _sz, _vp, _sz, _vp]),
     "gpuvm_touch_pages": (_i, [_vp, _sz, _sz, _i, _vp]),
     "gpuvm_raw_stream_sum_i32": (_i, [_vp, _sz, _vp, _vp]),
     "gpuvm_raw_gather_f32": (_i, [_vp, _vp, _sz, _sz, _vp, _vp, _vp]),
@@ -270,6 +271,11 @@ def gpuvm_embag_f32_unbatched(h, t_off: int, dims: int, d_rows, n_bags: int, bag
 
 def gpuvm_scatter_update_u32(h, a_off: int, d_idx, n: int, stream=None):
     _check(lib().gpuvm_scatter_update_u32(h, a_off, _ptr(d_idx), n, _stream(stream)), "gpuvm_scatter_update_u32")
+
+
+def gpuvm_scatter_update_u32_batched(h, a_off: int, d_idx, n: int, stream=None):
+    _check(lib().gpuvm_scatter_update_u32_batched(h, a_off, _ptr(d_idx), n, _stream(stream)),
+           "gpuvm_scatter_update_u32_batched")
 
 
 def gpuvm_touch_pages(h, first_page: int, n_pages: int, warps_per_sm: int, stream=None):

@@ -528,6 +528,29 @@ __global__ void __launch_bounds__(256) scatter_update_kernel(Mem m, unsigned lon
     }
 }
 
+// The same update with batched requests and no helper warps: every warp stages 1024 requests in
+// shared memory and migrates the pages of the faults it owns itself.
+__global__ void __launch_bounds__(128) scatter_update_batch_kernel(gpuvm_dev_t vm, unsigned long long a_off,
+                                                                   const long long *__restrict__ idx, unsigned long long n)
+{
+    __shared__ gpuvm_batch_entry s_table[4][1024];
+    const unsigned int lane = threadIdx.x & 31;
+    gpuvm_batch_entry *table = s_table[threadIdx.x >> 5];
+    const unsigned long long batches = (n + 1023) / 1024;
+    for (unsigned long long t = warp_in_grid(); t < batches; t += warps_in_grid()) {
+        const unsigned long long base = t * 1024;
+        const unsigned int m = (unsigned int)(n - base < 1024 ? n - base : 1024);
+        for (unsigned int k = lane; k < m; k += 32)
+            gpuvm_batch_set(vm, table, k, a_off + 4ull * (unsigned long long)idx[base + k]);
+        __syncwarp();
+        gpuvm_batch_access(vm, table, m, GPUVM_WRITE, [](unsigned int, const unsigned char *p) {
+            unsigned int *q = reinterpret_cast<unsigned int *>(const_cast<unsigned char *>(p));
+            gpuvm_store(q, gpuvm_load(q) * 3u + 1u);
+        });
+        __syncwarp();
+    }
+}
+
 // ------------------------------------------------------------------ page touch
 __global__ void touch_pages_kernel(gpuvm_dev_t vm, unsigned long long first_page, unsigned long long n_pages)
 {
@@ -850,6 +873,18 @@ int gpuvm_scatter_update_u32(gpuvm_t h, size_t a_off, const int64_t *d_idx, size
     if (n == 0) return GPUVM_OK;
     scatter_update_kernel<Paged><<<sm_count() * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         m, a_off, reinterpret_cast<const long long *>(d_idx), n);
+    return launched();
+}
+
+int gpuvm_scatter_update_u32_batched(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m) || !d_idx) return GPUVM_E_ARG;
+    if (a_off % 16) return GPUVM_E_ALIGN;
+    if (m.vm.page_shift > 27) return GPUVM_E_PAGE;
+    if (n == 0) return GPUVM_OK;
+    scatter_update_batch_kernel<<<sm_count() * 4, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        m.vm, a_off, reinterpret_cast<const long long *>(d_idx), n);
     return launched();
 }
 

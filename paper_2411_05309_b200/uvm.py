@@ -58,9 +58,14 @@ def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0) -> dict:
             balloon = B.gpuvm_balloon_alloc(w.pool_bytes + SLACK)
             out["free_bytes_under_balloon"] = B.gpuvm_mem_info()[0]
             read_only = cfg != 4
-            for advise in ([False, True] if read_only else [False]):
+            # cfg 2 is not run with read-mostly: under the balloon, the random gather over
+            # read-duplicated managed pages once ended in an illegal-address fault raised while the
+            # driver serviced it (the same kernel and arguments had just run without the advice);
+            # the combination is left alone rather than probed further
+            variants = [False] if cfg in (2, 4) else [False, True]
+            for advise in variants:
                 rec = {"read_mostly": advise}
-                rec.update(_one(torch, w, cfg, p, timeout_s / (2 if read_only else 1), bufs, advise))
+                rec.update(_one(torch, w, cfg, p, timeout_s / len(variants), bufs, advise))
                 out["runs"].append(rec)
         finally:
             if balloon:
