@@ -111,6 +111,47 @@ def test_wait_that_runs_out_returns_an_error_status(B):
         assert int(out.item()) == int(a.astype(np.int64).sum())
 
 
+@pytest.mark.parametrize("which", ["gather", "gather_unbatched", "scatter_batched", "embag"])
+def test_batched_waits_run_out_too(B, which):
+    """The batched engine and the migrator warps give up in the same way: a page that stays
+    BUSY makes its requests fail after spin_limit_us, everything else is served, the kernel
+    ends, the error is reported, and after a reset the same call succeeds."""
+    import torch
+    page, n = 4096, 1 << 14
+    x = inputs.fill_f32_pm1(np.empty(n, np.float32), n, 3)
+    idx = np.random.default_rng(1).permutation(n).astype(np.int64)[:8192]
+    ar = Arena(page, {"x": x})
+    d_idx = torch.from_numpy(idx).cuda()
+    fs = torch.zeros(8, dtype=torch.float32, device="cuda")
+    bs = torch.zeros(8, dtype=torch.int64, device="cuda")
+    out = torch.zeros(256 * 128, dtype=torch.float32, device="cuda")
+    rows = torch.from_numpy((idx % (n // 128))[:256 * 32].copy()).cuda()
+
+    def call(h):
+        if which == "gather":
+            B.gpuvm_gather_f32(h, 0, d_idx, idx.size, 1024, fs, bs)
+        elif which == "gather_unbatched":
+            B.gpuvm_gather_f32_unbatched(h, 0, d_idx, idx.size, 1024, fs, bs)
+        elif which == "scatter_batched":
+            B.gpuvm_scatter_update_u32_batched(h, 0, d_idx, idx.size)
+        else:
+            B.gpuvm_embag_f32(h, 0, 128, rows, 256, 32, out)
+
+    with paged(ar.host, page, 6, spin_limit_us=30_000) as h:
+        B.gpuvm_debug_poke_pte(h, 5, BUSY)
+        call(h)
+        torch.cuda.synchronize()
+        st = B.gpuvm_stats(h, raise_on_error=False)
+        assert st["error"] == B.E_TIMEOUT and st["error_page"] == 5
+        B.gpuvm_reset(h)
+        ar.views["x"][...] = x
+        call(h)
+        st, ck = finish(h)
+        if which.startswith("gather"):
+            import oracle
+            assert np.array_equal(bs.cpu().numpy(), oracle.gather_block_sums_direct(x, idx, 1024)[1])
+
+
 def test_offset_past_the_end_is_a_range_error(B):
     import torch
     host = aligned_bytes(8 * 4096)
