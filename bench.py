@@ -167,6 +167,19 @@ def oracle_step(cfg: int, w=None, shrink: int = 0):
         deg = np.diff(off)
         vis = lvl >= 0
         return int(16 * vis.sum() + 4 * deg[vis].sum()), dt, f"direct BFS on an RMAT graph of scale {scale}"
+    if cfg in (6, 7):
+        scale = min(24 - shrink, 22)
+        off, col = inputs.rmat_csr(scale, 16 << scale, inputs.config_seed(3))
+        if cfg == 6:
+            t0 = time.perf_counter()
+            oracle.cc_labels_direct(off, col)
+            return 8 * off.size + 4 * col.size, time.perf_counter() - t0, f"union-find over an RMAT graph of scale {scale} (one pass over the edges)"
+        w = inputs.fill_i32_range(np.empty(col.size, np.int32), col.size, inputs.config_seed(3, 2), 1, 255)
+        t0 = time.perf_counter()
+        d = oracle.sssp_direct(off, col, w, 0)
+        dt = time.perf_counter() - t0
+        reached = d != 0x7FFFFFFF
+        return int(16 * reached.sum() + 8 * np.diff(off)[reached].sum()), dt, f"Dijkstra on an RMAT graph of scale {scale}"
     if cfg == 5:
         rows_n, dims, bag = 1 << 20, 128, 32
         t = inputs.fill_f32_pm1(np.empty(rows_n * dims, np.float32), rows_n * dims, inputs.config_seed(5)).reshape(rows_n, dims)
@@ -203,8 +216,10 @@ NAMES = {1: "cfg1 streaming read-reduce: int64 sum over 64 MiB int32, 4 KiB page
          2: "cfg2 random gather: 1 GiB fp32 array, 2^26 uniform int64 indices, sum per 1024, 64 KiB pages, 256 MiB pool",
          3: "cfg3 BFS on RMAT scale 24 (avg degree 16), CSR paged at 64 KiB, pool = half",
          4: "cfg4 vector add c=a+b over three 4 GiB fp32 arrays, 64 KiB pages, 4 GiB pool",
-         5: "cfg5 Zipf(1.05) embedding bag: 64 GiB table, 2^24 lookups, bags of 32, 2 MiB pages, 16 GiB pool"}
-DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32"}
+         5: "cfg5 Zipf(1.05) embedding bag: 64 GiB table, 2^24 lookups, bags of 32, 2 MiB pages, 16 GiB pool",
+         6: "connected components on the cfg3 graph (RMAT scale 24), CSR paged at 64 KiB, pool = half",
+         7: "SSSP from vertex 0 on the cfg3 graph with int32 weights in a third paged array, 64 KiB pages, pool = half"}
+DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32", 6: "int32", 7: "int32"}
 
 
 # ---------------------------------------------------------------------- rank plumbing
@@ -242,7 +257,7 @@ def e2e_step(torch, B, w, cfg: int):
         h2d = w.rows_host.numel() * 8
     w.launch(stream)
     B.gpuvm_flush(w.h, stream)
-    outs = {1: ["d_sum"], 2: ["d_fsum", "d_bsum"], 3: ["d_level"], 4: [], 5: ["d_out"]}[cfg]
+    outs = {1: ["d_sum"], 2: ["d_fsum", "d_bsum"], 3: ["d_level"], 4: [], 5: ["d_out"], 6: ["d_level"], 7: ["d_dist"]}[cfg]
     for name in outs:
         t = getattr(w, name)
         buf = w.__dict__.setdefault("_host_" + name, torch.empty(t.shape, dtype=t.dtype).pin_memory())
@@ -359,7 +374,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7])
     ap.add_argument("--shrink", type=int, default=0, help="divide all sizes by 2**shrink")
     ap.add_argument("--uvm", action="store_true", help="also run the workload over cudaMallocManaged")
     ap.add_argument("--uvm-timeout", type=float, default=120.0)

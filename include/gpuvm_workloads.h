@@ -12,8 +12,8 @@
  *   - calls enqueue work and return without synchronising unless stated; device
  *     errors (a wait that ran out, an offset out of range) are sticky in the handle
  *     and show up in gpuvm_stats().  Return value: 0 or a negative gpuvm_status.
- *   - nothing here allocates device memory except gpuvm_bfs_csr (1 MiB of scratch,
- *     freed before it returns) and the first gpuvm_gather_f32 / gpuvm_embag_f32 on
+ *   - nothing here allocates device memory except the graph workloads (2 MiB of
+ *     scratch, plus 2 bytes per vertex for SSSP, freed before they return) and the first gpuvm_gather_f32 / gpuvm_embag_f32 on
  *     a handle (request tables and row staging, kept by the handle).
  */
 #ifndef GPUVM_WORKLOADS_H
@@ -67,10 +67,38 @@ int gpuvm_gather_f32_unbatched(gpuvm_t h, size_t x_off, const int64_t *d_idx, si
  * spread over the whole grid (the imbalance Section 5.2 describes).  Synchronises the
  * stream between levels; *n_levels (host pointer, may be NULL) receives the number
  * of levels expanded, counting the last one that discovers nothing.  Allocates and
- * frees 1 MiB of device scratch (queue of neighbour-list pieces, counters).
+ * frees 2 MiB of device scratch (queue of neighbour-list pieces, counters).
  */
 int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
                   int32_t *d_level, int *n_levels, void *stream);
+
+/*
+ * Connected components of the same kind of graph (Section 5.2 evaluates CC next to
+ * BFS): d_label[v] receives the smallest vertex number of the weakly connected
+ * component of v (edges count in both directions).  Label propagation: every sweep
+ * visits every edge (u, c) and lowers the larger of the two labels to the smaller
+ * with atomicMin, until a sweep changes nothing.  Sweeps alternate direction like
+ * the BFS levels.  *n_sweeps (host pointer, may be NULL) receives the number of
+ * sweeps.  Allocates and frees 2 MiB of device scratch.  Synchronises per sweep.
+ */
+int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps,
+                 void *stream);
+
+/*
+ * Single-source shortest paths with int32 edge weights >= 0 stored in a third paged
+ * array parallel to the column indices (Section 5.2; the weights are a separate
+ * array as in the paper's Table 2).  w_off must differ from col_off by a multiple of
+ * the page size, so that the weights of an edge range sit at the same place in their
+ * page as the columns do in theirs; both pages are held together while the range is
+ * relaxed, hence the pool needs at least two frames per warp of the grid
+ * (GPUVM_E_POOL otherwise).  Bellman-Ford rounds over the vertices that changed in
+ * the previous round; d_dist[v] receives the distance from `source`, 0x7FFFFFFF
+ * where unreachable (path lengths must stay below that).  *n_rounds (host pointer,
+ * may be NULL) receives the number of rounds.  Allocates and frees 2 MiB + 2 nv bytes
+ * of device scratch.  Synchronises per round.
+ */
+int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source,
+                   int32_t *d_dist, int *n_rounds, void *stream);
 
 /*
  * gpuvm_bfs_csr for callers that must not allocate.  (The paper has no counterpart:
@@ -83,13 +111,13 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
  * all free device memory to their own pool, where cudaMalloc would simply fail.
  * For them this variant does exactly what gpuvm_bfs_csr does, same kernels, same
  * arguments, same results, but takes its scratch (the queue of neighbour-list
- * pieces and the level counters, 1 MiB + 16 bytes) from an array that is part of
+ * pieces and the level counters, 2 MiB + 16 bytes) from an array that is part of
  * the library's device image.  It calls no cudaMalloc, cudaFree or other
  * allocating routine.
  *
  *   - Limit: nv <= GPUVM_BFS_NOALLOC_MAX_VERTICES, the graph size the fixed queue
  *     is sized for; anything larger returns GPUVM_E_RANGE and runs nothing.
- *   - Cost: every device that loads the library holds the 1 MiB array until the
+ *   - Cost: every device that loads the library holds the 2 MiB array until the
  *     process exits, whether or not this function is ever called.
  *   - The first call on a device looks up the array's device address (once per
  *     device, with that device current).  Make that first call during set-up,
@@ -162,6 +190,10 @@ int gpuvm_raw_gather_f32(const float *x, const int64_t *d_idx, size_t n_idx, siz
                          float *d_fsum, int64_t *d_bsum, void *stream);
 int gpuvm_raw_bfs_csr(const int64_t *row_off, const int32_t *col, size_t nv, size_t source,
                       int32_t *d_level, int *n_levels, void *stream);
+int gpuvm_raw_cc_csr(const int64_t *row_off, const int32_t *col, size_t nv, int32_t *d_label, int *n_sweeps,
+                     void *stream);
+int gpuvm_raw_sssp_csr(const int64_t *row_off, const int32_t *col, const int32_t *weight, size_t nv,
+                       size_t source, int32_t *d_dist, int *n_rounds, void *stream);
 int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void *stream);
 int gpuvm_raw_embag_f32(const float *table, size_t dims, const int64_t *d_rows, size_t n_bags,
                         size_t bag, float *d_out, void *stream);

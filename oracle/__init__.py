@@ -44,6 +44,8 @@ def _load():
             "orc_stream_sum_i32_direct": (ctypes.c_int64, [vp, u64]),
             "orc_gather_block_sums_direct": (None, [vp, vp, u64, u64, vp, vp]),
             "orc_bfs_levels_direct": (None, [vp, vp, u64, u64, vp]),
+            "orc_cc_labels_direct": (None, [vp, vp, u64, vp]),
+            "orc_sssp_direct": (None, [vp, vp, vp, u64, u64, vp]),
             "orc_vadd_f32_direct": (None, [vp, vp, vp, u64]),
             "orc_embag_f32_direct": (None, [vp, u64, vp, u64, u64, vp]),
             "orc_pager_create": (vp, [vp, u64, u64, u64, i32, i32]),
@@ -95,6 +97,21 @@ def bfs_levels_direct(row_off: np.ndarray, col: np.ndarray, source: int) -> np.n
     _load().orc_bfs_levels_direct(_p(row_off, np.int64), _p(col, np.int32), nv, source,
                                   _p(level, np.int32))
     return level
+
+
+def cc_labels_direct(row_off: np.ndarray, col: np.ndarray) -> np.ndarray:
+    nv = row_off.size - 1
+    label = np.empty(nv, dtype=np.int32)
+    _load().orc_cc_labels_direct(_p(row_off, np.int64), _p(col, np.int32), nv, _p(label, np.int32))
+    return label
+
+
+def sssp_direct(row_off: np.ndarray, col: np.ndarray, weight: np.ndarray, source: int) -> np.ndarray:
+    nv = row_off.size - 1
+    dist = np.empty(nv, dtype=np.int32)
+    _load().orc_sssp_direct(_p(row_off, np.int64), _p(col, np.int32), _p(weight, np.int32), nv, source,
+                            _p(dist, np.int32))
+    return dist
 
 
 def vadd_f32_direct(a: np.ndarray, b: np.ndarray) -> np.ndarray:

@@ -99,6 +99,87 @@ void orc_bfs_levels_direct(const int64_t *row_off, const int32_t *col, uint64_t 
     free(queue);
 }
 
+/*
+ * Weakly connected components (Section 5.2 runs CC on the same graphs): label[v] = the
+ * smallest vertex number in the component of v when edges count in both directions.
+ * Union-find with the smaller root as the representative.
+ */
+static uint64_t uf_find(uint64_t *parent, uint64_t v)
+{
+    while (parent[v] != v) {
+        parent[v] = parent[parent[v]];
+        v = parent[v];
+    }
+    return v;
+}
+
+void orc_cc_labels_direct(const int64_t *row_off, const int32_t *col, uint64_t nv, int32_t *label)
+{
+    uint64_t *parent = (uint64_t *)malloc(nv * sizeof(uint64_t));
+    for (uint64_t v = 0; v < nv; ++v) parent[v] = v;
+    for (uint64_t u = 0; u < nv; ++u)
+        for (int64_t e = row_off[u]; e < row_off[u + 1]; ++e) {
+            uint64_t a = uf_find(parent, u), b = uf_find(parent, (uint64_t)col[e]);
+            if (a < b) parent[b] = a;
+            else if (b < a) parent[a] = b;
+        }
+    for (uint64_t v = 0; v < nv; ++v) label[v] = (int32_t)uf_find(parent, v);
+    free(parent);
+}
+
+/*
+ * Single-source shortest paths with non-negative int32 weights (Section 5.2 runs SSSP with a
+ * separate weight array): Dijkstra with a binary heap of (distance, vertex) pairs and lazy
+ * deletion.  dist[v] = 0x7FFFFFFF when v cannot be reached.
+ */
+typedef struct { int64_t d; uint64_t v; } orc_heap_item;
+
+static void heap_push(orc_heap_item *h, uint64_t *n, orc_heap_item it)
+{
+    uint64_t i = (*n)++;
+    while (i > 0 && h[(i - 1) / 2].d > it.d) { h[i] = h[(i - 1) / 2]; i = (i - 1) / 2; }
+    h[i] = it;
+}
+
+static orc_heap_item heap_pop(orc_heap_item *h, uint64_t *n)
+{
+    orc_heap_item top = h[0], last = h[--(*n)];
+    uint64_t i = 0;
+    for (;;) {
+        uint64_t c = 2 * i + 1;
+        if (c >= *n) break;
+        if (c + 1 < *n && h[c + 1].d < h[c].d) ++c;
+        if (h[c].d >= last.d) break;
+        h[i] = h[c];
+        i = c;
+    }
+    h[i] = last;
+    return top;
+}
+
+void orc_sssp_direct(const int64_t *row_off, const int32_t *col, const int32_t *weight, uint64_t nv, uint64_t source,
+                     int32_t *dist)
+{
+    const int64_t INF = 0x7FFFFFFF;
+    int64_t *d = (int64_t *)malloc(nv * sizeof(int64_t));
+    for (uint64_t v = 0; v < nv; ++v) d[v] = INF;
+    uint64_t cap = (uint64_t)row_off[nv] + 1, n = 0;
+    orc_heap_item *heap = (orc_heap_item *)malloc(cap * sizeof(orc_heap_item));
+    d[source] = 0;
+    heap_push(heap, &n, (orc_heap_item){0, source});
+    while (n) {
+        orc_heap_item it = heap_pop(heap, &n);
+        if (it.d != d[it.v]) continue;                  /* stale entry */
+        for (int64_t e = row_off[it.v]; e < row_off[it.v + 1]; ++e) {
+            int64_t nd = it.d + (int64_t)weight[e];
+            uint64_t c = (uint64_t)col[e];
+            if (nd < d[c]) { d[c] = nd; heap_push(heap, &n, (orc_heap_item){nd, c}); }
+        }
+    }
+    for (uint64_t v = 0; v < nv; ++v) dist[v] = (int32_t)d[v];
+    free(heap); free(d);
+}
+
 /* c[i] = a[i] + b[i], one correctly rounded binary32 addition per element. */
 void orc_vadd_f32_direct(const float *a, const float *b, float *c, uint64_t n)
 {

@@ -73,6 +73,10 @@ SYMBOLS = {
     "gpuvm_gather_f32_unbatched": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp, _vp]),
     "gpuvm_bfs_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_bfs_csr_noalloc": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
+    "gpuvm_cc_csr": (_i, [_vp, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
+    "gpuvm_sssp_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
+    "gpuvm_raw_cc_csr": (_i, [_vp, _vp, _sz, _vp, ctypes.POINTER(_i), _vp]),
+    "gpuvm_raw_sssp_csr": (_i, [_vp, _vp, _vp, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_vadd_f32": (_i, [_vp, _sz, _sz, _sz, _sz, _vp]),
     "gpuvm_embag_f32": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_embag_f32_unbatched": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
@@ -241,6 +245,34 @@ def gpuvm_bfs_csr(h, off_off: int, col_off: int, nv: int, source: int, d_level, 
     _check(lib().gpuvm_bfs_csr(h, off_off, col_off, nv, source, _ptr(d_level), ctypes.byref(levels), _stream(stream)),
            "gpuvm_bfs_csr")
     return levels.value
+
+
+def gpuvm_cc_csr(h, off_off: int, col_off: int, nv: int, d_label, stream=None) -> int:
+    sweeps = _i(0)
+    _check(lib().gpuvm_cc_csr(h, off_off, col_off, nv, _ptr(d_label), ctypes.byref(sweeps), _stream(stream)),
+           "gpuvm_cc_csr")
+    return sweeps.value
+
+
+def gpuvm_sssp_csr(h, off_off: int, col_off: int, w_off: int, nv: int, source: int, d_dist, stream=None) -> int:
+    rounds = _i(0)
+    _check(lib().gpuvm_sssp_csr(h, off_off, col_off, w_off, nv, source, _ptr(d_dist), ctypes.byref(rounds),
+                                _stream(stream)), "gpuvm_sssp_csr")
+    return rounds.value
+
+
+def gpuvm_raw_cc_csr(row_off, col, nv: int, d_label, stream=None) -> int:
+    sweeps = _i(0)
+    _check(lib().gpuvm_raw_cc_csr(_ptr(row_off), _ptr(col), nv, _ptr(d_label), ctypes.byref(sweeps), _stream(stream)),
+           "gpuvm_raw_cc_csr")
+    return sweeps.value
+
+
+def gpuvm_raw_sssp_csr(row_off, col, weight, nv: int, source: int, d_dist, stream=None) -> int:
+    rounds = _i(0)
+    _check(lib().gpuvm_raw_sssp_csr(_ptr(row_off), _ptr(col), _ptr(weight), nv, source, _ptr(d_dist),
+                                    ctypes.byref(rounds), _stream(stream)), "gpuvm_raw_sssp_csr")
+    return rounds.value
 
 
 BFS_NOALLOC_MAX_VERTICES = 1 << 26

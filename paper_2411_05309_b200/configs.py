@@ -194,6 +194,49 @@ class Bfs(Workload):
         return int(16 * visited.sum() + 4 * self.traversed_edges)
 
 
+class Cc(Bfs):
+    """Connected components on the BFS configuration's graph and pool (the paper's second graph workload)."""
+    name, cfg = "cc_rmat_csr", 6
+
+    def launch(self, stream):
+        self.sweeps = B.gpuvm_cc_csr(self.h, self.off["off"], self.off["col"], self.nv, self.d_level, stream)
+        return {"sweeps": self.sweeps}
+
+    def effective_bytes(self):
+        # every sweep reads every row offset and every edge
+        return int(self.sweeps * (8 * (self.nv + 1) + 4 * self.ne))
+
+
+class Sssp(Workload):
+    """SSSP from vertex 0 on the same RMAT graph with int32 weights in [1, 255] in a third paged array;
+    pool = half of the three arrays."""
+    name, cfg, page_bytes = "sssp_rmat_csr", 7, 64 * KiB
+
+    def setup(self):
+        import torch
+        self.scale = 24 - self.shrink
+        self.nv = 1 << self.scale
+        self.ne = 16 << self.scale
+        self._create({"off": _pad(8 * (self.nv + 1), 16), "col": 4 * self.ne, "w": 4 * self.ne}, lambda total: total // 2)
+        base = B.gpuvm_host_ptr(self.h)
+        inputs.rmat_csr(self.scale, self.ne, inputs.config_seed(3), base + self.off["off"], base + self.off["col"])
+        inputs.fill_i32_range(base + self.off["w"], self.ne, inputs.config_seed(3, 2), 1, 255)
+        self.d_dist = torch.zeros(self.nv, dtype=torch.int32, device="cuda")
+        self.rounds = 0
+        return self
+
+    def launch(self, stream):
+        self.rounds = B.gpuvm_sssp_csr(self.h, self.off["off"], self.off["col"], self.off["w"], self.nv, 0, self.d_dist,
+                                       stream)
+        return {"rounds": self.rounds}
+
+    def effective_bytes(self):
+        d = self.d_dist.cpu().numpy()
+        off = self.view("off", np.int64, self.nv + 1)
+        reached = d != 0x7FFFFFFF
+        return int(16 * reached.sum() + 8 * np.diff(off)[reached].sum())     # offsets + (column, weight) per edge, once
+
+
 class VAdd(Workload):
     """c = a + b over three fp32 arrays, 64 KiB pages, pool = one array (3x oversubscribed)."""
     name, cfg, page_bytes = "vector_add_f32", 4, 64 * KiB
@@ -239,7 +282,7 @@ class EmbeddingBag(Workload):
         return 4 * self.dims * self.n_lookups
 
 
-WORKLOADS = {1: StreamSum, 2: Gather, 3: Bfs, 4: VAdd, 5: EmbeddingBag}
+WORKLOADS = {1: StreamSum, 2: Gather, 3: Bfs, 4: VAdd, 5: EmbeddingBag, 6: Cc, 7: Sssp}
 
 
 def make(cfg: int, shrink: int = 0) -> Workload:

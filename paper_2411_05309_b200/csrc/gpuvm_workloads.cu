@@ -210,37 +210,79 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
     if (lane == 0) gpuvm_requester_done(queue);
 }
 
-// ------------------------------------------------------------------------ BFS
+// ------------------------------------------------------- graph sweeps (BFS, CC, SSSP)
 constexpr long long kBigDegree = 4096;     // neighbour lists at least this long are spread over the grid
-constexpr unsigned int kBigQueue = 65536;  // entries of the span queue (two int64 each)
+constexpr unsigned int kBigQueue = 65536;  // entries of the span queue (four int64 each: first edge, end, vertex, -)
 
-// counters: [0] vertices discovered in this level, [1] span queue size, [2] chunk ticket, [3] span ticket
+// counters: [0] updates made in this sweep, [1] span queue size, [2] chunk ticket, [3] span ticket
 
-// Visit the edges [elo, ehi) that lie inside the pinned unit starting at edge `first`.
-template <class Mem>
-__device__ __forceinline__ unsigned int bfs_visit(const unsigned char *unit_ptr, long long first, long long elo,
-                                                  long long ehi, unsigned int lane, int *__restrict__ level, int depth)
+// What a sweep does with a vertex and with each of its edges.
+struct BfsOp {                              // level-synchronous BFS: expand the vertices of the current level
+    int *level;
+    int depth;
+    __device__ __forceinline__ bool active(unsigned long long v) const { return level[v] == depth; }
+    __device__ __forceinline__ unsigned int edge(long long, int c, int) const
+    {
+        return level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1;
+    }
+};
+
+struct CcOp {                               // label propagation over every edge, both ways, minimum label wins
+    int *label;
+    __device__ __forceinline__ bool active(unsigned long long) const { return true; }
+    __device__ __forceinline__ unsigned int edge(long long u, int c, int) const
+    {
+        const int lu = label[u], lc = label[c];
+        if (lu < lc) return atomicMin(label + c, lu) > lu;
+        if (lc < lu) return atomicMin(label + u, lc) > lc;
+        return 0;
+    }
+};
+
+struct SsspOp {                             // Bellman-Ford rounds: relax the edges of vertices that changed last round
+    int *dist;
+    const unsigned char *cur;
+    unsigned char *next;
+    __device__ __forceinline__ bool active(unsigned long long v) const { return cur[v] != 0; }
+    __device__ __forceinline__ unsigned int edge(long long u, int c, int w) const
+    {
+        const int du = dist[u];
+        if (du == 0x7FFFFFFF) return 0;
+        const int nd = du + w;
+        if (nd < dist[c] && atomicMin(dist + c, nd) > nd) { next[c] = 1; return 1; }
+        return 0;
+    }
+};
+
+// Visit the edges [elo, ehi) of vertex u that lie inside the pinned unit starting at edge `first`.
+template <class Mem, class Op, bool WEIGHTED>
+__device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned char *col_unit, const unsigned char *w_unit,
+                                                    long long first, long long u, long long elo, long long ehi,
+                                                    unsigned int lane)
 {
     unsigned int found = 0;
     for (long long e = elo + lane; e < ehi; e += 32) {
-        const int c = Mem::load_i32(unit_ptr + 4 * (e - first));
-        if (level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1) ++found;
+        const int c = Mem::load_i32(col_unit + 4 * (e - first));
+        const int w = WEIGHTED ? Mem::load_i32(w_unit + 4 * (e - first)) : 0;
+        found += op.edge(u, c, w);
     }
     return found;
 }
 
-// One level = one sweep over the vertices in ascending order: a warp draws the next chunk
-// of 32 consecutive vertices from a ticket counter, so at any moment the whole grid works
-// inside a narrow window of the row-offset and column arrays and a level touches every page
-// at most about once, in address order.  Per chunk the warp reads the 33 row offsets with
-// two accessor calls and then walks the column pages that the chunk's edges span, holding
-// one page at a time: one pin per page and chunk instead of one per neighbour list, which
-// keeps the atomic traffic on the entries of the few pages under the window low.
-template <class Mem>
-__global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long long off_off, unsigned long long col_off,
-                                                        int *__restrict__ level, unsigned int nv,
-                                                        long long *__restrict__ span_q, unsigned int *__restrict__ counters,
-                                                        int depth)
+// One sweep over the vertices in address order: a warp draws the next chunk of 32 consecutive
+// vertices from a ticket counter, so at any moment the whole grid works inside a narrow window
+// of the row-offset and column arrays and a sweep touches every page at most about once.
+// Per chunk the warp reads the 33 row offsets with two accessor calls and then walks the
+// column pages that the chunk's edges span, holding one page at a time (two with weights, which
+// sit at the same offset inside their own page): one pin per page and chunk instead of one per
+// neighbour list, which keeps the atomic traffic on the entries of the few pages under the
+// window low.  Odd sweeps run downwards: the pages a sweep used last are still resident when the
+// next one starts with them (a one-directional cyclic sweep defeats any LRU-like policy).
+template <class Mem, class Op, bool WEIGHTED>
+__global__ void __launch_bounds__(256) graph_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
+                                                          unsigned long long w_off, unsigned int nv,
+                                                          long long *__restrict__ span_q, unsigned int *__restrict__ counters,
+                                                          int sweep)
 {
     const unsigned int lane = threadIdx.x & 31;
     const unsigned long long unit = m.unit();
@@ -251,11 +293,9 @@ __global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long lon
         if (lane == 0) chunk = atomicAdd(counters + 2, 1u);
         chunk = __shfl_sync(0xFFFFFFFFu, chunk, 0);
         if (chunk >= n_chunks) break;
-        // odd levels sweep downwards: the pages a sweep used last are still resident when the
-        // next sweep starts with them (a one-directional cyclic sweep defeats any LRU-like policy)
-        const unsigned long long v0 = 32ull * ((depth & 1) ? n_chunks - 1 - chunk : chunk);
+        const unsigned long long v0 = 32ull * ((sweep & 1) ? n_chunks - 1 - chunk : chunk);
         const unsigned long long v = v0 + lane;
-        const bool active = v < nv && level[v] == depth;
+        const bool active = v < nv && op.active(v);
         if (!__any_sync(0xFFFFFFFFu, active)) continue;
         // row offsets of the chunk: off[v0 .. v0+32], clamped to the nv + 1 entries that exist
         long long lo = m.template read<long long>(off_off, v < nv ? v : nv);
@@ -274,14 +314,15 @@ __global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long lon
             if (lane == 0) slot = atomicAdd(counters + 1, pieces);
             slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
             if (slot + pieces > kBigQueue) {                       // queue full: expand the list here
-                for (unsigned int k = slot + lane; k < kBigQueue; k += 32) { span_q[2 * k] = 0; span_q[2 * k + 1] = 0; }
+                for (unsigned int k = slot + lane; k < kBigQueue; k += 32) { span_q[4 * k] = 0; span_q[4 * k + 1] = 0; }
                 continue;
             }
             for (unsigned int k = lane; k < pieces; k += 32) {
                 const long long s = (long long)(((b0 + k) * unit - col_off + 3) / 4);
                 const long long t = (long long)(((b0 + k + 1) * unit - col_off) / 4);
-                span_q[2 * (slot + k)] = k == 0 ? blo : s;
-                span_q[2 * (slot + k) + 1] = t < bhi ? t : bhi;
+                span_q[4 * (slot + k)] = k == 0 ? blo : s;
+                span_q[4 * (slot + k) + 1] = t < bhi ? t : bhi;
+                span_q[4 * (slot + k) + 2] = (long long)(v0 + L);
             }
             if ((int)lane == L) { lo = 0; hi = 0; }
         }
@@ -299,17 +340,23 @@ __global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long lon
             if (last > rhi) last = rhi;
             unsigned int touch = __ballot_sync(0xFFFFFFFFu, lo < last && hi > first);
             if (touch) {
-                gpuvm_token tok;
+                gpuvm_token tok, tok_w;
                 const unsigned char *p = m.pin(byte, GPUVM_READ, tok);
                 if (!p) return;
+                const unsigned char *pw = nullptr;
+                if (WEIGHTED) {
+                    pw = m.pin(w_off + 4ull * first, GPUVM_READ, tok_w);
+                    if (!pw) { m.release(tok); return; }
+                }
                 while (touch) {
                     const int L = __ffs(touch) - 1;
                     touch &= touch - 1;
                     long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
                     if (blo < first) blo = first;
                     if (bhi > last) bhi = last;
-                    found += bfs_visit<Mem>(p, first, blo, bhi, lane, level, depth);
+                    found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, (long long)(v0 + L), blo, bhi, lane);
                 }
+                if (WEIGHTED) m.release(tok_w);
                 m.release(tok);
             }
             first = last;
@@ -320,10 +367,10 @@ __global__ void __launch_bounds__(256) bfs_sweep_kernel(Mem m, unsigned long lon
 }
 
 // Pieces of long neighbour lists, one warp per piece (a piece never crosses a unit).
-template <class Mem>
-__global__ void __launch_bounds__(256) bfs_span_kernel(Mem m, unsigned long long col_off, int *__restrict__ level,
-                                                       const long long *__restrict__ span_q,
-                                                       unsigned int *__restrict__ counters, int depth)
+template <class Mem, class Op, bool WEIGHTED>
+__global__ void __launch_bounds__(256) graph_span_kernel(Mem m, Op op, unsigned long long col_off, unsigned long long w_off,
+                                                         const long long *__restrict__ span_q,
+                                                         unsigned int *__restrict__ counters)
 {
     const unsigned int lane = threadIdx.x & 31;
     const unsigned int n = counters[1] < kBigQueue ? counters[1] : kBigQueue;
@@ -333,12 +380,18 @@ __global__ void __launch_bounds__(256) bfs_span_kernel(Mem m, unsigned long long
         if (lane == 0) i = atomicAdd(counters + 3, 1u);
         i = __shfl_sync(0xFFFFFFFFu, i, 0);
         if (i >= n) break;
-        const long long elo = span_q[2 * i], ehi = span_q[2 * i + 1];
+        const long long elo = span_q[4 * i], ehi = span_q[4 * i + 1], u = span_q[4 * i + 2];
         if (ehi <= elo) continue;
-        gpuvm_token tok;
+        gpuvm_token tok, tok_w;
         const unsigned char *p = m.pin(col_off + 4ull * elo, GPUVM_READ, tok);
         if (!p) return;
-        found += bfs_visit<Mem>(p, elo, elo, ehi, lane, level, depth);
+        const unsigned char *pw = nullptr;
+        if (WEIGHTED) {
+            pw = m.pin(w_off + 4ull * elo, GPUVM_READ, tok_w);
+            if (!pw) { m.release(tok); return; }
+        }
+        found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, elo, u, elo, ehi, lane);
+        if (WEIGHTED) m.release(tok_w);
         m.release(tok);
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
@@ -346,6 +399,19 @@ __global__ void __launch_bounds__(256) bfs_span_kernel(Mem m, unsigned long long
 }
 
 __global__ void bfs_init_kernel(int *level, int source) { level[source] = 0; }
+
+__global__ void cc_init_kernel(int *label, unsigned int nv)
+{
+    for (unsigned int v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += gridDim.x * blockDim.x) label[v] = (int)v;
+}
+
+__global__ void sssp_init_kernel(int *dist, unsigned char *cur, unsigned int nv, unsigned int source)
+{
+    for (unsigned int v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += gridDim.x * blockDim.x) {
+        dist[v] = v == source ? 0 : 0x7FFFFFFF;
+        cur[v] = v == source;
+    }
+}
 
 // ----------------------------------------------------------------- vector add
 // A warp owns one unit (page) of the element range and walks it in chunks of at most 4 KiB.
@@ -653,30 +719,39 @@ int run_gather(const Mem &m, size_t x_off, const int64_t *d_idx, size_t n_idx, s
 }
 
 constexpr int kVaddBlocksPerSm = 4;
-constexpr size_t kBfsScratchBytes = 2 * kBigQueue * sizeof(long long) + 4 * sizeof(unsigned int);
+constexpr size_t kBfsScratchBytes = 4 * kBigQueue * sizeof(long long) + 4 * sizeof(unsigned int);
+
+// One sweep (both kernels) and its update count.
+template <class Mem, class Op, bool WEIGHTED>
+int graph_sweep(const Mem &m, const Op &op, size_t off_off, size_t col_off, size_t w_off, size_t nv, void *scratch, int sweep,
+                unsigned int *updates, cudaStream_t s)
+{
+    long long *span_q = static_cast<long long *>(scratch);
+    unsigned int *counters = reinterpret_cast<unsigned int *>(span_q + 4 * kBigQueue);
+    const int grid = sm_count() * 2;
+    cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
+    graph_sweep_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, off_off, col_off, w_off, (unsigned int)nv, span_q, counters, sweep);
+    graph_span_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, col_off, w_off, span_q, counters);
+    int rc = launched(2);
+    unsigned int host_counters[2] = {0, 0};
+    if (cudaMemcpyAsync(host_counters, counters, sizeof(host_counters), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+    *updates = host_counters[0];
+    return rc;
+}
 
 // One BFS on caller-provided scratch (kBfsScratchBytes, 16-byte aligned).
 template <class Mem>
 int bfs_levels(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
                void *scratch, cudaStream_t s)
 {
-    long long *span_q = static_cast<long long *>(scratch);
-    unsigned int *counters = reinterpret_cast<unsigned int *>(span_q + 2 * kBigQueue);
     cudaMemsetAsync(d_level, 0xFF, nv * sizeof(int32_t), s);
     bfs_init_kernel<<<1, 1, 0, s>>>(d_level, (int)source);
     int rc = launched();
     int depth = 0;
-    const int grid = sm_count() * 2;
     unsigned int found = 1;
     while (rc == GPUVM_OK && found > 0) {
-        cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
-        bfs_sweep_kernel<Mem><<<grid, 256, 0, s>>>(m, off_off, col_off, d_level, (unsigned int)nv, span_q, counters, depth);
-        bfs_span_kernel<Mem><<<grid, 256, 0, s>>>(m, col_off, d_level, span_q, counters, depth);
-        rc = launched(2);
-        unsigned int host_counters[2] = {0, 0};
-        if (cudaMemcpyAsync(host_counters, counters, sizeof(host_counters), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-            cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); rc = GPUVM_E_CUDA; break; }
-        found = host_counters[0];
+        rc = graph_sweep<Mem, BfsOp, false>(m, BfsOp{d_level, depth}, off_off, col_off, 0, nv, scratch, depth, &found, s);
         ++depth;
     }
     if (n_levels) *n_levels = depth;
@@ -694,6 +769,59 @@ int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t sour
     int rc = bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, s);
     cudaStreamSynchronize(s);
     cudaFree(scratch);
+    return rc;
+}
+
+struct Scratch {                     // device scratch for one call, freed on scope exit
+    void *p = nullptr;
+    explicit Scratch(size_t bytes) { if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); p = nullptr; } }
+    ~Scratch() { if (p) cudaFree(p); }
+};
+
+template <class Mem>
+int run_cc(const Mem &m, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, cudaStream_t s)
+{
+    if (!d_label || nv == 0 || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
+    if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
+    Scratch scratch(kBfsScratchBytes);
+    if (!scratch.p) return GPUVM_E_ALLOC;
+    cc_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
+    int rc = launched();
+    int sweep = 0;
+    unsigned int updates = 1;
+    while (rc == GPUVM_OK && updates > 0) {
+        rc = graph_sweep<Mem, CcOp, false>(m, CcOp{d_label}, off_off, col_off, 0, nv, scratch.p, sweep, &updates, s);
+        ++sweep;
+    }
+    cudaStreamSynchronize(s);
+    if (n_sweeps) *n_sweeps = sweep;
+    return rc;
+}
+
+template <class Mem>
+int run_sssp(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source, int32_t *d_dist,
+             int *n_rounds, cudaStream_t s)
+{
+    if (!d_dist || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
+    if (off_off % 16 || col_off % 16 || w_off % 16) return GPUVM_E_ALIGN;
+    if ((w_off > col_off ? w_off - col_off : col_off - w_off) % m.unit_host() != 0) return GPUVM_E_ALIGN;
+    Scratch scratch(kBfsScratchBytes + 2 * nv);
+    if (!scratch.p) return GPUVM_E_ALLOC;
+    unsigned char *flags = static_cast<unsigned char *>(scratch.p) + kBfsScratchBytes;
+    unsigned char *cur = flags, *next = flags + nv;
+    sssp_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_dist, cur, (unsigned int)nv, (unsigned int)source);
+    int rc = launched();
+    int round = 0;
+    unsigned int updates = 1;
+    while (rc == GPUVM_OK && updates > 0) {
+        cudaMemsetAsync(next, 0, nv, s);
+        rc = graph_sweep<Mem, SsspOp, true>(m, SsspOp{d_dist, cur, next}, off_off, col_off, w_off, nv, scratch.p, round,
+                                            &updates, s);
+        unsigned char *t = cur; cur = next; next = t;
+        ++round;
+    }
+    cudaStreamSynchronize(s);
+    if (n_rounds) *n_rounds = round;
     return rc;
 }
 
@@ -824,6 +952,23 @@ int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, 
     return bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, static_cast<cudaStream_t>(stream));
 }
 
+int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_cc(m, off_off, col_off, nv, d_label, n_sweeps, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source, int32_t *d_dist,
+                   int *n_rounds, void *stream)
+{
+    PagedH m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    // column and weight page of an edge range are held together: two frames per warp of the grid
+    if (gpuvm_safe_warps(h, 2) < sm_count() * 2 * 8) return GPUVM_E_POOL;
+    return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, static_cast<cudaStream_t>(stream));
+}
+
 int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n, void *stream)
 {
     PagedH m;
@@ -926,6 +1071,32 @@ int gpuvm_raw_bfs_csr(const int64_t *row_off, const int32_t *col, size_t nv, siz
     if ((ro - base) % 16 || (co - base) % 16) return GPUVM_E_ALIGN;
     Raw m{base, 65536};
     return run_bfs(m, (size_t)(ro - base), (size_t)(co - base), nv, source, d_level, n_levels, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_raw_cc_csr(const int64_t *row_off, const int32_t *col, size_t nv, int32_t *d_label, int *n_sweeps, void *stream)
+{
+    if (!row_off || !col) return GPUVM_E_ARG;
+    unsigned char *ro = reinterpret_cast<unsigned char *>(const_cast<int64_t *>(row_off));
+    unsigned char *co = reinterpret_cast<unsigned char *>(const_cast<int32_t *>(col));
+    unsigned char *base = ro < co ? ro : co;
+    if ((ro - base) % 16 || (co - base) % 16) return GPUVM_E_ALIGN;
+    Raw m{base, 65536};
+    return run_cc(m, (size_t)(ro - base), (size_t)(co - base), nv, d_label, n_sweeps, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_raw_sssp_csr(const int64_t *row_off, const int32_t *col, const int32_t *weight, size_t nv, size_t source,
+                       int32_t *d_dist, int *n_rounds, void *stream)
+{
+    if (!row_off || !col || !weight) return GPUVM_E_ARG;
+    unsigned char *ro = reinterpret_cast<unsigned char *>(const_cast<int64_t *>(row_off));
+    unsigned char *co = reinterpret_cast<unsigned char *>(const_cast<int32_t *>(col));
+    unsigned char *we = reinterpret_cast<unsigned char *>(const_cast<int32_t *>(weight));
+    unsigned char *base = ro < co ? (ro < we ? ro : we) : (co < we ? co : we);
+    RawH m;
+    m.base = base;
+    m.unit_bytes = 65536;
+    return run_sssp(m, (size_t)(ro - base), (size_t)(co - base), (size_t)(we - base), nv, source, d_dist, n_rounds,
+                    static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void *stream)

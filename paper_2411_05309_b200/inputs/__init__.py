@@ -53,6 +53,8 @@ def _load():
         lib.gvi_fill_i32_u20.argtypes = [vp, u64, u64, u64]
         lib.gvi_fill_f32_pm1.argtypes = [vp, u64, u64, u64]
         lib.gvi_fill_index_i64.argtypes = [vp, u64, u64, u64, u64]
+        lib.gvi_fill_i32_range.argtypes = [vp, u64, u64, u64, ctypes.c_int32, ctypes.c_uint32]
+        lib.gvi_fill_i32_range.restype = None
         lib.gvi_rmat_csr.restype = ctypes.c_int
         lib.gvi_rmat_csr.argtypes = [ctypes.c_int, u64, u64, ctypes.c_uint32, ctypes.c_uint32,
                                      ctypes.c_uint32, vp, vp]
@@ -83,6 +85,12 @@ def fill_i32_u20(dst, n: int, seed: int, first: int = 0):
 
 def fill_f32_pm1(dst, n: int, seed: int, first: int = 0):
     _load().gvi_fill_f32_pm1(_addr(dst, np.float32, n), first, n, seed)
+    return dst
+
+
+def fill_i32_range(dst, n: int, seed: int, lo: int, span: int, first: int = 0):
+    """int32 values uniform in [lo, lo + span): synthetic edge weights."""
+    _load().gvi_fill_i32_range(_addr(dst, np.int32, n), first, n, seed, lo, span)
     return dst
 
 

@@ -47,6 +47,14 @@ void gvi_fill_f32_pm1(float *dst, uint64_t first, uint64_t n, uint64_t seed)
     }
 }
 
+/* int32 values uniform in [lo, lo + span): edge weights. */
+void gvi_fill_i32_range(int32_t *dst, uint64_t first, uint64_t n, uint64_t seed, int32_t lo, uint32_t span)
+{
+#pragma omp parallel for schedule(static)
+    for (uint64_t k = 0; k < n; ++k)
+        dst[k] = lo + (int32_t)(mix64(seed, first + k) % span);
+}
+
 /* int64 indices uniform in [0, modulo). */
 void gvi_fill_index_i64(int64_t *dst, uint64_t first, uint64_t n, uint64_t seed,
                         uint64_t modulo)

@@ -26,7 +26,7 @@ SLACK = 16 << 20          # device memory left to the driver on top of the pool
 
 # Extra size reduction (log2) of the twin per configuration: UVM thrashes badly on the
 # write-back and Zipf workloads, and a running kernel cannot be stopped from the host.
-TWIN_SHRINK = {1: 0, 2: 0, 3: 0, 4: 3, 5: 3}
+TWIN_SHRINK = {1: 0, 2: 0, 3: 0, 4: 3, 5: 3, 6: 0, 7: 0}
 
 
 def _timed(torch, fn):
@@ -83,7 +83,7 @@ def _outputs(torch, w, cfg: int) -> dict:
         nb = (w.n_idx + w.block - 1) // w.block
         return {"fs": torch.zeros(nb, dtype=torch.float32, device="cuda"),
                 "bs": torch.zeros(nb, dtype=torch.int64, device="cuda")}
-    if cfg == 3:
+    if cfg in (3, 6, 7):
         return {"lvl": torch.zeros(w.nv, dtype=torch.int32, device="cuda")}
     if cfg == 5:
         return {"out": torch.zeros(w.n_bags * w.dims, dtype=torch.float32, device="cuda")}
@@ -129,6 +129,18 @@ def _one_inner(torch, w, cfg: int, p: int, budget_s: float, bufs: dict, cold) ->
         t = _timed(torch, lambda: B.gpuvm_raw_bfs_csr(p + w.off["off"], p + w.off["col"], w.nv, 0, lvl))
         return {"seconds": t, "effective_gbs": w.effective_bytes() / t / 1e9,
                 "matches_paged_result": bool(torch.equal(lvl, w.d_level)), "scaled": False}
+    if cfg == 6:
+        lab = bufs["lvl"]
+        cold()
+        t = _timed(torch, lambda: B.gpuvm_raw_cc_csr(p + w.off["off"], p + w.off["col"], w.nv, lab))
+        return {"seconds": t, "effective_gbs": w.effective_bytes() / t / 1e9,
+                "matches_paged_result": bool(torch.equal(lab, w.d_level)), "scaled": False}
+    if cfg == 7:
+        dist = bufs["lvl"]
+        cold()
+        t = _timed(torch, lambda: B.gpuvm_raw_sssp_csr(p + w.off["off"], p + w.off["col"], p + w.off["w"], w.nv, 0, dist))
+        return {"seconds": t, "effective_gbs": w.effective_bytes() / t / 1e9,
+                "matches_paged_result": bool(torch.equal(dist, w.d_dist)), "scaled": False}
     if cfg == 4:
         cold()
         t = _timed(torch, lambda: B.gpuvm_raw_vadd_f32(p + w.off["a"], p + w.off["b"], p + w.off["c"], w.n))

@@ -65,6 +65,32 @@ def test_cfg3_bfs_rmat24():
         w.close()
 
 
+def test_cc_and_sssp_on_the_cfg3_graph():
+    """The two further graph workloads of the paper's evaluation on the same RMAT graph."""
+    w, res = run(6)
+    try:
+        off, col = w.view("off", np.int64, w.nv + 1), w.view("col", np.int32, w.ne)
+        ref = oracle.cc_labels_direct(off, col)
+        assert np.array_equal(w.d_level.cpu().numpy(), ref)
+        assert ref[0] == 0 and np.all(ref <= np.arange(w.nv))
+    finally:
+        w.close()
+    w, res = run(7)
+    try:
+        off, col, wt = w.view("off", np.int64, w.nv + 1), w.view("col", np.int32, w.ne), w.view("w", np.int32, w.ne)
+        assert wt.min() >= 1 and wt.max() <= 255
+        ref = oracle.sssp_direct(off, col, wt, 0)
+        got = w.d_dist.cpu().numpy()
+        assert np.array_equal(got, ref)
+        # certificate: no edge out of a reached vertex can still be relaxed
+        src = np.repeat(np.arange(w.nv, dtype=np.int64), np.diff(off))[: 1 << 24]
+        e = np.arange(src.size)
+        ok = got[src] != 0x7FFFFFFF
+        assert np.all(got[col[e]][ok].astype(np.int64) <= got[src][ok].astype(np.int64) + wt[e][ok])
+    finally:
+        w.close()
+
+
 def test_cfg4_vector_add_12GiB():
     w, res = run(4)
     try:

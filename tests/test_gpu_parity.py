@@ -207,6 +207,65 @@ def test_bfs_rmat_with_hub_vertices(B, scale, page, frames):
     assert st["writebacks"] == 0
 
 
+def graph_arena(page, off, col, weight=None):
+    off_p = np.zeros((off.size + 1) // 2 * 2, np.int64)
+    off_p[:off.size] = off
+    pad4 = lambda a: np.concatenate([a, np.zeros((-a.size) % 4, a.dtype)])
+    arrays = {"off": off_p, "col": pad4(col)}
+    if weight is not None:
+        arrays["w"] = pad4(weight)
+    return Arena(page, arrays)
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+def test_cc_small_graphs_and_rmat(B, policy):
+    import torch
+    cases = [(nv, edges) for nv, edges, _ in small_graphs()]
+    graphs = [csr(nv, edges) for nv, edges in cases]
+    graphs.append(inputs.rmat_csr(12, 4 << 12, inputs.config_seed(3)))      # sparse: many components
+    graphs.append(inputs.rmat_csr(14, 16 << 14, inputs.config_seed(3)))     # hub vertices: long lists are split
+    for off, col in graphs:
+        nv = off.size - 1
+        ref = oracle.cc_labels_direct(off, col[:max(int(off[-1]), 0)] if off[-1] else col)
+        for page, frames in ((64, 1), (4096, 6), (65536, 3)):
+            ar = graph_arena(page, off, col)
+            label = torch.zeros(nv, dtype=torch.int32, device="cuda")
+            with paged(ar.host, page, frames, policy) as h:
+                sweeps = B.gpuvm_cc_csr(h, ar.off["off"], ar.off["col"], nv, label)
+                st, ck = finish(h)
+            assert np.array_equal(label.cpu().numpy(), ref)
+            assert sweeps >= 1 and st["writebacks"] == 0
+
+
+@pytest.mark.parametrize("policy", POLICIES)
+def test_sssp_small_graphs_and_rmat(B, policy):
+    import torch
+    graphs = [csr(nv, edges) + (src,) for nv, edges, src in small_graphs()]
+    graphs.append(inputs.rmat_csr(12, 8 << 12, inputs.config_seed(3)) + (0,))
+    graphs.append(inputs.rmat_csr(14, 16 << 14, inputs.config_seed(3)) + (0,))
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    need = 2 * sms * 2 * 8                                   # two frames per warp of the grid
+    for off, col, src in graphs:
+        nv = off.size - 1
+        weight = inputs.fill_i32_range(np.empty(col.size, np.int32), col.size, inputs.config_seed(3, 2), 1, 255)
+        ref = oracle.sssp_direct(off, col, weight, src)
+        for page in (64, 4096):
+            ar = graph_arena(page, off, col, weight)
+            dist = torch.zeros(nv, dtype=torch.int32, device="cuda")
+            with paged(ar.host, page, need + 3, policy) as h:
+                rounds = B.gpuvm_sssp_csr(h, ar.off["off"], ar.off["col"], ar.off["w"], nv, src, dist)
+                st, ck = finish(h)
+            assert np.array_equal(dist.cpu().numpy(), ref)
+            assert rounds >= 1
+    # a pool that cannot hold two pages per warp is refused, nothing runs
+    ar = graph_arena(4096, *graphs[1][:2], np.ones(graphs[1][1].size, np.int32))
+    with paged(ar.host, 4096, 8) as h:
+        with pytest.raises(B.GpuvmError) as e:
+            B.gpuvm_sssp_csr(h, ar.off["off"], ar.off["col"], ar.off["w"], graphs[1][0].size - 1, 0,
+                             torch.zeros(8, dtype=torch.int32, device="cuda"))
+        assert e.value.status == B.E_POOL
+
+
 @pytest.mark.parametrize("page,n_rows,n_bags,frames,dims,bag", [
     (4096, 512, 64, 64, 128, 32),
     (4096, 4096, 1000, 8, 128, 32),

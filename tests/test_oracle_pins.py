@@ -373,3 +373,70 @@ def test_uniform_independent_reference_hit_ratio():
         c = pg.counters()
         assert abs(c["faults"] / n - (1 - F / P)) < 0.01
         pg.close()
+
+
+def test_cc_against_scipy_and_brute_force():
+    from scipy.sparse import csr_matrix
+    from scipy.sparse.csgraph import connected_components
+    rng = np.random.default_rng(31)
+    cases = [(1, []), (4, []), (5, [(0, 0), (3, 1), (1, 3), (4, 2)]), (6, [(5, 0), (4, 5), (1, 2)])]
+    for _ in range(30):
+        nv = int(rng.integers(2, 30))
+        cases.append((nv, [(int(rng.integers(0, nv)), int(rng.integers(0, nv))) for _ in range(int(rng.integers(0, 30)))]))
+    for nv, edges in cases:
+        off, col = csr_from_edges(nv, edges)
+        got = oracle.cc_labels_direct(off, col)
+        # brute force: repeat "every edge pulls both ends to the smaller label" until nothing changes
+        lab = list(range(nv))
+        changed = True
+        while changed:
+            changed = False
+            for u, v in edges:
+                m = min(lab[u], lab[v])
+                if lab[u] != m or lab[v] != m:
+                    lab[u] = lab[v] = m
+                    changed = True
+        assert list(got) == lab
+        if edges:
+            m = csr_matrix((np.ones(len(edges)), ([e[0] for e in edges], [e[1] for e in edges])), shape=(nv, nv))
+            n_comp, part = connected_components(m, directed=True, connection="weak")
+            assert len(set(got)) == n_comp
+            for c in range(n_comp):                       # same partition, labelled by its smallest member
+                members = np.nonzero(part == c)[0]
+                assert set(got[members]) == {members.min()}
+
+
+def test_sssp_against_bellman_ford_and_scipy():
+    from scipy.sparse import csr_matrix
+    from scipy.sparse.csgraph import dijkstra
+    rng = np.random.default_rng(47)
+    INF = 0x7FFFFFFF
+    cases = [(1, [], 0), (3, [(0, 1, 5), (0, 1, 2), (1, 2, 0), (2, 2, 1)], 0), (4, [(1, 0, 3)], 0)]
+    for _ in range(30):
+        nv = int(rng.integers(2, 25))
+        ne = int(rng.integers(0, 60))
+        cases.append((nv, [(int(rng.integers(0, nv)), int(rng.integers(0, nv)), int(rng.integers(0, 300))) for _ in range(ne)],
+                      int(rng.integers(0, nv))))
+    for nv, wedges, src in cases:
+        off, col = csr_from_edges(nv, [(u, v) for u, v, _ in wedges])
+        w = np.zeros(col.size, dtype=np.int32)
+        cur = off[:-1].copy()
+        for u, v, ww in wedges:                           # same stable placement as csr_from_edges
+            w[cur[u]] = ww
+            cur[u] += 1
+        got = oracle.sssp_direct(off, col, w, src)
+        d = [INF] * nv
+        d[src] = 0
+        for _ in range(nv):                                # Bellman-Ford, V rounds over all edges
+            for u, v, ww in wedges:
+                if d[u] != INF and d[u] + ww < d[v]:
+                    d[v] = d[u] + ww
+        assert list(got) == d
+        best = {}
+        for u, v, ww in wedges:                            # scipy sums duplicate entries: keep the lightest edge
+            best[(u, v)] = min(ww, best.get((u, v), 1 << 40))
+        pos = {k: x for k, x in best.items() if x > 0 and k[0] != k[1]}
+        if pos and all(x > 0 for x in best.values()):
+            m = csr_matrix((list(pos.values()), ([k[0] for k in pos], [k[1] for k in pos])), shape=(nv, nv))
+            sp = dijkstra(m, directed=True, indices=src)
+            assert list(got) == [int(x) if np.isfinite(x) else INF for x in sp]
