@@ -10,6 +10,7 @@
  *   void* gpuvm_ptr(vm, byte_off, mode, &token)                pin and hand out a frame pointer
  *   void  gpuvm_release(vm, token)                             unpin what gpuvm_ptr pinned
  *   void  gpuvm_clean(vm, token, p)                            write a pinned page back now (eager write-back)
+ *   void  gpuvm_prefetch(vm, byte_off)                         fetch a page ahead of its use, unpinned
  *
  * What happens on an access (Section 3.1, Fig. 2; Section 3.3):
  *   1. address split: page number = byte offset >> page_shift, offset = the rest;
@@ -605,6 +606,63 @@ __device__ __forceinline__ void gpuvm_clean(const gpuvm_dev_t &vm, const gpuvm_t
     if (token.leader) {
         gpuvm::stat_add(vm, gpuvm::kWritebacks, 1);
         gpuvm::stat_add(vm, gpuvm::kBytesOut, len);
+    }
+}
+
+/*
+ * Prefetch: if the page that holds `byte_off` is neither resident nor being fetched, the
+ * calling lanes (which must all pass the same offset) fetch it now and leave it resident,
+ * unpinned, with its reference bit set; otherwise they return at once.  Used by sweeps to
+ * fetch pages ahead of the window in which all warps work: without it every warp of the
+ * window waits for the same few pages and only those few are in flight on the link.  Gives
+ * up quietly (page left INVALID) when no frame is free after a few ring slots.
+ */
+static __device__ __noinline__ void gpuvm_prefetch(const gpuvm_dev_t vm, unsigned long long byte_off)
+{
+    using namespace gpuvm;
+    if (byte_off >= vm.bytes) return;
+    const unsigned long long vpn = byte_off >> vm.page_shift;
+    const unsigned int active = __activemask();
+    const unsigned int lane = lane_id(), L = __ffs(active) - 1;
+    const unsigned int rank = __popc(active & ((1u << lane) - 1u)), n = __popc(active);
+    unsigned long long *pte = vm.pte + vpn;
+    int go = 0;
+    unsigned int h = 0;
+    unsigned long long victim = ~0ull;
+    bool vdirty = false;
+    if (lane == L) {
+        const unsigned long long w = ld_relaxed_u64(pte);
+        if ((w & kStMask) == kInvalid && atomicCAS(pte, w, w | kBusy) == w) {
+            go = try_claim(vm, vpn, 8, h, victim, vdirty) ? 1 : 0;
+            if (!go) atomicXor(pte, kBusy);                       /* no frame at hand: BUSY -> INVALID */
+        }
+    }
+    if (!__shfl_sync(active, go, L)) return;
+    const unsigned int bh = __shfl_sync(active, h, L);
+    const unsigned long long bq = __shfl_sync(active, victim, L);
+    const int bd = __shfl_sync(active, (int)vdirty, L);
+    unsigned char *fr = vm.pool + ((unsigned long long)bh << vm.page_shift);
+    if (bq != ~0ull) {
+        if (bd) {
+            warp_copy<8, true>(vm.host + (bq << vm.page_shift), fr, page_len(vm, bq) >> 4, rank, n);
+            __threadfence_system();
+            __syncwarp(active);
+        }
+        if (lane == L) {
+            atomicXor(vm.pte + bq, kEvicting | ((unsigned long long)bh << kFrameShift) | (bd ? kDirty : 0ull));
+            stat_add(vm, kEvictions, 1);
+            if (bd) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, bq)); }
+        }
+    }
+    warp_copy<8, false>(fr, vm.host + (vpn << vm.page_shift), page_len(vm, vpn) >> 4, rank, n);
+    __threadfence();
+    __syncwarp(active);
+    if (lane == L) {
+        st_relaxed_u32(vm.frame_vpn + bh, (unsigned int)vpn);
+        atomicXor(pte, (kBusy ^ kValid) | ((unsigned long long)bh << kFrameShift) |
+                           (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull));
+        stat_add(vm, kFaults, 1);
+        stat_add(vm, kBytesIn, page_len(vm, vpn));
     }
 }
 

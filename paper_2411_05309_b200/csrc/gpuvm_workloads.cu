@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <cstdint>
+#include <cstring>
 
 #include "gpuvm.h"
 #include "gpuvm_batch.cuh"
@@ -18,6 +19,7 @@ std::atomic<unsigned long long> g_launches{0};
 
 struct Paged {
     gpuvm_dev_t vm;
+    unsigned long long edges_hint = 0;
     __device__ __forceinline__ unsigned long long unit() const { return 1ull << vm.page_shift; }
     template <typename T>
     __device__ __forceinline__ T read(unsigned long long base, unsigned long long i) const { return gpuvm_read<T>(vm, i, base); }
@@ -29,6 +31,7 @@ struct Paged {
     }
     __device__ __forceinline__ void release(const gpuvm_token &t) const { gpuvm_release(vm, t); }
     __device__ __forceinline__ void clean(const gpuvm_token &t, const void *p) const { gpuvm_clean(vm, t, p); }
+    __device__ __forceinline__ void prefetch(unsigned long long off) const { gpuvm_prefetch(vm, off); }
     static __device__ __forceinline__ uint4 load16(const void *p) { return gpuvm_load16(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { gpuvm_store16(p, v); }
     static __device__ __forceinline__ int load_i32(const void *p) { return gpuvm_load(static_cast<const int *>(p)); }
@@ -37,6 +40,7 @@ struct Paged {
 struct Raw {
     unsigned char *base;
     unsigned long long unit_bytes;
+    unsigned long long edges_hint = 0;
     __device__ __forceinline__ unsigned long long unit() const { return unit_bytes; }
     template <typename T>
     __device__ __forceinline__ T read(unsigned long long off, unsigned long long i) const { return reinterpret_cast<const T *>(base + off)[i]; }
@@ -45,6 +49,7 @@ struct Raw {
     __device__ __forceinline__ unsigned char *pin(unsigned long long off, int, gpuvm_token &) const { return base + off; }
     __device__ __forceinline__ void release(const gpuvm_token &) const {}
     __device__ __forceinline__ void clean(const gpuvm_token &, const void *) const {}
+    __device__ __forceinline__ void prefetch(unsigned long long) const {}
     static __device__ __forceinline__ uint4 load16(const void *p) { return *static_cast<const uint4 *>(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { *static_cast<uint4 *>(p) = v; }
     static __device__ __forceinline__ int load_i32(const void *p) { return *static_cast<const int *>(p); }
@@ -213,6 +218,7 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
 // ------------------------------------------------------- graph sweeps (BFS, CC, SSSP)
 constexpr long long kBigDegree = 4096;     // neighbour lists at least this long are spread over the grid
 constexpr unsigned int kBigQueue = 65536;  // entries of the span queue (four int64 each: first edge, end, vertex, -)
+constexpr long long kAhead = 16;           // pages of look-ahead of the sweeps' prefetches
 
 // counters: [0] updates made in this sweep, [1] span queue size, [2] chunk ticket, [3] span ticket
 
@@ -281,8 +287,8 @@ __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned
 template <class Mem, class Op, bool WEIGHTED>
 __global__ void __launch_bounds__(256) graph_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
                                                           unsigned long long w_off, unsigned int nv,
-                                                          long long *__restrict__ span_q, unsigned int *__restrict__ counters,
-                                                          int sweep)
+                                                          unsigned long long n_edges, long long *__restrict__ span_q,
+                                                          unsigned int *__restrict__ counters, int sweep)
 {
     const unsigned int lane = threadIdx.x & 31;
     const unsigned long long unit = m.unit();
@@ -297,6 +303,13 @@ __global__ void __launch_bounds__(256) graph_sweep_kernel(Mem m, Op op, unsigned
         const unsigned long long v = v0 + lane;
         const bool active = v < nv && op.active(v);
         if (!__any_sync(0xFFFFFFFFu, active)) continue;
+        // fetch the row-offset page the sweep will reach kAhead pages from now (one warp wins the
+        // page, the others return at once), so that the window does not stall on one page at a time
+        const bool dense = __popc(__ballot_sync(0xFFFFFFFFu, active)) >= 8;   // a sparse frontier may never get there
+        if (dense) {
+            const long long ahead = (long long)(off_off + 8ull * v0) + ((sweep & 1) ? -kAhead : kAhead) * (long long)unit;
+            if (ahead >= (long long)off_off && ahead < (long long)(off_off + 8ull * nv)) m.prefetch((unsigned long long)ahead);
+        }
         // row offsets of the chunk: off[v0 .. v0+32], clamped to the nv + 1 entries that exist
         long long lo = m.template read<long long>(off_off, v < nv ? v : nv);
         long long hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
@@ -332,6 +345,14 @@ __global__ void __launch_bounds__(256) graph_sweep_kernel(Mem m, Op op, unsigned
             const long long a = __shfl_xor_sync(0xFFFFFFFFu, rlo, o), b = __shfl_xor_sync(0xFFFFFFFFu, rhi, o);
             rlo = a < rlo ? a : rlo;
             rhi = b > rhi ? b : rhi;
+        }
+        if (dense && rhi > rlo) {                        // and the column page the sweep will reach
+            const long long ahead = (long long)(col_off + 4ull * ((sweep & 1) ? rlo : rhi)) +
+                                    ((sweep & 1) ? -kAhead : kAhead) * (long long)unit;
+            if (ahead >= (long long)col_off && ahead < (long long)(col_off + 4ull * n_edges)) {
+                m.prefetch((unsigned long long)ahead);
+                if (WEIGHTED) m.prefetch((unsigned long long)ahead - col_off + w_off);
+            }
         }
         long long first = rlo;
         while (first < rhi) {
@@ -691,6 +712,17 @@ int launched(unsigned long long n = 1)
 
 bool view_of(gpuvm_t h, Paged &m) { return h && gpuvm_device_view(h, &m.vm) == GPUVM_OK; }
 
+// The number of edges is the last row offset; it is read from the backing store on the host
+// (row offsets are never written) and only bounds the sweeps' prefetches.
+void hint_edges(gpuvm_t h, Paged &m, size_t off_off, size_t nv)
+{
+    const unsigned char *host = static_cast<const unsigned char *>(gpuvm_host_ptr(h));
+    if (!host || off_off + 8 * (nv + 1) > m.vm.bytes) return;
+    long long ne = 0;
+    memcpy(&ne, host + off_off + 8 * nv, sizeof(ne));
+    if (ne > 0) m.edges_hint = (unsigned long long)ne;
+}
+
 template <class Mem>
 int run_stream_sum(const Mem &m, size_t a_off, size_t n, int64_t *d_sum, cudaStream_t s)
 {
@@ -726,11 +758,13 @@ template <class Mem, class Op, bool WEIGHTED>
 int graph_sweep(const Mem &m, const Op &op, size_t off_off, size_t col_off, size_t w_off, size_t nv, void *scratch, int sweep,
                 unsigned int *updates, cudaStream_t s)
 {
+    // number of edges = last row offset; only used to keep prefetches inside the column array
+    const unsigned long long n_edges = m.edges_hint;
     long long *span_q = static_cast<long long *>(scratch);
     unsigned int *counters = reinterpret_cast<unsigned int *>(span_q + 4 * kBigQueue);
     const int grid = sm_count() * 2;
     cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
-    graph_sweep_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, off_off, col_off, w_off, (unsigned int)nv, span_q, counters, sweep);
+    graph_sweep_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, off_off, col_off, w_off, (unsigned int)nv, n_edges, span_q, counters, sweep);
     graph_span_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, col_off, w_off, span_q, counters);
     int rc = launched(2);
     unsigned int host_counters[2] = {0, 0};
@@ -933,6 +967,7 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
 {
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
+    hint_edges(h, m, off_off, nv);
     return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, static_cast<cudaStream_t>(stream));
 }
 
@@ -947,6 +982,7 @@ int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, 
     void *scratch = nullptr;
     int rc = bfs_static_scratch(&scratch);
     if (rc != GPUVM_OK) return rc;
+    hint_edges(h, m, off_off, nv);
     // bfs_levels zeroes the counters at the start of every level and writes each queue entry
     // before reading it, so whatever the previous call left in the array does not matter
     return bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, static_cast<cudaStream_t>(stream));
@@ -956,6 +992,7 @@ int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *
 {
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
+    hint_edges(h, m, off_off, nv);
     return run_cc(m, off_off, col_off, nv, d_label, n_sweeps, static_cast<cudaStream_t>(stream));
 }
 
@@ -966,6 +1003,7 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
     if (!view_of(h, m)) return GPUVM_E_ARG;
     // column and weight page of an edge range are held together: two frames per warp of the grid
     if (gpuvm_safe_warps(h, 2) < sm_count() * 2 * 8) return GPUVM_E_POOL;
+    hint_edges(h, m, off_off, nv);
     return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, static_cast<cudaStream_t>(stream));
 }
 
