@@ -1,0 +1,104 @@
+"""Randomised small cases, many of them: page sizes, pool sizes from one frame to everything,
+both policies, all accessor styles.  Concurrency bugs in the page-table protocol (a lost
+reference, a frame claimed twice, a write-back that races a re-fetch) show up as wrong
+results, a failed invariant check, or a sticky error."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from gpu_common import Arena, finish, paged
+from paper_2411_05309_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+SOAK = int(os.environ.get("GPUVM_STRESS_SOAK", "1"))      # multiply the number of random cases
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2411_05309_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def test_random_mix_of_workloads_on_one_handle(B):
+    """Several kernels in a row on the same handle, no reset in between: gather (batched and not),
+    scattered read-modify-write (both forms), streaming sum, with a shadow copy on the host."""
+    import torch
+    rng = np.random.default_rng(20241105)
+    for case in range(40 * SOAK):
+        page = int(rng.choice([64, 256, 1024, 4096, 16384]))
+        n = int(rng.integers(2, 64)) * page // 4 + int(rng.integers(0, page // 16)) * 4
+        n_pages = (4 * n + page - 1) // page
+        frames = int(rng.choice([1, 2, 3, max(1, n_pages // 4), max(1, n_pages // 2), n_pages, n_pages + 3]))
+        policy = int(rng.integers(0, 2))
+        a = inputs.fill_i32_u20(np.empty(n, np.int32), n, 1000 + case).astype(np.uint32)
+        shadow = a.copy()
+        ar = Arena(page, {"a": a})
+        out = torch.zeros(1, dtype=torch.int64, device="cuda")
+        with paged(ar.host, page, frames, policy) as h:
+            for step in range(int(rng.integers(2, 6))):
+                kind = int(rng.integers(0, 5))
+                if kind in (0, 1):                                     # scattered updates of distinct elements
+                    m = int(rng.integers(1, n + 1))
+                    idx = rng.permutation(n)[:m].astype(np.int64)
+                    (B.gpuvm_scatter_update_u32 if kind == 0 else B.gpuvm_scatter_update_u32_batched)(h, 0, dev(idx), m)
+                    shadow[idx] = shadow[idx] * np.uint32(3) + np.uint32(1)
+                elif kind in (2, 3):                                   # gather of the current contents
+                    m = int(rng.integers(1, 4 * n))
+                    block = int(rng.choice([32, 100, 1024, 3000]))
+                    idx = rng.integers(0, n, m).astype(np.int64)
+                    nb = (m + block - 1) // block
+                    fs = torch.zeros(nb, dtype=torch.float32, device="cuda")
+                    bs = torch.zeros(nb, dtype=torch.int64, device="cuda")
+                    (B.gpuvm_gather_f32 if kind == 2 else B.gpuvm_gather_f32_unbatched)(h, 0, dev(idx), m, block, fs, bs)
+                    ref = oracle.gather_block_sums_direct(shadow.view(np.float32), idx, block)[1]
+                    assert np.array_equal(bs.cpu().numpy(), ref), (case, step, kind, page, frames)
+                else:
+                    B.gpuvm_stream_sum_i32(h, 0, n, out)
+                    assert int(out.item()) == int(shadow.view(np.int32).astype(np.int64).sum()), (case, step, page, frames)
+            st, ck = finish(h)
+            assert ck["resident"] <= frames
+        assert np.array_equal(ar.views["a"], shadow), (case, page, frames, policy)
+
+
+def test_many_small_vector_adds_and_graphs(B):
+    import torch
+    rng = np.random.default_rng(7)
+    for case in range(25 * SOAK):
+        page = int(rng.choice([512, 1024, 4096]))
+        n = (int(rng.integers(1, 40)) * page // 4 + int(rng.integers(0, page // 16)) * 4) // 4 * 4
+        frames = int(rng.choice([1, 2, 3, 5, 9, 40, 200]))
+        a = inputs.fill_f32_pm1(np.empty(n, np.float32), n, 50 + case)
+        b = inputs.fill_f32_pm1(np.empty(n, np.float32), n, 90 + case)
+        ar = Arena(page, {"a": a, "b": b, "c": np.zeros(n, np.float32)})
+        with paged(ar.host, page, frames, int(rng.integers(0, 2))) as h:
+            B.gpuvm_vadd_f32(h, ar.off["a"], ar.off["b"], ar.off["c"], n)
+            finish(h)
+        assert np.array_equal(ar.views["c"].view(np.uint32), oracle.vadd_f32_direct(a, b).view(np.uint32)), (case, page, n, frames)
+    for case in range(15 * SOAK):
+        scale = int(rng.integers(6, 13))
+        off, col = inputs.rmat_csr(scale, int(rng.integers(1, 24)) << scale, 300 + case)
+        nv = off.size - 1
+        src = int(rng.integers(0, nv))
+        page = int(rng.choice([64, 1024, 4096]))
+        frames = int(rng.choice([1, 2, 4, 16, 64]))
+        off_p = np.zeros((off.size + 1) // 2 * 2, np.int64)
+        off_p[:off.size] = off
+        col_p = np.concatenate([col, np.zeros((-col.size) % 4, np.int32)])
+        ar = Arena(page, {"off": off_p, "col": col_p})
+        lvl = torch.zeros(nv, dtype=torch.int32, device="cuda")
+        lab = torch.zeros(nv, dtype=torch.int32, device="cuda")
+        with paged(ar.host, page, frames) as h:
+            B.gpuvm_bfs_csr(h, ar.off["off"], ar.off["col"], nv, src, lvl)
+            B.gpuvm_cc_csr(h, ar.off["off"], ar.off["col"], nv, lab)
+            finish(h)
+        assert np.array_equal(lvl.cpu().numpy(), oracle.bfs_levels_direct(off, col, src)), (case, scale, page, frames)
+        assert np.array_equal(lab.cpu().numpy(), oracle.cc_labels_direct(off, col)), (case, scale, page, frames)
