@@ -43,6 +43,18 @@ def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0) -> dict:
     outputs and its time at that size), then the same kernels over managed memory."""
     import torch
     from . import configs
+    if cfg == 2:
+        # Not run any more.  Over managed memory under the balloon the random gather ended twice in
+        # an illegal-address fault (once with, once without read-mostly) after an earlier run of
+        # the same code had completed.  The kernel's accesses are in bounds by construction (indices
+        # are generated modulo the array length; the same kernel is clean on device memory and, for
+        # the other workloads, on managed memory), so the fault is attributed to fault servicing
+        # under extreme oversubscription and the combination is left alone instead of being probed.
+        return {"unavailable": "random gather over managed memory under the balloon raised illegal-address "
+                               "faults; not re-run",
+                "recorded_earlier_run": {"units_total": 1 << 26, "runs": [
+                    {"read_mostly": False, "units_run": 262144, "seconds": 10.269, "effective_gbs": 0.000102},
+                    {"read_mostly": True, "units_run": 1048576, "seconds": 25.785, "effective_gbs": 0.000163}]}}
     w = configs.make(cfg, shrink + TWIN_SHRINK[cfg])
     try:
         ours = w.run()
@@ -58,11 +70,7 @@ def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0) -> dict:
             balloon = B.gpuvm_balloon_alloc(w.pool_bytes + SLACK)
             out["free_bytes_under_balloon"] = B.gpuvm_mem_info()[0]
             read_only = cfg != 4
-            # cfg 2 is not run with read-mostly: under the balloon, the random gather over
-            # read-duplicated managed pages once ended in an illegal-address fault raised while the
-            # driver serviced it (the same kernel and arguments had just run without the advice);
-            # the combination is left alone rather than probed further
-            variants = [False] if cfg in (2, 4) else [False, True]
+            variants = [False] if cfg == 4 else [False, True]
             for advise in variants:
                 rec = {"read_mostly": advise}
                 rec.update(_one(torch, w, cfg, p, timeout_s / len(variants), bufs, advise))
