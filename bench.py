@@ -314,7 +314,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     w = configs.make(args.workload, args.shrink)
     for _ in range(args.warmup):
         w.run(check=False)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, args.clock_period)
     launches0 = B.gpuvm_launch_count()
     barrier()
     sampler.start()
@@ -377,6 +377,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "e2e": {"value": replica_throughput(world, eff_bytes, e2e_s) / 1e9, "unit": UNIT, "h2d_bytes_per_step": e2e[-1][1],
                 "d2h_bytes_per_step": e2e[-1][2], "ms_per_step": e2e_s * 1e3},
         "gpu_launches": launches, "clocks": clocks, "wall_s": wall,
+        "step_ms": [r.seconds * 1e3 for r in results],
+        "ms_median": statistics.median(r.seconds for r in results) * 1e3, "ms_min": min(r.seconds for r in results) * 1e3,
     }
     if not args.no_cpu_baseline:
         nbytes, dt, sample = oracle_step(args.workload, w if args.workload in (1, 2) else None, args.shrink)
@@ -403,6 +405,7 @@ def main():
     ap.add_argument("--uvm", action="store_true", help="also run the workload over cudaMallocManaged")
     ap.add_argument("--uvm-timeout", type=float, default=120.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--clock-period", type=float, default=0.5, help="seconds between NVML clock samples")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
