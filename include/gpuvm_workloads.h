@@ -12,9 +12,13 @@
  *   - calls enqueue work and return without synchronising unless stated; device
  *     errors (a wait that ran out, an offset out of range) are sticky in the handle
  *     and show up in gpuvm_stats().  Return value: 0 or a negative gpuvm_status.
- *   - nothing here allocates device memory except the graph workloads (2 MiB of
- *     scratch, plus 2 bytes per vertex for SSSP, freed before they return) and the first gpuvm_gather_f32 / gpuvm_embag_f32 on
- *     a handle (request tables and row staging, kept by the handle).
+ *   - device scratch (queues of the graph workloads, request tables of the gather, row
+ *     staging of the embedding bag) belongs to the handle: it is allocated the first
+ *     time a workload needs it, grown when a later call needs more, and freed by
+ *     gpuvm_destroy; calls that do not outgrow it allocate nothing (a per-call
+ *     cudaMalloc / cudaFree pair was measured to stall for 0.1-0.5 s now and then).
+ *     All workload calls on one handle share that scratch: do not let two of them
+ *     overlap on the GPU.  The gpuvm_raw_* twins allocate and free per call.
  */
 #ifndef GPUVM_WORKLOADS_H
 #define GPUVM_WORKLOADS_H
@@ -66,8 +70,8 @@ int gpuvm_gather_f32_unbatched(gpuvm_t h, size_t x_off, const int64_t *d_idx, si
  * one launch for very long neighbour lists, which are cut at page boundaries and
  * spread over the whole grid (the imbalance Section 5.2 describes).  Synchronises the
  * stream between levels; *n_levels (host pointer, may be NULL) receives the number
- * of levels expanded, counting the last one that discovers nothing.  Allocates and
- * frees 2 MiB of device scratch (queue of neighbour-list pieces, counters).
+ * of levels expanded, counting the last one that discovers nothing.  Uses 2 MiB of
+ * the handle's device scratch (queue of neighbour-list pieces, counters).
  */
 int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
                   int32_t *d_level, int *n_levels, void *stream);
@@ -79,7 +83,7 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
  * visits every edge (u, c) and lowers the larger of the two labels to the smaller
  * with atomicMin, until a sweep changes nothing.  Sweeps alternate direction like
  * the BFS levels.  *n_sweeps (host pointer, may be NULL) receives the number of
- * sweeps.  Allocates and frees 2 MiB of device scratch.  Synchronises per sweep.
+ * sweeps.  Uses 2 MiB of the handle's device scratch.  Synchronises per sweep.
  */
 int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps,
                  void *stream);
@@ -94,8 +98,8 @@ int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *
  * (GPUVM_E_POOL otherwise).  Bellman-Ford rounds over the vertices that changed in
  * the previous round; d_dist[v] receives the distance from `source`, 0x7FFFFFFF
  * where unreachable (path lengths must stay below that).  *n_rounds (host pointer,
- * may be NULL) receives the number of rounds.  Allocates and frees 2 MiB + 2 nv bytes
- * of device scratch.  Synchronises per round.
+ * may be NULL) receives the number of rounds.  Uses 2 MiB + 2 nv bytes of the
+ * handle's device scratch.  Synchronises per round.
  */
 int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source,
                    int32_t *d_dist, int *n_rounds, void *stream);

@@ -794,15 +794,13 @@ int bfs_levels(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t s
 
 template <class Mem>
 int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
-            cudaStream_t s)
+            void *scratch, cudaStream_t s)
 {
     if (!d_level || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
-    void *scratch = nullptr;                       // span queue + 4 counters
-    if (cudaMalloc(&scratch, kBfsScratchBytes) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_ALLOC; }
+    if (!scratch) return GPUVM_E_ALLOC;
     int rc = bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, s);
     cudaStreamSynchronize(s);
-    cudaFree(scratch);
     return rc;
 }
 
@@ -813,12 +811,13 @@ struct Scratch {                     // device scratch for one call, freed on sc
 };
 
 template <class Mem>
-int run_cc(const Mem &m, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, cudaStream_t s)
+int run_cc(const Mem &m, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, void *scratch_p,
+           cudaStream_t s)
 {
     if (!d_label || nv == 0 || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
-    Scratch scratch(kBfsScratchBytes);
-    if (!scratch.p) return GPUVM_E_ALLOC;
+    if (!scratch_p) return GPUVM_E_ALLOC;
+    struct { void *p; } scratch{scratch_p};
     cc_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
     int rc = launched();
     int sweep = 0;
@@ -834,13 +833,13 @@ int run_cc(const Mem &m, size_t off_off, size_t col_off, size_t nv, int32_t *d_l
 
 template <class Mem>
 int run_sssp(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source, int32_t *d_dist,
-             int *n_rounds, cudaStream_t s)
+             int *n_rounds, void *scratch_p, cudaStream_t s)
 {
     if (!d_dist || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16 || w_off % 16) return GPUVM_E_ALIGN;
     if ((w_off > col_off ? w_off - col_off : col_off - w_off) % m.unit_host() != 0) return GPUVM_E_ALIGN;
-    Scratch scratch(kBfsScratchBytes + 2 * nv);
-    if (!scratch.p) return GPUVM_E_ALLOC;
+    if (!scratch_p) return GPUVM_E_ALLOC;          // kBfsScratchBytes + 2 * nv bytes
+    struct { void *p; } scratch{scratch_p};
     unsigned char *flags = static_cast<unsigned char *>(scratch.p) + kBfsScratchBytes;
     unsigned char *cur = flags, *next = flags + nv;
     sssp_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_dist, cur, (unsigned int)nv, (unsigned int)source);
@@ -968,7 +967,8 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
     hint_edges(h, m, off_off, nv);
-    return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, static_cast<cudaStream_t>(stream));
+    return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, gpuvm_scratch_(h, kBfsScratchBytes),
+                   static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level,
@@ -993,7 +993,8 @@ int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
     hint_edges(h, m, off_off, nv);
-    return run_cc(m, off_off, col_off, nv, d_label, n_sweeps, static_cast<cudaStream_t>(stream));
+    return run_cc(m, off_off, col_off, nv, d_label, n_sweeps, gpuvm_scratch_(h, kBfsScratchBytes),
+                  static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source, int32_t *d_dist,
@@ -1004,7 +1005,8 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
     // column and weight page of an edge range are held together: two frames per warp of the grid
     if (gpuvm_safe_warps(h, 2) < sm_count() * 2 * 8) return GPUVM_E_POOL;
     hint_edges(h, m, off_off, nv);
-    return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, static_cast<cudaStream_t>(stream));
+    return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, gpuvm_scratch_(h, kBfsScratchBytes + 2 * nv),
+                    static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n, void *stream)
@@ -1108,7 +1110,9 @@ int gpuvm_raw_bfs_csr(const int64_t *row_off, const int32_t *col, size_t nv, siz
     unsigned char *base = ro < co ? ro : co;
     if ((ro - base) % 16 || (co - base) % 16) return GPUVM_E_ALIGN;
     Raw m{base, 65536};
-    return run_bfs(m, (size_t)(ro - base), (size_t)(co - base), nv, source, d_level, n_levels, static_cast<cudaStream_t>(stream));
+    Scratch scratch(kBfsScratchBytes);
+    return run_bfs(m, (size_t)(ro - base), (size_t)(co - base), nv, source, d_level, n_levels, scratch.p,
+                   static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_raw_cc_csr(const int64_t *row_off, const int32_t *col, size_t nv, int32_t *d_label, int *n_sweeps, void *stream)
@@ -1119,7 +1123,9 @@ int gpuvm_raw_cc_csr(const int64_t *row_off, const int32_t *col, size_t nv, int3
     unsigned char *base = ro < co ? ro : co;
     if ((ro - base) % 16 || (co - base) % 16) return GPUVM_E_ALIGN;
     Raw m{base, 65536};
-    return run_cc(m, (size_t)(ro - base), (size_t)(co - base), nv, d_label, n_sweeps, static_cast<cudaStream_t>(stream));
+    Scratch scratch(kBfsScratchBytes);
+    return run_cc(m, (size_t)(ro - base), (size_t)(co - base), nv, d_label, n_sweeps, scratch.p,
+                  static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_raw_sssp_csr(const int64_t *row_off, const int32_t *col, const int32_t *weight, size_t nv, size_t source,
@@ -1133,8 +1139,9 @@ int gpuvm_raw_sssp_csr(const int64_t *row_off, const int32_t *col, const int32_t
     RawH m;
     m.base = base;
     m.unit_bytes = 65536;
+    Scratch scratch(kBfsScratchBytes + 2 * nv);
     return run_sssp(m, (size_t)(ro - base), (size_t)(co - base), (size_t)(we - base), nv, source, d_dist, n_rounds,
-                    static_cast<cudaStream_t>(stream));
+                    scratch.p, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void *stream)
