@@ -188,6 +188,11 @@ int gpuvm_scatter_update_u32_batched(gpuvm_t h, size_t a_off, const int64_t *d_i
  */
 int gpuvm_touch_pages(gpuvm_t h, size_t first_page, size_t n_pages, int warps_per_sm, void *stream);
 
+/* The same with a given total number of warps (rounded up to whole thread blocks of at most 8
+ * warps, spread over the SMs): how many migrating warps the link needs (Section 3.2, Little's
+ * law; Section 5.2, sensitivity to the number of queues). */
+int gpuvm_touch_pages_warps(gpuvm_t h, size_t first_page, size_t n_pages, int total_warps, void *stream);
+
 /* ---- the same kernels on plain pointers (cudaMallocManaged or device memory) */
 int gpuvm_raw_stream_sum_i32(const int32_t *a, size_t n, int64_t *d_sum, void *stream);
 int gpuvm_raw_gather_f32(const float *x, const int64_t *d_idx, size_t n_idx, size_t block,

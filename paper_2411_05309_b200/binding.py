@@ -83,6 +83,7 @@ SYMBOLS = {
     "gpuvm_scatter_update_u32": (_i, [_vp, _sz, _vp, _sz, _vp]),
     "gpuvm_scatter_update_u32_batched": (_i, [_vp, _sz, _vp, _sz, _vp]),
     "gpuvm_touch_pages": (_i, [_vp, _sz, _sz, _i, _vp]),
+    "gpuvm_touch_pages_warps": (_i, [_vp, _sz, _sz, _i, _vp]),
     "gpuvm_raw_stream_sum_i32": (_i, [_vp, _sz, _vp, _vp]),
     "gpuvm_raw_gather_f32": (_i, [_vp, _vp, _sz, _sz, _vp, _vp, _vp]),
     "gpuvm_raw_bfs_csr": (_i, [_vp, _vp, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
@@ -312,6 +313,11 @@ def gpuvm_scatter_update_u32_batched(h, a_off: int, d_idx, n: int, stream=None):
 
 def gpuvm_touch_pages(h, first_page: int, n_pages: int, warps_per_sm: int, stream=None):
     _check(lib().gpuvm_touch_pages(h, first_page, n_pages, warps_per_sm, _stream(stream)), "gpuvm_touch_pages")
+
+
+def gpuvm_touch_pages_warps(h, first_page: int, n_pages: int, total_warps: int, stream=None):
+    _check(lib().gpuvm_touch_pages_warps(h, first_page, n_pages, total_warps, _stream(stream)),
+           "gpuvm_touch_pages_warps")
 
 
 def gpuvm_raw_stream_sum_i32(a, n: int, d_sum, stream=None):

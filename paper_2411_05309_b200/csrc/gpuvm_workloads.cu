@@ -1079,9 +1079,22 @@ int gpuvm_touch_pages(gpuvm_t h, size_t first_page, size_t n_pages, int warps_pe
     if (!view_of(h, m) || warps_per_sm <= 0 || warps_per_sm > 64) return GPUVM_E_ARG;
     if (first_page + n_pages > m.vm.n_pages) return GPUVM_E_RANGE;
     if (n_pages == 0) return GPUVM_OK;
-    int threads = warps_per_sm * 32 > 1024 ? 1024 : warps_per_sm * 32;
+    int threads = warps_per_sm * 32 > 256 ? 256 : warps_per_sm * 32;      // 128 registers per thread: 256-thread blocks
     int blocks_per_sm = (warps_per_sm * 32 + threads - 1) / threads;
     touch_pages_kernel<<<sm_count() * blocks_per_sm, threads, 0, static_cast<cudaStream_t>(stream)>>>(m.vm, first_page, n_pages);
+    return launched();
+}
+
+int gpuvm_touch_pages_warps(gpuvm_t h, size_t first_page, size_t n_pages, int total_warps, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m) || total_warps <= 0 || total_warps > 65536) return GPUVM_E_ARG;
+    if (first_page + n_pages > m.vm.n_pages) return GPUVM_E_RANGE;
+    if (n_pages == 0) return GPUVM_OK;
+    // spread the warps over the SMs: one-warp blocks up to the SM count, wider blocks beyond
+    const int per_block = (total_warps + sm_count() - 1) / sm_count() > 8 ? 8 : (total_warps + sm_count() - 1) / sm_count();
+    const int blocks = (total_warps + per_block - 1) / per_block;
+    touch_pages_kernel<<<blocks, per_block * 32, 0, static_cast<cudaStream_t>(stream)>>>(m.vm, first_page, n_pages);
     return launched();
 }
 

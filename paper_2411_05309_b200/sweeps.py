@@ -2,11 +2,16 @@
 oversubscription analysis), printed as JSON lines.
 
     python -m paper_2411_05309_b200.sweeps pages   [--gib 4] [--warps-per-sm 16]
+    python -m paper_2411_05309_b200.sweeps warps   [--gib 2]
     python -m paper_2411_05309_b200.sweeps oversub [--workload 1|2|3|4] [--shrink S]
 
 pages   -- Section 5.1 / Fig. 7: move a fixed amount of host memory into the pool with one
            warp per page, consecutive pages, for page sizes from 4 KiB to 2 MiB; reports the
            migration bandwidth against the pinned-copy peak measured in the same run.
+warps   -- Section 5.2 / Fig. 10 (sensitivity to the number of queue pairs): here the number of
+           warps that migrate pages at the same time, 1 .. 32 per SM, at 4 KiB and 64 KiB pages;
+           with Little's law (Section 3.2) the link saturates once warps x bytes in flight per
+           warp (4 KiB) reach bandwidth x latency.
 oversub -- Section 5.4 / Fig. 14 with Eq. 1: run a workload with the pool shrunk step by step,
            level = paged bytes / pool bytes - 1, under the clock policy and under FIFO (the
            paper's ring), reporting time relative to level 0.
@@ -58,6 +63,31 @@ def sweep_pages(gib: float, warps_per_sm: int):
             B.gpuvm_destroy(h)
 
 
+def sweep_warps(gib: float):
+    import torch
+    from . import binding as B
+    nbytes = int(gib * (1 << 30))
+    host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for page in (4096, 65536):
+        h = B.gpuvm_create(host.data_ptr(), nbytes, page, nbytes)
+        try:
+            for warps in (1, 2, 4, 8, 16, 32, 64, sms, 4 * sms, 32 * sms):
+                n_pages = min(nbytes // page, max(64, warps * (1 << 22) // page))     # a few MiB per warp
+                times = []
+                for r in range(3):
+                    B.gpuvm_reset(h)
+                    times.append(_time(torch, lambda: B.gpuvm_touch_pages_warps(h, 0, n_pages, warps)))
+                t = min(times[1:])
+                gbs = n_pages * page / t / 1e9
+                print(json.dumps({"sweep": "warps", "page_bytes": page, "migrating_warps": warps,
+                                  "bytes_in_flight": warps * 4096, "bytes": n_pages * page, "seconds": t,
+                                  "migration_gbs": gbs, "gbs_per_warp": gbs / warps,
+                                  "implied_latency_us": warps * 4096 / (gbs * 1e9) * 1e6}), flush=True)
+        finally:
+            B.gpuvm_destroy(h)
+
+
 def sweep_oversub(cfg: int, shrink: int):
     from . import binding as B
     from . import configs
@@ -86,7 +116,7 @@ def sweep_oversub(cfg: int, shrink: int):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("which", choices=["pages", "oversub"])
+    ap.add_argument("which", choices=["pages", "warps", "oversub"])
     ap.add_argument("--gib", type=float, default=4.0)
     ap.add_argument("--warps-per-sm", type=int, default=16)
     ap.add_argument("--workload", type=int, default=1)
@@ -94,6 +124,8 @@ def main(argv=None):
     a = ap.parse_args(argv)
     if a.which == "pages":
         sweep_pages(a.gib, a.warps_per_sm)
+    elif a.which == "warps":
+        sweep_warps(min(a.gib, 2.0))
     else:
         sweep_oversub(a.workload, a.shrink)
 
