@@ -296,6 +296,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     import torch
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the paged path has no CPU fallback")
+    local_rank %= max(1, torch.cuda.device_count())
     torch.cuda.set_device(local_rank)
     from paper_2411_05309_b200 import binding as B
     from paper_2411_05309_b200 import configs

@@ -584,8 +584,11 @@ __device__ __forceinline__ void gpuvm_release(const gpuvm_dev_t &vm, const gpuvm
  * paper names synchronous write-back on the fault path as its weak spot, Section 5.3).
  * Called by the lanes that pinned the page together (token.group), converged, before
  * gpuvm_release; `p` is any address inside the page's frame.  The dirty bit is cleared
- * before the copy starts: a store that lands during or after the copy sets it again and
- * the page is written back once more later, so nothing is lost.
+ * before the copy starts, so a writer that pins the page after that marks it dirty again and
+ * it is written back once more later.  A writer that pinned the page BEFORE the call and
+ * stores during or after the copy is not covered (its pin saw the dirty bit already set and
+ * did not set it again): clean only pages whose writers have all released them, or that
+ * the calling warp alone writes, as the vector add does.
  */
 __device__ __forceinline__ void gpuvm_clean(const gpuvm_dev_t &vm, const gpuvm_token &token, const void *p)
 {

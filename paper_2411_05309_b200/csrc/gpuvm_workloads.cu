@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(256) stream_sum_kernel(Mem m, unsigned long lo
 
 // -------------------------------------------------------------- random gather
 template <class Mem>
-__global__ void __launch_bounds__(1024) gather_kernel(Mem m, unsigned long long x_off, const long long *__restrict__ idx,
+__global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long long x_off, const long long *__restrict__ idx,
                                                       unsigned long long n_idx, unsigned long long block,
                                                       float *__restrict__ fsum, long long *__restrict__ bsum)
 {
