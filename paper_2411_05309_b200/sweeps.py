@@ -3,6 +3,7 @@ oversubscription analysis), printed as JSON lines.
 
     python -m paper_2411_05309_b200.sweeps pages   [--gib 4] [--warps-per-sm 16]
     python -m paper_2411_05309_b200.sweeps warps   [--gib 2]
+    python -m paper_2411_05309_b200.sweeps resident
     python -m paper_2411_05309_b200.sweeps oversub [--workload 1|2|3|4] [--shrink S]
 
 pages   -- Section 5.1 / Fig. 7: move a fixed amount of host memory into the pool with one
@@ -12,6 +13,9 @@ warps   -- Section 5.2 / Fig. 10 (sensitivity to the number of queue pairs): her
            warps that migrate pages at the same time, 1 .. 32 per SM, at 4 KiB and 64 KiB pages;
            with Little's law (Section 3.2) the link saturates once warps x bytes in flight per
            warp (4 KiB) reach bandwidth x latency.
+resident -- the hit path: streaming sum and random gather over an array that is entirely resident
+           in the pool (no fault in the timed runs), against the same kernels on a plain device
+           pointer and against the measured HBM copy bandwidth.
 oversub -- Section 5.4 / Fig. 14 with Eq. 1: run a workload with the pool shrunk step by step,
            level = paged bytes / pool bytes - 1, under the clock policy and under FIFO (the
            paper's ring), reporting time relative to level 0.
@@ -88,6 +92,44 @@ def sweep_warps(gib: float):
             B.gpuvm_destroy(h)
 
 
+def sweep_resident():
+    import torch
+    from . import binding as B
+    nbytes, n_idx = 1 << 30, 1 << 26
+    host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    host.zero_()
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    dev = torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda")
+    idx = torch.randint(0, nbytes // 4, (n_idx,), device="cuda", dtype=torch.int64)
+    fs = torch.zeros(n_idx // 1024, dtype=torch.float32, device="cuda")
+    bs = torch.zeros(n_idx // 1024, dtype=torch.int64, device="cuda")
+
+    def best(fn, reps=4):
+        fn()
+        torch.cuda.synchronize()
+        return min(_time(torch, fn) for _ in range(reps))
+
+    t = best(lambda: B.gpuvm_raw_stream_sum_i32(dev.data_ptr(), nbytes // 4, out))
+    print(json.dumps({"sweep": "resident", "kernel": "stream_sum on a device pointer", "gbs": nbytes / t / 1e9}), flush=True)
+    t = best(lambda: B.gpuvm_raw_gather_f32(dev.data_ptr(), idx, n_idx, 1024, fs, bs))
+    print(json.dumps({"sweep": "resident", "kernel": "gather on a device pointer", "g_accesses_per_s": n_idx / t / 1e9}), flush=True)
+    for page in (4096, 65536, 2 << 20):
+        h = B.gpuvm_create(host.data_ptr(), nbytes, page, nbytes)
+        try:
+            t = best(lambda: B.gpuvm_stream_sum_i32(h, 0, nbytes // 4, out))
+            faults = B.gpuvm_stats(h)["faults"]
+            print(json.dumps({"sweep": "resident", "kernel": "stream_sum, all pages resident", "page_bytes": page,
+                              "gbs": nbytes / t / 1e9, "faults_in_warm_up_only": faults == nbytes // page}), flush=True)
+            for name, fn in (("gather (batched), all pages resident", B.gpuvm_gather_f32),
+                             ("gather (one request per lane), all pages resident", B.gpuvm_gather_f32_unbatched)):
+                t = best(lambda: fn(h, 0, idx, n_idx, 1024, fs, bs), 3)
+                print(json.dumps({"sweep": "resident", "kernel": name, "page_bytes": page,
+                                  "g_accesses_per_s": n_idx / t / 1e9}), flush=True)
+            assert B.gpuvm_stats(h)["faults"] == nbytes // page
+        finally:
+            B.gpuvm_destroy(h)
+
+
 def sweep_oversub(cfg: int, shrink: int):
     from . import binding as B
     from . import configs
@@ -116,7 +158,7 @@ def sweep_oversub(cfg: int, shrink: int):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("which", choices=["pages", "warps", "oversub"])
+    ap.add_argument("which", choices=["pages", "warps", "resident", "oversub"])
     ap.add_argument("--gib", type=float, default=4.0)
     ap.add_argument("--warps-per-sm", type=int, default=16)
     ap.add_argument("--workload", type=int, default=1)
@@ -124,6 +166,8 @@ def main(argv=None):
     a = ap.parse_args(argv)
     if a.which == "pages":
         sweep_pages(a.gib, a.warps_per_sm)
+    elif a.which == "resident":
+        sweep_resident()
     elif a.which == "warps":
         sweep_warps(min(a.gib, 2.0))
     else:
