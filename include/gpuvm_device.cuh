@@ -139,6 +139,15 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
     return v;
 }
 
+/* take one reference; acquire order: what the publisher of a VALID entry wrote to the frame
+ * before publishing is visible to the accesses that follow in this thread */
+__device__ __forceinline__ unsigned long long pin_acquire(unsigned long long *pte)
+{
+    unsigned long long old;
+    asm volatile("atom.acquire.gpu.global.add.u64 %0, [%1], 1;" : "=l"(old) : "l"(pte) : "memory");
+    return old;
+}
+
 __device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int *p)
 {
     unsigned int v;
@@ -471,7 +480,7 @@ __device__ __forceinline__ bool access(const gpuvm_dev_t &vm, unsigned long long
     unsigned long long *pte = vm.pte + vpn;
     unsigned long long w = 0;
     if (is_leader) {
-        w = atomicAdd(pte, 1ull) + 1ull;                     /* pin first, look afterwards */
+        w = pin_acquire(pte) + 1ull;                         /* pin first, look afterwards */
         if (group & (group - 1)) stat_add(vm, kLanes, __popc(group) - 1);
     }
     w = __shfl_sync(active, w, leader);
@@ -486,7 +495,6 @@ __device__ __forceinline__ bool access(const gpuvm_dev_t &vm, unsigned long long
         }
         unsigned char *p = vm.pool + ((unsigned long long)frame << vm.page_shift) + off;
         if (OP_BYTES == 0) {
-            __threadfence();
             *ptr_out = p;
         } else {
             if (OP_BYTES == 16) { if (mode == kWrite) st_frame16(p, val); else val = ld_frame16(p); }
