@@ -182,7 +182,7 @@ def oracle_step(cfg: int, w=None, shrink: int = 0):
         t0 = time.perf_counter()
         oracle.vadd_f32_direct(a, b)
         return 12 * n, time.perf_counter() - t0, f"direct vector add of the first {n} elements"
-    if cfg == 3:
+    if cfg in (3, 8):
         scale = min(24 - shrink, 22)
         off, col = inputs.rmat_csr(scale, 16 << scale, inputs.config_seed(3))
         t0 = time.perf_counter()
@@ -242,8 +242,9 @@ NAMES = {1: "cfg1 streaming read-reduce: int64 sum over 64 MiB int32, 4 KiB page
          4: "cfg4 vector add c=a+b over three 4 GiB fp32 arrays, 64 KiB pages, 4 GiB pool",
          5: "cfg5 Zipf(1.05) embedding bag: 64 GiB table, 2^24 lookups, bags of 32, 2 MiB pages, 16 GiB pool",
          6: "connected components on the cfg3 graph (RMAT scale 24), CSR paged at 64 KiB, pool = half",
-         7: "SSSP from vertex 0 on the cfg3 graph with int32 weights in a third paged array, 64 KiB pages, pool = half"}
-DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32", 6: "int32", 7: "int32"}
+         7: "SSSP from vertex 0 on the cfg3 graph with int32 weights in a third paged array, 64 KiB pages, pool = half",
+         8: "BFS on the cfg3 graph stored as Balanced CSR (chunks of 16 Ki edges), 64 KiB pages, pool = half"}
+DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32", 6: "int32", 7: "int32", 8: "int32"}
 
 
 # ---------------------------------------------------------------------- rank plumbing
@@ -281,7 +282,7 @@ def e2e_step(torch, B, w, cfg: int):
         h2d = w.rows_host.numel() * 8
     w.launch(stream)
     B.gpuvm_flush(w.h, stream)
-    outs = {1: ["d_sum"], 2: ["d_fsum", "d_bsum"], 3: ["d_level"], 4: [], 5: ["d_out"], 6: ["d_level"], 7: ["d_dist"]}[cfg]
+    outs = {1: ["d_sum"], 2: ["d_fsum", "d_bsum"], 3: ["d_level"], 4: [], 5: ["d_out"], 6: ["d_level"], 7: ["d_dist"], 8: ["d_level"]}[cfg]
     for name in outs:
         t = getattr(w, name)
         buf = w.__dict__.setdefault("_host_" + name, torch.empty(t.shape, dtype=t.dtype).pin_memory())
@@ -401,7 +402,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8])
     ap.add_argument("--shrink", type=int, default=0, help="divide all sizes by 2**shrink")
     ap.add_argument("--uvm", action="store_true", help="also run the workload over cudaMallocManaged")
     ap.add_argument("--uvm-timeout", type=float, default=120.0)

@@ -77,6 +77,21 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
                   int32_t *d_level, int *n_levels, void *stream);
 
 /*
+ * BFS over Balanced CSR (Section 5.2, Fig. 8): besides the row offsets and the column
+ * indices, a third paged array at chunk_off holds, for every chunk of `chunk_edges`
+ * consecutive edges, the number of the vertex whose neighbour list contains the chunk's
+ * first edge (int32, ceil(n_edges / chunk_edges) + 1 entries, the last one = the vertex
+ * of the last edge; see inputs.balanced_chunks).  Workers take chunks instead of
+ * vertices, so each gets the same number of edges and exactly one column page however
+ * skewed the degrees are, and a long list is expanded by as many warps as it has chunks.
+ * A chunk must lie inside one page: col_off is a multiple of the page size and the page
+ * size a multiple of 4 * chunk_edges.  Same result as gpuvm_bfs_csr.  Uses 16 bytes of
+ * the handle's device scratch.  One launch and one synchronisation per level.
+ */
+int gpuvm_bfs_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, size_t nv, size_t n_edges,
+                   size_t chunk_edges, size_t source, int32_t *d_level, int *n_levels, void *stream);
+
+/*
  * Connected components of the same kind of graph (Section 5.2 evaluates CC next to
  * BFS): d_label[v] receives the smallest vertex number of the weakly connected
  * component of v (edges count in both directions).  Label propagation: every sweep

@@ -73,6 +73,7 @@ SYMBOLS = {
     "gpuvm_gather_f32_unbatched": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp, _vp]),
     "gpuvm_bfs_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_bfs_csr_noalloc": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
+    "gpuvm_bfs_bcsr": (_i, [_vp, _sz, _sz, _sz, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_cc_csr": (_i, [_vp, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_sssp_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_raw_cc_csr": (_i, [_vp, _vp, _sz, _vp, ctypes.POINTER(_i), _vp]),
@@ -245,6 +246,14 @@ def gpuvm_bfs_csr(h, off_off: int, col_off: int, nv: int, source: int, d_level, 
     levels = _i(0)
     _check(lib().gpuvm_bfs_csr(h, off_off, col_off, nv, source, _ptr(d_level), ctypes.byref(levels), _stream(stream)),
            "gpuvm_bfs_csr")
+    return levels.value
+
+
+def gpuvm_bfs_bcsr(h, off_off: int, col_off: int, chunk_off: int, nv: int, n_edges: int, chunk_edges: int,
+                   source: int, d_level, stream=None) -> int:
+    levels = _i(0)
+    _check(lib().gpuvm_bfs_bcsr(h, off_off, col_off, chunk_off, nv, n_edges, chunk_edges, source, _ptr(d_level),
+                                ctypes.byref(levels), _stream(stream)), "gpuvm_bfs_bcsr")
     return levels.value
 
 

@@ -194,6 +194,34 @@ class Bfs(Workload):
         return int(16 * visited.sum() + 4 * self.traversed_edges)
 
 
+class BfsBalanced(Bfs):
+    """BFS on the cfg 3 graph stored as Balanced CSR: chunks of one page of edges (16 Ki edges), the chunk
+    table paged with the other two arrays; pool = half."""
+    name, cfg = "bfs_rmat_balanced_csr", 8
+
+    def setup(self):
+        import torch
+        self.scale = 24 - self.shrink
+        self.nv = 1 << self.scale
+        self.ne = 16 << self.scale
+        self.chunk_edges = self.page_bytes // 4
+        n_chunks = (self.ne + self.chunk_edges - 1) // self.chunk_edges
+        self._create({"off": _pad(8 * (self.nv + 1), 16), "col": 4 * self.ne, "chunk": _pad(4 * (n_chunks + 1), 16)},
+                     lambda total: total // 2)
+        base = B.gpuvm_host_ptr(self.h)
+        inputs.rmat_csr(self.scale, self.ne, inputs.config_seed(3), base + self.off["off"], base + self.off["col"])
+        chunks = inputs.balanced_chunks(self.view("off", np.int64, self.nv + 1), self.chunk_edges)
+        self.view("chunk", np.int32, chunks.size)[...] = chunks
+        self.d_level = torch.zeros(self.nv, dtype=torch.int32, device="cuda")
+        self.levels = 0
+        return self
+
+    def launch(self, stream):
+        self.levels = B.gpuvm_bfs_bcsr(self.h, self.off["off"], self.off["col"], self.off["chunk"], self.nv, self.ne,
+                                       self.chunk_edges, 0, self.d_level, stream)
+        return {"levels": self.levels}
+
+
 class Cc(Bfs):
     """Connected components on the BFS configuration's graph and pool (the paper's second graph workload)."""
     name, cfg = "cc_rmat_csr", 6
@@ -282,7 +310,7 @@ class EmbeddingBag(Workload):
         return 4 * self.dims * self.n_lookups
 
 
-WORKLOADS = {1: StreamSum, 2: Gather, 3: Bfs, 4: VAdd, 5: EmbeddingBag, 6: Cc, 7: Sssp}
+WORKLOADS = {1: StreamSum, 2: Gather, 3: Bfs, 4: VAdd, 5: EmbeddingBag, 6: Cc, 7: Sssp, 8: BfsBalanced}
 
 
 def make(cfg: int, shrink: int = 0) -> Workload:

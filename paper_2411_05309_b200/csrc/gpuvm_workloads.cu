@@ -419,6 +419,63 @@ __global__ void __launch_bounds__(256) graph_span_kernel(Mem m, Op op, unsigned 
     if (lane == 0 && found) atomicAdd(counters, found);
 }
 
+// Balanced CSR (Section 5.2, Fig. 8): the edge array is cut into chunks of equal length and a
+// small array names the vertex whose list holds the first edge of each chunk.  Workers take
+// chunks, not vertices: every worker gets the same number of edges and, a chunk lying inside one
+// page, exactly one page of columns, however the degrees are distributed; a long neighbour list
+// is shared by as many workers as it has chunks.  A warp draws a chunk ticket, walks the chunk's
+// vertices 32 at a time, and expands the part of each active vertex's list that lies in the chunk.  counters: [0] updates, [2] chunk ticket.
+template <class Mem, class Op>
+__global__ void __launch_bounds__(256) bcsr_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
+                                                         unsigned long long chunk_off, unsigned int nv,
+                                                         unsigned long long n_edges, unsigned int chunk_edges,
+                                                         unsigned int *__restrict__ counters, int sweep)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    const unsigned int n_chunks = (unsigned int)((n_edges + chunk_edges - 1) / chunk_edges);
+    unsigned int found = 0;
+    for (;;) {
+        unsigned int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(counters + 2, 1u);
+        ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+        if (ticket >= n_chunks) break;
+        const unsigned int c = (sweep & 1) ? n_chunks - 1 - ticket : ticket;
+        const long long c_lo = (long long)c * chunk_edges;
+        const long long c_hi = c_lo + chunk_edges < (long long)n_edges ? c_lo + chunk_edges : (long long)n_edges;
+        // vertices whose lists reach into this chunk: first vertex of this chunk .. first vertex of the next
+        int vr = 0;
+        if (lane < 2) vr = m.template read<int>(chunk_off, (unsigned long long)c + lane);   // chunk table has n_chunks + 1 entries
+        const unsigned int v_first = (unsigned int)__shfl_sync(0xFFFFFFFFu, vr, 0);
+        const unsigned int v_last = (unsigned int)__shfl_sync(0xFFFFFFFFu, vr, 1);
+        for (unsigned int v0 = v_first; v0 <= v_last && v0 < nv; v0 += 32) {
+            const unsigned long long v = (unsigned long long)v0 + lane;
+            const bool active = v <= v_last && v < nv && op.active(v);
+            if (!__any_sync(0xFFFFFFFFu, active)) continue;
+            long long lo = m.template read<long long>(off_off, v < nv ? v : nv);
+            long long hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+            if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
+            if (lo < c_lo) lo = c_lo;
+            if (hi > c_hi) hi = c_hi;
+            unsigned int touch = __ballot_sync(0xFFFFFFFFu, active && hi > lo);
+            if (!touch) continue;
+            // the chunk's column page is held only while these 32 vertices are expanded, never
+            // while row offsets are read: one page at a time, no pool is too small
+            gpuvm_token tok;
+            const unsigned char *p = m.pin(col_off + 4ull * c_lo, GPUVM_READ, tok);
+            if (!p) return;
+            while (touch) {
+                const int L = __ffs(touch) - 1;
+                touch &= touch - 1;
+                const long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
+                found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), blo, bhi, lane);
+            }
+            m.release(tok);
+        }
+    }
+    for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
+    if (lane == 0 && found) atomicAdd(counters, found);
+}
+
 __global__ void bfs_init_kernel(int *level, int source) { level[source] = 0; }
 
 __global__ void cc_init_kernel(int *label, unsigned int nv)
@@ -804,6 +861,39 @@ int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t sour
     return rc;
 }
 
+// BFS over Balanced CSR: one chunk sweep per level.
+template <class Mem>
+int run_bfs_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off, size_t nv, size_t n_edges,
+                 size_t chunk_edges, size_t source, int32_t *d_level, int *n_levels, void *scratch, cudaStream_t s)
+{
+    if (!d_level || nv == 0 || source >= nv || nv > 0x7FFFFFFFull || chunk_edges == 0 || chunk_edges > 0x7FFFFFFFull)
+        return GPUVM_E_ARG;
+    if (off_off % 16 || col_off % 16 || chunk_off % 16) return GPUVM_E_ALIGN;
+    // a chunk must lie inside one unit (page) of the column array
+    if (col_off % m.unit_host() || m.unit_host() % (4 * chunk_edges)) return GPUVM_E_ALIGN;
+    if (!scratch) return GPUVM_E_ALLOC;
+    unsigned int *counters = static_cast<unsigned int *>(scratch);
+    cudaMemsetAsync(d_level, 0xFF, nv * sizeof(int32_t), s);
+    bfs_init_kernel<<<1, 1, 0, s>>>(d_level, (int)source);
+    int rc = launched();
+    int depth = 0;
+    unsigned int found = 1;
+    while (rc == GPUVM_OK && found > 0 && n_edges > 0) {
+        cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
+        bcsr_sweep_kernel<Mem, BfsOp><<<sm_count() * 2, 256, 0, s>>>(m, BfsOp{d_level, depth}, off_off, col_off, chunk_off,
+                                                                     (unsigned int)nv, n_edges, (unsigned int)chunk_edges,
+                                                                     counters, depth);
+        rc = launched();
+        if (cudaMemcpyAsync(&found, counters, sizeof(found), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); rc = GPUVM_E_CUDA; break; }
+        ++depth;
+    }
+    if (n_edges == 0) depth = 1;
+    cudaStreamSynchronize(s);
+    if (n_levels) *n_levels = depth;
+    return rc;
+}
+
 struct Scratch {                     // device scratch for one call, freed on scope exit
     void *p = nullptr;
     explicit Scratch(size_t bytes) { if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); p = nullptr; } }
@@ -986,6 +1076,15 @@ int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, 
     // bfs_levels zeroes the counters at the start of every level and writes each queue entry
     // before reading it, so whatever the previous call left in the array does not matter
     return bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_bfs_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, size_t nv, size_t n_edges,
+                   size_t chunk_edges, size_t source, int32_t *d_level, int *n_levels, void *stream)
+{
+    PagedH m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_bfs_bcsr(m, off_off, col_off, chunk_off, nv, n_edges, chunk_edges, source, d_level, n_levels,
+                        gpuvm_scratch_(h, kBfsScratchBytes), static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, void *stream)

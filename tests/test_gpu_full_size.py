@@ -91,6 +91,16 @@ def test_cc_and_sssp_on_the_cfg3_graph():
         w.close()
 
 
+def test_bfs_over_balanced_csr_rmat24():
+    w, res = run(8)
+    try:
+        off, col = w.view("off", np.int64, w.nv + 1), w.view("col", np.int32, w.ne)
+        assert np.array_equal(w.d_level.cpu().numpy(), oracle.bfs_levels_direct(off, col, 0))
+        assert res.stats["writebacks"] == 0
+    finally:
+        w.close()
+
+
 def test_cfg4_vector_add_12GiB():
     w, res = run(4)
     try:

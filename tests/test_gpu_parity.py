@@ -218,6 +218,39 @@ def graph_arena(page, off, col, weight=None):
 
 
 @pytest.mark.parametrize("policy", POLICIES)
+def test_bfs_over_balanced_csr(B, policy):
+    """Same levels as the oracle's BFS when workers take equal-size edge chunks instead of vertices."""
+    import torch
+    graphs = [csr(nv, edges) + (src,) for nv, edges, src in small_graphs()]
+    graphs.append(inputs.rmat_csr(12, 16 << 12, inputs.config_seed(3)) + (0,))
+    graphs.append(inputs.rmat_csr(14, 16 << 14, inputs.config_seed(3)) + (7,))
+    for off, col, src in graphs:
+        nv, ne = off.size - 1, int(off[-1])
+        ref = oracle.bfs_levels_direct(off, col, src)
+        for page, chunk_edges, frames in ((64, 16, 1), (64, 4, 3), (4096, 1024, 5), (4096, 256, 64)):
+            chunks = inputs.balanced_chunks(off, chunk_edges)
+            # brute-force check of the chunk table: the owner of edge e is the vertex with off[v] <= e < off[v+1]
+            for c in range(min(chunks.size - 1, 50)):
+                v = int(chunks[c])
+                assert off[v] <= c * chunk_edges < off[v + 1]
+            off_p = np.zeros((off.size + 1) // 2 * 2, np.int64)
+            off_p[:off.size] = off
+            pad4 = lambda a: np.concatenate([a, np.zeros((-a.size) % 4, a.dtype)])
+            ar = Arena(page, {"off": off_p, "col": pad4(col), "chunk": pad4(chunks)})
+            level = torch.zeros(nv, dtype=torch.int32, device="cuda")
+            with paged(ar.host, page, frames, policy) as h:
+                depth = B.gpuvm_bfs_bcsr(h, ar.off["off"], ar.off["col"], ar.off["chunk"], nv, ne, chunk_edges, src, level)
+                st, ck = finish(h)
+            assert np.array_equal(level.cpu().numpy(), ref), (nv, ne, page, chunk_edges, frames)
+            assert depth == ref.max() + 1
+    # a chunk that would straddle pages is refused
+    with paged(ar.host, 4096, 8) as h:
+        with pytest.raises(B.GpuvmError) as e:
+            B.gpuvm_bfs_bcsr(h, ar.off["off"], ar.off["col"], ar.off["chunk"], nv, ne, 1536, src, level)
+        assert e.value.status == B.E_ALIGN
+
+
+@pytest.mark.parametrize("policy", POLICIES)
 def test_cc_small_graphs_and_rmat(B, policy):
     import torch
     cases = [(nv, edges) for nv, edges, _ in small_graphs()]
