@@ -55,6 +55,8 @@ def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0) -> dict:
                 "recorded_earlier_run": {"units_total": 1 << 26, "runs": [
                     {"read_mostly": False, "units_run": 262144, "seconds": 10.269, "effective_gbs": 0.000102},
                     {"read_mostly": True, "units_run": 1048576, "seconds": 25.785, "effective_gbs": 0.000163}]}}
+    if cfg not in TWIN_SHRINK:
+        return {"unavailable": "no plain-pointer twin of this workload; see workload 3 for BFS over managed memory"}
     w = configs.make(cfg, shrink + TWIN_SHRINK[cfg])
     try:
         ours = w.run()
