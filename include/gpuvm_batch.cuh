@@ -13,7 +13,8 @@
  *   - row by row, the requests of a row are grouped with __match_any_sync; the leader
  *     of a group pins the page (atomicAdd on the entry) and becomes hit, waiter or
  *     owner exactly as in gpuvm_device.cuh; followers take the frame number from their
- *     leader by shuffle when the page is there;
+ *     leader by shuffle when the page is there (the grouping is redone over the unfinished
+ *     lanes of the row each time: a group finishes as a whole, so it comes out the same);
  *   - every round, each unfinished row is visited: leaders re-read their entry; groups
  *     whose page is resident call `consume(i, ptr)` on each of their requests and the
  *     leader drops the reference at once (no page is held while frames are claimed:
@@ -39,8 +40,8 @@
  * with coalesced 16-byte loads.  gpuvm_batch_skip(table, i) marks slot i as unused.  Requests that fail
  * (offset out of range, wait ran out) are not consumed; the sticky error is set as for the
  * other accessors.  Returns the number of requests served for the calling lane.
- * Pages must not be larger than 128 MiB (the in-page offset shares a word with the
- * leader's lane number).
+ * gpuvm_batch_run is the engine itself: tables of up to 64 * W rows in any layout that a
+ * small accessor type can read (for instance bare 32-bit element indices).
  */
 #ifndef GPUVM_BATCH_CUH
 #define GPUVM_BATCH_CUH
@@ -49,7 +50,7 @@
 
 struct gpuvm_batch_entry {
     unsigned int vpn;       /* page number; 0xFFFFFFFF = rejected request */
-    unsigned int offl;      /* bits 0-26 offset in the page, bits 27-31 lane of the group's leader */
+    unsigned int offl;      /* offset in the page */
 };
 
 constexpr unsigned int GPUVM_BATCH_MAX = 2048;
@@ -67,7 +68,6 @@ struct gpuvm_fault_queue {
 
 namespace gpuvm {
 
-constexpr unsigned int kOffMask = 0x07FFFFFFu;
 constexpr unsigned int kNotReady = 0xFFFFFFFFu;   /* "frame" values a leader hands to its followers */
 constexpr unsigned int kFailed = 0xFFFFFFFEu;
 constexpr unsigned int kRejected = 0xFFFFFFFFu;   /* vpn of a request that was refused when it was set */
@@ -191,8 +191,8 @@ __device__ __forceinline__ void gpuvm_batch_set(const gpuvm_dev_t &vm, gpuvm_bat
                                                 unsigned long long byte_off)
 {
     gpuvm_batch_entry e;
-    if (byte_off >= vm.bytes || vm.page_shift > 27) {
-        gpuvm::set_error(vm, byte_off >= vm.bytes ? GPUVM_E_RANGE : GPUVM_E_PAGE, byte_off >> vm.page_shift);
+    if (byte_off >= vm.bytes) {
+        gpuvm::set_error(vm, GPUVM_E_RANGE, byte_off >> vm.page_shift);
         e.vpn = gpuvm::kRejected; e.offl = 0;
     } else {
         e.vpn = (unsigned int)(byte_off >> vm.page_shift);
@@ -207,41 +207,59 @@ __device__ __forceinline__ void gpuvm_batch_skip(gpuvm_batch_entry *table, unsig
     table[i].offl = 0;
 }
 
-template <bool WARP_CONSUME = false, class Consume>
-static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t vm, gpuvm_batch_entry *table,
-                                                               unsigned int n, int mode, Consume consume,
-                                                               gpuvm_fault_queue *queue = nullptr)
+/* How the engine reads a request table.  valid(i): slot i holds a request; vpn(i) / off(i):
+ * its page number and the offset inside the page.  The engine never writes the table. */
+struct gpuvm_entry_table {
+    const gpuvm_batch_entry *e;
+    __device__ __forceinline__ bool valid(unsigned int i) const { return e[i].vpn != gpuvm::kRejected; }
+    __device__ __forceinline__ unsigned int vpn(unsigned int i) const { return e[i].vpn; }
+    __device__ __forceinline__ unsigned int off(unsigned int i) const { return e[i].offl; }
+};
+
+/*
+ * The engine.  W: the table has up to 64 * W rows of 32 requests (state of a lane's requests
+ * is kept in W 64-bit masks per kind).  Table: see gpuvm_entry_table.  Groups are formed with
+ * __match_any_sync when the requests are registered and again, over the lanes that are not
+ * finished, whenever a row is visited: a group finishes as a whole, so the lanes and the
+ * leader (lowest lane) are the same every time.
+ */
+template <int W, bool WARP_CONSUME, class Table, class Consume>
+static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm, const Table table, unsigned int n,
+                                                            int mode, Consume consume, gpuvm_fault_queue *queue)
 {
     using namespace gpuvm;
     const unsigned int lane = lane_id();
     const unsigned int rows = (n + 31) >> 5;
-    unsigned long long todo = 0;     /* bit j: my request in row j is not finished                */
-    unsigned long long lead = 0;     /* bit j: I lead my group in row j (I hold its reference)     */
-    unsigned long long own = 0;      /* bit j: my group's page is BUSY by my CAS and not handed on */
-    unsigned long long failed = 0;   /* bit j: I gave up on row j (leader only)                    */
+    unsigned long long todo[W], lead[W], own[W], failed[W];
+    /* bit j of word k: row 64 k + j.  todo: my request is not finished; lead: I lead my group
+     * (I hold its reference); own: my group's page is BUSY by my CAS and not handed on;
+     * failed: I gave up on the row (leader only) */
+#pragma unroll
+    for (int k = 0; k < W; ++k) { todo[k] = 0; lead[k] = 0; own[k] = 0; failed[k] = 0; }
     unsigned int served = 0;
 
     /* register every request in the page table (steps 1-4 of the access path) */
-    for (unsigned int j = 0; j < rows; ++j) {
-        const unsigned int i = j * 32 + lane;
-        const bool active = i < n && table[i].vpn != kRejected;
-        const unsigned int m = __ballot_sync(0xFFFFFFFFu, active);
-        if (active) {
-            const unsigned int vpn = table[i].vpn;
-            const unsigned int group = __match_any_sync(m, vpn);
-            const unsigned int leader = __ffs(group) - 1;
-            table[i].offl = (table[i].offl & kOffMask) | (leader << 27);
-            if (lane == leader) {
-                unsigned long long *pte = vm.pte + vpn;
-                unsigned int frame;
-                const int st = advance(vm, pte, atomicAdd(pte, 1ull) + 1ull, mode, frame);
-                if (st == kReady) { if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1); }
-                else if (st == kWait) stat_add(vm, kWaits, 1);
-                else own |= 1ull << j;
-                if (group & (group - 1)) stat_add(vm, kLanes, __popc(group) - 1);
-                lead |= 1ull << j;
+#pragma unroll
+    for (int k = 0; k < W; ++k) {
+        for (unsigned int jj = 0; jj < 64 && 64u * k + jj < rows; ++jj) {
+            const unsigned int i = (64u * k + jj) * 32 + lane;
+            const bool active = i < n && table.valid(i);
+            const unsigned int m = __ballot_sync(0xFFFFFFFFu, active);
+            if (active) {
+                const unsigned int vpn = table.vpn(i);
+                const unsigned int group = __match_any_sync(m, vpn);
+                if (lane == (unsigned int)(__ffs(group) - 1)) {
+                    unsigned long long *pte = vm.pte + vpn;
+                    unsigned int frame;
+                    const int st = advance(vm, pte, pin_acquire(pte) + 1ull, mode, frame);
+                    if (st == kReady) { if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1); }
+                    else if (st == kWait) stat_add(vm, kWaits, 1);
+                    else own[k] |= 1ull << jj;
+                    if (group & (group - 1)) stat_add(vm, kLanes, __popc(group) - 1);
+                    lead[k] |= 1ull << jj;
+                }
+                todo[k] |= 1ull << jj;
             }
-            todo |= 1ull << j;
         }
     }
     __syncwarp();
@@ -250,70 +268,77 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
     unsigned int sleep_ns = 64;
     for (;;) {
         bool progress = false, any_rows = false;
-        for (unsigned int j = 0; j < rows; ++j) {
-            const bool mine = (todo >> j) & 1ull;
-            const unsigned int rowmask = __ballot_sync(0xFFFFFFFFu, mine);
-            if (!rowmask) continue;
-            any_rows = true;
-            unsigned int frame = kNotReady, off = 0;
-            unsigned long long *pte = nullptr;
-            bool is_leader = false;
-            const unsigned int i = j * 32 + lane;
-            if (mine) {
-                const gpuvm_batch_entry e = table[i];
-                const unsigned int leader = e.offl >> 27;
-                off = e.offl & kOffMask;
-                pte = vm.pte + e.vpn;
-                is_leader = (lead >> j) & 1ull;
-                if (is_leader) {
-                    if ((failed >> j) & 1ull) {
-                        frame = kFailed;
-                    } else if (!((own >> j) & 1ull)) {
-                        unsigned int f;
-                        const int st = advance(vm, pte, ld_acquire_u64(pte), mode, f);   /* acquire: pairs with the publish */
-                        if (st == kReady) frame = f;
-                        else if (st == kOwn) { own |= 1ull << j; progress = true; }
+#pragma unroll
+        for (int k = 0; k < W; ++k) {
+            for (unsigned int jj = 0; jj < 64 && 64u * k + jj < rows; ++jj) {
+                const unsigned long long bit = 1ull << jj;
+                const bool mine = (todo[k] & bit) != 0;
+                const unsigned int rowmask = __ballot_sync(0xFFFFFFFFu, mine);
+                if (!rowmask) continue;
+                any_rows = true;
+                const unsigned int i = (64u * k + jj) * 32 + lane;
+                unsigned int frame = kNotReady, off = 0;
+                unsigned long long *pte = nullptr;
+                bool is_leader = false;
+                if (mine) {
+                    const unsigned int vpn = table.vpn(i);
+                    const unsigned int leader = __ffs(__match_any_sync(rowmask, vpn)) - 1;
+                    off = table.off(i);
+                    pte = vm.pte + vpn;
+                    is_leader = (lead[k] & bit) != 0;            /* == (lane == leader) */
+                    if (is_leader) {
+                        if (failed[k] & bit) {
+                            frame = kFailed;
+                        } else if (!(own[k] & bit)) {
+                            unsigned int f;
+                            const int st = advance(vm, pte, ld_acquire_u64(pte), mode, f);   /* pairs with the publish */
+                            if (st == kReady) frame = f;
+                            else if (st == kOwn) { own[k] |= bit; progress = true; }
+                        }
                     }
+                    frame = __shfl_sync(rowmask, frame, leader);
+                    if (frame == kFailed) todo[k] &= ~bit;
                 }
-                frame = __shfl_sync(rowmask, frame, leader);
-                if (frame == kFailed) todo &= ~(1ull << j);
-            }
-            const bool ready = mine && frame < kFailed;
-            if (WARP_CONSUME) {
-                unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
-                while (ready_lanes) {
-                    const unsigned int L = __ffs(ready_lanes) - 1;
-                    ready_lanes &= ready_lanes - 1;
-                    const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame, L), o = __shfl_sync(0xFFFFFFFFu, off, L);
-                    consume(j * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o);
+                const bool ready = mine && frame < kFailed;
+                if (WARP_CONSUME) {
+                    unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
+                    while (ready_lanes) {
+                        const unsigned int L = __ffs(ready_lanes) - 1;
+                        ready_lanes &= ready_lanes - 1;
+                        const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame, L), o = __shfl_sync(0xFFFFFFFFu, off, L);
+                        consume((64u * k + jj) * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o);
+                    }
+                    __syncwarp();                               /* every group has used its frame */
+                } else {
+                    if (ready) consume(i, vm.pool + ((unsigned long long)frame << vm.page_shift) + off);
+                    if (mine) __syncwarp(rowmask);              /* the whole group has used the frame */
                 }
-                __syncwarp();                                   /* every group has used its frame */
-            } else {
                 if (ready) {
-                    consume(i, vm.pool + ((unsigned long long)frame << vm.page_shift) + off);
+                    todo[k] &= ~bit;
+                    ++served;
+                    progress = true;
+                    if (is_leader) unpin(pte);                  /* step 8 */
                 }
-                if (mine) __syncwarp(rowmask);                  /* the whole group has used the frame */
-            }
-            if (ready) {
-                todo &= ~(1ull << j);
-                ++served;
-                progress = true;
-                if (is_leader) unpin(pte);                      /* step 8 */
             }
         }
         if (!any_rows) break;
 
         if (queue) {
             /* hand owned faults to the migrator warps; afterwards wait for the page like anyone */
-            while (own) {
-                const unsigned int j = __ffsll((long long)own) - 1;
-                if (!fault_queue_push(queue, table[j * 32 + lane].vpn, mode)) break;
-                own &= own - 1;
-                progress = true;
-            }
+#pragma unroll
+            for (int k = 0; k < W; ++k)
+                while (own[k]) {
+                    const unsigned int jj = __ffsll((long long)own[k]) - 1;
+                    if (!fault_queue_push(queue, table.vpn((64u * k + jj) * 32 + lane), mode)) break;
+                    own[k] &= own[k] - 1;
+                    progress = true;
+                }
         } else {
             /* no helpers: the first lane that owns a fault takes a frame and the warp migrates the page */
-            const unsigned int owners = __ballot_sync(0xFFFFFFFFu, own != 0);
+            bool has_own = false;
+#pragma unroll
+            for (int k = 0; k < W; ++k) has_own |= own[k] != 0;
+            const unsigned int owners = __ballot_sync(0xFFFFFFFFu, has_own);
             if (owners) {
                 const unsigned int L = __ffs(owners) - 1;
                 unsigned int h = 0, vpn = 0;
@@ -321,13 +346,24 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
                 bool vdirty = false;
                 int claimed = 0;
                 if (lane == L) {
-                    vpn = table[(__ffsll((long long)own) - 1) * 32 + lane].vpn;
+                    int kk = 0;
+#pragma unroll
+                    for (int k = W - 1; k >= 0; --k) if (own[k]) kk = k;
+                    unsigned long long word = 0;
+#pragma unroll
+                    for (int k = 0; k < W; ++k) if (k == kk) word = own[k];
+                    vpn = table.vpn((64u * kk + (__ffsll((long long)word) - 1)) * 32 + lane);
                     claimed = try_claim(vm, vpn, 4, h, victim, vdirty);
                 }
                 if (__shfl_sync(0xFFFFFFFFu, claimed, L)) {
                     migrate_page(vm, __shfl_sync(0xFFFFFFFFu, vpn, L), mode, __shfl_sync(0xFFFFFFFFu, h, L),
                                  __shfl_sync(0xFFFFFFFFu, victim, L), __shfl_sync(0xFFFFFFFFu, (int)vdirty, L), lane, L);
-                    if (lane == L) own &= own - 1;
+                    if (lane == L) {
+                        bool cleared = false;
+#pragma unroll
+                        for (int k = 0; k < W; ++k)
+                            if (!cleared && own[k]) { own[k] &= own[k] - 1; cleared = true; }
+                    }
                     progress = true;
                 }
             }
@@ -340,16 +376,19 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
         bool expired = (t - t_start) > (unsigned long long)vm.spin_limit_us * 1000ull || has_error(vm);
         expired = __any_sync(0xFFFFFFFFu, expired);
         if (expired) {
-            unsigned long long give_up = todo & lead & ~failed;
-            while (give_up) {
-                const unsigned int j = __ffsll((long long)give_up) - 1;
-                give_up &= give_up - 1;
-                unsigned long long *pte = vm.pte + table[j * 32 + lane].vpn;
-                set_error(vm, GPUVM_E_TIMEOUT, table[j * 32 + lane].vpn);
-                if ((own >> j) & 1ull) atomicXor(pte, kBusy);   /* BUSY -> INVALID: never handed on */
-                unpin(pte);
-                own &= ~(1ull << j);
-                failed |= 1ull << j;
+#pragma unroll
+            for (int k = 0; k < W; ++k) {
+                unsigned long long give_up = todo[k] & lead[k] & ~failed[k];
+                while (give_up) {
+                    const unsigned int jj = __ffsll((long long)give_up) - 1;
+                    give_up &= give_up - 1;
+                    const unsigned int vpn = table.vpn((64u * k + jj) * 32 + lane);
+                    set_error(vm, GPUVM_E_TIMEOUT, vpn);
+                    if ((own[k] >> jj) & 1ull) atomicXor(vm.pte + vpn, kBusy);   /* BUSY -> INVALID: never handed on */
+                    unpin(vm.pte + vpn);
+                    own[k] &= ~(1ull << jj);
+                    failed[k] |= 1ull << jj;
+                }
             }
             continue;                                           /* followers learn of it in the next round */
         }
@@ -358,6 +397,15 @@ static __device__ __noinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t
         if (sleep_ns < 4096) sleep_ns *= 2;
     }
     return served;
+}
+
+/* One table of up to 2048 eight-byte entries (see the top of this file). */
+template <bool WARP_CONSUME = false, class Consume>
+static __device__ __forceinline__ unsigned int gpuvm_batch_access(const gpuvm_dev_t &vm, gpuvm_batch_entry *table,
+                                                                  unsigned int n, int mode, Consume consume,
+                                                                  gpuvm_fault_queue *queue = nullptr)
+{
+    return gpuvm_batch_run<1, WARP_CONSUME>(vm, gpuvm_entry_table{table}, n, mode, consume, queue);
 }
 
 #endif /* GPUVM_BATCH_CUH */

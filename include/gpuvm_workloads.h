@@ -176,7 +176,7 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
  * device scratch and added per bag in list order once the batch is complete, so the
  * result has the bits of a sequential fp32 sum.  Scratch owned by the handle: 8 KiB +
  * 1024 rows per requester warp (2.1 GiB for dims = 128 on a full grid of 148 SMs),
- * allocated at the first call, freed by gpuvm_destroy.  Pages up to 128 MiB.
+ * allocated at the first call, freed by gpuvm_destroy.
  * gpuvm_embag_f32_unbatched: one warp per bag, one row request at a time through
  * gpuvm_read; no scratch.
  */

@@ -1125,7 +1125,6 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     if (!d_rows || !d_out || dims == 0 || dims % 4 || dims / 4 > 32 || bag == 0 || bag > 0xFFFFFFFFull) return GPUVM_E_ARG;
     if (t_off % 16) return GPUVM_E_ALIGN;
     if (n_bags == 0) return GPUVM_OK;
-    if (m.vm.page_shift > 27) return GPUVM_E_PAGE;
     const int requesters = kEmbagRequesters, migrators = kEmbagMigrators;
     const size_t items = (n_bags + 31) / 32;
     const size_t blocks_needed = (items + requesters - 1) / requesters;
@@ -1165,7 +1164,6 @@ int gpuvm_scatter_update_u32_batched(gpuvm_t h, size_t a_off, const int64_t *d_i
     Paged m;
     if (!view_of(h, m) || !d_idx) return GPUVM_E_ARG;
     if (a_off % 16) return GPUVM_E_ALIGN;
-    if (m.vm.page_shift > 27) return GPUVM_E_PAGE;
     if (n == 0) return GPUVM_OK;
     scatter_update_batch_kernel<<<sm_count() * 4, 128, 0, static_cast<cudaStream_t>(stream)>>>(
         m.vm, a_off, reinterpret_cast<const long long *>(d_idx), n);
