@@ -44,13 +44,13 @@ int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void
  * x: fp32 array at x_off; d_idx: n_idx int64 element indices in device memory.
  * d_fsum, d_bsum: ceil(n_idx / block) elements.  block <= 2^20.
  *
- * gpuvm_gather_f32: a requester warp stages 2048 page requests at a time and keeps all
- * of them registered in the page table at once (gpuvm_batch.cuh), so that one migrated
- * page serves many waiting requests (Section 3.3: inter-warp coalescing); the faults
- * go through a ring of page ids in shared memory to the thread block's migrator warps.
- * The request tables (16 KiB per requester warp, 68 MiB for a full grid on 148 SMs) are
- * device scratch owned by the handle: allocated at the first call, freed by
- * gpuvm_destroy.
+ * gpuvm_gather_f32: a requester warp stages 4096 requests at a time (32-bit element indices,
+ * so the array must have fewer than 2^32 - 1 elements: GPUVM_E_RANGE otherwise) and keeps
+ * all of them registered in the page table at once (gpuvm_batch.cuh), so that one migrated
+ * page serves many waiting requests (Section 3.3: inter-warp coalescing); the faults go
+ * through a ring of page ids in shared memory to the thread block's migrator warps.  The
+ * request tables (16 KiB per requester warp, 68 MiB for a full grid on 148 SMs) are device
+ * scratch owned by the handle: allocated at the first call, freed by gpuvm_destroy.
  * gpuvm_gather_f32_unbatched: one thread per index through gpuvm_read<float>, one
  * thread block per index block; at most 32 requests per warp are in flight.
  */

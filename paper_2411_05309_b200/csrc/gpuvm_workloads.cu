@@ -130,8 +130,8 @@ __global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long lo
 }
 
 // A requester warp takes a run of consecutive indices (whole index blocks when they fit),
-// stages their page requests in its request table (handle-owned device scratch: it stays in
-// L2), registers them all in the page table, and as the pages arrive replaces each request by
+// stages their element indices in its request table (handle-owned device scratch: it stays in
+// L2), registers them all in the page table, and as the pages arrive replaces each index by
 // the value it asked for (gpuvm_batch.cuh); then it adds the values up block by block.  The
 // faults it owns go to the thread block's ring of page ids in shared memory, which the
 // block's migrator warps serve.  No block-wide barrier after start-up: warps never wait for
@@ -139,18 +139,32 @@ __global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long lo
 constexpr int kGatherRequesters = 28;
 constexpr int kGatherMigrators = 4;
 constexpr int kGatherMaxWarps = 32;
-constexpr unsigned int kGatherBatch = GPUVM_BATCH_MAX;   // requests per requester warp
+constexpr unsigned int kGatherBatch = 4096;              // requests per requester warp: 128 rows of 32
+constexpr unsigned int kNoIndex = 0xFFFFFFFFu;
+
+// Request table of the gather: one 32-bit element index per request (the array has fewer than
+// 2^32 - 1 elements), replaced by the value's bit pattern when the request is served.
+struct GatherTable {
+    unsigned int *e;
+    unsigned long long x_off;
+    unsigned int page_shift;
+    __device__ __forceinline__ bool valid(unsigned int i) const { return e[i] != kNoIndex; }
+    __device__ __forceinline__ unsigned int vpn(unsigned int i) const { return (unsigned int)((x_off + 4ull * e[i]) >> page_shift); }
+    __device__ __forceinline__ unsigned int off(unsigned int i) const
+    {
+        return (unsigned int)((x_off + 4ull * e[i]) & ((1ull << page_shift) - 1ull));
+    }
+};
 
 __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(gpuvm_dev_t vm, unsigned long long x_off,
-                                                                            const long long *__restrict__ idx,
-                                                                            unsigned long long n_idx, unsigned long long block,
-                                                                            float *__restrict__ fsum, long long *__restrict__ bsum,
-                                                                            int requesters, unsigned int batch,
-                                                                            gpuvm_batch_entry *g_tables)
+                                                                               const long long *__restrict__ idx,
+                                                                               unsigned long long n_idx, unsigned long long block,
+                                                                               float *__restrict__ fsum, long long *__restrict__ bsum,
+                                                                               int requesters, unsigned int batch,
+                                                                               unsigned int *g_tables)
 {
-    extern __shared__ __align__(16) unsigned char s_raw[];
-    gpuvm_fault_queue *queue = reinterpret_cast<gpuvm_fault_queue *>(s_raw);
-    gpuvm_batch_entry *tables = g_tables + (size_t)blockIdx.x * requesters * batch;
+    __shared__ gpuvm_fault_queue queue_s;
+    gpuvm_fault_queue *queue = &queue_s;
     const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
         reinterpret_cast<unsigned int *>(queue)[k] = 0;
@@ -161,7 +175,8 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
         gpuvm_migrator_loop(vm, queue);
         return;
     }
-    gpuvm_batch_entry *table = tables + (size_t)warp * batch;
+    unsigned int *table = g_tables + ((size_t)blockIdx.x * requesters + warp) * batch;
+    const unsigned long long n_elems = (vm.bytes - x_off) / 4;
     const unsigned long long nb = (n_idx + block - 1) / block;
     const unsigned long long per = block <= batch ? batch / block : 1;      // index blocks per work item
     const unsigned long long items = (nb + per - 1) / per;
@@ -173,15 +188,19 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
         long long carry_b = 0;
         for (unsigned long long base = lo; base < hi; base += batch) {
             const unsigned int n = (unsigned int)(hi - base < batch ? hi - base : batch);
-            for (unsigned int k = lane; k < n; k += 32)
-                gpuvm_batch_set(vm, table, k, x_off + 4ull * (unsigned long long)idx[base + k]);
+            for (unsigned int k = lane; k < n; k += 32) {
+                const unsigned long long i = (unsigned long long)idx[base + k];
+                if (i >= n_elems) gpuvm::set_error(vm, GPUVM_E_RANGE, (x_off + 4 * i) >> vm.page_shift);
+                table[k] = i < n_elems ? (unsigned int)i : kNoIndex;
+            }
             __syncwarp();
-            gpuvm_batch_access(vm, table, n, GPUVM_READ, [table](unsigned int i, const unsigned char *p) {
-                table[i].vpn = gpuvm_load(reinterpret_cast<const unsigned int *>(p));
-                table[i].offl = 1u;                              // served
-            }, queue);
+            gpuvm_batch_run<2, false>(vm, GatherTable{table, x_off, vm.page_shift}, n, GPUVM_READ,
+                                      [table](unsigned int i, const unsigned char *p) {
+                                          table[i] = gpuvm_load(reinterpret_cast<const unsigned int *>(p));
+                                      }, queue);
             __syncwarp();
-            // sum the values of this piece, index block by index block
+            // sum the values of this piece, index block by index block (a rejected index left
+            // kNoIndex in its slot and has set the sticky error: the sums are then meaningless)
             unsigned long long pos = base;
             while (pos < base + n) {
                 const unsigned long long b = pos / block;
@@ -190,11 +209,9 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
                 double f = 0.0;
                 long long bits = 0;
                 for (unsigned long long k = pos + lane; k < end; k += 32) {
-                    const gpuvm_batch_entry e = table[k - base];
-                    if (e.offl == 1u) {
-                        f += (double)__uint_as_float(e.vpn);
-                        bits += (long long)e.vpn;
-                    }
+                    const unsigned int v = table[k - base];
+                    f += (double)__uint_as_float(v);
+                    bits += (long long)v;
                 }
                 for (int o = 16; o; o >>= 1) {
                     f += __shfl_down_sync(0xFFFFFFFFu, f, o);
@@ -1027,6 +1044,7 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     if (!d_idx || !d_fsum || !d_bsum || block == 0 || block > (size_t(1) << 20)) return GPUVM_E_ARG;
     if (x_off % 16) return GPUVM_E_ALIGN;
     if (n_idx == 0) return GPUVM_OK;
+    if ((m.vm.bytes - x_off) / 4 >= kNoIndex) return GPUVM_E_RANGE;      // element indices are staged as 32-bit numbers
     const int requesters = kGatherRequesters, migrators = kGatherMigrators;
     const unsigned int batch = kGatherBatch;
     const size_t nb = (n_idx + block - 1) / block;
@@ -1034,10 +1052,9 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     const size_t items = (nb + per - 1) / per;
     const size_t blocks_needed = (items + requesters - 1) / requesters;
     const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
-    gpuvm_batch_entry *tables = static_cast<gpuvm_batch_entry *>(
-        gpuvm_scratch_(h, (size_t)grid * requesters * batch * sizeof(gpuvm_batch_entry)));
+    unsigned int *tables = static_cast<unsigned int *>(gpuvm_scratch_(h, (size_t)grid * requesters * batch * sizeof(unsigned int)));
     if (!tables) return GPUVM_E_ALLOC;
-    gather_batch_kernel<<<grid, (requesters + migrators) * 32, sizeof(gpuvm_fault_queue), static_cast<cudaStream_t>(stream)>>>(
+    gather_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
         m.vm, x_off, reinterpret_cast<const long long *>(d_idx), n_idx, block, d_fsum, reinterpret_cast<long long *>(d_bsum),
         requesters, batch, tables);
     return launched();
