@@ -152,6 +152,34 @@ def test_batched_waits_run_out_too(B, which):
             assert np.array_equal(bs.cpu().numpy(), oracle.gather_block_sums_direct(x, idx, 1024)[1])
 
 
+def test_concurrent_kernels_on_one_handle_and_on_two(B):
+    """Kernels launched on different streams may share a page table (Section 4, "Multi-kernel
+    support": a stream of concurrent kernels reading the same data on demand): a warp only ever
+    waits for pages that a running warp is fetching, so no launch waits for another launch."""
+    import torch
+    n = 1 << 18
+    a = inputs.fill_i32_u20(np.empty(n, np.int32), n, 11)
+    b = inputs.fill_i32_u20(np.empty(n, np.int32), n, 12)
+    ar, br = Arena(4096, {"a": a}), Arena(4096, {"a": b})
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    outs = [torch.zeros(1, dtype=torch.int64, device="cuda") for _ in range(4)]
+    with paged(ar.host, 4096, 24) as h1, paged(br.host, 4096, 24) as h2:
+        for rep in range(5):
+            B.gpuvm_reset(h1)
+            B.gpuvm_reset(h2)
+            # two kernels on one handle (overlapping halves), a third on another handle
+            B.gpuvm_stream_sum_i32(h1, 0, 3 * n // 4, outs[0], s1)
+            B.gpuvm_stream_sum_i32(h1, n, 3 * n // 4, outs[1], s2)          # byte offset n = element n/4
+            B.gpuvm_stream_sum_i32(h2, 0, n, outs[2], s1)
+            B.gpuvm_stream_sum_i32(h2, 0, n, outs[3], s2)
+            torch.cuda.synchronize()
+            assert int(outs[0].item()) == int(a[: 3 * n // 4].astype(np.int64).sum())
+            assert int(outs[1].item()) == int(a[n // 4:].astype(np.int64).sum())
+            assert int(outs[2].item()) == int(outs[3].item()) == int(b.astype(np.int64).sum())
+            finish(h1)
+            finish(h2)
+
+
 def test_offset_past_the_end_is_a_range_error(B):
     import torch
     host = aligned_bytes(8 * 4096)
