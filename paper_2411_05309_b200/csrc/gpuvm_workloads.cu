@@ -302,7 +302,7 @@ __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned
 // window low.  Odd sweeps run downwards: the pages a sweep used last are still resident when the
 // next one starts with them (a one-directional cyclic sweep defeats any LRU-like policy).
 template <class Mem, class Op, bool WEIGHTED>
-__global__ void __launch_bounds__(256) graph_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
+__global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
                                                           unsigned long long w_off, unsigned int nv,
                                                           unsigned long long n_edges, long long *__restrict__ span_q,
                                                           unsigned int *__restrict__ counters, int sweep)
@@ -406,7 +406,7 @@ __global__ void __launch_bounds__(256) graph_sweep_kernel(Mem m, Op op, unsigned
 
 // Pieces of long neighbour lists, one warp per piece (a piece never crosses a unit).
 template <class Mem, class Op, bool WEIGHTED>
-__global__ void __launch_bounds__(256) graph_span_kernel(Mem m, Op op, unsigned long long col_off, unsigned long long w_off,
+__global__ void __launch_bounds__(256, 4) graph_span_kernel(Mem m, Op op, unsigned long long col_off, unsigned long long w_off,
                                                          const long long *__restrict__ span_q,
                                                          unsigned int *__restrict__ counters)
 {
@@ -443,7 +443,7 @@ __global__ void __launch_bounds__(256) graph_span_kernel(Mem m, Op op, unsigned 
 // is shared by as many workers as it has chunks.  A warp draws a chunk ticket, walks the chunk's
 // vertices 32 at a time, and expands the part of each active vertex's list that lies in the chunk.  counters: [0] updates, [2] chunk ticket.
 template <class Mem, class Op>
-__global__ void __launch_bounds__(256) bcsr_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
+__global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
                                                          unsigned long long chunk_off, unsigned int nv,
                                                          unsigned long long n_edges, unsigned int chunk_edges,
                                                          unsigned int *__restrict__ counters, int sweep)
@@ -836,7 +836,7 @@ int graph_sweep(const Mem &m, const Op &op, size_t off_off, size_t col_off, size
     const unsigned long long n_edges = m.edges_hint;
     long long *span_q = static_cast<long long *>(scratch);
     unsigned int *counters = reinterpret_cast<unsigned int *>(span_q + 4 * kBigQueue);
-    const int grid = sm_count() * 2;
+    const int grid = sm_count() * 4;
     cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
     graph_sweep_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, off_off, col_off, w_off, (unsigned int)nv, n_edges, span_q, counters, sweep);
     graph_span_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, col_off, w_off, span_q, counters);
