@@ -163,6 +163,16 @@ int gpuvm_check(gpuvm_t h, gpuvm_check_t *out);
 int gpuvm_set_policy(gpuvm_t h, int policy);
 int gpuvm_set_spin_limit_us(gpuvm_t h, unsigned int spin_limit_us);
 
+/* Device scratch of the batched workload entry points (request tables, staging of gathered
+ * rows; not pages of the backing store).  It belongs to the handle, is allocated at the first
+ * call that needs it and grown on demand.  More scratch lets a kernel keep more page requests
+ * registered at once, and so lets one migrated page serve more of them (the counterpart of the
+ * paper's deeper queues, Section 3.2): gpuvm_set_scratch_limit bounds it (bytes; 0 = no bound,
+ * the default), the workloads then choose the deepest batch that fits and never less than their
+ * smallest one.  gpuvm_scratch_bytes returns what is allocated now. */
+int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes);
+size_t gpuvm_scratch_bytes(gpuvm_t h);
+
 /* Largest number of simultaneously resident warps that can each hold
  * `pins_per_warp` pages pinned without exhausting the pool (a warp that holds
  * pins while faulting needs a free frame; Section 3.3: a frame is reused only

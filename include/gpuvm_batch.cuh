@@ -1,5 +1,5 @@
 /*
- * gpuvm_batch.cuh -- batched access: one warp keeps up to 2048 page requests in flight.
+ * gpuvm_batch.cuh -- batched access: one warp keeps thousands of page requests in flight.
  *
  * gpuvm_read / gpuvm_write return when the slowest of a warp's 32 requests has been
  * served, so a warp never has more than 32 requests outstanding.  For scattered
@@ -40,11 +40,14 @@
  * with coalesced 16-byte loads.  gpuvm_batch_skip(table, i) marks slot i as unused.  Requests that fail
  * (offset out of range, wait ran out) are not consumed; the sticky error is set as for the
  * other accessors.  Returns the number of requests served for the calling lane.
- * gpuvm_batch_run is the engine itself: tables of up to 64 * W rows in any layout that a
- * small accessor type can read (for instance bare 32-bit element indices).
+ * gpuvm_batch_run is the engine itself: longer tables, in any layout that a small accessor
+ * type can read (for instance bare 32-bit element indices), with the per-lane state words in
+ * memory the caller provides.
  */
 #ifndef GPUVM_BATCH_CUH
 #define GPUVM_BATCH_CUH
+
+#include <type_traits>
 
 #include "gpuvm_device.cuh"
 
@@ -58,36 +61,67 @@ constexpr unsigned int GPUVM_BATCH_MAX = 2048;
 /* Ring of owned faults of one thread block, in shared memory.  Zero it (all fields) before
  * use, set `requesters` to the number of requester warps, __syncthreads(). */
 constexpr unsigned int GPUVM_FAULT_QUEUE_SLOTS = 2048;
+constexpr unsigned int GPUVM_SHARED_QUEUE_SLOTS = 1u << 16;
+constexpr unsigned int GPUVM_FAULT_QUEUE_SPILL = 8;       /* entries a block keeps for its own migrators */
+
+/* Optional ring in device memory that all thread blocks of a grid share: a block whose own
+ * ring already holds GPUVM_FAULT_QUEUE_SPILL entries pushes here instead, and migrator warps
+ * that find their block's ring empty pop from here, so no block is left to move a long
+ * backlog alone while the migrators of the others idle.  Zero it before the launch. */
+struct gpuvm_shared_queue {
+    unsigned int head;
+    unsigned int pad0[31];
+    unsigned int tail;
+    unsigned int pad1[31];
+    unsigned int slot[GPUVM_SHARED_QUEUE_SLOTS];  /* as gpuvm_fault_queue::slot */
+};
+
 struct gpuvm_fault_queue {
     unsigned int head;          /* next slot to pop  */
     unsigned int tail;          /* next slot to push */
     unsigned int requesters;    /* requester warps that have not called gpuvm_requester_done yet */
     unsigned int pad;
+    gpuvm_shared_queue *shared; /* nullptr: none */
     unsigned int slot[GPUVM_FAULT_QUEUE_SLOTS];   /* 0 = empty, else (vpn + 1) | write << 31 */
 };
 
 namespace gpuvm {
 
 constexpr unsigned int kNotReady = 0xFFFFFFFFu;   /* "frame" values a leader hands to its followers */
-constexpr unsigned int kFailed = 0xFFFFFFFEu;
 constexpr unsigned int kRejected = 0xFFFFFFFFu;   /* vpn of a request that was refused when it was set */
 
 /* Any lane.  False when the ring is (nearly) full: the caller keeps the fault and retries. */
 __device__ __forceinline__ bool fault_queue_push(gpuvm_fault_queue *q, unsigned int vpn, int mode)
 {
     volatile unsigned int *vh = &q->head, *vt = &q->tail;
+    const unsigned int item = (vpn + 1u) | (mode == kWrite ? 0x80000000u : 0u);
+    gpuvm_shared_queue *g = q->shared;
+    if (g && *vt - *vh >= GPUVM_FAULT_QUEUE_SPILL) {
+        /* the block has enough of its own: the shared ring, unless that is (nearly) full.  Any
+         * lane of the grid may pass the check at the same moment: 2^15 slots stay spare. */
+        const unsigned int gh = ld_relaxed_u32(&g->head), gt = ld_relaxed_u32(&g->tail);
+        if (gt - gh < GPUVM_SHARED_QUEUE_SLOTS - (1u << 15)) {
+            const unsigned int pos = atomicAdd(&g->tail, 1u);
+            st_relaxed_u32(&g->slot[pos % GPUVM_SHARED_QUEUE_SLOTS], item);
+            return true;
+        }
+    }
     /* up to 1024 lanes may pass this check at the same moment: keep that many slots spare */
     if (*vt - *vh >= GPUVM_FAULT_QUEUE_SLOTS - 1024u) return false;
     const unsigned int pos = atomicAdd(&q->tail, 1u);
     volatile unsigned int *slot = &q->slot[pos % GPUVM_FAULT_QUEUE_SLOTS];
-    *slot = (vpn + 1u) | (mode == kWrite ? 0x80000000u : 0u);
+    *slot = item;
     return true;
 }
 
 /* All 32 lanes: frame `h` has been claimed for page `vpn` by lane `L` (steps 6 and 7 of the
- * access path): write a dirty victim back, unmap it, copy the page in, publish. */
-__device__ __forceinline__ void migrate_page(const gpuvm_dev_t &vm, unsigned long long vpn, int mode, unsigned int h,
-                                             unsigned long long victim, int vdirty, unsigned int lane, unsigned int L)
+ * access path): write a dirty victim back, unmap it, copy the page in, publish.  With `bulk`
+ * (state held by lane L) the page comes in through the bulk-copy unit; false is returned when
+ * that copy did not finish within the bound: the sticky error is set, the page's entry goes
+ * back to INVALID and the frame is free again. */
+__device__ __forceinline__ bool migrate_page(const gpuvm_dev_t &vm, unsigned long long vpn, int mode, unsigned int h,
+                                             unsigned long long victim, int vdirty, unsigned int lane, unsigned int L,
+                                             BulkStage *bulk = nullptr)
 {
     unsigned char *fr = vm.pool + ((unsigned long long)h << vm.page_shift);
     if (victim != ~0ull) {
@@ -102,7 +136,21 @@ __device__ __forceinline__ void migrate_page(const gpuvm_dev_t &vm, unsigned lon
             if (vdirty) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, victim)); }
         }
     }
-    warp_copy<8, false>(fr, vm.host + (vpn << vm.page_shift), page_len(vm, vpn) >> 4, lane, 32);
+    if (bulk) {
+        int ok = 1;
+        if (lane == L) {
+            ok = bulk_copy_in(*bulk, fr, vm.host + (vpn << vm.page_shift), (unsigned int)page_len(vm, vpn),
+                              (unsigned long long)vm.spin_limit_us * 1000ull);
+            if (!ok) {
+                set_error(vm, GPUVM_E_TIMEOUT, vpn);
+                atomicXor(vm.pte + vpn, kBusy);                      /* BUSY -> INVALID */
+                st_relaxed_u32(vm.frame_vpn + h, kFrameFree);
+            }
+        }
+        if (!__shfl_sync(0xFFFFFFFFu, ok, L)) return false;
+    } else {
+        warp_copy<8, false>(fr, vm.host + (vpn << vm.page_shift), page_len(vm, vpn) >> 4, lane, 32);
+    }
     __threadfence();
     __syncwarp();
     if (lane == L) {
@@ -112,6 +160,7 @@ __device__ __forceinline__ void migrate_page(const gpuvm_dev_t &vm, unsigned lon
         stat_add(vm, kFaults, 1);
         stat_add(vm, kBytesIn, page_len(vm, vpn));
     }
+    return true;
 }
 
 }  // namespace gpuvm
@@ -129,10 +178,17 @@ __device__ __forceinline__ void gpuvm_requester_done(gpuvm_fault_queue *q)
  * within the bound, the sticky error is set and the page's entry goes back to INVALID, so
  * that its waiters give up instead of waiting forever.
  */
-static __device__ __noinline__ void gpuvm_migrator_loop(const gpuvm_dev_t vm, gpuvm_fault_queue *q)
+static __device__ __noinline__ void gpuvm_migrator_loop(const gpuvm_dev_t vm, gpuvm_fault_queue *q,
+                                                        unsigned char *stage_buf = nullptr,
+                                                        unsigned long long *stage_mbar = nullptr,
+                                                        unsigned int chunk = 0, unsigned int stages = 0)
 {
     using namespace gpuvm;
     const unsigned int lane = lane_id();
+    BulkStage bulk{stage_buf, stage_mbar, chunk, stages, 0u, 0u};
+    const bool use_bulk = stage_buf != nullptr && stages != 0u;
+    if (use_bulk && lane == 0) bulk_stage_init(bulk);
+    __syncwarp();
     volatile unsigned int *vh = &q->head, *vt = &q->tail, *vr = &q->requesters;
     unsigned int idle_ns = 32;
     for (;;) {
@@ -146,9 +202,21 @@ static __device__ __noinline__ void gpuvm_migrator_loop(const gpuvm_dev_t vm, gp
                 *slot = 0u;
             }
         }
+        if (lane == 0 && item == 0u && q->shared) {
+            gpuvm_shared_queue *g = q->shared;
+            const unsigned int h = ld_relaxed_u32(&g->head);
+            if (h != ld_relaxed_u32(&g->tail) && atomicCAS(&g->head, h, h + 1u) == h) {
+                unsigned int *slot = &g->slot[h % GPUVM_SHARED_QUEUE_SLOTS];
+                unsigned int spins = 0;
+                while ((item = ld_relaxed_u32(slot)) == 0u && ++spins < (1u << 22)) { }   /* the pusher is between its two stores */
+                st_relaxed_u32(slot, 0u);
+            }
+        }
         item = __shfl_sync(0xFFFFFFFFu, item, 0);
         if (item == 0u) {
-            const unsigned int done = (lane == 0) ? (unsigned int)(*vr == 0u && *vh == *vt) : 0u;
+            const unsigned int done = (lane == 0) ? (unsigned int)(*vr == 0u && *vh == *vt &&
+                                                                   (!q->shared || ld_relaxed_u32(&q->shared->head) ==
+                                                                                      ld_relaxed_u32(&q->shared->tail))) : 0u;
             if (__shfl_sync(0xFFFFFFFFu, done, 0)) return;
             __nanosleep(idle_ns);
             if (idle_ns < 1024) idle_ns *= 2;
@@ -182,8 +250,14 @@ static __device__ __noinline__ void gpuvm_migrator_loop(const gpuvm_dev_t vm, gp
             }
             continue;
         }
-        migrate_page(vm, vpn, mode, __shfl_sync(0xFFFFFFFFu, h, 0), __shfl_sync(0xFFFFFFFFu, victim, 0),
-                     __shfl_sync(0xFFFFFFFFu, (int)vdirty, 0), lane, 0);
+        if (!migrate_page(vm, vpn, mode, __shfl_sync(0xFFFFFFFFu, h, 0), __shfl_sync(0xFFFFFFFFu, victim, 0),
+                          __shfl_sync(0xFFFFFFFFu, (int)vdirty, 0), lane, 0, use_bulk ? &bulk : nullptr)) {
+            /* the bulk copy ran out of time: the error is set, requesters give up; let the copies
+             * still in flight land before the shared memory is given up, and stop serving */
+            if (lane == 0) bulk_stage_drain(bulk, (unsigned long long)vm.spin_limit_us * 1000ull);
+            __syncwarp();
+            return;
+        }
     }
 }
 
@@ -217,153 +291,262 @@ struct gpuvm_entry_table {
 };
 
 /*
- * The engine.  W: the table has up to 64 * W rows of 32 requests (state of a lane's requests
- * is kept in W 64-bit masks per kind).  Table: see gpuvm_entry_table.  Groups are formed with
- * __match_any_sync when the requests are registered and again, over the lanes that are not
- * finished, whenever a row is visited: a group finishes as a whole, so the lanes and the
- * leader (lowest lane) are the same every time.
+ * The engine.  Table: see gpuvm_entry_table.  The table has up to GPUVM_BATCH_ROWS_MAX rows of
+ * 32 requests.  The state of a lane's requests is two bits per row, kept in 64-bit words that
+ * the caller provides: `masks` points at the calling lane's first word, word w of kind c
+ * (0: todo, my request is not finished; 1: own, my group's page is BUSY by my compare-and-swap
+ * and not handed to a migrator yet) is masks[(c * words + w) * mask_stride] with
+ * words = ceil(rows / 64).  Shared memory with mask_stride = 32 and one base per lane, or a
+ * per-thread array with mask_stride = 1, both work; gpuvm_batch_mask_words(n) gives the count
+ * per lane.  Groups are formed with __match_any_sync when the requests are registered and
+ * again, over the lanes that are not finished, whenever a row is visited: a group finishes as
+ * a whole, so the lanes and the leader (lowest lane, it holds the group's reference) are the
+ * same every time.
+ * eager_push: a fault the warp comes to own goes to the ring while the rest of the table is
+ * still being registered, instead of after the first round of visits.  Right when the table
+ * holds all the requests the warp will ever make (the link starts at once); wrong when tables
+ * follow one another, because pages that later rows of this table would have pinned are
+ * still unprotected when the migrators look for victims (measured: 20-25 % more faults on the
+ * Zipf embedding bag).
  */
-template <int W, bool WARP_CONSUME, class Table, class Consume>
+constexpr unsigned int GPUVM_BATCH_ROWS_MAX = 1u << 16;
+#ifndef GPUVM_BATCH_REGISTER_PER_ROUND
+#define GPUVM_BATCH_REGISTER_PER_ROUND 1024u   /* words of 64 rows registered before each round of visits */
+#endif
+#ifndef GPUVM_BATCH_ACQ
+#define GPUVM_BATCH_ACQ 1
+#endif
+#ifndef GPUVM_BATCH_ROWS_AT_ONCE
+#define GPUVM_BATCH_ROWS_AT_ONCE 4     /* 1, 2, 4 or 8: rows whose memory accesses are issued together */
+#endif
+
+__host__ __device__ __forceinline__ unsigned int gpuvm_batch_mask_words(unsigned int n)
+{
+    return 2u * ((((n + 31u) >> 5) + 63u) >> 6);
+}
+
+namespace gpuvm {
+/* call a consume function; what a non-void one returns is folded into `dep` */
+template <class Consume>
+__device__ __forceinline__ void call_consume(Consume &consume, unsigned int i, const unsigned char *p, unsigned int &dep)
+{
+    if constexpr (std::is_void<decltype(consume(i, p))>::value) consume(i, p);
+    else dep ^= (unsigned int)consume(i, p);
+}
+}  // namespace gpuvm
+
+template <bool WARP_CONSUME, class Table, class Consume>
 static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm, const Table table, unsigned int n,
-                                                            int mode, Consume consume, gpuvm_fault_queue *queue)
+                                                            int mode, Consume consume, gpuvm_fault_queue *queue,
+                                                            unsigned long long *masks, unsigned int mask_stride,
+                                                            bool eager_push = false)
 {
     using namespace gpuvm;
     const unsigned int lane = lane_id();
     const unsigned int rows = (n + 31) >> 5;
-    unsigned long long todo[W], lead[W], own[W], failed[W];
-    /* bit j of word k: row 64 k + j.  todo: my request is not finished; lead: I lead my group
-     * (I hold its reference); own: my group's page is BUSY by my CAS and not handed on;
-     * failed: I gave up on the row (leader only) */
-#pragma unroll
-    for (int k = 0; k < W; ++k) { todo[k] = 0; lead[k] = 0; own[k] = 0; failed[k] = 0; }
+    const unsigned int words = (rows + 63) >> 6;
+    unsigned long long *const m_todo = masks, *const m_own = masks + (size_t)words * mask_stride;
     unsigned int served = 0;
+    constexpr bool kConsumeReturns = !std::is_void<decltype(consume(0u, static_cast<const unsigned char *>(nullptr)))>::value;
+    unsigned int n_hits = 0, n_waits = 0, n_lanes = 0;      /* this lane's share of the counters, added up at the end */
+    constexpr int R = GPUVM_BATCH_ROWS_AT_ONCE;
 
-    /* register every request in the page table (steps 1-4 of the access path) */
+    /* Register the requests of 64 rows in the page table (steps 1-4 of the access path); a
+     * fault this lane comes to own goes to the migrators at once when there is a ring.  The
+     * pin is a relaxed add: nothing is read from a frame before the acquire load of a visit. */
+    auto register_word = [&](unsigned int k) {
+        unsigned long long todo = 0, own = 0;
+        const unsigned int jn = rows - 64u * k < 64u ? rows - 64u * k : 64u;
+        for (unsigned int j0 = 0; j0 < jn; j0 += R) {          /* R rows at a time: their loads and atomics overlap */
+            unsigned int vpn[R], m[R];
+            unsigned long long old[R];
+            bool active[R], leads[R];
 #pragma unroll
-    for (int k = 0; k < W; ++k) {
-        for (unsigned int jj = 0; jj < 64 && 64u * k + jj < rows; ++jj) {
-            const unsigned int i = (64u * k + jj) * 32 + lane;
-            const bool active = i < n && table.valid(i);
-            const unsigned int m = __ballot_sync(0xFFFFFFFFu, active);
-            if (active) {
-                const unsigned int vpn = table.vpn(i);
-                const unsigned int group = __match_any_sync(m, vpn);
-                if (lane == (unsigned int)(__ffs(group) - 1)) {
-                    unsigned long long *pte = vm.pte + vpn;
-                    unsigned int frame;
-                    const int st = advance(vm, pte, pin_acquire(pte) + 1ull, mode, frame);
-                    if (st == kReady) { if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1); }
-                    else if (st == kWait) stat_add(vm, kWaits, 1);
-                    else own[k] |= 1ull << jj;
-                    if (group & (group - 1)) stat_add(vm, kLanes, __popc(group) - 1);
-                    lead[k] |= 1ull << jj;
+            for (int u = 0; u < R; ++u) {
+                const unsigned int i = (64u * k + j0 + u) * 32 + lane;
+                active[u] = j0 + u < jn && i < n && table.valid(i);
+                vpn[u] = active[u] ? table.vpn(i) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < R; ++u) m[u] = __ballot_sync(0xFFFFFFFFu, active[u]);
+#pragma unroll
+            for (int u = 0; u < R; ++u) {
+                leads[u] = false;
+                old[u] = 0;
+                if (active[u]) {
+                    const unsigned int group = __match_any_sync(m[u], vpn[u]);
+                    leads[u] = lane == (unsigned int)(__ffs(group) - 1);
+                    if (leads[u]) {
+                        old[u] = atomicAdd(vm.pte + vpn[u], 1ull);
+                        n_lanes += __popc(group) - 1;
+                    }
+                    todo |= 1ull << (j0 + u);
                 }
-                todo[k] |= 1ull << jj;
+            }
+#pragma unroll
+            for (int u = 0; u < R; ++u) {
+                if (leads[u]) {
+                    unsigned int frame;
+                    const int st = advance(vm, vm.pte + vpn[u], old[u] + 1ull, mode, frame);
+                    if (st == kReady) ++n_hits;
+                    else if (st == kWait) ++n_waits;
+                    else if (!(eager_push && queue && fault_queue_push(queue, vpn[u], mode))) own |= 1ull << (j0 + u);
+                }
             }
         }
-    }
-    __syncwarp();
+        m_todo[(size_t)k * mask_stride] = todo;
+        m_own[(size_t)k * mask_stride] = own;
+        __syncwarp();
+    };
 
+    /* Each round registers the next 64 rows and then visits every registered row, so pages that
+     * are there are used and released while the rest of the table is still being registered. */
+    unsigned int registered = 0;
     unsigned long long t_start = 0;
     unsigned int sleep_ns = 64;
     for (;;) {
-        bool progress = false, any_rows = false;
+        bool progress = false, any_rows = false, has_own = false;
+        for (unsigned int r = 0; r < GPUVM_BATCH_REGISTER_PER_ROUND && registered < words; ++r) {
+            register_word(registered++);
+            progress = true;
+        }
+        for (unsigned int k = 0; k < registered; ++k) {
+            unsigned long long todo = m_todo[(size_t)k * mask_stride], own = m_own[(size_t)k * mask_stride];
+            if (!__any_sync(0xFFFFFFFFu, todo != 0ull)) continue;
+            const unsigned long long todo_in = todo, own_in = own;
+            const unsigned int jn = rows - 64u * k < 64u ? rows - 64u * k : 64u;
+            for (unsigned int j0 = 0; j0 < jn; j0 += R) {
+                /* R rows at a time: their table entries and page-table words are fetched together */
+                unsigned int rowmask[R], vpn[R], off[R], leader[R], any = 0;
+                unsigned long long peek[R];
 #pragma unroll
-        for (int k = 0; k < W; ++k) {
-            for (unsigned int jj = 0; jj < 64 && 64u * k + jj < rows; ++jj) {
-                const unsigned long long bit = 1ull << jj;
-                const bool mine = (todo[k] & bit) != 0;
-                const unsigned int rowmask = __ballot_sync(0xFFFFFFFFu, mine);
-                if (!rowmask) continue;
+                for (int u = 0; u < R; ++u) {
+                    rowmask[u] = __ballot_sync(0xFFFFFFFFu, j0 + u < jn && ((todo >> (j0 + u)) & 1ull) != 0);
+                    any |= rowmask[u];
+                }
+                if (!any) continue;
                 any_rows = true;
-                const unsigned int i = (64u * k + jj) * 32 + lane;
-                unsigned int frame = kNotReady, off = 0;
-                unsigned long long *pte = nullptr;
-                bool is_leader = false;
-                if (mine) {
-                    const unsigned int vpn = table.vpn(i);
-                    const unsigned int leader = __ffs(__match_any_sync(rowmask, vpn)) - 1;
-                    off = table.off(i);
-                    pte = vm.pte + vpn;
-                    is_leader = (lead[k] & bit) != 0;            /* == (lane == leader) */
-                    if (is_leader) {
-                        if (failed[k] & bit) {
-                            frame = kFailed;
-                        } else if (!(own[k] & bit)) {
-                            unsigned int f;
-                            const int st = advance(vm, pte, ld_acquire_u64(pte), mode, f);   /* pairs with the publish */
-                            if (st == kReady) frame = f;
-                            else if (st == kOwn) { own[k] |= bit; progress = true; }
+#pragma unroll
+                for (int u = 0; u < R; ++u) {
+                    vpn[u] = 0; off[u] = 0;
+                    if ((rowmask[u] >> lane) & 1u) {
+                        const unsigned int i = (64u * k + j0 + u) * 32 + lane;
+                        vpn[u] = table.vpn(i);
+                        off[u] = table.off(i);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < R; ++u) {
+                    leader[u] = 32; peek[u] = 0;
+                    if ((rowmask[u] >> lane) & 1u) {
+                        leader[u] = __ffs(__match_any_sync(rowmask[u], vpn[u])) - 1;
+                        if (lane == leader[u] && !((own >> (j0 + u)) & 1ull)) peek[u] = ld_relaxed_u64(vm.pte + vpn[u]);
+                    }
+                }
+                /* leaders: what the entries say.  An entry that looks VALID is read again with
+                 * acquire (it pairs with the fence before the publish); a VALID that turns up any
+                 * other way gets a fence. */
+                unsigned int frame[R];
+                bool need_fence = false;
+#pragma unroll
+                for (int u = 0; u < R; ++u) {
+                    frame[u] = kNotReady;
+                    const unsigned long long bit = 1ull << (j0 + u);
+                    if (lane == leader[u] && !(own & bit)) {
+                        unsigned long long w = peek[u];
+                        const bool looks_valid = (w & kStMask) == kValid;
+                        if (GPUVM_BATCH_ACQ == 1 && looks_valid) w = ld_acquire_u64(vm.pte + vpn[u]);
+                        unsigned int f;
+                        const int st = advance(vm, vm.pte + vpn[u], w, mode, f);
+                        if (st == kReady) { frame[u] = f; need_fence |= GPUVM_BATCH_ACQ == 2 || (GPUVM_BATCH_ACQ == 1 && !looks_valid); }
+                        else if (st == kOwn) { own |= bit; progress = true; }
+                    }
+                }
+                if (__any_sync(0xFFFFFFFFu, need_fence)) __threadfence();
+                /* followers take the frame from their leader; every ready request is consumed */
+                bool any_ready = false;
+                unsigned int dep = 0;          /* what consume returned, folded: see below */
+#pragma unroll
+                for (int u = 0; u < R; ++u) {
+                    if (!rowmask[u]) continue;
+                    const bool mine = ((rowmask[u] >> lane) & 1u) != 0;
+                    if (mine) frame[u] = __shfl_sync(rowmask[u], frame[u], leader[u]);
+                    const bool ready = mine && frame[u] != kNotReady;
+                    if (WARP_CONSUME) {
+                        unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
+                        while (ready_lanes) {
+                            const unsigned int L = __ffs(ready_lanes) - 1;
+                            ready_lanes &= ready_lanes - 1;
+                            const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame[u], L), o = __shfl_sync(0xFFFFFFFFu, off[u], L);
+                            call_consume(consume, (64u * k + j0 + u) * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o, dep);
+                        }
+                    } else if (ready) {
+                        call_consume(consume, (64u * k + j0 + u) * 32 + lane,
+                                     vm.pool + ((unsigned long long)frame[u] << vm.page_shift) + off[u], dep);
+                    }
+                    any_ready |= ready;
+                }
+                /* step 8 for all of them.  The decrements must not overtake the groups' accesses
+                 * to their frames.  A consume that only reads and returns (something computed
+                 * from) what it read gives the engine a value that does not exist before the
+                 * loads have returned: `hold` below is zero, but it is computed from those values
+                 * of all 32 lanes, so the decrement that adds it cannot be issued earlier.  Any
+                 * other consume, and write mode, get a warp barrier and a fence instead. */
+                if (__any_sync(0xFFFFFFFFu, any_ready)) {
+                    unsigned long long hold = 0;
+                    if (kConsumeReturns && mode == kRead) {
+                        hold = __ballot_sync(0xFFFFFFFFu, (dep & (vm.n_frames >> 31)) != 0u);   /* n_frames < 2^31 */
+                    } else {
+                        __syncwarp();
+                        __threadfence();
+                    }
+#pragma unroll
+                    for (int u = 0; u < R; ++u) {
+                        if (((rowmask[u] >> lane) & 1u) && frame[u] != kNotReady) {
+                            todo &= ~(1ull << (j0 + u));
+                            ++served;
+                            if (lane == leader[u]) atomicAdd(vm.pte + vpn[u], ~0ull + hold);
                         }
                     }
-                    frame = __shfl_sync(rowmask, frame, leader);
-                    if (frame == kFailed) todo[k] &= ~bit;
-                }
-                const bool ready = mine && frame < kFailed;
-                if (WARP_CONSUME) {
-                    unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
-                    while (ready_lanes) {
-                        const unsigned int L = __ffs(ready_lanes) - 1;
-                        ready_lanes &= ready_lanes - 1;
-                        const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame, L), o = __shfl_sync(0xFFFFFFFFu, off, L);
-                        consume((64u * k + jj) * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o);
-                    }
-                    __syncwarp();                               /* every group has used its frame */
-                } else {
-                    if (ready) consume(i, vm.pool + ((unsigned long long)frame << vm.page_shift) + off);
-                    if (mine) __syncwarp(rowmask);              /* the whole group has used the frame */
-                }
-                if (ready) {
-                    todo[k] &= ~bit;
-                    ++served;
                     progress = true;
-                    if (is_leader) unpin(pte);                  /* step 8 */
                 }
             }
-        }
-        if (!any_rows) break;
-
-        if (queue) {
-            /* hand owned faults to the migrator warps; afterwards wait for the page like anyone */
-#pragma unroll
-            for (int k = 0; k < W; ++k)
-                while (own[k]) {
-                    const unsigned int jj = __ffsll((long long)own[k]) - 1;
+            if (queue) {
+                /* hand owned faults to the migrator warps; afterwards wait for the page like anyone */
+                while (own) {
+                    const unsigned int jj = __ffsll((long long)own) - 1;
                     if (!fault_queue_push(queue, table.vpn((64u * k + jj) * 32 + lane), mode)) break;
-                    own[k] &= own[k] - 1;
+                    own &= own - 1;
                     progress = true;
                 }
-        } else {
+            }
+            has_own |= own != 0ull;
+            if (todo != todo_in) m_todo[(size_t)k * mask_stride] = todo;
+            if (own != own_in) m_own[(size_t)k * mask_stride] = own;
+        }
+        if (!any_rows && registered == words) break;
+
+        if (!queue) {
             /* no helpers: the first lane that owns a fault takes a frame and the warp migrates the page */
-            bool has_own = false;
-#pragma unroll
-            for (int k = 0; k < W; ++k) has_own |= own[k] != 0;
             const unsigned int owners = __ballot_sync(0xFFFFFFFFu, has_own);
             if (owners) {
                 const unsigned int L = __ffs(owners) - 1;
-                unsigned int h = 0, vpn = 0;
-                unsigned long long victim = ~0ull;
+                unsigned int h = 0, vpn = 0, kk = 0;
+                unsigned long long victim = ~0ull, word = 0;
                 bool vdirty = false;
                 int claimed = 0;
                 if (lane == L) {
-                    int kk = 0;
-#pragma unroll
-                    for (int k = W - 1; k >= 0; --k) if (own[k]) kk = k;
-                    unsigned long long word = 0;
-#pragma unroll
-                    for (int k = 0; k < W; ++k) if (k == kk) word = own[k];
-                    vpn = table.vpn((64u * kk + (__ffsll((long long)word) - 1)) * 32 + lane);
-                    claimed = try_claim(vm, vpn, 4, h, victim, vdirty);
+                    for (kk = 0; kk < registered; ++kk)
+                        if ((word = m_own[(size_t)kk * mask_stride]) != 0ull) break;
+                    if (word) {
+                        vpn = table.vpn((64u * kk + (__ffsll((long long)word) - 1)) * 32 + lane);
+                        claimed = try_claim(vm, vpn, 4, h, victim, vdirty);
+                    }
                 }
                 if (__shfl_sync(0xFFFFFFFFu, claimed, L)) {
                     migrate_page(vm, __shfl_sync(0xFFFFFFFFu, vpn, L), mode, __shfl_sync(0xFFFFFFFFu, h, L),
                                  __shfl_sync(0xFFFFFFFFu, victim, L), __shfl_sync(0xFFFFFFFFu, (int)vdirty, L), lane, L);
-                    if (lane == L) {
-                        bool cleared = false;
-#pragma unroll
-                        for (int k = 0; k < W; ++k)
-                            if (!cleared && own[k]) { own[k] &= own[k] - 1; cleared = true; }
-                    }
+                    if (lane == L) m_own[(size_t)kk * mask_stride] = word & (word - 1);
                     progress = true;
                 }
             }
@@ -376,25 +559,41 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
         bool expired = (t - t_start) > (unsigned long long)vm.spin_limit_us * 1000ull || has_error(vm);
         expired = __any_sync(0xFFFFFFFFu, expired);
         if (expired) {
-#pragma unroll
-            for (int k = 0; k < W; ++k) {
-                unsigned long long give_up = todo[k] & lead[k] & ~failed[k];
-                while (give_up) {
-                    const unsigned int jj = __ffsll((long long)give_up) - 1;
-                    give_up &= give_up - 1;
+            /* every request that is left is abandoned: its group's leader drops the reference
+             * (and takes back a fault it still owns), nobody consumes */
+            for (unsigned int k = 0; k < registered; ++k) {
+                const unsigned long long todo = m_todo[(size_t)k * mask_stride], own = m_own[(size_t)k * mask_stride];
+                const unsigned int jn = rows - 64u * k < 64u ? rows - 64u * k : 64u;
+                for (unsigned int jj = 0; jj < jn; ++jj) {
+                    const bool mine = ((todo >> jj) & 1ull) != 0;
+                    const unsigned int rowmask = __ballot_sync(0xFFFFFFFFu, mine);
+                    if (!mine) continue;
                     const unsigned int vpn = table.vpn((64u * k + jj) * 32 + lane);
-                    set_error(vm, GPUVM_E_TIMEOUT, vpn);
-                    if ((own[k] >> jj) & 1ull) atomicXor(vm.pte + vpn, kBusy);   /* BUSY -> INVALID: never handed on */
-                    unpin(vm.pte + vpn);
-                    own[k] &= ~(1ull << jj);
-                    failed[k] |= 1ull << jj;
+                    if (lane == (unsigned int)(__ffs(__match_any_sync(rowmask, vpn)) - 1)) {
+                        set_error(vm, GPUVM_E_TIMEOUT, vpn);
+                        if ((own >> jj) & 1ull) atomicXor(vm.pte + vpn, kBusy);   /* BUSY -> INVALID: never handed on */
+                        unpin(vm.pte + vpn);
+                    }
                 }
+                m_todo[(size_t)k * mask_stride] = 0ull;
+                m_own[(size_t)k * mask_stride] = 0ull;
             }
-            continue;                                           /* followers learn of it in the next round */
+            break;
         }
         if (lane == 0) stat_add(vm, kRetries, 1);
         __nanosleep(sleep_ns);
         if (sleep_ns < 4096) sleep_ns *= 2;
+    }
+    __syncwarp();
+    for (int o = 16; o; o >>= 1) {
+        n_hits += __shfl_down_sync(0xFFFFFFFFu, n_hits, o);
+        n_waits += __shfl_down_sync(0xFFFFFFFFu, n_waits, o);
+        n_lanes += __shfl_down_sync(0xFFFFFFFFu, n_lanes, o);
+    }
+    if (lane == 0) {
+        if (GPUVM_COUNT_HITS && n_hits) stat_add(vm, kHits, n_hits);
+        if (n_waits) stat_add(vm, kWaits, n_waits);
+        if (n_lanes) stat_add(vm, kLanes, n_lanes);
     }
     return served;
 }
@@ -405,7 +604,9 @@ static __device__ __forceinline__ unsigned int gpuvm_batch_access(const gpuvm_de
                                                                   unsigned int n, int mode, Consume consume,
                                                                   gpuvm_fault_queue *queue = nullptr)
 {
-    return gpuvm_batch_run<1, WARP_CONSUME>(vm, gpuvm_entry_table{table}, n, mode, consume, queue);
+    unsigned long long masks[2] = {0ull, 0ull};
+    return gpuvm_batch_run<WARP_CONSUME>(vm, gpuvm_entry_table{table}, n < GPUVM_BATCH_MAX ? n : GPUVM_BATCH_MAX, mode,
+                                         consume, queue, masks, 1u);
 }
 
 #endif /* GPUVM_BATCH_CUH */

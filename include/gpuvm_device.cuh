@@ -251,6 +251,107 @@ __device__ __forceinline__ void warp_copy(unsigned char *dst, const unsigned cha
     }
 }
 
+/*
+ * Page copy by the bulk-copy unit (cp.async.bulk): one thread moves a page host -> shared
+ * memory -> frame in pieces of `chunk` bytes through `stages` staging buffers, each with its
+ * own mbarrier.  The copies do not pass through the load/store unit or registers, so a single
+ * thread keeps stages * chunk bytes in flight (a warp copying through registers has 4 KiB)
+ * and the warps that issue ordinary loads are not queued behind the migration traffic.
+ * The staging memory belongs to the calling warp; buf is 128-byte aligned, chunk a multiple
+ * of 16.  All addresses and lengths of the path are multiples of 16 bytes by construction
+ * (page sizes are powers of two >= 16, the backing store is 16-byte aligned and a multiple of
+ * 16 bytes long).
+ */
+struct BulkStage {
+    unsigned char *buf;            /* stages * chunk bytes of shared memory */
+    unsigned long long *mbar;      /* `stages` mbarriers in shared memory   */
+    unsigned int chunk, stages;
+    unsigned int phases;           /* bit s: parity the next wait on mbar[s] uses */
+    unsigned int pending;          /* bit s: a copy into stage s has been issued and not waited for */
+};
+
+__device__ __forceinline__ unsigned int smem_addr(const void *p) { return (unsigned int)__cvta_generic_to_shared(p); }
+
+/* one thread, once, before the first copy */
+__device__ __forceinline__ void bulk_stage_init(BulkStage &s)
+{
+    for (unsigned int i = 0; i < s.stages; ++i)
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(s.mbar + i)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    s.phases = 0;
+    s.pending = 0;
+}
+
+/* one thread: wait for the copy into stage `st`; false when `limit_ns` went by first */
+__device__ __forceinline__ bool bulk_stage_wait(BulkStage &s, unsigned int st, unsigned long long limit_ns)
+{
+    const unsigned int mb = smem_addr(s.mbar + st), parity = (s.phases >> st) & 1u;
+    unsigned long long t0 = 0;
+    for (unsigned int spins = 0;; ++spins) {
+        unsigned int ok;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(ok) : "r"(mb), "r"(parity) : "memory");
+        if (ok) break;
+        if ((spins & 63u) == 63u) {
+            const unsigned long long t = now_ns();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > limit_ns) return false;
+        }
+    }
+    s.phases ^= 1u << st;
+    s.pending &= ~(1u << st);
+    return true;
+}
+
+/* one thread, after a failed copy: give the copies still in flight one more bounded wait each */
+__device__ __forceinline__ void bulk_stage_drain(BulkStage &s, unsigned long long limit_ns)
+{
+    for (unsigned int st = 0; st < s.stages; ++st)
+        if ((s.pending >> st) & 1u) bulk_stage_wait(s, st, limit_ns);
+}
+
+/*
+ * One thread: copy `bytes` from the backing store to a frame.  Returns false when a wait ran
+ * out; copies may then still be in flight into the staging buffers (the caller sets the
+ * sticky error and waits once more, bounded, before it gives the shared memory up).
+ * On success every byte is in the frame: the group wait covers the writes, the proxy fence
+ * orders them before the generic-proxy publish that follows in the caller.
+ */
+__device__ __forceinline__ bool bulk_copy_in(BulkStage &s, unsigned char *frame, const unsigned char *src,
+                                             unsigned int bytes, unsigned long long limit_ns)
+{
+    const unsigned int nchunks = (bytes + s.chunk - 1) / s.chunk;
+    auto issue = [&](unsigned int c, unsigned int st) {
+        const unsigned int len = bytes - c * s.chunk < s.chunk ? bytes - c * s.chunk : s.chunk;
+        const unsigned int mb = smem_addr(s.mbar + st);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mb), "r"(len) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_addr(s.buf + (size_t)st * s.chunk)), "l"(__cvta_generic_to_global(src + (size_t)c * s.chunk)),
+                       "r"(len), "r"(mb) : "memory");
+        s.pending |= 1u << st;
+    };
+    unsigned int issued = 0;
+    while (issued < nchunks && issued < s.stages) { issue(issued, issued); ++issued; }
+    for (unsigned int done = 0; done < nchunks; ++done) {
+        const unsigned int st = done % s.stages;
+        const unsigned int len = bytes - done * s.chunk < s.chunk ? bytes - done * s.chunk : s.chunk;
+        if (!bulk_stage_wait(s, st, limit_ns)) return false;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     ::"l"(__cvta_generic_to_global(frame + (size_t)done * s.chunk)), "r"(smem_addr(s.buf + (size_t)st * s.chunk)),
+                       "r"(len) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        if (issued < nchunks) {
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   /* the buffer has been read */
+            issue(issued, st);
+            ++issued;
+        }
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    return true;
+}
+
 /* ------------------------------------------------------------ fault machinery */
 
 enum LaneState { kNew = 0, kWait, kOwn, kReady, kDone, kFail };

@@ -63,6 +63,8 @@ SYMBOLS = {
     "gpuvm_check": (_i, [_vp, ctypes.POINTER(Check)]),
     "gpuvm_set_policy": (_i, [_vp, _i]),
     "gpuvm_set_spin_limit_us": (_i, [_vp, ctypes.c_uint]),
+    "gpuvm_set_scratch_limit": (_i, [_vp, ctypes.c_size_t]),
+    "gpuvm_scratch_bytes": (ctypes.c_size_t, [_vp]),
     "gpuvm_safe_warps": (_i, [_vp, _i]),
     "gpuvm_inflight_pages": (ctypes.c_double, [ctypes.c_double, ctypes.c_double, ctypes.c_double]),
     "gpuvm_debug_poke_pte": (_i, [_vp, _u64, _u64]),
@@ -197,6 +199,14 @@ def gpuvm_check(h, raise_on_error: bool = True) -> dict:
 
 def gpuvm_set_policy(h, policy: int):
     _check(lib().gpuvm_set_policy(h, policy), "gpuvm_set_policy")
+
+
+def gpuvm_set_scratch_limit(h, nbytes: int):
+    _check(lib().gpuvm_set_scratch_limit(h, nbytes), "gpuvm_set_scratch_limit")
+
+
+def gpuvm_scratch_bytes(h) -> int:
+    return int(lib().gpuvm_scratch_bytes(h))
 
 
 def gpuvm_set_spin_limit_us(h, us: int):

@@ -21,6 +21,7 @@ struct gpuvm_handle {
     unsigned long long *check_buf;   // device, 8 words
     void *scratch;                   // device scratch for workload kernels (request tables)
     size_t scratch_bytes;
+    size_t scratch_limit;      /* 0: none */
 };
 
 namespace {
@@ -281,6 +282,17 @@ void *gpuvm_scratch_(gpuvm_handle *h, size_t bytes)
     h->scratch_bytes = bytes;
     return h->scratch;
 }
+
+size_t gpuvm_scratch_limit_(gpuvm_handle *h) { return h && h->scratch_limit ? h->scratch_limit : ~size_t(0); }
+
+int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes)
+{
+    if (!h) return GPUVM_E_ARG;
+    h->scratch_limit = bytes;
+    return GPUVM_OK;
+}
+
+size_t gpuvm_scratch_bytes(gpuvm_t h) { return h ? h->scratch_bytes : 0; }
 
 int gpuvm_device_view(gpuvm_t h, gpuvm_dev_t *out)
 {

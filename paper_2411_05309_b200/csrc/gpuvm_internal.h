@@ -12,6 +12,8 @@ void gpuvm_note_launch_(unsigned long long n);
  * allocation fails.  Growing synchronises the device. */
 struct gpuvm_handle;
 void *gpuvm_scratch_(struct gpuvm_handle *h, size_t bytes);
+/* bound set with gpuvm_set_scratch_limit, SIZE_MAX when there is none */
+size_t gpuvm_scratch_limit_(struct gpuvm_handle *h);
 #ifdef __cplusplus
 }
 #endif

@@ -141,8 +141,10 @@ __global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long lo
 constexpr int kGatherRequesters = 28;
 constexpr int kGatherMigrators = 4;
 constexpr int kGatherMaxWarps = 32;
-constexpr unsigned int kGatherBatch = 4096;              // requests per requester warp: 128 rows of 32
+constexpr unsigned int kGatherBatch = 16384;             // most requests per requester warp: 512 rows of 32
 constexpr unsigned int kNoIndex = 0xFFFFFFFFu;
+constexpr unsigned int kGatherChunk = 8192;              // bytes per bulk copy of a migrator warp
+constexpr unsigned int kGatherStages = 2;                // staging buffers per migrator warp
 
 // Request table of the gather: one 32-bit element index per request (the array has fewer than
 // 2^32 - 1 elements), replaced by the value's bit pattern when the request is served.
@@ -163,20 +165,30 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
                                                                                unsigned long long n_idx, unsigned long long block,
                                                                                float *__restrict__ fsum, long long *__restrict__ bsum,
                                                                                int requesters, unsigned int batch,
-                                                                               unsigned int *g_tables)
+                                                                               unsigned int *g_tables, unsigned int stage_chunk,
+                                                                               unsigned int stage_count, bool one_pass,
+                                                                               gpuvm_shared_queue *shared_queue)
 {
     __shared__ gpuvm_fault_queue queue_s;
+    // dynamic: per requester warp its mask words x 32 lanes; per migrator warp its staging
+    // buffers for the bulk copies; the mbarriers of those
+    extern __shared__ __align__(128) unsigned long long gather_masks[];
     gpuvm_fault_queue *queue = &queue_s;
     const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
         reinterpret_cast<unsigned int *>(queue)[k] = 0;
     __syncthreads();
-    if (threadIdx.x == 0) queue->requesters = (unsigned int)requesters;
+    if (threadIdx.x == 0) { queue->requesters = (unsigned int)requesters; queue->shared = shared_queue; }
     __syncthreads();
     if ((int)warp >= requesters) {
-        gpuvm_migrator_loop(vm, queue);
+        const unsigned int mig = warp - requesters, n_mig = (blockDim.x >> 5) - requesters;
+        unsigned char *stage0 = reinterpret_cast<unsigned char *>(gather_masks + (size_t)requesters * gpuvm_batch_mask_words(batch) * 32);
+        unsigned long long *mbar0 = reinterpret_cast<unsigned long long *>(stage0 + (size_t)n_mig * stage_count * stage_chunk);
+        gpuvm_migrator_loop(vm, queue, stage_count ? stage0 + (size_t)mig * stage_count * stage_chunk : nullptr,
+                            mbar0 + (size_t)mig * stage_count, stage_chunk, stage_count);
         return;
     }
+    unsigned long long *masks = gather_masks + (size_t)warp * gpuvm_batch_mask_words(batch) * 32 + lane;
     unsigned int *table = g_tables + ((size_t)blockIdx.x * requesters + warp) * batch;
     const unsigned long long n_elems = (vm.bytes - x_off) / 4;
     const unsigned long long nb = (n_idx + block - 1) / block;
@@ -196,10 +208,12 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
                 table[k] = i < n_elems ? (unsigned int)i : kNoIndex;
             }
             __syncwarp();
-            gpuvm_batch_run<2, false>(vm, GatherTable{table, x_off, vm.page_shift}, n, GPUVM_READ,
-                                      [table](unsigned int i, const unsigned char *p) {
-                                          table[i] = gpuvm_load(reinterpret_cast<const unsigned int *>(p));
-                                      }, queue);
+            gpuvm_batch_run<false>(vm, GatherTable{table, x_off, vm.page_shift}, n, GPUVM_READ,
+                                   [table](unsigned int i, const unsigned char *p) {
+                                       const unsigned int v = gpuvm_load(reinterpret_cast<const unsigned int *>(p));
+                                       table[i] = v;
+                                       return v;                  // read-only consume: lets the engine skip its fence
+                                   }, queue, masks, 32u, one_pass);
             __syncwarp();
             // sum the values of this piece, index block by index block (a rejected index left
             // kNoIndex in its slot and has set the sticky error: the sums are then meaningless)
@@ -613,11 +627,14 @@ __global__ void __launch_bounds__(256) embag_kernel(Mem m, unsigned long long t_
 constexpr int kEmbagRequesters = 28;
 constexpr int kEmbagMigrators = 4;
 constexpr unsigned int kEmbagLookups = 32;                 // lookups of a bag per batch (table rows)
+constexpr unsigned int kEmbagMaxGroups = 8;                // groups of 32 bags a requester warp takes at a time
 
 __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
                                                               const long long *__restrict__ rows, unsigned long long n_bags,
                                                               unsigned int bag, float *__restrict__ out, int requesters,
-                                                              gpuvm_batch_entry *g_tables, unsigned char *g_staging)
+                                                              gpuvm_batch_entry *g_tables, unsigned char *g_staging,
+                                                              unsigned int groups, bool one_pass,
+                                                              gpuvm_shared_queue *shared_queue)
 {
     __shared__ gpuvm_fault_queue queue_s;
     gpuvm_fault_queue *queue = &queue_s;
@@ -625,7 +642,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
     for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
         reinterpret_cast<unsigned int *>(queue)[k] = 0;
     __syncthreads();
-    if (threadIdx.x == 0) queue->requesters = (unsigned int)requesters;
+    if (threadIdx.x == 0) { queue->requesters = (unsigned int)requesters; queue->shared = shared_queue; }
     __syncthreads();
     if ((int)warp >= requesters) {
         gpuvm_migrator_loop(vm, queue);
@@ -634,36 +651,48 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
     const unsigned int q = dims >> 2;                            // 16-byte pieces per row
     const unsigned long long row_bytes = 4ull * dims;
     const size_t slot = (size_t)blockIdx.x * requesters + warp;
-    gpuvm_batch_entry *table = g_tables + slot * (32 * kEmbagLookups);
-    uint4 *staging = reinterpret_cast<uint4 *>(g_staging + slot * (32 * kEmbagLookups) * row_bytes);
-    const unsigned long long items = (n_bags + 31) / 32;
+    const size_t per_warp = (size_t)groups * 32 * (bag < kEmbagLookups ? bag : kEmbagLookups);
+    gpuvm_batch_entry *table = g_tables + slot * per_warp;
+    uint4 *staging = reinterpret_cast<uint4 *>(g_staging + slot * per_warp * row_bytes);
+    unsigned long long masks[2 * ((kEmbagMaxGroups * kEmbagLookups + 63) / 64)];
+    const unsigned long long per_item = 32ull * groups;
+    const unsigned long long items = (n_bags + per_item - 1) / per_item;
     const unsigned long long stride = (unsigned long long)gridDim.x * requesters;
     for (unsigned long long t = slot; t < items; t += stride) {
-        const unsigned long long g0 = 32 * t;
+        const unsigned long long g0 = per_item * t;
         for (unsigned int k0 = 0; k0 < bag; k0 += kEmbagLookups) {
             const unsigned int nk = bag - k0 < kEmbagLookups ? bag - k0 : kEmbagLookups;
-            // request (k, b): lookup k0 + k of bag g0 + b
-            for (unsigned int k = 0; k < nk; ++k) {
-                const unsigned long long g = g0 + lane;
-                if (g < n_bags)
-                    gpuvm_batch_set(vm, table, k * 32 + lane,
-                                    t_off + (unsigned long long)rows[g * bag + k0 + k] * row_bytes);
-                else
-                    gpuvm_batch_skip(table, k * 32 + lane);
-            }
+            // request ((gi * nk + k) * 32 + b): lookup k0 + k of bag g0 + 32 gi + b
+            for (unsigned int gi = 0; gi < groups; ++gi)
+                for (unsigned int k = 0; k < nk; ++k) {
+                    const unsigned long long g = g0 + 32ull * gi + lane;
+                    if (g < n_bags)
+                        gpuvm_batch_set(vm, table, (gi * nk + k) * 32 + lane,
+                                        t_off + (unsigned long long)rows[g * bag + k0 + k] * row_bytes);
+                    else
+                        gpuvm_batch_skip(table, (gi * nk + k) * 32 + lane);
+                }
             __syncwarp();
-            gpuvm_batch_access<true>(vm, table, nk * 32, GPUVM_READ, [=](unsigned int i, const unsigned char *p) {
-                if (lane < q) staging[(size_t)i * q + lane] = gpuvm_load16(p + 16u * lane);
-            }, queue);
+            gpuvm_batch_run<true>(vm, gpuvm_entry_table{table}, groups * nk * 32, GPUVM_READ,
+                                         [=](unsigned int i, const unsigned char *p) {
+                unsigned int seen = 0;                             // read-only consume: lets the engine skip its fence
+                if (lane < q) {
+                    const uint4 v = gpuvm_load16(p + 16u * lane);
+                    staging[(size_t)i * q + lane] = v;
+                    seen = v.x;
+                }
+                return seen;
+            }, queue, masks, 1u, one_pass);
             __syncwarp();
             // add the staged rows of each bag in list order
-            for (unsigned int b = 0; b < 32 && g0 + b < n_bags; ++b) {
+            for (unsigned int gb = 0; gb < 32 * groups && g0 + gb < n_bags; ++gb) {
                 if (lane < q) {
-                    float4 *dst = reinterpret_cast<float4 *>(out + (g0 + b) * dims) + lane;
+                    const unsigned int gi = gb >> 5, b = gb & 31;
+                    float4 *dst = reinterpret_cast<float4 *>(out + (g0 + gb) * dims) + lane;
                     float4 acc = k0 == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *dst;
 #pragma unroll 8
                     for (unsigned int k = 0; k < nk; ++k) {
-                        const uint4 v = staging[(size_t)(k * 32 + b) * q + lane];
+                        const uint4 v = staging[(size_t)((gi * nk + k) * 32 + b) * q + lane];
                         acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
                         acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
                         acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
@@ -784,6 +813,21 @@ int launched(unsigned long long n = 1)
     gpuvm_note_launch_(n);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? GPUVM_OK : GPUVM_E_CUDA;
+}
+
+// The grid-wide fault ring of a batched kernel, zeroed on the stream; nullptr when pages are
+// small.  Sharing the backlog pays when one page takes a migrator warp long to move (a 2 MiB
+// page: 0.8 ms, so a block that owns more faults than the others finishes long after them:
+// 1.52 s -> 1.34 s on the embedding bag); with 64 KiB pages the blocks' backlogs even out by
+// themselves and the extra migrators only add to the contention for frames (23.2 -> 24.0 ms
+// on the gather).
+constexpr size_t kSharedQueueMinPage = size_t(256) << 10;
+
+gpuvm_shared_queue *shared_queue_at(const gpuvm_dev_t &vm, unsigned char *where, cudaStream_t stream)
+{
+    if ((size_t(1) << vm.page_shift) < kSharedQueueMinPage) return nullptr;
+    if (cudaMemsetAsync(where, 0, sizeof(gpuvm_shared_queue), stream) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return reinterpret_cast<gpuvm_shared_queue *>(where);
 }
 
 bool view_of(gpuvm_t h, Paged &m) { return h && gpuvm_device_view(h, &m.vm) == GPUVM_OK; }
@@ -1049,17 +1093,38 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     if (n_idx == 0) return GPUVM_OK;
     if ((m.vm.bytes - x_off) / 4 >= kNoIndex) return GPUVM_E_RANGE;      // element indices are staged as 32-bit numbers
     const int requesters = kGatherRequesters, migrators = kGatherMigrators;
-    const unsigned int batch = kGatherBatch;
+    // Requests per requester warp: all of a warp's share of the index list when that is at most
+    // kGatherBatch (then every page is fetched once per run), whole index blocks, at least 2048.
+    const size_t warps_all = (size_t)sm_count() * requesters;
+    size_t share = (n_idx + warps_all - 1) / warps_all;
+    if (block <= kGatherBatch) share = (share + block - 1) / block * block;
+    unsigned int batch = 2048;
+    while (batch < kGatherBatch && batch < share && warps_all * (size_t)batch * 2 * sizeof(unsigned int) <= gpuvm_scratch_limit_(h))
+        batch *= 2;
     const size_t nb = (n_idx + block - 1) / block;
     const size_t per = block <= batch ? batch / block : 1;
     const size_t items = (nb + per - 1) / per;
     const size_t blocks_needed = (items + requesters - 1) / requesters;
     const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
-    unsigned int *tables = static_cast<unsigned int *>(gpuvm_scratch_(h, (size_t)grid * requesters * batch * sizeof(unsigned int)));
+    const size_t slots = items < (size_t)grid * requesters ? items : (size_t)grid * requesters;   // warps that get work
+    const size_t tables_bytes = (slots * batch * sizeof(unsigned int) + 255) & ~size_t(255);
+    unsigned int *tables = static_cast<unsigned int *>(gpuvm_scratch_(h, tables_bytes + sizeof(gpuvm_shared_queue)));
     if (!tables) return GPUVM_E_ALLOC;
-    gather_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+    gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, reinterpret_cast<unsigned char *>(tables) + tables_bytes,
+                                                       static_cast<cudaStream_t>(stream));
+    // staging of the migrator warps: kGatherStages pieces of at most kGatherChunk bytes each
+    const unsigned int stage_chunk = (unsigned int)((size_t(1) << m.vm.page_shift) < kGatherChunk ? (size_t(1) << m.vm.page_shift) : kGatherChunk);
+    const unsigned int stage_count = stage_chunk >= 128 ? kGatherStages : 0;     // tiny pages: copy through registers
+    const size_t mask_bytes = (size_t)requesters * gpuvm_batch_mask_words(batch) * 32 * sizeof(unsigned long long) +
+                              (size_t)migrators * stage_count * (stage_chunk + sizeof(unsigned long long));
+    if (mask_bytes > 40 * 1024 &&
+        cudaFuncSetAttribute(gather_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mask_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return GPUVM_E_CUDA;
+    }
+    gather_batch_kernel<<<grid, (requesters + migrators) * 32, mask_bytes, static_cast<cudaStream_t>(stream)>>>(
         m.vm, x_off, reinterpret_cast<const long long *>(d_idx), n_idx, block, d_fsum, reinterpret_cast<long long *>(d_bsum),
-        requesters, batch, tables);
+        requesters, batch, tables, stage_chunk, stage_count, /* one_pass = */ items <= (size_t)grid * requesters, shared_queue);
     return launched();
 }
 
@@ -1146,17 +1211,28 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     if (t_off % 16) return GPUVM_E_ALIGN;
     if (n_bags == 0) return GPUVM_OK;
     const int requesters = kEmbagRequesters, migrators = kEmbagMigrators;
-    const size_t items = (n_bags + 31) / 32;
+    // Groups of 32 bags per requester warp: enough for every bag to be in flight at once when
+    // that takes at most kEmbagMaxGroups, within the scratch bound (table + staged rows).
+    const size_t warps_all = (size_t)sm_count() * requesters;
+    const size_t lookups_now = bag < kEmbagLookups ? bag : kEmbagLookups;
+    unsigned int groups = 1;
+    while (groups < kEmbagMaxGroups && (n_bags + 32 * groups - 1) / (32 * groups) > warps_all &&
+           warps_all * (2 * groups) * 32 * lookups_now * (sizeof(gpuvm_batch_entry) + 4 * dims) <= gpuvm_scratch_limit_(h))
+        groups *= 2;
+    const size_t items = (n_bags + 32 * groups - 1) / (32 * groups);
     const size_t blocks_needed = (items + requesters - 1) / requesters;
     const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
-    const size_t per_warp = 32 * kEmbagLookups;
-    const size_t table_bytes = ((size_t)grid * requesters * per_warp * sizeof(gpuvm_batch_entry) + 255) & ~size_t(255);
-    const size_t staging_bytes = (size_t)grid * requesters * per_warp * 4 * dims;
-    unsigned char *scratch = static_cast<unsigned char *>(gpuvm_scratch_(h, table_bytes + staging_bytes));
+    const size_t per_warp = (size_t)groups * 32 * lookups_now;
+    const size_t slots = items < (size_t)grid * requesters ? items : (size_t)grid * requesters;   // warps that get work
+    const size_t table_bytes = (slots * per_warp * sizeof(gpuvm_batch_entry) + 255) & ~size_t(255);
+    const size_t staging_bytes = (slots * per_warp * 4 * dims + 255) & ~size_t(255);
+    unsigned char *scratch = static_cast<unsigned char *>(gpuvm_scratch_(h, table_bytes + staging_bytes + sizeof(gpuvm_shared_queue)));
     if (!scratch) return GPUVM_E_ALLOC;
+    gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, scratch + table_bytes + staging_bytes, static_cast<cudaStream_t>(stream));
     embag_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
         m.vm, t_off, (unsigned int)dims, reinterpret_cast<const long long *>(d_rows), n_bags, (unsigned int)bag, d_out,
-        requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes);
+        requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes, groups,
+        /* one_pass = */ items <= (size_t)grid * requesters && bag <= kEmbagLookups, shared_queue);
     return launched();
 }
 
@@ -1327,3 +1403,4 @@ int gpuvm_link_peak(void *host_ptr, void *d_buf, size_t bytes, int reps, double 
 }
 
 }  // extern "C"
+
