@@ -314,6 +314,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     link = measure_link(torch, B)
     w = configs.make(args.workload, args.shrink)
+    if args.scratch_limit_mib:
+        B.gpuvm_set_scratch_limit(w.h, args.scratch_limit_mib << 20)
     for _ in range(args.warmup):
         w.run(check=False)
     sampler = ClockSampler(local_rank, args.clock_period)
@@ -366,6 +368,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             "fault_rate_ceiling_per_s": link["ce_h2d_gbs"] * 1e9 / w.page_bytes,
         },
         "link_peak": link,
+        "scratch": {"bytes": B.gpuvm_scratch_bytes(w.h), "limit_bytes": args.scratch_limit_mib << 20,
+                    "what": "device memory of the workload beside the pool: request tables, staged rows, queues"},
         "stats": st, "invariants": ck,
         "roofline": {
             "bound": "host_link", "achieved": moved / kern_s / 1e9, "peak": link_peak, "unit": "GB/s",
@@ -407,6 +411,9 @@ def main():
     ap.add_argument("--shrink", type=int, default=0, help="divide all sizes by 2**shrink")
     ap.add_argument("--uvm", action="store_true", help="also run the workload over cudaMallocManaged")
     ap.add_argument("--uvm-timeout", type=float, default=120.0)
+    ap.add_argument("--scratch-limit-mib", type=int, default=0,
+                    help="bound of the workload's device scratch (request tables, staged rows); 0 = none. Less scratch "
+                         "means fewer page requests in flight per warp and more faults")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--clock-period", type=float, default=0.5, help="seconds between NVML clock samples")
     args = ap.parse_args()

@@ -44,13 +44,16 @@ int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void
  * x: fp32 array at x_off; d_idx: n_idx int64 element indices in device memory.
  * d_fsum, d_bsum: ceil(n_idx / block) elements.  block <= 2^20.
  *
- * gpuvm_gather_f32: a requester warp stages 4096 requests at a time (32-bit element indices,
- * so the array must have fewer than 2^32 - 1 elements: GPUVM_E_RANGE otherwise) and keeps
- * all of them registered in the page table at once (gpuvm_batch.cuh), so that one migrated
- * page serves many waiting requests (Section 3.3: inter-warp coalescing); the faults go
- * through a ring of page ids in shared memory to the thread block's migrator warps.  The
- * request tables (16 KiB per requester warp, 68 MiB for a full grid on 148 SMs) are device
- * scratch owned by the handle: allocated at the first call, freed by gpuvm_destroy.
+ * gpuvm_gather_f32: a requester warp stages 2048 to 16384 requests at a time (32-bit element
+ * indices, so the array must have fewer than 2^32 - 1 elements: GPUVM_E_RANGE otherwise) and
+ * keeps all of them registered in the page table at once (gpuvm_batch.cuh), so that one
+ * migrated page serves many waiting requests (Section 3.3: inter-warp coalescing); the faults
+ * go through a ring of page ids in shared memory to the thread block's migrator warps, which
+ * move pages with bulk copies.  The request tables are device scratch owned by the handle
+ * (allocated at the first call, freed by gpuvm_destroy): the warps take the deepest power of
+ * two that covers their share of the index list and fits gpuvm_set_scratch_limit, 4 bytes per
+ * request; with no limit and up to 16384 * 28 * (number of SMs) indices every request is in
+ * flight at once (n_idx * 4 bytes of tables) and each page is fetched once.
  * gpuvm_gather_f32_unbatched: one thread per index through gpuvm_read<float>, one
  * thread block per index block; at most 32 requests per warp are in flight.
  */
@@ -171,12 +174,13 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
  * dims a multiple of 4 with dims/4 <= 32 lanes (a lane owns 4 consecutive dims);
  * d_rows: n_bags * bag int64 row ids; d_out: n_bags * dims fp32.
  *
- * gpuvm_embag_f32: a requester warp registers the rows of 32 bags (up to 32 lookups
- * each, 1024 page requests) at once (gpuvm_batch.cuh); rows that arrive are staged in
- * device scratch and added per bag in list order once the batch is complete, so the
- * result has the bits of a sequential fp32 sum.  Scratch owned by the handle: 8 KiB +
- * 1024 rows per requester warp (2.1 GiB for dims = 128 on a full grid of 148 SMs),
- * allocated at the first call, freed by gpuvm_destroy.
+ * gpuvm_embag_f32: a requester warp registers the rows of 32 to 256 bags (up to 32 lookups
+ * each) at once (gpuvm_batch.cuh); rows that arrive are staged in device scratch and added
+ * per bag in list order once the batch is complete, so the result has the bits of a
+ * sequential fp32 sum.  Scratch owned by the handle (allocated at the first call, freed by
+ * gpuvm_destroy): 8 + 4 * dims bytes per request in flight.  The warps take as many groups
+ * of 32 bags (1, 2, 4 or 8) as it takes to have every bag in flight at once, within
+ * gpuvm_set_scratch_limit: 2.1 GiB for one group, dims = 128, on a full grid of 148 SMs.
  * gpuvm_embag_f32_unbatched: one warp per bag, one row request at a time through
  * gpuvm_read; no scratch.
  */

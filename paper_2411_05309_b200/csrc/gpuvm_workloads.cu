@@ -144,7 +144,7 @@ constexpr int kGatherMaxWarps = 32;
 constexpr unsigned int kGatherBatch = 16384;             // most requests per requester warp: 512 rows of 32
 constexpr unsigned int kNoIndex = 0xFFFFFFFFu;
 constexpr unsigned int kGatherChunk = 8192;              // bytes per bulk copy of a migrator warp
-constexpr unsigned int kGatherStages = 2;                // staging buffers per migrator warp
+constexpr unsigned int kGatherStages = 1;                // staging buffers per migrator warp (more in flight only delays each page)
 
 // Request table of the gather: one 32-bit element index per request (the array has fewer than
 // 2^32 - 1 elements), replaced by the value's bit pattern when the request is served.
@@ -627,6 +627,7 @@ __global__ void __launch_bounds__(256) embag_kernel(Mem m, unsigned long long t_
 constexpr int kEmbagRequesters = 28;
 constexpr int kEmbagMigrators = 4;
 constexpr unsigned int kEmbagLookups = 32;                 // lookups of a bag per batch (table rows)
+constexpr unsigned int kEmbagChunk = 8192;                 // bytes per bulk copy of a migrator warp
 constexpr unsigned int kEmbagMaxGroups = 8;                // groups of 32 bags a requester warp takes at a time
 
 __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
@@ -637,6 +638,8 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                                                               gpuvm_shared_queue *shared_queue)
 {
     __shared__ gpuvm_fault_queue queue_s;
+    __shared__ __align__(128) unsigned char stage_s[kEmbagMigrators][kEmbagChunk];   // bulk-copy staging of the migrator warps
+    __shared__ __align__(8) unsigned long long mbar_s[kEmbagMigrators];
     gpuvm_fault_queue *queue = &queue_s;
     const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
@@ -645,7 +648,12 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
     if (threadIdx.x == 0) { queue->requesters = (unsigned int)requesters; queue->shared = shared_queue; }
     __syncthreads();
     if ((int)warp >= requesters) {
-        gpuvm_migrator_loop(vm, queue);
+        const unsigned int mig = warp - requesters;
+        const unsigned int chunk = (1ull << vm.page_shift) < kEmbagChunk ? (unsigned int)(1ull << vm.page_shift) : kEmbagChunk;
+        if (mig < kEmbagMigrators && chunk >= 128)
+            gpuvm_migrator_loop(vm, queue, stage_s[mig], &mbar_s[mig], chunk, 1);
+        else
+            gpuvm_migrator_loop(vm, queue);
         return;
     }
     const unsigned int q = dims >> 2;                            // 16-byte pieces per row

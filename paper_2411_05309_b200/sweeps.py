@@ -5,6 +5,7 @@ oversubscription analysis), printed as JSON lines.
     python -m paper_2411_05309_b200.sweeps warps   [--gib 2]
     python -m paper_2411_05309_b200.sweeps resident
     python -m paper_2411_05309_b200.sweeps oversub [--workload 1|2|3|4] [--shrink S]
+    python -m paper_2411_05309_b200.sweeps depth   [--workload 2|5] [--shrink S]
 
 pages   -- Section 5.1 / Fig. 7: move a fixed amount of host memory into the pool with one
            warp per page, consecutive pages, for page sizes from 4 KiB to 2 MiB; reports the
@@ -19,6 +20,9 @@ resident -- the hit path: streaming sum and random gather over an array that is 
 oversub -- Section 5.4 / Fig. 14 with Eq. 1: run a workload with the pool shrunk step by step,
            level = paged bytes / pool bytes - 1, under the clock policy and under FIFO (the
            paper's ring), reporting time relative to level 0.
+depth   -- Section 3.2 (queue depth by Little's law) carried over to page requests: the batched
+           workloads under a growing bound of their device scratch, i.e. with more and more page
+           requests registered per warp; reports scratch bytes, faults and time.
 """
 from __future__ import annotations
 
@@ -156,9 +160,29 @@ def sweep_oversub(cfg: int, shrink: int):
                 w.close()
 
 
+def sweep_depth(cfg: int, shrink: int):
+    from . import binding as B
+    from . import configs
+    limits_mib = {2: [40, 80, 150, 0], 5: [2300, 4500, 0]}[cfg]
+    for limit in limits_mib:
+        w = configs.make(cfg, shrink)
+        try:
+            B.gpuvm_set_scratch_limit(w.h, (limit << 20) >> shrink)
+            w.run(check=False)
+            runs = [w.run() for _ in range(3)]
+            res = min(runs, key=lambda r: r.seconds)
+            print(json.dumps({"sweep": "depth", "workload": w.name, "scratch_limit_bytes": (limit << 20) >> shrink,
+                              "scratch_bytes": B.gpuvm_scratch_bytes(w.h), "pool_bytes": w.pool_bytes,
+                              "seconds": res.seconds, "faults": res.stats["faults"], "pages": w.nbytes // w.page_bytes,
+                              "bytes_in": res.stats["bytes_in"], "in_gbs": res.stats["bytes_in"] / res.seconds / 1e9,
+                              "effective_gbs": res.effective_bytes / res.seconds / 1e9}), flush=True)
+        finally:
+            w.close()
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("which", choices=["pages", "warps", "resident", "oversub"])
+    ap.add_argument("which", choices=["pages", "warps", "resident", "oversub", "depth"])
     ap.add_argument("--gib", type=float, default=4.0)
     ap.add_argument("--warps-per-sm", type=int, default=16)
     ap.add_argument("--workload", type=int, default=1)
@@ -170,6 +194,8 @@ def main(argv=None):
         sweep_resident()
     elif a.which == "warps":
         sweep_warps(min(a.gib, 2.0))
+    elif a.which == "depth":
+        sweep_depth(a.workload if a.workload in (2, 5) else 2, a.shrink)
     else:
         sweep_oversub(a.workload, a.shrink)
 
