@@ -200,6 +200,13 @@ int gpuvm_scatter_update_u32(gpuvm_t h, size_t a_off, const int64_t *d_idx, size
  * shared memory, without migrator warps: each warp migrates the pages of its own faults. */
 int gpuvm_scatter_update_u32_batched(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream);
 
+/* The same update in write mode with the thread block's fault ring and two migrator warps per
+ * block of six requester warps (512 requests per requester warp staged in shared memory):
+ * migrators write dirty victims back with 16-byte stores and bring pages in with bulk copies;
+ * with pages of 256 KiB or more the grid-wide ring is used as well (256 KiB of the handle's
+ * device scratch). */
+int gpuvm_scatter_update_u32_queued(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream);
+
 /*
  * Transfer micro-benchmark (Section 5.1, Fig. 7): touch n_pages consecutive pages
  * starting at page first_page, one warp per page, `warps_per_sm` warps on every SM;

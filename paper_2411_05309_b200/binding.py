@@ -85,6 +85,7 @@ SYMBOLS = {
     "gpuvm_embag_f32_unbatched": (_i, [_vp, _sz, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_scatter_update_u32": (_i, [_vp, _sz, _vp, _sz, _vp]),
     "gpuvm_scatter_update_u32_batched": (_i, [_vp, _sz, _vp, _sz, _vp]),
+    "gpuvm_scatter_update_u32_queued": (_i, [_vp, _sz, _vp, _sz, _vp]),
     "gpuvm_touch_pages": (_i, [_vp, _sz, _sz, _i, _vp]),
     "gpuvm_touch_pages_warps": (_i, [_vp, _sz, _sz, _i, _vp]),
     "gpuvm_raw_stream_sum_i32": (_i, [_vp, _sz, _vp, _vp]),
@@ -323,6 +324,11 @@ def gpuvm_embag_f32_unbatched(h, t_off: int, dims: int, d_rows, n_bags: int, bag
 
 def gpuvm_scatter_update_u32(h, a_off: int, d_idx, n: int, stream=None):
     _check(lib().gpuvm_scatter_update_u32(h, a_off, _ptr(d_idx), n, _stream(stream)), "gpuvm_scatter_update_u32")
+
+
+def gpuvm_scatter_update_u32_queued(h, a_off: int, d_idx, n: int, stream=None):
+    _check(lib().gpuvm_scatter_update_u32_queued(h, a_off, _ptr(d_idx), n, _stream(stream)),
+           "gpuvm_scatter_update_u32_queued")
 
 
 def gpuvm_scatter_update_u32_batched(h, a_off: int, d_idx, n: int, stream=None):

@@ -751,6 +751,54 @@ __global__ void __launch_bounds__(128) scatter_update_batch_kernel(gpuvm_dev_t v
     }
 }
 
+// The same update with the block's fault ring: six requester warps with 512 requests each, two
+// migrator warps (write mode: victims are dirty and are written back by the migrators; pages come
+// in by bulk copy).
+constexpr int kScatterRequesters = 6;
+constexpr int kScatterMigrators = 2;
+constexpr unsigned int kScatterBatch = 512;
+constexpr unsigned int kScatterChunk = 4096;
+
+__global__ void __launch_bounds__((kScatterRequesters + kScatterMigrators) * 32)
+scatter_update_queued_kernel(gpuvm_dev_t vm, unsigned long long a_off, const long long *__restrict__ idx,
+                             unsigned long long n, gpuvm_shared_queue *shared_queue)
+{
+    __shared__ gpuvm_fault_queue queue_s;
+    __shared__ gpuvm_batch_entry s_table[kScatterRequesters][kScatterBatch];
+    __shared__ __align__(128) unsigned char stage_s[kScatterMigrators][kScatterChunk];
+    __shared__ __align__(8) unsigned long long mbar_s[kScatterMigrators];
+    gpuvm_fault_queue *queue = &queue_s;
+    const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
+        reinterpret_cast<unsigned int *>(queue)[k] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) { queue->requesters = kScatterRequesters; queue->shared = shared_queue; }
+    __syncthreads();
+    if (warp >= kScatterRequesters) {
+        const unsigned int mig = warp - kScatterRequesters;
+        const unsigned int chunk = (1ull << vm.page_shift) < kScatterChunk ? (unsigned int)(1ull << vm.page_shift) : kScatterChunk;
+        if (chunk >= 128) gpuvm_migrator_loop(vm, queue, stage_s[mig], &mbar_s[mig], chunk, 1);
+        else gpuvm_migrator_loop(vm, queue);
+        return;
+    }
+    gpuvm_batch_entry *table = s_table[warp];
+    const unsigned long long batches = (n + kScatterBatch - 1) / kScatterBatch;
+    const unsigned long long stride = (unsigned long long)gridDim.x * kScatterRequesters;
+    for (unsigned long long t = (unsigned long long)blockIdx.x * kScatterRequesters + warp; t < batches; t += stride) {
+        const unsigned long long base = t * kScatterBatch;
+        const unsigned int m = (unsigned int)(n - base < kScatterBatch ? n - base : kScatterBatch);
+        for (unsigned int k = lane; k < m; k += 32)
+            gpuvm_batch_set(vm, table, k, a_off + 4ull * (unsigned long long)idx[base + k]);
+        __syncwarp();
+        gpuvm_batch_access(vm, table, m, GPUVM_WRITE, [](unsigned int, const unsigned char *p) {
+            unsigned int *q = reinterpret_cast<unsigned int *>(const_cast<unsigned char *>(p));
+            gpuvm_store(q, gpuvm_load(q) * 3u + 1u);
+        }, queue);
+        __syncwarp();
+    }
+    if (lane == 0) gpuvm_requester_done(queue);
+}
+
 // ------------------------------------------------------------------ page touch
 __global__ void touch_pages_kernel(gpuvm_dev_t vm, unsigned long long first_page, unsigned long long n_pages)
 {
@@ -1271,6 +1319,20 @@ int gpuvm_scatter_update_u32_batched(gpuvm_t h, size_t a_off, const int64_t *d_i
     if (n == 0) return GPUVM_OK;
     scatter_update_batch_kernel<<<sm_count() * 4, 128, 0, static_cast<cudaStream_t>(stream)>>>(
         m.vm, a_off, reinterpret_cast<const long long *>(d_idx), n);
+    return launched();
+}
+
+int gpuvm_scatter_update_u32_queued(gpuvm_t h, size_t a_off, const int64_t *d_idx, size_t n, void *stream)
+{
+    Paged m;
+    if (!view_of(h, m) || !d_idx) return GPUVM_E_ARG;
+    if (a_off % 16) return GPUVM_E_ALIGN;
+    if (n == 0) return GPUVM_OK;
+    unsigned char *scratch = static_cast<unsigned char *>(gpuvm_scratch_(h, sizeof(gpuvm_shared_queue)));
+    if (!scratch) return GPUVM_E_ALLOC;
+    gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, scratch, static_cast<cudaStream_t>(stream));
+    scatter_update_queued_kernel<<<sm_count() * 2, (kScatterRequesters + kScatterMigrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        m.vm, a_off, reinterpret_cast<const long long *>(d_idx), n, shared_queue);
     return launched();
 }
 

@@ -325,16 +325,18 @@ def test_embag(B, page, n_rows, n_bags, frames, dims, bag, batched):
     assert st["faults"] >= np.unique(rows * dims * 4 // page).size
 
 
-@pytest.mark.parametrize("page,n,frames", [(4096, 1 << 16, 64), (4096, 1 << 16, 7), (64, 2048, 1), (1024, 50000, 13)])
+@pytest.mark.parametrize("page,n,frames", [(4096, 1 << 16, 64), (4096, 1 << 16, 7), (64, 2048, 1), (1024, 50000, 13),
+                                           (1 << 18, 1 << 22, 5)])           # 256 KiB pages: the grid-wide ring too
 @pytest.mark.parametrize("policy", POLICIES)
-@pytest.mark.parametrize("batched", [False, True])
+@pytest.mark.parametrize("batched", [False, True, "queued"])
 def test_scatter_update_through_element_accessors(B, page, n, frames, policy, batched):
     n = n // 4 * 4
     a = (inputs.fill_i32_u20(np.empty(n, np.int32), n, 77)).astype(np.uint32)
     perm = np.random.default_rng(3).permutation(n)[: (3 * n) // 4].astype(np.int64)
     ar = Arena(page, {"a": a})
     with paged(ar.host, page, frames, policy) as h:
-        run = B.gpuvm_scatter_update_u32_batched if batched else B.gpuvm_scatter_update_u32
+        run = {False: B.gpuvm_scatter_update_u32, True: B.gpuvm_scatter_update_u32_batched,
+               "queued": B.gpuvm_scatter_update_u32_queued}[batched]
         run(h, ar.off["a"], dev(perm), perm.size)
         st, ck = finish(h)
     ref = a.copy()

@@ -111,7 +111,7 @@ def test_wait_that_runs_out_returns_an_error_status(B):
         assert int(out.item()) == int(a.astype(np.int64).sum())
 
 
-@pytest.mark.parametrize("which", ["gather", "gather_unbatched", "scatter_batched", "embag"])
+@pytest.mark.parametrize("which", ["gather", "gather_unbatched", "scatter_batched", "scatter_queued", "embag"])
 def test_batched_waits_run_out_too(B, which):
     """The batched engine and the migrator warps give up in the same way: a page that stays
     BUSY makes its requests fail after spin_limit_us, everything else is served, the kernel
@@ -134,6 +134,8 @@ def test_batched_waits_run_out_too(B, which):
             B.gpuvm_gather_f32_unbatched(h, 0, d_idx, idx.size, 1024, fs, bs)
         elif which == "scatter_batched":
             B.gpuvm_scatter_update_u32_batched(h, 0, d_idx, idx.size)
+        elif which == "scatter_queued":
+            B.gpuvm_scatter_update_u32_queued(h, 0, d_idx, idx.size)
         else:
             B.gpuvm_embag_f32(h, 0, 128, rows, 256, 32, out)
 

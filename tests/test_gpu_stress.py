@@ -49,7 +49,9 @@ def test_random_mix_of_workloads_on_one_handle(B):
                 if kind in (0, 1):                                     # scattered updates of distinct elements
                     m = int(rng.integers(1, n + 1))
                     idx = rng.permutation(n)[:m].astype(np.int64)
-                    (B.gpuvm_scatter_update_u32 if kind == 0 else B.gpuvm_scatter_update_u32_batched)(h, 0, dev(idx), m)
+                    variant = int(rng.integers(0, 2))
+                    (B.gpuvm_scatter_update_u32 if kind == 0 else
+                     (B.gpuvm_scatter_update_u32_batched, B.gpuvm_scatter_update_u32_queued)[variant])(h, 0, dev(idx), m)
                     shadow[idx] = shadow[idx] * np.uint32(3) + np.uint32(1)
                 elif kind in (2, 3):                                   # gather of the current contents
                     m = int(rng.integers(1, 4 * n))
