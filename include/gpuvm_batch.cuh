@@ -97,13 +97,20 @@ __device__ __forceinline__ bool fault_queue_push(gpuvm_fault_queue *q, unsigned 
     const unsigned int item = (vpn + 1u) | (mode == kWrite ? 0x80000000u : 0u);
     gpuvm_shared_queue *g = q->shared;
     if (g && *vt - *vh >= GPUVM_FAULT_QUEUE_SPILL) {
-        /* the block has enough of its own: the shared ring, unless that is (nearly) full.  Any
-         * lane of the grid may pass the check at the same moment: 2^15 slots stay spare. */
-        const unsigned int gh = ld_relaxed_u32(&g->head), gt = ld_relaxed_u32(&g->tail);
-        if (gt - gh < GPUVM_SHARED_QUEUE_SLOTS - (1u << 15)) {
-            const unsigned int pos = atomicAdd(&g->tail, 1u);
-            st_relaxed_u32(&g->slot[pos % GPUVM_SHARED_QUEUE_SLOTS], item);
-            return true;
+        /* the block has enough of its own: the shared ring, unless that is full.  A slot is
+         * reserved with a compare-and-swap on the tail, so the ring cannot be overrun however
+         * many lanes of the grid push at the same moment; after 32 lost races the block's
+         * own ring takes the fault. */
+        for (int tries = 0; tries < 32; ++tries) {
+            const unsigned int gt = ld_relaxed_u32(&g->tail);
+            if (gt - ld_relaxed_u32(&g->head) >= GPUVM_SHARED_QUEUE_SLOTS - 1u) break;
+            if (atomicCAS(&g->tail, gt, gt + 1u) == gt) {
+                unsigned int *slot = &g->slot[gt % GPUVM_SHARED_QUEUE_SLOTS];
+                unsigned int spins = 0;
+                while (ld_relaxed_u32(slot) != 0u && ++spins < (1u << 20)) { }   /* its last reader has not cleared it yet */
+                st_relaxed_u32(slot, item);
+                return true;
+            }
         }
     }
     /* up to 1024 lanes may pass this check at the same moment: keep that many slots spare */
