@@ -69,9 +69,11 @@ int gpuvm_gather_f32_unbatched(gpuvm_t h, size_t x_off, const int64_t *d_idx, si
  * receives the hop distance from `source`, -1 where unreachable.  Per level one
  * sweep over the vertices in ascending order (warps draw chunks of 32 consecutive
  * vertices from a ticket counter, so the grid moves through the arrays in address
- * order; per chunk the column pages its edges span are pinned one at a time) plus
- * one launch for very long neighbour lists, which are cut at page boundaries and
- * spread over the whole grid (the imbalance Section 5.2 describes).  Synchronises the
+ * order; per chunk the column pages its edges span are pinned one at a time).
+ * Very long neighbour lists are cut at page boundaries into pieces that go to a
+ * queue which all warps of the same launch serve between their chunks (the
+ * imbalance Section 5.2 describes), so the pieces are expanded while their pages
+ * are under the sweep window.  One launch per level.  Synchronises the
  * stream between levels; *n_levels (host pointer, may be NULL) receives the number
  * of levels expanded, counting the last one that discovers nothing.  Uses 2 MiB of
  * the handle's device scratch (queue of neighbour-list pieces, counters).
@@ -133,7 +135,7 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
  * all free device memory to their own pool, where cudaMalloc would simply fail.
  * For them this variant does exactly what gpuvm_bfs_csr does, same kernels, same
  * arguments, same results, but takes its scratch (the queue of neighbour-list
- * pieces and the level counters, 2 MiB + 16 bytes) from an array that is part of
+ * pieces and the level counters, 2 MiB + 640 bytes) from an array that is part of
  * the library's device image.  It calls no cudaMalloc, cudaFree or other
  * allocating routine.
  *
@@ -147,8 +149,8 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
  *   - All calls on one device share the array.  Two calls whose kernels overlap
  *     on the GPU (different streams, different threads) race on it and give wrong
  *     levels; issue them one after the other.  Nothing needs clearing between
- *     calls: each level re-zeroes the counters, and queue entries are written
- *     before they are read.
+ *     calls: each call zeroes the queue's ready words on its stream before its
+ *     first level, each level re-zeroes the counters.
  * d_level, n_levels, stream, return value: as for gpuvm_bfs_csr.
  */
 #define GPUVM_BFS_NOALLOC_MAX_VERTICES ((size_t)1 << 26)

@@ -33,6 +33,8 @@ struct Paged {
     __device__ __forceinline__ void release(const gpuvm_token &t) const { gpuvm_release(vm, t); }
     __device__ __forceinline__ void clean(const gpuvm_token &t, const void *p) const { gpuvm_clean(vm, t, p); }
     __device__ __forceinline__ void prefetch(unsigned long long off) const { gpuvm_prefetch(vm, off); }
+    __device__ __forceinline__ unsigned long long wait_ns() const { return (unsigned long long)vm.spin_limit_us * 1000ull; }
+    __device__ __forceinline__ void wait_ran_out(unsigned long long where) const { gpuvm::set_error(vm, GPUVM_E_TIMEOUT, where); }
     static __device__ __forceinline__ uint4 load16(const void *p) { return gpuvm_load16(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { gpuvm_store16(p, v); }
     static __device__ __forceinline__ int load_i32(const void *p) { return gpuvm_load(static_cast<const int *>(p)); }
@@ -52,6 +54,8 @@ struct Raw {
     __device__ __forceinline__ void release(const gpuvm_token &) const {}
     __device__ __forceinline__ void clean(const gpuvm_token &, const void *) const {}
     __device__ __forceinline__ void prefetch(unsigned long long) const {}
+    __device__ __forceinline__ unsigned long long wait_ns() const { return 10000000000ull; }
+    __device__ __forceinline__ void wait_ran_out(unsigned long long) const {}
     static __device__ __forceinline__ uint4 load16(const void *p) { return *static_cast<const uint4 *>(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { *static_cast<uint4 *>(p) = v; }
     static __device__ __forceinline__ int load_i32(const void *p) { return *static_cast<const int *>(p); }
@@ -251,9 +255,17 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
 // ------------------------------------------------------- graph sweeps (BFS, CC, SSSP)
 constexpr long long kBigDegree = 4096;     // neighbour lists at least this long are spread over the grid
 constexpr unsigned int kBigQueue = 65536;  // entries of the span queue (four int64 each: first edge, end, vertex, -)
+constexpr unsigned int kSpanPoll = 4;       // a warp looks into the span queue before every kSpanPoll-th chunk
 constexpr long long kAhead = 16;           // pages of look-ahead of the sweeps' prefetches
 
-// counters: [0] updates made in this sweep, [1] span queue size, [2] chunk ticket, [3] span ticket
+// counters of a sweep, each in a 128-byte line of its own (the chunk ticket is hit by every warp all
+// the time; a load of a word in the same line would queue behind those atomics)
+constexpr int kCntUpdates = 0;       // updates made in this sweep
+constexpr int kCntPushed = 32;       // span queue entries reserved
+constexpr int kCntTicket = 64;       // chunk ticket
+constexpr int kCntTaken = 96;        // span ticket
+constexpr int kCntDone = 128;        // chunks finished
+constexpr int kCntWords = 160;
 
 // What a sweep does with a vertex and with each of its edges.
 struct BfsOp {                              // level-synchronous BFS: expand the vertices of the current level
@@ -308,6 +320,96 @@ __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned
     return found;
 }
 
+__device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p) { return *reinterpret_cast<const volatile unsigned int *>(p); }
+
+// Expand one queued piece of a long neighbour list (all 32 lanes).  Returns this lane's number of
+// updates, or -1 when a wait ran out.  Out of line: it is the rare path of the sweep kernel and
+// would only add to the register pressure of the common one.
+template <class Mem, class Op, bool WEIGHTED>
+__device__ __noinline__ int expand_piece(const Mem m, const Op op, unsigned long long col_off, unsigned long long w_off,
+                                         const long long *span_q, unsigned int piece, long long epoch, unsigned int lane)
+{
+    // its producer is between reserving the slot and publishing it
+    const volatile long long *ready = span_q + 4 * (size_t)piece + 3;
+    unsigned long long t0 = 0;
+    bool ok = true;
+    while (*ready != epoch) {
+        const unsigned long long t = gpuvm::now_ns();
+        if (t0 == 0) t0 = t;
+        else if (t - t0 > m.wait_ns()) { ok = false; break; }
+        __nanosleep(64);
+    }
+    if (!__all_sync(0xFFFFFFFFu, ok)) { if (lane == 0) m.wait_ran_out(0); return -1; }
+    __threadfence();                                      // the entry's fields were written before its ready word
+    const long long elo = span_q[4 * (size_t)piece], ehi = span_q[4 * (size_t)piece + 1], u = span_q[4 * (size_t)piece + 2];
+    if (ehi <= elo) return 0;
+    gpuvm_token tok, tok_w;
+    const unsigned char *p = m.pin(col_off + 4ull * elo, GPUVM_READ, tok);
+    if (!p) return -1;
+    const unsigned char *pw = nullptr;
+    if (WEIGHTED) {
+        pw = m.pin(w_off + 4ull * elo, GPUVM_READ, tok_w);
+        if (!pw) { m.release(tok); return -1; }
+    }
+    const unsigned int found = visit_edges<Mem, Op, WEIGHTED>(op, p, pw, elo, u, elo, ehi, lane);
+    if (WEIGHTED) m.release(tok_w);
+    m.release(tok);
+    return (int)found;
+}
+
+// All 32 lanes: claim the next queued piece; 0xFFFFFFFF when none is waiting.
+__device__ __forceinline__ unsigned int take_piece(unsigned int *counters, unsigned int lane)
+{
+    unsigned int piece = 0xFFFFFFFFu;
+    if (lane == 0) {
+        unsigned int pushed = ld_volatile_u32(counters + kCntPushed);
+        if (pushed > kBigQueue) pushed = kBigQueue;
+        const unsigned int taken = ld_volatile_u32(counters + kCntTaken);
+        if (taken < pushed && atomicCAS(counters + kCntTaken, taken, taken + 1u) == taken) piece = taken;
+    }
+    return __shfl_sync(0xFFFFFFFFu, piece, 0);
+}
+
+// End of a warp's sweep (all 32 lanes): expand pieces until every chunk of the sweep is finished
+// and every piece is taken.  Returns this lane's number of updates.  The wait is bounded.
+template <class Mem, class Op, bool WEIGHTED>
+__device__ __noinline__ unsigned int drain_pieces(const Mem m, const Op op, unsigned long long col_off, unsigned long long w_off,
+                                                  const long long *span_q, unsigned int *counters, unsigned int n_chunks,
+                                                  long long epoch, unsigned int lane)
+{
+    unsigned int found = 0, sleep_ns = 64;
+    unsigned long long idle_since = 0;
+    for (;;) {
+        const unsigned int piece = take_piece(counters, lane);
+        if (piece != 0xFFFFFFFFu) {
+            const int r = expand_piece<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, piece, epoch, lane);
+            if (r < 0) return found;
+            found += (unsigned int)r;
+            idle_since = 0;
+            sleep_ns = 64;
+            continue;
+        }
+        int state = 0;                                        // 0 wait, 1 done, 2 gave up
+        if (lane == 0) {
+            unsigned int pushed = ld_volatile_u32(counters + kCntPushed);
+            if (pushed > kBigQueue) pushed = kBigQueue;
+            // Nothing queued in this sweep so far: leave at once (a warp that queues pieces later also
+            // comes through here and sees to them); thousands of idle warps polling would only be in
+            // the way of the ones still at work.  Otherwise stay and help until all chunks are finished.
+            if (pushed == 0u) state = 1;
+            else if (ld_volatile_u32(counters + kCntDone) >= n_chunks && ld_volatile_u32(counters + kCntTaken) >= pushed) state = 1;
+            else {
+                const unsigned long long t = gpuvm::now_ns();
+                if (idle_since == 0) idle_since = t;
+                else if (t - idle_since > m.wait_ns()) { m.wait_ran_out(0); state = 2; }
+            }
+        }
+        if (__shfl_sync(0xFFFFFFFFu, state, 0)) return found;
+        __nanosleep(sleep_ns);
+        if (sleep_ns < 16384) sleep_ns *= 2;
+    }
+}
+
 // One sweep over the vertices in address order: a warp draws the next chunk of 32 consecutive
 // vertices from a ticket counter, so at any moment the whole grid works inside a narrow window
 // of the row-offset and column arrays and a sweep touches every page at most about once.
@@ -317,6 +419,12 @@ __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned
 // neighbour list, which keeps the atomic traffic on the entries of the few pages under the
 // window low.  Odd sweeps run downwards: the pages a sweep used last are still resident when the
 // next one starts with them (a one-directional cyclic sweep defeats any LRU-like policy).
+// Very long neighbour lists are cut at unit boundaries into pieces that go to a queue; every warp
+// looks into that queue before it draws its next chunk, so the pieces are expanded by the whole
+// grid while their pages are still under (or just ahead of) the sweep window.  An entry is
+// published by its `ready` word (= sweep + 1, written after a fence; the queue is zeroed once per
+// call).  A warp leaves when all chunks are finished and all pieces are taken; every wait is
+// bounded.
 template <class Mem, class Op, bool WEIGHTED>
 __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
                                                           unsigned long long w_off, unsigned int nv,
@@ -326,12 +434,31 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
     const unsigned int lane = threadIdx.x & 31;
     const unsigned long long unit = m.unit();
     const unsigned int n_chunks = (nv + 31) / 32;
-    unsigned int found = 0;
+    const long long epoch = sweep + 1;
+    unsigned int found = 0, my_done = 0, iter = 0;
     for (;;) {
+        // ---- a piece of a long neighbour list, if one is waiting (looked for before every kSpanPoll-th chunk)
+        if ((iter++ & (kSpanPoll - 1)) == 0) {
+            const unsigned int piece = take_piece(counters, lane);
+            if (piece != 0xFFFFFFFFu) {
+                const int r = expand_piece<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, piece, epoch, lane);
+                if (r < 0) break;
+                found += (unsigned int)r;
+                continue;
+            }
+        }
+        // ---- the next chunk of 32 vertices
         unsigned int chunk = 0;
-        if (lane == 0) chunk = atomicAdd(counters + 2, 1u);
+        if (lane == 0) chunk = atomicAdd(counters + kCntTicket, 1u);
         chunk = __shfl_sync(0xFFFFFFFFu, chunk, 0);
-        if (chunk >= n_chunks) break;
+        if (chunk >= n_chunks) {
+            // no chunk left: report the finished ones, then help with the pieces until all chunks
+            // are finished and all pieces taken
+            if (lane == 0 && my_done) { __threadfence(); atomicAdd(counters + kCntDone, my_done); }
+            found += drain_pieces<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, counters, n_chunks, epoch, lane);
+            break;
+        }
+        ++my_done;
         const unsigned long long v0 = 32ull * ((sweep & 1) ? n_chunks - 1 - chunk : chunk);
         const unsigned long long v = v0 + lane;
         const bool active = v < nv && op.active(v);
@@ -357,20 +484,23 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             const unsigned long long b0 = (col_off + 4ull * blo) / unit, b1 = (col_off + 4ull * bhi - 1) / unit;
             const unsigned int pieces = (unsigned int)(b1 - b0 + 1);
             unsigned int slot = 0;
-            if (lane == 0) slot = atomicAdd(counters + 1, pieces);
+            if (lane == 0) slot = atomicAdd(counters + kCntPushed, pieces);
             slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
-            if (slot + pieces > kBigQueue) {                       // queue full: expand the list here
-                for (unsigned int k = slot + lane; k < kBigQueue; k += 32) { span_q[4 * k] = 0; span_q[4 * k + 1] = 0; }
-                continue;
-            }
-            for (unsigned int k = lane; k < pieces; k += 32) {
+            const bool fits = slot + pieces <= kBigQueue;
+            const unsigned int n_write = fits ? pieces : (slot < kBigQueue ? kBigQueue - slot : 0u);
+            for (unsigned int k = lane; k < n_write; k += 32) {
                 const long long s = (long long)(((b0 + k) * unit - col_off + 3) / 4);
                 const long long t = (long long)(((b0 + k + 1) * unit - col_off) / 4);
-                span_q[4 * (slot + k)] = k == 0 ? blo : s;
-                span_q[4 * (slot + k) + 1] = t < bhi ? t : bhi;
-                span_q[4 * (slot + k) + 2] = (long long)(v0 + L);
+                // queue full: the slots that were reserved are published empty and the list is expanded here
+                span_q[4 * (size_t)(slot + k)] = fits ? (k == 0 ? blo : s) : 0;
+                span_q[4 * (size_t)(slot + k) + 1] = fits ? (t < bhi ? t : bhi) : 0;
+                span_q[4 * (size_t)(slot + k) + 2] = (long long)(v0 + L);
             }
-            if ((int)lane == L) { lo = 0; hi = 0; }
+            __threadfence();
+            __syncwarp();
+            for (unsigned int k = lane; k < n_write; k += 32)
+                *reinterpret_cast<volatile long long *>(span_q + 4 * (size_t)(slot + k) + 3) = epoch;
+            if (fits && (int)lane == L) { lo = 0; hi = 0; }
         }
         // the edges of this chunk, unit by unit
         long long rlo = hi > lo ? lo : 0x7FFFFFFFFFFFFFFFll, rhi = hi > lo ? hi : 0;
@@ -388,6 +518,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             }
         }
         long long first = rlo;
+        bool failed = false;
         while (first < rhi) {
             const unsigned long long byte = col_off + 4ull * first;
             long long last = (long long)(((byte / unit + 1) * unit - col_off) / 4);   // first edge of the next unit
@@ -396,11 +527,11 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             if (touch) {
                 gpuvm_token tok, tok_w;
                 const unsigned char *p = m.pin(byte, GPUVM_READ, tok);
-                if (!p) return;
+                if (!p) { failed = true; break; }
                 const unsigned char *pw = nullptr;
                 if (WEIGHTED) {
                     pw = m.pin(w_off + 4ull * first, GPUVM_READ, tok_w);
-                    if (!pw) { m.release(tok); return; }
+                    if (!pw) { m.release(tok); failed = true; break; }
                 }
                 while (touch) {
                     const int L = __ffs(touch) - 1;
@@ -415,41 +546,10 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             }
             first = last;
         }
+        if (failed) break;                               // a wait ran out: the sticky error is set, the others give up too
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
-    if (lane == 0 && found) atomicAdd(counters, found);
-}
-
-// Pieces of long neighbour lists, one warp per piece (a piece never crosses a unit).
-template <class Mem, class Op, bool WEIGHTED>
-__global__ void __launch_bounds__(256, 4) graph_span_kernel(Mem m, Op op, unsigned long long col_off, unsigned long long w_off,
-                                                         const long long *__restrict__ span_q,
-                                                         unsigned int *__restrict__ counters)
-{
-    const unsigned int lane = threadIdx.x & 31;
-    const unsigned int n = counters[1] < kBigQueue ? counters[1] : kBigQueue;
-    unsigned int found = 0;
-    for (;;) {
-        unsigned int i = 0;
-        if (lane == 0) i = atomicAdd(counters + 3, 1u);
-        i = __shfl_sync(0xFFFFFFFFu, i, 0);
-        if (i >= n) break;
-        const long long elo = span_q[4 * i], ehi = span_q[4 * i + 1], u = span_q[4 * i + 2];
-        if (ehi <= elo) continue;
-        gpuvm_token tok, tok_w;
-        const unsigned char *p = m.pin(col_off + 4ull * elo, GPUVM_READ, tok);
-        if (!p) return;
-        const unsigned char *pw = nullptr;
-        if (WEIGHTED) {
-            pw = m.pin(w_off + 4ull * elo, GPUVM_READ, tok_w);
-            if (!pw) { m.release(tok); return; }
-        }
-        found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, elo, u, elo, ehi, lane);
-        if (WEIGHTED) m.release(tok_w);
-        m.release(tok);
-    }
-    for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
-    if (lane == 0 && found) atomicAdd(counters, found);
+    if (lane == 0 && found) atomicAdd(counters + kCntUpdates, found);
 }
 
 // Balanced CSR (Section 5.2, Fig. 8): the edge array is cut into chunks of equal length and a
@@ -927,9 +1027,9 @@ int run_gather(const Mem &m, size_t x_off, const int64_t *d_idx, size_t n_idx, s
 }
 
 constexpr int kVaddBlocksPerSm = 4;
-constexpr size_t kBfsScratchBytes = 4 * kBigQueue * sizeof(long long) + 4 * sizeof(unsigned int);
+constexpr size_t kBfsScratchBytes = 4 * kBigQueue * sizeof(long long) + kCntWords * sizeof(unsigned int);
 
-// One sweep (both kernels) and its update count.
+// One sweep and its update count.  `sweep` counts from 0 within a call.
 template <class Mem, class Op, bool WEIGHTED>
 int graph_sweep(const Mem &m, const Op &op, size_t off_off, size_t col_off, size_t w_off, size_t nv, void *scratch, int sweep,
                 unsigned int *updates, cudaStream_t s)
@@ -940,10 +1040,10 @@ int graph_sweep(const Mem &m, const Op &op, size_t off_off, size_t col_off, size
     unsigned int *counters = reinterpret_cast<unsigned int *>(span_q + 4 * kBigQueue);
     // paged: 4 blocks per SM; over managed memory a narrower window of 2 blocks per SM is 10x faster
     const int grid = sm_count() * Mem::kSweepBlocksPerSm;
-    cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
+    if (sweep == 0) cudaMemsetAsync(span_q, 0, 4 * kBigQueue * sizeof(long long), s);     // ready words: once per call
+    cudaMemsetAsync(counters, 0, kCntWords * sizeof(unsigned int), s);
     graph_sweep_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, off_off, col_off, w_off, (unsigned int)nv, n_edges, span_q, counters, sweep);
-    graph_span_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, col_off, w_off, span_q, counters);
-    int rc = launched(2);
+    int rc = launched(1);
     unsigned int host_counters[2] = {0, 0};
     if (cudaMemcpyAsync(host_counters, counters, sizeof(host_counters), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
         cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }

@@ -154,6 +154,47 @@ def test_batched_waits_run_out_too(B, which):
             assert np.array_equal(bs.cpu().numpy(), oracle.gather_block_sums_direct(x, idx, 1024)[1])
 
 
+@pytest.mark.parametrize("which", ["bfs", "cc"])
+def test_graph_sweep_waits_run_out_too(B, which):
+    """A column page that stays BUSY: the sweep (chunks, queued pieces of hub lists, the wait for
+    the other warps at its end) gives up after spin_limit_us, the kernel ends, the error is
+    reported; after a reset the same call gives the oracle's result."""
+    import torch
+    import oracle
+    off, col = inputs.rmat_csr(14, 16 << 14, inputs.config_seed(3))
+    assert np.diff(off).max() >= 4096                     # hub vertices: pieces are queued
+    nv = off.size - 1
+    off_p = np.zeros((off.size + 1) // 2 * 2, np.int64)
+    off_p[:off.size] = off
+    col_p = np.concatenate([col, np.zeros((-col.size) % 4, col.dtype)])
+    page = 4096
+    ar = Arena(page, {"off": off_p, "col": col_p})
+    out = torch.zeros(nv, dtype=torch.int32, device="cuda")
+    hub = int(np.argmax(np.diff(off)))
+    stuck = (ar.off["col"] + 4 * int(off[hub]) + 8 * page) // page      # a page in the middle of the longest list
+
+    def call(h):
+        if which == "bfs":
+            B.gpuvm_bfs_csr(h, ar.off["off"], ar.off["col"], nv, 0, out)
+        else:
+            B.gpuvm_cc_csr(h, ar.off["off"], ar.off["col"], nv, out)
+
+    with paged(ar.host, page, 64, spin_limit_us=30_000) as h:
+        B.gpuvm_debug_poke_pte(h, stuck, BUSY)
+        try:
+            call(h)
+        except B.GpuvmError:
+            pass
+        torch.cuda.synchronize()
+        st = B.gpuvm_stats(h, raise_on_error=False)
+        assert st["error"] == B.E_TIMEOUT
+        B.gpuvm_reset(h)
+        call(h)
+        finish(h)
+    ref = oracle.bfs_levels_direct(off, col, 0) if which == "bfs" else oracle.cc_labels_direct(off, col)
+    assert np.array_equal(out.cpu().numpy(), ref)
+
+
 def test_concurrent_kernels_on_one_handle_and_on_two(B):
     """Kernels launched on different streams may share a page table (Section 4, "Multi-kernel
     support": a stream of concurrent kernels reading the same data on demand): a warp only ever
