@@ -267,23 +267,26 @@ constexpr int kCntTaken = 96;        // span ticket
 constexpr int kCntDone = 128;        // chunks finished
 constexpr int kCntWords = 160;
 
-// What a sweep does with a vertex and with each of its edges.
+// What a sweep does with a vertex and with each of its edges.  peek reads what the edge's other
+// end holds now (a plain load: several edges' peeks are issued together), edge decides and updates.
 struct BfsOp {                              // level-synchronous BFS: expand the vertices of the current level
     int *level;
     int depth;
     __device__ __forceinline__ bool active(unsigned long long v) const { return level[v] == depth; }
-    __device__ __forceinline__ unsigned int edge(long long, int c, int) const
+    __device__ __forceinline__ int peek(int c) const { return level[c]; }
+    __device__ __forceinline__ unsigned int edge(long long, int c, int, int seen) const
     {
-        return level[c] == -1 && atomicCAS(level + c, -1, depth + 1) == -1;
+        return seen == -1 && atomicCAS(level + c, -1, depth + 1) == -1;
     }
 };
 
 struct CcOp {                               // label propagation over every edge, both ways, minimum label wins
     int *label;
     __device__ __forceinline__ bool active(unsigned long long) const { return true; }
-    __device__ __forceinline__ unsigned int edge(long long u, int c, int) const
+    __device__ __forceinline__ int peek(int c) const { return label[c]; }
+    __device__ __forceinline__ unsigned int edge(long long u, int c, int, int lc) const
     {
-        const int lu = label[u], lc = label[c];
+        const int lu = label[u];
         if (lu < lc) return atomicMin(label + c, lu) > lu;
         if (lc < lu) return atomicMin(label + u, lc) > lc;
         return 0;
@@ -295,27 +298,40 @@ struct SsspOp {                             // Bellman-Ford rounds: relax the ed
     const unsigned char *cur;
     unsigned char *next;
     __device__ __forceinline__ bool active(unsigned long long v) const { return cur[v] != 0; }
-    __device__ __forceinline__ unsigned int edge(long long u, int c, int w) const
+    __device__ __forceinline__ int peek(int c) const { return dist[c]; }
+    __device__ __forceinline__ unsigned int edge(long long u, int c, int w, int dc) const
     {
         const int du = dist[u];
         if (du == 0x7FFFFFFF) return 0;
         const int nd = du + w;
-        if (nd < dist[c] && atomicMin(dist + c, nd) > nd) { next[c] = 1; return 1; }
+        if (nd < dc && atomicMin(dist + c, nd) > nd) { next[c] = 1; return 1; }
         return 0;
     }
 };
 
-// Visit the edges [elo, ehi) of vertex u that lie inside the pinned unit starting at edge `first`.
+// Visit the edges [elo, ehi) of vertex u that lie inside the pinned unit starting at edge `first`,
+// four per lane at a time: the column (and weight) loads of the four are issued together, then
+// the peeks at their other ends, then the updates.
 template <class Mem, class Op, bool WEIGHTED>
 __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned char *col_unit, const unsigned char *w_unit,
                                                     long long first, long long u, long long elo, long long ehi,
                                                     unsigned int lane)
 {
+    constexpr int U = 4;
     unsigned int found = 0;
-    for (long long e = elo + lane; e < ehi; e += 32) {
-        const int c = Mem::load_i32(col_unit + 4 * (e - first));
-        const int w = WEIGHTED ? Mem::load_i32(w_unit + 4 * (e - first)) : 0;
-        found += op.edge(u, c, w);
+    for (long long e0 = elo + lane; e0 < ehi; e0 += 32 * U) {
+        int c[U], w[U], seen[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long e = e0 + 32 * k;
+            c[k] = e < ehi ? Mem::load_i32(col_unit + 4 * (e - first)) : -1;
+            w[k] = (WEIGHTED && e < ehi) ? Mem::load_i32(w_unit + 4 * (e - first)) : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) seen[k] = c[k] >= 0 ? op.peek(c[k]) : 0;
+#pragma unroll
+        for (int k = 0; k < U; ++k)
+            if (c[k] >= 0) found += op.edge(u, c[k], w[k], seen[k]);
     }
     return found;
 }
