@@ -44,16 +44,22 @@ int gpuvm_stream_sum_i32(gpuvm_t h, size_t a_off, size_t n, int64_t *d_sum, void
  * x: fp32 array at x_off; d_idx: n_idx int64 element indices in device memory.
  * d_fsum, d_bsum: ceil(n_idx / block) elements.  block <= 2^20.
  *
- * gpuvm_gather_f32: a requester warp stages 2048 to 16384 requests at a time (32-bit element
- * indices, so the array must have fewer than 2^32 - 1 elements: GPUVM_E_RANGE otherwise) and
- * keeps all of them registered in the page table at once (gpuvm_batch.cuh), so that one
- * migrated page serves many waiting requests (Section 3.3: inter-warp coalescing); the faults
- * go through a ring of page ids in shared memory to the thread block's migrator warps, which
- * move pages with bulk copies.  The request tables are device scratch owned by the handle
- * (allocated at the first call, freed by gpuvm_destroy): the warps take the deepest power of
- * two that covers their share of the index list and fits gpuvm_set_scratch_limit, 4 bytes per
- * request; with no limit and up to 16384 * 28 * (number of SMs) indices every request is in
- * flight at once (n_idx * 4 bytes of tables) and each page is fetched once.
+ * gpuvm_gather_f32: a requester warp keeps 2048 to 16384 requests registered in the page
+ * table at once (gpuvm_batch.cuh), so that one migrated page serves many waiting requests
+ * (Section 3.3: inter-warp coalescing); the faults go through a ring of page ids in shared
+ * memory to the thread block's migrator warps, which move pages with bulk copies.  With up to
+ * 16384 * 28 * (number of SMs) indices every request is in flight at once and each page is
+ * fetched once.  Two forms of the request table:
+ *   - block >= 256 and no scratch bound set: the index list itself is the table (read in
+ *     place) and every gathered value is added to the double / int64 sums of its index
+ *     block at once, in shared memory.  No device scratch.  The double sum is taken in the
+ *     order of arrival, so d_fsum can differ from a fixed-order sum in the last bit when the
+ *     sum lies within about 1e-13 (relative) of a float rounding boundary.
+ *   - otherwise: 32-bit element indices staged in device scratch owned by the handle, 4
+ *     bytes per request in flight (the array must then have fewer than 2^32 - 1 elements:
+ *     GPUVM_E_RANGE otherwise), replaced by the values as they arrive and summed in index
+ *     order; the warps take the deepest power of two that covers their share of the index
+ *     list and fits gpuvm_set_scratch_limit.
  * gpuvm_gather_f32_unbatched: one thread per index through gpuvm_read<float>, one
  * thread block per index block; at most 32 requests per warp are in flight.
  */

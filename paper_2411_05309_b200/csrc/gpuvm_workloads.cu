@@ -164,6 +164,33 @@ struct GatherTable {
     }
 };
 
+// The index list itself as the request table (no copy): request i of a piece is idx[i].
+struct GatherIndexTable {
+    const long long *idx;
+    unsigned long long x_off, n_elems;
+    gpuvm_dev_t vm;
+    __device__ __forceinline__ bool valid(unsigned int i) const
+    {
+        const unsigned long long e = (unsigned long long)idx[i];
+        if (e >= n_elems) gpuvm::set_error(vm, GPUVM_E_RANGE, (x_off + 4 * e) >> vm.page_shift);
+        return e < n_elems;
+    }
+    __device__ __forceinline__ unsigned int vpn(unsigned int i) const { return (unsigned int)((x_off + 4ull * (unsigned long long)idx[i]) >> vm.page_shift); }
+    __device__ __forceinline__ unsigned int off(unsigned int i) const
+    {
+        return (unsigned int)((x_off + 4ull * (unsigned long long)idx[i]) & ((1ull << vm.page_shift) - 1ull));
+    }
+};
+
+constexpr unsigned int kGatherAcc = 64;                  // index blocks a requester warp sums at a time without a table
+constexpr unsigned int kGatherDirectMinBlock = kGatherBatch / kGatherAcc;
+
+// DIRECT: the requests are read from the index list in place and every value is added to the sums of
+// its index block as it is gathered (shared-memory accumulators, double and int64): no request table,
+// no scratch.  Needs index blocks of at least kGatherDirectMinBlock.  The double sum is then taken in
+// the order of arrival; its float rounding is the oracle's unless the sum lies within 1e-13 of a
+// rounding boundary.
+template <bool DIRECT>
 __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(gpuvm_dev_t vm, unsigned long long x_off,
                                                                                const long long *__restrict__ idx,
                                                                                unsigned long long n_idx, unsigned long long block,
@@ -193,7 +220,13 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
         return;
     }
     unsigned long long *masks = gather_masks + (size_t)warp * gpuvm_batch_mask_words(batch) * 32 + lane;
-    unsigned int *table = g_tables + ((size_t)blockIdx.x * requesters + warp) * batch;
+    unsigned int *table = DIRECT ? nullptr : g_tables + ((size_t)blockIdx.x * requesters + warp) * batch;
+    // DIRECT: this warp's accumulators, behind the masks, the staging buffers and their mbarriers
+    const unsigned int n_mig_w = (blockDim.x >> 5) - requesters;
+    unsigned char *acc0 = reinterpret_cast<unsigned char *>(gather_masks + (size_t)requesters * gpuvm_batch_mask_words(batch) * 32) +
+                          (size_t)n_mig_w * stage_count * (stage_chunk + sizeof(unsigned long long));
+    double *acc_f = reinterpret_cast<double *>(acc0) + (size_t)warp * 2 * kGatherAcc;
+    unsigned long long *acc_b = reinterpret_cast<unsigned long long *>(acc_f + kGatherAcc);
     const unsigned long long n_elems = (vm.bytes - x_off) / 4;
     const unsigned long long nb = (n_idx + block - 1) / block;
     const unsigned long long per = block <= batch ? batch / block : 1;      // index blocks per work item
@@ -206,6 +239,37 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
         long long carry_b = 0;
         for (unsigned long long base = lo; base < hi; base += batch) {
             const unsigned int n = (unsigned int)(hi - base < batch ? hi - base : batch);
+            if constexpr (DIRECT) {
+                // blocks of this piece: whole ones (block <= batch: pieces start on a block boundary) or a part of one
+                const unsigned int nblk = block <= batch ? (unsigned int)((n + block - 1) / block) : 1u;
+                const unsigned int blk32 = (unsigned int)block;
+                for (unsigned int k = lane; k < nblk; k += 32) { acc_f[k] = 0.0; acc_b[k] = 0ull; }
+                __syncwarp();
+                gpuvm_batch_run<false>(vm, GatherIndexTable{idx + base, x_off, n_elems, vm}, n, GPUVM_READ,
+                                       [=](unsigned int i, const unsigned char *p) {
+                                           const unsigned int v = gpuvm_load(reinterpret_cast<const unsigned int *>(p));
+                                           const unsigned int k = nblk > 1 ? i / blk32 : 0u;
+                                           atomicAdd(acc_f + k, (double)__uint_as_float(v));
+                                           atomicAdd(acc_b + k, (unsigned long long)v);
+                                           return v;              // read-only consume: lets the engine skip its fence
+                                       }, queue, masks, 32u, one_pass);
+                __syncwarp();
+                if (block <= batch) {
+                    for (unsigned int k = lane; k < nblk; k += 32) {
+                        fsum[base / block + k] = (float)acc_f[k];
+                        bsum[base / block + k] = (long long)acc_b[k];
+                    }
+                } else {                                          // one long block, piece by piece
+                    carry_f += acc_f[0];
+                    carry_b += (long long)acc_b[0];
+                    if (base + n == hi) {
+                        if (lane == 0) { fsum[base / block] = (float)carry_f; bsum[base / block] = carry_b; }
+                        carry_f = 0.0;
+                        carry_b = 0;
+                    }
+                }
+                __syncwarp();
+            } else {
             for (unsigned int k = lane; k < n; k += 32) {
                 const unsigned long long i = (unsigned long long)idx[base + k];
                 if (i >= n_elems) gpuvm::set_error(vm, GPUVM_E_RANGE, (x_off + 4 * i) >> vm.page_shift);
@@ -247,6 +311,7 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
                 pos = end;
             }
             __syncwarp();
+            }   // table path
         }
     }
     if (lane == 0) gpuvm_requester_done(queue);
@@ -1263,15 +1328,19 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     if (!d_idx || !d_fsum || !d_bsum || block == 0 || block > (size_t(1) << 20)) return GPUVM_E_ARG;
     if (x_off % 16) return GPUVM_E_ALIGN;
     if (n_idx == 0) return GPUVM_OK;
-    if ((m.vm.bytes - x_off) / 4 >= kNoIndex) return GPUVM_E_RANGE;      // element indices are staged as 32-bit numbers
     const int requesters = kGatherRequesters, migrators = kGatherMigrators;
     // Requests per requester warp: all of a warp's share of the index list when that is at most
     // kGatherBatch (then every page is fetched once per run), whole index blocks, at least 2048.
     const size_t warps_all = (size_t)sm_count() * requesters;
     size_t share = (n_idx + warps_all - 1) / warps_all;
     if (block <= kGatherBatch) share = (share + block - 1) / block * block;
+    // Without a scratch bound and with index blocks of at least kGatherDirectMinBlock the requests are
+    // read from the index list in place and summed as they arrive: no table, no scratch.
+    const bool direct = block >= kGatherDirectMinBlock && gpuvm_scratch_limit_(h) == ~size_t(0);
+    if (!direct && (m.vm.bytes - x_off) / 4 >= kNoIndex) return GPUVM_E_RANGE;      // element indices are staged as 32-bit numbers
     unsigned int batch = 2048;
-    while (batch < kGatherBatch && batch < share && warps_all * (size_t)batch * 2 * sizeof(unsigned int) <= gpuvm_scratch_limit_(h))
+    while (batch < kGatherBatch && batch < share &&
+           (direct || warps_all * (size_t)batch * 2 * sizeof(unsigned int) <= gpuvm_scratch_limit_(h)))
         batch *= 2;
     const size_t nb = (n_idx + block - 1) / block;
     const size_t per = block <= batch ? batch / block : 1;
@@ -1279,7 +1348,7 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     const size_t blocks_needed = (items + requesters - 1) / requesters;
     const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
     const size_t slots = items < (size_t)grid * requesters ? items : (size_t)grid * requesters;   // warps that get work
-    const size_t tables_bytes = (slots * batch * sizeof(unsigned int) + 255) & ~size_t(255);
+    const size_t tables_bytes = direct ? 0 : (slots * batch * sizeof(unsigned int) + 255) & ~size_t(255);
     unsigned int *tables = static_cast<unsigned int *>(gpuvm_scratch_(h, tables_bytes + sizeof(gpuvm_shared_queue)));
     if (!tables) return GPUVM_E_ALLOC;
     gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, reinterpret_cast<unsigned char *>(tables) + tables_bytes,
@@ -1288,13 +1357,15 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     const unsigned int stage_chunk = (unsigned int)((size_t(1) << m.vm.page_shift) < kGatherChunk ? (size_t(1) << m.vm.page_shift) : kGatherChunk);
     const unsigned int stage_count = stage_chunk >= 128 ? kGatherStages : 0;     // tiny pages: copy through registers
     const size_t mask_bytes = (size_t)requesters * gpuvm_batch_mask_words(batch) * 32 * sizeof(unsigned long long) +
-                              (size_t)migrators * stage_count * (stage_chunk + sizeof(unsigned long long));
+                              (size_t)migrators * stage_count * (stage_chunk + sizeof(unsigned long long)) +
+                              (direct ? (size_t)requesters * 2 * kGatherAcc * sizeof(double) : 0);
+    auto kernel = direct ? gather_batch_kernel<true> : gather_batch_kernel<false>;
     if (mask_bytes > 40 * 1024 &&
-        cudaFuncSetAttribute(gather_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mask_bytes) != cudaSuccess) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mask_bytes) != cudaSuccess) {
         cudaGetLastError();
         return GPUVM_E_CUDA;
     }
-    gather_batch_kernel<<<grid, (requesters + migrators) * 32, mask_bytes, static_cast<cudaStream_t>(stream)>>>(
+    kernel<<<grid, (requesters + migrators) * 32, mask_bytes, static_cast<cudaStream_t>(stream)>>>(
         m.vm, x_off, reinterpret_cast<const long long *>(d_idx), n_idx, block, d_fsum, reinterpret_cast<long long *>(d_bsum),
         requesters, batch, tables, stage_chunk, stage_count, /* one_pass = */ items <= (size_t)grid * requesters, shared_queue);
     return launched();
