@@ -384,7 +384,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             "traffic": NCU_LINK_BYTES.get(args.workload) if args.shrink == 0 and not args.scratch_limit_mib else None,
             "traffic_source": "host-link bytes of one launch counted by ncu (sysmem read sector misses x 32 B) in the "
                               "committed capture of this kernel at this size; equals the kernel's own bytes_in counter. "
-                              "DRAM traffic is not the bound on this path (8.5 % of DRAM peak in the capture of cfg 2)",
+                              "DRAM traffic is not the bound on this path (9.4 % of DRAM peak in the capture of cfg 2)",
             "hbm": {"achieved": (bytes_in + bytes_out + eff_bytes) / kern_s / 1e9, "peak": hbm_peak,
                     "frac": ((bytes_in + bytes_out + eff_bytes) / kern_s / 1e9) / hbm_peak,
                     "peak_source": "MEASURED_PEAKS.json" if peaks else "fallback"},
