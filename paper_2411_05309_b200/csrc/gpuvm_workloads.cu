@@ -135,13 +135,13 @@ __global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long lo
     }
 }
 
-// A requester warp takes a run of consecutive indices (whole index blocks when they fit),
-// stages their element indices in its request table (handle-owned device scratch: it stays in
-// L2), registers them all in the page table, and as the pages arrive replaces each index by
-// the value it asked for (gpuvm_batch.cuh); then it adds the values up block by block.  The
-// faults it owns go to the thread block's ring of page ids in shared memory, which the
-// block's migrator warps serve.  No block-wide barrier after start-up: warps never wait for
-// one another.
+// A requester warp takes a run of consecutive indices (whole index blocks when they fit) and
+// registers them all in the page table (gpuvm_batch.cuh).  Table form: their element indices are
+// staged in the warp's request table (handle-owned device scratch), each index is replaced by the
+// value it asked for as the pages arrive, and the values are added up block by block afterwards.
+// Direct form: see the template parameter below.  The faults a warp owns go to the thread block's
+// ring of page ids in shared memory, which the block's migrator warps serve.  No block-wide barrier
+// after start-up: warps never wait for one another.
 constexpr int kGatherRequesters = 28;
 constexpr int kGatherMigrators = 4;
 constexpr int kGatherMaxWarps = 32;
