@@ -1250,7 +1250,7 @@ int run_sssp(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t 
 }
 
 template <class Mem>
-int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, bool hold_c, cudaStream_t s)
+int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, bool hold_c, int blocks, cudaStream_t s)
 {
     unsigned long long unit = 0;
     if (n % 4) return GPUVM_E_ALIGN;
@@ -1260,9 +1260,9 @@ int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, b
     if (chunk < 512) return GPUVM_E_PAGE;             // a warp moves 512 bytes per instruction
     if (a_off % chunk || b_off % chunk || c_off % chunk) return GPUVM_E_ALIGN;
     if (hold_c && c_off % unit == 0)
-        vadd_kernel<Mem, true><<<sm_count() * kVaddBlocksPerSm, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
+        vadd_kernel<Mem, true><<<blocks, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
     else
-        vadd_kernel<Mem, false><<<sm_count() * kVaddBlocksPerSm, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
+        vadd_kernel<Mem, false><<<blocks, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
     return launched();
 }
 
@@ -1440,9 +1440,13 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
 {
     PagedH m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
-    // two pages per warp are held at once on the no-fetch path: only when the pool can take it
-    const bool hold_c = gpuvm_safe_warps(h, 2) >= sm_count() * kVaddBlocksPerSm * 8;
-    return run_vadd(m, a_off, b_off, c_off, n, hold_c, static_cast<cudaStream_t>(stream));
+    // Two pages per warp are held at once on the no-fetch path: only when the pool can take it.  A small
+    // pool gets a smaller grid first (down to one thread block per SM, which is what is resident at
+    // this kernel's register count anyway) before the kernel falls back to one page at a time.
+    int blocks = sm_count() * kVaddBlocksPerSm;
+    while (blocks > sm_count() && gpuvm_safe_warps(h, 2) < blocks * 8) blocks -= sm_count();
+    const bool hold_c = gpuvm_safe_warps(h, 2) >= blocks * 8;
+    return run_vadd(m, a_off, b_off, c_off, n, hold_c, blocks, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
@@ -1617,7 +1621,7 @@ int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void 
     RawH m;
     m.base = base;
     m.unit_bytes = 65536;
-    return run_vadd(m, (size_t)(pa - base), (size_t)(pb - base), (size_t)(pc - base), n, false, static_cast<cudaStream_t>(stream));
+    return run_vadd(m, (size_t)(pa - base), (size_t)(pb - base), (size_t)(pc - base), n, false, sm_count() * kVaddBlocksPerSm, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_raw_embag_f32(const float *table, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
