@@ -62,6 +62,10 @@ def test_create_rejects_bad_arguments_before_cuda(B):
     assert L.gpuvm_flush(None, None) == B.E_ARG and L.gpuvm_safe_warps(None, 1) == B.E_ARG
     assert L.gpuvm_stream_sum_i32(None, 0, 16, None, None) == B.E_ARG
     assert L.gpuvm_bfs_csr_noalloc(None, 0, 0, 1, 0, None, None, None) == B.E_ARG
+    assert L.gpuvm_set_scratch_limit(None, 1 << 20) == B.E_ARG and L.gpuvm_scratch_bytes(None) == 0
+    assert L.gpuvm_gather_f32(None, 0, None, 16, 1024, None, None, None) == B.E_ARG
+    assert L.gpuvm_embag_f32(None, 0, 128, None, 1, 32, None, None) == B.E_ARG
+    assert L.gpuvm_scatter_update_u32_queued(None, 0, None, 1, None) == B.E_ARG
 
 
 def test_no_device_no_fallback(B):
