@@ -424,7 +424,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8])
@@ -435,7 +435,7 @@ def main():
                     help="bound of the workload's device scratch (request tables, staged rows); 0 = none. Less scratch "
                          "means fewer page requests in flight per warp and more faults")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--clock-period", type=float, default=0.5, help="seconds between NVML clock samples")
+    ap.add_argument("--clock-period", type=float, default=0.1, help="seconds between NVML clock samples")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
