@@ -1349,10 +1349,16 @@ int gpuvm_gather_f32(gpuvm_t h, size_t x_off, const int64_t *d_idx, size_t n_idx
     const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
     const size_t slots = items < (size_t)grid * requesters ? items : (size_t)grid * requesters;   // warps that get work
     const size_t tables_bytes = direct ? 0 : (slots * batch * sizeof(unsigned int) + 255) & ~size_t(255);
-    unsigned int *tables = static_cast<unsigned int *>(gpuvm_scratch_(h, tables_bytes + sizeof(gpuvm_shared_queue)));
-    if (!tables) return GPUVM_E_ALLOC;
-    gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, reinterpret_cast<unsigned char *>(tables) + tables_bytes,
-                                                       static_cast<cudaStream_t>(stream));
+    const bool want_ring = (size_t(1) << m.vm.page_shift) >= kSharedQueueMinPage;
+    unsigned int *tables = nullptr;
+    gpuvm_shared_queue *shared_queue = nullptr;
+    if (tables_bytes || want_ring) {                          // the table-free form with small pages needs no scratch at all
+        tables = static_cast<unsigned int *>(gpuvm_scratch_(h, tables_bytes + (want_ring ? sizeof(gpuvm_shared_queue) : 0)));
+        if (!tables) return GPUVM_E_ALLOC;
+        if (want_ring)
+            shared_queue = shared_queue_at(m.vm, reinterpret_cast<unsigned char *>(tables) + tables_bytes,
+                                           static_cast<cudaStream_t>(stream));
+    }
     // staging of the migrator warps: kGatherStages pieces of at most kGatherChunk bytes each
     const unsigned int stage_chunk = (unsigned int)((size_t(1) << m.vm.page_shift) < kGatherChunk ? (size_t(1) << m.vm.page_shift) : kGatherChunk);
     const unsigned int stage_count = stage_chunk >= 128 ? kGatherStages : 0;     // tiny pages: copy through registers
