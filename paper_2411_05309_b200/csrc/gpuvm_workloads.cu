@@ -38,6 +38,7 @@ struct Paged {
     static __device__ __forceinline__ uint4 load16(const void *p) { return gpuvm_load16(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { gpuvm_store16(p, v); }
     static __device__ __forceinline__ int load_i32(const void *p) { return gpuvm_load(static_cast<const int *>(p)); }
+    static __device__ __forceinline__ long long load_i64(const void *p) { return gpuvm_load(static_cast<const long long *>(p)); }
 };
 
 struct Raw {
@@ -59,6 +60,7 @@ struct Raw {
     static __device__ __forceinline__ uint4 load16(const void *p) { return *static_cast<const uint4 *>(p); }
     static __device__ __forceinline__ void store16(void *p, uint4 v) { *static_cast<uint4 *>(p) = v; }
     static __device__ __forceinline__ int load_i32(const void *p) { return *static_cast<const int *>(p); }
+    static __device__ __forceinline__ long long load_i64(const void *p) { return *static_cast<const long long *>(p); }
 };
 
 __device__ __forceinline__ unsigned int warp_in_grid() { return (blockIdx.x * blockDim.x + threadIdx.x) >> 5; }
@@ -552,9 +554,22 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             if (ahead >= (long long)off_off && ahead < (long long)(off_off + 8ull * nv)) m.prefetch((unsigned long long)ahead);
         }
         // row offsets of the chunk: off[v0 .. v0+32], clamped to the nv + 1 entries that exist
-        long long lo = m.template read<long long>(off_off, v < nv ? v : nv);
-        long long hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
-        if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
+        // (one pin for all 33 when they lie in one unit, which they do except at unit ends and at the last chunk)
+        long long lo, hi;
+        const unsigned long long ob = off_off + 8ull * v0;
+        if (v0 + 32 <= nv && ob % unit + 33 * 8 <= unit) {
+            gpuvm_token tok_o;
+            const unsigned char *po = m.pin(ob, GPUVM_READ, tok_o);
+            if (!po) break;
+            lo = Mem::load_i64(po + 8 * lane);
+            hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+            if (lane == 31) hi = Mem::load_i64(po + 8 * 32);
+            m.release(tok_o);
+        } else {
+            lo = m.template read<long long>(off_off, v < nv ? v : nv);
+            hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+            if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
+        }
         if (!active) { lo = 0; hi = 0; }
         // long neighbour lists: cut them at unit boundaries and queue the pieces for the grid
         unsigned int bigs = __ballot_sync(0xFFFFFFFFu, hi - lo >= kBigDegree);
