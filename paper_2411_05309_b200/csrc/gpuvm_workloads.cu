@@ -322,6 +322,7 @@ __global__ void __launch_bounds__(kGatherMaxWarps * 32, 1) gather_batch_kernel(g
 // ------------------------------------------------------- graph sweeps (BFS, CC, SSSP)
 constexpr long long kBigDegree = 4096;     // neighbour lists at least this long are spread over the grid
 constexpr unsigned int kBigQueue = 65536;  // entries of the span queue (four int64 each: first edge, end, vertex, -)
+constexpr unsigned int kChunksPerTicket = 2;  // consecutive chunks of 32 vertices a warp draws at a time
 constexpr unsigned int kSpanPoll = 4;       // a warp looks into the span queue before every kSpanPoll-th chunk
 constexpr long long kAhead = 16;           // pages of look-ahead of the sweeps' prefetches
 
@@ -518,7 +519,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
     const unsigned long long unit = m.unit();
     const unsigned int n_chunks = (nv + 31) / 32;
     const long long epoch = sweep + 1;
-    unsigned int found = 0, my_done = 0, iter = 0;
+    unsigned int found = 0, my_done = 0, iter = 0, next_chunk = 0, last_chunk = 0;
     for (;;) {
         // ---- a piece of a long neighbour list, if one is waiting (looked for before every kSpanPoll-th chunk)
         if ((iter++ & (kSpanPoll - 1)) == 0) {
@@ -530,17 +531,22 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
                 continue;
             }
         }
-        // ---- the next chunk of 32 vertices
-        unsigned int chunk = 0;
-        if (lane == 0) chunk = atomicAdd(counters + kCntTicket, 1u);
-        chunk = __shfl_sync(0xFFFFFFFFu, chunk, 0);
-        if (chunk >= n_chunks) {
-            // no chunk left: report the finished ones, then help with the pieces until all chunks
-            // are finished and all pieces taken
-            if (lane == 0 && my_done) { __threadfence(); atomicAdd(counters + kCntDone, my_done); }
-            found += drain_pieces<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, counters, n_chunks, epoch, lane);
-            break;
+        // ---- the next chunk of 32 vertices (a ticket is good for kChunksPerTicket consecutive chunks)
+        if (next_chunk == last_chunk) {
+            unsigned int t = 0;
+            if (lane == 0) t = atomicAdd(counters + kCntTicket, kChunksPerTicket);
+            t = __shfl_sync(0xFFFFFFFFu, t, 0);
+            if (t >= n_chunks) {
+                // no chunk left: report the finished ones, then help with the pieces until all chunks
+                // are finished and all pieces taken
+                if (lane == 0 && my_done) { __threadfence(); atomicAdd(counters + kCntDone, my_done); }
+                found += drain_pieces<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, counters, n_chunks, epoch, lane);
+                break;
+            }
+            next_chunk = t;
+            last_chunk = t + kChunksPerTicket < n_chunks ? t + kChunksPerTicket : n_chunks;
         }
+        const unsigned int chunk = next_chunk++;
         ++my_done;
         const unsigned long long v0 = 32ull * ((sweep & 1) ? n_chunks - 1 - chunk : chunk);
         const unsigned long long v = v0 + lane;
