@@ -682,13 +682,36 @@ __global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsign
         if (lane < 2) vr = m.template read<int>(chunk_off, (unsigned long long)c + lane);   // chunk table has n_chunks + 1 entries
         const unsigned int v_first = (unsigned int)__shfl_sync(0xFFFFFFFFu, vr, 0);
         const unsigned int v_last = (unsigned int)__shfl_sync(0xFFFFFFFFu, vr, 1);
-        for (unsigned int v0 = v_first; v0 <= v_last && v0 < nv; v0 += 32) {
+        // which groups of 32 vertices have an active one: eight groups' flags are loaded at a time (a chunk
+        // in a region of low degrees spans tens of thousands of vertices)
+        for (unsigned int g0 = v_first; g0 <= v_last && g0 < nv; g0 += 256) {
+        unsigned int group_active = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const unsigned long long vk = (unsigned long long)g0 + 32u * k + lane;
+            const bool a = vk <= v_last && vk < nv && op.active(vk);
+            group_active |= (__any_sync(0xFFFFFFFFu, a) ? 1u : 0u) << k;
+        }
+        for (unsigned int v0 = g0; group_active; v0 += 32, group_active >>= 1) {
+            if (!(group_active & 1u)) continue;
             const unsigned long long v = (unsigned long long)v0 + lane;
             const bool active = v <= v_last && v < nv && op.active(v);
             if (!__any_sync(0xFFFFFFFFu, active)) continue;
-            long long lo = m.template read<long long>(off_off, v < nv ? v : nv);
-            long long hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
-            if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
+            long long lo, hi;                                    // one pin for the 33 row offsets when they lie in one unit
+            const unsigned long long ob = off_off + 8ull * v0;
+            if ((unsigned long long)v0 + 32 <= nv && ob % m.unit() + 33 * 8 <= m.unit()) {
+                gpuvm_token tok_o;
+                const unsigned char *po = m.pin(ob, GPUVM_READ, tok_o);
+                if (!po) return;
+                lo = Mem::load_i64(po + 8 * lane);
+                hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+                if (lane == 31) hi = Mem::load_i64(po + 8 * 32);
+                m.release(tok_o);
+            } else {
+                lo = m.template read<long long>(off_off, v < nv ? v : nv);
+                hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+                if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
+            }
             if (lo < c_lo) lo = c_lo;
             if (hi > c_hi) hi = c_hi;
             unsigned int touch = __ballot_sync(0xFFFFFFFFu, active && hi > lo);
@@ -705,6 +728,7 @@ __global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsign
                 found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), blo, bhi, lane);
             }
             m.release(tok);
+        }
         }
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
