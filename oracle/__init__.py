@@ -55,6 +55,10 @@ def _load():
             "orc_pager_flush": (None, [vp]),
             "orc_pager_counters": (None, [vp, vp]),
             "orc_pager_check": (i32, [vp]),
+            "orc_pager_debug_poke": (i32, [vp, i32, u64, u64]),
+            "orc_pager_trace": (None, [vp, vp, u64]),
+            "orc_pager_trace_len": (u64, [vp]),
+            "orc_belady_faults": (u64, [vp, u64, u64, u64]),
             "orc_stream_sum_i32_paged": (ctypes.c_int64, [vp, u64, u64]),
             "orc_gather_block_sums_paged": (None, [vp, u64, vp, u64, u64, vp, vp]),
             "orc_bfs_levels_paged": (None, [vp, u64, u64, u64, u64, vp]),
@@ -175,6 +179,26 @@ class Pager:
     def check(self) -> int:
         return int(_load().orc_pager_check(self._h))
 
+    def debug_poke(self, which: str, i: int, v: int) -> None:
+        """Test hook: damage one word of the tables (which: 'map', 'frame_page', 'resident')."""
+        rc = _load().orc_pager_debug_poke(self._h, {"map": 0, "frame_page": 1, "resident": 2}[which], i,
+                                          v & 0xFFFFFFFFFFFFFFFF)
+        if rc != 0:
+            raise IndexError((which, i))
+
+    def record_trace(self, capacity: int) -> np.ndarray:
+        """Record the page numbers of the accesses that follow (runs of one page collapsed) into a
+        new array of `capacity` entries; trace() returns the part that was filled."""
+        self._trace = np.empty(capacity, dtype=np.uint64)
+        _load().orc_pager_trace(self._h, self._trace.ctypes.data, capacity)
+        return self._trace
+
+    def trace(self) -> np.ndarray:
+        n = int(_load().orc_pager_trace_len(self._h))
+        if n > self._trace.size:
+            raise OverflowError(f"trace needs {n} entries, {self._trace.size} were provided")
+        return self._trace[:n]
+
     # workloads through the pager; offsets are byte offsets inside the backing store
     def stream_sum_i32(self, a_off: int, n: int) -> int:
         return int(_load().orc_stream_sum_i32_paged(self._h, a_off, n))
@@ -201,6 +225,35 @@ class Pager:
         _load().orc_embag_f32_paged(self._h, t_off, dims, _p(rows, np.int64), n_bags, bag,
                                     _p(out, np.float32))
         return out
+
+
+NONE = 0xFFFFFFFFFFFFFFFF
+
+
+def belady_faults(trace: np.ndarray, n_pages: int, n_frames: int) -> int:
+    """Faults of Belady's optimal replacement on a trace of page numbers."""
+    t = np.ascontiguousarray(trace, dtype=np.uint64)
+    assert t.size == 0 or int(t.max()) < n_pages
+    return int(_load().orc_belady_faults(t.ctypes.data, t.size, n_pages, n_frames))
+
+
+def replay_counts(trace: np.ndarray, n_pages: int, page_bytes: int, n_frames: int, belady: bool = True) -> dict:
+    """Fault counts of a read-only page trace under the sequential replay's two policies and
+    under optimal replacement (what no policy can beat with this many frames)."""
+    out = {}
+    host = np.zeros(1, dtype=np.uint8)
+    for name, policy in (("clock", CLOCK), ("fifo", FIFO)):
+        h = _load().orc_pager_create(host.ctypes.data, n_pages * page_bytes, page_bytes, n_frames, policy, 0)
+        t = np.ascontiguousarray(trace, dtype=np.uint64)
+        _load().orc_pager_replay(h, t.ctypes.data, None, t.size)
+        c = np.zeros(10, dtype=np.uint64)
+        _load().orc_pager_counters(h, c.ctypes.data)
+        out[name] = int(c[2])
+        _load().orc_pager_destroy(h)
+    if belady:
+        out["belady"] = belady_faults(trace, n_pages, n_frames)
+    out["distinct"] = int(np.unique(trace).size)
+    return out
 
 
 def oversubscription_level(workload_bytes: float, gpu_bytes: float) -> float:

@@ -227,6 +227,9 @@ typedef struct {
     /* counters */
     uint64_t accesses, hits, faults, evictions, writebacks;
     uint64_t bytes_in, bytes_out, resident, max_resident, hand_steps;
+    /* optional record of the page numbers accessed, runs of one page collapsed to one entry */
+    uint64_t *trace;
+    uint64_t trace_cap, trace_len, trace_last;
 } orc_pager;
 
 static uint64_t page_len(const orc_pager *p, uint64_t vpn)
@@ -255,8 +258,27 @@ orc_pager *orc_pager_create(void *host, uint64_t bytes, uint64_t page_bytes,
     for (uint64_t i = 0; i < p->n_pages; ++i) p->map[i] = ORC_NONE;
     for (uint64_t i = 0; i < n_frames; ++i) p->frame_page[i] = ORC_NONE;
     if (move_bytes) p->frames = (uint8_t *)malloc(n_frames * page_bytes);
+    p->trace_last = ORC_NONE;
     return p;
 }
+
+/*
+ * Record the sequence of page numbers that orc_pager_access sees from now on into buf (caller's
+ * memory, cap entries).  Consecutive accesses to one page are recorded once: every access of such
+ * a run after the first is a hit under any policy and leaves reference and dirty state as the
+ * first access of the run left it (for read-only traces), so fault counts of the collapsed trace
+ * equal those of the full one.  orc_pager_trace_len returns the number of entries the run would
+ * have needed; entries beyond cap are counted but not stored.
+ */
+void orc_pager_trace(orc_pager *p, uint64_t *buf, uint64_t cap)
+{
+    p->trace = buf;
+    p->trace_cap = cap;
+    p->trace_len = 0;
+    p->trace_last = ORC_NONE;
+}
+
+uint64_t orc_pager_trace_len(const orc_pager *p) { return p->trace_len; }
 
 void orc_pager_destroy(orc_pager *p)
 {
@@ -287,6 +309,11 @@ static void evict_frame(orc_pager *p, uint64_t f)
 uint64_t orc_pager_access(orc_pager *p, uint64_t vpn, int is_write)
 {
     p->accesses++;
+    if (p->trace && vpn != p->trace_last) {
+        if (p->trace_len < p->trace_cap) p->trace[p->trace_len] = vpn;
+        p->trace_len++;
+        p->trace_last = vpn;
+    }
     uint64_t f = p->map[vpn];
     if (f != ORC_NONE) {                      /* Fig. 2 step 2: resident */
         p->hits++;
@@ -366,6 +393,57 @@ int orc_pager_check(const orc_pager *p)
         }
     if (mapped != used || mapped != p->resident || mapped > p->n_frames) return 5;
     return 0;
+}
+
+/*
+ * Test hook for the checker above: overwrite one word of the replay's tables so that a test can
+ * see orc_pager_check report each kind of damage.  which: 0 = map[i] (page table), 1 =
+ * frame_page[i] (ring), 2 = the resident counter (i ignored).  v = UINT64_MAX means "none".
+ */
+int orc_pager_debug_poke(orc_pager *p, int which, uint64_t i, uint64_t v)
+{
+    if (which == 0 && i < p->n_pages) { p->map[i] = v; return 0; }
+    if (which == 1 && i < p->n_frames) { p->frame_page[i] = v; return 0; }
+    if (which == 2) { p->resident = v; return 0; }
+    return -1;
+}
+
+/*
+ * Belady's optimal replacement (the lower bound of any policy, used next to the FIFO ring of
+ * Section 3.3 and the clock variant): number of faults of `trace` with n_frames frames when, on
+ * a fault with no free frame, the resident page whose next use lies farthest in the future (or
+ * that is never used again) is evicted.  Plain form: next-use positions are computed by one
+ * backward pass, the victim is found by a linear scan over the frames.
+ */
+uint64_t orc_belady_faults(const uint64_t *trace, uint64_t n, uint64_t n_pages, uint64_t n_frames)
+{
+    const uint64_t NEVER = UINT64_MAX;
+    uint64_t *next = (uint64_t *)malloc((n ? n : 1) * sizeof(uint64_t));     /* next[i]: next position of trace[i] */
+    uint64_t *last_seen = (uint64_t *)malloc((n_pages ? n_pages : 1) * sizeof(uint64_t));
+    uint64_t *where = (uint64_t *)malloc((n_pages ? n_pages : 1) * sizeof(uint64_t)); /* page -> frame or NONE */
+    uint64_t *frame_page = (uint64_t *)malloc(n_frames * sizeof(uint64_t));
+    uint64_t *frame_next = (uint64_t *)malloc(n_frames * sizeof(uint64_t));
+    for (uint64_t v = 0; v < n_pages; ++v) { last_seen[v] = NEVER; where[v] = ORC_NONE; }
+    for (uint64_t i = n; i-- > 0;) { next[i] = last_seen[trace[i]]; last_seen[trace[i]] = i; }
+    uint64_t used = 0, faults = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        uint64_t v = trace[i], f = where[v];
+        if (f == ORC_NONE) {
+            faults++;
+            if (used < n_frames) f = used++;
+            else {
+                f = 0;
+                for (uint64_t g = 1; g < n_frames; ++g)
+                    if (frame_next[g] > frame_next[f]) f = g;
+                where[frame_page[f]] = ORC_NONE;
+            }
+            frame_page[f] = v;
+            where[v] = f;
+        }
+        frame_next[f] = next[i];
+    }
+    free(next); free(last_seen); free(where); free(frame_page); free(frame_next);
+    return faults;
 }
 
 /* Element accessors through the pager.  An element never straddles a page

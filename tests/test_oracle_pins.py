@@ -440,3 +440,89 @@ def test_sssp_against_bellman_ford_and_scipy():
             m = csr_matrix((list(pos.values()), ([k[0] for k in pos], [k[1] for k in pos])), shape=(nv, nv))
             sp = dijkstra(m, directed=True, indices=src)
             assert list(got) == [int(x) if np.isfinite(x) else INF for x in sp]
+
+
+def test_pager_check_reports_each_kind_of_damage():
+    """The replay's own invariant checker is only worth something if it can say no: damage its
+    tables one word at a time and see each return code (a checker that always answers 0 would pass
+    every other test)."""
+    n_pages, frames = 12, 4
+
+    def fresh():
+        pg = make_pager(n_pages, 16, frames, oracle.CLOCK)
+        for p in (0, 5, 7):                          # frames 0, 1, 2 taken; frame 3 free; pages 1.. unmapped
+            pg.access(p)
+        assert pg.check() == 0
+        return pg
+
+    pg = fresh(); pg.debug_poke("map", 5, frames); assert pg.check() == 1         # page table names a frame that does not exist
+    pg = fresh(); pg.debug_poke("map", 3, 0); assert pg.check() == 2              # two pages claim frame 0
+    pg = fresh(); pg.debug_poke("frame_page", 3, n_pages + 5); assert pg.check() == 3   # ring names a page that does not exist
+    pg = fresh(); pg.debug_poke("frame_page", 3, 9); assert pg.check() == 4       # ring names a page that is not mapped there
+    pg = fresh(); pg.debug_poke("resident", 0, 2); assert pg.check() == 5         # counter disagrees with the tables
+    pg = fresh(); pg.debug_poke("map", 7, oracle.NONE); assert pg.check() == 4    # a mapping lost, its frame still names the page
+    pg = fresh(); pg.debug_poke("frame_page", 1, oracle.NONE); assert pg.check() == 2   # a frame emptied under a mapped page
+    with pytest.raises(IndexError):
+        fresh().debug_poke("map", n_pages, 0)
+
+
+@pytest.mark.parametrize("frames", [1, 2, 3, 4, 8, 17])
+def test_belady_count_against_brute_force(frames):
+    for trace in random_traces():
+        trace = [int(t) for t in trace]
+        n_pages = max(trace) + 1
+        assert oracle.belady_faults(np.array(trace), n_pages, frames) == belady_opt_faults(trace, frames)
+    assert oracle.belady_faults(np.empty(0, np.uint64), 4, frames) == 0
+
+
+def test_belady_count_on_the_textbook_strings():
+    for _, frames, policy, faults, string in _rows("page_replacement_strings.txt"):
+        if policy != "fifo":
+            trace = np.array([int(t) for t in string.split()])
+            assert oracle.belady_faults(trace, int(trace.max()) + 1, int(frames)) == int(faults)
+
+
+def test_recorded_trace_collapses_runs_and_keeps_the_fault_counts():
+    rng = np.random.default_rng(11)
+    pages = rng.integers(0, 40, 500)
+    full = np.repeat(pages, rng.integers(1, 6, pages.size))           # runs of 1..5 accesses per page
+    for frames in (1, 3, 8, 40):
+        for policy, name in ((oracle.CLOCK, "clock"), (oracle.FIFO, "fifo")):
+            pg = make_pager(40, 16, frames, policy, move=False)
+            pg.record_trace(full.size)
+            pg.replay(full)
+            got = pg.trace()
+            keep = np.concatenate([[True], full[1:] != full[:-1]])
+            assert np.array_equal(got, full[keep].astype(np.uint64))   # exactly the run heads, in order
+            counts = oracle.replay_counts(got, 40, 16, frames)
+            assert counts[name] == pg.counters()["faults"]             # collapsed trace: same faults
+            assert counts["belady"] == belady_opt_faults([int(t) for t in full], frames)
+            assert counts["belady"] <= min(counts["clock"], counts["fifo"]) and counts["distinct"] == np.unique(full).size
+            pg.close()
+    pg = make_pager(40, 16, 4, oracle.CLOCK, move=False)
+    pg.record_trace(3)
+    pg.replay(full)
+    with pytest.raises(OverflowError):
+        pg.trace()
+
+
+def test_bfs_page_trace_is_the_canonical_order():
+    """Level by level, vertices ascending, per vertex its two row offsets and then its edges: on a
+    hand-made graph the recorded page trace is written out and compared."""
+    # 4 vertices; page = 16 bytes = 2 row offsets or 4 columns; offsets at byte 0 (5 int64 = 40 bytes -> 3 pages),
+    # columns from byte 48 (page 3)
+    off = np.array([0, 2, 3, 3, 6], dtype=np.int64)         # 0 -> {1, 3}; 1 -> {3}; 2 -> {}; 3 -> {0, 1, 2}
+    col = np.array([1, 3, 3, 0, 1, 2], dtype=np.int32)
+    host = np.zeros(48 + 32, dtype=np.uint8)
+    host[:40] = np.frombuffer(off.tobytes(), np.uint8)
+    host[48:48 + 24] = np.frombuffer(col.tobytes(), np.uint8)
+    pg = oracle.Pager(host, 16, 2, oracle.CLOCK, True)
+    pg.record_trace(64)
+    lvl = pg.bfs_levels(0, 48, 4, 0)
+    assert lvl.tolist() == [0, 1, 2, 1]
+    # level 0: vertex 0: off[0], off[1] (page 0), edges 0..1 (page 3)
+    # level 1: vertex 1: off[1] (page 0), off[2] (page 1), edge 2 (page 3); vertex 3: off[3] (page 1), off[4] (page 2),
+    #          edges 3 (page 3), 4..5 (page 4)
+    # level 2: vertex 2: off[2], off[3] (page 1), no edges
+    assert pg.trace().tolist() == [0, 3, 0, 1, 3, 1, 2, 3, 4, 1]
+    pg.close()
