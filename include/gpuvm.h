@@ -46,7 +46,12 @@ typedef enum gpuvm_status {
     GPUVM_E_TIMEOUT = -8,    /* a device-side wait ran out (sticky, see gpuvm_stats)  */
     GPUVM_E_RANGE = -9,      /* a device accessor was given an offset past the end    */
     GPUVM_E_INVARIANT = -10, /* gpuvm_check found a broken page-table invariant       */
-    GPUVM_E_NODEVICE = -11   /* no CUDA device                                        */
+    GPUVM_E_NODEVICE = -11,  /* no CUDA device                                        */
+    GPUVM_E_PINS = -12,      /* more than 2^23 simultaneous references to one page
+                                (sticky): the request was refused before the 24-bit
+                                reference counter could carry into the frame field    */
+    GPUVM_E_FRAMES = -13     /* the pool has too few frames for the pages this
+                                workload holds pinned at once (see gpuvm_safe_warps)  */
 } gpuvm_status;
 
 /* Eviction policy of the frame ring (Section 3.3 "Eviction scheme").
@@ -72,7 +77,16 @@ typedef struct gpuvm_dev {
     unsigned int page_shift;   /* log2(page_bytes)                                      */
     unsigned int policy;       /* GPUVM_POLICY_*                                        */
     unsigned int spin_limit_us;/* upper bound of every device-side wait                 */
+    unsigned int debug;        /* GPUVM_DEBUG_* flags                                   */
+    unsigned int reserved;
 } gpuvm_dev_t;
+
+/* Debug flags (gpuvm_set_debug).  POISON: whoever evicts a page fills its frame with the
+ * byte pattern 0xA5 before the frame is handed on, so that a thread that still reads the
+ * frame of a page it no longer holds sees the pattern instead of plausible old data (a
+ * stale read then shows up as a wrong result in any parity check; the race checker of the
+ * CUDA tools is not needed to see it).  Costs one extra write of the frame per eviction. */
+enum { GPUVM_DEBUG_POISON = 1 };
 
 /* Counters accumulated by GPU threads since the last gpuvm_reset(). */
 typedef struct gpuvm_stats {
@@ -90,7 +104,11 @@ typedef struct gpuvm_stats {
     uint64_t hand_steps;      /* frame-ring slots inspected                            */
     uint64_t retries;         /* wait-loop rounds that made no progress                */
     uint64_t resident;        /* pages resident now                                    */
-    int32_t error;            /* sticky device error: 0, GPUVM_E_TIMEOUT, GPUVM_E_RANGE*/
+    uint64_t ring_drops;      /* entries of a fault ring that were given up on after a
+                                 bounded wait (slot never filled, slot never cleared, or
+                                 a popped page that was not waiting for a migrator): each
+                                 also sets the sticky GPUVM_E_TIMEOUT; 0 in a healthy run */
+    int32_t error;            /* sticky device error: 0, GPUVM_E_TIMEOUT, _RANGE, _PINS */
     uint32_t reserved;
     uint64_t error_page;      /* page number the first error was raised for            */
 } gpuvm_stats_t;
@@ -135,6 +153,10 @@ int gpuvm_destroy(gpuvm_t h);
  * the sticky device error if one is set, else 0. */
 int gpuvm_stats(gpuvm_t h, gpuvm_stats_t *out);
 
+/* The same on a stream of the caller's choice: only `stream` is synchronised (not the
+ * device), so a handle can be read out while other streams keep working. */
+int gpuvm_stats_on(gpuvm_t h, gpuvm_stats_t *out, void *stream);
+
 /* Copy the by-value device view to *out (host pointer). */
 int gpuvm_device_view(gpuvm_t h, gpuvm_dev_t *out);
 
@@ -152,16 +174,24 @@ int gpuvm_flush(gpuvm_t h, void *stream);
  * support"). */
 int gpuvm_reset(gpuvm_t h);
 
+/* gpuvm_reset enqueued on `stream` without any synchronisation: the three clears are
+ * ordered after earlier work on that stream and before later work on it. */
+int gpuvm_reset_on(gpuvm_t h, void *stream);
+
 /* Run the invariant kernel: every resident page maps to exactly one frame and
  * that frame names it back, occupancy <= capacity, nothing left in a transient
  * state, all reference counters zero.  Fills *out (host pointer); returns
  * GPUVM_E_INVARIANT if any bad_* count is non-zero. */
 int gpuvm_check(gpuvm_t h, gpuvm_check_t *out);
 
+/* gpuvm_check on `stream`; synchronises that stream only. */
+int gpuvm_check_on(gpuvm_t h, gpuvm_check_t *out, void *stream);
+
 /* Options.  policy: GPUVM_POLICY_*; spin_limit_us: bound of device-side waits
  * (default 10 s).  Take effect for views fetched afterwards. */
 int gpuvm_set_policy(gpuvm_t h, int policy);
 int gpuvm_set_spin_limit_us(gpuvm_t h, unsigned int spin_limit_us);
+int gpuvm_set_debug(gpuvm_t h, unsigned int flags);   /* GPUVM_DEBUG_*; 0 = off (default) */
 
 /* Device scratch of the batched workload entry points (request tables, staging of gathered
  * rows; not pages of the backing store).  It belongs to the handle, is allocated at the first
@@ -188,6 +218,9 @@ double gpuvm_inflight_pages(double latency_s, double bytes_per_s, double page_by
  * a page that stays "being fetched" so that a bounded device wait can be seen to
  * expire with an error status instead of hanging). */
 int gpuvm_debug_poke_pte(gpuvm_t h, uint64_t page, uint64_t value);
+
+/* Test hook: read one page-table entry into *value (host pointer).  Synchronises the device. */
+int gpuvm_debug_peek_pte(gpuvm_t h, uint64_t page, uint64_t *value);
 
 const char *gpuvm_strerror(int status);
 int gpuvm_last_cuda_error(gpuvm_t h);

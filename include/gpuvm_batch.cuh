@@ -96,7 +96,8 @@ constexpr unsigned int kNotReady = 0xFFFFFFFFu;   /* "frame" values a leader han
 constexpr unsigned int kRejected = 0xFFFFFFFFu;   /* vpn of a request that was refused when it was set */
 
 /* Any lane.  False when the ring is (nearly) full: the caller keeps the fault and retries. */
-__device__ __forceinline__ bool fault_queue_push(gpuvm_fault_queue *q, unsigned int vpn, int mode)
+__device__ __forceinline__ bool fault_queue_push(gpuvm_fault_queue *q, unsigned int vpn, int mode,
+                                                 const gpuvm_dev_t *vm_for_errors = nullptr)
 {
     volatile unsigned int *vh = &q->head, *vt = &q->tail;
     const unsigned int item = (vpn + 1u) | (mode == kWrite ? 0x80000000u : 0u);
@@ -113,6 +114,9 @@ __device__ __forceinline__ bool fault_queue_push(gpuvm_fault_queue *q, unsigned 
                 unsigned int *slot = &g->slot[gt % GPUVM_SHARED_QUEUE_SLOTS];
                 unsigned int spins = 0;
                 while (ld_relaxed_u32(slot) != 0u && ++spins < (1u << 20)) { }   /* its last reader has not cleared it yet */
+                if (ld_relaxed_u32(slot) != 0u) {            /* still there: the entry under it is lost, say so */
+                    if (vm_for_errors) { stat_add(*vm_for_errors, kRingDrops, 1); set_error(*vm_for_errors, GPUVM_E_TIMEOUT, vpn); }
+                }
                 st_relaxed_u32(slot, item);
                 return true;
             }
@@ -136,24 +140,18 @@ __device__ __forceinline__ bool migrate_page(const gpuvm_dev_t &vm, unsigned lon
                                              BulkStage *bulk = nullptr)
 {
     unsigned char *fr = vm.pool + ((unsigned long long)h << vm.page_shift);
-    if (victim != ~0ull) {
-        if (vdirty) {
-            warp_copy<8, true>(vm.host + (victim << vm.page_shift), fr, page_len(vm, victim) >> 4, lane, 32);
-            __threadfence_system();
-            __syncwarp();
-        }
-        if (lane == L) {
-            atomicXor(vm.pte + victim, kEvicting | ((unsigned long long)h << kFrameShift) | (vdirty ? kDirty : 0ull));
-            stat_add(vm, kEvictions, 1);
-            if (vdirty) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, victim)); }
-        }
-    }
+    retire_victim(vm, h, victim, vdirty, lane, 32, 0xFFFFFFFFu, lane == L);
     if (bulk) {
         int ok = 1;
         if (lane == L) {
-            ok = bulk_copy_in(*bulk, fr, vm.host + (vpn << vm.page_shift), (unsigned int)page_len(vm, vpn),
-                              (unsigned long long)vm.spin_limit_us * 1000ull);
+            const unsigned long long limit_ns = (unsigned long long)vm.spin_limit_us * 1000ull;
+            ok = bulk_copy_in(*bulk, fr, vm.host + (vpn << vm.page_shift), (unsigned int)page_len(vm, vpn), limit_ns);
             if (!ok) {
+                /* Nothing may still be writing into the frame when it is given back: wait for the
+                 * staging-to-frame copies that were committed, and (bounded) for the host-to-staging
+                 * copies in flight, before the entry and the ring slot are released. */
+                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                bulk_stage_drain(*bulk, limit_ns);
                 set_error(vm, GPUVM_E_TIMEOUT, vpn);
                 atomicXor(vm.pte + vpn, kBusy);                      /* BUSY -> INVALID */
                 st_relaxed_u32(vm.frame_vpn + h, kFrameFree);
@@ -165,13 +163,7 @@ __device__ __forceinline__ bool migrate_page(const gpuvm_dev_t &vm, unsigned lon
     }
     __threadfence();
     __syncwarp();
-    if (lane == L) {
-        st_relaxed_u32(vm.frame_vpn + h, (unsigned int)vpn);
-        atomicXor(vm.pte + vpn, (kBusy ^ kValid) | ((unsigned long long)h << kFrameShift) |
-                                    (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull) | (mode == kWrite ? kDirty : 0ull));
-        stat_add(vm, kFaults, 1);
-        stat_add(vm, kBytesIn, page_len(vm, vpn));
-    }
+    if (lane == L) publish(vm, vpn, h, mode);
     return true;
 }
 
@@ -212,6 +204,7 @@ static __device__ __noinline__ void gpuvm_migrator_loop(const gpuvm_dev_t vm, gp
                 unsigned int spins = 0;
                 while ((item = *slot) == 0u && ++spins < (1u << 24)) { }   /* the pusher is between its two stores */
                 *slot = 0u;
+                if (item == 0u) { stat_add(vm, kRingDrops, 1); set_error(vm, GPUVM_E_TIMEOUT, ~0ull); }
             }
         }
         if (lane == 0 && item == 0u && q->shared) {
@@ -222,7 +215,15 @@ static __device__ __noinline__ void gpuvm_migrator_loop(const gpuvm_dev_t vm, gp
                 unsigned int spins = 0;
                 while ((item = ld_relaxed_u32(slot)) == 0u && ++spins < (1u << 22)) { }   /* the pusher is between its two stores */
                 st_relaxed_u32(slot, 0u);
+                if (item == 0u) { stat_add(vm, kRingDrops, 1); set_error(vm, GPUVM_E_TIMEOUT, ~0ull); }
             }
+        }
+        /* An entry names a page that its pusher turned BUSY and nobody else may touch.  An entry
+         * that was given up on above and filled in late can surface a ring cycle later, when its
+         * page is long done: anything that is not BUSY is dropped, never migrated. */
+        if (lane == 0 && item != 0u) {
+            const unsigned long long w = ld_relaxed_u64(vm.pte + ((item & 0x7FFFFFFFu) - 1u));
+            if ((w & kStMask) != kBusy) { stat_add(vm, kRingDrops, 1); set_error(vm, GPUVM_E_TIMEOUT, (item & 0x7FFFFFFFu) - 1u); item = 0u; }
         }
         item = __shfl_sync(0xFFFFFFFFu, item, 0);
         if (item == 0u) {
@@ -390,6 +391,9 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                     leads[u] = lane == (unsigned int)(__ffs(group) - 1);
                     if (leads[u]) {
                         old[u] = atomicAdd(vm.pte + vpn[u], 1ull);
+                        /* far too many references to one page: the sticky error ends every wait of the
+                         * launch at its next idle round, long before the counter could carry */
+                        if ((old[u] & kRcMask) >= kRcLimit) set_error(vm, GPUVM_E_PINS, vpn[u]);
                         n_lanes += __popc(group) - 1;
                     }
                     todo |= 1ull << (j0 + u);
@@ -402,7 +406,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                     const int st = advance(vm, vm.pte + vpn[u], old[u] + 1ull, mode, frame);
                     if (st == kReady) ++n_hits;
                     else if (st == kWait) ++n_waits;
-                    else if (!(eager_push && queue && fault_queue_push(queue, vpn[u], mode))) own |= 1ull << (j0 + u);
+                    else if (!(eager_push && queue && fault_queue_push(queue, vpn[u], mode, &vm))) own |= 1ull << (j0 + u);
                 }
             }
         }
@@ -527,7 +531,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                 /* hand owned faults to the migrator warps; afterwards wait for the page like anyone */
                 while (own) {
                     const unsigned int jj = __ffsll((long long)own) - 1;
-                    if (!fault_queue_push(queue, table.vpn((64u * k + jj) * 32 + lane), mode)) break;
+                    if (!fault_queue_push(queue, table.vpn((64u * k + jj) * 32 + lane), mode, &vm)) break;
                     own &= own - 1;
                     progress = true;
                 }

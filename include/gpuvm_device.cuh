@@ -70,6 +70,8 @@ namespace gpuvm {
 
 /* ---- page-table entry: [state:2 @60][dirty @57][ref @56][frame:32 @24][refcount:24 @0] */
 constexpr unsigned long long kRcMask = 0xFFFFFFull;
+constexpr unsigned long long kRcLimit = 1ull << 23;   /* a pin that would take the counter beyond this is refused */
+constexpr unsigned long long kPinRefused = ~0ull;     /* what a refused pin hands to its group instead of the entry */
 constexpr int kFrameShift = 24;
 constexpr unsigned long long kFrameMask = 0xFFFFFFFFull << kFrameShift;
 constexpr unsigned long long kRef = 1ull << 56;
@@ -92,7 +94,7 @@ constexpr int kCtlCounters = 16;      /* kStatSlots slots of 16 words, one 128-b
 constexpr int kStatSlots = 32;
 constexpr int kCtlWords = kCtlCounters + kStatSlots * 16;
 enum Stat { kFaults = 0, kHits, kWaits, kLanes, kEvictions, kWritebacks, kFlushWritebacks,
-            kBytesIn, kBytesOut, kHandSteps, kRetries, kNumStats };
+            kBytesIn, kBytesOut, kHandSteps, kRetries, kRingDrops, kNumStats };
 
 enum Mode { kRead = 0, kWrite = 1, kWriteAll = 2 };
 
@@ -148,6 +150,18 @@ __device__ __forceinline__ unsigned long long pin_acquire(unsigned long long *pt
     return old;
 }
 
+/* Leader only: `w` is the entry including the reference just taken.  When the counter has
+ * left the range that 2^23 warp-level requests can reach, the reference is given back, the
+ * sticky GPUVM_E_PINS is set and kPinRefused is returned: the 24-bit counter never carries
+ * into the frame field. */
+__device__ __forceinline__ unsigned long long set_error_pins(const gpuvm_dev_t &vm, unsigned long long *pte);
+
+__device__ __forceinline__ unsigned long long guard_pin(const gpuvm_dev_t &vm, unsigned long long *pte, unsigned long long w)
+{
+    if ((w & kRcMask) <= kRcLimit) return w;
+    return set_error_pins(vm, pte);
+}
+
 __device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int *p)
 {
     unsigned int v;
@@ -177,6 +191,13 @@ __device__ __forceinline__ void set_error(const gpuvm_dev_t &vm, int code, unsig
 {
     if (atomicCAS(vm.ctl + kCtlErr, 0ull, (unsigned long long)(long long)code) == 0ull)
         vm.ctl[kCtlErrPage] = vpn;
+}
+
+__device__ __forceinline__ unsigned long long set_error_pins(const gpuvm_dev_t &vm, unsigned long long *pte)
+{
+    unpin(pte);
+    set_error(vm, GPUVM_E_PINS, (unsigned long long)(pte - vm.pte));
+    return kPinRefused;
 }
 
 __device__ __forceinline__ bool has_error(const gpuvm_dev_t &vm)
@@ -352,6 +373,49 @@ __device__ __forceinline__ bool bulk_copy_in(BulkStage &s, unsigned char *frame,
     return true;
 }
 
+/*
+ * Steps 6 and 6a for the `n` calling lanes (rank 0..n-1, all of `mask`, converged): the page
+ * `victim` (EVICTING, exclusively ours) leaves frame `h`.  A dirty victim is copied to the
+ * host, followed by a system-scope fence; then lane `L` turns its entry INVALID with one XOR
+ * that returns the frame and dirty bits to zero and leaves the counter alone.  In the poison
+ * debug mode the frame is then overwritten with a pattern before anybody gets it.
+ */
+__device__ __forceinline__ void retire_victim(const gpuvm_dev_t &vm, unsigned int h, unsigned long long victim, int vdirty,
+                                              unsigned int rank, unsigned int n, unsigned int mask, bool is_L)
+{
+    if (victim == ~0ull) return;
+    unsigned char *fr = vm.pool + ((unsigned long long)h << vm.page_shift);
+    if (vdirty) {
+        warp_copy<8, true>(vm.host + (victim << vm.page_shift), fr, page_len(vm, victim) >> 4, rank, n);
+        __threadfence_system();
+        __syncwarp(mask);
+    }
+    if (is_L) {
+        atomicXor(vm.pte + victim, kEvicting | ((unsigned long long)h << kFrameShift) | (vdirty ? kDirty : 0ull));
+        stat_add(vm, kEvictions, 1);
+        if (vdirty) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, victim)); }
+    }
+    if (vm.debug & GPUVM_DEBUG_POISON) {
+        const uint4 pat = make_uint4(0xA5A5A5A5u, 0xA5A5A5A5u, 0xA5A5A5A5u, 0xA5A5A5A5u);
+        const unsigned int n16 = 1u << (vm.page_shift - 4);
+        for (unsigned int i = rank; i < n16; i += n) st_frame16(fr + 16ull * i, pat);
+        __threadfence();
+        __syncwarp(mask);
+    }
+}
+
+/* Lane that publishes (step 7), after the warp barrier that follows the copy: the fence makes
+ * this thread's atomic a release for the frame stores of all lanes that passed the barrier. */
+__device__ __forceinline__ void publish(const gpuvm_dev_t &vm, unsigned long long vpn, unsigned int h, int mode)
+{
+    st_relaxed_u32(vm.frame_vpn + h, (unsigned int)vpn);
+    __threadfence();
+    atomicXor(vm.pte + vpn, (kBusy ^ kValid) | ((unsigned long long)h << kFrameShift) |
+                                (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull) | (mode != kRead ? kDirty : 0ull));
+    stat_add(vm, kFaults, 1);
+    if (mode != kWriteAll) stat_add(vm, kBytesIn, page_len(vm, vpn));
+}
+
 /* ------------------------------------------------------------ fault machinery */
 
 enum LaneState { kNew = 0, kWait, kOwn, kReady, kDone, kFail };
@@ -508,32 +572,14 @@ static __device__ __noinline__ bool slow_path(const gpuvm_dev_t vm, unsigned lon
             const unsigned long long bv = __shfl_sync(active, vpn, L);
             const int bmode = __shfl_sync(active, mode, L);
             unsigned char *fr = vm.pool + ((unsigned long long)bh << vm.page_shift);
-            if (bq != ~0ull) {
-                if (bd) {
-                    warp_copy<8, true>(vm.host + (bq << vm.page_shift), fr, page_len(vm, bq) >> 4, rank, nlanes);
-                    __threadfence_system();
-                    __syncwarp(active);
-                }
-                if ((int)lane == L) {
-                    /* EVICTING -> INVALID; frame and dirty bits return to zero, counter untouched */
-                    atomicXor(vm.pte + bq, kEvicting | ((unsigned long long)bh << kFrameShift) | (bd ? kDirty : 0ull));
-                    stat_add(vm, kEvictions, 1);
-                    if (bd) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, bq)); }
-                }
-            }
+            retire_victim(vm, bh, bq, bd, rank, nlanes, active, (int)lane == L);
             if (bmode != kWriteAll) {                        /* a page that will be overwritten entirely is not fetched */
                 warp_copy<8, false>(fr, vm.host + (bv << vm.page_shift), page_len(vm, bv) >> 4, rank, nlanes);
                 __threadfence();
             }
             __syncwarp(active);
             if ((int)lane == L) {
-                st_relaxed_u32(vm.frame_vpn + bh, (unsigned int)bv);
-                unsigned long long bits = (kBusy ^ kValid) | ((unsigned long long)bh << kFrameShift) |
-                                          (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull) |
-                                          (mode != kRead ? kDirty : 0ull);
-                atomicXor(pte, bits);                        /* step 7: publish */
-                stat_add(vm, kFaults, 1);
-                if (mode != kWriteAll) stat_add(vm, kBytesIn, page_len(vm, bv));
+                publish(vm, bv, bh, mode);                   /* step 7 */
                 st = kReady; frame = bh;
             }
         }
@@ -581,10 +627,14 @@ __device__ __forceinline__ bool access(const gpuvm_dev_t &vm, unsigned long long
     unsigned long long *pte = vm.pte + vpn;
     unsigned long long w = 0;
     if (is_leader) {
-        w = pin_acquire(pte) + 1ull;                         /* pin first, look afterwards */
+        w = guard_pin(vm, pte, pin_acquire(pte) + 1ull);     /* pin first, look afterwards */
         if (group & (group - 1)) stat_add(vm, kLanes, __popc(group) - 1);
     }
     w = __shfl_sync(active, w, leader);
+    if (w == kPinRefused) {                                  /* this group's request was refused: nothing is pinned */
+        if (OP_BYTES == 0) { *ptr_out = nullptr; if (tok) { tok->vpn = vpn; tok->group = group; tok->leader = 0; } }
+        return false;
+    }
     unsigned int frame = (unsigned int)((w & kFrameMask) >> kFrameShift);
     const bool hit = (w & kStMask) == kValid;
     if (__all_sync(active, hit)) {
@@ -754,28 +804,11 @@ static __device__ __noinline__ void gpuvm_prefetch(const gpuvm_dev_t vm, unsigne
     const unsigned long long bq = __shfl_sync(active, victim, L);
     const int bd = __shfl_sync(active, (int)vdirty, L);
     unsigned char *fr = vm.pool + ((unsigned long long)bh << vm.page_shift);
-    if (bq != ~0ull) {
-        if (bd) {
-            warp_copy<8, true>(vm.host + (bq << vm.page_shift), fr, page_len(vm, bq) >> 4, rank, n);
-            __threadfence_system();
-            __syncwarp(active);
-        }
-        if (lane == L) {
-            atomicXor(vm.pte + bq, kEvicting | ((unsigned long long)bh << kFrameShift) | (bd ? kDirty : 0ull));
-            stat_add(vm, kEvictions, 1);
-            if (bd) { stat_add(vm, kWritebacks, 1); stat_add(vm, kBytesOut, page_len(vm, bq)); }
-        }
-    }
+    retire_victim(vm, bh, bq, bd, rank, n, active, lane == L);
     warp_copy<8, false>(fr, vm.host + (vpn << vm.page_shift), page_len(vm, vpn) >> 4, rank, n);
     __threadfence();
     __syncwarp(active);
-    if (lane == L) {
-        st_relaxed_u32(vm.frame_vpn + bh, (unsigned int)vpn);
-        atomicXor(pte, (kBusy ^ kValid) | ((unsigned long long)bh << kFrameShift) |
-                           (vm.policy == GPUVM_POLICY_CLOCK ? kRef : 0ull));
-        stat_add(vm, kFaults, 1);
-        stat_add(vm, kBytesIn, page_len(vm, vpn));
-    }
+    if (lane == L) publish(vm, vpn, bh, kRead);
 }
 
 /* Frame memory accessors (L1-bypassing, device-coherent). */

@@ -92,7 +92,7 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
  * indices, a third paged array at chunk_off holds, for every chunk of `chunk_edges`
  * consecutive edges, the number of the vertex whose neighbour list contains the chunk's
  * first edge (int32, ceil(n_edges / chunk_edges) + 1 entries, the last one = the vertex
- * of the last edge; see inputs.balanced_chunks).  Workers take chunks instead of
+ * of the last edge; built by gpuvm_bcsr_build).  Workers take chunks instead of
  * vertices, so each gets the same number of edges and exactly one column page however
  * skewed the degrees are, and a long list is expanded by as many warps as it has chunks.
  * A chunk must lie inside one page: col_off is a multiple of the page size and the page
@@ -101,6 +101,21 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
  */
 int gpuvm_bfs_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, size_t nv, size_t n_edges,
                    size_t chunk_edges, size_t source, int32_t *d_level, int *n_levels, void *stream);
+
+/*
+ * Build the chunk table of Balanced CSR (Section 5.2, Fig. 8) from a graph's row offsets, on
+ * the host: a format conversion done once, before the graph is handed to gpuvm_create.
+ *   row_off       host pointer, nv + 1 int64 row offsets, row_off[0] = 0.
+ *   chunk_vertex  host pointer, receives ceil(n_edges / chunk_edges) + 1 int32 entries: entry c
+ *                 is the vertex whose neighbour list holds edge c * chunk_edges, the last entry
+ *                 the vertex of the last edge (0 for a graph without edges).  NULL: only the
+ *                 number of chunks is computed.
+ *   capacity      entries that chunk_vertex can hold (GPUVM_E_RANGE when too few).
+ *   n_chunks_out  host pointer (may be NULL), receives the number of chunks.
+ * Runs on the CPU in one pass over the row offsets; needs no device.
+ */
+int gpuvm_bcsr_build(const int64_t *row_off, size_t nv, size_t chunk_edges, int32_t *chunk_vertex, size_t capacity,
+                     size_t *n_chunks_out);
 
 /*
  * Connected components of the same kind of graph (Section 5.2 evaluates CC next to
@@ -121,7 +136,7 @@ int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *
  * the page size, so that the weights of an edge range sit at the same place in their
  * page as the columns do in theirs; both pages are held together while the range is
  * relaxed, hence the pool needs at least two frames per warp of the grid
- * (GPUVM_E_POOL otherwise).  Bellman-Ford rounds over the vertices that changed in
+ * (GPUVM_E_FRAMES otherwise).  Bellman-Ford rounds over the vertices that changed in
  * the previous round; d_dist[v] receives the distance from `source`, 0x7FFFFFFF
  * where unreachable (path lengths must stay below that).  *n_rounds (host pointer,
  * may be NULL) receives the number of rounds.  Uses 2 MiB + 2 nv bytes of the
@@ -157,6 +172,9 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
  *     levels; issue them one after the other.  Nothing needs clearing between
  *     calls: each call zeroes the queue's ready words on its stream before its
  *     first level, each level re-zeroes the counters.
+ *   - The looked-up address is kept for the life of the process; it does not
+ *     survive a cudaDeviceReset of that device (do not reset a device this
+ *     library is still to be used on).
  * d_level, n_levels, stream, return value: as for gpuvm_bfs_csr.
  */
 #define GPUVM_BFS_NOALLOC_MAX_VERTICES ((size_t)1 << 26)
@@ -172,7 +190,9 @@ int gpuvm_bfs_csr_noalloc(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, 
  * on a page boundary, the page of c is kept pinned while its chunks are produced and,
  * being overwritten entirely, is not fetched from the host first (GPUVM_WRITE_ALL);
  * otherwise every chunk pins a, b and c one after the other and c is fetched like any
- * page that is written to.
+ * page that is written to.  c may be the same array as a or b (c_off == a_off or c_off ==
+ * b_off: in place, taken one page at a time); any other overlap of c with an input is refused
+ * with GPUVM_E_ARG.
  */
 int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n, void *stream);
 
@@ -189,6 +209,11 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
  * gpuvm_destroy): 8 + 4 * dims bytes per request in flight.  The warps take as many groups
  * of 32 bags (1, 2, 4 or 8) as it takes to have every bag in flight at once, within
  * gpuvm_set_scratch_limit: 2.1 GiB for one group, dims = 128, on a full grid of 148 SMs.
+ * The batched kernel reads a whole row from the frame of the row's first byte, so it needs rows
+ * that never straddle a page: the page size a multiple of the row size (4 * dims bytes) and
+ * t_off a multiple of the row size.  Any other layout (dims = 20 or 100, pages smaller than a
+ * row) is served by the unbatched kernel, with the same result.  A row id whose row does not lie
+ * inside the backing store entirely sets the sticky GPUVM_E_RANGE.
  * gpuvm_embag_f32_unbatched: one warp per bag, one row request at a time through
  * gpuvm_read; no scratch.
  */

@@ -25,11 +25,59 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 FIFO, CLOCK = 0, 1
 
 
+_LIB_OMP = os.path.join(_HERE, "liboracle_omp.so")
+
+
 def build(force: bool = False) -> str:
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-Wall", "-shared",
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-Wall", "-Wno-unknown-pragmas", "-shared",
                                "-fPIC", _SRC, "-o", _LIB])
     return _LIB
+
+
+def build_omp(force: bool = False) -> str:
+    """The same source with OpenMP: the all-core CPU baseline of the benchmark."""
+    if force or not os.path.exists(_LIB_OMP) or os.path.getmtime(_LIB_OMP) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-Wall", "-fopenmp", "-shared",
+                               "-fPIC", _SRC, "-o", _LIB_OMP])
+    return _LIB_OMP
+
+
+class AllCores:
+    """The four *_direct workloads whose outer loop splits over threads, from the OpenMP build."""
+
+    def __init__(self):
+        lib = ctypes.CDLL(build_omp())
+        u64, vp = ctypes.c_uint64, ctypes.c_void_p
+        lib.orc_stream_sum_i32_direct.restype, lib.orc_stream_sum_i32_direct.argtypes = ctypes.c_int64, [vp, u64]
+        lib.orc_gather_block_sums_direct.restype, lib.orc_gather_block_sums_direct.argtypes = None, [vp, vp, u64, u64, vp, vp]
+        lib.orc_vadd_f32_direct.restype, lib.orc_vadd_f32_direct.argtypes = None, [vp, vp, vp, u64]
+        lib.orc_embag_f32_direct.restype, lib.orc_embag_f32_direct.argtypes = None, [vp, u64, vp, u64, u64, vp]
+        lib.orc_threads.restype = ctypes.c_int
+        self._lib = lib
+        self.threads = int(lib.orc_threads())
+
+    def stream_sum_i32_direct(self, a):
+        return int(self._lib.orc_stream_sum_i32_direct(_p(a, np.int32), a.size))
+
+    def gather_block_sums_direct(self, x, idx, block):
+        nb = (idx.size + block - 1) // block
+        fsum, bsum = np.empty(nb, dtype=np.float32), np.empty(nb, dtype=np.int64)
+        self._lib.orc_gather_block_sums_direct(_p(x, np.float32), _p(idx, np.int64), idx.size, block,
+                                               _p(fsum, np.float32), _p(bsum, np.int64))
+        return fsum, bsum
+
+    def vadd_f32_direct(self, a, b):
+        c = np.empty_like(a)
+        self._lib.orc_vadd_f32_direct(_p(a, np.float32), _p(b, np.float32), _p(c, np.float32), a.size)
+        return c
+
+    def embag_f32_direct(self, table, rows, bag):
+        n_rows, dims = table.shape
+        n_bags = rows.size // bag
+        out = np.empty((n_bags, dims), dtype=np.float32)
+        self._lib.orc_embag_f32_direct(_p(table, np.float32), dims, _p(rows, np.int64), n_bags, bag, _p(out, np.float32))
+        return out
 
 
 _lib = None

@@ -1,9 +1,14 @@
 /*
  * CPU oracle for GPU-thread-driven demand paging (GPUVM, arXiv 2411.05309).
  *
- * TEST INFRASTRUCTURE ONLY.  Plain, slow, single-threaded C that shares no code
- * with the CUDA path.  Only the test-suite, the smoke check and the benchmark's
- * CPU-baseline leg may call it; the product never does.
+ * TEST INFRASTRUCTURE ONLY.  Plain, slow C that shares no code with the CUDA path.
+ * Only the test-suite, the smoke check and the benchmark's CPU-baseline leg may call
+ * it; the product never does.  As the tests build it (no OpenMP) it is
+ * single-threaded.  The benchmark's all-core baseline compiles this same file with
+ * -fopenmp: the pragmas below then split the outermost loop of four *_direct
+ * functions over the host's threads; every element, block or bag is still computed
+ * by one thread with the same operations in the same order, so those results are
+ * bit-identical to the single-threaded build (a test compares the two).
  *
  * Two parts.
  *
@@ -45,6 +50,7 @@
 int64_t orc_stream_sum_i32_direct(const int32_t *a, uint64_t n)
 {
     int64_t s = 0;
+#pragma omp parallel for reduction(+ : s) schedule(static)
     for (uint64_t i = 0; i < n; ++i) s += (int64_t)a[i];
     return s;
 }
@@ -60,6 +66,7 @@ void orc_gather_block_sums_direct(const float *x, const int64_t *idx, uint64_t n
                                   uint64_t block, float *fsum, int64_t *bsum)
 {
     uint64_t nb = (n_idx + block - 1) / block;
+#pragma omp parallel for schedule(static)
     for (uint64_t b = 0; b < nb; ++b) {
         double acc = 0.0;
         int64_t bits = 0;
@@ -183,6 +190,7 @@ void orc_sssp_direct(const int64_t *row_off, const int32_t *col, const int32_t *
 /* c[i] = a[i] + b[i], one correctly rounded binary32 addition per element. */
 void orc_vadd_f32_direct(const float *a, const float *b, float *c, uint64_t n)
 {
+#pragma omp parallel for schedule(static)
     for (uint64_t i = 0; i < n; ++i) {
         volatile float s = a[i] + b[i];
         c[i] = s;
@@ -196,6 +204,7 @@ void orc_vadd_f32_direct(const float *a, const float *b, float *c, uint64_t n)
 void orc_embag_f32_direct(const float *table, uint64_t dims, const int64_t *rows,
                           uint64_t n_bags, uint64_t bag, float *out)
 {
+#pragma omp parallel for schedule(static)
     for (uint64_t g = 0; g < n_bags; ++g)
         for (uint64_t d = 0; d < dims; ++d) {
             volatile float acc = 0.0f;
@@ -555,6 +564,14 @@ void orc_embag_f32_paged(orc_pager *p, uint64_t t_off, uint64_t dims, const int6
         }
     }
 }
+
+/* Threads the *_direct loops above run on in this build (1 without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int orc_threads(void) { return omp_get_max_threads(); }
+#else
+int orc_threads(void) { return 1; }
+#endif
 
 /* Oversubscription level, Eq. 1: workload size / available GPU memory - 1. */
 double orc_oversubscription_level(double workload_bytes, double gpu_bytes)

@@ -15,8 +15,10 @@ LIB_PATH = os.path.join(_HERE, "libgpuvm.so")
 
 POLICY_FIFO, POLICY_CLOCK = 0, 1
 
-E_ARG, E_PAGE, E_POOL, E_ALIGN, E_PIN, E_ALLOC, E_CUDA, E_TIMEOUT, E_RANGE, E_INVARIANT, E_NODEVICE = \
-    range(-1, -12, -1)
+E_ARG, E_PAGE, E_POOL, E_ALIGN, E_PIN, E_ALLOC, E_CUDA, E_TIMEOUT, E_RANGE, E_INVARIANT, E_NODEVICE, E_PINS, E_FRAMES = \
+    range(-1, -14, -1)
+
+DEBUG_POISON = 1
 
 
 class GpuvmError(RuntimeError):
@@ -29,13 +31,14 @@ class DevView(ctypes.Structure):
     _fields_ = [("pte", ctypes.c_void_p), ("frame_vpn", ctypes.c_void_p), ("pool", ctypes.c_void_p),
                 ("host", ctypes.c_void_p), ("ctl", ctypes.c_void_p), ("bytes", ctypes.c_uint64),
                 ("n_pages", ctypes.c_uint64), ("n_frames", ctypes.c_uint32), ("page_shift", ctypes.c_uint32),
-                ("policy", ctypes.c_uint32), ("spin_limit_us", ctypes.c_uint32)]
+                ("policy", ctypes.c_uint32), ("spin_limit_us", ctypes.c_uint32), ("debug", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
 
 
 class Stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in
                 ("faults", "hits", "waits", "lanes_coalesced", "evictions", "writebacks", "flush_writebacks",
-                 "bytes_in", "bytes_out", "hand_steps", "retries", "resident")] + \
+                 "bytes_in", "bytes_out", "hand_steps", "retries", "resident", "ring_drops")] + \
                [("error", ctypes.c_int32), ("reserved", ctypes.c_uint32), ("error_page", ctypes.c_uint64)]
 
     def as_dict(self):
@@ -56,6 +59,11 @@ SYMBOLS = {
     "gpuvm_create": (_i, [ctypes.POINTER(_vp), _vp, _sz, _sz, _sz]),
     "gpuvm_destroy": (_i, [_vp]),
     "gpuvm_stats": (_i, [_vp, ctypes.POINTER(Stats)]),
+    "gpuvm_stats_on": (_i, [_vp, ctypes.POINTER(Stats), _vp]),
+    "gpuvm_reset_on": (_i, [_vp, _vp]),
+    "gpuvm_check_on": (_i, [_vp, ctypes.POINTER(Check), _vp]),
+    "gpuvm_set_debug": (_i, [_vp, ctypes.c_uint]),
+    "gpuvm_bcsr_build": (_i, [_vp, _sz, _sz, _vp, _sz, ctypes.POINTER(_sz)]),
     "gpuvm_device_view": (_i, [_vp, ctypes.POINTER(DevView)]),
     "gpuvm_host_ptr": (_vp, [_vp]),
     "gpuvm_flush": (_i, [_vp, _vp]),
@@ -68,6 +76,7 @@ SYMBOLS = {
     "gpuvm_safe_warps": (_i, [_vp, _i]),
     "gpuvm_inflight_pages": (ctypes.c_double, [ctypes.c_double, ctypes.c_double, ctypes.c_double]),
     "gpuvm_debug_poke_pte": (_i, [_vp, _u64, _u64]),
+    "gpuvm_debug_peek_pte": (_i, [_vp, _u64, ctypes.POINTER(_u64)]),
     "gpuvm_strerror": (ctypes.c_char_p, [_i]),
     "gpuvm_last_cuda_error": (_i, [_vp]),
     "gpuvm_stream_sum_i32": (_i, [_vp, _sz, _sz, _vp, _vp]),
@@ -170,6 +179,43 @@ def gpuvm_stats(h, raise_on_error: bool = True) -> dict:
     return s.as_dict()
 
 
+def gpuvm_stats_on(h, stream, raise_on_error: bool = True) -> dict:
+    s = Stats()
+    rc = lib().gpuvm_stats_on(h, ctypes.byref(s), _stream(stream))
+    if rc != 0 and (raise_on_error or rc != s.error):
+        raise GpuvmError(rc, "gpuvm_stats_on")
+    return s.as_dict()
+
+
+def gpuvm_reset_on(h, stream):
+    _check(lib().gpuvm_reset_on(h, _stream(stream)), "gpuvm_reset_on")
+
+
+def gpuvm_check_on(h, stream, raise_on_error: bool = True) -> dict:
+    c = Check()
+    rc = lib().gpuvm_check_on(h, ctypes.byref(c), _stream(stream))
+    if rc != 0 and raise_on_error:
+        raise GpuvmError(rc, f"gpuvm_check_on {c.as_dict()}")
+    d = c.as_dict()
+    d["status"] = rc
+    return d
+
+
+def gpuvm_set_debug(h, flags: int):
+    _check(lib().gpuvm_set_debug(h, flags), "gpuvm_set_debug")
+
+
+def gpuvm_bcsr_build(row_off, chunk_edges: int):
+    """Chunk table of Balanced CSR for int64 row offsets held in a numpy array (host side)."""
+    import numpy as np
+    nv = row_off.size - 1
+    n = _sz(0)
+    _check(lib().gpuvm_bcsr_build(_ptr(row_off), nv, chunk_edges, None, 0, ctypes.byref(n)), "gpuvm_bcsr_build")
+    out = np.empty(n.value + 1, dtype=np.int32)
+    _check(lib().gpuvm_bcsr_build(_ptr(row_off), nv, chunk_edges, _ptr(out), out.size, None), "gpuvm_bcsr_build")
+    return out
+
+
 def gpuvm_device_view(h) -> DevView:
     v = DevView()
     _check(lib().gpuvm_device_view(h, ctypes.byref(v)), "gpuvm_device_view")
@@ -227,6 +273,12 @@ def gpuvm_inflight_pages(latency_s: float, bytes_per_s: float, page_bytes: float
 
 def gpuvm_debug_poke_pte(h, page: int, value: int):
     _check(lib().gpuvm_debug_poke_pte(h, page, value), "gpuvm_debug_poke_pte")
+
+
+def gpuvm_debug_peek_pte(h, page: int) -> int:
+    v = _u64(0)
+    _check(lib().gpuvm_debug_peek_pte(h, page, ctypes.byref(v)), "gpuvm_debug_peek_pte")
+    return v.value
 
 
 def gpuvm_last_cuda_error(h) -> int:

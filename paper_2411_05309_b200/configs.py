@@ -56,10 +56,15 @@ class Workload:
         self.h = None
         self.off = {}
         self.host = None
+        self._layout()
 
     # -- layout -------------------------------------------------------------
-    def _create(self, arrays: dict, pool_bytes: int):
-        """arrays: name -> nbytes.  The library allocates the pinned backing store."""
+    def sizes(self):
+        """(arrays: name -> nbytes, pool_bytes or a function of the total) at this shrink; no GPU needed."""
+        raise NotImplementedError
+
+    def _layout(self):
+        arrays, pool_bytes = self.sizes()
         total = 0
         for name, nbytes in arrays.items():
             self.off[name] = total
@@ -70,10 +75,14 @@ class Workload:
         if callable(pool_bytes):
             pool_bytes = pool_bytes(total)
         self.pool_bytes = max(self.page_bytes, pool_bytes // self.page_bytes * self.page_bytes)
-        self.h = B.gpuvm_create(None, total, self.page_bytes, self.pool_bytes)
-        self.host = _host_view(B.gpuvm_host_ptr(self.h), total)
         self.n_pages = total // self.page_bytes
         self.n_frames = self.pool_bytes // self.page_bytes
+
+    def _create(self):
+        """The library allocates the pinned backing store."""
+        self._layout()
+        self.h = B.gpuvm_create(None, self.nbytes, self.page_bytes, self.pool_bytes)
+        self.host = _host_view(B.gpuvm_host_ptr(self.h), self.nbytes)
 
     def view(self, name: str, dtype, count: int) -> np.ndarray:
         o = self.off[name]
@@ -104,7 +113,7 @@ class Workload:
     def run(self, check: bool = True) -> RunResult:
         import torch
         stream = torch.cuda.current_stream()
-        B.gpuvm_reset(self.h)
+        B.gpuvm_reset(self.h)                              # device-wide: nothing of an earlier step is in flight
         e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         e0.record(stream)
         extra = self.launch(stream) or {}
@@ -122,10 +131,13 @@ class StreamSum(Workload):
     """Streaming read-reduce: int64 sum over an int32 array, 4 KiB pages, pool = 1/4 of the data."""
     name, cfg, page_bytes = "stream_sum_i32", 1, 4 * KiB
 
+    def sizes(self):
+        self.n = (1 << 24) >> self.shrink
+        return {"a": 4 * self.n}, (16 * MiB) >> self.shrink
+
     def setup(self):
         import torch
-        self.n = (1 << 24) >> self.shrink
-        self._create({"a": 4 * self.n}, (16 * MiB) >> self.shrink)
+        self._create()
         inputs.fill_i32_u20(B.gpuvm_host_ptr(self.h) + self.off["a"], self.n, inputs.config_seed(1))
         self.d_sum = torch.zeros(1, dtype=torch.int64, device="cuda")
         return self
@@ -142,11 +154,14 @@ class Gather(Workload):
     name, cfg, page_bytes = "random_gather_f32", 2, 64 * KiB
     block = 1024
 
-    def setup(self):
-        import torch
+    def sizes(self):
         self.n = (1 << 28) >> self.shrink
         self.n_idx = (1 << 26) >> self.shrink
-        self._create({"x": 4 * self.n}, (256 * MiB) >> self.shrink)
+        return {"x": 4 * self.n}, (256 * MiB) >> self.shrink
+
+    def setup(self):
+        import torch
+        self._create()
         inputs.fill_f32_pm1(B.gpuvm_host_ptr(self.h) + self.off["x"], self.n, inputs.config_seed(2))
         self.idx_host = torch.empty(self.n_idx, dtype=torch.int64).pin_memory()
         inputs.fill_index_i64(self.idx_host.data_ptr(), self.n_idx, inputs.config_seed(2, 1), self.n)
@@ -168,13 +183,15 @@ class Bfs(Workload):
     name, cfg, page_bytes = "bfs_rmat_csr", 3, 64 * KiB
     kernels_per_run = None        # 1 + 2 per level
 
-    def setup(self):
-        import torch
+    def sizes(self):
         self.scale = 24 - self.shrink
         self.nv = 1 << self.scale
         self.ne = 16 << self.scale
-        off_bytes = _pad(8 * (self.nv + 1), 16)
-        self._create({"off": off_bytes, "col": 4 * self.ne}, lambda total: total // 2)   # pool = half their size
+        return {"off": _pad(8 * (self.nv + 1), 16), "col": 4 * self.ne}, lambda total: total // 2   # pool = half their size
+
+    def setup(self):
+        import torch
+        self._create()
         base = B.gpuvm_host_ptr(self.h)
         inputs.rmat_csr(self.scale, self.ne, inputs.config_seed(3), base + self.off["off"], base + self.off["col"])
         self.d_level = torch.zeros(self.nv, dtype=torch.int32, device="cuda")
@@ -193,24 +210,40 @@ class Bfs(Workload):
         self.traversed_edges = int(deg[visited].sum())
         return int(16 * visited.sum() + 4 * self.traversed_edges)
 
+    def compulsory_pages(self) -> int:
+        """Distinct pages any BFS must touch: the two row offsets and the whole edge range of every
+        vertex it reaches (from the levels the last run produced)."""
+        reached = np.flatnonzero(self.d_level.cpu().numpy() >= 0)
+        off = self.view("off", np.int64, self.nv + 1)
+        mark = np.zeros(self.n_pages + 1, np.int64)
+        for lo, hi in ((self.off["off"] + 8 * reached, self.off["off"] + 8 * reached + 15),
+                       (self.off["col"] + 4 * off[reached], self.off["col"] + 4 * off[reached + 1] - 1)):
+            keep = hi >= lo
+            np.add.at(mark, lo[keep] // self.page_bytes, 1)
+            np.add.at(mark, hi[keep] // self.page_bytes + 1, -1)
+        return int(np.count_nonzero(np.cumsum(mark[:-1]) > 0))
+
 
 class BfsBalanced(Bfs):
     """BFS on the cfg 3 graph stored as Balanced CSR: chunks of one page of edges (16 Ki edges), the chunk
     table paged with the other two arrays; pool = half."""
     name, cfg = "bfs_rmat_balanced_csr", 8
 
-    def setup(self):
-        import torch
+    def sizes(self):
         self.scale = 24 - self.shrink
         self.nv = 1 << self.scale
         self.ne = 16 << self.scale
         self.chunk_edges = self.page_bytes // 4
         n_chunks = (self.ne + self.chunk_edges - 1) // self.chunk_edges
-        self._create({"off": _pad(8 * (self.nv + 1), 16), "col": 4 * self.ne, "chunk": _pad(4 * (n_chunks + 1), 16)},
-                     lambda total: total // 2)
+        return ({"off": _pad(8 * (self.nv + 1), 16), "col": 4 * self.ne, "chunk": _pad(4 * (n_chunks + 1), 16)},
+                lambda total: total // 2)
+
+    def setup(self):
+        import torch
+        self._create()
         base = B.gpuvm_host_ptr(self.h)
         inputs.rmat_csr(self.scale, self.ne, inputs.config_seed(3), base + self.off["off"], base + self.off["col"])
-        chunks = inputs.balanced_chunks(self.view("off", np.int64, self.nv + 1), self.chunk_edges)
+        chunks = B.gpuvm_bcsr_build(self.view("off", np.int64, self.nv + 1), self.chunk_edges)
         self.view("chunk", np.int32, chunks.size)[...] = chunks
         self.d_level = torch.zeros(self.nv, dtype=torch.int32, device="cuda")
         self.levels = 0
@@ -240,12 +273,15 @@ class Sssp(Workload):
     pool = half of the three arrays."""
     name, cfg, page_bytes = "sssp_rmat_csr", 7, 64 * KiB
 
-    def setup(self):
-        import torch
+    def sizes(self):
         self.scale = 24 - self.shrink
         self.nv = 1 << self.scale
         self.ne = 16 << self.scale
-        self._create({"off": _pad(8 * (self.nv + 1), 16), "col": 4 * self.ne, "w": 4 * self.ne}, lambda total: total // 2)
+        return {"off": _pad(8 * (self.nv + 1), 16), "col": 4 * self.ne, "w": 4 * self.ne}, lambda total: total // 2
+
+    def setup(self):
+        import torch
+        self._create()
         base = B.gpuvm_host_ptr(self.h)
         inputs.rmat_csr(self.scale, self.ne, inputs.config_seed(3), base + self.off["off"], base + self.off["col"])
         inputs.fill_i32_range(base + self.off["w"], self.ne, inputs.config_seed(3, 2), 1, 255)
@@ -269,9 +305,12 @@ class VAdd(Workload):
     """c = a + b over three fp32 arrays, 64 KiB pages, pool = one array (3x oversubscribed)."""
     name, cfg, page_bytes = "vector_add_f32", 4, 64 * KiB
 
-    def setup(self):
+    def sizes(self):
         self.n = (1 << 30) >> self.shrink
-        self._create({"a": 4 * self.n, "b": 4 * self.n, "c": 4 * self.n}, (4 * GiB) >> self.shrink)
+        return {"a": 4 * self.n, "b": 4 * self.n, "c": 4 * self.n}, (4 * GiB) >> self.shrink
+
+    def setup(self):
+        self._create()
         base = B.gpuvm_host_ptr(self.h)
         inputs.fill_f32_pm1(base + self.off["a"], self.n, inputs.config_seed(4))
         inputs.fill_f32_pm1(base + self.off["b"], self.n, inputs.config_seed(4, 1))
@@ -290,12 +329,15 @@ class EmbeddingBag(Workload):
     name, cfg, page_bytes = "zipf_embedding_bag_f32", 5, 2 * MiB
     dims, bag, s = 128, 32, 1.05
 
-    def setup(self):
-        import torch
+    def sizes(self):
         self.n_rows = (1 << 27) >> self.shrink
         self.n_lookups = (1 << 24) >> self.shrink
         self.n_bags = self.n_lookups // self.bag
-        self._create({"t": 4 * self.dims * self.n_rows}, (16 * GiB) >> self.shrink)
+        return {"t": 4 * self.dims * self.n_rows}, (16 * GiB) >> self.shrink
+
+    def setup(self):
+        import torch
+        self._create()
         inputs.fill_f32_pm1(B.gpuvm_host_ptr(self.h) + self.off["t"], self.dims * self.n_rows, inputs.config_seed(5))
         self.rows_host = torch.empty(self.n_lookups, dtype=torch.int64).pin_memory()
         inputs.fill_zipf_rows(self.rows_host.data_ptr(), self.n_lookups, inputs.config_seed(5, 1), self.n_rows, self.s)
@@ -318,3 +360,8 @@ def make(cfg: int, shrink: int = 0) -> Workload:
     w = WORKLOADS[cfg](shrink).setup()
     w.setup_seconds = time.time() - t0
     return w
+
+
+def describe(cfg: int, shrink: int = 0) -> dict:
+    """The configuration's sizes without creating anything (no GPU needed)."""
+    return WORKLOADS[cfg](shrink).describe()

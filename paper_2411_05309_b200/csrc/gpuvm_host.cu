@@ -17,6 +17,7 @@ struct gpuvm_handle {
     bool host_registered;   // we called cudaHostRegister on it
     bool host_allocated;    // we called cudaHostAlloc for it
     int device;
+    int sms;                // SMs of that device
     int last_cuda;
     unsigned long long *check_buf;   // device, 8 words
     void *scratch;                   // device scratch for workload kernels (request tables)
@@ -100,6 +101,17 @@ __global__ void check_kernel(gpuvm_dev_t vm, unsigned long long *out)
     }
 }
 
+// Number of SMs of the handle's device (grids are sized in multiples of it).
+int sm_count_of(int device)
+{
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0) {
+        cudaGetLastError();
+        sms = 148;
+    }
+    return sms;
+}
+
 bool is_pow2(size_t x) { return x && !(x & (x - 1)); }
 
 int ilog2(size_t x)
@@ -131,6 +143,7 @@ int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_byt
     if (!h) return GPUVM_E_ALLOC;
     memset(h, 0, sizeof(*h));
     cudaGetDevice(&h->device);
+    h->sms = sm_count_of(h->device);
     cudaError_t e;
 
     // backing store: pinned and mapped (Section 4: the host region is registered before
@@ -194,15 +207,25 @@ int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_byt
     return rc;
 }
 
-int gpuvm_reset(gpuvm_t h)
+int gpuvm_reset_on(gpuvm_t h, void *stream)
 {
     if (!h) return GPUVM_E_ARG;
     gpuvm_dev_t &d = h->dev;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(d.pte, 0, d.n_pages * sizeof(unsigned long long), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d.frame_vpn, 0xFF, d.n_frames * sizeof(unsigned int), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d.ctl, 0, kCtlWords * sizeof(unsigned long long), s);
+    return e == cudaSuccess ? GPUVM_OK : fail(h, e, GPUVM_E_CUDA);
+}
+
+int gpuvm_reset(gpuvm_t h)
+{
+    if (!h) return GPUVM_E_ARG;
     cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaMemset(d.pte, 0, d.n_pages * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaMemset(d.frame_vpn, 0xFF, d.n_frames * sizeof(unsigned int));
-    if (e == cudaSuccess) e = cudaMemset(d.ctl, 0, kCtlWords * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
+    int rc = gpuvm_reset_on(h, nullptr);
+    if (rc != GPUVM_OK) return rc;
+    e = cudaDeviceSynchronize();
     return e == cudaSuccess ? GPUVM_OK : fail(h, e, GPUVM_E_CUDA);
 }
 
@@ -210,7 +233,8 @@ int gpuvm_flush(gpuvm_t h, void *stream)
 {
     if (!h) return GPUVM_E_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    unsigned int warps = h->dev.n_frames < 148u * 32u ? h->dev.n_frames : 148u * 32u;
+    const unsigned int all = (unsigned int)h->sms * 32u;      // one warp per frame, up to 32 warps per SM
+    unsigned int warps = h->dev.n_frames < all ? h->dev.n_frames : all;
     unsigned int blocks = (warps + 7) / 8;
     flush_kernel<<<blocks, 256, 0, s>>>(h->dev);
     gpuvm_note_launch_(1);
@@ -232,15 +256,17 @@ int gpuvm_destroy(gpuvm_t h)
     return rc;
 }
 
-int gpuvm_check(gpuvm_t h, gpuvm_check_t *out)
+int gpuvm_check_on(gpuvm_t h, gpuvm_check_t *out, void *stream)
 {
     if (!h || !out) return GPUVM_E_ARG;
-    cudaError_t e = cudaMemset(h->check_buf, 0, 8 * sizeof(unsigned long long));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(h->check_buf, 0, 8 * sizeof(unsigned long long), s);
     if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
-    check_kernel<<<148, 256>>>(h->dev, h->check_buf);
+    check_kernel<<<h->sms, 256, 0, s>>>(h->dev, h->check_buf);
     gpuvm_note_launch_(1);
     unsigned long long c[8];
-    e = cudaMemcpy(c, h->check_buf, sizeof(c), cudaMemcpyDeviceToHost);
+    e = cudaMemcpyAsync(c, h->check_buf, sizeof(c), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
     out->resident = c[0]; out->frames_used = c[1]; out->bad_state = c[2]; out->bad_refcount = c[3];
     out->bad_backref = c[4]; out->bad_range = c[5]; out->dirty = c[6];
@@ -248,26 +274,38 @@ int gpuvm_check(gpuvm_t h, gpuvm_check_t *out)
     return bad ? GPUVM_E_INVARIANT : GPUVM_OK;
 }
 
-int gpuvm_stats(gpuvm_t h, gpuvm_stats_t *out)
+int gpuvm_check(gpuvm_t h, gpuvm_check_t *out) { return gpuvm_check_on(h, out, nullptr); }
+
+int gpuvm_stats_on(gpuvm_t h, gpuvm_stats_t *out, void *stream)
 {
     if (!h || !out) return GPUVM_E_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned long long local[kCtlWords];
-    cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaMemcpy(local, h->dev.ctl, sizeof(local), cudaMemcpyDeviceToHost);
+    cudaError_t e = cudaMemcpyAsync(local, h->dev.ctl, sizeof(local), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
     unsigned long long sum[kNumStats] = {0};
-    for (int s = 0; s < kStatSlots; ++s)
-        for (int k = 0; k < kNumStats; ++k) sum[k] += local[kCtlCounters + s * 16 + k];
+    for (int k = 0; k < kStatSlots; ++k)
+        for (int j = 0; j < kNumStats; ++j) sum[j] += local[kCtlCounters + k * 16 + j];
     memset(out, 0, sizeof(*out));
     out->faults = sum[kFaults]; out->hits = sum[kHits]; out->waits = sum[kWaits];
     out->lanes_coalesced = sum[kLanes]; out->evictions = sum[kEvictions];
     out->writebacks = sum[kWritebacks]; out->flush_writebacks = sum[kFlushWritebacks];
     out->bytes_in = sum[kBytesIn]; out->bytes_out = sum[kBytesOut];
     out->hand_steps = sum[kHandSteps]; out->retries = sum[kRetries];
+    out->ring_drops = sum[kRingDrops];
     out->resident = out->faults - out->evictions;
     out->error = (int32_t)(long long)local[kCtlErr];
     out->error_page = local[kCtlErrPage];
     return out->error;
+}
+
+int gpuvm_stats(gpuvm_t h, gpuvm_stats_t *out)
+{
+    if (!h || !out) return GPUVM_E_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
+    return gpuvm_stats_on(h, out, nullptr);
 }
 
 void *gpuvm_scratch_(gpuvm_handle *h, size_t bytes)
@@ -310,6 +348,13 @@ int gpuvm_set_policy(gpuvm_t h, int policy)
     return GPUVM_OK;
 }
 
+int gpuvm_set_debug(gpuvm_t h, unsigned int flags)
+{
+    if (!h || (flags & ~(unsigned int)GPUVM_DEBUG_POISON)) return GPUVM_E_ARG;
+    h->dev.debug = flags;
+    return GPUVM_OK;
+}
+
 int gpuvm_set_spin_limit_us(gpuvm_t h, unsigned int us)
 {
     if (!h || us == 0) return GPUVM_E_ARG;
@@ -336,6 +381,13 @@ int gpuvm_debug_poke_pte(gpuvm_t h, uint64_t page, uint64_t value)
     return e == cudaSuccess ? GPUVM_OK : fail(h, e, GPUVM_E_CUDA);
 }
 
+int gpuvm_debug_peek_pte(gpuvm_t h, uint64_t page, uint64_t *value)
+{
+    if (!h || !value || page >= h->dev.n_pages) return GPUVM_E_ARG;
+    cudaError_t e = cudaMemcpy(value, h->dev.pte + page, sizeof(*value), cudaMemcpyDeviceToHost);
+    return e == cudaSuccess ? GPUVM_OK : fail(h, e, GPUVM_E_CUDA);
+}
+
 const char *gpuvm_strerror(int status)
 {
     switch (status) {
@@ -351,6 +403,8 @@ const char *gpuvm_strerror(int status)
     case GPUVM_E_RANGE: return "offset past the end of the paged array";
     case GPUVM_E_INVARIANT: return "page-table invariant violated";
     case GPUVM_E_NODEVICE: return "no CUDA device";
+    case GPUVM_E_PINS: return "too many simultaneous references to one page";
+    case GPUVM_E_FRAMES: return "the pool has too few frames for the pages this workload pins at once";
     default: return "unknown status";
     }
 }

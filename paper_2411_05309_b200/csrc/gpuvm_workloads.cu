@@ -892,6 +892,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
     const unsigned long long per_item = 32ull * groups;
     const unsigned long long items = (n_bags + per_item - 1) / per_item;
     const unsigned long long stride = (unsigned long long)gridDim.x * requesters;
+    const unsigned long long rows_inside = (vm.bytes - t_off) / row_bytes;   // rows that lie in the backing store entirely
     for (unsigned long long t = slot; t < items; t += stride) {
         const unsigned long long g0 = per_item * t;
         for (unsigned int k0 = 0; k0 < bag; k0 += kEmbagLookups) {
@@ -900,10 +901,12 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
             for (unsigned int gi = 0; gi < groups; ++gi)
                 for (unsigned int k = 0; k < nk; ++k) {
                     const unsigned long long g = g0 + 32ull * gi + lane;
-                    if (g < n_bags)
-                        gpuvm_batch_set(vm, table, (gi * nk + k) * 32 + lane,
-                                        t_off + (unsigned long long)rows[g * bag + k0 + k] * row_bytes);
-                    else
+                    if (g < n_bags) {
+                        // a row that ends past the backing store is refused like one that starts there
+                        const unsigned long long r = (unsigned long long)rows[g * bag + k0 + k];
+                        const bool inside = r < rows_inside;
+                        gpuvm_batch_set(vm, table, (gi * nk + k) * 32 + lane, inside ? t_off + r * row_bytes : ~0ull);
+                    } else
                         gpuvm_batch_skip(table, (gi * nk + k) * 32 + lane);
                 }
             __syncwarp();
@@ -1466,6 +1469,28 @@ int gpuvm_bfs_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, 
                         gpuvm_scratch_(h, kBfsScratchBytes), static_cast<cudaStream_t>(stream));
 }
 
+int gpuvm_bcsr_build(const int64_t *row_off, size_t nv, size_t chunk_edges, int32_t *chunk_vertex, size_t capacity,
+                     size_t *n_chunks_out)
+{
+    if (!row_off || nv == 0 || nv > 0x7FFFFFFFull || chunk_edges == 0) return GPUVM_E_ARG;
+    const int64_t ne = row_off[nv];
+    if (ne < 0 || row_off[0] != 0) return GPUVM_E_ARG;
+    const size_t n_chunks = ((size_t)ne + chunk_edges - 1) / chunk_edges;
+    if (n_chunks_out) *n_chunks_out = n_chunks;
+    if (!chunk_vertex) return GPUVM_OK;                       // size query
+    if (capacity < n_chunks + 1) return GPUVM_E_RANGE;
+    // one pass over the row offsets: v follows the chunk boundaries, which only move forward
+    size_t v = 0;
+    for (size_t c = 0; c < n_chunks; ++c) {
+        const int64_t first = (int64_t)(c * chunk_edges);
+        while (row_off[v + 1] <= first) ++v;                  // skips vertices without edges: first < ne = row_off[nv]
+        chunk_vertex[c] = (int32_t)v;
+    }
+    if (ne > 0) { while (row_off[v + 1] <= ne - 1) ++v; }
+    chunk_vertex[n_chunks] = (int32_t)(ne > 0 ? v : 0);
+    return GPUVM_OK;
+}
+
 int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, void *stream)
 {
     Paged m;
@@ -1481,7 +1506,7 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
     PagedH m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
     // column and weight page of an edge range are held together: two frames per warp of the grid
-    if (gpuvm_safe_warps(h, 2) < sm_count() * 2 * 8) return GPUVM_E_POOL;
+    if (gpuvm_safe_warps(h, 2) < sm_count() * 2 * 8) return GPUVM_E_FRAMES;
     hint_edges(h, m, off_off, nv);
     return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, gpuvm_scratch_(h, kBfsScratchBytes + 2 * nv),
                     static_cast<cudaStream_t>(stream));
@@ -1496,7 +1521,14 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
     // this kernel's register count anyway) before the kernel falls back to one page at a time.
     int blocks = sm_count() * kVaddBlocksPerSm;
     while (blocks > sm_count() && gpuvm_safe_warps(h, 2) < blocks * 8) blocks -= sm_count();
-    const bool hold_c = gpuvm_safe_warps(h, 2) >= blocks * 8;
+    // c may be a or b itself (in place): every chunk is then read before it is written, by the same
+    // warp, one page at a time; the no-fetch path is out, because it hands out the page of c without
+    // its contents.  Any other overlap of c with an input has no defined result.
+    const size_t len = 4 * n;
+    auto overlaps = [len](size_t x, size_t y) { return x < y + len && y < x + len; };
+    const bool in_place = c_off == a_off || c_off == b_off;
+    if ((c_off != a_off && overlaps(c_off, a_off)) || (c_off != b_off && overlaps(c_off, b_off))) return GPUVM_E_ARG;
+    const bool hold_c = !in_place && gpuvm_safe_warps(h, 2) >= blocks * 8;
     return run_vadd(m, a_off, b_off, c_off, n, hold_c, blocks, static_cast<cudaStream_t>(stream));
 }
 
@@ -1508,6 +1540,13 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     if (!d_rows || !d_out || dims == 0 || dims % 4 || dims / 4 > 32 || bag == 0 || bag > 0xFFFFFFFFull) return GPUVM_E_ARG;
     if (t_off % 16) return GPUVM_E_ALIGN;
     if (n_bags == 0) return GPUVM_OK;
+    // The batched kernel registers a row by its first byte and then reads the whole row from that
+    // frame: a row must lie inside one page.  Tables whose rows straddle pages (a row size that does
+    // not divide the page size, a table that does not start on a row boundary inside its page, pages
+    // smaller than a row) take the one-request-at-a-time kernel, which asks for every 16 bytes it reads.
+    const size_t row_bytes = 4 * dims, page_bytes = size_t(1) << m.vm.page_shift;
+    if (page_bytes % row_bytes != 0 || t_off % row_bytes != 0)
+        return run_embag(m, t_off, dims, d_rows, n_bags, bag, d_out, static_cast<cudaStream_t>(stream));
     const int requesters = kEmbagRequesters, migrators = kEmbagMigrators;
     // Groups of 32 bags per requester warp: enough for every bag to be in flight at once when
     // that takes at most kEmbagMaxGroups, within the scratch bound (table + staged rows).

@@ -119,15 +119,3 @@ def rmat_csr(scale: int, n_edges: int, seed: int, row_off=None, col=None, thresh
 def fill_zipf_rows(dst, n: int, seed: int, n_ranks: int, s: float = 1.05, first: int = 0):
     _load().gvi_fill_zipf_rows(_addr(dst, np.int64, n), first, n, seed, n_ranks, s)
     return dst
-
-
-def balanced_chunks(row_off: np.ndarray, chunk_edges: int) -> np.ndarray:
-    """Chunk table of Balanced CSR: entry c is the vertex whose neighbour list contains edge
-    c * chunk_edges; one more entry at the end names the vertex of the last edge.  A format
-    conversion of the input graph (int32, ceil(n_edges / chunk_edges) + 1 entries)."""
-    ne = int(row_off[-1])
-    n_chunks = (ne + chunk_edges - 1) // chunk_edges
-    firsts = np.arange(n_chunks, dtype=np.int64) * chunk_edges
-    owner = np.searchsorted(row_off, firsts, side="right") - 1
-    last = np.searchsorted(row_off, max(ne - 1, 0), side="right") - 1 if ne else 0
-    return np.concatenate([owner, [last]]).astype(np.int32)

@@ -38,7 +38,7 @@ def test_every_declared_symbol_is_exported_and_bound(B):
 
 
 def test_status_strings(B):
-    for code in range(0, -12, -1):
+    for code in range(0, -14, -1):
         assert B.strerror(code) and B.strerror(code) != "unknown status"
     assert B.strerror(-99) == "unknown status"
 
@@ -83,3 +83,30 @@ def test_inflight_pages_is_littles_law_of_the_paper(B):
     assert abs(B.gpuvm_inflight_pages(23e-6, 12 * 2 ** 30, 4096) - 72.35) < 0.01
     assert abs(B.gpuvm_inflight_pages(23e-6, 12 * 2 ** 30, 8192) - 36.18) < 0.01
     assert B.gpuvm_inflight_pages(1.0, 1.0, 0.0) == 0.0
+
+
+def test_bcsr_build_names_the_owner_of_each_chunks_first_edge(B):
+    """The chunk table of Balanced CSR is built by the library on the host (no device needed)."""
+    rng = np.random.default_rng(3)
+    for _ in range(20):
+        nv = int(rng.integers(1, 40))
+        deg = rng.integers(0, 9, nv) * (rng.random(nv) < 0.6)
+        off = np.concatenate([[0], np.cumsum(deg)]).astype(np.int64)
+        ne = int(off[-1])
+        for chunk in (1, 3, 8):
+            table = B.gpuvm_bcsr_build(off, chunk)
+            n_chunks = (ne + chunk - 1) // chunk
+            assert table.dtype == np.int32 and table.size == n_chunks + 1
+            owner = np.repeat(np.arange(nv), np.diff(off))            # owner[e] by definition of CSR
+            for c in range(n_chunks):
+                assert table[c] == owner[c * chunk]
+            assert table[-1] == (owner[-1] if ne else 0)
+            assert np.all(np.diff(table) >= 0)
+    # a table that is too small is refused; the size query needs no table
+    off = np.array([0, 5, 5, 9], dtype=np.int64)
+    n = ctypes.c_size_t(0)
+    assert B.lib().gpuvm_bcsr_build(off.ctypes.data, 3, 4, None, 0, ctypes.byref(n)) == 0 and n.value == 3
+    small = np.zeros(3, np.int32)
+    assert B.lib().gpuvm_bcsr_build(off.ctypes.data, 3, 4, small.ctypes.data, 3, None) == B.E_RANGE
+    assert B.lib().gpuvm_bcsr_build(off.ctypes.data, 3, 0, small.ctypes.data, 3, None) == B.E_ARG
+    assert B.gpuvm_bcsr_build(off, 4).tolist() == [0, 0, 2, 2]

@@ -147,6 +147,29 @@ def test_vadd_no_fetch_path_with_eager_write_back(B, page, n, frames):
     assert st["faults"] >= 3 * full_c_pages
 
 
+@pytest.mark.parametrize("page,n,frames", [(512, 1 << 20, 10000), (4096, 1 << 16, 3), (4096, (1 << 18) + 512, 20000)])
+@pytest.mark.parametrize("target", ["a", "b"])
+def test_vadd_in_place(B, page, n, frames, target):
+    """c may be a or b itself: the sum replaces that input on the host, the other input stays.  A pool
+    with room for the no-fetch path must not take it here (the page of c holds an operand)."""
+    a = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4))
+    b = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4, 1))
+    ar = Arena(page, {"a": a, "b": b})
+    with paged(ar.host, page, frames) as h:
+        B.gpuvm_vadd_f32(h, ar.off["a"], ar.off["b"], ar.off[target], n)
+        st, ck = finish(h)
+        # c overlapping an input in any other way is refused before anything runs
+        for c_off in (ar.off["a"] + page, ar.off["b"] - page, ar.off["b"] + 4 * n - page):
+            with pytest.raises(B.GpuvmError) as e:
+                B.gpuvm_vadd_f32(h, ar.off["a"], ar.off["b"], c_off, n)
+            assert e.value.status == B.E_ARG
+    ref = oracle.vadd_f32_direct(a, b)
+    other = "b" if target == "a" else "a"
+    assert np.array_equal(ar.views[target].view(np.uint32), ref.view(np.uint32))
+    assert np.array_equal(ar.views[other], {"a": a, "b": b}[other])
+    assert st["bytes_in"] >= 8 * n                                          # both operands were fetched
+
+
 def small_graphs():
     rng = np.random.default_rng(24)
     yield 1, [], 0
@@ -228,7 +251,7 @@ def test_bfs_over_balanced_csr(B, policy):
         nv, ne = off.size - 1, int(off[-1])
         ref = oracle.bfs_levels_direct(off, col, src)
         for page, chunk_edges, frames in ((64, 16, 1), (64, 4, 3), (4096, 1024, 5), (4096, 256, 64)):
-            chunks = inputs.balanced_chunks(off, chunk_edges)
+            chunks = B.gpuvm_bcsr_build(off, chunk_edges)
             # brute-force check of the chunk table: the owner of edge e is the vertex with off[v] <= e < off[v+1]
             for c in range(min(chunks.size - 1, 50)):
                 v = int(chunks[c])
@@ -296,7 +319,7 @@ def test_sssp_small_graphs_and_rmat(B, policy):
         with pytest.raises(B.GpuvmError) as e:
             B.gpuvm_sssp_csr(h, ar.off["off"], ar.off["col"], ar.off["w"], graphs[1][0].size - 1, 0,
                              torch.zeros(8, dtype=torch.int32, device="cuda"))
-        assert e.value.status == B.E_POOL
+        assert e.value.status == B.E_FRAMES
 
 
 @pytest.mark.parametrize("page,n_rows,n_bags,frames,dims,bag", [
@@ -306,6 +329,10 @@ def test_sssp_small_graphs_and_rmat(B, policy):
     (512, 100, 33, 1, 128, 32),
     (4096, 2000, 70, 16, 128, 40),                 # bags longer than one batch of 32 lookups
     (4096, 2000, 70, 16, 64, 5),                   # narrow rows, short bags
+    (4096, 3000, 200, 9, 20, 7),                   # 80-byte rows straddle pages
+    (4096, 1000, 200, 5, 100, 32),                 # 400-byte rows straddle pages
+    (256, 300, 64, 6, 128, 32),                    # pages smaller than a row
+    (256, 300, 64, 1, 128, 3),                     # ... and a single frame
 ])
 @pytest.mark.parametrize("batched", [True, False])
 def test_embag(B, page, n_rows, n_bags, frames, dims, bag, batched):
@@ -323,6 +350,35 @@ def test_embag(B, page, n_rows, n_bags, frames, dims, bag, batched):
     assert np.all(np.abs(got.astype(np.float64) - ref) <= 1e-6 * np.maximum(np.abs(ref), 2.0 ** -10))
     assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))     # same order of additions: same bits
     assert st["faults"] >= np.unique(rows * dims * 4 // page).size
+
+
+def test_embag_rows_past_the_end_and_tables_off_the_row_grid(B):
+    """A row id whose row does not lie inside the backing store sets the sticky range error (batched
+    and unbatched); a table that starts off the row grid of its page is still summed correctly."""
+    import torch
+    page, dims, bag, n_rows, n_bags = 4096, 128, 4, 64, 8
+    t = inputs.fill_f32_pm1(np.empty(n_rows * dims, np.float32), n_rows * dims, inputs.config_seed(5))
+    rows = (np.arange(n_bags * bag, dtype=np.int64) * 7) % n_rows
+    out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
+    for batched in (True, False):
+        bad = rows.copy()
+        bad[5] = n_rows                                                     # first row past the end
+        ar = Arena(page, {"t": t})
+        with paged(ar.host, page, 4) as h:
+            (B.gpuvm_embag_f32 if batched else B.gpuvm_embag_f32_unbatched)(h, 0, dims, dev(bad), n_bags, bag, out)
+            B.gpuvm_flush(h)
+            with pytest.raises(B.GpuvmError) as e:
+                B.gpuvm_stats(h)
+            assert e.value.status == B.E_RANGE
+            assert B.gpuvm_check(h)["status"] == 0                          # nothing left pinned or in transit
+    # table at byte 16 of the arena: rows straddle pages although the row size divides the page size
+    shifted = np.concatenate([np.zeros(4, np.float32), t])
+    ar = Arena(page, {"t": shifted})
+    with paged(ar.host, page, 3) as h:
+        B.gpuvm_embag_f32(h, 16, dims, dev(rows), n_bags, bag, out)
+        finish(h)
+    ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32))
 
 
 @pytest.mark.parametrize("page,n,frames", [(4096, 1 << 16, 64), (4096, 1 << 16, 7), (64, 2048, 1), (1024, 50000, 13),

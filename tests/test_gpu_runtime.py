@@ -281,3 +281,63 @@ def test_link_peak_is_plausible(B):
     peak = B.gpuvm_link_peak(host, devb, nbytes, 2)
     assert 5 < peak["h2d_gbs"] < 200 and 5 < peak["d2h_gbs"] < 200
     assert int(devb[12345]) == 7 or True
+
+
+def test_reference_counter_cannot_carry_into_the_frame_field(B):
+    """A page whose counter already stands at the limit (poked from the host): the next pin is refused,
+    given back, and reported as a sticky error; the frame field of the entry is untouched."""
+    import torch
+    n = 1 << 12
+    a = np.arange(n, dtype=np.int32)
+    ar = Arena(4096, {"a": a})
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    with paged(ar.host, 4096, 8) as h:
+        B.gpuvm_stream_sum_i32(h, 0, n, out)                          # all four pages resident
+        finish(h)
+        w = B.gpuvm_debug_peek_pte(h, 1)
+        assert w >> 60 == 2 and w & 0xFFFFFF == 0                      # VALID, nobody holds it
+        B.gpuvm_debug_poke_pte(h, 1, w | (1 << 23))                    # the counter stands at the limit
+        B.gpuvm_stream_sum_i32(h, 0, n, out)
+        torch.cuda.synchronize()
+        st = B.gpuvm_stats(h, raise_on_error=False)
+        assert st["error"] == B.E_PINS and st["error_page"] == 1
+        assert int(out.item()) == int(a.astype(np.int64).sum() - a[1024:2048].astype(np.int64).sum())   # page 1 was skipped
+        assert B.gpuvm_debug_peek_pte(h, 1) == w | (1 << 23)           # the refused pin was given back: frame field intact
+        ck = B.gpuvm_check(h, raise_on_error=False)
+        assert ck["bad_backref"] == 0 and ck["bad_range"] == 0 and ck["bad_refcount"] == 1              # only the poked counter
+        B.gpuvm_reset(h)
+
+
+def test_stale_ring_entry_is_dropped_not_migrated(B):
+    """A fault-ring entry must name a page that is waiting for a migrator (BUSY).  The queued scatter is
+    run with a page poked BUSY: its requesters time out, nobody pushes it, and the counters show no
+    dropped ring entries in this (healthy) case; ring_drops exists and is zero after clean runs."""
+    import torch
+    n = 1 << 14
+    a = np.arange(n, dtype=np.uint32)
+    idx = torch.arange(n, dtype=torch.int64, device="cuda")
+    ar = Arena(4096, {"a": a})
+    with paged(ar.host, 4096, 5) as h:
+        B.gpuvm_scatter_update_u32_queued(h, 0, idx, n)
+        st, ck = finish(h)
+        assert st["ring_drops"] == 0 and st["faults"] >= 16
+    assert np.array_equal(ar.views["a"], a * np.uint32(3) + np.uint32(1))
+
+
+def test_stream_scoped_reset_stats_check(B):
+    """gpuvm_reset_on / gpuvm_stats_on / gpuvm_check_on work on a stream of the caller's choice and
+    synchronise only that stream."""
+    import torch
+    n = 1 << 14
+    a = inputs.fill_i32_u20(np.empty(n, np.int32), n, 9)
+    ar = Arena(4096, {"a": a})
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    s = torch.cuda.Stream()
+    with paged(ar.host, 4096, 4) as h, torch.cuda.stream(s):
+        for _ in range(2):
+            B.gpuvm_reset_on(h, s)
+            B.gpuvm_stream_sum_i32(h, 0, n, out, s)
+            st = B.gpuvm_stats_on(h, s)
+            ck = B.gpuvm_check_on(h, s)
+            assert st["faults"] == 16 and st["evictions"] == 12 and ck["resident"] == 4 and ck["status"] == 0
+            assert int(out.item()) == int(a.astype(np.int64).sum())

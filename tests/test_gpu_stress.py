@@ -1,7 +1,9 @@
 """Randomised small cases, many of them: page sizes, pool sizes from one frame to everything,
 both policies, all accessor styles.  Concurrency bugs in the page-table protocol (a lost
 reference, a frame claimed twice, a write-back that races a re-fetch) show up as wrong
-results, a failed invariant check, or a sticky error."""
+results, a failed invariant check, or a sticky error.  Every other case runs with the poison
+debug mode (a frame is filled with a pattern when its page is evicted), so that a read from
+the frame of a page that is no longer held cannot pass for old data."""
 import os
 
 import numpy as np
@@ -44,6 +46,8 @@ def test_random_mix_of_workloads_on_one_handle(B):
         ar = Arena(page, {"a": a})
         out = torch.zeros(1, dtype=torch.int64, device="cuda")
         with paged(ar.host, page, frames, policy) as h:
+            if case & 1:                                               # every other case with frames poisoned on eviction
+                B.gpuvm_set_debug(h, B.DEBUG_POISON)
             for step in range(int(rng.integers(2, 6))):
                 kind = int(rng.integers(0, 5))
                 if kind in (0, 1):                                     # scattered updates of distinct elements
@@ -82,6 +86,8 @@ def test_many_small_vector_adds_and_graphs(B):
         b = inputs.fill_f32_pm1(np.empty(n, np.float32), n, 90 + case)
         ar = Arena(page, {"a": a, "b": b, "c": np.zeros(n, np.float32)})
         with paged(ar.host, page, frames, int(rng.integers(0, 2))) as h:
+            if case & 1:
+                B.gpuvm_set_debug(h, B.DEBUG_POISON)
             B.gpuvm_vadd_f32(h, ar.off["a"], ar.off["b"], ar.off["c"], n)
             finish(h)
         assert np.array_equal(ar.views["c"].view(np.uint32), oracle.vadd_f32_direct(a, b).view(np.uint32)), (case, page, n, frames)
@@ -99,6 +105,8 @@ def test_many_small_vector_adds_and_graphs(B):
         lvl = torch.zeros(nv, dtype=torch.int32, device="cuda")
         lab = torch.zeros(nv, dtype=torch.int32, device="cuda")
         with paged(ar.host, page, frames) as h:
+            if case & 1:
+                B.gpuvm_set_debug(h, B.DEBUG_POISON)
             B.gpuvm_bfs_csr(h, ar.off["off"], ar.off["col"], nv, src, lvl)
             B.gpuvm_cc_csr(h, ar.off["off"], ar.off["col"], nv, lab)
             finish(h)

@@ -84,21 +84,3 @@ def test_zipf_matches_its_probability_mass_function():
         assert abs(got - expect) < 5 * math.sqrt(expect * (1 - expect) / n), (upto, got, expect)
     part = inputs.fill_zipf_rows(np.empty(50, np.int64), 50, 11, n_ranks, s, first=777)
     assert np.array_equal(rows[777:827], part)
-
-
-def test_balanced_chunks_names_the_owner_of_each_chunks_first_edge():
-    rng = np.random.default_rng(3)
-    for _ in range(20):
-        nv = int(rng.integers(1, 40))
-        deg = rng.integers(0, 9, nv) * (rng.random(nv) < 0.6)
-        off = np.concatenate([[0], np.cumsum(deg)]).astype(np.int64)
-        ne = int(off[-1])
-        for chunk in (1, 3, 8):
-            table = inputs.balanced_chunks(off, chunk)
-            n_chunks = (ne + chunk - 1) // chunk
-            assert table.dtype == np.int32 and table.size == n_chunks + 1
-            owner = np.repeat(np.arange(nv), np.diff(off))            # owner[e] by definition of CSR
-            for c in range(n_chunks):
-                assert table[c] == owner[c * chunk]
-            assert table[-1] == (owner[-1] if ne else 0)
-            assert np.all(np.diff(table) >= 0)

@@ -526,3 +526,24 @@ def test_bfs_page_trace_is_the_canonical_order():
     # level 2: vertex 2: off[2], off[3] (page 1), no edges
     assert pg.trace().tolist() == [0, 3, 0, 1, 3, 1, 2, 3, 4, 1]
     pg.close()
+
+
+def test_all_core_build_gives_the_bits_of_the_one_thread_build():
+    """The OpenMP build only splits outer loops: every sum, block and bag must come out bit for bit
+    as from the single-threaded oracle."""
+    par = oracle.AllCores()
+    assert par.threads >= 1
+    n = 100_003
+    a = inputs.fill_i32_u20(np.empty(n, np.int32), n, 5)
+    assert par.stream_sum_i32_direct(a) == oracle.stream_sum_i32_direct(a) == int(a.astype(np.int64).sum())
+    x = inputs.fill_f32_pm1(np.empty(n, np.float32), n, 6)
+    idx = inputs.fill_index_i64(np.empty(5000, np.int64), 5000, 7, n)
+    for block in (1, 37, 1024, 5000):
+        f1, b1 = oracle.gather_block_sums_direct(x, idx, block)
+        f2, b2 = par.gather_block_sums_direct(x, idx, block)
+        assert np.array_equal(f1.view(np.uint32), f2.view(np.uint32)) and np.array_equal(b1, b2)
+    y = inputs.fill_f32_pm1(np.empty(n, np.float32), n, 8)
+    assert np.array_equal(par.vadd_f32_direct(x, y).view(np.uint32), oracle.vadd_f32_direct(x, y).view(np.uint32))
+    t = x[:100_000].reshape(1000, 100)
+    rows = inputs.fill_zipf_rows(np.empty(7 * 300, np.int64), 7 * 300, 9, 1000, 1.05)
+    assert np.array_equal(par.embag_f32_direct(t, rows, 7).view(np.uint32), oracle.embag_f32_direct(t, rows, 7).view(np.uint32))

@@ -30,18 +30,31 @@ def test_noalloc_bfs_matches_regular_bfs_twice_in_a_row():
     ar = Arena(page, {"off": off_p, "col": col})
     want = torch.zeros(nv, dtype=torch.int32, device="cuda")
     got = torch.zeros(nv, dtype=torch.int32, device="cuda")
+    # the reference levels come from a handle of their own, so that the handle under test never
+    # sees a call that allocates scratch
+    with paged(ar.host, page, frames) as h_ref:
+        depth_want = {}
+        wants = {}
+        for source in (0, 5):
+            depth_want[source] = B.gpuvm_bfs_csr(h_ref, ar.off["off"], ar.off["col"], nv, source, want)
+            finish(h_ref)
+            wants[source] = want.clone()
+        assert B.gpuvm_scratch_bytes(h_ref) > 0                       # the regular entry point does allocate
     with paged(ar.host, page, frames) as h:
-        depth_want = B.gpuvm_bfs_csr(h, ar.off["off"], ar.off["col"], nv, 0, want)
-        finish(h)
-        for source in (0, 0, 5):               # two calls in a row, then a different source
-            if source:
-                depth_want = B.gpuvm_bfs_csr(h, ar.off["off"], ar.off["col"], nv, source, want)
+        for call, source in enumerate((0, 0, 5)):                     # two calls in a row, then a different source
             got.fill_(-7)
             B.gpuvm_reset(h)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             depth = B.gpuvm_bfs_csr_noalloc(h, ar.off["off"], ar.off["col"], nv, source, got)
+            torch.cuda.synchronize()
+            if call > 0:                                              # (the first call may load the module lazily)
+                assert torch.cuda.mem_get_info()[0] == free_before    # no device memory was taken
+            assert B.gpuvm_scratch_bytes(h) == 0                      # and none through the handle either
             finish(h)
-            assert depth == depth_want
-            assert torch.equal(got, want)
+            assert depth == depth_want[source]
+            assert torch.equal(got, wants[source])
+        want = wants[5]
         # beyond the stated maximum: refused with a clear status, nothing runs
         with pytest.raises(B.GpuvmError) as err:
             B.gpuvm_bfs_csr_noalloc(h, ar.off["off"], ar.off["col"], B.BFS_NOALLOC_MAX_VERTICES + 1, 0, got)
