@@ -1,14 +1,18 @@
 #!/usr/bin/env python
 """Benchmark of the demand-paging hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload CFG] [--shrink S]
-                    [--impl ours|reference] [--uvm] [--no-cpu-baseline]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload CFG | --configs 1,2,3,4,5]
+                    [--shrink S] [--impl ours|reference] [--no-uvm] [--no-cpu-baseline] [--no-replay]
 
 One step = one cold pass of the whole path over one workload: reset the page table, run the
 workload kernel(s) (translation, fault coalescing, frame claim, eviction, write-back,
-migration, the application arithmetic), flush dirty pages.  The default workload is the
-random gather (configuration 2: 1 GiB fp32 array, 2^26 uniform indices, 64 KiB pages,
-256 MiB pool); --workload 1..5 selects another configuration.
+migration, the application arithmetic), flush dirty pages.
+
+With no --workload all five configurations are run, the largest one last: configuration 5
+(Zipf embedding bag: 64 GiB table, 2 MiB pages, 16 GiB pool) is the headline record, timed
+for exactly K steps after W warm-up steps, and `per_config` carries the same fields for each of
+the five (configurations 1-4 with min(K, 10) steps after min(W, 3)).  --workload N runs one
+workload (1-5 the configurations, 6 CC, 7 SSSP, 8 BFS over Balanced CSR) as the headline.
 
 Rank 0 prints ONE JSON line.  `value` is the effective application GB/s (useful payload
 bytes / CUDA-event time) with all inputs resident (paged array in pinned host memory, which
@@ -113,10 +117,14 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------- link peaks
 
-# Host-link bytes per launch that ncu counted for the full-size workloads that have a committed
-# capture under profiles/ (stream_sum_kernel cfg 1: 2 097 152 sectors; gather_batch_kernel cfg 2:
-# 33 554 432 sectors of 32 bytes).
-NCU_LINK_BYTES = {1: 2097152 * 32, 2: 33554432 * 32}
+# Host-link bytes of one launch as ncu counted them (sysmem read sector misses x 32 B, plus sysmem write
+# sectors for the written workload) in the capture committed under profiles/, scaled to the full
+# launch where the capture was taken on a reduced case (traffic grows with the pages moved).
+# cfg -> (bytes per launch at full size, file under profiles/, how it was scaled)
+NCU_LINK_TRAFFIC = {
+    1: (2097152 * 32, "stream_sum_kernel_cfg1_full_set.md", "full size"),
+    2: (33554432 * 32, "gather_batch_kernel_cfg2_full_set.md", "full size"),
+}
 
 
 def measure_link(torch, B, nbytes=1 << 30, reps=5) -> dict:
@@ -150,14 +158,47 @@ def measured_peaks() -> dict:
         return {}
 
 
+def link_roofline(bytes_in: float, bytes_out: float, kernel_s: float, link: dict) -> dict:
+    """The two directions of the link work at the same time, so the floor of a launch is the slower
+    of (bytes in / inbound peak) and (bytes out / outbound peak); the fraction is that floor over
+    the measured kernel time, i.e. achieved / peak in the direction that bounds the launch."""
+    t_in = bytes_in / (link["ce_h2d_gbs"] * 1e9)
+    t_out = bytes_out / (link["ce_d2h_gbs"] * 1e9)
+    inbound = t_in >= t_out
+    moved, peak = (bytes_in, link["ce_h2d_gbs"]) if inbound else (bytes_out, link["ce_d2h_gbs"])
+    achieved = moved / kernel_s / 1e9 if kernel_s else 0.0
+    return {"bound": "host_link", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "direction": "host_to_device" if inbound else "device_to_host",
+            "floor_ms": max(t_in, t_out) * 1e3, "kernel_ms": kernel_s * 1e3,
+            "other_direction_gbs": (bytes_out if inbound else bytes_in) / kernel_s / 1e9 if kernel_s else 0.0,
+            "peak_source": "pinned cudaMemcpy measured in this run, in the direction that bounds the launch "
+                           "(floor = max(bytes in / H2D peak, bytes out / D2H peak))",
+            "frac_of_sm_issued_peak": achieved / (link["sm_h2d_gbs"] if inbound else link["sm_d2h_gbs"])}
+
+
 # ------------------------------------------------------------------- CPU oracle timing
 
-def oracle_step(cfg: int, w=None, shrink: int = 0):
-    """Time the CPU oracle (as it stands, one thread) on a bounded sample of the workload.
-    Returns (effective bytes, seconds, description of the sample)."""
+def _best_of(fn, reps=2):
+    best = None
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        fn()
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best
+
+
+def oracle_sample(cfg: int, w=None, shrink: int = 0):
+    """The bounded sample of workload `cfg` that the CPU oracle is timed on.
+    Returns (effective bytes of the sample, description, fn(impl) that runs it with `impl` = the oracle
+    module or its all-core build, whether an all-core form exists)."""
     import numpy as np
-    import oracle
     from paper_2411_05309_b200 import inputs
+    if cfg == 1:
+        n = (1 << 24) >> shrink
+        a = w.view("a", np.int32, w.n) if w is not None else inputs.fill_i32_u20(np.empty(n, np.int32), n, inputs.config_seed(1))
+        return 8 * 4 * a.size, "8 direct passes over the whole array", \
+            (lambda impl: [impl.stream_sum_i32_direct(a) for _ in range(8)]), True
     if cfg == 2:
         n, n_idx = (1 << 28) >> shrink, (1 << 26) >> shrink
         if w is not None:
@@ -165,81 +206,83 @@ def oracle_step(cfg: int, w=None, shrink: int = 0):
         else:
             x = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(2))
             idx = inputs.fill_index_i64(np.empty(n_idx, np.int64), n_idx, inputs.config_seed(2, 1), n)
-        t0 = time.perf_counter()
-        oracle.gather_block_sums_direct(x, idx, 1024)
-        pg = oracle.Pager(x.view(np.uint8), 64 << 10, max(1, (4096 >> shrink)), oracle.CLOCK, False)
-        sample = idx[: max(1, idx.size // 4)]
-        pg.gather_block_sums(0, sample, 1024)
-        dt = time.perf_counter() - t0
-        pg.close()
-        return 4 * idx.size, dt, (f"direct results for all {idx.size} indices + sequential paging replay of the first "
-                                  f"{sample.size} (no byte movement)")
-    if cfg == 1:
-        n = (1 << 24) >> shrink
-        a = w.view("a", np.int32, w.n) if w is not None else inputs.fill_i32_u20(np.empty(n, np.int32), n, inputs.config_seed(1))
-        t0 = time.perf_counter()
-        for _ in range(8):
-            oracle.stream_sum_i32_direct(a)
-        return 8 * 4 * a.size, time.perf_counter() - t0, "8 direct passes over the whole array"
+        return 4 * idx.size, f"direct block sums for all {idx.size} indices", \
+            (lambda impl: impl.gather_block_sums_direct(x, idx, 1024)), True
     if cfg == 4:
         n = min((1 << 30) >> shrink, 1 << 27)
         a = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4))
         b = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4, 1))
-        t0 = time.perf_counter()
-        oracle.vadd_f32_direct(a, b)
-        return 12 * n, time.perf_counter() - t0, f"direct vector add of the first {n} elements"
-    if cfg in (3, 8):
+        return 12 * n, f"direct vector add of the first {n} elements", (lambda impl: impl.vadd_f32_direct(a, b)), True
+    if cfg in (3, 8, 6, 7):
         scale = min(24 - shrink, 22)
         off, col = inputs.rmat_csr(scale, 16 << scale, inputs.config_seed(3))
-        t0 = time.perf_counter()
-        lvl = oracle.bfs_levels_direct(off, col, 0)
-        dt = time.perf_counter() - t0
-        deg = np.diff(off)
-        vis = lvl >= 0
-        return int(16 * vis.sum() + 4 * deg[vis].sum()), dt, f"direct BFS on an RMAT graph of scale {scale}"
-    if cfg in (6, 7):
-        scale = min(24 - shrink, 22)
-        off, col = inputs.rmat_csr(scale, 16 << scale, inputs.config_seed(3))
+        import oracle
+        if cfg in (3, 8):
+            lvl = oracle.bfs_levels_direct(off, col, 0)
+            vis = lvl >= 0
+            nbytes = int(16 * vis.sum() + 4 * np.diff(off)[vis].sum())
+            return nbytes, f"queue BFS on an RMAT graph of scale {scale} (sequential by nature: one thread)", \
+                (lambda impl: impl.bfs_levels_direct(off, col, 0)), False
         if cfg == 6:
-            t0 = time.perf_counter()
-            oracle.cc_labels_direct(off, col)
-            return 8 * off.size + 4 * col.size, time.perf_counter() - t0, f"union-find over an RMAT graph of scale {scale} (one pass over the edges)"
-        w = inputs.fill_i32_range(np.empty(col.size, np.int32), col.size, inputs.config_seed(3, 2), 1, 255)
-        t0 = time.perf_counter()
-        d = oracle.sssp_direct(off, col, w, 0)
-        dt = time.perf_counter() - t0
+            return 8 * off.size + 4 * col.size, f"union-find over an RMAT graph of scale {scale} (one pass over the edges)", \
+                (lambda impl: impl.cc_labels_direct(off, col)), False
+        wt = inputs.fill_i32_range(np.empty(col.size, np.int32), col.size, inputs.config_seed(3, 2), 1, 255)
+        d = oracle.sssp_direct(off, col, wt, 0)
         reached = d != 0x7FFFFFFF
-        return int(16 * reached.sum() + 8 * np.diff(off)[reached].sum()), dt, f"Dijkstra on an RMAT graph of scale {scale}"
+        return int(16 * reached.sum() + 8 * np.diff(off)[reached].sum()), f"Dijkstra on an RMAT graph of scale {scale}", \
+            (lambda impl: impl.sssp_direct(off, col, wt, 0)), False
     if cfg == 5:
         rows_n, dims, bag = 1 << 20, 128, 32
         t = inputs.fill_f32_pm1(np.empty(rows_n * dims, np.float32), rows_n * dims, inputs.config_seed(5)).reshape(rows_n, dims)
         n_lookups = 1 << 21
         rows = inputs.fill_zipf_rows(np.empty(n_lookups, np.int64), n_lookups, inputs.config_seed(5, 1), rows_n, 1.05)
-        t0 = time.perf_counter()
-        oracle.embag_f32_direct(t, rows, bag)
-        return 4 * dims * n_lookups, time.perf_counter() - t0, f"{n_lookups} lookups into a {rows_n}-row table"
+        return 4 * dims * n_lookups, f"{n_lookups} Zipf lookups (bags of {bag}) into a {rows_n}-row table", \
+            (lambda impl: impl.embag_f32_direct(t, rows, bag)), True
     raise ValueError(cfg)
 
 
-def run_reference(args, rank: int):
-    """The reference arm of this benchmark is the CPU oracle timed on the host cores."""
-    if rank != 0:
-        return
-    times, nbytes, sample = [], 0, ""
-    for i in range(args.warmup + args.steps):
-        nbytes, dt, sample = oracle_step(args.workload, None, args.shrink)
-        if i >= args.warmup:
-            times.append(dt)
-    t = sum(times) / len(times)
-    value = nbytes / t / 1e9
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": DTYPES[args.workload], "data": "synthetic",
-            "config": {"workload": NAMES[args.workload], "shrink": args.shrink},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
-            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-            "gpu_launches": 0}
-    print(json.dumps(line), flush=True)
+def cpu_baseline(cfg: int, w=None, shrink: int = 0) -> dict:
+    """The CPU oracle as it stands, timed on a bounded sample of the workload: on one thread and,
+    where its outer loop splits over threads, on all host cores (the OpenMP build of the same file)."""
+    import oracle
+    nbytes, sample, run, splits = oracle_sample(cfg, w, shrink)
+    dt1 = _best_of(lambda: run(oracle))
+    out = {"value": nbytes / dt1 / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample, "seconds": dt1,
+           "host_cores": os.cpu_count()}
+    if splits:
+        par = oracle.AllCores()
+        dtn = _best_of(lambda: run(par))
+        out["one_thread"] = {"value": out["value"], "seconds": dt1}
+        out.update({"value": nbytes / dtn / 1e9, "cores": par.threads, "seconds": dtn,
+                    "kind": "oracle (same source built with OpenMP: outer loop split over threads)"})
+    return out
+
+
+def replay_counts(cfg: int, w) -> dict:
+    """Fault counts of the workload's canonical (sequential) page trace through the oracle's replay:
+    clock, FIFO and Belady's optimum with the configuration's number of frames.  For the order-dependent
+    GPU fault counts these say what a one-request-at-a-time pager would take."""
+    import numpy as np
+    import oracle
+    t0 = time.perf_counter()
+    if cfg == 3:
+        pg = oracle.Pager(w.host, w.page_bytes, w.n_frames, oracle.CLOCK, False)
+        pg.record_trace(1 << 28)
+        pg.bfs_levels(w.off["off"], w.off["col"], w.nv, 0)
+        trace = pg.trace().copy()
+        pg.close()
+        what = "level by level, vertices ascending, both row offsets then the edge range of each vertex"
+    elif cfg == 5:
+        rows = w.rows_host.numpy()
+        trace = ((w.off["t"] + rows.astype(np.uint64) * np.uint64(4 * w.dims)) >> np.uint64(21)).astype(np.uint64)
+        keep = np.concatenate([[True], trace[1:] != trace[:-1]])
+        trace = np.ascontiguousarray(trace[keep])
+        what = "lookups in list order, one page per row"
+    else:
+        return {}
+    out = oracle.replay_counts(trace, w.n_pages, w.page_bytes, w.n_frames)
+    out.update({"trace_records": int(trace.size), "order": what, "frames": w.n_frames, "seconds": time.perf_counter() - t0})
+    return out
 
 
 NAMES = {1: "cfg1 streaming read-reduce: int64 sum over 64 MiB int32, 4 KiB pages, 16 MiB pool",
@@ -251,6 +294,62 @@ NAMES = {1: "cfg1 streaming read-reduce: int64 sum over 64 MiB int32, 4 KiB page
          7: "SSSP from vertex 0 on the cfg3 graph with int32 weights in a third paged array, 64 KiB pages, pool = half",
          8: "BFS on the cfg3 graph stored as Balanced CSR (chunks of 16 Ki edges), 64 KiB pages, pool = half"}
 DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32", 6: "int32", 7: "int32", 8: "int32"}
+
+
+def config_of(cfg: int, shrink: int) -> dict:
+    """`config` of the JSON line: the same keys from both arms."""
+    from paper_2411_05309_b200 import configs
+    d = configs.describe(cfg, shrink)
+    d["kernel"] = d["workload"]
+    d["workload"] = NAMES[cfg]
+    return d
+
+
+def headline_of(args, world: int) -> int:
+    """The workload the top-level record is quoted on: the one asked for, else the largest configuration
+    (5) when its 64 GiB pinned table fits the host once per rank, else the next largest."""
+    if args.workload:
+        return args.workload
+    order = [int(c) for c in args.configs.split(",")]
+    try:
+        import psutil
+        ram = psutil.virtual_memory().total
+    except Exception:
+        ram = 1 << 62
+    from paper_2411_05309_b200 import configs
+    by_size = sorted(order, key=lambda c: configs.describe(c, args.shrink)["paged_bytes"], reverse=True)
+    for c in by_size:
+        if world * configs.describe(c, args.shrink)["paged_bytes"] <= 0.6 * ram:
+            return c
+    return by_size[-1]
+
+
+def run_reference(args, rank: int, world: int):
+    """The reference arm of this benchmark is the CPU oracle timed on the host cores."""
+    if rank != 0:
+        return
+    import oracle
+    cfg = headline_of(args, world)
+    nbytes, sample, run, splits = oracle_sample(cfg, None, args.shrink)
+    impl = oracle.AllCores() if splits else oracle
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        run(impl)
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    t = sum(times) / len(times)
+    value = nbytes / t / 1e9
+    cores = impl.threads if splits else 1
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": DTYPES[cfg], "data": "synthetic",
+            "config": config_of(cfg, args.shrink),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                             "host_cores": os.cpu_count()},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
 
 
 # ---------------------------------------------------------------------- rank plumbing
@@ -272,6 +371,10 @@ def replica_throughput(world: int, units_per_rank: float, slowest_seconds: float
 
 # ------------------------------------------------------------------------------- ours
 
+OUTPUTS = {1: ["d_sum"], 2: ["d_fsum", "d_bsum"], 3: ["d_level"], 4: [], 5: ["d_out"], 6: ["d_level"], 7: ["d_dist"],
+           8: ["d_level"]}
+
+
 def e2e_step(torch, B, w, cfg: int):
     """One step through the C ABI with the step's device operands coming from pinned host
     memory and the results going back to the host, all inside the timed region."""
@@ -288,8 +391,7 @@ def e2e_step(torch, B, w, cfg: int):
         h2d = w.rows_host.numel() * 8
     w.launch(stream)
     B.gpuvm_flush(w.h, stream)
-    outs = {1: ["d_sum"], 2: ["d_fsum", "d_bsum"], 3: ["d_level"], 4: [], 5: ["d_out"], 6: ["d_level"], 7: ["d_dist"], 8: ["d_level"]}[cfg]
-    for name in outs:
+    for name in OUTPUTS[cfg]:
         t = getattr(w, name)
         buf = w.__dict__.setdefault("_host_" + name, torch.empty(t.shape, dtype=t.dtype).pin_memory())
         buf.copy_(t, non_blocking=True)
@@ -297,6 +399,98 @@ def e2e_step(torch, B, w, cfg: int):
     e1.record(stream)
     e1.synchronize()
     return e0.elapsed_time(e1) / 1e3, h2d, d2h
+
+
+def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link: dict, dist, world: int,
+               local_rank: int, rank: int, barrier) -> dict:
+    """All measurements of one workload: K timed cold steps, the end-to-end steps, the run under a
+    scratch bound (cfg 2 and 5), and on rank 0 the CPU baseline, the oracle's replay counts and the same
+    kernels over managed memory."""
+    w = configs.make(cfg, args.shrink)
+    try:
+        if args.scratch_limit_mib:
+            B.gpuvm_set_scratch_limit(w.h, args.scratch_limit_mib << 20)
+        for _ in range(warmup):
+            w.run(check=False)
+        sampler = ClockSampler(local_rank, args.clock_period)
+        launches0 = B.gpuvm_launch_count()
+        barrier()
+        sampler.start()
+        t_wall0 = time.perf_counter()
+        results = [w.run(check=True) for _ in range(steps)]
+        barrier()
+        wall = time.perf_counter() - t_wall0
+        clocks = sampler.stop()
+        launches = B.gpuvm_launch_count() - launches0
+        e2e_step(torch, B, w, cfg)                                # untimed: allocates the pinned result buffers
+        e2e = [e2e_step(torch, B, w, cfg) for _ in range(max(1, min(steps, 3)))]
+
+        step_s = sum(r.seconds for r in results) / len(results)
+        kern_s = sum(r.kernel_seconds for r in results) / len(results)
+        e2e_s = sum(t for t, _, _ in e2e) / len(e2e)
+        step_s, kern_s, e2e_s = max_over_ranks(dist, [step_s, kern_s, e2e_s], "cuda")
+        eff_bytes = results[-1].effective_bytes
+        bytes_in = sum(r.stats["bytes_in"] for r in results) / len(results)
+        bytes_out = sum(r.stats["bytes_out"] for r in results) / len(results)
+        faults = sum(r.stats["faults"] for r in results) / len(results)
+        peaks = measured_peaks()
+        hbm_peak = peaks.get("hbm_gbs", 6650.0)
+        roof = link_roofline(bytes_in, bytes_out, kern_s, link)
+        traffic = NCU_LINK_TRAFFIC.get(cfg) if args.shrink == 0 and not args.scratch_limit_mib else None
+        roof["traffic"] = traffic[0] if traffic else None
+        roof["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[2]}): host-link bytes of one launch counted by ncu"
+                                  if traffic else None)
+        roof["hbm"] = {"achieved": (bytes_in + bytes_out + eff_bytes) / kern_s / 1e9, "peak": hbm_peak,
+                       "frac": ((bytes_in + bytes_out + eff_bytes) / kern_s / 1e9) / hbm_peak,
+                       "peak_source": "MEASURED_PEAKS.json" if peaks else "fallback"}
+        rec = {
+            "value": replica_throughput(world, eff_bytes, step_s) / 1e9, "unit": UNIT, "steps": steps, "warmup": warmup,
+            "ms_per_step": step_s * 1e3, "dtype": DTYPES[cfg], "config": config_of(cfg, args.shrink),
+            "migration": {
+                "in_gbs": bytes_in / step_s / 1e9, "out_gbs": bytes_out / step_s / 1e9,
+                "faults_per_s": faults / step_s, "faults": faults, "bytes_in": bytes_in, "bytes_out": bytes_out,
+                "io_amplification": bytes_in / eff_bytes if eff_bytes else None,
+                "fault_rate_ceiling_per_s": link["ce_h2d_gbs"] * 1e9 / w.page_bytes,
+            },
+            "scratch": {"bytes": B.gpuvm_scratch_bytes(w.h), "limit_bytes": args.scratch_limit_mib << 20,
+                        "what": "device memory of the workload beside the pool: request tables, staged rows, queues"},
+            "stats": results[-1].stats, "invariants": results[-1].check, "roofline": roof,
+            "e2e": {"value": replica_throughput(world, eff_bytes, e2e_s) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": e2e[-1][1], "d2h_bytes_per_step": e2e[-1][2], "ms_per_step": e2e_s * 1e3},
+            "gpu_launches": launches, "clocks": clocks, "wall_s": wall, "setup_s": w.setup_seconds,
+            "step_ms": [r.seconds * 1e3 for r in results],
+            "ms_median": statistics.median(r.seconds for r in results) * 1e3,
+            "ms_min": min(r.seconds for r in results) * 1e3,
+            "extra": results[-1].extra,
+        }
+        if cfg in (3, 8) and rank == 0:
+            pages = w.compulsory_pages()
+            rec["roofline"]["compulsory_pages"] = pages
+            rec["roofline"]["frac_compulsory"] = pages * w.page_bytes / kern_s / 1e9 / link["ce_h2d_gbs"]
+        if cfg in (2, 5) and not args.scratch_limit_mib:
+            # the same workload with its scratch bounded to an eighth of the pool: fewer requests in flight
+            # per warp, so a page serves fewer of them per visit and is fetched more often
+            bound = max(w.pool_bytes // 8, 1 << 20)
+            B.gpuvm_set_scratch_limit(w.h, bound)
+            w.run(check=False)
+            r = w.run(check=True)
+            rec["scratch"]["bounded_to_an_eighth_of_the_pool"] = {
+                "limit_bytes": bound, "scratch_bytes_used_by_this_run": None, "ms_per_step": r.seconds * 1e3,
+                "value": r.effective_bytes / r.seconds / 1e9, "faults": r.stats["faults"],
+                "in_gbs": r.stats["bytes_in"] / r.seconds / 1e9, "invariants_status": r.check["status"]}
+            B.gpuvm_set_scratch_limit(w.h, 0)
+        if rank == 0:
+            if not args.no_cpu_baseline:
+                rec["cpu_baseline"] = cpu_baseline(cfg, w if cfg in (1, 2) else None, args.shrink)
+            if not args.no_replay and cfg in (3, 5) and args.shrink >= 0:
+                rec["oracle_replay_faults"] = replay_counts(cfg, w)
+            if not args.no_uvm and (args.uvm or cfg in (1, 3)):
+                from paper_2411_05309_b200 import uvm
+                rec["uvm"] = uvm.run_twin(cfg, args.shrink, timeout_s=args.uvm_timeout, w=w if cfg in (1, 3) else None)
+        return rec
+    finally:
+        w.close()
+        torch.cuda.empty_cache()
 
 
 def run_ours(args, rank: int, world: int, local_rank: int):
@@ -319,105 +513,32 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         torch.cuda.synchronize()
 
     link = measure_link(torch, B)
-    w = configs.make(args.workload, args.shrink)
-    if args.scratch_limit_mib:
-        B.gpuvm_set_scratch_limit(w.h, args.scratch_limit_mib << 20)
-    for _ in range(args.warmup):
-        w.run(check=False)
-    sampler = ClockSampler(local_rank, args.clock_period)
-    launches0 = B.gpuvm_launch_count()
-    barrier()
-    sampler.start()
-    t_wall0 = time.perf_counter()
-    results = [w.run(check=True) for _ in range(args.steps)]
-    barrier()
-    wall = time.perf_counter() - t_wall0
-    clocks = sampler.stop()
-    launches = B.gpuvm_launch_count() - launches0
-    e2e_step(torch, B, w, args.workload)                       # untimed: allocates the pinned result buffers
-    e2e = [e2e_step(torch, B, w, args.workload) for _ in range(max(1, min(args.steps, 3)))]
-
-    step_s = sum(r.seconds for r in results) / len(results)
-    kern_s = sum(r.kernel_seconds for r in results) / len(results)
-    e2e_s = sum(t for t, _, _ in e2e) / len(e2e)
-    step_s, kern_s, e2e_s = max_over_ranks(dist, [step_s, kern_s, e2e_s], "cuda")
-    eff_bytes = results[-1].effective_bytes
-    st = results[-1].stats
-    ck = results[-1].check
-    bytes_in = sum(r.stats["bytes_in"] for r in results) / len(results)
-    bytes_out = sum(r.stats["bytes_out"] for r in results) / len(results)
-    faults = sum(r.stats["faults"] for r in results) / len(results)
-    peaks = measured_peaks()
-    hbm_peak = peaks.get("hbm_gbs", 6650.0)
-    link_peak = link["ce_h2d_gbs"] if bytes_out == 0 else link["ce_h2d_gbs"] + link["ce_d2h_gbs"]
-    moved = bytes_in + bytes_out
-
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        w.close()
-        return
-
-    line = {
-        "metric": METRIC, "value": replica_throughput(world, eff_bytes, step_s) / 1e9, "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": DTYPES[args.workload], "data": "synthetic",
-        "config": {**w.describe(), "workload": NAMES[args.workload], "replicas": world,
-                   "cache_state": "cold every step: page table reset, paged array (>= 8x L2 at full size) re-read "
-                                  "from host memory; nothing of a previous step stays resident"},
-        "migration": {
-            "in_gbs": bytes_in / step_s / 1e9, "out_gbs": bytes_out / step_s / 1e9,
-            "faults_per_s": faults / step_s, "faults": faults, "bytes_in": bytes_in, "bytes_out": bytes_out,
-            "io_amplification": bytes_in / eff_bytes if eff_bytes else None,
-            "frac_of_pinned_copy_peak": (moved / step_s / 1e9) / link_peak,
-            "frac_of_sm_link_peak": (bytes_in / step_s / 1e9) / link["sm_h2d_gbs"] if link["sm_h2d_gbs"] else None,
-            "fault_rate_ceiling_per_s": link["ce_h2d_gbs"] * 1e9 / w.page_bytes,
-        },
-        "link_peak": link,
-        "scratch": {"bytes": B.gpuvm_scratch_bytes(w.h), "limit_bytes": args.scratch_limit_mib << 20,
-                    "what": "device memory of the workload beside the pool: request tables, staged rows, queues"},
-        "stats": st, "invariants": ck,
-        "roofline": {
-            "bound": "host_link", "achieved": moved / kern_s / 1e9, "peak": link_peak, "unit": "GB/s",
-            "frac": (moved / kern_s / 1e9) / link_peak,
-            "peak_source": "pinned cudaMemcpy measured in this run (H2D; H2D + D2H when pages are written back)",
-            "traffic": NCU_LINK_BYTES.get(args.workload) if args.shrink == 0 and not args.scratch_limit_mib else None,
-            "traffic_source": "host-link bytes of one launch counted by ncu (sysmem read sector misses x 32 B) in the "
-                              "committed capture of this kernel at this size; equals the kernel's own bytes_in counter. "
-                              "DRAM traffic is not the bound on this path (9.4 % of DRAM peak in the capture of cfg 2)",
-            "hbm": {"achieved": (bytes_in + bytes_out + eff_bytes) / kern_s / 1e9, "peak": hbm_peak,
-                    "frac": ((bytes_in + bytes_out + eff_bytes) / kern_s / 1e9) / hbm_peak,
-                    "peak_source": "MEASURED_PEAKS.json" if peaks else "fallback"},
-            "kernel_ms": kern_s * 1e3,
-        },
-        "e2e": {"value": replica_throughput(world, eff_bytes, e2e_s) / 1e9, "unit": UNIT, "h2d_bytes_per_step": e2e[-1][1],
-                "d2h_bytes_per_step": e2e[-1][2], "ms_per_step": e2e_s * 1e3},
-        "gpu_launches": launches, "clocks": clocks, "wall_s": wall,
-        "step_ms": [r.seconds * 1e3 for r in results],
-        "ms_median": statistics.median(r.seconds for r in results) * 1e3, "ms_min": min(r.seconds for r in results) * 1e3,
-    }
-    if args.workload == 2 and not args.scratch_limit_mib:
-        # the same workload with request tables bounded to 80 MiB (4096 requests per warp in flight instead
-        # of all 16 384 read from the index list in place): every page fetched about once per quarter of the list
-        quarter = max(1, (80 << 20) >> args.shrink)
-        B.gpuvm_set_scratch_limit(w.h, quarter)
-        w.run(check=False)
-        r = w.run(check=True)
-        B.gpuvm_set_scratch_limit(w.h, 0)
-        line["scratch"]["with_a_quarter_of_the_requests_in_flight"] = {
-            "limit_bytes": quarter, "ms_per_step": r.seconds * 1e3, "value": r.effective_bytes / r.seconds / 1e9,
-            "faults": r.stats["faults"], "in_gbs": r.stats["bytes_in"] / r.seconds / 1e9}
-    if not args.no_cpu_baseline:
-        nbytes, dt, sample = oracle_step(args.workload, w if args.workload in (1, 2) else None, args.shrink)
-        line["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": sample, "seconds": dt}
-    if args.uvm:
-        from paper_2411_05309_b200 import uvm
-        w.close()
-        line["uvm"] = uvm.run_twin(args.workload, args.shrink, timeout_s=args.uvm_timeout)
-    w.close()
+    head = headline_of(args, world)
+    order = [args.workload] if args.workload else [int(c) for c in args.configs.split(",")]
+    order = [c for c in order if c != head] + [head]               # the headline workload runs last
+    per_config = {}
+    for cfg in order:
+        steps, warmup = (args.steps, args.warmup) if cfg == head else (min(args.steps, 10), min(args.warmup, 3))
+        per_config[str(cfg)] = run_config(torch, B, configs, cfg, args, steps, warmup, link, dist, world, local_rank,
+                                          rank, barrier)
     if dist is not None:
         dist.destroy_process_group()
+    if rank != 0:
+        return
+    h = per_config[str(head)]
+    line = {"metric": METRIC, "value": h["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": h["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": h["dtype"], "data": "synthetic", "config": h["config"],
+            "replicas": world,
+            "cache_state": "cold every step: page table reset, the paged array (>= 8x L2 at full size) is re-read "
+                           "from host memory; nothing of a previous step stays resident",
+            "link_peak": link}
+    for k in ("migration", "scratch", "stats", "invariants", "roofline", "e2e", "gpu_launches", "clocks", "wall_s",
+              "step_ms", "ms_median", "ms_min", "cpu_baseline", "oracle_replay_faults", "uvm", "extra"):
+        if k in h:
+            line[k] = h[k]
+    if len(per_config) > 1:
+        line["per_config"] = per_config
     print(json.dumps(line), flush=True)
 
 
@@ -427,21 +548,25 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8])
+    ap.add_argument("--workload", type=int, default=0, choices=[0, 1, 2, 3, 4, 5, 6, 7, 8],
+                    help="run this workload only (0: all of --configs, the largest as the headline)")
+    ap.add_argument("--configs", default="1,2,3,4,5", help="configurations of the default run")
     ap.add_argument("--shrink", type=int, default=0, help="divide all sizes by 2**shrink")
-    ap.add_argument("--uvm", action="store_true", help="also run the workload over cudaMallocManaged")
+    ap.add_argument("--uvm", action="store_true", help="run every workload over cudaMallocManaged too (default: cfg 1 and 3)")
+    ap.add_argument("--no-uvm", action="store_true")
     ap.add_argument("--uvm-timeout", type=float, default=120.0)
     ap.add_argument("--scratch-limit-mib", type=int, default=0,
                     help="bound of the workload's device scratch (request tables, staged rows); 0 = none. Less scratch "
                          "means fewer page requests in flight per warp and more faults")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-replay", action="store_true", help="skip the oracle's sequential replay counts (cfg 3 and 5)")
     ap.add_argument("--clock-period", type=float, default=0.1, help="seconds between NVML clock samples")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
-        run_reference(args, rank)
+        run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)
 

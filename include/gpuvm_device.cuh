@@ -8,6 +8,7 @@
  *   T     gpuvm_read <T>(vm, elem_index, base_byte_off)        pin, load, unpin
  *   void  gpuvm_write<T>(vm, elem_index, value, base_byte_off) pin, mark dirty, store, unpin
  *   void* gpuvm_ptr(vm, byte_off, mode, &token)                pin and hand out a frame pointer
+ *   void* gpuvm_ptr_if_resident(vm, byte_off, &token)          the same, but only if the page is there: no fault, no wait
  *   void  gpuvm_release(vm, token)                             unpin what gpuvm_ptr pinned
  *   void  gpuvm_clean(vm, token, p)                            write a pinned page back now (eager write-back)
  *   void  gpuvm_prefetch(vm, byte_off)                         fetch a page ahead of its use, unpinned
@@ -727,6 +728,41 @@ __device__ __forceinline__ void *gpuvm_ptr(const gpuvm_dev_t &vm, unsigned long 
     token->leader = 0; token->group = 0; token->vpn = 0;
     gpuvm::access<0>(vm, byte_off, mode, v, token, &p);
     return p;
+}
+
+/*
+ * gpuvm_ptr in read mode for callers that want a page only if it is there already: never faults,
+ * never waits.  A resident page is pinned and its frame address returned (release it with
+ * gpuvm_release, as after gpuvm_ptr); for a page that is absent or in transit nullptr is returned
+ * and nothing stays pinned.  Lanes that call together may ask for different pages.  Used by the
+ * graph sweeps to re-expand a vertex behind the sweep position while its pages are still in the pool.
+ */
+__device__ __forceinline__ void *gpuvm_ptr_if_resident(const gpuvm_dev_t &vm, unsigned long long byte_off,
+                                                       gpuvm_token *token)
+{
+    using namespace gpuvm;
+    token->leader = 0; token->group = 0; token->vpn = 0;
+    if (byte_off >= vm.bytes) { set_error(vm, GPUVM_E_RANGE, byte_off >> vm.page_shift); return nullptr; }
+    const unsigned long long vpn = byte_off >> vm.page_shift;
+    const unsigned int active = __activemask();
+    const unsigned int group = __match_any_sync(active, vpn);
+    const unsigned int leader = __ffs(group) - 1;
+    const bool is_leader = lane_id() == leader;
+    unsigned long long *pte = vm.pte + vpn;
+    unsigned long long w = 0;
+    if (is_leader) {
+        w = guard_pin(vm, pte, pin_acquire(pte) + 1ull);
+        if (w == kPinRefused) w = 0;
+        else if ((w & kStMask) != kValid) { unpin(pte); w = 0; }
+        else {
+            if (vm.policy == GPUVM_POLICY_CLOCK && !(w & kRef)) atomicOr(pte, kRef);
+            if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1);
+        }
+    }
+    w = __shfl_sync(group, w, leader);
+    if ((w & kStMask) != kValid) return nullptr;
+    token->vpn = vpn; token->group = group; token->leader = is_leader;
+    return vm.pool + (((w & kFrameMask) >> kFrameShift) << vm.page_shift) + (byte_off & ((1ull << vm.page_shift) - 1ull));
 }
 
 /* Called by the same lanes that called gpuvm_ptr together. */

@@ -69,20 +69,29 @@ int gpuvm_gather_f32_unbatched(gpuvm_t h, size_t x_off, const int64_t *d_idx, si
                                float *d_fsum, int64_t *d_bsum, void *stream);
 
 /*
- * Level-synchronous BFS over a CSR graph whose int64 row offsets (nv + 1 of them,
- * at off_off) and int32 column indices (at col_off) are paged (Section 5.2 runs
- * BFS on CSR through the paged arrays).  d_level: nv int32 in device memory,
- * receives the hop distance from `source`, -1 where unreachable.  Per level one
- * sweep over the vertices in ascending order (warps draw chunks of 32 consecutive
- * vertices from a ticket counter, so the grid moves through the arrays in address
- * order; per chunk the column pages its edges span are pinned one at a time).
- * Very long neighbour lists are cut at page boundaries into pieces that go to a
- * queue which all warps of the same launch serve between their chunks (the
- * imbalance Section 5.2 describes), so the pieces are expanded while their pages
- * are under the sweep window.  One launch per level.  Synchronises the
- * stream between levels; *n_levels (host pointer, may be NULL) receives the number
- * of levels expanded, counting the last one that discovers nothing.  Uses 2 MiB of
- * the handle's device scratch (queue of neighbour-list pieces, counters).
+ * BFS over a CSR graph whose int64 row offsets (nv + 1 of them, at off_off) and int32
+ * column indices (at col_off) are paged (Section 5.2 runs BFS on CSR through the paged
+ * arrays).  d_level: nv int32 in device memory, receives the hop distance from `source`,
+ * -1 where unreachable (nv < 2^30).
+ *
+ * The sweeps go over the vertices in address order (warps draw chunks of 32 consecutive
+ * vertices from a ticket counter, so the grid moves through the arrays as a narrow window;
+ * per chunk the column pages its edges span are pinned one at a time), alternating
+ * direction.  They are label-correcting rather than level-synchronous: a vertex is
+ * expanded whenever its level has been lowered since it was last expanded (the level
+ * array holds level << 1 | dirty while the sweeps run; lowering is an atomicMin that sets
+ * the bit), so one sweep carries as many hops as the vertex order allows, and a vertex
+ * that is lowered behind the sweep position is queued and re-expanded in the same sweep by
+ * whichever warp is free, provided its pages are still in the pool (gpuvm_ptr_if_resident:
+ * no fault is taken for it; otherwise it stays dirty for the next sweep).  The fixed point
+ * is the BFS level.  With a pool of half the graph almost every page is fetched once per
+ * run, where one sweep per level fetched most of the graph once per level.
+ * Very long neighbour lists are cut at page boundaries into pieces that go to a queue which
+ * all warps of the same launch serve between their chunks (the imbalance Section 5.2
+ * describes).  The first sweep expands the source alone.  One launch per sweep; the stream is
+ * synchronised between sweeps.  *n_levels (host pointer, may be NULL) receives the largest
+ * level + 1.  Uses 2 MiB + max(nv, 2^18) bytes of the handle's device scratch (the two
+ * queues and the counters).
  */
 int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
                   int32_t *d_level, int *n_levels, void *stream);
@@ -118,13 +127,15 @@ int gpuvm_bcsr_build(const int64_t *row_off, size_t nv, size_t chunk_edges, int3
                      size_t *n_chunks_out);
 
 /*
- * Connected components of the same kind of graph (Section 5.2 evaluates CC next to
- * BFS): d_label[v] receives the smallest vertex number of the weakly connected
- * component of v (edges count in both directions).  Label propagation: every sweep
- * visits every edge (u, c) and lowers the larger of the two labels to the smaller
- * with atomicMin, until a sweep changes nothing.  Sweeps alternate direction like
- * the BFS levels.  *n_sweeps (host pointer, may be NULL) receives the number of
- * sweeps.  Uses 2 MiB of the handle's device scratch.  Synchronises per sweep.
+ * Connected components of the same kind of graph (Section 5.2 evaluates CC next to BFS):
+ * d_label[v] receives the smallest vertex number of the weakly connected component of v
+ * (edges count in both directions).  Concurrent union-find in ONE sweep over the edges:
+ * d_label starts as the identity and serves as the parent array; for every edge the roots
+ * of both ends are found (with path halving) and the larger root is hooked under the
+ * smaller with a compare-and-swap that succeeds only while it still is a root; a finishing
+ * kernel replaces every parent by its root.  Every page of the graph is fetched once.
+ * *n_sweeps (host pointer, may be NULL) receives the number of sweeps over the edges (1).
+ * Uses 2 MiB of the handle's device scratch.  Synchronises the stream.
  */
 int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps,
                  void *stream);
@@ -136,11 +147,11 @@ int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *
  * the page size, so that the weights of an edge range sit at the same place in their
  * page as the columns do in theirs; both pages are held together while the range is
  * relaxed, hence the pool needs at least two frames per warp of the grid
- * (GPUVM_E_FRAMES otherwise).  Bellman-Ford rounds over the vertices that changed in
- * the previous round; d_dist[v] receives the distance from `source`, 0x7FFFFFFF
- * where unreachable (path lengths must stay below that).  *n_rounds (host pointer,
- * may be NULL) receives the number of rounds.  Uses 2 MiB + 2 nv bytes of the
- * handle's device scratch.  Synchronises per round.
+ * (GPUVM_E_FRAMES otherwise).  The same label-correcting sweeps as gpuvm_bfs_csr with
+ * the edge weight in place of 1; d_dist[v] receives the distance from `source`,
+ * 0x7FFFFFFF where unreachable (path lengths must stay below 2^30).  *n_rounds (host
+ * pointer, may be NULL) receives the number of sweeps.  Uses 2 MiB + max(nv, 2^18) bytes of
+ * the handle's device scratch.  Synchronises per sweep.
  */
 int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source,
                    int32_t *d_dist, int *n_rounds, void *stream);
@@ -154,10 +165,11 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
  * allocation synchronises the whole device and may take a driver lock), plug-ins
  * whose host forbids allocation after start-up, and processes that have handed
  * all free device memory to their own pool, where cudaMalloc would simply fail.
- * For them this variant does exactly what gpuvm_bfs_csr does, same kernels, same
- * arguments, same results, but takes its scratch (the queue of neighbour-list
- * pieces and the level counters, 2 MiB + 640 bytes) from an array that is part of
- * the library's device image.  It calls no cudaMalloc, cudaFree or other
+ * For them this variant computes what gpuvm_bfs_csr computes, same arguments, same
+ * results, with one sweep per level (the queue that gpuvm_bfs_csr keeps for vertices
+ * lowered behind the sweep grows with the graph and has no place in a fixed array),
+ * and takes its scratch (the queue of neighbour-list pieces and the sweep counters,
+ * 2 MiB + 1 KiB) from an array that is part of the library's device image.  It calls no cudaMalloc, cudaFree or other
  * allocating routine.
  *
  *   - Limit: nv <= GPUVM_BFS_NOALLOC_MAX_VERTICES, the graph size the fixed queue

@@ -4,7 +4,10 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <chrono>
 #include <cstdint>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "gpuvm.h"
@@ -30,6 +33,10 @@ struct Paged {
     {
         return static_cast<unsigned char *>(gpuvm_ptr(vm, off, mode, &t));
     }
+    __device__ __forceinline__ unsigned char *pin_if_resident(unsigned long long off, gpuvm_token &t) const
+    {
+        return static_cast<unsigned char *>(gpuvm_ptr_if_resident(vm, off, &t));
+    }
     __device__ __forceinline__ void release(const gpuvm_token &t) const { gpuvm_release(vm, t); }
     __device__ __forceinline__ void clean(const gpuvm_token &t, const void *p) const { gpuvm_clean(vm, t, p); }
     __device__ __forceinline__ void prefetch(unsigned long long off) const { gpuvm_prefetch(vm, off); }
@@ -52,6 +59,7 @@ struct Raw {
     template <typename T>
     __device__ __forceinline__ void write(unsigned long long off, unsigned long long i, T v) const { reinterpret_cast<T *>(base + off)[i] = v; }
     __device__ __forceinline__ unsigned char *pin(unsigned long long off, int, gpuvm_token &) const { return base + off; }
+    __device__ __forceinline__ unsigned char *pin_if_resident(unsigned long long off, gpuvm_token &) const { return base + off; }
     __device__ __forceinline__ void release(const gpuvm_token &) const {}
     __device__ __forceinline__ void clean(const gpuvm_token &, const void *) const {}
     __device__ __forceinline__ void prefetch(unsigned long long) const {}
@@ -325,6 +333,7 @@ constexpr unsigned int kBigQueue = 65536;  // entries of the span queue (four in
 constexpr unsigned int kChunksPerTicket = 2;  // consecutive chunks of 32 vertices a warp draws at a time
 constexpr unsigned int kSpanPoll = 4;       // a warp looks into the span queue before every kSpanPoll-th chunk
 constexpr long long kAhead = 16;           // pages of look-ahead of the sweeps' prefetches
+constexpr unsigned int kNoVertex = 0xFFFFFFFFu;
 
 // counters of a sweep, each in a 128-byte line of its own (the chunk ticket is hit by every warp all
 // the time; a load of a word in the same line would queue behind those atomics)
@@ -333,47 +342,119 @@ constexpr int kCntPushed = 32;       // span queue entries reserved
 constexpr int kCntTicket = 64;       // chunk ticket
 constexpr int kCntTaken = 96;        // span ticket
 constexpr int kCntDone = 128;        // chunks finished
-constexpr int kCntWords = 160;
+constexpr int kCntBehindTail = 160;  // entries reserved in the queue of vertices that changed behind the sweep position
+constexpr int kCntBehindHead = 192;  // entries of that queue taken
+constexpr int kCntMax = 224;         // largest label (written by the finishing kernel)
+constexpr int kCntWords = 256;
 
-// What a sweep does with a vertex and with each of its edges.  peek reads what the edge's other
-// end holds now (a plain load: several edges' peeks are issued together), edge decides and updates.
+// What a sweep does with a vertex and with each of its edges.
+//   active(v)   does the sweep expand v?
+//   begin(v)    called once by the lane that owns an active v before its edges are visited; returns the
+//               value of v that its edges are visited with
+//   value(u)    the same value without side effects (for pieces of a long list that are expanded later)
+//   peek(c)     what the edge's other end holds now (a plain load: several edges' peeks are issued together)
+//   edge(...)   decides and updates; returns 1 when it changed something.  `pos` is how far the sweep has
+//               got (in chunks, in sweep order), for operations that care what lies behind it
 struct BfsOp {                              // level-synchronous BFS: expand the vertices of the current level
+    static constexpr bool kBehind = false;
     int *level;
     int depth;
     __device__ __forceinline__ bool active(unsigned long long v) const { return level[v] == depth; }
+    __device__ __forceinline__ int begin(unsigned long long) const { return depth; }
+    __device__ __forceinline__ int value(unsigned long long) const { return depth; }
     __device__ __forceinline__ int peek(int c) const { return level[c]; }
-    __device__ __forceinline__ unsigned int edge(long long, int c, int, int seen) const
+    __device__ __forceinline__ unsigned int edge(int, long long, int c, int, int seen, unsigned int) const
     {
         return seen == -1 && atomicCAS(level + c, -1, depth + 1) == -1;
     }
 };
 
-struct CcOp {                               // label propagation over every edge, both ways, minimum label wins
-    int *label;
-    __device__ __forceinline__ bool active(unsigned long long) const { return true; }
-    __device__ __forceinline__ int peek(int c) const { return label[c]; }
-    __device__ __forceinline__ unsigned int edge(long long u, int c, int, int lc) const
+// Connected components by concurrent union-find in ONE pass over the edges (the lock-free scheme of
+// Anderson and Woll as used by ECL-CC): parent[] starts as the identity; for every edge the roots of its
+// two ends are found (with path halving) and the larger root is hooked under the smaller one with a
+// compare-and-swap that only succeeds while it still is a root.  Parents only ever decrease, so the root
+// of a tree is the smallest vertex in it; a finishing kernel replaces every parent by its root.
+struct CcOp {
+    static constexpr bool kBehind = false;
+    int *parent;
+    __device__ __forceinline__ static int ld(const int *p) { return __ldcg(p); }
+    __device__ __forceinline__ int find(int x) const
     {
-        const int lu = label[u];
-        if (lu < lc) return atomicMin(label + c, lu) > lu;
-        if (lc < lu) return atomicMin(label + u, lc) > lc;
+        int p = ld(parent + x);
+        while (p != x) {
+            const int gp = ld(parent + p);
+            if (gp != p) parent[x] = gp;                 // path halving: any ancestor is a valid parent
+            x = p;
+            p = gp;
+        }
+        return x;
+    }
+    __device__ __forceinline__ int find_read_only(int x) const
+    {
+        for (int p = ld(parent + x); p != x; p = ld(parent + x)) x = p;
+        return x;
+    }
+    __device__ __forceinline__ bool active(unsigned long long) const { return true; }
+    __device__ __forceinline__ int begin(unsigned long long v) const { return (int)v; }
+    __device__ __forceinline__ int value(unsigned long long u) const { return (int)u; }
+    __device__ __forceinline__ int peek(int c) const { return ld(parent + c); }
+    __device__ __forceinline__ unsigned int edge(int, long long u, int c, int, int pc, unsigned int) const
+    {
+        int ra = find((int)u), rb = pc == c ? c : find(pc);
+        while (ra != rb) {
+            if (ra < rb) { const int t = ra; ra = rb; rb = t; }          // ra is the larger root: it goes under rb
+            const int old = atomicCAS(parent + ra, ra, rb);
+            if (old == ra) return 1;
+            ra = find(old);                                              // ra was no longer a root
+            rb = find(rb);
+        }
         return 0;
     }
 };
 
-struct SsspOp {                             // Bellman-Ford rounds: relax the edges of vertices that changed last round
+// Label-correcting relaxation: BFS (every edge has length 1) and SSSP (edge weights).  dist[v] holds
+// (distance << 1) | dirty.  A vertex is expanded when its dirty bit is set; expanding clears the bit with
+// an atomic AND whose return value is the distance the edges are relaxed with; lowering a distance is an
+// atomicMin with the bit set, so whoever is lowered is expanded (again) later.  The fixed point is the
+// shortest distance.  One sweep carries as many hops as the order of the vertices allows, and a vertex
+// that is lowered BEHIND the sweep position goes to a queue from which idle moments of all warps
+// re-expand it in the same sweep, provided its pages are still resident (no fault is taken for it;
+// otherwise it simply stays dirty for the next sweep).  Level-synchronous sweeps fetch most of the graph
+// once per level; this way almost every page is fetched once per run.
+constexpr int kLcInf = 0x7FFFFFFE;          // unreached, not dirty
+template <bool WEIGHTED>
+struct LcOp {
+    static constexpr bool kBehind = true;
     int *dist;
-    const unsigned char *cur;
-    unsigned char *next;
-    __device__ __forceinline__ bool active(unsigned long long v) const { return cur[v] != 0; }
-    __device__ __forceinline__ int peek(int c) const { return dist[c]; }
-    __device__ __forceinline__ unsigned int edge(long long u, int c, int w, int dc) const
+    unsigned int *behind_q;                 // vertex numbers, kNoVertex = not written yet
+    unsigned int *counters;
+    unsigned int behind_cap, n_chunks;
+    int backward;
+    unsigned int only;                      // kNoVertex, or the one vertex this sweep expands (the first sweep: the source)
+    __device__ __forceinline__ bool active(unsigned long long v) const
     {
-        const int du = dist[u];
-        if (du == 0x7FFFFFFF) return 0;
-        const int nd = du + w;
-        if (nd < dc && atomicMin(dist + c, nd) > nd) { next[c] = 1; return 1; }
-        return 0;
+        return only == kNoVertex ? (__ldcg(dist + v) & 1) != 0 : v == only;
+    }
+    __device__ __forceinline__ int begin(unsigned long long v) const { return atomicAnd(dist + v, ~1) >> 1; }
+    __device__ __forceinline__ void redirty(unsigned long long v) const { atomicOr(dist + v, 1); }
+    __device__ __forceinline__ int value(unsigned long long u) const { return __ldcg(dist + u) >> 1; }
+    __device__ __forceinline__ int peek(int c) const { return dist[c]; }
+    __device__ __forceinline__ unsigned int edge(int du, long long, int c, int w, int seen, unsigned int pos) const
+    {
+        const int nd = ((du + (WEIGHTED ? w : 1)) << 1) | 1;
+        if (nd >= seen || atomicMin(dist + c, nd) <= nd) return 0;
+        // lowered.  Has the sweep passed c already (or is it just about to)?  Then nobody will look at it
+        // again in this sweep unless it is queued.
+        const unsigned int ci = (unsigned int)c >> 5, si = backward ? n_chunks - 1u - ci : ci;
+        if (si < pos && only == kNoVertex) {
+            const unsigned int m = __activemask(), lane = gpuvm::lane_id(), leader = __ffs(m) - 1;
+            unsigned int base = 0;
+            if (lane == leader) base = atomicAdd(counters + kCntBehindTail, (unsigned int)__popc(m));
+            base = __shfl_sync(m, base, leader);
+            const unsigned int slot = base + __popc(m & ((1u << lane) - 1u));
+            if (slot < behind_cap) gpuvm::st_relaxed_u32(behind_q + slot, (unsigned int)c);   // full: c stays dirty for the next sweep
+        }
+        return 1;
     }
 };
 
@@ -382,8 +463,8 @@ struct SsspOp {                             // Bellman-Ford rounds: relax the ed
 // the peeks at their other ends, then the updates.
 template <class Mem, class Op, bool WEIGHTED>
 __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned char *col_unit, const unsigned char *w_unit,
-                                                    long long first, long long u, long long elo, long long ehi,
-                                                    unsigned int lane)
+                                                    long long first, long long u, int uval, long long elo, long long ehi,
+                                                    unsigned int lane, unsigned int pos)
 {
     constexpr int U = 4;
     unsigned int found = 0;
@@ -399,19 +480,28 @@ __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned
         for (int k = 0; k < U; ++k) seen[k] = c[k] >= 0 ? op.peek(c[k]) : 0;
 #pragma unroll
         for (int k = 0; k < U; ++k)
-            if (c[k] >= 0) found += op.edge(u, c[k], w[k], seen[k]);
+            if (c[k] >= 0) found += op.edge(uval, u, c[k], w[k], seen[k], pos);
     }
     return found;
 }
 
 __device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p) { return *reinterpret_cast<const volatile unsigned int *>(p); }
 
+// How far the sweep has got, for operations that queue what changes behind it: the chunk ticket (chunks
+// below it are drawn) plus the chunks that may be drawn while a unit of edges is being visited.
+__device__ __forceinline__ unsigned int sweep_pos(const unsigned int *counters, unsigned int n_chunks)
+{
+    const unsigned int t = ld_volatile_u32(counters + kCntTicket), margin = 2u * kChunksPerTicket * warps_in_grid();
+    return t >= n_chunks || t + margin >= n_chunks ? n_chunks : t + margin;
+}
+
 // Expand one queued piece of a long neighbour list (all 32 lanes).  Returns this lane's number of
 // updates, or -1 when a wait ran out.  Out of line: it is the rare path of the sweep kernel and
 // would only add to the register pressure of the common one.
 template <class Mem, class Op, bool WEIGHTED>
 __device__ __noinline__ int expand_piece(const Mem m, const Op op, unsigned long long col_off, unsigned long long w_off,
-                                         const long long *span_q, unsigned int piece, long long epoch, unsigned int lane)
+                                         const long long *span_q, unsigned int *counters, unsigned int n_chunks,
+                                         unsigned int piece, long long epoch, unsigned int lane)
 {
     // its producer is between reserving the slot and publishing it
     const volatile long long *ready = span_q + 4 * (size_t)piece + 3;
@@ -435,7 +525,8 @@ __device__ __noinline__ int expand_piece(const Mem m, const Op op, unsigned long
         pw = m.pin(w_off + 4ull * elo, GPUVM_READ, tok_w);
         if (!pw) { m.release(tok); return -1; }
     }
-    const unsigned int found = visit_edges<Mem, Op, WEIGHTED>(op, p, pw, elo, u, elo, ehi, lane);
+    const unsigned int pos = Op::kBehind ? sweep_pos(counters, n_chunks) : 0u;
+    const unsigned int found = visit_edges<Mem, Op, WEIGHTED>(op, p, pw, elo, u, op.value((unsigned long long)u), elo, ehi, lane, pos);
     if (WEIGHTED) m.release(tok_w);
     m.release(tok);
     return (int)found;
@@ -454,33 +545,122 @@ __device__ __forceinline__ unsigned int take_piece(unsigned int *counters, unsig
     return __shfl_sync(0xFFFFFFFFu, piece, 0);
 }
 
-// End of a warp's sweep (all 32 lanes): expand pieces until every chunk of the sweep is finished
-// and every piece is taken.  Returns this lane's number of updates.  The wait is bounded.
+// All 32 lanes: take up to 32 vertices from the queue of vertices that were lowered behind the sweep
+// position and re-expand those whose pages are resident.  Returns this lane's number of updates, or -1 when
+// the queue was empty.  A vertex whose row offsets or edges are not in the pool is left dirty (no fault is
+// taken for it: the next sweep finds it); so is one with a very long list.
 template <class Mem, class Op, bool WEIGHTED>
-__device__ __noinline__ unsigned int drain_pieces(const Mem m, const Op op, unsigned long long col_off, unsigned long long w_off,
-                                                  const long long *span_q, unsigned int *counters, unsigned int n_chunks,
-                                                  long long epoch, unsigned int lane)
+__device__ __noinline__ int expand_behind(const Mem m, const Op op, unsigned long long off_off, unsigned long long col_off,
+                                          unsigned long long w_off, unsigned int nv, unsigned int *counters, unsigned int lane)
+{
+    // 32 slots are reserved with one fetch-and-add, and only when the queue was seen non-empty: no retry
+    // storms when thousands of warps come here at once.  Warps that saw the same state may reserve slots past
+    // the tail; such a slot is read if its producer fills it within a short wait and is given up otherwise
+    // (its vertex stays dirty and is found by the next sweep).
+    unsigned int n = 0xFFFFFFFFu, h = 0;
+    if (lane == 0) {
+        unsigned int t = ld_volatile_u32(counters + kCntBehindTail);
+        if (t > op.behind_cap) t = op.behind_cap;
+        if (ld_volatile_u32(counters + kCntBehindHead) < t) {
+            h = atomicAdd(counters + kCntBehindHead, 32u);
+            n = h < op.behind_cap ? (op.behind_cap - h < 32u ? op.behind_cap - h : 32u) : 0u;
+        }
+    }
+    n = __shfl_sync(0xFFFFFFFFu, n, 0);
+    h = __shfl_sync(0xFFFFFFFFu, h, 0);
+    if (n == 0xFFFFFFFFu) return -1;
+    unsigned int u = kNoVertex;
+    if (lane < n) {
+        unsigned int spins = 0;                               // its producer is between reserving the slot and filling it
+        while ((u = gpuvm::ld_relaxed_u32(op.behind_q + h + lane)) == kNoVertex && ++spins < 256u) __nanosleep(32);
+    }
+    bool have = u != kNoVertex && u < nv && op.active(u);
+    long long lo = 0, hi = 0;
+    if (have) {
+        gpuvm_token tok;
+        const unsigned char *p = m.pin_if_resident(off_off + 8ull * u, tok);
+        if (p) { lo = Mem::load_i64(p); m.release(tok); }
+        const unsigned char *q = p ? m.pin_if_resident(off_off + 8ull * u + 8, tok) : nullptr;
+        if (q) { hi = Mem::load_i64(q); m.release(tok); }
+        have = p && q;
+        if (have && hi <= lo) { op.begin(u); have = false; }  // nothing to expand: just not dirty any more
+        if (have && hi - lo >= kBigDegree) have = false;
+    }
+    unsigned int found = 0;
+    unsigned int todo = __ballot_sync(0xFFFFFFFFu, have);
+    const unsigned long long unit = m.unit();
+    const unsigned int pos = sweep_pos(counters, op.n_chunks);
+    while (todo) {
+        const int L = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const long long bu = __shfl_sync(0xFFFFFFFFu, u, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
+        long long first = __shfl_sync(0xFFFFFFFFu, lo, L);
+        int uval = 0;
+        bool begun = false, complete = true;
+        while (first < bhi) {
+            const unsigned long long byte = col_off + 4ull * first;
+            long long last = (long long)(((byte / unit + 1) * unit - col_off) / 4);
+            if (last > bhi) last = bhi;
+            gpuvm_token tok, tok_w;
+            const unsigned char *p = m.pin_if_resident(byte, tok);
+            if (!p) { complete = false; break; }
+            const unsigned char *pw = nullptr;
+            if (WEIGHTED) {
+                pw = m.pin_if_resident(w_off + 4ull * first, tok_w);
+                if (!pw) { m.release(tok); complete = false; break; }
+            }
+            if (!begun) {
+                if (lane == 0) uval = op.begin((unsigned long long)bu);
+                uval = __shfl_sync(0xFFFFFFFFu, uval, 0);
+                begun = true;
+            }
+            found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, bu, uval, first, last, lane, pos);
+            if (WEIGHTED) m.release(tok_w);
+            m.release(tok);
+            first = last;
+        }
+        if (begun && !complete && lane == 0) op.redirty((unsigned long long)bu);   // the rest of its list waits for the next sweep
+    }
+    return (int)found;
+}
+
+// End of a warp's sweep (all 32 lanes): expand pieces (and vertices lowered behind the sweep) until every
+// chunk of the sweep is finished and every piece is taken.  Returns this lane's number of updates.  The wait is bounded.
+template <class Mem, class Op, bool WEIGHTED>
+__device__ __noinline__ unsigned int drain_pieces(const Mem m, const Op op, unsigned long long off_off, unsigned long long col_off,
+                                                  unsigned long long w_off, unsigned int nv, const long long *span_q,
+                                                  unsigned int *counters, unsigned int n_chunks, long long epoch, unsigned int lane)
 {
     unsigned int found = 0, sleep_ns = 64;
     unsigned long long idle_since = 0;
     for (;;) {
         const unsigned int piece = take_piece(counters, lane);
         if (piece != 0xFFFFFFFFu) {
-            const int r = expand_piece<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, piece, epoch, lane);
+            const int r = expand_piece<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, counters, n_chunks, piece, epoch, lane);
             if (r < 0) return found;
             found += (unsigned int)r;
             idle_since = 0;
             sleep_ns = 64;
             continue;
         }
+        if constexpr (Op::kBehind) {
+            const int r = expand_behind<Mem, Op, WEIGHTED>(m, op, off_off, col_off, w_off, nv, counters, lane);
+            if (r >= 0) {
+                found += (unsigned int)r;
+                idle_since = 0;
+                sleep_ns = 64;
+                continue;
+            }
+        }
         int state = 0;                                        // 0 wait, 1 done, 2 gave up
         if (lane == 0) {
             unsigned int pushed = ld_volatile_u32(counters + kCntPushed);
             if (pushed > kBigQueue) pushed = kBigQueue;
+            const unsigned int queued_behind = Op::kBehind ? ld_volatile_u32(counters + kCntBehindTail) : 0u;
             // Nothing queued in this sweep so far: leave at once (a warp that queues pieces later also
             // comes through here and sees to them); thousands of idle warps polling would only be in
             // the way of the ones still at work.  Otherwise stay and help until all chunks are finished.
-            if (pushed == 0u) state = 1;
+            if (pushed == 0u && queued_behind == 0u) state = 1;
             else if (ld_volatile_u32(counters + kCntDone) >= n_chunks && ld_volatile_u32(counters + kCntTaken) >= pushed) state = 1;
             else {
                 const unsigned long long t = gpuvm::now_ns();
@@ -507,13 +687,14 @@ __device__ __noinline__ unsigned int drain_pieces(const Mem m, const Op op, unsi
 // looks into that queue before it draws its next chunk, so the pieces are expanded by the whole
 // grid while their pages are still under (or just ahead of) the sweep window.  An entry is
 // published by its `ready` word (= sweep + 1, written after a fence; the queue is zeroed once per
-// call).  A warp leaves when all chunks are finished and all pieces are taken; every wait is
-// bounded.
+// call).  Operations with kBehind also keep a queue of vertices that changed behind the sweep position
+// (see LcOp), served in the same way.  A warp leaves when all chunks are finished and all pieces are
+// taken; every wait is bounded.
 template <class Mem, class Op, bool WEIGHTED>
 __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
                                                           unsigned long long w_off, unsigned int nv,
                                                           unsigned long long n_edges, long long *__restrict__ span_q,
-                                                          unsigned int *__restrict__ counters, int sweep)
+                                                          unsigned int *__restrict__ counters, int sweep, int backward)
 {
     const unsigned int lane = threadIdx.x & 31;
     const unsigned long long unit = m.unit();
@@ -525,10 +706,17 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
         if ((iter++ & (kSpanPoll - 1)) == 0) {
             const unsigned int piece = take_piece(counters, lane);
             if (piece != 0xFFFFFFFFu) {
-                const int r = expand_piece<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, piece, epoch, lane);
+                const int r = expand_piece<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, counters, n_chunks, piece, epoch, lane);
                 if (r < 0) break;
                 found += (unsigned int)r;
                 continue;
+            }
+        }
+        // ---- vertices that were lowered behind the sweep position, while their pages are still there
+        if constexpr (Op::kBehind) {
+            if ((iter & (kSpanPoll - 1)) == 1) {
+                const int r = expand_behind<Mem, Op, WEIGHTED>(m, op, off_off, col_off, w_off, nv, counters, lane);
+                if (r > 0) found += (unsigned int)r;
             }
         }
         // ---- the next chunk of 32 vertices (a ticket is good for kChunksPerTicket consecutive chunks)
@@ -540,7 +728,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
                 // no chunk left: report the finished ones, then help with the pieces until all chunks
                 // are finished and all pieces taken
                 if (lane == 0 && my_done) { __threadfence(); atomicAdd(counters + kCntDone, my_done); }
-                found += drain_pieces<Mem, Op, WEIGHTED>(m, op, col_off, w_off, span_q, counters, n_chunks, epoch, lane);
+                found += drain_pieces<Mem, Op, WEIGHTED>(m, op, off_off, col_off, w_off, nv, span_q, counters, n_chunks, epoch, lane);
                 break;
             }
             next_chunk = t;
@@ -548,7 +736,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
         }
         const unsigned int chunk = next_chunk++;
         ++my_done;
-        const unsigned long long v0 = 32ull * ((sweep & 1) ? n_chunks - 1 - chunk : chunk);
+        const unsigned long long v0 = 32ull * (backward ? n_chunks - 1 - chunk : chunk);
         const unsigned long long v = v0 + lane;
         const bool active = v < nv && op.active(v);
         if (!__any_sync(0xFFFFFFFFu, active)) continue;
@@ -556,7 +744,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
         // page, the others return at once), so that the window does not stall on one page at a time
         const bool dense = __popc(__ballot_sync(0xFFFFFFFFu, active)) >= 8;   // a sparse frontier may never get there
         if (dense) {
-            const long long ahead = (long long)(off_off + 8ull * v0) + ((sweep & 1) ? -kAhead : kAhead) * (long long)unit;
+            const long long ahead = (long long)(off_off + 8ull * v0) + (backward ? -kAhead : kAhead) * (long long)unit;
             if (ahead >= (long long)off_off && ahead < (long long)(off_off + 8ull * nv)) m.prefetch((unsigned long long)ahead);
         }
         // row offsets of the chunk: off[v0 .. v0+32], clamped to the nv + 1 entries that exist
@@ -577,6 +765,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
         }
         if (!active) { lo = 0; hi = 0; }
+        const int uval = active ? op.begin(v) : 0;          // the value this vertex's edges are visited with
         // long neighbour lists: cut them at unit boundaries and queue the pieces for the grid
         unsigned int bigs = __ballot_sync(0xFFFFFFFFu, hi - lo >= kBigDegree);
         while (bigs) {
@@ -612,8 +801,8 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             rhi = b > rhi ? b : rhi;
         }
         if (dense && rhi > rlo) {                        // and the column page the sweep will reach
-            const long long ahead = (long long)(col_off + 4ull * ((sweep & 1) ? rlo : rhi)) +
-                                    ((sweep & 1) ? -kAhead : kAhead) * (long long)unit;
+            const long long ahead = (long long)(col_off + 4ull * (backward ? rlo : rhi)) +
+                                    (backward ? -kAhead : kAhead) * (long long)unit;
             if (ahead >= (long long)col_off && ahead < (long long)(col_off + 4ull * n_edges)) {
                 m.prefetch((unsigned long long)ahead);
                 if (WEIGHTED) m.prefetch((unsigned long long)ahead - col_off + w_off);
@@ -635,13 +824,15 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
                     pw = m.pin(w_off + 4ull * first, GPUVM_READ, tok_w);
                     if (!pw) { m.release(tok); failed = true; break; }
                 }
+                const unsigned int pos = Op::kBehind ? sweep_pos(counters, n_chunks) : 0u;
                 while (touch) {
                     const int L = __ffs(touch) - 1;
                     touch &= touch - 1;
                     long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
+                    const int bval = __shfl_sync(0xFFFFFFFFu, uval, L);
                     if (blo < first) blo = first;
                     if (bhi > last) bhi = last;
-                    found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, (long long)(v0 + L), blo, bhi, lane);
+                    found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, (long long)(v0 + L), bval, blo, bhi, lane, pos);
                 }
                 if (WEIGHTED) m.release(tok_w);
                 m.release(tok);
@@ -725,7 +916,7 @@ __global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsign
                 const int L = __ffs(touch) - 1;
                 touch &= touch - 1;
                 const long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
-                found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), blo, bhi, lane);
+                found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), op.depth, blo, bhi, lane, 0u);
             }
             m.release(tok);
         }
@@ -742,12 +933,34 @@ __global__ void cc_init_kernel(int *label, unsigned int nv)
     for (unsigned int v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += gridDim.x * blockDim.x) label[v] = (int)v;
 }
 
-__global__ void sssp_init_kernel(int *dist, unsigned char *cur, unsigned int nv, unsigned int source)
+// Every parent becomes its root (= the smallest vertex of its component).  The only stores of this kernel
+// are roots (no path halving here: a halving store that lands after the root was stored would undo it).
+__global__ void cc_finish_kernel(int *parent, unsigned int nv)
 {
+    const CcOp op{parent};
+    for (unsigned int v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += gridDim.x * blockDim.x)
+        parent[v] = op.find_read_only((int)v);
+}
+
+// label-correcting runs: everything unreached and clean, the source at distance 0 and dirty
+__global__ void lc_init_kernel(int *dist, unsigned int nv, unsigned int source)
+{
+    for (unsigned int v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += gridDim.x * blockDim.x)
+        dist[v] = v == source ? 1 : kLcInf;
+}
+
+// packed words back to distances; `unreached` for what was never lowered; the largest distance goes to *max_out
+__global__ void lc_finish_kernel(int *dist, unsigned int nv, int unreached, unsigned int *max_out)
+{
+    int best = 0;
     for (unsigned int v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += gridDim.x * blockDim.x) {
-        dist[v] = v == source ? 0 : 0x7FFFFFFF;
-        cur[v] = v == source;
+        const int w = dist[v];
+        const int d = w >= kLcInf ? unreached : w >> 1;
+        dist[v] = d;
+        if (w < kLcInf && d > best) best = d;
     }
+    for (int o = 16; o; o >>= 1) { const int t = __shfl_down_sync(0xFFFFFFFFu, best, o); best = t > best ? t : best; }
+    if ((threadIdx.x & 31) == 0 && best > 0) atomicMax(max_out, (unsigned int)best);
 }
 
 // ----------------------------------------------------------------- vector add
@@ -1158,11 +1371,18 @@ int run_gather(const Mem &m, size_t x_off, const int64_t *d_idx, size_t n_idx, s
 constexpr int kVaddBlocksPerSm = 4;
 constexpr size_t kBfsScratchBytes = 4 * kBigQueue * sizeof(long long) + kCntWords * sizeof(unsigned int);
 
+// Scratch of the sweeps: queue of pieces, counters, then (label-correcting runs) the queue of vertices
+// lowered behind the sweep position.
+constexpr size_t kBehindMin = 1u << 16;
+size_t behind_capacity(size_t nv) { return nv / 4 > kBehindMin ? nv / 4 : kBehindMin; }
+size_t lc_scratch_bytes(size_t nv) { return kBfsScratchBytes + behind_capacity(nv) * sizeof(unsigned int); }
+
 // One sweep and its update count.  `sweep` counts from 0 within a call.
 template <class Mem, class Op, bool WEIGHTED>
 int graph_sweep(const Mem &m, const Op &op, size_t off_off, size_t col_off, size_t w_off, size_t nv, void *scratch, int sweep,
-                unsigned int *updates, cudaStream_t s)
+                unsigned int *updates, cudaStream_t s, int backward = -1)
 {
+    if (backward < 0) backward = sweep & 1;                  // odd sweeps run downwards
     // number of edges = last row offset; only used to keep prefetches inside the column array
     const unsigned long long n_edges = m.edges_hint;
     long long *span_q = static_cast<long long *>(scratch);
@@ -1171,16 +1391,25 @@ int graph_sweep(const Mem &m, const Op &op, size_t off_off, size_t col_off, size
     const int grid = sm_count() * Mem::kSweepBlocksPerSm;
     if (sweep == 0) cudaMemsetAsync(span_q, 0, 4 * kBigQueue * sizeof(long long), s);     // ready words: once per call
     cudaMemsetAsync(counters, 0, kCntWords * sizeof(unsigned int), s);
-    graph_sweep_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, off_off, col_off, w_off, (unsigned int)nv, n_edges, span_q, counters, sweep);
+    graph_sweep_kernel<Mem, Op, WEIGHTED><<<grid, 256, 0, s>>>(m, op, off_off, col_off, w_off, (unsigned int)nv, n_edges, span_q, counters, sweep, backward);
     int rc = launched(1);
-    unsigned int host_counters[2] = {0, 0};
-    if (cudaMemcpyAsync(host_counters, counters, sizeof(host_counters), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+    static const bool trace = getenv("GPUVM_TRACE_SWEEPS") != nullptr;     // one line per sweep on stderr
+    unsigned int host_counters[kCntWords] = {0};
+    const size_t want = trace ? sizeof(host_counters) : 2 * sizeof(unsigned int);
+    const auto t0 = std::chrono::steady_clock::now();
+    if (cudaMemcpyAsync(host_counters, counters, want, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
         cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+    if (trace)
+        fprintf(stderr, "sweep %d: %.3f ms (host clock, from launch to counters read), updates %u, pieces %u/%u, chunks done %u, "
+                        "behind queued %u taken %u\n", sweep,
+                std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count(), host_counters[kCntUpdates],
+                host_counters[kCntTaken], host_counters[kCntPushed], host_counters[kCntDone], host_counters[kCntBehindTail],
+                host_counters[kCntBehindHead]);
     *updates = host_counters[0];
     return rc;
 }
 
-// One BFS on caller-provided scratch (kBfsScratchBytes, 16-byte aligned).
+// One level-synchronous BFS on caller-provided scratch (kBfsScratchBytes, 16-byte aligned): one sweep per level.
 template <class Mem>
 int bfs_levels(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
                void *scratch, cudaStream_t s)
@@ -1198,15 +1427,52 @@ int bfs_levels(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t s
     return rc;
 }
 
+// Label-correcting sweeps until nothing changes (BFS: unit lengths; SSSP: the weights at w_off).  d_dist holds
+// the packed words while the sweeps run and the distances afterwards.  scratch: lc_scratch_bytes(nv).
+// *max_dist receives the largest distance reached.
+template <class Mem, bool WEIGHTED>
+int lc_sweeps(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source, int32_t *d_dist,
+              int unreached, int *n_sweeps, unsigned int *max_dist, void *scratch, cudaStream_t s)
+{
+    unsigned int *counters = reinterpret_cast<unsigned int *>(static_cast<long long *>(scratch) + 4 * kBigQueue);
+    unsigned int *behind_q = counters + kCntWords;
+    const unsigned int cap = (unsigned int)behind_capacity(nv);
+    lc_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_dist, (unsigned int)nv, (unsigned int)source);
+    int rc = launched();
+    int sweep = 0;
+    unsigned int updates = 1;
+    while (rc == GPUVM_OK && updates > 0) {
+        cudaMemsetAsync(behind_q, 0xFF, (size_t)cap * sizeof(unsigned int), s);
+        // The first sweep expands the source alone.  (A sweep draws its chunks as fast as it can skip them: with
+        // one dirty vertex it would be over before that vertex's neighbours are lowered, and they would all count
+        // as "behind".)  The second one runs upwards again, from the pages the first one left; then they alternate.
+        const int backward = sweep == 0 ? 0 : (sweep - 1) & 1;
+        const LcOp<WEIGHTED> op{d_dist, behind_q, counters, cap, (unsigned int)((nv + 31) / 32), backward,
+                                sweep == 0 ? (unsigned int)source : kNoVertex};
+        rc = graph_sweep<Mem, LcOp<WEIGHTED>, WEIGHTED>(m, op, off_off, col_off, w_off, nv, scratch, sweep, &updates, s, backward);
+        ++sweep;
+    }
+    cudaMemsetAsync(counters + kCntMax, 0, sizeof(unsigned int), s);
+    lc_finish_kernel<<<sm_count() * 4, 256, 0, s>>>(d_dist, (unsigned int)nv, unreached, counters + kCntMax);
+    if (rc == GPUVM_OK) rc = launched(); else launched();
+    unsigned int far = 0;
+    if (cudaMemcpyAsync(&far, counters + kCntMax, sizeof(far), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+    if (max_dist) *max_dist = far;
+    if (n_sweeps) *n_sweeps = sweep;
+    return rc;
+}
+
 template <class Mem>
 int run_bfs(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t source, int32_t *d_level, int *n_levels,
             void *scratch, cudaStream_t s)
 {
-    if (!d_level || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
+    if (!d_level || nv == 0 || source >= nv || nv > 0x3FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
     if (!scratch) return GPUVM_E_ALLOC;
-    int rc = bfs_levels(m, off_off, col_off, nv, source, d_level, n_levels, scratch, s);
-    cudaStreamSynchronize(s);
+    unsigned int far = 0;
+    int rc = lc_sweeps<Mem, false>(m, off_off, col_off, 0, nv, source, d_level, -1, nullptr, &far, scratch, s);
+    if (n_levels) *n_levels = (int)far + 1;               // levels 0 .. far were expanded, the last one found nothing
     return rc;
 }
 
@@ -1250,51 +1516,32 @@ struct Scratch {                     // device scratch for one call, freed on sc
 };
 
 template <class Mem>
-int run_cc(const Mem &m, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, void *scratch_p,
+int run_cc(const Mem &m, size_t off_off, size_t col_off, size_t nv, int32_t *d_label, int *n_sweeps, void *scratch,
            cudaStream_t s)
 {
     if (!d_label || nv == 0 || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16) return GPUVM_E_ALIGN;
-    if (!scratch_p) return GPUVM_E_ALLOC;
-    struct { void *p; } scratch{scratch_p};
+    if (!scratch) return GPUVM_E_ALLOC;
     cc_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
     int rc = launched();
-    int sweep = 0;
-    unsigned int updates = 1;
-    while (rc == GPUVM_OK && updates > 0) {
-        rc = graph_sweep<Mem, CcOp, false>(m, CcOp{d_label}, off_off, col_off, 0, nv, scratch.p, sweep, &updates, s);
-        ++sweep;
-    }
+    unsigned int hooks = 0;
+    if (rc == GPUVM_OK) rc = graph_sweep<Mem, CcOp, false>(m, CcOp{d_label}, off_off, col_off, 0, nv, scratch, 0, &hooks, s);
+    cc_finish_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
+    if (rc == GPUVM_OK) rc = launched(); else launched();
     cudaStreamSynchronize(s);
-    if (n_sweeps) *n_sweeps = sweep;
+    if (n_sweeps) *n_sweeps = 1;
     return rc;
 }
 
 template <class Mem>
 int run_sssp(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source, int32_t *d_dist,
-             int *n_rounds, void *scratch_p, cudaStream_t s)
+             int *n_rounds, void *scratch, cudaStream_t s)
 {
     if (!d_dist || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16 || w_off % 16) return GPUVM_E_ALIGN;
     if ((w_off > col_off ? w_off - col_off : col_off - w_off) % m.unit_host() != 0) return GPUVM_E_ALIGN;
-    if (!scratch_p) return GPUVM_E_ALLOC;          // kBfsScratchBytes + 2 * nv bytes
-    struct { void *p; } scratch{scratch_p};
-    unsigned char *flags = static_cast<unsigned char *>(scratch.p) + kBfsScratchBytes;
-    unsigned char *cur = flags, *next = flags + nv;
-    sssp_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_dist, cur, (unsigned int)nv, (unsigned int)source);
-    int rc = launched();
-    int round = 0;
-    unsigned int updates = 1;
-    while (rc == GPUVM_OK && updates > 0) {
-        cudaMemsetAsync(next, 0, nv, s);
-        rc = graph_sweep<Mem, SsspOp, true>(m, SsspOp{d_dist, cur, next}, off_off, col_off, w_off, nv, scratch.p, round,
-                                            &updates, s);
-        unsigned char *t = cur; cur = next; next = t;
-        ++round;
-    }
-    cudaStreamSynchronize(s);
-    if (n_rounds) *n_rounds = round;
-    return rc;
+    if (!scratch) return GPUVM_E_ALLOC;          // lc_scratch_bytes(nv)
+    return lc_sweeps<Mem, true>(m, off_off, col_off, w_off, nv, source, d_dist, 0x7FFFFFFF, n_rounds, nullptr, scratch, s);
 }
 
 template <class Mem>
@@ -1439,7 +1686,7 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
     hint_edges(h, m, off_off, nv);
-    return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, gpuvm_scratch_(h, kBfsScratchBytes),
+    return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, gpuvm_scratch_(h, lc_scratch_bytes(nv)),
                    static_cast<cudaStream_t>(stream));
 }
 
@@ -1508,7 +1755,7 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
     // column and weight page of an edge range are held together: two frames per warp of the grid
     if (gpuvm_safe_warps(h, 2) < sm_count() * 2 * 8) return GPUVM_E_FRAMES;
     hint_edges(h, m, off_off, nv);
-    return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, gpuvm_scratch_(h, kBfsScratchBytes + 2 * nv),
+    return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, gpuvm_scratch_(h, lc_scratch_bytes(nv)),
                     static_cast<cudaStream_t>(stream));
 }
 
@@ -1667,7 +1914,7 @@ int gpuvm_raw_bfs_csr(const int64_t *row_off, const int32_t *col, size_t nv, siz
     unsigned char *base = ro < co ? ro : co;
     if ((ro - base) % 16 || (co - base) % 16) return GPUVM_E_ALIGN;
     Raw m{base, 65536};
-    Scratch scratch(kBfsScratchBytes);
+    Scratch scratch(lc_scratch_bytes(nv));
     return run_bfs(m, (size_t)(ro - base), (size_t)(co - base), nv, source, d_level, n_levels, scratch.p,
                    static_cast<cudaStream_t>(stream));
 }
@@ -1696,7 +1943,7 @@ int gpuvm_raw_sssp_csr(const int64_t *row_off, const int32_t *col, const int32_t
     RawH m;
     m.base = base;
     m.unit_bytes = 65536;
-    Scratch scratch(kBfsScratchBytes + 2 * nv);
+    Scratch scratch(lc_scratch_bytes(nv));
     return run_sssp(m, (size_t)(ro - base), (size_t)(co - base), (size_t)(we - base), nv, source, d_dist, n_rounds,
                     scratch.p, static_cast<cudaStream_t>(stream));
 }

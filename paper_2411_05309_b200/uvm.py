@@ -38,10 +38,10 @@ def _timed(torch, fn):
     return e0.elapsed_time(e1) / 1e3
 
 
-def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0) -> dict:
-    """Build the workload at shrink + TWIN_SHRINK[cfg], run the paged path (one warm-up, the better
-    of two cold runs: reference outputs and its time at that size), then the same kernels over
-    managed memory."""
+def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0, w=None) -> dict:
+    """Build the workload at shrink + TWIN_SHRINK[cfg] (or take a prepared one of that size, which
+    stays the caller's), run the paged path (one warm-up, the better of two cold runs: reference
+    outputs and its time at that size), then the same kernels over managed memory."""
     import torch
     from . import configs
     if cfg == 2:
@@ -58,7 +58,9 @@ def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0) -> dict:
                     {"read_mostly": True, "units_run": 1048576, "seconds": 25.785, "effective_gbs": 0.000163}]}}
     if cfg not in TWIN_SHRINK:
         return {"unavailable": "no plain-pointer twin of this workload; see workload 3 for BFS over managed memory"}
-    w = configs.make(cfg, shrink + TWIN_SHRINK[cfg])
+    own = w is None or w.shrink != shrink + TWIN_SHRINK[cfg]
+    if own:
+        w = configs.make(cfg, shrink + TWIN_SHRINK[cfg])
     try:
         w.run(check=False)                                   # warm: scratch allocation, first touch of the arena
         ours = min((w.run() for _ in range(2)), key=lambda r: r.seconds)
@@ -85,7 +87,8 @@ def run_twin(cfg: int, shrink: int = 0, timeout_s: float = 120.0) -> dict:
             B.gpuvm_uvm_free(p)
         return out
     finally:
-        w.close()
+        if own:
+            w.close()
 
 
 def _outputs(torch, w, cfg: int) -> dict:

@@ -70,3 +70,24 @@ def test_reference_arm_prints_only_on_rank_zero():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
+
+
+def test_direction_aware_roofline_and_config_record():
+    """Host logic of the benchmark line: the floor of a launch is the slower direction of the link,
+    both arms describe the configuration with the same keys, and every ncu figure the line quotes
+    names a summary that is in the tree."""
+    import os
+    import bench
+    link = {"ce_h2d_gbs": 50.0, "ce_d2h_gbs": 60.0, "sm_h2d_gbs": 48.0, "sm_d2h_gbs": 52.0}
+    r = bench.link_roofline(8e9, 4e9, 0.2, link)                  # 8 GB in, 4 GB out in 200 ms
+    assert r["direction"] == "host_to_device" and abs(r["floor_ms"] - 160.0) < 1e-9
+    assert abs(r["frac"] - 0.8) < 1e-12 and abs(r["achieved"] - 40.0) < 1e-9 and r["peak"] == 50.0
+    r = bench.link_roofline(1e9, 6e9, 0.2, link)
+    assert r["direction"] == "device_to_host" and abs(r["frac"] - 0.5) < 1e-12
+    a, b = bench.config_of(5, 0), bench.config_of(5, 0)
+    assert a == b and a["cfg"] == 5 and a["pool_bytes"] == 16 << 30 and a["page_bytes"] == 2 << 20
+    assert bench.config_of(3, 0)["frames"] == 9216
+    root = os.path.dirname(os.path.abspath(bench.__file__))
+    for cfg, (nbytes, name, how) in bench.NCU_LINK_TRAFFIC.items():
+        text = open(os.path.join(root, "profiles", name)).read().replace(" ", "").replace(",", "")
+        assert str(nbytes // 32) in text, (cfg, name)             # the sector count is in the committed summary
