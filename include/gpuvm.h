@@ -78,7 +78,8 @@ typedef struct gpuvm_dev {
     unsigned int policy;       /* GPUVM_POLICY_*                                        */
     unsigned int spin_limit_us;/* upper bound of every device-side wait                 */
     unsigned int debug;        /* GPUVM_DEBUG_* flags                                   */
-    unsigned int reserved;
+    unsigned int clean_ahead;  /* ring positions the cleaners may run ahead of the head
+                                  cursor; 0: write-back only on the fault path          */
 } gpuvm_dev_t;
 
 /* Debug flags (gpuvm_set_debug).  POISON: whoever evicts a page fills its frame with the
@@ -97,13 +98,16 @@ typedef struct gpuvm_stats {
     uint64_t lanes_coalesced; /* threads that shared their warp leader's request
                                  (intra-warp coalescing)                               */
     uint64_t evictions;       /* pages unmapped to make room                           */
-    uint64_t writebacks;      /* dirty victims copied pool -> host while running       */
+    uint64_t writebacks;      /* dirty victims copied pool -> host by the warp that
+                                 needed their frame (on the fault path)               */
     uint64_t flush_writebacks;/* dirty pages copied by gpuvm_flush                     */
     uint64_t bytes_in;        /* host -> pool bytes                                    */
     uint64_t bytes_out;       /* pool -> host bytes (evictions + flush)                */
     uint64_t hand_steps;      /* frame-ring slots inspected                            */
     uint64_t retries;         /* wait-loop rounds that made no progress                */
     uint64_t resident;        /* pages resident now                                    */
+    uint64_t cleaned;         /* dirty pages written back off the fault path, by idle
+                                 warps, while they stayed resident                    */
     uint64_t ring_drops;      /* entries of a fault ring that were given up on after a
                                  bounded wait (slot never filled, slot never cleared, or
                                  a popped page that was not waiting for a migrator): each
@@ -192,6 +196,18 @@ int gpuvm_check_on(gpuvm_t h, gpuvm_check_t *out, void *stream);
 int gpuvm_set_policy(gpuvm_t h, int policy);
 int gpuvm_set_spin_limit_us(gpuvm_t h, unsigned int spin_limit_us);
 int gpuvm_set_debug(gpuvm_t h, unsigned int flags);   /* GPUVM_DEBUG_*; 0 = off (default) */
+
+/* Write-back off the fault path (Section 5.3 names synchronous write-back as the method's weak spot):
+ * warps with nothing to do write back dirty pages that lie up to `frames` ring positions ahead of the
+ * head cursor and would be its victims, so that the warp that takes the frame does not have to.  The
+ * order of eviction is unchanged.  What it costs: a page that is written to again between its early
+ * write-back and its eviction is written back twice.  Off by default (frames = 0): with thousands of
+ * warps faulting at once, the write-backs of some overlap the fetches of others and both directions
+ * of the link are busy anyway; measured on scattered updates over a thrashing pool it moved two thirds
+ * of the write-backs off the fault path and made the run no faster (requesters migrate their own
+ * pages) or slower by half (migrator warps: the extra write-backs take link time from the fetches).
+ * A setting for workloads whose dirty pages are written once and whose faulting warps are few. */
+int gpuvm_set_clean_ahead(gpuvm_t h, unsigned int frames);
 
 /* Device scratch of the batched workload entry points (request tables, staging of gathered
  * rows; not pages of the backing store).  It belongs to the handle, is allocated at the first

@@ -227,6 +227,9 @@ static __device__ __noinline__ void gpuvm_migrator_loop(const gpuvm_dev_t vm, gp
         }
         item = __shfl_sync(0xFFFFFFFFu, item, 0);
         if (item == 0u) {
+            /* no fault to serve: write back a dirty page that is about to become a victim, so that whoever needs a
+             * frame next gets it without a write-back */
+            if (clean_ahead(vm, 0xFFFFFFFFu, lane, 32, lane == 0)) { idle_ns = 32; continue; }
             const unsigned int done = (lane == 0) ? (unsigned int)(*vr == 0u && *vh == *vt &&
                                                                    (!q->shared || ld_relaxed_u32(&q->shared->head) ==
                                                                                       ld_relaxed_u32(&q->shared->tail))) : 0u;
@@ -597,6 +600,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
             break;
         }
         if (lane == 0) stat_add(vm, kRetries, 1);
+        if (clean_ahead(vm, 0xFFFFFFFFu, lane, 32, lane == 0)) continue;   /* idle: write back a page that is about to be a victim */
         __nanosleep(sleep_ns);
         if (sleep_ns < 4096) sleep_ns *= 2;
     }

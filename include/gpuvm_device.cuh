@@ -93,9 +93,10 @@ constexpr int kCtlErr = 1;
 constexpr int kCtlErrPage = 2;
 constexpr int kCtlCounters = 16;      /* kStatSlots slots of 16 words, one 128-byte line each */
 constexpr int kStatSlots = 32;
-constexpr int kCtlWords = kCtlCounters + kStatSlots * 16;
+constexpr int kCtlCleanCursor = kCtlCounters + kStatSlots * 16;   /* ring position of the cleaners (a line of its own) */
+constexpr int kCtlWords = kCtlCleanCursor + 16;
 enum Stat { kFaults = 0, kHits, kWaits, kLanes, kEvictions, kWritebacks, kFlushWritebacks,
-            kBytesIn, kBytesOut, kHandSteps, kRetries, kRingDrops, kNumStats };
+            kBytesIn, kBytesOut, kHandSteps, kRetries, kRingDrops, kCleaned, kNumStats };
 
 enum Mode { kRead = 0, kWrite = 1, kWriteAll = 2 };
 
@@ -452,7 +453,7 @@ __device__ __forceinline__ int advance(const gpuvm_dev_t &vm, unsigned long long
  */
 __device__ __forceinline__ bool try_claim(const gpuvm_dev_t &vm, unsigned long long vpn,
                                           int tries, unsigned int &frame,
-                                          unsigned long long &victim, bool &victim_dirty)
+                                          unsigned long long &victim, bool &victim_dirty, bool allow_dirty = true)
 {
     for (int t = 0; t < tries; ++t) {
         unsigned long long ticket = atomicAdd(vm.ctl + kCtlHand, 1ull);
@@ -476,6 +477,7 @@ __device__ __forceinline__ bool try_claim(const gpuvm_dev_t &vm, unsigned long l
             atomicAnd(qpte, ~kRef);                         /* second chance */
             continue;
         }
+        if ((w & kDirty) && !allow_dirty) continue;         /* a prefetch does not pay for a write-back */
         unsigned long long evicting = (w & ~(kStMask | kRef)) | kEvicting;
         if (atomicCAS(qpte, w, evicting) != w) continue;    /* lost against a pin or another evictor */
         st_relaxed_u32(vm.frame_vpn + h, kFrameLock | (unsigned int)vpn);
@@ -485,6 +487,69 @@ __device__ __forceinline__ bool try_claim(const gpuvm_dev_t &vm, unsigned long l
     }
     stat_add(vm, kHandSteps, tries);
     return false;
+}
+
+/*
+ * Write-back off the fault path (the paper names synchronous write-back by the faulting thread as
+ * its weak spot, Section 5.3, and eviction work inside the fault handler as the cause of the step at
+ * oversubscription level 1, Section 5.4).  The frame ring has a second cursor that runs ahead of the
+ * head cursor: warps with nothing to do -- a migrator warp whose fault ring is empty, a warp that
+ * waits for somebody else's fault -- take the next ring position from it, and if the page in that
+ * frame would be the head cursor's victim when it gets there (resident, nobody holds it, not
+ * referenced since its last chance, dirty) they write it back now.  One compare-and-swap on the
+ * exact entry takes a reference and clears the dirty bit: all earlier writers have released the page,
+ * and any later writer marks it dirty again.  Copy, system fence, drop the reference: the page stays
+ * resident, and when the head cursor arrives its frame is handed on without a write-back.  The order
+ * in which frames are claimed is untouched, so no fault is added; pages written back early and
+ * written to again before they are evicted cost one more write-back.  Nothing depends on the
+ * cleaners: a victim that is still dirty is written back by the warp that takes its frame, as before.
+ */
+/*
+ * The `n` calling lanes (rank 0..n-1, all of `mask`, converged; `is_L` on the lowest of them): look
+ * at the next ring position ahead of the head cursor and write its page back if it qualifies.
+ * Returns true when a page was written back.
+ */
+static __device__ __noinline__ bool clean_ahead(const gpuvm_dev_t vm, unsigned int mask, unsigned int rank, unsigned int n,
+                                                bool is_L)
+{
+    if (vm.clean_ahead == 0u) return false;
+    const unsigned int L = __ffs(mask) - 1;
+    unsigned int f = kFrameFree, e = kFrameFree;
+    if (is_L) {
+        const unsigned long long hand = ld_relaxed_u64(vm.ctl + kCtlHand);
+        unsigned long long c = ld_relaxed_u64(vm.ctl + kCtlCleanCursor);
+        const unsigned long long ahead = vm.clean_ahead;
+        const unsigned long long pos = c < hand ? hand : c;              /* the head cursor has overtaken: start from it */
+        if (hand >= vm.n_frames && pos < hand + ahead &&                 /* (a ring that has not filled once evicts nothing) */
+            atomicCAS(vm.ctl + kCtlCleanCursor, c, pos + 1ull) == c) {
+            f = (unsigned int)(pos % vm.n_frames);
+            e = ld_relaxed_u32(vm.frame_vpn + f);
+            if (e != kFrameFree && !(e & kFrameLock) && e < vm.n_pages) {
+                const unsigned long long w = ld_relaxed_u64(vm.pte + e);
+                const bool fits = (w & kStMask) == kValid && (w & kRcMask) == 0ull && (w & kDirty) &&
+                                  !(vm.policy == GPUVM_POLICY_CLOCK && (w & kRef)) &&
+                                  (unsigned int)((w & kFrameMask) >> kFrameShift) == f;
+                if (!fits || atomicCAS(vm.pte + e, w, (w & ~kDirty) + 1ull) != w) e = kFrameFree;
+            } else {
+                e = kFrameFree;
+            }
+        }
+    }
+    f = __shfl_sync(mask, f, L);
+    e = __shfl_sync(mask, e, L);
+    if (e == kFrameFree) return false;
+    __threadfence();                                          /* acquire side of the writers' releases */
+    const unsigned int len = page_len(vm, e);
+    warp_copy<8, true>(vm.host + ((unsigned long long)e << vm.page_shift), vm.pool + ((unsigned long long)f << vm.page_shift),
+                       len >> 4, rank, n);
+    __threadfence_system();
+    __syncwarp(mask);
+    if (is_L) {
+        unpin(vm.pte + e);
+        stat_add(vm, kCleaned, 1);
+        stat_add(vm, kBytesOut, len);
+    }
+    return true;
 }
 
 /*
@@ -602,6 +667,8 @@ static __device__ __noinline__ bool slow_path(const gpuvm_dev_t vm, unsigned lon
             continue;                                        /* READY groups still finish */
         }
         if (lane == (unsigned int)(__ffs(active) - 1)) stat_add(vm, kRetries, 1);
+        /* nothing to do but wait: write back a dirty page that is about to become a victim, if there is one */
+        if (clean_ahead(vm, active, rank, nlanes, lane == (unsigned int)(__ffs(active) - 1))) continue;
         __nanosleep(sleep_ns);
         if (sleep_ns < 2048) sleep_ns *= 2;
     }
@@ -831,7 +898,7 @@ static __device__ __noinline__ void gpuvm_prefetch(const gpuvm_dev_t vm, unsigne
     if (lane == L) {
         const unsigned long long w = ld_relaxed_u64(pte);
         if ((w & kStMask) == kInvalid && atomicCAS(pte, w, w | kBusy) == w) {
-            go = try_claim(vm, vpn, 8, h, victim, vdirty) ? 1 : 0;
+            go = try_claim(vm, vpn, 8, h, victim, vdirty, /* allow_dirty = */ false) ? 1 : 0;
             if (!go) atomicXor(pte, kBusy);                       /* no frame at hand: BUSY -> INVALID */
         }
     }

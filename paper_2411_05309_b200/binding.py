@@ -32,13 +32,13 @@ class DevView(ctypes.Structure):
                 ("host", ctypes.c_void_p), ("ctl", ctypes.c_void_p), ("bytes", ctypes.c_uint64),
                 ("n_pages", ctypes.c_uint64), ("n_frames", ctypes.c_uint32), ("page_shift", ctypes.c_uint32),
                 ("policy", ctypes.c_uint32), ("spin_limit_us", ctypes.c_uint32), ("debug", ctypes.c_uint32),
-                ("reserved", ctypes.c_uint32)]
+                ("clean_ahead", ctypes.c_uint32)]
 
 
 class Stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in
                 ("faults", "hits", "waits", "lanes_coalesced", "evictions", "writebacks", "flush_writebacks",
-                 "bytes_in", "bytes_out", "hand_steps", "retries", "resident", "ring_drops")] + \
+                 "bytes_in", "bytes_out", "hand_steps", "retries", "resident", "cleaned", "ring_drops")] + \
                [("error", ctypes.c_int32), ("reserved", ctypes.c_uint32), ("error_page", ctypes.c_uint64)]
 
     def as_dict(self):
@@ -63,6 +63,7 @@ SYMBOLS = {
     "gpuvm_reset_on": (_i, [_vp, _vp]),
     "gpuvm_check_on": (_i, [_vp, ctypes.POINTER(Check), _vp]),
     "gpuvm_set_debug": (_i, [_vp, ctypes.c_uint]),
+    "gpuvm_set_clean_ahead": (_i, [_vp, ctypes.c_uint]),
     "gpuvm_bcsr_build": (_i, [_vp, _sz, _sz, _vp, _sz, ctypes.POINTER(_sz)]),
     "gpuvm_device_view": (_i, [_vp, ctypes.POINTER(DevView)]),
     "gpuvm_host_ptr": (_vp, [_vp]),
@@ -199,6 +200,10 @@ def gpuvm_check_on(h, stream, raise_on_error: bool = True) -> dict:
     d = c.as_dict()
     d["status"] = rc
     return d
+
+
+def gpuvm_set_clean_ahead(h, frames: int):
+    _check(lib().gpuvm_set_clean_ahead(h, frames), "gpuvm_set_clean_ahead")
 
 
 def gpuvm_set_debug(h, flags: int):

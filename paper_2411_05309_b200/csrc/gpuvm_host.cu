@@ -186,6 +186,7 @@ int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_byt
     d.n_frames = (unsigned int)(pool_bytes / page_bytes);
     d.policy = GPUVM_POLICY_CLOCK;
     d.spin_limit_us = 10u * 1000u * 1000u;
+    d.clean_ahead = 0;                              // write-back off the fault path is opt-in: gpuvm_set_clean_ahead
 
     bool ok = cudaMalloc(&d.pte, d.n_pages * sizeof(unsigned long long)) == cudaSuccess &&
               cudaMalloc(&d.frame_vpn, d.n_frames * sizeof(unsigned int)) == cudaSuccess &&
@@ -294,6 +295,7 @@ int gpuvm_stats_on(gpuvm_t h, gpuvm_stats_t *out, void *stream)
     out->bytes_in = sum[kBytesIn]; out->bytes_out = sum[kBytesOut];
     out->hand_steps = sum[kHandSteps]; out->retries = sum[kRetries];
     out->ring_drops = sum[kRingDrops];
+    out->cleaned = sum[kCleaned];
     out->resident = out->faults - out->evictions;
     out->error = (int32_t)(long long)local[kCtlErr];
     out->error_page = local[kCtlErrPage];
@@ -352,6 +354,13 @@ int gpuvm_set_debug(gpuvm_t h, unsigned int flags)
 {
     if (!h || (flags & ~(unsigned int)GPUVM_DEBUG_POISON)) return GPUVM_E_ARG;
     h->dev.debug = flags;
+    return GPUVM_OK;
+}
+
+int gpuvm_set_clean_ahead(gpuvm_t h, unsigned int frames)
+{
+    if (!h) return GPUVM_E_ARG;
+    h->dev.clean_ahead = frames < h->dev.n_frames ? frames : h->dev.n_frames;
     return GPUVM_OK;
 }
 

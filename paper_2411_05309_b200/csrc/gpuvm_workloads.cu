@@ -1545,7 +1545,8 @@ int run_sssp(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t 
 }
 
 template <class Mem>
-int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, bool hold_c, int blocks, cudaStream_t s)
+int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, bool hold_c, int blocks, int threads,
+             cudaStream_t s)
 {
     unsigned long long unit = 0;
     if (n % 4) return GPUVM_E_ALIGN;
@@ -1555,9 +1556,9 @@ int run_vadd(const Mem &m, size_t a_off, size_t b_off, size_t c_off, size_t n, b
     if (chunk < 512) return GPUVM_E_PAGE;             // a warp moves 512 bytes per instruction
     if (a_off % chunk || b_off % chunk || c_off % chunk) return GPUVM_E_ALIGN;
     if (hold_c && c_off % unit == 0)
-        vadd_kernel<Mem, true><<<blocks, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
+        vadd_kernel<Mem, true><<<blocks, threads, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
     else
-        vadd_kernel<Mem, false><<<blocks, 256, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
+        vadd_kernel<Mem, false><<<blocks, threads, 0, s>>>(m, a_off, b_off, c_off, n, chunk);
     return launched();
 }
 
@@ -1763,11 +1764,6 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
 {
     PagedH m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
-    // Two pages per warp are held at once on the no-fetch path: only when the pool can take it.  A small
-    // pool gets a smaller grid first (down to one thread block per SM, which is what is resident at
-    // this kernel's register count anyway) before the kernel falls back to one page at a time.
-    int blocks = sm_count() * kVaddBlocksPerSm;
-    while (blocks > sm_count() && gpuvm_safe_warps(h, 2) < blocks * 8) blocks -= sm_count();
     // c may be a or b itself (in place): every chunk is then read before it is written, by the same
     // warp, one page at a time; the no-fetch path is out, because it hands out the page of c without
     // its contents.  Any other overlap of c with an input has no defined result.
@@ -1775,8 +1771,16 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
     auto overlaps = [len](size_t x, size_t y) { return x < y + len && y < x + len; };
     const bool in_place = c_off == a_off || c_off == b_off;
     if ((c_off != a_off && overlaps(c_off, a_off)) || (c_off != b_off && overlaps(c_off, b_off))) return GPUVM_E_ARG;
-    const bool hold_c = !in_place && gpuvm_safe_warps(h, 2) >= blocks * 8;
-    return run_vadd(m, a_off, b_off, c_off, n, hold_c, blocks, static_cast<cudaStream_t>(stream));
+    // The grid is sized to the pool: a warp works on three pages at a time (it holds the page of c, or comes
+    // back to it, and comes back to its pages of a and b chunk by chunk).  More warps than that would evict
+    // one another's pages between chunks and fetch every page many times (measured: 13 times); the link
+    // is full from a few dozen migrating warps anyway, so a small pool costs warps, not bandwidth.
+    const int safe = gpuvm_safe_warps(h, 4);                // three pages in rotation and one to spare for the ring's slack
+    int blocks = sm_count() * kVaddBlocksPerSm, threads = 256;
+    if (safe >= 8) blocks = blocks < safe / 8 ? blocks : safe / 8;
+    else { blocks = 1; threads = 32 * (safe > 0 ? safe : 1); }
+    const bool hold_c = !in_place && gpuvm_safe_warps(h, 2) >= 1;
+    return run_vadd(m, a_off, b_off, c_off, n, hold_c, blocks, threads, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,
@@ -1958,7 +1962,7 @@ int gpuvm_raw_vadd_f32(const float *a, const float *b, float *c, size_t n, void 
     RawH m;
     m.base = base;
     m.unit_bytes = 65536;
-    return run_vadd(m, (size_t)(pa - base), (size_t)(pb - base), (size_t)(pc - base), n, false, sm_count() * kVaddBlocksPerSm, static_cast<cudaStream_t>(stream));
+    return run_vadd(m, (size_t)(pa - base), (size_t)(pb - base), (size_t)(pc - base), n, false, sm_count() * kVaddBlocksPerSm, 256, static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_raw_embag_f32(const float *table, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag, float *d_out,

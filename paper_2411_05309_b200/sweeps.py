@@ -6,6 +6,7 @@ oversubscription analysis), printed as JSON lines.
     python -m paper_2411_05309_b200.sweeps resident
     python -m paper_2411_05309_b200.sweeps oversub [--workload 1|2|3|4] [--shrink S]
     python -m paper_2411_05309_b200.sweeps depth   [--workload 2|5] [--shrink S]
+    python -m paper_2411_05309_b200.sweeps writeback
 
 pages   -- Section 5.1 / Fig. 7: move a fixed amount of host memory into the pool with one
            warp per page, consecutive pages, for page sizes from 4 KiB to 2 MiB; reports the
@@ -23,6 +24,11 @@ oversub -- Section 5.4 / Fig. 14 with Eq. 1: run a workload with the pool shrunk
 depth   -- Section 3.2 (queue depth by Little's law) carried over to page requests: the batched
            workloads under a growing bound of their device scratch, i.e. with more and more page
            requests registered per warp; reports scratch bytes, faults and time.
+writeback -- Section 5.3 (vector add: synchronous write-back named as the weak spot) and Section 5.4
+           (eviction adds to the fault latency): workloads whose victims are dirty, at pools of all,
+           a quarter and a twelfth of the data: the scattered read-modify-write in its three forms and
+           the vector add on a pool too small for its no-fetch path; reports time, faults, write-backs
+           on and off the fault path, and both directions of the link.
 """
 from __future__ import annotations
 
@@ -180,9 +186,71 @@ def sweep_depth(cfg: int, shrink: int):
             w.close()
 
 
+def sweep_writeback():
+    import torch
+    from . import binding as B
+    from . import configs
+    n, n_upd, page = 1 << 28, 1 << 24, 65536
+    host = torch.zeros(n, dtype=torch.int32).pin_memory()
+    idx = torch.randperm(n, device="cuda")[:n_upd].contiguous()
+    forms = (("scatter, one access per lane", B.gpuvm_scatter_update_u32),
+             ("scatter, batched, requester migrates", B.gpuvm_scatter_update_u32_batched),
+             ("scatter, batched, migrator warps", B.gpuvm_scatter_update_u32_queued))
+
+    def record(name, extra, t, st):
+        print(json.dumps({"sweep": "writeback", "workload": name, **extra, "seconds": t, "faults": st["faults"],
+                          "writebacks_on_fault_path": st["writebacks"], "writebacks_by_cleaners": st["cleaned"],
+                          "flush_writebacks": st["flush_writebacks"], "in_gbs": st["bytes_in"] / t / 1e9,
+                          "out_gbs": st["bytes_out"] / t / 1e9}), flush=True)
+
+    for frac in (1, 4, 12):
+        pool = (4 * n // frac) // page * page
+        h = B.gpuvm_create(host.data_ptr(), 4 * n, page, pool)
+        try:
+            for name, fn in forms[1:] if frac > 1 else forms:       # (one access per lane thrashes for 15-20 s at small pools)
+                for ahead in (0, None):
+                    if ahead is not None:
+                        B.gpuvm_set_clean_ahead(h, ahead)
+                    else:
+                        B.gpuvm_set_clean_ahead(h, min(pool // page // 32, 128))
+                    best = None
+                    for r in range(3):
+                        B.gpuvm_reset(h)
+                        t = _time(torch, lambda: (fn(h, 0, idx, n_upd), B.gpuvm_flush(h, torch.cuda.current_stream())))
+                        st = B.gpuvm_stats(h)
+                        assert B.gpuvm_check(h)["status"] == 0
+                        if r and (best is None or t < best[0]):
+                            best = (t, st)
+                    record(name, {"pool_fraction": f"1/{frac}", "page_bytes": page,
+                                  "clean_ahead": B.gpuvm_device_view(h).clean_ahead}, *best)
+        finally:
+            B.gpuvm_destroy(h)
+    del host, idx
+    torch.cuda.empty_cache()
+    # vector add on small pools: out of place (the page of c is held, not fetched, and written back by its
+    # producer) and in place (c = a: pages of a are read, written and left dirty: the case for the cleaners)
+    for frames in (2048, 256):
+        for in_place in (False, True):
+            for ahead in (0, None):
+                w = configs.WORKLOADS[4](2)                          # three 1 GiB arrays
+                w.pool_override = frames * 65536
+                w.setup()
+                try:
+                    if ahead is not None:
+                        B.gpuvm_set_clean_ahead(w.h, ahead)
+                    if in_place:
+                        w.launch = lambda stream, w=w: B.gpuvm_vadd_f32(w.h, w.off["a"], w.off["b"], w.off["a"], w.n, stream)
+                    w.run(check=False)
+                    res = min((w.run() for _ in range(3)), key=lambda r: r.seconds)
+                    record("vector add in place" if in_place else "vector add", {"frames": frames, "pool_bytes": w.pool_bytes,
+                           "clean_ahead": B.gpuvm_device_view(w.h).clean_ahead}, res.seconds, res.stats)
+                finally:
+                    w.close()
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("which", choices=["pages", "warps", "resident", "oversub", "depth"])
+    ap.add_argument("which", choices=["pages", "warps", "resident", "oversub", "depth", "writeback"])
     ap.add_argument("--gib", type=float, default=4.0)
     ap.add_argument("--warps-per-sm", type=int, default=16)
     ap.add_argument("--workload", type=int, default=1)
@@ -194,6 +262,8 @@ def main(argv=None):
         sweep_resident()
     elif a.which == "warps":
         sweep_warps(min(a.gib, 2.0))
+    elif a.which == "writeback":
+        sweep_writeback()
     elif a.which == "depth":
         sweep_depth(a.workload if a.workload in (2, 5) else 2, a.shrink)
     else:

@@ -48,6 +48,8 @@ def test_random_mix_of_workloads_on_one_handle(B):
         with paged(ar.host, page, frames, policy) as h:
             if case & 1:                                               # every other case with frames poisoned on eviction
                 B.gpuvm_set_debug(h, B.DEBUG_POISON)
+            if case % 3 == 0:                                          # every third with write-back off the fault path
+                B.gpuvm_set_clean_ahead(h, max(1, frames // 4))
             for step in range(int(rng.integers(2, 6))):
                 kind = int(rng.integers(0, 5))
                 if kind in (0, 1):                                     # scattered updates of distinct elements
