@@ -333,8 +333,10 @@ constexpr unsigned int GPUVM_BATCH_ROWS_MAX = 1u << 16;
 #define GPUVM_BATCH_ACQ 1
 #endif
 #ifndef GPUVM_BATCH_ROWS_AT_ONCE
-#define GPUVM_BATCH_ROWS_AT_ONCE 4     /* 1, 2, 4 or 8: rows whose memory accesses are issued together */
+#define GPUVM_BATCH_ROWS_AT_ONCE 2     /* 1, 2, 4 or 8: rows whose memory accesses are issued together (2: no spills to speak
+                                          of at 64 registers; 4 spilled ten times as much for the same speed, 8 was slower) */
 #endif
+
 
 __host__ __device__ __forceinline__ unsigned int gpuvm_batch_mask_words(unsigned int n)
 {
@@ -367,168 +369,162 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
     unsigned int n_hits = 0, n_waits = 0, n_lanes = 0;      /* this lane's share of the counters, added up at the end */
     constexpr int R = GPUVM_BATCH_ROWS_AT_ONCE;
 
-    /* Register the requests of 64 rows in the page table (steps 1-4 of the access path); a
-     * fault this lane comes to own goes to the migrators at once when there is a ring.  The
-     * pin is a relaxed add: nothing is read from a frame before the acquire load of a visit. */
-    auto register_word = [&](unsigned int k) {
-        unsigned long long todo = 0, own = 0;
-        const unsigned int jn = rows - 64u * k < 64u ? rows - 64u * k : 64u;
-        for (unsigned int j0 = 0; j0 < jn; j0 += R) {          /* R rows at a time: their loads and atomics overlap */
-            unsigned int vpn[R], m[R];
-            unsigned long long old[R];
-            bool active[R], leads[R];
+    /*
+     * R rows of word k, starting at row j0 of the word.  first: the requests are registered in the page
+     * table (steps 1-4 of the access path: grouped, pinned by their leader, hit / wait / own); otherwise
+     * the unfinished ones are looked at again.  Either way every group whose page is there is consumed
+     * and released on the spot, so a request that hits costs one visit and one pin / unpin pair.
+     * The R rows' table entries, page-table accesses and frame loads are issued together.
+     * Returns true when something moved.
+     */
+    auto visit = [&](unsigned int k, unsigned int j0, unsigned int jn, bool first, unsigned long long &todo,
+                     unsigned long long &own) -> bool {
+        unsigned int rowmask[R], vpn[R], off[R], leader[R], any = 0;
+        unsigned long long word[R];
+        bool progress = false;
 #pragma unroll
-            for (int u = 0; u < R; ++u) {
+        for (int u = 0; u < R; ++u) {
+            const unsigned int i = (64u * k + j0 + u) * 32 + lane;
+            const bool mine = j0 + u < jn && (first ? (i < n && table.valid(i)) : ((todo >> (j0 + u)) & 1ull) != 0);
+            rowmask[u] = __ballot_sync(0xFFFFFFFFu, mine);
+            any |= rowmask[u];
+        }
+        if (!any) return false;
+#pragma unroll
+        for (int u = 0; u < R; ++u) {
+            vpn[u] = 0; off[u] = 0;
+            if ((rowmask[u] >> lane) & 1u) {
                 const unsigned int i = (64u * k + j0 + u) * 32 + lane;
-                active[u] = j0 + u < jn && i < n && table.valid(i);
-                vpn[u] = active[u] ? table.vpn(i) : 0u;
+                vpn[u] = table.vpn(i);
+                off[u] = table.off(i);
+                if (first) todo |= 1ull << (j0 + u);
             }
+        }
 #pragma unroll
-            for (int u = 0; u < R; ++u) m[u] = __ballot_sync(0xFFFFFFFFu, active[u]);
-#pragma unroll
-            for (int u = 0; u < R; ++u) {
-                leads[u] = false;
-                old[u] = 0;
-                if (active[u]) {
-                    const unsigned int group = __match_any_sync(m[u], vpn[u]);
-                    leads[u] = lane == (unsigned int)(__ffs(group) - 1);
-                    if (leads[u]) {
-                        old[u] = atomicAdd(vm.pte + vpn[u], 1ull);
+        for (int u = 0; u < R; ++u) {
+            leader[u] = 32; word[u] = 0;
+            if ((rowmask[u] >> lane) & 1u) {
+                const unsigned int group = __match_any_sync(rowmask[u], vpn[u]);
+                leader[u] = __ffs(group) - 1;
+                if (lane == leader[u]) {
+                    if (first) {
+                        word[u] = pin_acquire(vm.pte + vpn[u]) + 1ull;
                         /* far too many references to one page: the sticky error ends every wait of the
                          * launch at its next idle round, long before the counter could carry */
-                        if ((old[u] & kRcMask) >= kRcLimit) set_error(vm, GPUVM_E_PINS, vpn[u]);
+                        if ((word[u] & kRcMask) > kRcLimit) set_error(vm, GPUVM_E_PINS, vpn[u]);
                         n_lanes += __popc(group) - 1;
+                    } else if (!((own >> (j0 + u)) & 1ull)) {
+                        word[u] = ld_relaxed_u64(vm.pte + vpn[u]);
                     }
-                    todo |= 1ull << (j0 + u);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < R; ++u) {
-                if (leads[u]) {
-                    unsigned int frame;
-                    const int st = advance(vm, vm.pte + vpn[u], old[u] + 1ull, mode, frame);
-                    if (st == kReady) ++n_hits;
-                    else if (st == kWait) ++n_waits;
-                    else if (!(eager_push && queue && fault_queue_push(queue, vpn[u], mode, &vm))) own |= 1ull << (j0 + u);
                 }
             }
         }
-        m_todo[(size_t)k * mask_stride] = todo;
-        m_own[(size_t)k * mask_stride] = own;
-        __syncwarp();
+        /* leaders: what the entries say.  A pin is an acquire; on a later visit an entry that looks VALID is
+         * read again with acquire (either pairs with the fence before the publish); a VALID that turns up
+         * any other way gets a fence. */
+        unsigned int frame[R];
+        bool need_fence = false;
+#pragma unroll
+        for (int u = 0; u < R; ++u) {
+            frame[u] = kNotReady;
+            const unsigned long long bit = 1ull << (j0 + u);
+            if (lane == leader[u] && (first || !(own & bit))) {
+                unsigned long long w = word[u];
+                const bool looks_valid = (w & kStMask) == kValid;
+                if (!first && GPUVM_BATCH_ACQ == 1 && looks_valid) w = ld_acquire_u64(vm.pte + vpn[u]);
+                unsigned int f;
+                const int st = advance(vm, vm.pte + vpn[u], w, mode, f);
+                if (st == kReady) {
+                    frame[u] = f;
+                    need_fence |= GPUVM_BATCH_ACQ == 2 || (GPUVM_BATCH_ACQ == 1 && !looks_valid);
+                    if (first) ++n_hits;
+                } else if (st == kOwn) {
+                    if (!(first && eager_push && queue && fault_queue_push(queue, vpn[u], mode, &vm))) own |= bit;
+                    progress = true;
+                } else if (first) {
+                    ++n_waits;
+                }
+            }
+        }
+        if (__any_sync(0xFFFFFFFFu, need_fence)) __threadfence();
+        /* followers take the frame from their leader; every ready request is consumed */
+        bool any_ready = false;
+        unsigned int dep = 0;          /* what consume returned, folded: see below */
+#pragma unroll
+        for (int u = 0; u < R; ++u) {
+            if (!rowmask[u]) continue;
+            const bool mine = ((rowmask[u] >> lane) & 1u) != 0;
+            if (mine) frame[u] = __shfl_sync(rowmask[u], frame[u], leader[u]);
+            const bool ready = mine && frame[u] != kNotReady;
+            if (WARP_CONSUME) {
+                unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
+                while (ready_lanes) {
+                    const unsigned int L = __ffs(ready_lanes) - 1;
+                    ready_lanes &= ready_lanes - 1;
+                    const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame[u], L), o = __shfl_sync(0xFFFFFFFFu, off[u], L);
+                    call_consume(consume, (64u * k + j0 + u) * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o, dep);
+                }
+            } else if (ready) {
+                call_consume(consume, (64u * k + j0 + u) * 32 + lane,
+                             vm.pool + ((unsigned long long)frame[u] << vm.page_shift) + off[u], dep);
+            }
+            any_ready |= ready;
+        }
+        /* step 8 for all of them.  The decrements must not overtake the groups' accesses
+         * to their frames.  A consume that only reads and returns (something computed
+         * from) what it read gives the engine a value that does not exist before the
+         * loads have returned: `hold` below is zero, but it is computed from those values
+         * of all 32 lanes, so the decrement that adds it cannot be issued earlier (this leans on
+         * the hardware executing a dependent instruction after its operands exist; the PTX memory
+         * model by itself does not order a relaxed atomic after earlier loads).  Any
+         * other consume, and write mode, get a warp barrier and a fence instead. */
+        if (__any_sync(0xFFFFFFFFu, any_ready)) {
+            unsigned long long hold = 0;
+            if (kConsumeReturns && mode == kRead) {
+                hold = __ballot_sync(0xFFFFFFFFu, (dep & (vm.n_frames >> 31)) != 0u);   /* n_frames < 2^31 */
+            } else {
+                __syncwarp();
+                __threadfence();
+            }
+#pragma unroll
+            for (int u = 0; u < R; ++u) {
+                if (((rowmask[u] >> lane) & 1u) && frame[u] != kNotReady) {
+                    todo &= ~(1ull << (j0 + u));
+                    ++served;
+                    if (lane == leader[u]) atomicAdd(vm.pte + vpn[u], ~0ull + hold);
+                }
+            }
+            progress = true;
+        }
+        return progress;
     };
 
-    /* Each round registers the next 64 rows and then visits every registered row, so pages that
-     * are there are used and released while the rest of the table is still being registered. */
+    /* Each round registers the next words of 64 rows and then visits every registered row that has
+     * unfinished requests, so pages that are there are used and released while the rest of the
+     * table is still being registered. */
     unsigned int registered = 0;
     unsigned long long t_start = 0;
     unsigned int sleep_ns = 64;
     for (;;) {
         bool progress = false, any_rows = false, has_own = false;
+        const unsigned int first_new = registered;
         for (unsigned int r = 0; r < GPUVM_BATCH_REGISTER_PER_ROUND && registered < words; ++r) {
-            register_word(registered++);
+            const unsigned int k = registered++;
+            unsigned long long todo = 0, own = 0;
+            const unsigned int jn = rows - 64u * k < 64u ? rows - 64u * k : 64u;
+            for (unsigned int j0 = 0; j0 < jn; j0 += R) visit(k, j0, jn, true, todo, own);
+            m_todo[(size_t)k * mask_stride] = todo;
+            m_own[(size_t)k * mask_stride] = own;
             progress = true;
         }
         for (unsigned int k = 0; k < registered; ++k) {
             unsigned long long todo = m_todo[(size_t)k * mask_stride], own = m_own[(size_t)k * mask_stride];
             if (!__any_sync(0xFFFFFFFFu, todo != 0ull)) continue;
+            any_rows = true;
             const unsigned long long todo_in = todo, own_in = own;
-            const unsigned int jn = rows - 64u * k < 64u ? rows - 64u * k : 64u;
-            for (unsigned int j0 = 0; j0 < jn; j0 += R) {
-                /* R rows at a time: their table entries and page-table words are fetched together */
-                unsigned int rowmask[R], vpn[R], off[R], leader[R], any = 0;
-                unsigned long long peek[R];
-#pragma unroll
-                for (int u = 0; u < R; ++u) {
-                    rowmask[u] = __ballot_sync(0xFFFFFFFFu, j0 + u < jn && ((todo >> (j0 + u)) & 1ull) != 0);
-                    any |= rowmask[u];
-                }
-                if (!any) continue;
-                any_rows = true;
-#pragma unroll
-                for (int u = 0; u < R; ++u) {
-                    vpn[u] = 0; off[u] = 0;
-                    if ((rowmask[u] >> lane) & 1u) {
-                        const unsigned int i = (64u * k + j0 + u) * 32 + lane;
-                        vpn[u] = table.vpn(i);
-                        off[u] = table.off(i);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < R; ++u) {
-                    leader[u] = 32; peek[u] = 0;
-                    if ((rowmask[u] >> lane) & 1u) {
-                        leader[u] = __ffs(__match_any_sync(rowmask[u], vpn[u])) - 1;
-                        if (lane == leader[u] && !((own >> (j0 + u)) & 1ull)) peek[u] = ld_relaxed_u64(vm.pte + vpn[u]);
-                    }
-                }
-                /* leaders: what the entries say.  An entry that looks VALID is read again with
-                 * acquire (it pairs with the fence before the publish); a VALID that turns up any
-                 * other way gets a fence. */
-                unsigned int frame[R];
-                bool need_fence = false;
-#pragma unroll
-                for (int u = 0; u < R; ++u) {
-                    frame[u] = kNotReady;
-                    const unsigned long long bit = 1ull << (j0 + u);
-                    if (lane == leader[u] && !(own & bit)) {
-                        unsigned long long w = peek[u];
-                        const bool looks_valid = (w & kStMask) == kValid;
-                        if (GPUVM_BATCH_ACQ == 1 && looks_valid) w = ld_acquire_u64(vm.pte + vpn[u]);
-                        unsigned int f;
-                        const int st = advance(vm, vm.pte + vpn[u], w, mode, f);
-                        if (st == kReady) { frame[u] = f; need_fence |= GPUVM_BATCH_ACQ == 2 || (GPUVM_BATCH_ACQ == 1 && !looks_valid); }
-                        else if (st == kOwn) { own |= bit; progress = true; }
-                    }
-                }
-                if (__any_sync(0xFFFFFFFFu, need_fence)) __threadfence();
-                /* followers take the frame from their leader; every ready request is consumed */
-                bool any_ready = false;
-                unsigned int dep = 0;          /* what consume returned, folded: see below */
-#pragma unroll
-                for (int u = 0; u < R; ++u) {
-                    if (!rowmask[u]) continue;
-                    const bool mine = ((rowmask[u] >> lane) & 1u) != 0;
-                    if (mine) frame[u] = __shfl_sync(rowmask[u], frame[u], leader[u]);
-                    const bool ready = mine && frame[u] != kNotReady;
-                    if (WARP_CONSUME) {
-                        unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
-                        while (ready_lanes) {
-                            const unsigned int L = __ffs(ready_lanes) - 1;
-                            ready_lanes &= ready_lanes - 1;
-                            const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame[u], L), o = __shfl_sync(0xFFFFFFFFu, off[u], L);
-                            call_consume(consume, (64u * k + j0 + u) * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o, dep);
-                        }
-                    } else if (ready) {
-                        call_consume(consume, (64u * k + j0 + u) * 32 + lane,
-                                     vm.pool + ((unsigned long long)frame[u] << vm.page_shift) + off[u], dep);
-                    }
-                    any_ready |= ready;
-                }
-                /* step 8 for all of them.  The decrements must not overtake the groups' accesses
-                 * to their frames.  A consume that only reads and returns (something computed
-                 * from) what it read gives the engine a value that does not exist before the
-                 * loads have returned: `hold` below is zero, but it is computed from those values
-                 * of all 32 lanes, so the decrement that adds it cannot be issued earlier.  Any
-                 * other consume, and write mode, get a warp barrier and a fence instead. */
-                if (__any_sync(0xFFFFFFFFu, any_ready)) {
-                    unsigned long long hold = 0;
-                    if (kConsumeReturns && mode == kRead) {
-                        hold = __ballot_sync(0xFFFFFFFFu, (dep & (vm.n_frames >> 31)) != 0u);   /* n_frames < 2^31 */
-                    } else {
-                        __syncwarp();
-                        __threadfence();
-                    }
-#pragma unroll
-                    for (int u = 0; u < R; ++u) {
-                        if (((rowmask[u] >> lane) & 1u) && frame[u] != kNotReady) {
-                            todo &= ~(1ull << (j0 + u));
-                            ++served;
-                            if (lane == leader[u]) atomicAdd(vm.pte + vpn[u], ~0ull + hold);
-                        }
-                    }
-                    progress = true;
-                }
+            if (k < first_new) {                              /* (what was registered in this round has just been looked at) */
+                const unsigned int jn = rows - 64u * k < 64u ? rows - 64u * k : 64u;
+                for (unsigned int j0 = 0; j0 < jn; j0 += R) progress |= visit(k, j0, jn, false, todo, own);
             }
             if (queue) {
                 /* hand owned faults to the migrator warps; afterwards wait for the page like anyone */
@@ -571,7 +567,10 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
             }
         }
 
-        if (__any_sync(0xFFFFFFFFu, progress)) { sleep_ns = 64; t_start = 0; continue; }
+        if (__any_sync(0xFFFFFFFFu, progress)) {
+            sleep_ns = 64; t_start = 0;
+            continue;
+        }
         /* nothing moved: back off; give up when the bound is reached */
         const unsigned long long t = now_ns();
         if (t_start == 0) t_start = t;

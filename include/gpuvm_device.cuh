@@ -148,7 +148,11 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 __device__ __forceinline__ unsigned long long pin_acquire(unsigned long long *pte)
 {
     unsigned long long old;
+#ifdef GPUVM_EXP_RELAXED_PIN
+    asm volatile("atom.relaxed.gpu.global.add.u64 %0, [%1], 1;" : "=l"(old) : "l"(pte) : "memory");
+#else
     asm volatile("atom.acquire.gpu.global.add.u64 %0, [%1], 1;" : "=l"(old) : "l"(pte) : "memory");
+#endif
     return old;
 }
 
@@ -180,7 +184,11 @@ __device__ __forceinline__ void st_relaxed_u32(unsigned int *p, unsigned int v)
  * barrier before it, its group's) frame accesses happen before the drop */
 __device__ __forceinline__ void unpin(unsigned long long *pte)
 {
+#ifdef GPUVM_EXP_RELAXED_UNPIN
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(pte), "l"(~0ull) : "memory");
+#else
     asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(pte), "l"(~0ull) : "memory");
+#endif
 }
 
 __device__ __forceinline__ void stat_add(const gpuvm_dev_t &vm, int kind, unsigned long long v)
@@ -493,8 +501,10 @@ __device__ __forceinline__ bool try_claim(const gpuvm_dev_t &vm, unsigned long l
  * Write-back off the fault path (the paper names synchronous write-back by the faulting thread as
  * its weak spot, Section 5.3, and eviction work inside the fault handler as the cause of the step at
  * oversubscription level 1, Section 5.4).  The frame ring has a second cursor that runs ahead of the
- * head cursor: warps with nothing to do -- a migrator warp whose fault ring is empty, a warp that
- * waits for somebody else's fault -- take the next ring position from it, and if the page in that
+ * head cursor: warps of the batched kernels with nothing to do -- a migrator warp whose fault ring is
+ * empty, a requester warp whose scan found nothing ready -- take the next ring position from it (the
+ * single-access path does not: the call alone cost its kernels a third of their resident
+ * throughput in registers), and if the page in that
  * frame would be the head cursor's victim when it gets there (resident, nobody holds it, not
  * referenced since its last chance, dirty) they write it back now.  One compare-and-swap on the
  * exact entry takes a reference and clears the dirty bit: all earlier writers have released the page,
@@ -579,9 +589,14 @@ static __device__ __noinline__ bool slow_path(const gpuvm_dev_t vm, unsigned lon
     unsigned int sleep_ns = 32;
 
     if (is_leader) {
-        st = advance(vm, pte, w, mode, frame);
-        if (st == kReady) { if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1); }
-        else if (st == kWait) stat_add(vm, kWaits, 1);
+        if ((w & kRcMask) > kRcLimit) {                      /* too many references to this page: refused, nothing stays pinned */
+            set_error_pins(vm, pte);
+            st = kFail;
+        } else {
+            st = advance(vm, pte, w, mode, frame);
+            if (st == kReady) { if (GPUVM_COUNT_HITS) stat_add(vm, kHits, 1); }
+            else if (st == kWait) stat_add(vm, kWaits, 1);
+        }
     }
 
     for (;;) {
@@ -667,8 +682,6 @@ static __device__ __noinline__ bool slow_path(const gpuvm_dev_t vm, unsigned lon
             continue;                                        /* READY groups still finish */
         }
         if (lane == (unsigned int)(__ffs(active) - 1)) stat_add(vm, kRetries, 1);
-        /* nothing to do but wait: write back a dirty page that is about to become a victim, if there is one */
-        if (clean_ahead(vm, active, rank, nlanes, lane == (unsigned int)(__ffs(active) - 1))) continue;
         __nanosleep(sleep_ns);
         if (sleep_ns < 2048) sleep_ns *= 2;
     }
@@ -695,16 +708,13 @@ __device__ __forceinline__ bool access(const gpuvm_dev_t &vm, unsigned long long
     unsigned long long *pte = vm.pte + vpn;
     unsigned long long w = 0;
     if (is_leader) {
-        w = guard_pin(vm, pte, pin_acquire(pte) + 1ull);     /* pin first, look afterwards */
+        w = pin_acquire(pte) + 1ull;                         /* pin first, look afterwards */
         if (group & (group - 1)) stat_add(vm, kLanes, __popc(group) - 1);
     }
     w = __shfl_sync(active, w, leader);
-    if (w == kPinRefused) {                                  /* this group's request was refused: nothing is pinned */
-        if (OP_BYTES == 0) { *ptr_out = nullptr; if (tok) { tok->vpn = vpn; tok->group = group; tok->leader = 0; } }
-        return false;
-    }
     unsigned int frame = (unsigned int)((w & kFrameMask) >> kFrameShift);
-    const bool hit = (w & kStMask) == kValid;
+    /* (a counter beyond the limit is not a hit: the slow path refuses the request) */
+    const bool hit = (w & kStMask) == kValid && (w & kRcMask) <= kRcLimit;
     if (__all_sync(active, hit)) {
         if (is_leader) {
             unsigned long long want = (mode != kRead ? kDirty : 0ull) |

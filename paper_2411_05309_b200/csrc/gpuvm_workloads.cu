@@ -1242,7 +1242,7 @@ scatter_update_queued_kernel(gpuvm_dev_t vm, unsigned long long a_off, const lon
 }
 
 // ------------------------------------------------------------------ page touch
-__global__ void touch_pages_kernel(gpuvm_dev_t vm, unsigned long long first_page, unsigned long long n_pages)
+__global__ void __launch_bounds__(256, 2) touch_pages_kernel(gpuvm_dev_t vm, unsigned long long first_page, unsigned long long n_pages)
 {
     for (unsigned long long p = warp_in_grid(); p < n_pages; p += warps_in_grid()) {
         gpuvm_token tok;

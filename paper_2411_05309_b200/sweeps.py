@@ -7,6 +7,7 @@ oversubscription analysis), printed as JSON lines.
     python -m paper_2411_05309_b200.sweeps oversub [--workload 1|2|3|4] [--shrink S]
     python -m paper_2411_05309_b200.sweeps depth   [--workload 2|5] [--shrink S]
     python -m paper_2411_05309_b200.sweeps writeback
+    python -m paper_2411_05309_b200.sweeps link    [--gib 0.25]
 
 pages   -- Section 5.1 / Fig. 7: move a fixed amount of host memory into the pool with one
            warp per page, consecutive pages, for page sizes from 4 KiB to 2 MiB; reports the
@@ -24,6 +25,8 @@ oversub -- Section 5.4 / Fig. 14 with Eq. 1: run a workload with the pool shrunk
 depth   -- Section 3.2 (queue depth by Little's law) carried over to page requests: the batched
            workloads under a growing bound of their device scratch, i.e. with more and more page
            requests registered per warp; reports scratch bytes, faults and time.
+link    -- the host link by itself: pinned-copy (copy engine) and SM-issued load / store bandwidth on a
+           buffer of the given size (the kernels that every roofline of this build is measured against).
 writeback -- Section 5.3 (vector add: synchronous write-back named as the weak spot) and Section 5.4
            (eviction adds to the fault latency): workloads whose victims are dirty, at pools of all,
            a quarter and a twelfth of the data: the scattered read-modify-write in its three forms and
@@ -186,6 +189,20 @@ def sweep_depth(cfg: int, shrink: int):
             w.close()
 
 
+def sweep_link(gib: float):
+    import torch
+    from . import binding as B
+    nbytes = int(gib * (1 << 30)) // 4096 * 4096
+    host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    devb = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    out = {"sweep": "link", "bytes": nbytes}
+    for name, (dst, src) in {"ce_h2d_gbs": (devb, host), "ce_d2h_gbs": (host, devb)}.items():
+        out[name] = max(nbytes / _time(torch, lambda: dst.copy_(src, non_blocking=True)) / 1e9 for _ in range(4))
+    sm = B.gpuvm_link_peak(host.data_ptr(), devb.data_ptr(), nbytes, 3)
+    out.update({"sm_h2d_gbs": sm["h2d_gbs"], "sm_d2h_gbs": sm["d2h_gbs"], "sm_duplex_gbs": sm["duplex_gbs"]})
+    print(json.dumps(out), flush=True)
+
+
 def sweep_writeback():
     import torch
     from . import binding as B
@@ -250,7 +267,7 @@ def sweep_writeback():
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("which", choices=["pages", "warps", "resident", "oversub", "depth", "writeback"])
+    ap.add_argument("which", choices=["pages", "warps", "resident", "oversub", "depth", "writeback", "link"])
     ap.add_argument("--gib", type=float, default=4.0)
     ap.add_argument("--warps-per-sm", type=int, default=16)
     ap.add_argument("--workload", type=int, default=1)
@@ -264,6 +281,8 @@ def main(argv=None):
         sweep_warps(min(a.gib, 2.0))
     elif a.which == "writeback":
         sweep_writeback()
+    elif a.which == "link":
+        sweep_link(a.gib if a.gib != 4.0 else 0.25)
     elif a.which == "depth":
         sweep_depth(a.workload if a.workload in (2, 5) else 2, a.shrink)
     else:
