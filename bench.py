@@ -117,13 +117,20 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------- link peaks
 
-# Host-link bytes of one launch as ncu counted them (sysmem read sector misses x 32 B, plus sysmem write
-# sectors for the written workload) in the capture committed under profiles/, scaled to the full
-# launch where the capture was taken on a reduced case (traffic grows with the pages moved).
-# cfg -> (bytes per launch at full size, file under profiles/, how it was scaled)
+# Host-link bytes of one launch of each configuration's dominant kernel as ncu counted them (sysmem read
+# sector misses x 32 B inbound; for the written workload also the outbound payload) in the capture
+# committed under profiles/.  Where the capture was taken on a reduced case the figure is scaled to the full
+# launch by the pages moved (every page crosses the link once in these launches, so traffic grows in
+# proportion).  cfg -> (bytes per launch at full size, file under profiles/, the count in that file, how scaled)
 NCU_LINK_TRAFFIC = {
-    1: (2097152 * 32, "stream_sum_kernel_cfg1_full_set.md", "full size"),
-    2: (33554432 * 32, "gather_batch_kernel_cfg2_full_set.md", "full size"),
+    1: (2097152 * 32, "stream_sum_kernel_cfg1_full_set.md", 2097152, "full size"),
+    2: (33554432 * 32, "gather_batch_kernel_cfg2_full_set.md", 33554432, "full size"),
+    3: (37699584 * 32, "graph_sweep_kernel_lc_cfg3_sweep1_full_set.md", 37699584,
+        "full size; sweep 1 of the five sweeps of a run, 85 % of its time"),
+    4: (33554432 * 32 * 8 + (4 << 30), "vadd_kernel_cfg4_eighth_full_set.md", 33554432,
+        "1/8 case x 8: 8 GiB in, plus the 4 GiB of c that go out"),
+    5: (134217728 * 32 * 16, "embag_batch_kernel_cfg5_sixteenth_full_set.md", 134217728, "1/16 case x 16"),
+    6: (37758976 * 32, "graph_sweep_kernel_cc_cfg6_full_set.md", 37758976, "full size"),
 }
 
 
@@ -232,9 +239,9 @@ def oracle_sample(cfg: int, w=None, shrink: int = 0):
         return int(16 * reached.sum() + 8 * np.diff(off)[reached].sum()), f"Dijkstra on an RMAT graph of scale {scale}", \
             (lambda impl: impl.sssp_direct(off, col, wt, 0)), False
     if cfg == 5:
-        rows_n, dims, bag = 1 << 20, 128, 32
+        rows_n, dims, bag = 1 << 25, 128, 32          # a 16 GiB table: far beyond the last-level cache, like the workload's
         t = inputs.fill_f32_pm1(np.empty(rows_n * dims, np.float32), rows_n * dims, inputs.config_seed(5)).reshape(rows_n, dims)
-        n_lookups = 1 << 21
+        n_lookups = 1 << 22
         rows = inputs.fill_zipf_rows(np.empty(n_lookups, np.int64), n_lookups, inputs.config_seed(5, 1), rows_n, 1.05)
         return 4 * dims * n_lookups, f"{n_lookups} Zipf lookups (bags of {bag}) into a {rows_n}-row table", \
             (lambda impl: impl.embag_f32_direct(t, rows, bag)), True
@@ -438,7 +445,7 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
         roof = link_roofline(bytes_in, bytes_out, kern_s, link)
         traffic = NCU_LINK_TRAFFIC.get(cfg) if args.shrink == 0 and not args.scratch_limit_mib else None
         roof["traffic"] = traffic[0] if traffic else None
-        roof["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[2]}): host-link bytes of one launch counted by ncu"
+        roof["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[3]}): host-link bytes of one launch counted by ncu"
                                   if traffic else None)
         roof["hbm"] = {"achieved": (bytes_in + bytes_out + eff_bytes) / kern_s / 1e9, "peak": hbm_peak,
                        "frac": ((bytes_in + bytes_out + eff_bytes) / kern_s / 1e9) / hbm_peak,
@@ -475,7 +482,7 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
             w.run(check=False)
             r = w.run(check=True)
             rec["scratch"]["bounded_to_an_eighth_of_the_pool"] = {
-                "limit_bytes": bound, "scratch_bytes_used_by_this_run": None, "ms_per_step": r.seconds * 1e3,
+                "limit_bytes": bound, "ms_per_step": r.seconds * 1e3,
                 "value": r.effective_bytes / r.seconds / 1e9, "faults": r.stats["faults"],
                 "in_gbs": r.stats["bytes_in"] / r.seconds / 1e9, "invariants_status": r.check["status"]}
             B.gpuvm_set_scratch_limit(w.h, 0)

@@ -88,6 +88,7 @@ def test_direction_aware_roofline_and_config_record():
     assert a == b and a["cfg"] == 5 and a["pool_bytes"] == 16 << 30 and a["page_bytes"] == 2 << 20
     assert bench.config_of(3, 0)["frames"] == 9216
     root = os.path.dirname(os.path.abspath(bench.__file__))
-    for cfg, (nbytes, name, how) in bench.NCU_LINK_TRAFFIC.items():
+    for cfg, (nbytes, name, sectors, how) in bench.NCU_LINK_TRAFFIC.items():
         text = open(os.path.join(root, "profiles", name)).read().replace(" ", "").replace(",", "")
-        assert str(nbytes // 32) in text, (cfg, name)             # the sector count is in the committed summary
+        assert str(sectors) in text, (cfg, name)                  # the sector count is in the committed summary
+        assert nbytes >= sectors * 32
