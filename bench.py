@@ -12,7 +12,7 @@ With no --workload all five configurations are run, the largest one last: config
 (Zipf embedding bag: 64 GiB table, 2 MiB pages, 16 GiB pool) is the headline record, timed
 for exactly K steps after W warm-up steps, and `per_config` carries the same fields for each of
 the five (configurations 1-4 with min(K, 10) steps after min(W, 3)).  --workload N runs one
-workload (1-5 the configurations, 6 CC, 7 SSSP, 8 BFS over Balanced CSR) as the headline.
+workload (1-5 the configurations, 6 CC, 7 SSSP, 8 and 9 BFS and CC over Balanced CSR) as the headline.
 
 Rank 0 prints ONE JSON line.  `value` is the effective application GB/s (useful payload
 bytes / CUDA-event time) with all inputs resident (paged array in pinned host memory, which
@@ -220,7 +220,7 @@ def oracle_sample(cfg: int, w=None, shrink: int = 0):
         a = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4))
         b = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(4, 1))
         return 12 * n, f"direct vector add of the first {n} elements", (lambda impl: impl.vadd_f32_direct(a, b)), True
-    if cfg in (3, 8, 6, 7):
+    if cfg in (3, 8, 6, 7, 9):
         scale = min(24 - shrink, 22)
         off, col = inputs.rmat_csr(scale, 16 << scale, inputs.config_seed(3))
         import oracle
@@ -230,7 +230,7 @@ def oracle_sample(cfg: int, w=None, shrink: int = 0):
             nbytes = int(16 * vis.sum() + 4 * np.diff(off)[vis].sum())
             return nbytes, f"queue BFS on an RMAT graph of scale {scale} (sequential by nature: one thread)", \
                 (lambda impl: impl.bfs_levels_direct(off, col, 0)), False
-        if cfg == 6:
+        if cfg in (6, 9):
             return 8 * off.size + 4 * col.size, f"union-find over an RMAT graph of scale {scale} (one pass over the edges)", \
                 (lambda impl: impl.cc_labels_direct(off, col)), False
         wt = inputs.fill_i32_range(np.empty(col.size, np.int32), col.size, inputs.config_seed(3, 2), 1, 255)
@@ -299,8 +299,9 @@ NAMES = {1: "cfg1 streaming read-reduce: int64 sum over 64 MiB int32, 4 KiB page
          5: "cfg5 Zipf(1.05) embedding bag: 64 GiB table, 2^24 lookups, bags of 32, 2 MiB pages, 16 GiB pool",
          6: "connected components on the cfg3 graph (RMAT scale 24), CSR paged at 64 KiB, pool = half",
          7: "SSSP from vertex 0 on the cfg3 graph with int32 weights in a third paged array, 64 KiB pages, pool = half",
-         8: "BFS on the cfg3 graph stored as Balanced CSR (chunks of 16 Ki edges), 64 KiB pages, pool = half"}
-DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32", 6: "int32", 7: "int32", 8: "int32"}
+         8: "BFS on the cfg3 graph stored as Balanced CSR (chunks of 16 Ki edges), 64 KiB pages, pool = half",
+         9: "connected components on the cfg3 graph stored as Balanced CSR, 64 KiB pages, pool = half"}
+DTYPES = {1: "int64", 2: "f32", 3: "int32", 4: "f32", 5: "f32", 6: "int32", 7: "int32", 8: "int32", 9: "int32"}
 
 
 def config_of(cfg: int, shrink: int) -> dict:
@@ -379,7 +380,7 @@ def replica_throughput(world: int, units_per_rank: float, slowest_seconds: float
 # ------------------------------------------------------------------------------- ours
 
 OUTPUTS = {1: ["d_sum"], 2: ["d_fsum", "d_bsum"], 3: ["d_level"], 4: [], 5: ["d_out"], 6: ["d_level"], 7: ["d_dist"],
-           8: ["d_level"]}
+           8: ["d_level"], 9: ["d_level"]}
 
 
 def e2e_step(torch, B, w, cfg: int):
@@ -555,7 +556,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=0, choices=[0, 1, 2, 3, 4, 5, 6, 7, 8],
+    ap.add_argument("--workload", type=int, default=0, choices=[0, 1, 2, 3, 4, 5, 6, 7, 8, 9],
                     help="run this workload only (0: all of --configs, the largest as the headline)")
     ap.add_argument("--configs", default="1,2,3,4,5", help="configurations of the default run")
     ap.add_argument("--shrink", type=int, default=0, help="divide all sizes by 2**shrink")

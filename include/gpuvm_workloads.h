@@ -112,6 +112,14 @@ int gpuvm_bfs_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, 
                    size_t chunk_edges, size_t source, int32_t *d_level, int *n_levels, void *stream);
 
 /*
+ * Connected components over Balanced CSR (Section 5.2, Fig. 8 runs CC on it): the union-find pass of
+ * gpuvm_cc_csr, with workers that take chunks of edges instead of vertices.  Arguments as for
+ * gpuvm_bfs_bcsr; d_label as for gpuvm_cc_csr.  One launch; synchronises the stream.
+ */
+int gpuvm_cc_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, size_t nv, size_t n_edges,
+                  size_t chunk_edges, int32_t *d_label, void *stream);
+
+/*
  * Build the chunk table of Balanced CSR (Section 5.2, Fig. 8) from a graph's row offsets, on
  * the host: a format conversion done once, before the graph is handed to gpuvm_create.
  *   row_off       host pointer, nv + 1 int64 row offsets, row_off[0] = 0.

@@ -86,6 +86,7 @@ SYMBOLS = {
     "gpuvm_bfs_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_bfs_csr_noalloc": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_bfs_bcsr": (_i, [_vp, _sz, _sz, _sz, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
+    "gpuvm_cc_bcsr": (_i, [_vp, _sz, _sz, _sz, _sz, _sz, _sz, _vp, _vp]),
     "gpuvm_cc_csr": (_i, [_vp, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_sssp_csr": (_i, [_vp, _sz, _sz, _sz, _sz, _sz, _vp, ctypes.POINTER(_i), _vp]),
     "gpuvm_raw_cc_csr": (_i, [_vp, _vp, _sz, _vp, ctypes.POINTER(_i), _vp]),
@@ -323,6 +324,12 @@ def gpuvm_bfs_bcsr(h, off_off: int, col_off: int, chunk_off: int, nv: int, n_edg
     _check(lib().gpuvm_bfs_bcsr(h, off_off, col_off, chunk_off, nv, n_edges, chunk_edges, source, _ptr(d_level),
                                 ctypes.byref(levels), _stream(stream)), "gpuvm_bfs_bcsr")
     return levels.value
+
+
+def gpuvm_cc_bcsr(h, off_off: int, col_off: int, chunk_off: int, nv: int, n_edges: int, chunk_edges: int, d_label,
+                  stream=None):
+    _check(lib().gpuvm_cc_bcsr(h, off_off, col_off, chunk_off, nv, n_edges, chunk_edges, _ptr(d_label), _stream(stream)),
+           "gpuvm_cc_bcsr")
 
 
 def gpuvm_cc_csr(h, off_off: int, col_off: int, nv: int, d_label, stream=None) -> int:

@@ -255,6 +255,22 @@ class BfsBalanced(Bfs):
         return {"levels": self.levels}
 
 
+class CcBalanced(BfsBalanced):
+    """Connected components on the cfg 3 graph stored as Balanced CSR."""
+    name, cfg = "cc_rmat_balanced_csr", 9
+
+    def launch(self, stream):
+        B.gpuvm_cc_bcsr(self.h, self.off["off"], self.off["col"], self.off["chunk"], self.nv, self.ne, self.chunk_edges,
+                        self.d_level, stream)
+        return {"sweeps": 1}
+
+    def effective_bytes(self):
+        return int(8 * (self.nv + 1) + 4 * self.ne)
+
+    def compulsory_pages(self):
+        return self.n_pages
+
+
 class Cc(Bfs):
     """Connected components on the BFS configuration's graph and pool (the paper's second graph workload)."""
     name, cfg = "cc_rmat_csr", 6
@@ -352,7 +368,7 @@ class EmbeddingBag(Workload):
         return 4 * self.dims * self.n_lookups
 
 
-WORKLOADS = {1: StreamSum, 2: Gather, 3: Bfs, 4: VAdd, 5: EmbeddingBag, 6: Cc, 7: Sssp, 8: BfsBalanced}
+WORKLOADS = {1: StreamSum, 2: Gather, 3: Bfs, 4: VAdd, 5: EmbeddingBag, 6: Cc, 7: Sssp, 8: BfsBalanced, 9: CcBalanced}
 
 
 def make(cfg: int, shrink: int = 0) -> Workload:

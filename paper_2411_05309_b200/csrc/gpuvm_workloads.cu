@@ -907,6 +907,7 @@ __global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsign
             if (hi > c_hi) hi = c_hi;
             unsigned int touch = __ballot_sync(0xFFFFFFFFu, active && hi > lo);
             if (!touch) continue;
+            const int uval = active ? op.begin(v) : 0;
             // the chunk's column page is held only while these 32 vertices are expanded, never
             // while row offsets are read: one page at a time, no pool is too small
             gpuvm_token tok;
@@ -916,7 +917,8 @@ __global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsign
                 const int L = __ffs(touch) - 1;
                 touch &= touch - 1;
                 const long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
-                found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), op.depth, blo, bhi, lane, 0u);
+                found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), __shfl_sync(0xFFFFFFFFu, uval, L),
+                                                     blo, bhi, lane, 0u);
             }
             m.release(tok);
         }
@@ -1509,6 +1511,30 @@ int run_bfs_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off,
     return rc;
 }
 
+// Connected components over Balanced CSR: the one union-find pass, chunk by chunk.
+template <class Mem>
+int run_cc_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off, size_t nv, size_t n_edges,
+                size_t chunk_edges, int32_t *d_label, void *scratch, cudaStream_t s)
+{
+    if (!d_label || nv == 0 || nv > 0x7FFFFFFFull || chunk_edges == 0 || chunk_edges > 0x7FFFFFFFull) return GPUVM_E_ARG;
+    if (off_off % 16 || col_off % 16 || chunk_off % 16) return GPUVM_E_ALIGN;
+    if (col_off % m.unit_host() || m.unit_host() % (4 * chunk_edges)) return GPUVM_E_ALIGN;
+    if (!scratch) return GPUVM_E_ALLOC;
+    unsigned int *counters = static_cast<unsigned int *>(scratch);
+    cc_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
+    int rc = launched();
+    if (rc == GPUVM_OK && n_edges > 0) {
+        cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
+        bcsr_sweep_kernel<Mem, CcOp><<<sm_count() * 2, 256, 0, s>>>(m, CcOp{d_label}, off_off, col_off, chunk_off, (unsigned int)nv,
+                                                                    n_edges, (unsigned int)chunk_edges, counters, 0);
+        rc = launched();
+    }
+    cc_finish_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
+    if (rc == GPUVM_OK) rc = launched(); else launched();
+    cudaStreamSynchronize(s);
+    return rc;
+}
+
 struct Scratch {                     // device scratch for one call, freed on scope exit
     void *p = nullptr;
     explicit Scratch(size_t bytes) { if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); p = nullptr; } }
@@ -1715,6 +1741,15 @@ int gpuvm_bfs_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, 
     if (!view_of(h, m)) return GPUVM_E_ARG;
     return run_bfs_bcsr(m, off_off, col_off, chunk_off, nv, n_edges, chunk_edges, source, d_level, n_levels,
                         gpuvm_scratch_(h, kBfsScratchBytes), static_cast<cudaStream_t>(stream));
+}
+
+int gpuvm_cc_bcsr(gpuvm_t h, size_t off_off, size_t col_off, size_t chunk_off, size_t nv, size_t n_edges, size_t chunk_edges,
+                  int32_t *d_label, void *stream)
+{
+    PagedH m;
+    if (!view_of(h, m)) return GPUVM_E_ARG;
+    return run_cc_bcsr(m, off_off, col_off, chunk_off, nv, n_edges, chunk_edges, d_label, gpuvm_scratch_(h, kBfsScratchBytes),
+                       static_cast<cudaStream_t>(stream));
 }
 
 int gpuvm_bcsr_build(const int64_t *row_off, size_t nv, size_t chunk_edges, int32_t *chunk_vertex, size_t capacity,

@@ -122,6 +122,16 @@ def test_bfs_over_balanced_csr_rmat24():
         w.close()
 
 
+def test_cc_over_balanced_csr_rmat24():
+    w, res = run(9)
+    try:
+        off, col = w.view("off", np.int64, w.nv + 1), w.view("col", np.int32, w.ne)
+        assert np.array_equal(w.d_level.cpu().numpy(), oracle.cc_labels_direct(off, col))
+        assert res.stats["writebacks"] == 0 and res.stats["faults"] >= w.n_pages - 1
+    finally:
+        w.close()
+
+
 def test_cfg4_vector_add_12GiB():
     w, res = run(4)
     try:

@@ -261,11 +261,15 @@ def test_bfs_over_balanced_csr(B, policy):
             pad4 = lambda a: np.concatenate([a, np.zeros((-a.size) % 4, a.dtype)])
             ar = Arena(page, {"off": off_p, "col": pad4(col), "chunk": pad4(chunks)})
             level = torch.zeros(nv, dtype=torch.int32, device="cuda")
+            label = torch.zeros(nv, dtype=torch.int32, device="cuda")
             with paged(ar.host, page, frames, policy) as h:
                 depth = B.gpuvm_bfs_bcsr(h, ar.off["off"], ar.off["col"], ar.off["chunk"], nv, ne, chunk_edges, src, level)
                 st, ck = finish(h)
+                B.gpuvm_cc_bcsr(h, ar.off["off"], ar.off["col"], ar.off["chunk"], nv, ne, chunk_edges, label)
+                finish(h)
             assert np.array_equal(level.cpu().numpy(), ref), (nv, ne, page, chunk_edges, frames)
             assert depth == ref.max() + 1
+            assert np.array_equal(label.cpu().numpy(), oracle.cc_labels_direct(off, col)), (nv, ne, page)
     # a chunk that would straddle pages is refused
     with paged(ar.host, 4096, 8) as h:
         with pytest.raises(B.GpuvmError) as e:
