@@ -401,8 +401,10 @@ def e2e_step(torch, B, w, cfg: int):
     B.gpuvm_flush(w.h, stream)
     for name in OUTPUTS[cfg]:
         t = getattr(w, name)
-        buf = w.__dict__.setdefault("_host_" + name, torch.empty(t.shape, dtype=t.dtype).pin_memory())
-        buf.copy_(t, non_blocking=True)
+        key = "_host_" + name
+        if key not in w.__dict__:                           # (allocated by the untimed first call)
+            w.__dict__[key] = torch.empty(t.shape, dtype=t.dtype).pin_memory()
+        w.__dict__[key].copy_(t, non_blocking=True)
         d2h += t.numel() * t.element_size()
     e1.record(stream)
     e1.synchronize()
@@ -441,9 +443,10 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
         bytes_in = sum(r.stats["bytes_in"] for r in results) / len(results)
         bytes_out = sum(r.stats["bytes_out"] for r in results) / len(results)
         faults = sum(r.stats["faults"] for r in results) / len(results)
+        direct = sum(r.stats.get("bytes_direct", 0) for r in results) / len(results)   # read in place, no page moved
         peaks = measured_peaks()
         hbm_peak = peaks.get("hbm_gbs", 6650.0)
-        roof = link_roofline(bytes_in, bytes_out, kern_s, link)
+        roof = link_roofline(bytes_in + direct, bytes_out, kern_s, link)
         traffic = NCU_LINK_TRAFFIC.get(cfg) if args.shrink == 0 and not args.scratch_limit_mib else None
         roof["traffic"] = traffic[0] if traffic else None
         roof["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[3]}): host-link bytes of one launch counted by ncu"
@@ -456,6 +459,7 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
             "ms_per_step": step_s * 1e3, "dtype": DTYPES[cfg], "config": config_of(cfg, args.shrink),
             "migration": {
                 "in_gbs": bytes_in / step_s / 1e9, "out_gbs": bytes_out / step_s / 1e9,
+                "direct_gbs": direct / step_s / 1e9, "bytes_direct": direct,
                 "faults_per_s": faults / step_s, "faults": faults, "bytes_in": bytes_in, "bytes_out": bytes_out,
                 "io_amplification": bytes_in / eff_bytes if eff_bytes else None,
                 "fault_rate_ceiling_per_s": link["ce_h2d_gbs"] * 1e9 / w.page_bytes,

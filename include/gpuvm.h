@@ -87,7 +87,11 @@ typedef struct gpuvm_dev {
  * frame of a page it no longer holds sees the pattern instead of plausible old data (a
  * stale read then shows up as a wrong result in any parity check; the race checker of the
  * CUDA tools is not needed to see it).  Costs one extra write of the frame per eviction. */
-enum { GPUVM_DEBUG_POISON = 1 };
+/* FENCED_RELEASE: the batched engine releases the pages of read-only requests after a warp barrier and
+ * a device fence (the form the PTX memory model orders by itself) instead of making the release depend
+ * on the loaded values (the default, which leans on the hardware issuing an instruction only when its
+ * operands exist).  Same results; a few per cent slower scans.  For cross-checking the default. */
+enum { GPUVM_DEBUG_POISON = 1, GPUVM_DEBUG_FENCED_RELEASE = 2 };
 
 /* Counters accumulated by GPU threads since the last gpuvm_reset(). */
 typedef struct gpuvm_stats {
@@ -108,6 +112,9 @@ typedef struct gpuvm_stats {
     uint64_t resident;        /* pages resident now                                    */
     uint64_t cleaned;         /* dirty pages written back off the fault path, by idle
                                  warps, while they stayed resident                    */
+    uint64_t bytes_direct;    /* bytes that kernels read in place from the backing store
+                                 instead of fetching their page (sparse accesses of the
+                                 graph sweeps to pages that are not resident)          */
     uint64_t ring_drops;      /* entries of a fault ring that were given up on after a
                                  bounded wait (slot never filled, slot never cleared, or
                                  a popped page that was not waiting for a migrator): each

@@ -480,7 +480,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
          * other consume, and write mode, get a warp barrier and a fence instead. */
         if (__any_sync(0xFFFFFFFFu, any_ready)) {
             unsigned long long hold = 0;
-            if (kConsumeReturns && mode == kRead) {
+            if (kConsumeReturns && mode == kRead && !(vm.debug & GPUVM_DEBUG_FENCED_RELEASE)) {
                 hold = __ballot_sync(0xFFFFFFFFu, (dep & (vm.n_frames >> 31)) != 0u);   /* n_frames < 2^31 */
             } else {
                 __syncwarp();

@@ -96,7 +96,7 @@ constexpr int kStatSlots = 32;
 constexpr int kCtlCleanCursor = kCtlCounters + kStatSlots * 16;   /* ring position of the cleaners (a line of its own) */
 constexpr int kCtlWords = kCtlCleanCursor + 16;
 enum Stat { kFaults = 0, kHits, kWaits, kLanes, kEvictions, kWritebacks, kFlushWritebacks,
-            kBytesIn, kBytesOut, kHandSteps, kRetries, kRingDrops, kCleaned, kNumStats };
+            kBytesIn, kBytesOut, kHandSteps, kRetries, kRingDrops, kCleaned, kBytesDirect, kNumStats };
 
 enum Mode { kRead = 0, kWrite = 1, kWriteAll = 2 };
 

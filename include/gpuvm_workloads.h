@@ -82,16 +82,21 @@ int gpuvm_gather_f32_unbatched(gpuvm_t h, size_t x_off, const int64_t *d_idx, si
  * array holds level << 1 | dirty while the sweeps run; lowering is an atomicMin that sets
  * the bit), so one sweep carries as many hops as the vertex order allows, and a vertex
  * that is lowered behind the sweep position is queued and re-expanded in the same sweep by
- * whichever warp is free, provided its pages are still in the pool (gpuvm_ptr_if_resident:
- * no fault is taken for it; otherwise it stays dirty for the next sweep).  The fixed point
- * is the BFS level.  With a pool of half the graph almost every page is fetched once per
+ * whichever warp is free.  No page is fetched for such a vertex: its two row offsets and its
+ * edges are read from their frames where the pages are still in the pool
+ * (gpuvm_ptr_if_resident) and in place from the backing store where they are not (the CSR
+ * arrays are never written, so the backing store is current; gpuvm_stats counts these bytes as
+ * bytes_direct).  A sweep that follows one with few updates works the same way throughout: it
+ * reads the few scattered lists it needs in place instead of fetching a page for each.  The
+ * fixed point is the BFS level.  With a pool of half the graph every page is fetched once per
  * run, where one sweep per level fetched most of the graph once per level.
  * Very long neighbour lists are cut at page boundaries into pieces that go to a queue which
  * all warps of the same launch serve between their chunks (the imbalance Section 5.2
  * describes).  The first sweep expands the source alone.  One launch per sweep; the stream is
  * synchronised between sweeps.  *n_levels (host pointer, may be NULL) receives the largest
  * level + 1.  Uses 2 MiB + max(nv, 2^18) bytes of the handle's device scratch (the two
- * queues and the counters).
+ * queues and the counters).  The row offsets and column indices must not be written through
+ * the runtime while the call runs.
  */
 int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t source,
                   int32_t *d_level, int *n_levels, void *stream);
@@ -158,7 +163,7 @@ int gpuvm_cc_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, int32_t *
  * (GPUVM_E_FRAMES otherwise).  The same label-correcting sweeps as gpuvm_bfs_csr with
  * the edge weight in place of 1; d_dist[v] receives the distance from `source`,
  * 0x7FFFFFFF where unreachable (path lengths must stay below 2^30).  *n_rounds (host
- * pointer, may be NULL) receives the number of sweeps.  Uses 2 MiB + max(nv, 2^18) bytes of
+ * pointer, may be NULL) receives the number of sweeps.  Uses 2 MiB + max(2 nv, 2^18) bytes of
  * the handle's device scratch.  Synchronises per sweep.
  */
 int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source,

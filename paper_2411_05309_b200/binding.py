@@ -18,7 +18,7 @@ POLICY_FIFO, POLICY_CLOCK = 0, 1
 E_ARG, E_PAGE, E_POOL, E_ALIGN, E_PIN, E_ALLOC, E_CUDA, E_TIMEOUT, E_RANGE, E_INVARIANT, E_NODEVICE, E_PINS, E_FRAMES = \
     range(-1, -14, -1)
 
-DEBUG_POISON = 1
+DEBUG_POISON, DEBUG_FENCED_RELEASE = 1, 2
 
 
 class GpuvmError(RuntimeError):
@@ -38,7 +38,7 @@ class DevView(ctypes.Structure):
 class Stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint64) for n in
                 ("faults", "hits", "waits", "lanes_coalesced", "evictions", "writebacks", "flush_writebacks",
-                 "bytes_in", "bytes_out", "hand_steps", "retries", "resident", "cleaned", "ring_drops")] + \
+                 "bytes_in", "bytes_out", "hand_steps", "retries", "resident", "cleaned", "bytes_direct", "ring_drops")] + \
                [("error", ctypes.c_int32), ("reserved", ctypes.c_uint32), ("error_page", ctypes.c_uint64)]
 
     def as_dict(self):

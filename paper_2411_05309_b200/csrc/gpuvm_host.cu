@@ -296,6 +296,7 @@ int gpuvm_stats_on(gpuvm_t h, gpuvm_stats_t *out, void *stream)
     out->hand_steps = sum[kHandSteps]; out->retries = sum[kRetries];
     out->ring_drops = sum[kRingDrops];
     out->cleaned = sum[kCleaned];
+    out->bytes_direct = sum[kBytesDirect];
     out->resident = out->faults - out->evictions;
     out->error = (int32_t)(long long)local[kCtlErr];
     out->error_page = local[kCtlErrPage];
@@ -352,7 +353,7 @@ int gpuvm_set_policy(gpuvm_t h, int policy)
 
 int gpuvm_set_debug(gpuvm_t h, unsigned int flags)
 {
-    if (!h || (flags & ~(unsigned int)GPUVM_DEBUG_POISON)) return GPUVM_E_ARG;
+    if (!h || (flags & ~(unsigned int)(GPUVM_DEBUG_POISON | GPUVM_DEBUG_FENCED_RELEASE))) return GPUVM_E_ARG;
     h->dev.debug = flags;
     return GPUVM_OK;
 }

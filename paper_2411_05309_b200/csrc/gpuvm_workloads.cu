@@ -22,9 +22,18 @@ std::atomic<unsigned long long> g_launches{0};
 
 struct Paged {
     static constexpr int kSweepBlocksPerSm = 4;
+    static constexpr bool kBehindQueue = true;
     gpuvm_dev_t vm;
     unsigned long long edges_hint = 0;
     __device__ __forceinline__ unsigned long long unit() const { return 1ull << vm.page_shift; }
+    // Host side.  Is it cheaper to read `vertices` scattered neighbour lists in place (about 256 bytes on the link
+    // each: two row offsets, a short list, each rounded up to a 128-byte read) than to fetch the pages a full
+    // sweep would miss (what does not fit the pool)?
+    bool sparse_sweep(unsigned long long vertices) const
+    {
+        const unsigned long long missing = vm.n_pages > vm.n_frames ? vm.n_pages - vm.n_frames : 0ull;
+        return vertices * 256ull < (missing << vm.page_shift);
+    }
     template <typename T>
     __device__ __forceinline__ T read(unsigned long long base, unsigned long long i) const { return gpuvm_read<T>(vm, i, base); }
     template <typename T>
@@ -37,6 +46,10 @@ struct Paged {
     {
         return static_cast<unsigned char *>(gpuvm_ptr_if_resident(vm, off, &t));
     }
+    // The backing-store copy of a byte, read in place over the link.  Current for arrays that are not written
+    // through the runtime during the launch (the graph arrays never are).
+    __device__ __forceinline__ const unsigned char *through(unsigned long long off) const { return vm.host + off; }
+    __device__ __forceinline__ void note_direct(unsigned long long bytes) const { gpuvm::stat_add(vm, gpuvm::kBytesDirect, bytes); }
     __device__ __forceinline__ void release(const gpuvm_token &t) const { gpuvm_release(vm, t); }
     __device__ __forceinline__ void clean(const gpuvm_token &t, const void *p) const { gpuvm_clean(vm, t, p); }
     __device__ __forceinline__ void prefetch(unsigned long long off) const { gpuvm_prefetch(vm, off); }
@@ -50,16 +63,20 @@ struct Paged {
 
 struct Raw {
     static constexpr int kSweepBlocksPerSm = 2;
+    static constexpr bool kBehindQueue = false;
     unsigned char *base;
     unsigned long long unit_bytes;
     unsigned long long edges_hint = 0;
     __device__ __forceinline__ unsigned long long unit() const { return unit_bytes; }
+    bool sparse_sweep(unsigned long long) const { return false; }
     template <typename T>
     __device__ __forceinline__ T read(unsigned long long off, unsigned long long i) const { return reinterpret_cast<const T *>(base + off)[i]; }
     template <typename T>
     __device__ __forceinline__ void write(unsigned long long off, unsigned long long i, T v) const { reinterpret_cast<T *>(base + off)[i] = v; }
     __device__ __forceinline__ unsigned char *pin(unsigned long long off, int, gpuvm_token &) const { return base + off; }
     __device__ __forceinline__ unsigned char *pin_if_resident(unsigned long long off, gpuvm_token &) const { return base + off; }
+    __device__ __forceinline__ const unsigned char *through(unsigned long long off) const { return base + off; }
+    __device__ __forceinline__ void note_direct(unsigned long long) const {}
     __device__ __forceinline__ void release(const gpuvm_token &) const {}
     __device__ __forceinline__ void clean(const gpuvm_token &, const void *) const {}
     __device__ __forceinline__ void prefetch(unsigned long long) const {}
@@ -431,6 +448,7 @@ struct LcOp {
     unsigned int behind_cap, n_chunks;
     int backward;
     unsigned int only;                      // kNoVertex, or the one vertex this sweep expands (the first sweep: the source)
+    int through_main;                       // a sparse sweep: pages that are not resident are read in place, not fetched
     __device__ __forceinline__ bool active(unsigned long long v) const
     {
         return only == kNoVertex ? (__ldcg(dist + v) & 1) != 0 : v == only;
@@ -446,7 +464,7 @@ struct LcOp {
         // lowered.  Has the sweep passed c already (or is it just about to)?  Then nobody will look at it
         // again in this sweep unless it is queued.
         const unsigned int ci = (unsigned int)c >> 5, si = backward ? n_chunks - 1u - ci : ci;
-        if (si < pos && only == kNoVertex) {
+        if (si < pos && only == kNoVertex && behind_cap != 0u) {
             const unsigned int m = __activemask(), lane = gpuvm::lane_id(), leader = __ffs(m) - 1;
             unsigned int base = 0;
             if (lane == leader) base = atomicAdd(counters + kCntBehindTail, (unsigned int)__popc(m));
@@ -546,9 +564,11 @@ __device__ __forceinline__ unsigned int take_piece(unsigned int *counters, unsig
 }
 
 // All 32 lanes: take up to 32 vertices from the queue of vertices that were lowered behind the sweep
-// position and re-expand those whose pages are resident.  Returns this lane's number of updates, or -1 when
-// the queue was empty.  A vertex whose row offsets or edges are not in the pool is left dirty (no fault is
-// taken for it: the next sweep finds it); so is one with a very long list.
+// position and re-expand them.  Returns this lane's number of updates, or -1 when the queue was empty.
+// No fault is taken for such a vertex: what it needs (two row offsets, its edges: a hundred bytes or so)
+// is read from the frame when its page is in the pool and in place from the backing store when it is not
+// (the CSR arrays are never written, so the backing store is current).  One with a very long list is left
+// dirty for the next sweep.
 template <class Mem, class Op, bool WEIGHTED>
 __device__ __noinline__ int expand_behind(const Mem m, const Op op, unsigned long long off_off, unsigned long long col_off,
                                           unsigned long long w_off, unsigned int nv, unsigned int *counters, unsigned int lane)
@@ -576,15 +596,19 @@ __device__ __noinline__ int expand_behind(const Mem m, const Op op, unsigned lon
     }
     bool have = u != kNoVertex && u < nv && op.active(u);
     long long lo = 0, hi = 0;
+    unsigned long long direct = 0;                            // bytes read in place from the backing store
     if (have) {
+        // the two row offsets: from their frame when the page is resident, else in place from the backing store
+        // (no page is fetched for a vertex behind the sweep)
         gpuvm_token tok;
         const unsigned char *p = m.pin_if_resident(off_off + 8ull * u, tok);
         if (p) { lo = Mem::load_i64(p); m.release(tok); }
-        const unsigned char *q = p ? m.pin_if_resident(off_off + 8ull * u + 8, tok) : nullptr;
+        else { lo = Mem::load_i64(m.through(off_off + 8ull * u)); direct += 8; }
+        const unsigned char *q = m.pin_if_resident(off_off + 8ull * u + 8, tok);
         if (q) { hi = Mem::load_i64(q); m.release(tok); }
-        have = p && q;
-        if (have && hi <= lo) { op.begin(u); have = false; }  // nothing to expand: just not dirty any more
-        if (have && hi - lo >= kBigDegree) have = false;
+        else { hi = Mem::load_i64(m.through(off_off + 8ull * u + 8)); direct += 8; }
+        if (hi <= lo) { op.begin(u); have = false; }          // nothing to expand: just not dirty any more
+        if (have && hi - lo >= kBigDegree) have = false;      // a hub: left dirty, the next sweep cuts it into pieces
     }
     unsigned int found = 0;
     unsigned int todo = __ballot_sync(0xFFFFFFFFu, have);
@@ -596,31 +620,32 @@ __device__ __noinline__ int expand_behind(const Mem m, const Op op, unsigned lon
         const long long bu = __shfl_sync(0xFFFFFFFFu, u, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
         long long first = __shfl_sync(0xFFFFFFFFu, lo, L);
         int uval = 0;
-        bool begun = false, complete = true;
+        if (lane == 0) uval = op.begin((unsigned long long)bu);
+        uval = __shfl_sync(0xFFFFFFFFu, uval, 0);
         while (first < bhi) {
             const unsigned long long byte = col_off + 4ull * first;
             long long last = (long long)(((byte / unit + 1) * unit - col_off) / 4);
             if (last > bhi) last = bhi;
+            // this part of the list: from its frame when the page is resident, else in place from the backing store
             gpuvm_token tok, tok_w;
             const unsigned char *p = m.pin_if_resident(byte, tok);
-            if (!p) { complete = false; break; }
+            const bool held = p != nullptr;
+            if (!held) { p = m.through(byte); if (lane == 0) direct += 4ull * (unsigned long long)(last - first); }
             const unsigned char *pw = nullptr;
+            bool held_w = false;
             if (WEIGHTED) {
                 pw = m.pin_if_resident(w_off + 4ull * first, tok_w);
-                if (!pw) { m.release(tok); complete = false; break; }
-            }
-            if (!begun) {
-                if (lane == 0) uval = op.begin((unsigned long long)bu);
-                uval = __shfl_sync(0xFFFFFFFFu, uval, 0);
-                begun = true;
+                held_w = pw != nullptr;
+                if (!held_w) { pw = m.through(w_off + 4ull * first); if (lane == 0) direct += 4ull * (unsigned long long)(last - first); }
             }
             found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, bu, uval, first, last, lane, pos);
-            if (WEIGHTED) m.release(tok_w);
-            m.release(tok);
+            if (held_w) m.release(tok_w);
+            if (held) m.release(tok);
             first = last;
         }
-        if (begun && !complete && lane == 0) op.redirty((unsigned long long)bu);   // the rest of its list waits for the next sweep
     }
+    for (int o = 16; o; o >>= 1) direct += __shfl_down_sync(0xFFFFFFFFu, direct, o);
+    if (lane == 0 && direct) m.note_direct(direct);
     return (int)found;
 }
 
@@ -701,6 +726,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
     const unsigned int n_chunks = (nv + 31) / 32;
     const long long epoch = sweep + 1;
     unsigned int found = 0, my_done = 0, iter = 0, next_chunk = 0, last_chunk = 0;
+    unsigned long long direct = 0;                           // bytes this lane read in place from the backing store
     for (;;) {
         // ---- a piece of a long neighbour list, if one is waiting (looked for before every kSpanPoll-th chunk)
         if ((iter++ & (kSpanPoll - 1)) == 0) {
@@ -751,14 +777,28 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
         // (one pin for all 33 when they lie in one unit, which they do except at unit ends and at the last chunk)
         long long lo, hi;
         const unsigned long long ob = off_off + 8ull * v0;
+        // a sparse sweep (few vertices left to expand, scattered over the graph) does not fetch pages: what is
+        // resident is read from its frame, the rest in place from the backing store
+        bool thru = false;
+        if constexpr (Op::kBehind) thru = op.through_main != 0;
         if (v0 + 32 <= nv && ob % unit + 33 * 8 <= unit) {
             gpuvm_token tok_o;
-            const unsigned char *po = m.pin(ob, GPUVM_READ, tok_o);
-            if (!po) break;
+            const unsigned char *po = thru ? m.pin_if_resident(ob, tok_o) : m.pin(ob, GPUVM_READ, tok_o);
+            const bool held = po != nullptr;
+            if (!held) {
+                if (!thru) break;
+                po = m.through(ob);
+                if (lane == 0) direct += 33 * 8;
+            }
             lo = Mem::load_i64(po + 8 * lane);
             hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
             if (lane == 31) hi = Mem::load_i64(po + 8 * 32);
-            m.release(tok_o);
+            if (held) m.release(tok_o);
+        } else if (thru) {
+            lo = Mem::load_i64(m.through(off_off + 8ull * (v < nv ? v : nv)));
+            hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+            if (lane == 31) hi = Mem::load_i64(m.through(off_off + 8ull * (v + 1 < nv ? v + 1 : nv)));
+            if (lane == 0) direct += 33 * 8;
         } else {
             lo = m.template read<long long>(off_off, v < nv ? v : nv);
             hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
@@ -817,12 +857,21 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
             unsigned int touch = __ballot_sync(0xFFFFFFFFu, lo < last && hi > first);
             if (touch) {
                 gpuvm_token tok, tok_w;
-                const unsigned char *p = m.pin(byte, GPUVM_READ, tok);
-                if (!p) { failed = true; break; }
+                const unsigned char *p = thru ? m.pin_if_resident(byte, tok) : m.pin(byte, GPUVM_READ, tok);
+                const bool held = p != nullptr;
+                if (!held) {
+                    if (!thru) { failed = true; break; }
+                    p = m.through(byte);
+                }
                 const unsigned char *pw = nullptr;
+                bool held_w = false;
                 if (WEIGHTED) {
-                    pw = m.pin(w_off + 4ull * first, GPUVM_READ, tok_w);
-                    if (!pw) { m.release(tok); failed = true; break; }
+                    pw = thru ? m.pin_if_resident(w_off + 4ull * first, tok_w) : m.pin(w_off + 4ull * first, GPUVM_READ, tok_w);
+                    held_w = pw != nullptr;
+                    if (!held_w) {
+                        if (!thru) { m.release(tok); failed = true; break; }
+                        pw = m.through(w_off + 4ull * first);
+                    }
                 }
                 const unsigned int pos = Op::kBehind ? sweep_pos(counters, n_chunks) : 0u;
                 while (touch) {
@@ -833,9 +882,10 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
                     if (blo < first) blo = first;
                     if (bhi > last) bhi = last;
                     found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, (long long)(v0 + L), bval, blo, bhi, lane, pos);
+                    if (lane == 0) direct += 4ull * (unsigned long long)(bhi - blo) * ((held ? 0u : 1u) + (WEIGHTED && !held_w ? 1u : 0u));
                 }
-                if (WEIGHTED) m.release(tok_w);
-                m.release(tok);
+                if (held_w) m.release(tok_w);
+                if (held) m.release(tok);
             }
             first = last;
         }
@@ -843,6 +893,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
     if (lane == 0 && found) atomicAdd(counters + kCntUpdates, found);
+    if (lane == 0 && direct) m.note_direct(direct);
 }
 
 // Balanced CSR (Section 5.2, Fig. 8): the edge array is cut into chunks of equal length and a
@@ -1376,8 +1427,13 @@ constexpr size_t kBfsScratchBytes = 4 * kBigQueue * sizeof(long long) + kCntWord
 // Scratch of the sweeps: queue of pieces, counters, then (label-correcting runs) the queue of vertices
 // lowered behind the sweep position.
 constexpr size_t kBehindMin = 1u << 16;
-size_t behind_capacity(size_t nv) { return nv / 4 > kBehindMin ? nv / 4 : kBehindMin; }
-size_t lc_scratch_bytes(size_t nv) { return kBfsScratchBytes + behind_capacity(nv) * sizeof(unsigned int); }
+size_t behind_capacity(size_t nv, bool weighted)
+{
+    // with weights a vertex is lowered several times per sweep (every shorter path found), with unit lengths about once
+    const size_t want = weighted ? nv / 2 : nv / 4;
+    return want > kBehindMin ? want : kBehindMin;
+}
+size_t lc_scratch_bytes(size_t nv, bool weighted) { return kBfsScratchBytes + behind_capacity(nv, weighted) * sizeof(unsigned int); }
 
 // One sweep and its update count.  `sweep` counts from 0 within a call.
 template <class Mem, class Op, bool WEIGHTED>
@@ -1430,7 +1486,7 @@ int bfs_levels(const Mem &m, size_t off_off, size_t col_off, size_t nv, size_t s
 }
 
 // Label-correcting sweeps until nothing changes (BFS: unit lengths; SSSP: the weights at w_off).  d_dist holds
-// the packed words while the sweeps run and the distances afterwards.  scratch: lc_scratch_bytes(nv).
+// the packed words while the sweeps run and the distances afterwards.  scratch: lc_scratch_bytes(nv, WEIGHTED).
 // *max_dist receives the largest distance reached.
 template <class Mem, bool WEIGHTED>
 int lc_sweeps(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t nv, size_t source, int32_t *d_dist,
@@ -1438,7 +1494,10 @@ int lc_sweeps(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t
 {
     unsigned int *counters = reinterpret_cast<unsigned int *>(static_cast<long long *>(scratch) + 4 * kBigQueue);
     unsigned int *behind_q = counters + kCntWords;
-    const unsigned int cap = (unsigned int)behind_capacity(nv);
+    // Over plain pointers (the managed-memory twin) the queue is off: re-expanding vertices at random places
+    // behind the sweep is only cheap when one can ask whether their pages are resident, which a plain pointer
+    // cannot; there the vertices simply stay dirty for the next sweep.
+    const unsigned int cap = Mem::kBehindQueue ? (unsigned int)behind_capacity(nv, WEIGHTED) : 0u;
     lc_init_kernel<<<sm_count() * 4, 256, 0, s>>>(d_dist, (unsigned int)nv, (unsigned int)source);
     int rc = launched();
     int sweep = 0;
@@ -1449,8 +1508,11 @@ int lc_sweeps(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t
         // one dirty vertex it would be over before that vertex's neighbours are lowered, and they would all count
         // as "behind".)  The second one runs upwards again, from the pages the first one left; then they alternate.
         const int backward = sweep == 0 ? 0 : (sweep - 1) & 1;
+        // A sweep that follows one with few updates has little to expand, scattered over the whole graph: it reads
+        // what it needs in place instead of fetching a page per vertex (see sparse_sweep).
+        const int sparse = sweep >= 2 && m.sparse_sweep(updates);
         const LcOp<WEIGHTED> op{d_dist, behind_q, counters, cap, (unsigned int)((nv + 31) / 32), backward,
-                                sweep == 0 ? (unsigned int)source : kNoVertex};
+                                sweep == 0 ? (unsigned int)source : kNoVertex, sparse};
         rc = graph_sweep<Mem, LcOp<WEIGHTED>, WEIGHTED>(m, op, off_off, col_off, w_off, nv, scratch, sweep, &updates, s, backward);
         ++sweep;
     }
@@ -1566,7 +1628,7 @@ int run_sssp(const Mem &m, size_t off_off, size_t col_off, size_t w_off, size_t 
     if (!d_dist || nv == 0 || source >= nv || nv > 0x7FFFFFFFull) return GPUVM_E_ARG;
     if (off_off % 16 || col_off % 16 || w_off % 16) return GPUVM_E_ALIGN;
     if ((w_off > col_off ? w_off - col_off : col_off - w_off) % m.unit_host() != 0) return GPUVM_E_ALIGN;
-    if (!scratch) return GPUVM_E_ALLOC;          // lc_scratch_bytes(nv)
+    if (!scratch) return GPUVM_E_ALLOC;          // lc_scratch_bytes(nv, true)
     return lc_sweeps<Mem, true>(m, off_off, col_off, w_off, nv, source, d_dist, 0x7FFFFFFF, n_rounds, nullptr, scratch, s);
 }
 
@@ -1713,7 +1775,7 @@ int gpuvm_bfs_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t nv, size_t s
     Paged m;
     if (!view_of(h, m)) return GPUVM_E_ARG;
     hint_edges(h, m, off_off, nv);
-    return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, gpuvm_scratch_(h, lc_scratch_bytes(nv)),
+    return run_bfs(m, off_off, col_off, nv, source, d_level, n_levels, gpuvm_scratch_(h, lc_scratch_bytes(nv, false)),
                    static_cast<cudaStream_t>(stream));
 }
 
@@ -1791,7 +1853,7 @@ int gpuvm_sssp_csr(gpuvm_t h, size_t off_off, size_t col_off, size_t w_off, size
     // column and weight page of an edge range are held together: two frames per warp of the grid
     if (gpuvm_safe_warps(h, 2) < sm_count() * 2 * 8) return GPUVM_E_FRAMES;
     hint_edges(h, m, off_off, nv);
-    return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, gpuvm_scratch_(h, lc_scratch_bytes(nv)),
+    return run_sssp(m, off_off, col_off, w_off, nv, source, d_dist, n_rounds, gpuvm_scratch_(h, lc_scratch_bytes(nv, true)),
                     static_cast<cudaStream_t>(stream));
 }
 
@@ -1953,7 +2015,7 @@ int gpuvm_raw_bfs_csr(const int64_t *row_off, const int32_t *col, size_t nv, siz
     unsigned char *base = ro < co ? ro : co;
     if ((ro - base) % 16 || (co - base) % 16) return GPUVM_E_ALIGN;
     Raw m{base, 65536};
-    Scratch scratch(lc_scratch_bytes(nv));
+    Scratch scratch(lc_scratch_bytes(nv, false));
     return run_bfs(m, (size_t)(ro - base), (size_t)(co - base), nv, source, d_level, n_levels, scratch.p,
                    static_cast<cudaStream_t>(stream));
 }
@@ -1982,7 +2044,7 @@ int gpuvm_raw_sssp_csr(const int64_t *row_off, const int32_t *col, const int32_t
     RawH m;
     m.base = base;
     m.unit_bytes = 65536;
-    Scratch scratch(lc_scratch_bytes(nv));
+    Scratch scratch(lc_scratch_bytes(nv, true));
     return run_sssp(m, (size_t)(ro - base), (size_t)(co - base), (size_t)(we - base), nv, source, d_dist, n_rounds,
                     scratch.p, static_cast<cudaStream_t>(stream));
 }

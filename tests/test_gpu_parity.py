@@ -431,6 +431,36 @@ def test_write_back_off_the_fault_path(B, page, n, frames, ahead, policy, form):
     assert st["bytes_out"] == (st["writebacks"] + st["cleaned"] + st["flush_writebacks"]) * page
 
 
+@pytest.mark.parametrize("frames", [1, 6, 64])
+def test_fenced_release_gives_the_same_results(B, frames):
+    """The batched engine normally releases the pages of read-only requests through a data dependency on
+    what was read; with GPUVM_DEBUG_FENCED_RELEASE it uses a warp barrier and a fence instead (the form
+    the memory model orders by itself).  Both must give the oracle's results, bit for bit."""
+    import torch
+    page, n, n_idx, dims, bag, n_bags = 4096, 1 << 16, 20000, 128, 8, 100
+    x = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(2))
+    idx = inputs.fill_index_i64(np.empty(n_idx, np.int64), n_idx, inputs.config_seed(2, 1), n)
+    rows = inputs.fill_zipf_rows(np.empty(n_bags * bag, np.int64), n_bags * bag, inputs.config_seed(5, 1), n // dims, 1.05)
+    ar = Arena(page, {"x": x})
+    nb = (n_idx + 1023) // 1024
+    ref_f, ref_b = oracle.gather_block_sums_direct(x, idx, 1024)
+    ref_e = oracle.embag_f32_direct(x.reshape(n // dims, dims), rows, bag).reshape(-1)
+    for flags in (0, B.DEBUG_FENCED_RELEASE, B.DEBUG_FENCED_RELEASE | B.DEBUG_POISON):
+        fs = torch.zeros(nb, dtype=torch.float32, device="cuda")
+        bs = torch.zeros(nb, dtype=torch.int64, device="cuda")
+        out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
+        with paged(ar.host, page, frames) as h:
+            B.gpuvm_set_debug(h, flags)
+            assert B.gpuvm_device_view(h).debug == flags
+            B.gpuvm_gather_f32(h, 0, dev(idx), n_idx, 1024, fs, bs)
+            B.gpuvm_embag_f32(h, 0, dims, dev(rows), n_bags, bag, out)
+            finish(h)
+        assert np.array_equal(bs.cpu().numpy(), ref_b), flags
+        got = fs.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref_f) <= 1e-6 * np.maximum(np.abs(ref_f), 2.0 ** -10))
+        assert np.array_equal(out.cpu().numpy().view(np.uint32), ref_e.view(np.uint32)), flags
+
+
 def test_two_kernels_share_mappings(B):
     """Mappings persist across launches: a read-only pass after a write pass sees the
     written values without any flush in between."""
