@@ -125,8 +125,8 @@ class ClockSampler:
 NCU_LINK_TRAFFIC = {
     1: (2097152 * 32, "stream_sum_kernel_cfg1_full_set.md", 2097152, "full size"),
     2: (33554432 * 32, "gather_batch_kernel_cfg2_full_set.md", 33554432, "full size"),
-    3: (37699584 * 32, "graph_sweep_kernel_lc_cfg3_sweep1_full_set.md", 37699584,
-        "full size; sweep 1 of the five sweeps of a run, 85 % of its time"),
+    3: (38354055 * 32, "graph_sweep_kernel_lc_cfg3_sweep1_full_set.md", 38354055,
+        "full size; sweep 1 of the four sweeps of a run, 95 % of its time"),
     4: (33554432 * 32 * 8 + (4 << 30), "vadd_kernel_cfg4_eighth_full_set.md", 33554432,
         "1/8 case x 8: 8 GiB in, plus the 4 GiB of c that go out"),
     5: (134217728 * 32 * 16, "embag_batch_kernel_cfg5_sixteenth_full_set.md", 134217728, "1/16 case x 16"),
