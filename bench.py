@@ -36,6 +36,7 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+DEFAULT_INPLACE_DIVISOR = 4          # the library's default (include/gpuvm.h, gpuvm_set_inplace_divisor)
 METRIC = "effective_app_GBps"
 UNIT = "GB/s"
 
@@ -129,7 +130,8 @@ NCU_LINK_TRAFFIC = {
         "full size; sweep 1 of the four sweeps of a run, 95 % of its time"),
     4: (33554432 * 32 * 8 + (4 << 30), "vadd_kernel_cfg4_eighth_full_set.md", 33554432,
         "1/8 case x 8: 8 GiB in, plus the 4 GiB of c that go out"),
-    5: (134217728 * 32 * 16, "embag_batch_kernel_cfg5_sixteenth_full_set.md", 134217728, "1/16 case x 16"),
+    "5_always_migrate": (134217728 * 32 * 16, "embag_batch_kernel_cfg5_sixteenth_full_set.md", 134217728,
+                         "1/16 case x 16, every first touch fetching its page"),
     6: (37758976 * 32, "graph_sweep_kernel_cc_cfg6_full_set.md", 37758976, "full size"),
 }
 
@@ -411,6 +413,44 @@ def e2e_step(torch, B, w, cfg: int):
     return e0.elapsed_time(e1) / 1e3, h2d, d2h
 
 
+def embag_policy_records(torch, B, w, args, link: dict, kern_s: float, direct: float, rec: dict) -> dict:
+    """cfg 5 runs with the library's rent-or-buy default (a page is fetched once its rows have moved a quarter of
+    its size in place).  Reported beside it: the ceiling of scattered row reads over this backing store, measured
+    here, which bounds the rows read in place; and the same launch with the policy off (the paper's way: every
+    first touch fetches the page), with its own link roofline."""
+    out = {}
+    row_bytes = 4 * w.dims
+    buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    scattered = B.gpuvm_link_peak_scattered(B.gpuvm_host_ptr(w.h), w.nbytes, row_bytes, 1 << 22, buf.data_ptr(), buf.numel())
+    del buf
+    out["in_place"] = {
+        "bytes": direct, "gbs": direct / kern_s / 1e9 if kern_s else 0.0, "scattered_read_peak_gbs": scattered,
+        "frac": direct / kern_s / 1e9 / scattered if kern_s and scattered else None,
+        "what": f"rows read in place from the backing store; the peak is {1 << 22} rows of {row_bytes} B at hashed "
+                f"positions of the same {w.nbytes >> 30} GiB region, four in flight per warp, measured in this run"}
+    if args.inplace_divisor < 0 and not args.scratch_limit_mib:
+        B.gpuvm_set_inplace_divisor(w.h, 0)
+        try:
+            w.run(check=False)
+            rs = [w.run(check=True) for _ in range(2)]
+        finally:
+            B.gpuvm_set_inplace_divisor(w.h, DEFAULT_INPLACE_DIVISOR)
+        secs = sum(r.seconds for r in rs) / len(rs)
+        ks = sum(r.kernel_seconds for r in rs) / len(rs)
+        st = rs[-1].stats
+        roof = link_roofline(st["bytes_in"], st["bytes_out"], ks, link)
+        traffic = NCU_LINK_TRAFFIC.get("5_always_migrate") if args.shrink == 0 else None
+        roof["traffic"] = traffic[0] if traffic else None
+        roof["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[3]}): host-link bytes of one launch counted by ncu"
+                                  if traffic else None)
+        out["always_migrate"] = {
+            "what": "gpuvm_set_inplace_divisor(h, 0): every first touch fetches the page, as in the paper",
+            "ms_per_step": secs * 1e3, "value": rs[-1].effective_bytes / secs / 1e9, "unit": UNIT, "steps": len(rs),
+            "faults": st["faults"], "bytes_in": st["bytes_in"], "in_gbs": st["bytes_in"] / secs / 1e9,
+            "invariants_status": rs[-1].check["status"], "roofline": roof}
+    return out
+
+
 def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link: dict, dist, world: int,
                local_rank: int, rank: int, barrier) -> dict:
     """All measurements of one workload: K timed cold steps, the end-to-end steps, the run under a
@@ -420,6 +460,8 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
     try:
         if args.scratch_limit_mib:
             B.gpuvm_set_scratch_limit(w.h, args.scratch_limit_mib << 20)
+        if args.inplace_divisor >= 0:
+            B.gpuvm_set_inplace_divisor(w.h, args.inplace_divisor)
         for _ in range(warmup):
             w.run(check=False)
         sampler = ClockSampler(local_rank, args.clock_period)
@@ -479,6 +521,10 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
             pages = w.compulsory_pages()
             rec["roofline"]["compulsory_pages"] = pages
             rec["roofline"]["frac_compulsory"] = pages * w.page_bytes / kern_s / 1e9 / link["ce_h2d_gbs"]
+        if cfg == 5:
+            rec["migration"]["inplace_divisor"] = args.inplace_divisor if args.inplace_divisor >= 0 else DEFAULT_INPLACE_DIVISOR
+        if cfg == 5 and rank == 0:
+            rec["roofline"].update(embag_policy_records(torch, B, w, args, link, kern_s, direct, rec))
         if cfg in (2, 5) and not args.scratch_limit_mib:
             # the same workload with its scratch bounded to an eighth of the pool: fewer requests in flight
             # per warp, so a page serves fewer of them per visit and is fetched more often
@@ -570,6 +616,8 @@ def main():
     ap.add_argument("--scratch-limit-mib", type=int, default=0,
                     help="bound of the workload's device scratch (request tables, staged rows); 0 = none. Less scratch "
                          "means fewer page requests in flight per warp and more faults")
+    ap.add_argument("--inplace-divisor", type=int, default=-1,
+                    help="rent-or-buy divisor of the batched row workloads (cfg 5): -1 = the library's default, 0 = off")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-replay", action="store_true", help="skip the oracle's sequential replay counts (cfg 3 and 5)")
     ap.add_argument("--clock-period", type=float, default=0.1, help="seconds between NVML clock samples")

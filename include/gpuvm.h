@@ -226,6 +226,20 @@ int gpuvm_set_clean_ahead(gpuvm_t h, unsigned int frames);
 int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes);
 size_t gpuvm_scratch_bytes(gpuvm_t h);
 
+/* Rent or buy (not in the paper, which fetches a page at its first fault).  The batched row workloads
+ * (gpuvm_embag_f32) do not fetch a page for its first requests: while the requests served from a page since it
+ * was last resident have read less than page_bytes / divisor over the link, the next one reads its row in place
+ * from the backing store (pinned host memory is as reachable for a load as for a page copy) and the page stays
+ * where it is; the request after that fetches it.  A page that is asked for a few times never costs a page of
+ * traffic; one that turns out hot costs at most 1 / divisor more than if it had been fetched at once.  Counted in
+ * gpuvm_stats as bytes_direct.  Only for reads, and only right for data that is not written through the
+ * runtime while such a kernel runs.  divisor: default 4; 0 = off (every first touch fetches the page).
+ * Why 4 and not 1 (the break-even point by bytes): a row read in place is a scattered link read, and over a
+ * 64 GiB backing store those were measured at 24.5 GB/s however many were in flight (51.4 GB/s over 1 GiB, 33.4
+ * over 8 GiB: address translation on the host side), while page copies run at 51.4 GB/s beside them; the two
+ * streams finish together near a quarter (measured on the 64 GiB Zipf table: 70 / 61 / 77 ms for 2 / 4 / 8). */
+int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor);
+
 /* Largest number of simultaneously resident warps that can each hold
  * `pins_per_warp` pages pinned without exhausting the pool (a warp that holds
  * pins while faulting needs a free frame; Section 3.3: a frame is reused only

@@ -93,6 +93,7 @@ struct gpuvm_fault_queue {
 namespace gpuvm {
 
 constexpr unsigned int kNotReady = 0xFFFFFFFFu;   /* "frame" values a leader hands to its followers */
+constexpr unsigned int kInPlaceFrame = 0xFFFFFFFEu; /* the group reads from the backing store, it holds no reference */
 constexpr unsigned int kRejected = 0xFFFFFFFFu;   /* vpn of a request that was refused when it was set */
 
 /* Any lane.  False when the ring is (nearly) full: the caller keeps the fault and retries. */
@@ -343,6 +344,19 @@ __host__ __device__ __forceinline__ unsigned int gpuvm_batch_mask_words(unsigned
     return 2u * ((((n + 31u) >> 5) + 63u) >> 6);
 }
 
+/*
+ * A consume "function" for WARP_CONSUME that the engine carries out itself: request i asks for a row of
+ * units16 x 16 bytes (at most 32 units), which goes to dst + i * units16 (in 16-byte units; ordinary device
+ * memory).  Because the engine knows what is to be done it can have the rows of four requests in flight at
+ * a time (four loads per lane, then four stores), which is what the rows that are read in place from the
+ * backing store need: one such read takes a link round trip.
+ */
+struct gpuvm_row_copy {
+    uint4 *dst;
+    unsigned int units16;
+    __device__ __forceinline__ unsigned int operator()(unsigned int, const unsigned char *) const { return 0u; }   /* (never called) */
+};
+
 namespace gpuvm {
 /* call a consume function; what a non-void one returns is folded into `dep` */
 template <class Consume>
@@ -357,10 +371,13 @@ template <bool WARP_CONSUME, class Table, class Consume>
 static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm, const Table table, unsigned int n,
                                                             int mode, Consume consume, gpuvm_fault_queue *queue,
                                                             unsigned long long *masks, unsigned int mask_stride,
-                                                            bool eager_push = false)
+                                                            bool eager_push = false, unsigned int inplace_limit = 0,
+                                                            unsigned int inplace_bytes = 0)
 {
     using namespace gpuvm;
     const unsigned int lane = lane_id();
+    if (mode != kRead) inplace_limit = 0;                   /* only reads can be served from the backing store */
+    unsigned int n_inplace = 0;                             /* this lane's requests served in place */
     const unsigned int rows = (n + 31) >> 5;
     const unsigned int words = (rows + 63) >> 6;
     unsigned long long *const m_todo = masks, *const m_own = masks + (size_t)words * mask_stride;
@@ -379,7 +396,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
      */
     auto visit = [&](unsigned int k, unsigned int j0, unsigned int jn, bool first, unsigned long long &todo,
                      unsigned long long &own) -> bool {
-        unsigned int rowmask[R], vpn[R], off[R], leader[R], any = 0;
+        unsigned int rowmask[R], vpn[R], off[R], leader[R], gsize[R], any = 0;
         unsigned long long word[R];
         bool progress = false;
 #pragma unroll
@@ -402,10 +419,11 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
         }
 #pragma unroll
         for (int u = 0; u < R; ++u) {
-            leader[u] = 32; word[u] = 0;
+            leader[u] = 32; word[u] = 0; gsize[u] = 1;
             if ((rowmask[u] >> lane) & 1u) {
                 const unsigned int group = __match_any_sync(rowmask[u], vpn[u]);
                 leader[u] = __ffs(group) - 1;
+                gsize[u] = __popc(group);
                 if (lane == leader[u]) {
                     if (first) {
                         word[u] = pin_acquire(vm.pte + vpn[u]) + 1ull;
@@ -433,11 +451,14 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                 const bool looks_valid = (w & kStMask) == kValid;
                 if (!first && GPUVM_BATCH_ACQ == 1 && looks_valid) w = ld_acquire_u64(vm.pte + vpn[u]);
                 unsigned int f;
-                const int st = advance(vm, vm.pte + vpn[u], w, mode, f);
+                const int st = advance(vm, vm.pte + vpn[u], w, mode, f, inplace_limit, gsize[u]);
                 if (st == kReady) {
                     frame[u] = f;
                     need_fence |= GPUVM_BATCH_ACQ == 2 || (GPUVM_BATCH_ACQ == 1 && !looks_valid);
                     if (first) ++n_hits;
+                } else if (st == kInPlace) {
+                    frame[u] = kInPlaceFrame;           /* served from the backing store; the reference is gone already */
+                    n_inplace += gsize[u];
                 } else if (st == kOwn) {
                     if (!(first && eager_push && queue && fault_queue_push(queue, vpn[u], mode, &vm))) own |= bit;
                     progress = true;
@@ -456,17 +477,52 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
             const bool mine = ((rowmask[u] >> lane) & 1u) != 0;
             if (mine) frame[u] = __shfl_sync(rowmask[u], frame[u], leader[u]);
             const bool ready = mine && frame[u] != kNotReady;
-            if (WARP_CONSUME) {
+            if constexpr (WARP_CONSUME && std::is_same<Consume, gpuvm_row_copy>::value) {
+                unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
+                while (ready_lanes) {
+                    constexpr int Q = 4;                    /* rows in flight per warp */
+                    const unsigned char *src[Q];
+                    unsigned int idx[Q];
+                    uint4 v[Q];
+                    int cnt = 0;
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) {
+                        src[q] = nullptr; idx[q] = 0;
+                        if (ready_lanes) {
+                            const unsigned int L = __ffs(ready_lanes) - 1;
+                            ready_lanes &= ready_lanes - 1;
+                            const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame[u], L), o = __shfl_sync(0xFFFFFFFFu, off[u], L);
+                            const unsigned int pv = __shfl_sync(0xFFFFFFFFu, vpn[u], L);
+                            src[q] = (f == kInPlaceFrame ? vm.host + ((unsigned long long)pv << vm.page_shift)
+                                                         : vm.pool + ((unsigned long long)f << vm.page_shift)) + o;
+                            idx[q] = (64u * k + j0 + u) * 32 + L;
+                            cnt = q + 1;
+                        }
+                    }
+                    if (lane < consume.units16) {
+#pragma unroll
+                        for (int q = 0; q < Q; ++q)
+                            if (q < cnt) v[q] = gpuvm_load16(src[q] + 16u * lane);
+#pragma unroll
+                        for (int q = 0; q < Q; ++q)
+                            if (q < cnt) { consume.dst[(size_t)idx[q] * consume.units16 + lane] = v[q]; dep ^= v[q].x; }
+                    }
+                }
+            } else if (WARP_CONSUME) {
                 unsigned int ready_lanes = __ballot_sync(0xFFFFFFFFu, ready);
                 while (ready_lanes) {
                     const unsigned int L = __ffs(ready_lanes) - 1;
                     ready_lanes &= ready_lanes - 1;
                     const unsigned int f = __shfl_sync(0xFFFFFFFFu, frame[u], L), o = __shfl_sync(0xFFFFFFFFu, off[u], L);
-                    call_consume(consume, (64u * k + j0 + u) * 32 + L, vm.pool + ((unsigned long long)f << vm.page_shift) + o, dep);
+                    const unsigned int pv = __shfl_sync(0xFFFFFFFFu, vpn[u], L);
+                    const unsigned char *src = f == kInPlaceFrame ? vm.host + ((unsigned long long)pv << vm.page_shift)
+                                                                  : vm.pool + ((unsigned long long)f << vm.page_shift);
+                    call_consume(consume, (64u * k + j0 + u) * 32 + L, src + o, dep);
                 }
             } else if (ready) {
-                call_consume(consume, (64u * k + j0 + u) * 32 + lane,
-                             vm.pool + ((unsigned long long)frame[u] << vm.page_shift) + off[u], dep);
+                const unsigned char *src = frame[u] == kInPlaceFrame ? vm.host + ((unsigned long long)vpn[u] << vm.page_shift)
+                                                                     : vm.pool + ((unsigned long long)frame[u] << vm.page_shift);
+                call_consume(consume, (64u * k + j0 + u) * 32 + lane, src + off[u], dep);
             }
             any_ready |= ready;
         }
@@ -491,7 +547,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                 if (((rowmask[u] >> lane) & 1u) && frame[u] != kNotReady) {
                     todo &= ~(1ull << (j0 + u));
                     ++served;
-                    if (lane == leader[u]) atomicAdd(vm.pte + vpn[u], ~0ull + hold);
+                    if (lane == leader[u] && frame[u] != kInPlaceFrame) atomicAdd(vm.pte + vpn[u], ~0ull + hold);
                 }
             }
             progress = true;
@@ -608,8 +664,10 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
         n_hits += __shfl_down_sync(0xFFFFFFFFu, n_hits, o);
         n_waits += __shfl_down_sync(0xFFFFFFFFu, n_waits, o);
         n_lanes += __shfl_down_sync(0xFFFFFFFFu, n_lanes, o);
+        n_inplace += __shfl_down_sync(0xFFFFFFFFu, n_inplace, o);
     }
     if (lane == 0) {
+        if (n_inplace) stat_add(vm, kBytesDirect, (unsigned long long)n_inplace * inplace_bytes);
         if (GPUVM_COUNT_HITS && n_hits) stat_add(vm, kHits, n_hits);
         if (n_waits) stat_add(vm, kWaits, n_waits);
         if (n_lanes) stat_add(vm, kLanes, n_lanes);

@@ -69,7 +69,8 @@
 
 namespace gpuvm {
 
-/* ---- page-table entry: [state:2 @60][dirty @57][ref @56][frame:32 @24][refcount:24 @0] */
+/* ---- page-table entry: [state:2 @60][dirty @57][ref @56][frame:32 @24][refcount:24 @0]
+ *      (while the state is INVALID the frame field counts the requests served in place, see advance) */
 constexpr unsigned long long kRcMask = 0xFFFFFFull;
 constexpr unsigned long long kRcLimit = 1ull << 23;   /* a pin that would take the counter beyond this is refused */
 constexpr unsigned long long kPinRefused = ~0ull;     /* what a refused pin hands to its group instead of the entry */
@@ -428,15 +429,26 @@ __device__ __forceinline__ void publish(const gpuvm_dev_t &vm, unsigned long lon
 
 /* ------------------------------------------------------------ fault machinery */
 
-enum LaneState { kNew = 0, kWait, kOwn, kReady, kDone, kFail };
+enum LaneState { kNew = 0, kWait, kOwn, kReady, kDone, kFail, kInPlace };
 
 /*
  * Leader only.  `w` is a fresh value of the entry that includes this group's
  * reference.  VALID: note the reference/dirty bits, READY.  BUSY or EVICTING:
  * WAIT.  INVALID: try to become the owner (step 4).
+ *
+ * Rent or buy.  With inplace_limit != 0 (read mode only) a page that is not resident is not
+ * fetched for its first requests: while fewer than inplace_limit requests have been served from it
+ * since it was last resident, this one is counted (in the frame field of the entry, which means
+ * nothing while the entry is INVALID), gives its reference back in the same compare-and-swap and
+ * returns IN PLACE: the caller reads what it wants from the backing store, which is current for a
+ * page that is not resident.  Only when a page has been asked for often enough that its requests
+ * have moved a stated fraction of its size over the link does the next request fetch it.  Pages
+ * that are touched a few times never cost a page of traffic; a page that turns out hot costs at
+ * most that fraction more than if it had been fetched at once.
  */
 __device__ __forceinline__ int advance(const gpuvm_dev_t &vm, unsigned long long *pte,
-                                       unsigned long long w, int mode, unsigned int &frame)
+                                       unsigned long long w, int mode, unsigned int &frame,
+                                       unsigned int inplace_limit = 0, unsigned int weight = 1)
 {
     for (;;) {
         unsigned long long st = w & kStMask;
@@ -448,9 +460,18 @@ __device__ __forceinline__ int advance(const gpuvm_dev_t &vm, unsigned long long
             return kReady;
         }
         if (st != kInvalid) return kWait;
-        unsigned long long seen = atomicCAS(pte, w, w | kBusy);
-        if (seen == w) return kOwn;
-        w = seen;                      /* somebody pinned, unpinned or took ownership */
+        unsigned long long next;
+        int result;
+        if (inplace_limit != 0u && ((w & kFrameMask) >> kFrameShift) < inplace_limit) {
+            next = w + ((unsigned long long)weight << kFrameShift) - 1ull;      /* count it, drop the reference */
+            result = kInPlace;
+        } else {
+            next = (w & ~kFrameMask) | kBusy;               /* ours to fetch; the count starts over */
+            result = kOwn;
+        }
+        unsigned long long seen = atomicCAS(pte, w, next);
+        if (seen == w) return result;
+        w = seen;                      /* somebody pinned, unpinned, counted or took ownership */
     }
 }
 
@@ -907,7 +928,7 @@ static __device__ __noinline__ void gpuvm_prefetch(const gpuvm_dev_t vm, unsigne
     bool vdirty = false;
     if (lane == L) {
         const unsigned long long w = ld_relaxed_u64(pte);
-        if ((w & kStMask) == kInvalid && atomicCAS(pte, w, w | kBusy) == w) {
+        if ((w & kStMask) == kInvalid && atomicCAS(pte, w, (w & ~kFrameMask) | kBusy) == w) {
             go = try_claim(vm, vpn, 8, h, victim, vdirty, /* allow_dirty = */ false) ? 1 : 0;
             if (!go) atomicXor(pte, kBusy);                       /* no frame at hand: BUSY -> INVALID */
         }

@@ -300,6 +300,17 @@ int gpuvm_raw_embag_f32(const float *table, size_t dims, const int64_t *d_rows, 
  */
 int gpuvm_link_peak(void *host_ptr, void *d_buf, size_t bytes, int reps, double *out);
 
+/*
+ * The same link read as scattered rows: n_rows rows of row_bytes (a multiple of 16, at most 512) at hashed
+ * positions of the pinned region [host_ptr, host_ptr + host_bytes) are loaded by warps, four rows in flight
+ * each, and stored to the device buffer d_buf of d_bytes (reused round-robin).  out[0] = GB/s, best of `reps`.
+ * This is the ceiling of rows read in place from the backing store; it falls with the size of the region
+ * (measured on one host: 51.4 GB/s over 1 GiB, 33.4 over 8 GiB, 24.5 over 64 GiB, whatever the number of reads
+ * in flight).  out: host pointer to 1 double.  Synchronises.
+ */
+int gpuvm_link_peak_scattered(void *host_ptr, size_t host_bytes, size_t row_bytes, size_t n_rows, void *d_buf,
+                              size_t d_bytes, int reps, double *out);
+
 /* Number of kernels this library has launched in the calling process. */
 unsigned long long gpuvm_launch_count(void);
 

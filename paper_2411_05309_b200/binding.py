@@ -64,6 +64,7 @@ SYMBOLS = {
     "gpuvm_check_on": (_i, [_vp, ctypes.POINTER(Check), _vp]),
     "gpuvm_set_debug": (_i, [_vp, ctypes.c_uint]),
     "gpuvm_set_clean_ahead": (_i, [_vp, ctypes.c_uint]),
+    "gpuvm_set_inplace_divisor": (_i, [_vp, ctypes.c_uint]),
     "gpuvm_bcsr_build": (_i, [_vp, _sz, _sz, _vp, _sz, ctypes.POINTER(_sz)]),
     "gpuvm_device_view": (_i, [_vp, ctypes.POINTER(DevView)]),
     "gpuvm_host_ptr": (_vp, [_vp]),
@@ -105,6 +106,7 @@ SYMBOLS = {
     "gpuvm_raw_vadd_f32": (_i, [_vp, _vp, _vp, _sz, _vp]),
     "gpuvm_raw_embag_f32": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_link_peak": (_i, [_vp, _vp, _sz, _i, ctypes.POINTER(ctypes.c_double)]),
+    "gpuvm_link_peak_scattered": (_i, [_vp, _sz, _sz, _sz, _vp, _sz, _i, ctypes.POINTER(ctypes.c_double)]),
     "gpuvm_launch_count": (ctypes.c_ulonglong, []),
     "gpuvm_uvm_alloc": (_i, [ctypes.POINTER(_vp), _sz]),
     "gpuvm_uvm_free": (_i, [_vp]),
@@ -201,6 +203,10 @@ def gpuvm_check_on(h, stream, raise_on_error: bool = True) -> dict:
     d = c.as_dict()
     d["status"] = rc
     return d
+
+
+def gpuvm_set_inplace_divisor(h, divisor: int):
+    _check(lib().gpuvm_set_inplace_divisor(h, divisor), "gpuvm_set_inplace_divisor")
 
 
 def gpuvm_set_clean_ahead(h, frames: int):
@@ -438,6 +444,13 @@ def gpuvm_link_peak(host_ptr, d_buf, nbytes: int, reps: int = 3):
     out = (ctypes.c_double * 3)()
     _check(lib().gpuvm_link_peak(_ptr(host_ptr), _ptr(d_buf), nbytes, reps, out), "gpuvm_link_peak")
     return {"h2d_gbs": out[0], "d2h_gbs": out[1], "duplex_gbs": out[2]}
+
+
+def gpuvm_link_peak_scattered(host_ptr, host_bytes: int, row_bytes: int, n_rows: int, d_buf, d_bytes: int, reps: int = 2) -> float:
+    out = (ctypes.c_double * 1)()
+    _check(lib().gpuvm_link_peak_scattered(_ptr(host_ptr), host_bytes, row_bytes, n_rows, _ptr(d_buf), d_bytes, reps, out),
+           "gpuvm_link_peak_scattered")
+    return out[0]
 
 
 # ------------------------------------------------------------ managed-memory helpers

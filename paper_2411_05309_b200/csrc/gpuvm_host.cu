@@ -23,6 +23,7 @@ struct gpuvm_handle {
     void *scratch;                   // device scratch for workload kernels (request tables)
     size_t scratch_bytes;
     size_t scratch_limit;      /* 0: none */
+    unsigned int inplace_divisor;
 };
 
 namespace {
@@ -80,7 +81,7 @@ __global__ void check_kernel(gpuvm_dev_t vm, unsigned long long *out)
             else if (vm.frame_vpn[f] != (unsigned int)v) c[4]++;
             if (w & ~(kStMask | kDirty | kRef | kFrameMask | kRcMask)) c[2]++;
         } else if (st == kInvalid) {
-            if (w & ~kRcMask) c[2]++;
+            if (w & ~(kRcMask | kFrameMask)) c[2]++;        // (the frame field counts in-place reads while INVALID)
         } else {
             c[2]++;
         }
@@ -144,6 +145,7 @@ int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_byt
     memset(h, 0, sizeof(*h));
     cudaGetDevice(&h->device);
     h->sms = sm_count_of(h->device);
+    h->inplace_divisor = 4;
     cudaError_t e;
 
     // backing store: pinned and mapped (Section 4: the host region is registered before
@@ -334,6 +336,15 @@ int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes)
 }
 
 size_t gpuvm_scratch_bytes(gpuvm_t h) { return h ? h->scratch_bytes : 0; }
+
+size_t gpuvm_inplace_divisor_(gpuvm_handle *h) { return h ? h->inplace_divisor : 0; }
+
+int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor)
+{
+    if (!h) return GPUVM_E_ARG;
+    h->inplace_divisor = divisor;
+    return GPUVM_OK;
+}
 
 int gpuvm_device_view(gpuvm_t h, gpuvm_dev_t *out)
 {

@@ -14,6 +14,8 @@ struct gpuvm_handle;
 void *gpuvm_scratch_(struct gpuvm_handle *h, size_t bytes);
 /* bound set with gpuvm_set_scratch_limit, SIZE_MAX when there is none */
 size_t gpuvm_scratch_limit_(struct gpuvm_handle *h);
+/* divisor set with gpuvm_set_inplace_divisor (default 2; 0: requests are never served in place) */
+size_t gpuvm_inplace_divisor_(struct gpuvm_handle *h);
 #ifdef __cplusplus
 }
 #endif

@@ -1127,7 +1127,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                                                               unsigned int bag, float *__restrict__ out, int requesters,
                                                               gpuvm_batch_entry *g_tables, unsigned char *g_staging,
                                                               unsigned int groups, bool one_pass,
-                                                              gpuvm_shared_queue *shared_queue)
+                                                              gpuvm_shared_queue *shared_queue, unsigned int inplace_limit)
 {
     __shared__ gpuvm_fault_queue queue_s;
     __shared__ __align__(128) unsigned char stage_s[kEmbagMigrators][kEmbagChunk];   // bulk-copy staging of the migrator warps
@@ -1176,16 +1176,10 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                         gpuvm_batch_skip(table, (gi * nk + k) * 32 + lane);
                 }
             __syncwarp();
-            gpuvm_batch_run<true>(vm, gpuvm_entry_table{table}, groups * nk * 32, GPUVM_READ,
-                                         [=](unsigned int i, const unsigned char *p) {
-                unsigned int seen = 0;                             // read-only consume: lets the engine skip its fence
-                if (lane < q) {
-                    const uint4 v = gpuvm_load16(p + 16u * lane);
-                    staging[(size_t)i * q + lane] = v;
-                    seen = v.x;
-                }
-                return seen;
-            }, queue, masks, 1u, one_pass);
+            // every served row is copied to its slot of the staging area by the whole warp (the engine does it
+            // itself, four rows in flight: gpuvm_row_copy), from its frame or in place from the backing store
+            gpuvm_batch_run<true>(vm, gpuvm_entry_table{table}, groups * nk * 32, GPUVM_READ, gpuvm_row_copy{staging, q},
+                                  queue, masks, 1u, one_pass, inplace_limit, (unsigned int)row_bytes);
             __syncwarp();
             // add the staged rows of each bag in list order
             for (unsigned int gb = 0; gb < 32 * groups && g0 + gb < n_bags; ++gb) {
@@ -1314,6 +1308,33 @@ __global__ void link_in_kernel(const uint4 *__restrict__ src, uint4 *__restrict_
         for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < n16) v[u] = gpuvm::ld_host16(src + i); }
 #pragma unroll
         for (int u = 0; u < 8; ++u) { size_t i = base + u * stride; if (i < n16) gpuvm::st_frame16(dst + i, v[u]); }
+    }
+}
+
+// Scattered rows over the link: row i of the launch is row hash(seed, i) of the host region; a warp has four
+// rows in flight (16 bytes per lane and row).  What a workload that reads rows in place can reach at most.
+__global__ void link_scattered_kernel(const unsigned char *__restrict__ host, unsigned long long host_rows, unsigned int units16,
+                                      unsigned long long n_rows, unsigned long long seed, uint4 *__restrict__ dst,
+                                      unsigned long long dst_rows)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    const unsigned long long warp = (blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x) >> 5;
+    const unsigned long long warps = ((unsigned long long)gridDim.x * blockDim.x) >> 5;
+    const unsigned long long row_bytes = 16ull * units16;
+    for (unsigned long long i = warp * 4; i < n_rows; i += warps * 4) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            unsigned long long z = seed + (i + u) * 0x9E3779B97F4A7C15ull;       // splitmix64 of the row's index
+            z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+            z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+            z ^= z >> 31;
+            if (i + u < n_rows && lane < units16)
+                v[u] = gpuvm::ld_host16(reinterpret_cast<const uint4 *>(host + (z % host_rows) * row_bytes) + lane);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (i + u < n_rows && lane < units16) gpuvm::st_frame16(dst + ((i + u) % dst_rows) * units16 + lane, v[u]);
     }
 }
 
@@ -1914,10 +1935,17 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     unsigned char *scratch = static_cast<unsigned char *>(gpuvm_scratch_(h, table_bytes + staging_bytes + sizeof(gpuvm_shared_queue)));
     if (!scratch) return GPUVM_E_ALLOC;
     gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, scratch + table_bytes + staging_bytes, static_cast<cudaStream_t>(stream));
+    // Rent or buy: a page is fetched only once its rows have been asked for often enough to have moved a stated
+    // fraction of its size over the link (gpuvm_set_inplace_divisor; a quarter of it by default); until then its rows
+    // are read in place from the backing store.  A row is a whole number of 128-byte link reads when it is a
+    // multiple of 128 bytes long; shorter rows are charged 128 bytes.
+    const size_t divisor = gpuvm_inplace_divisor_(h);
+    const size_t charged = row_bytes < 128 ? 128 : row_bytes;
+    const unsigned int inplace_limit = divisor ? (unsigned int)(page_bytes / divisor / charged) : 0u;
     embag_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
         m.vm, t_off, (unsigned int)dims, reinterpret_cast<const long long *>(d_rows), n_bags, (unsigned int)bag, d_out,
         requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes, groups,
-        /* one_pass = */ items <= (size_t)grid * requesters && bag <= kEmbagLookups, shared_queue);
+        /* one_pass = */ items <= (size_t)grid * requesters && bag <= kEmbagLookups, shared_queue, inplace_limit);
     return launched();
 }
 
@@ -2098,6 +2126,37 @@ int gpuvm_link_peak(void *host_ptr, void *d_buf, size_t bytes, int reps, double 
     cudaEventDestroy(a);
     cudaEventDestroy(b);
     out[0] = best[0]; out[1] = best[1]; out[2] = best[2];
+    return GPUVM_OK;
+}
+
+int gpuvm_link_peak_scattered(void *host_ptr, size_t host_bytes, size_t row_bytes, size_t n_rows, void *d_buf, size_t d_bytes,
+                              int reps, double *out)
+{
+    if (!host_ptr || !d_buf || !out || row_bytes < 16 || row_bytes % 16 || row_bytes > 512 || host_bytes < row_bytes ||
+        d_bytes < row_bytes || n_rows == 0 || reps <= 0)
+        return GPUVM_E_ARG;
+    void *dh = nullptr;
+    if (cudaHostGetDevicePointer(&dh, host_ptr, 0) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_PIN; }
+    cudaEvent_t a, b;
+    cudaEventCreate(&a);
+    cudaEventCreate(&b);
+    double best = 0;
+    for (int r = 0; r <= reps; ++r) {
+        cudaEventRecord(a);
+        link_scattered_kernel<<<sm_count(), 1024>>>(static_cast<const unsigned char *>(dh), host_bytes / row_bytes,
+                                                    (unsigned int)(row_bytes / 16), n_rows, 0x5CA77E2ull + r,
+                                                    static_cast<uint4 *>(d_buf), d_bytes / row_bytes);
+        gpuvm_note_launch_(1);
+        cudaEventRecord(b);
+        if (cudaEventSynchronize(b) != cudaSuccess) { cudaGetLastError(); cudaEventDestroy(a); cudaEventDestroy(b); return GPUVM_E_CUDA; }
+        float ms = 0;
+        cudaEventElapsedTime(&ms, a, b);
+        const double gbs = (double)n_rows * row_bytes / (ms * 1e6);
+        if (r > 0 && gbs > best) best = gbs;                      // r == 0 is the warm-up
+    }
+    cudaEventDestroy(a);
+    cudaEventDestroy(b);
+    out[0] = best;
     return GPUVM_OK;
 }
 

@@ -353,7 +353,48 @@ def test_embag(B, page, n_rows, n_bags, frames, dims, bag, batched):
     got = out.cpu().numpy()
     assert np.all(np.abs(got.astype(np.float64) - ref) <= 1e-6 * np.maximum(np.abs(ref), 2.0 ** -10))
     assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))     # same order of additions: same bits
-    assert st["faults"] >= np.unique(rows * dims * 4 // page).size
+    # every looked-up row crossed the link, as part of a fetched page or read in place
+    touched = np.unique(rows * dims * 4 // page).size
+    assert st["faults"] * page + st["bytes_direct"] >= touched * min(page, 4 * dims)
+    if not batched:
+        assert st["bytes_direct"] == 0 and st["faults"] >= touched
+
+
+@pytest.mark.parametrize("frames", [1, 4, 64])
+def test_embag_rent_or_buy(B, frames):
+    """The batched embedding bag reads the first rows of a page in place and fetches the page only when its requests
+    have moved the stated fraction of its size (a quarter unless set otherwise): cold pages are never fetched, a hot page is fetched once after the stated number of
+    in-place reads, and with the divisor 0 every first touch fetches.  Results are exact either way."""
+    import torch
+    page, dims, bag = 4096, 128, 4                       # 8 rows per page; a quarter of a page = 2 rows
+    n_rows = 512
+    t = inputs.fill_f32_pm1(np.empty(n_rows * dims, np.float32), n_rows * dims, inputs.config_seed(5))
+    ar = Arena(page, {"t": t})
+    cold = np.arange(0, n_rows, 8, dtype=np.int64)[:64]                      # one row of each of 64 pages
+    hot = np.full(1024, 17, dtype=np.int64)                                   # one page, over and over
+    mixed = np.concatenate([cold, hot, cold + 1])
+    for rows, name in ((cold, "cold"), (hot, "hot"), (mixed, "mixed")):
+        n_bags = rows.size // bag
+        ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
+        for divisor in (None, 2, 0, 8):
+            out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
+            with paged(ar.host, page, frames) as h:
+                if divisor is None:
+                    divisor = 4                                                # the default
+                else:
+                    B.gpuvm_set_inplace_divisor(h, divisor)
+                B.gpuvm_embag_f32(h, 0, dims, dev(rows), n_bags, bag, out)
+                st, ck = finish(h)
+            assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32)), (name, divisor)
+            limit = page // divisor // 512 if divisor else 0                  # rows of a page that are read in place
+            if divisor == 0:
+                assert st["bytes_direct"] == 0 and st["faults"] >= np.unique(rows // 8).size
+            elif name == "cold":                                               # one row per page: below any limit
+                assert st["faults"] == 0 and st["bytes_direct"] == rows.size * 512
+            elif name == "hot":                                                # the page is bought after `limit` rows
+                assert st["faults"] >= 1
+                assert limit * 512 <= st["bytes_direct"] <= (limit + 31) * 512 * st["faults"]
+            assert st["bytes_direct"] % 512 == 0
 
 
 def test_embag_rows_past_the_end_and_tables_off_the_row_grid(B):
