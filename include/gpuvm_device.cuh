@@ -6,6 +6,7 @@
  * paged array only through:
  *
  *   T     gpuvm_read <T>(vm, elem_index, base_byte_off)        pin, load, unpin
+ *   void  gpuvm_read_n<T, N>(vm, elem[N], out[N], base, count) N such reads per lane with their round trips overlapped
  *   void  gpuvm_write<T>(vm, elem_index, value, base_byte_off) pin, mark dirty, store, unpin
  *   void* gpuvm_ptr(vm, byte_off, mode, &token)                pin and hand out a frame pointer
  *   void* gpuvm_ptr_if_resident(vm, byte_off, &token)          the same, but only if the page is there: no fault, no wait
@@ -796,6 +797,92 @@ __device__ __forceinline__ T gpuvm_read(const gpuvm_dev_t &vm, unsigned long lon
     T out;
     memcpy(&out, &v, sizeof(T));
     return out;
+}
+
+namespace gpuvm {
+/* gpuvm_read as a call, for callers that reach it rarely and do not want its code in their loop */
+template <typename T>
+static __device__ __noinline__ T read_out_of_line(const gpuvm_dev_t vm, unsigned long long elem, unsigned long long base_off)
+{
+    return gpuvm_read<T>(vm, elem, base_off);
+}
+}  // namespace gpuvm
+
+/*
+ * N independent reads per lane, issued together: out[j] = element elem[j] of the array of T at base_off, for
+ * j < count (count <= N may differ between lanes).  The resident case of gpuvm_read without its round trips in
+ * series: every lane pins the pages of its own requests (no grouping: lanes that happen to ask for the same page
+ * take one reference each), all N pins are in flight together, then the N loads, then the N unpins.  Ordering is
+ * by dependency, as in the batched engine: a load's address is computed from the entry its pin returned, so it
+ * is issued after the entry was seen VALID and is served by L2, where the publisher's stores already are; an
+ * unpin adds a zero that is computed from the loaded value, so it is issued after the value has arrived.  (This
+ * leans on the hardware executing a dependent instruction after its operands exist; the PTX memory model by
+ * itself does not order relaxed operations by dependency.  With GPUVM_DEBUG_FENCED_RELEASE in vm.debug a fence
+ * is placed on either side of the loads instead.)  A request whose page is not resident gives its reference
+ * back, and the lanes that called together then repeat that slot through gpuvm_read, so nothing is held while
+ * a frame is waited for (deadlock-free for any pool size, as gpuvm_read is).  Call it converged: `here` below
+ * must name the same lanes in all of them.  Each served request counts as one hit.  T of 4, 8 or 16 bytes.
+ */
+template <typename T, int N>
+__device__ __forceinline__ void gpuvm_read_n(const gpuvm_dev_t &vm, const unsigned long long (&elem)[N], T (&out)[N],
+                                             unsigned long long base_off = 0, int count = N)
+{
+    using namespace gpuvm;
+    static_assert(sizeof(T) == 4 || sizeof(T) == 8 || sizeof(T) == 16, "element size must be 4, 8 or 16 bytes");
+    const bool fenced = (vm.debug & GPUVM_DEBUG_FENCED_RELEASE) != 0;
+    unsigned long long w[N];
+    unsigned int slots = 0, hits = 0;                           /* bit j: slot j holds a reference / was served */
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const unsigned long long byte_off = base_off + elem[j] * sizeof(T);
+        w[j] = 0;
+        if (j < count && byte_off + sizeof(T) <= vm.bytes) {
+            slots |= 1u << j;
+            asm volatile("atom.relaxed.gpu.global.add.u64 %0, [%1], 1;" : "=l"(w[j]) : "l"(vm.pte + (byte_off >> vm.page_shift)) : "memory");
+        }
+    }
+    if (fenced) __threadfence();
+    uint4 v[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        v[j] = make_uint4(0, 0, 0, 0);
+        w[j] += 1ull;
+        if (((slots >> j) & 1u) && (w[j] & kStMask) == kValid && (w[j] & kRcMask) <= kRcLimit) {
+            const unsigned long long byte_off = base_off + elem[j] * sizeof(T);
+            hits |= 1u << j;
+            const unsigned char *p = vm.pool + (((w[j] & kFrameMask) >> kFrameShift) << vm.page_shift) +
+                                     (byte_off & ((1ull << vm.page_shift) - 1ull));
+            if (sizeof(T) == 16) v[j] = ld_frame16(p);
+            else if (sizeof(T) == 8) asm volatile("ld.relaxed.gpu.global.v2.u32 {%0,%1}, [%2];" : "=r"(v[j].x), "=r"(v[j].y) : "l"(p) : "memory");
+            else asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v[j].x) : "l"(p) : "memory");
+        }
+    }
+    if (fenced) __threadfence();
+#pragma unroll
+    for (int j = 0; j < N; ++j)
+        if ((slots >> j) & 1u) {
+            unsigned long long *pte = vm.pte + ((base_off + elem[j] * sizeof(T)) >> vm.page_shift);
+            if (((hits >> j) & 1u) && vm.policy == GPUVM_POLICY_CLOCK && !(w[j] & kRef)) atomicOr(pte, kRef);
+            /* zero, but not before v[j] exists (n_frames < 2^31) */
+            const unsigned long long hold = (unsigned long long)(v[j].x & (vm.n_frames >> 31));
+            asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(pte), "l"(~0ull + hold) : "memory");
+        }
+    if (GPUVM_COUNT_HITS && hits) {
+        /* one counter update per warp instruction: the lowest lane adds up what the lanes with it served */
+        const unsigned int active = __activemask();
+        const unsigned int n = __reduce_add_sync(active, (unsigned int)__popc(hits));
+        if (lane_id() == (unsigned int)__ffs(active) - 1u) stat_add(vm, kHits, n);
+    }
+    /* Slots that were not served (absent, in transit, out of range) take the full path.  All lanes that came in
+     * together go there together, the served ones too: the warp that faults copies the page with the lanes it
+     * has, and a few stragglers on their own would move a page sixteen bytes at a time. */
+    const unsigned int here = __activemask();
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const bool missed = j < count && !((hits >> j) & 1u);
+        if ((hits >> j) & 1u) memcpy(&out[j], &v[j], sizeof(T));
+        if (__any_sync(here, missed) && j < count) out[j] = gpuvm::read_out_of_line<T>(vm, elem[j], base_off);
+    }
 }
 
 /* A[i] = value (Listing 1, left-hand side).  A write miss fetches the page first. */

@@ -26,9 +26,19 @@ struct Paged {
     gpuvm_dev_t vm;
     unsigned long long edges_hint = 0;
     __device__ __forceinline__ unsigned long long unit() const { return 1ull << vm.page_shift; }
+    // what one lane group of a streaming kernel takes at a time: large pages are shared out in 64 KiB pieces
+    // (one pin per piece), so that a few hundred pages still occupy the whole grid
+    __device__ __forceinline__ unsigned long long stream_unit() const { return vm.page_shift > 16 ? 65536ull : 1ull << vm.page_shift; }
     // Host side.  Is it cheaper to read `vertices` scattered neighbour lists in place (about 256 bytes on the link
     // each: two row offsets, a short list, each rounded up to a 128-byte read) than to fetch the pages a full
     // sweep would miss (what does not fit the pool)?
+    // Host side.  How many pages (at most `want`) may each of `warps` warps hold pinned at the same time?
+    int pins_per_warp(int warps, int want) const
+    {
+        int g = want;
+        while (g > 1 && (unsigned long long)warps * g > vm.n_frames) g >>= 1;
+        return g;
+    }
     bool sparse_sweep(unsigned long long vertices) const
     {
         const unsigned long long missing = vm.n_pages > vm.n_frames ? vm.n_pages - vm.n_frames : 0ull;
@@ -36,6 +46,11 @@ struct Paged {
     }
     template <typename T>
     __device__ __forceinline__ T read(unsigned long long base, unsigned long long i) const { return gpuvm_read<T>(vm, i, base); }
+    template <typename T, int N>
+    __device__ __forceinline__ void read_n(unsigned long long base, const unsigned long long (&i)[N], T (&out)[N], int count) const
+    {
+        gpuvm_read_n<T, N>(vm, i, out, base, count);
+    }
     template <typename T>
     __device__ __forceinline__ void write(unsigned long long base, unsigned long long i, T v) const { gpuvm_write<T>(vm, i, v, base); }
     __device__ __forceinline__ unsigned char *pin(unsigned long long off, int mode, gpuvm_token &t) const
@@ -68,9 +83,18 @@ struct Raw {
     unsigned long long unit_bytes;
     unsigned long long edges_hint = 0;
     __device__ __forceinline__ unsigned long long unit() const { return unit_bytes; }
+    __device__ __forceinline__ unsigned long long stream_unit() const { return unit_bytes; }
+    int pins_per_warp(int, int) const { return 1; }
     bool sparse_sweep(unsigned long long) const { return false; }
     template <typename T>
     __device__ __forceinline__ T read(unsigned long long off, unsigned long long i) const { return reinterpret_cast<const T *>(base + off)[i]; }
+    template <typename T, int N>
+    __device__ __forceinline__ void read_n(unsigned long long off, const unsigned long long (&i)[N], T (&out)[N], int count) const
+    {
+#pragma unroll
+        for (int j = 0; j < N; ++j)
+            if (j < count) out[j] = reinterpret_cast<const T *>(base + off)[i[j]];
+    }
     template <typename T>
     __device__ __forceinline__ void write(unsigned long long off, unsigned long long i, T v) const { reinterpret_cast<T *>(base + off)[i] = v; }
     __device__ __forceinline__ unsigned char *pin(unsigned long long off, int, gpuvm_token &) const { return base + off; }
@@ -92,16 +116,21 @@ __device__ __forceinline__ unsigned int warp_in_grid() { return (blockIdx.x * bl
 __device__ __forceinline__ unsigned int warps_in_grid() { return (gridDim.x * blockDim.x) >> 5; }
 
 // ------------------------------------------------------------- streaming sum
-template <class Mem>
+// G units (pages) per warp at a time, 32 / G lanes each: the G pins are issued together, so the round trip of
+// the translation is paid once per G pages, and every lane group streams its own page.
+template <class Mem, int G>
 __global__ void __launch_bounds__(256) stream_sum_kernel(Mem m, unsigned long long a_off, unsigned long long n,
                                                          unsigned long long *out)
 {
-    const unsigned int lane = threadIdx.x & 31;
-    const unsigned long long unit = m.unit();
+    constexpr unsigned int L = 32 / G;                            // lanes per page
+    const unsigned int lane = threadIdx.x & 31, sub = lane / L, sl = lane % L;
+    const unsigned long long unit = m.stream_unit();             // a page, or a 64 KiB piece of a larger one
     const unsigned long long start = a_off, end = a_off + 4ull * n;
     const unsigned long long first = start / unit, units = (end + unit - 1) / unit - first;
     long long acc = 0;
-    for (unsigned long long u = warp_in_grid(); u < units; u += warps_in_grid()) {
+    for (unsigned long long u0 = (unsigned long long)warp_in_grid() * G; u0 < units; u0 += (unsigned long long)warps_in_grid() * G) {
+        const unsigned long long u = u0 + sub;
+        if (u >= units) continue;
         unsigned long long lo = (first + u) * unit, hi = lo + unit;
         if (lo < start) lo = start;
         if (hi > end) hi = end;
@@ -109,27 +138,34 @@ __global__ void __launch_bounds__(256) stream_sum_kernel(Mem m, unsigned long lo
         const unsigned char *p = m.pin(lo, GPUVM_READ, tok);
         if (!p) continue;
         const unsigned int len = (unsigned int)(hi - lo), n16 = len >> 4;
-#pragma unroll 4
-        for (unsigned int i = lane; i < n16; i += 32) {
+#pragma unroll 8
+        for (unsigned int i = sl; i < n16; i += L) {
             uint4 v = Mem::load16(p + 16ull * i);
             acc += (long long)(int)v.x + (long long)(int)v.y + (long long)(int)v.z + (long long)(int)v.w;
         }
         const unsigned int tail = (len & 15u) >> 2;
-        if (lane < tail) acc += (long long)Mem::load_i32(p + 16ull * n16 + 4u * lane);
+        if (sl < tail) acc += (long long)Mem::load_i32(p + 16ull * n16 + 4u * sl);
         m.release(tok);
     }
+    __syncwarp();
     for (int o = 16; o; o >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, o);
     if (lane == 0 && acc != 0) atomicAdd(out, (unsigned long long)acc);
 }
 
 // -------------------------------------------------------------- random gather
+// One request per lane and slot, kGatherSlots slots at a time (gpuvm_read_n): a thread block adds up one index
+// block at a time.
+// Two blocks of 256 threads per SM at up to 128 registers: with four blocks at 64 registers the loop spills and
+// a resident gather is a quarter slower (23.8 against 31.8 G accesses/s), the cold one the same.
+constexpr int kGatherSlots = 4;
+constexpr int kGatherPlainBlocksPerSm = 2;
 template <class Mem>
-__global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long long x_off, const long long *__restrict__ idx,
-                                                      unsigned long long n_idx, unsigned long long block,
-                                                      float *__restrict__ fsum, long long *__restrict__ bsum)
+__global__ void __launch_bounds__(256, kGatherPlainBlocksPerSm) gather_kernel(Mem m, unsigned long long x_off, const long long *__restrict__ idx,
+                                                        unsigned long long n_idx, unsigned long long block,
+                                                        float *__restrict__ fsum, long long *__restrict__ bsum)
 {
-    __shared__ double s_f[32];
-    __shared__ long long s_b[32];
+    __shared__ double s_f[8];
+    __shared__ long long s_b[8];
     const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned long long nb = (n_idx + block - 1) / block;
     for (unsigned long long b = blockIdx.x; b < nb; b += gridDim.x) {
@@ -137,11 +173,22 @@ __global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long lo
         const unsigned long long hi = lo + block < n_idx ? lo + block : n_idx;
         double f = 0.0;
         long long bits = 0;
-        for (unsigned long long k = lo + threadIdx.x; k < hi; k += blockDim.x) {
-            float v = m.template read<float>(x_off, (unsigned long long)idx[k]);
-            f += (double)v;
-            bits += (long long)__float_as_uint(v);
+        for (unsigned long long k = lo + threadIdx.x; k < hi; k += (unsigned long long)kGatherSlots * blockDim.x) {
+            unsigned long long e[kGatherSlots];
+            float v[kGatherSlots];
+            int count = 0;
+#pragma unroll
+            for (int j = 0; j < kGatherSlots; ++j) {
+                const unsigned long long kj = k + (unsigned long long)j * blockDim.x;
+                e[j] = kj < hi ? (unsigned long long)idx[kj] : 0ull;
+                count += kj < hi;
+            }
+            m.template read_n<float, kGatherSlots>(x_off, e, v, count);
+#pragma unroll
+            for (int j = 0; j < kGatherSlots; ++j)
+                if (j < count) { f += (double)v[j]; bits += (long long)__float_as_uint(v[j]); }
         }
+        __syncwarp();
         for (int o = 16; o; o >>= 1) {
             f += __shfl_down_sync(0xFFFFFFFFu, f, o);
             bits += __shfl_down_sync(0xFFFFFFFFu, bits, o);
@@ -152,7 +199,7 @@ __global__ void __launch_bounds__(1024, 1) gather_kernel(Mem m, unsigned long lo
             const unsigned int nw = blockDim.x >> 5;
             f = lane < nw ? s_f[lane] : 0.0;
             bits = lane < nw ? s_b[lane] : 0;
-            for (int o = 16; o; o >>= 1) {
+            for (int o = 4; o; o >>= 1) {
                 f += __shfl_down_sync(0xFFFFFFFFu, f, o);
                 bits += __shfl_down_sync(0xFFFFFFFFu, bits, o);
             }
@@ -1422,7 +1469,14 @@ int run_stream_sum(const Mem &m, size_t a_off, size_t n, int64_t *d_sum, cudaStr
     if (a_off % 16) return GPUVM_E_ALIGN;
     if (cudaMemsetAsync(d_sum, 0, sizeof(int64_t), s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
     if (n == 0) return GPUVM_OK;
-    stream_sum_kernel<Mem><<<sm_count() * 4, 256, 0, s>>>(m, a_off, n, reinterpret_cast<unsigned long long *>(d_sum));
+    // Pages per warp at a time: as many as the pool lets every warp of the grid hold at once (a warp that
+    // holds pins while it faults needs a free frame), at most four.
+    const int blocks = sm_count() * 4, warps = blocks * 8;
+    int g = m.pins_per_warp(warps, 4);
+    unsigned long long *out = reinterpret_cast<unsigned long long *>(d_sum);
+    if (g >= 4) stream_sum_kernel<Mem, 4><<<blocks, 256, 0, s>>>(m, a_off, n, out);
+    else if (g >= 2) stream_sum_kernel<Mem, 2><<<blocks, 256, 0, s>>>(m, a_off, n, out);
+    else stream_sum_kernel<Mem, 1><<<blocks, 256, 0, s>>>(m, a_off, n, out);
     return launched();
 }
 
@@ -1434,8 +1488,8 @@ int run_gather(const Mem &m, size_t x_off, const int64_t *d_idx, size_t n_idx, s
     if (x_off % 16) return GPUVM_E_ALIGN;
     if (n_idx == 0) return GPUVM_OK;
     size_t nb = (n_idx + block - 1) / block;
-    unsigned int threads = block >= 1024 ? 1024u : (unsigned int)((block + 31) / 32 * 32);
-    size_t resident = (size_t)sm_count() * (2048 / threads);
+    unsigned int threads = block >= 256 ? 256u : (unsigned int)((block + 31) / 32 * 32);
+    size_t resident = (size_t)sm_count() * (256 * kGatherPlainBlocksPerSm / threads);
     unsigned int grid = (unsigned int)(nb < resident ? nb : resident);
     gather_kernel<Mem><<<grid, threads, 0, s>>>(m, x_off, reinterpret_cast<const long long *>(d_idx), n_idx, block,
                                                  d_fsum, reinterpret_cast<long long *>(d_bsum));

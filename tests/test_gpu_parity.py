@@ -502,6 +502,40 @@ def test_fenced_release_gives_the_same_results(B, frames):
         assert np.array_equal(out.cpu().numpy().view(np.uint32), ref_e.view(np.uint32)), flags
 
 
+@pytest.mark.parametrize("frames", [2, 64])
+def test_read_n_hits_misses_and_fenced_mode(B, frames):
+    """The one-request-per-lane gather issues four reads per lane together (gpuvm_read_n): a second pass over a
+    pool that holds everything is served by hits alone (one per request), a pool of two frames sends almost
+    every slot through the full path, and the fenced debug mode (fences instead of dependency order around the
+    loads) gives the same bits."""
+    import torch
+    page, n, n_idx = 4096, 1 << 16, 20000 + 13
+    x = inputs.fill_f32_pm1(np.empty(n, np.float32), n, inputs.config_seed(2))
+    idx = inputs.fill_index_i64(np.empty(n_idx, np.int64), n_idx, inputs.config_seed(2, 1), n)
+    ar = Arena(page, {"x": x})
+    nb = (n_idx + 1023) // 1024
+    ref_f, ref_b = oracle.gather_block_sums_direct(x, idx, 1024)
+    for flags in (0, B.DEBUG_FENCED_RELEASE):
+        fs = torch.zeros(nb, dtype=torch.float32, device="cuda")
+        bs = torch.zeros(nb, dtype=torch.int64, device="cuda")
+        with paged(ar.host, page, frames) as h:
+            B.gpuvm_set_debug(h, flags)
+            B.gpuvm_gather_f32_unbatched(h, 0, dev(idx), n_idx, 1024, fs, bs)
+            st1, _ = finish(h)
+            assert np.array_equal(bs.cpu().numpy(), ref_b), flags
+            bs.zero_()
+            B.gpuvm_gather_f32_unbatched(h, 0, dev(idx), n_idx, 1024, fs, bs)
+            st2, _ = finish(h)
+        assert np.array_equal(bs.cpu().numpy(), ref_b), flags
+        got = fs.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref_f) <= 1e-6 * np.maximum(np.abs(ref_f), 2.0 ** -10))
+        if frames >= ar.n_pages:
+            assert st2["faults"] == st1["faults"] == np.unique(idx * 4 // page).size
+            assert st2["hits"] - st1["hits"] == n_idx          # every request of the second pass is a hit of its own
+        else:
+            assert st2["faults"] > st1["faults"] > frames
+
+
 def test_two_kernels_share_mappings(B):
     """Mappings persist across launches: a read-only pass after a write pass sees the
     written values without any flush in between."""
