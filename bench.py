@@ -414,10 +414,11 @@ def e2e_step(torch, B, w, cfg: int):
 
 
 def embag_policy_records(torch, B, w, args, link: dict, kern_s: float, direct: float, rec: dict) -> dict:
-    """cfg 5 runs with the library's rent-or-buy default (a page is fetched once its rows have moved a quarter of
-    its size in place).  Reported beside it: the ceiling of scattered row reads over this backing store, measured
-    here, which bounds the rows read in place; and the same launch with the policy off (the paper's way: every
-    first touch fetches the page), with its own link roofline."""
+    """cfg 5 runs with the library's default: lookups are counted per page first, rows of pages with fewer lookups
+    than a quarter of their rows are read in place, the other pages are fetched at their first touch.  Reported
+    beside it: the ceiling of scattered row reads over this backing store, measured here, which bounds the rows
+    read in place; the online form of the policy (no count beforehand); and the same launch with the policy off
+    (the paper's way: every first touch fetches the page), each with its own link roofline."""
     out = {}
     row_bytes = 4 * w.dims
     buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -429,25 +430,34 @@ def embag_policy_records(torch, B, w, args, link: dict, kern_s: float, direct: f
         "what": f"rows read in place from the backing store; the peak is {1 << 22} rows of {row_bytes} B at hashed "
                 f"positions of the same {w.nbytes >> 30} GiB region, four in flight per warp, measured in this run"}
     if args.inplace_divisor < 0 and not args.scratch_limit_mib:
-        B.gpuvm_set_inplace_divisor(w.h, 0)
-        try:
-            w.run(check=False)
-            rs = [w.run(check=True) for _ in range(2)]
-        finally:
-            B.gpuvm_set_inplace_divisor(w.h, DEFAULT_INPLACE_DIVISOR)
-        secs = sum(r.seconds for r in rs) / len(rs)
-        ks = sum(r.kernel_seconds for r in rs) / len(rs)
-        st = rs[-1].stats
-        roof = link_roofline(st["bytes_in"], st["bytes_out"], ks, link)
+        def other_policy(what, setup, restore):
+            setup()
+            try:
+                w.run(check=False)
+                rs = [w.run(check=True) for _ in range(2)]
+            finally:
+                restore()
+            secs = sum(r.seconds for r in rs) / len(rs)
+            ks = sum(r.kernel_seconds for r in rs) / len(rs)
+            st = rs[-1].stats
+            roof = link_roofline(st["bytes_in"] + st.get("bytes_direct", 0), st["bytes_out"], ks, link)
+            return {"what": what, "ms_per_step": secs * 1e3, "value": rs[-1].effective_bytes / secs / 1e9, "unit": UNIT,
+                    "steps": len(rs), "faults": st["faults"], "bytes_in": st["bytes_in"],
+                    "bytes_direct": st.get("bytes_direct", 0), "in_gbs": st["bytes_in"] / secs / 1e9,
+                    "invariants_status": rs[-1].check["status"], "roofline": roof}
+
+        out["online"] = other_policy(
+            "gpuvm_set_inplace_counted(h, 0): no count beforehand; the first requests that find a page absent read "
+            "their rows in place, the one after them fetches the page",
+            lambda: B.gpuvm_set_inplace_counted(w.h, False), lambda: B.gpuvm_set_inplace_counted(w.h, True))
+        rec_am = other_policy(
+            "gpuvm_set_inplace_divisor(h, 0): every first touch fetches the page, as in the paper",
+            lambda: B.gpuvm_set_inplace_divisor(w.h, 0), lambda: B.gpuvm_set_inplace_divisor(w.h, DEFAULT_INPLACE_DIVISOR))
         traffic = NCU_LINK_TRAFFIC.get("5_always_migrate") if args.shrink == 0 else None
-        roof["traffic"] = traffic[0] if traffic else None
-        roof["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[3]}): host-link bytes of one launch counted by ncu"
-                                  if traffic else None)
-        out["always_migrate"] = {
-            "what": "gpuvm_set_inplace_divisor(h, 0): every first touch fetches the page, as in the paper",
-            "ms_per_step": secs * 1e3, "value": rs[-1].effective_bytes / secs / 1e9, "unit": UNIT, "steps": len(rs),
-            "faults": st["faults"], "bytes_in": st["bytes_in"], "in_gbs": st["bytes_in"] / secs / 1e9,
-            "invariants_status": rs[-1].check["status"], "roofline": roof}
+        rec_am["roofline"]["traffic"] = traffic[0] if traffic else None
+        rec_am["roofline"]["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[3]}): host-link bytes of one launch "
+                                                "counted by ncu" if traffic else None)
+        out["always_migrate"] = rec_am
     return out
 
 

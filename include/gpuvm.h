@@ -240,6 +240,14 @@ size_t gpuvm_scratch_bytes(gpuvm_t h);
  * streams finish together near a quarter (measured on the 64 GiB Zipf table: 70 / 61 / 77 ms for 2 / 4 / 8). */
 int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor);
 
+/* How the batched row workloads decide which pages are worth fetching.  counted != 0 (default): a short kernel
+ * first counts, per page, the lookups of the whole list (the list is the kernel's input, so the demand is
+ * known before the first access); rows of pages with fewer than page_bytes / divisor / row_bytes lookups are
+ * read in place without the page table being touched, every other page is fetched at its first touch: no
+ * row of a page that will be fetched anyway is read in place first.  counted == 0: the online form described
+ * above, which needs no pass over the list. */
+int gpuvm_set_inplace_counted(gpuvm_t h, int counted);
+
 /* Largest number of simultaneously resident warps that can each hold
  * `pins_per_warp` pages pinned without exhausting the pool (a warp that holds
  * pins while faulting needs a free frame; Section 3.3: a frame is reused only

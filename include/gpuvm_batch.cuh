@@ -48,6 +48,13 @@
  * gpuvm_batch_run is the engine itself: longer tables, in any layout that a small accessor
  * type can read (for instance bare 32-bit element indices), with the per-lane state words in
  * memory the caller provides.
+ * Reads in place (read mode, data that nobody writes through the runtime meanwhile): with inplace_limit != 0
+ * a request for a page that is not resident need not fetch it; consume then gets a pointer into the backing
+ * store (inplace_bytes: what one such request moves, for the bytes_direct counter).  Which requests: with
+ * `demand` (one 32-bit count per page: how many requests of the whole launch name it, counted by the caller
+ * beforehand) those of pages with fewer than inplace_limit requests, without the page table being touched at
+ * all, and every other page is fetched at its first touch; without `demand` the first inplace_limit requests
+ * that find a page absent, counted in the frame field of its entry, and the one after them fetches it.
  */
 #ifndef GPUVM_BATCH_CUH
 #define GPUVM_BATCH_CUH
@@ -95,6 +102,7 @@ namespace gpuvm {
 constexpr unsigned int kNotReady = 0xFFFFFFFFu;   /* "frame" values a leader hands to its followers */
 constexpr unsigned int kInPlaceFrame = 0xFFFFFFFEu; /* the group reads from the backing store, it holds no reference */
 constexpr unsigned int kRejected = 0xFFFFFFFFu;   /* vpn of a request that was refused when it was set */
+constexpr unsigned long long kColdWord = ~0ull;   /* stands for the entry of a page that is read in place unseen (no entry has all bits set) */
 
 /* Any lane.  False when the ring is (nearly) full: the caller keeps the fault and retries. */
 __device__ __forceinline__ bool fault_queue_push(gpuvm_fault_queue *q, unsigned int vpn, int mode,
@@ -372,7 +380,7 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                                                             int mode, Consume consume, gpuvm_fault_queue *queue,
                                                             unsigned long long *masks, unsigned int mask_stride,
                                                             bool eager_push = false, unsigned int inplace_limit = 0,
-                                                            unsigned int inplace_bytes = 0)
+                                                            unsigned int inplace_bytes = 0, const unsigned int *demand = nullptr)
 {
     using namespace gpuvm;
     const unsigned int lane = lane_id();
@@ -425,7 +433,9 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                 leader[u] = __ffs(group) - 1;
                 gsize[u] = __popc(group);
                 if (lane == leader[u]) {
-                    if (first) {
+                    if (first && demand && inplace_limit != 0u && demand[vpn[u]] < inplace_limit) {
+                        word[u] = kColdWord;                /* known cold: read in place, the page table is not touched */
+                    } else if (first) {
                         word[u] = pin_acquire(vm.pte + vpn[u]) + 1ull;
                         /* far too many references to one page: the sticky error ends every wait of the
                          * launch at its next idle round, long before the counter could carry */
@@ -451,7 +461,8 @@ static __device__ __noinline__ unsigned int gpuvm_batch_run(const gpuvm_dev_t vm
                 const bool looks_valid = (w & kStMask) == kValid;
                 if (!first && GPUVM_BATCH_ACQ == 1 && looks_valid) w = ld_acquire_u64(vm.pte + vpn[u]);
                 unsigned int f;
-                const int st = advance(vm, vm.pte + vpn[u], w, mode, f, inplace_limit, gsize[u]);
+                const int st = w == kColdWord ? (int)kInPlace
+                                              : advance(vm, vm.pte + vpn[u], w, mode, f, demand ? 0u : inplace_limit, gsize[u]);
                 if (st == kReady) {
                     frame[u] = f;
                     need_fence |= GPUVM_BATCH_ACQ == 2 || (GPUVM_BATCH_ACQ == 1 && !looks_valid);

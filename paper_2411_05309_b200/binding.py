@@ -65,6 +65,7 @@ SYMBOLS = {
     "gpuvm_set_debug": (_i, [_vp, ctypes.c_uint]),
     "gpuvm_set_clean_ahead": (_i, [_vp, ctypes.c_uint]),
     "gpuvm_set_inplace_divisor": (_i, [_vp, ctypes.c_uint]),
+    "gpuvm_set_inplace_counted": (_i, [_vp, _i]),
     "gpuvm_bcsr_build": (_i, [_vp, _sz, _sz, _vp, _sz, ctypes.POINTER(_sz)]),
     "gpuvm_device_view": (_i, [_vp, ctypes.POINTER(DevView)]),
     "gpuvm_host_ptr": (_vp, [_vp]),
@@ -207,6 +208,10 @@ def gpuvm_check_on(h, stream, raise_on_error: bool = True) -> dict:
 
 def gpuvm_set_inplace_divisor(h, divisor: int):
     _check(lib().gpuvm_set_inplace_divisor(h, divisor), "gpuvm_set_inplace_divisor")
+
+
+def gpuvm_set_inplace_counted(h, counted: bool):
+    _check(lib().gpuvm_set_inplace_counted(h, int(bool(counted))), "gpuvm_set_inplace_counted")
 
 
 def gpuvm_set_clean_ahead(h, frames: int):

@@ -24,6 +24,7 @@ struct gpuvm_handle {
     size_t scratch_bytes;
     size_t scratch_limit;      /* 0: none */
     unsigned int inplace_divisor;
+    bool inplace_counted;   // the batched row workloads count the lookups per page first
 };
 
 namespace {
@@ -146,6 +147,7 @@ int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_byt
     cudaGetDevice(&h->device);
     h->sms = sm_count_of(h->device);
     h->inplace_divisor = 4;
+    h->inplace_counted = true;
     cudaError_t e;
 
     // backing store: pinned and mapped (Section 4: the host region is registered before
@@ -338,11 +340,19 @@ int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes)
 size_t gpuvm_scratch_bytes(gpuvm_t h) { return h ? h->scratch_bytes : 0; }
 
 size_t gpuvm_inplace_divisor_(gpuvm_handle *h) { return h ? h->inplace_divisor : 0; }
+int gpuvm_inplace_counted_(gpuvm_handle *h) { return h && h->inplace_counted; }
 
 int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor)
 {
     if (!h) return GPUVM_E_ARG;
     h->inplace_divisor = divisor;
+    return GPUVM_OK;
+}
+
+int gpuvm_set_inplace_counted(gpuvm_t h, int counted)
+{
+    if (!h) return GPUVM_E_ARG;
+    h->inplace_counted = counted != 0;
     return GPUVM_OK;
 }
 

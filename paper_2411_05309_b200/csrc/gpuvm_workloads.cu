@@ -1169,12 +1169,34 @@ constexpr unsigned int kEmbagLookups = 32;                 // lookups of a bag p
 constexpr unsigned int kEmbagChunk = 8192;                 // bytes per bulk copy of a migrator warp
 constexpr unsigned int kEmbagMaxGroups = 8;                // groups of 32 bags a requester warp takes at a time
 
+// How many lookups of the whole list name each page: the batched kernel reads the rows of pages with few
+// lookups in place and fetches the others at their first touch.  One atomic per group of equal pages in a warp.
+__global__ void embag_demand_kernel(const long long *__restrict__ rows, unsigned long long n, unsigned long long t_off,
+                                    unsigned long long row_bytes, unsigned int page_shift, unsigned long long rows_inside,
+                                    unsigned int *__restrict__ demand)
+{
+    const unsigned int lane = threadIdx.x & 31;
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    for (unsigned long long base = (blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x) & ~31ull; base < n; base += stride) {
+        const unsigned long long i = base + lane;
+        const unsigned long long r = i < n ? (unsigned long long)rows[i] : ~0ull;
+        const bool inside = r < rows_inside;
+        const unsigned int vpn = inside ? (unsigned int)((t_off + r * row_bytes) >> page_shift) : 0u;
+        const unsigned int mask = __ballot_sync(0xFFFFFFFFu, inside);
+        if (inside) {
+            const unsigned int group = __match_any_sync(mask, vpn);
+            if (lane == (unsigned int)__ffs(group) - 1u) atomicAdd(demand + vpn, (unsigned int)__popc(group));
+        }
+    }
+}
+
 __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
                                                               const long long *__restrict__ rows, unsigned long long n_bags,
                                                               unsigned int bag, float *__restrict__ out, int requesters,
                                                               gpuvm_batch_entry *g_tables, unsigned char *g_staging,
                                                               unsigned int groups, bool one_pass,
-                                                              gpuvm_shared_queue *shared_queue, unsigned int inplace_limit)
+                                                              gpuvm_shared_queue *shared_queue, unsigned int inplace_limit,
+                                                              const unsigned int *demand)
 {
     __shared__ gpuvm_fault_queue queue_s;
     __shared__ __align__(128) unsigned char stage_s[kEmbagMigrators][kEmbagChunk];   // bulk-copy staging of the migrator warps
@@ -1226,7 +1248,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
             // every served row is copied to its slot of the staging area by the whole warp (the engine does it
             // itself, four rows in flight: gpuvm_row_copy), from its frame or in place from the backing store
             gpuvm_batch_run<true>(vm, gpuvm_entry_table{table}, groups * nk * 32, GPUVM_READ, gpuvm_row_copy{staging, q},
-                                  queue, masks, 1u, one_pass, inplace_limit, (unsigned int)row_bytes);
+                                  queue, masks, 1u, one_pass, inplace_limit, (unsigned int)row_bytes, demand);
             __syncwarp();
             // add the staged rows of each bag in list order
             for (unsigned int gb = 0; gb < 32 * groups && g0 + gb < n_bags; ++gb) {
@@ -1986,7 +2008,9 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     const size_t slots = items < (size_t)grid * requesters ? items : (size_t)grid * requesters;   // warps that get work
     const size_t table_bytes = (slots * per_warp * sizeof(gpuvm_batch_entry) + 255) & ~size_t(255);
     const size_t staging_bytes = (slots * per_warp * 4 * dims + 255) & ~size_t(255);
-    unsigned char *scratch = static_cast<unsigned char *>(gpuvm_scratch_(h, table_bytes + staging_bytes + sizeof(gpuvm_shared_queue)));
+    const size_t demand_bytes = (m.vm.n_pages * sizeof(unsigned int) + 255) & ~size_t(255);
+    unsigned char *scratch = static_cast<unsigned char *>(
+        gpuvm_scratch_(h, table_bytes + staging_bytes + sizeof(gpuvm_shared_queue) + demand_bytes));
     if (!scratch) return GPUVM_E_ALLOC;
     gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, scratch + table_bytes + staging_bytes, static_cast<cudaStream_t>(stream));
     // Rent or buy: a page is fetched only once its rows have been asked for often enough to have moved a stated
@@ -1996,11 +2020,23 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     const size_t divisor = gpuvm_inplace_divisor_(h);
     const size_t charged = row_bytes < 128 ? 128 : row_bytes;
     const unsigned int inplace_limit = divisor ? (unsigned int)(page_bytes / divisor / charged) : 0u;
+    // The lookup list is at hand, so the lookups per page can be counted before the first access: pages below the
+    // limit are then read in place throughout and the others fetched at once (gpuvm_set_inplace_counted).
+    unsigned int *demand = nullptr;
+    unsigned long long launches = 1;
+    if (inplace_limit != 0u && gpuvm_inplace_counted_(h)) {
+        demand = reinterpret_cast<unsigned int *>(scratch + table_bytes + staging_bytes + sizeof(gpuvm_shared_queue));
+        if (cudaMemsetAsync(demand, 0, demand_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+        embag_demand_kernel<<<sm_count() * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            reinterpret_cast<const long long *>(d_rows), (unsigned long long)n_bags * bag, t_off, row_bytes, m.vm.page_shift,
+            (m.vm.bytes - t_off) / row_bytes, demand);
+        ++launches;
+    }
     embag_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
         m.vm, t_off, (unsigned int)dims, reinterpret_cast<const long long *>(d_rows), n_bags, (unsigned int)bag, d_out,
         requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes, groups,
-        /* one_pass = */ items <= (size_t)grid * requesters && bag <= kEmbagLookups, shared_queue, inplace_limit);
-    return launched();
+        /* one_pass = */ items <= (size_t)grid * requesters && bag <= kEmbagLookups, shared_queue, inplace_limit, demand);
+    return launched(launches);
 }
 
 int gpuvm_embag_f32_unbatched(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows, size_t n_bags, size_t bag,

@@ -161,18 +161,24 @@ def test_cfg5_zipf_embedding_bag_64GiB():
             assert np.array_equal(ref.view(np.uint32), out[start:start + step].view(np.uint32)), start
         st = res.stats
         distinct = np.unique(rows >> 12).size                   # 4096 rows per 2 MiB page
-        # Rent or buy: a page is fetched only after 1024 of its rows (a quarter of its size) have been read in place, so
-        # at most the pages with that many lookups are fetched, each once (all requests are in flight together),
-        # and no row is read in place from a page more often than the limit allows (+ one row of 32 requests per
-        # warp that was counting at the same moment)
+        # Pages with fewer than 1024 lookups (a quarter of their 4096 rows) are never fetched: their rows are read
+        # in place, every one of them; the others are fetched once, at their first touch (all requests are in
+        # flight together and 615 pages fit the pool)
         per_page = np.bincount(rows >> 12, minlength=w.n_pages)
         limit = (2 << 20) // 4 // 512
-        assert st["faults"] <= np.count_nonzero(per_page > limit) + 1 and st["faults"] >= np.count_nonzero(per_page > limit + 4096)
-        in_place = st["bytes_direct"] // 512
-        assert in_place <= int(np.minimum(per_page, limit + 4096).sum())
-        assert in_place >= int(per_page[per_page <= limit].sum())                # cold pages are served in place entirely
-        # the paper's way (every first touch fetches the page): never fewer than one fault per page touched
+        assert st["faults"] == np.count_nonzero(per_page >= limit)
+        assert st["bytes_direct"] == int(per_page[per_page < limit].sum()) * 512
         B = __import__("paper_2411_05309_b200.binding", fromlist=["x"])
+        # the online form (no count beforehand): a page is fetched after 1024 of its rows have been read in place
+        B.gpuvm_set_inplace_counted(w.h, False)
+        res1 = w.run()
+        st1 = res1.stats
+        assert np.count_nonzero(per_page > limit + 4096) <= st1["faults"] <= np.count_nonzero(per_page > limit) + 1
+        in_place = st1["bytes_direct"] // 512
+        assert int(per_page[per_page <= limit].sum()) <= in_place <= int(np.minimum(per_page, limit + 4096).sum())
+        assert np.array_equal(w.d_out.cpu().numpy().reshape(w.n_bags, w.dims)[:4096].view(np.uint32), out[:4096].view(np.uint32))
+        B.gpuvm_set_inplace_counted(w.h, True)
+        # the paper's way (every first touch fetches the page): never fewer than one fault per page touched
         B.gpuvm_set_inplace_divisor(w.h, 0)
         res0 = w.run()
         assert res0.stats["bytes_direct"] == 0 and distinct <= res0.stats["faults"] <= 1.3 * 1.06e6

@@ -360,11 +360,14 @@ def test_embag(B, page, n_rows, n_bags, frames, dims, bag, batched):
         assert st["bytes_direct"] == 0 and st["faults"] >= touched
 
 
+@pytest.mark.parametrize("counted", [True, False])
 @pytest.mark.parametrize("frames", [1, 4, 64])
-def test_embag_rent_or_buy(B, frames):
-    """The batched embedding bag reads the first rows of a page in place and fetches the page only when its requests
-    have moved the stated fraction of its size (a quarter unless set otherwise): cold pages are never fetched, a hot page is fetched once after the stated number of
-    in-place reads, and with the divisor 0 every first touch fetches.  Results are exact either way."""
+def test_embag_rent_or_buy(B, frames, counted):
+    """The batched embedding bag does not fetch a page for a few rows.  Counted (default): the lookups per page are
+    counted first; rows of pages below the limit (page / divisor / row size; a quarter of a page unless set
+    otherwise) are read in place, all of them, and the other pages are fetched at their first touch.  Online: the
+    first `limit` requests that find a page absent read their rows in place, the next one fetches it.  Divisor 0:
+    every first touch fetches, as in the paper.  Results are exact either way."""
     import torch
     page, dims, bag = 4096, 128, 4                       # 8 rows per page; a quarter of a page = 2 rows
     n_rows = 512
@@ -376,9 +379,11 @@ def test_embag_rent_or_buy(B, frames):
     for rows, name in ((cold, "cold"), (hot, "hot"), (mixed, "mixed")):
         n_bags = rows.size // bag
         ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
+        per_page = np.bincount(rows // 8, minlength=ar.n_pages)
         for divisor in (None, 2, 0, 8):
             out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
             with paged(ar.host, page, frames) as h:
+                B.gpuvm_set_inplace_counted(h, counted)
                 if divisor is None:
                     divisor = 4                                                # the default
                 else:
@@ -387,14 +392,18 @@ def test_embag_rent_or_buy(B, frames):
                 st, ck = finish(h)
             assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32)), (name, divisor)
             limit = page // divisor // 512 if divisor else 0                  # rows of a page that are read in place
+            assert st["bytes_direct"] % 512 == 0
             if divisor == 0:
-                assert st["bytes_direct"] == 0 and st["faults"] >= np.unique(rows // 8).size
+                assert st["bytes_direct"] == 0 and st["faults"] >= np.count_nonzero(per_page)
+            elif counted:
+                bought = np.count_nonzero(per_page >= limit)
+                assert st["bytes_direct"] == int(per_page[per_page < limit].sum()) * 512
+                assert st["faults"] >= bought and (frames < bought or st["faults"] == bought)
             elif name == "cold":                                               # one row per page: below any limit
                 assert st["faults"] == 0 and st["bytes_direct"] == rows.size * 512
             elif name == "hot":                                                # the page is bought after `limit` rows
                 assert st["faults"] >= 1
                 assert limit * 512 <= st["bytes_direct"] <= (limit + 31) * 512 * st["faults"]
-            assert st["bytes_direct"] % 512 == 0
 
 
 def test_embag_rows_past_the_end_and_tables_off_the_row_grid(B):
