@@ -130,6 +130,8 @@ NCU_LINK_TRAFFIC = {
         "full size; sweep 1 of the four sweeps of a run, 95 % of its time"),
     4: (33554432 * 32 * 8 + (4 << 30), "vadd_kernel_cfg4_eighth_full_set.md", 33554432,
         "1/8 case x 8: 8 GiB in, plus the 4 GiB of c that go out"),
+    5: (76624608 * 32, "embag_batch_kernel_cfg5_counted_policy.md", 76624608,
+        "full size, default policy; one metric, one pass"),
     "5_always_migrate": (134217728 * 32 * 16, "embag_batch_kernel_cfg5_sixteenth_full_set.md", 134217728,
                          "1/16 case x 16, every first touch fetching its page"),
     6: (37758976 * 32, "graph_sweep_kernel_cc_cfg6_full_set.md", 37758976, "full size"),
@@ -499,7 +501,8 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
         peaks = measured_peaks()
         hbm_peak = peaks.get("hbm_gbs", 6650.0)
         roof = link_roofline(bytes_in + direct, bytes_out, kern_s, link)
-        traffic = NCU_LINK_TRAFFIC.get(cfg) if args.shrink == 0 and not args.scratch_limit_mib else None
+        traffic = (NCU_LINK_TRAFFIC.get(cfg) if args.shrink == 0 and not args.scratch_limit_mib and args.inplace_divisor < 0
+                   else None)
         roof["traffic"] = traffic[0] if traffic else None
         roof["traffic_source"] = (f"profiles/{traffic[1]} ({traffic[3]}): host-link bytes of one launch counted by ncu"
                                   if traffic else None)

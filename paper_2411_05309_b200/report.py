@@ -23,9 +23,14 @@ def _mib(nbytes: float) -> str:
 def _row(cfg: str, r: dict) -> str:
     m, roof, sc = r["migration"], r["roofline"], r["scratch"]
     mig = f"{m['in_gbs']:.1f} in" + (f" + {m['out_gbs']:.1f} out" if m["out_gbs"] > 0.05 else "")
+    if m.get("direct_gbs", 0.0) > 0.05:
+        mig += f" + {m['direct_gbs']:.1f} read in place"
     frac = f"{roof['frac']:.3f}"
     if "frac_compulsory" in roof:
         frac += f" by faults, {roof['frac_compulsory']:.3f} of the compulsory floor"
+    if roof.get("in_place", {}).get("frac"):
+        frac += (f"; rows in place at {roof['in_place']['frac']:.2f} of the {roof['in_place']['scattered_read_peak_gbs']:.1f} GB/s "
+                 "scattered reads reach")
     cpu = r.get("cpu_baseline")
     cpu_s = "-"
     if cpu:
@@ -35,11 +40,26 @@ def _row(cfg: str, r: dict) -> str:
     bounded = sc.get("bounded_to_an_eighth_of_the_pool")
     b_s = "-"
     if bounded:
-        b_s = f"{_mib(bounded['limit_bytes'])}: {bounded['ms_per_step']:.0f} ms, {bounded['faults'] / 1e3:.0f} K faults"
+        n = bounded["faults"]
+        b_s = f"{_mib(bounded['limit_bytes'])}: {bounded['ms_per_step']:.0f} ms, " + (f"{n / 1e3:.0f} K faults" if n >= 10000 else f"{n} faults")
     ms = r["ms_per_step"]
     t = f"{ms:.2f} ms" if ms < 1000 else f"{ms / 1e3:.3f} s"
     return (f"| {cfg} {r['config']['workload'].split(':')[0].split(',')[0].split(' ', 1)[-1]} | {t} | {r['value']:.2f} | {mig} | {frac} | "
             f"{m['faults']:.0f} of {r['config']['pages']} pages | {_mib(sc['bytes'])} | {r['e2e']['value']:.2f} | {cpu_s} | {b_s} |")
+
+
+def policies(line: dict) -> str:
+    """cfg 5 under the other two policies, when the line has them."""
+    recs = line.get("per_config") or {str(line["config"]["cfg"]): line}
+    roof = recs.get("5", {}).get("roofline", {})
+    out = []
+    for key, name in (("online", "online rent-or-buy (no count beforehand)"), ("always_migrate", "the paper's policy (every first touch fetches)")):
+        r = roof.get(key)
+        if r:
+            out.append(f"cfg 5 under {name}: {r['ms_per_step']:.1f} ms, {r['value']:.2f} GB/s, {r['faults']} faults, "
+                       f"{r['bytes_in'] / 1e9:.2f} GB paged in + {r.get('bytes_direct', 0) / 1e9:.2f} GB read in place, "
+                       f"roofline.frac {r['roofline']['frac']:.3f}.")
+    return "\n".join(out)
 
 
 def table(line: dict) -> str:
@@ -65,6 +85,10 @@ def main(argv=None) -> int:
     text = open(argv[0]).read() if argv else sys.stdin.read()
     line = json.loads([l for l in text.splitlines() if l.startswith("{")][-1])
     print(table(line))
+    extra = policies(line)
+    if extra:
+        print()
+        print(extra)
     return 0
 
 

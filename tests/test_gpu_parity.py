@@ -61,6 +61,37 @@ def test_stream_sum(B, page, n, frames, policy):
     assert np.array_equal(ar.host, before)
 
 
+@pytest.mark.parametrize("page,frames", [
+    (256, 20000),                 # four pages per warp at a time (eight lanes each): the pool lets every warp hold four
+    (256, 10000),                 # two
+    (256, 4000),                  # one
+    (1 << 18, 40),                # pages above 64 KiB are shared out in 64 KiB pieces, one pin per piece
+])
+def test_stream_sum_lane_groups(B, page, frames):
+    """The streaming kernel takes as many pages per warp at a time as the pool lets every warp of its grid hold
+    (4, 2 or 1), and splits large pages into 64 KiB pieces: same sum, every page fetched once when the pool holds
+    them all, ragged first and last pages included."""
+    import torch
+    n = (1 << 20) + 4 * 37 + 3
+    a = inputs.fill_i32_u20(np.empty(n + 16, np.int32), n + 16, inputs.config_seed(1))
+    ar = Arena(page, {"a": a})
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    with paged(ar.host, page, frames) as h:
+        for skip in (0, 12):                                                 # start off the page grid (16-byte aligned)
+            B.gpuvm_reset(h)
+            B.gpuvm_stream_sum_i32(h, ar.off["a"] + 4 * skip, n, out)
+            st, ck = finish(h)
+            assert int(out.item()) == oracle.stream_sum_i32_direct(a[skip:skip + n])
+            touched = (4 * (skip + n) + page - 1) // page - (4 * skip) // page
+            if frames >= touched:
+                assert st["faults"] == touched and st["evictions"] == 0
+                B.gpuvm_stream_sum_i32(h, ar.off["a"] + 4 * skip, n, out)     # all hits now
+                st2, _ = finish(h)
+                assert st2["faults"] == touched and int(out.item()) == oracle.stream_sum_i32_direct(a[skip:skip + n])
+            else:
+                assert st["faults"] >= touched and st["evictions"] >= touched - frames
+
+
 @pytest.mark.parametrize("page,n,n_idx,block,frames", [
     (4096, 1 << 16, 1 << 14, 1024, 64),
     (4096, 1 << 16, (1 << 14) + 77, 1024, 16),     # ragged last block

@@ -341,3 +341,16 @@ def test_stream_scoped_reset_stats_check(B):
             ck = B.gpuvm_check_on(h, s)
             assert st["faults"] == 16 and st["evictions"] == 12 and ck["resident"] == 4 and ck["status"] == 0
             assert int(out.item()) == int(a.astype(np.int64).sum())
+
+
+def test_scattered_link_peak_runs_and_checks_its_arguments(B):
+    """gpuvm_link_peak_scattered reads rows at hashed positions of a pinned region and reports a rate; bad row
+    sizes and empty requests are refused."""
+    import torch
+    host = torch.zeros(64 << 20, dtype=torch.uint8).pin_memory()
+    buf = torch.empty(8 << 20, dtype=torch.uint8, device="cuda")
+    gbs = B.gpuvm_link_peak_scattered(host.data_ptr(), host.numel(), 512, 1 << 16, buf.data_ptr(), buf.numel(), 1)
+    assert 0.5 < gbs < 200.0
+    for row_bytes, n_rows in ((24, 16), (1024, 16), (512, 0)):
+        with pytest.raises(B.GpuvmError):
+            B.gpuvm_link_peak_scattered(host.data_ptr(), host.numel(), row_bytes, n_rows, buf.data_ptr(), buf.numel(), 1)
