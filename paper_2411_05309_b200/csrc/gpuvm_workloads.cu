@@ -1169,11 +1169,13 @@ constexpr unsigned int kEmbagLookups = 32;                 // lookups of a bag p
 constexpr unsigned int kEmbagChunk = 8192;                 // bytes per bulk copy of a migrator warp
 constexpr unsigned int kEmbagMaxGroups = 8;                // groups of 32 bags a requester warp takes at a time
 
-// How many lookups of the whole list name each page: the batched kernel reads the rows of pages with few
-// lookups in place and fetches the others at their first touch.  One atomic per group of equal pages in a warp.
+// How many lookups of the whole list name each page, up to `limit` (all the batched kernel asks is whether a page
+// reaches it): it reads the rows of pages below the limit in place and fetches the others at their first touch.
+// One atomic per group of equal pages in a warp, and none once a page's count has reached the limit, so the
+// hottest pages, which would serialise hundreds of thousands of atomics on one word each, cost a load.
 __global__ void embag_demand_kernel(const long long *__restrict__ rows, unsigned long long n, unsigned long long t_off,
                                     unsigned long long row_bytes, unsigned int page_shift, unsigned long long rows_inside,
-                                    unsigned int *__restrict__ demand)
+                                    unsigned int *__restrict__ demand, unsigned int limit)
 {
     const unsigned int lane = threadIdx.x & 31;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
@@ -1185,7 +1187,8 @@ __global__ void embag_demand_kernel(const long long *__restrict__ rows, unsigned
         const unsigned int mask = __ballot_sync(0xFFFFFFFFu, inside);
         if (inside) {
             const unsigned int group = __match_any_sync(mask, vpn);
-            if (lane == (unsigned int)__ffs(group) - 1u) atomicAdd(demand + vpn, (unsigned int)__popc(group));
+            if (lane == (unsigned int)__ffs(group) - 1u && gpuvm::ld_relaxed_u32(demand + vpn) < limit)
+                atomicAdd(demand + vpn, (unsigned int)__popc(group));
         }
     }
 }
@@ -2029,7 +2032,7 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
         if (cudaMemsetAsync(demand, 0, demand_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
         embag_demand_kernel<<<sm_count() * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
             reinterpret_cast<const long long *>(d_rows), (unsigned long long)n_bags * bag, t_off, row_bytes, m.vm.page_shift,
-            (m.vm.bytes - t_off) / row_bytes, demand);
+            (m.vm.bytes - t_off) / row_bytes, demand, inplace_limit);
         ++launches;
     }
     embag_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
