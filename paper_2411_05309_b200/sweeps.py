@@ -173,20 +173,28 @@ def sweep_depth(cfg: int, shrink: int):
     from . import binding as B
     from . import configs
     limits_mib = {2: [40, 80, 150, 0], 5: [2300, 4500, 0]}[cfg]
-    for limit in limits_mib:
-        w = configs.make(cfg, shrink)
-        try:
-            B.gpuvm_set_scratch_limit(w.h, (limit << 20) >> shrink)
-            w.run(check=False)
-            runs = [w.run() for _ in range(3)]
-            res = min(runs, key=lambda r: r.seconds)
-            print(json.dumps({"sweep": "depth", "workload": w.name, "scratch_limit_bytes": (limit << 20) >> shrink,
-                              "scratch_bytes": B.gpuvm_scratch_bytes(w.h), "pool_bytes": w.pool_bytes,
-                              "seconds": res.seconds, "faults": res.stats["faults"], "pages": w.nbytes // w.page_bytes,
-                              "bytes_in": res.stats["bytes_in"], "in_gbs": res.stats["bytes_in"] / res.seconds / 1e9,
-                              "effective_gbs": res.effective_bytes / res.seconds / 1e9}), flush=True)
-        finally:
-            w.close()
+    # the embedding bag under the paper's policy (every first touch fetches its page) and under the library's default
+    # (rows of pages with few lookups are read in place)
+    policies = {2: [("default", None)], 5: [("every first touch fetches", 0), ("default", None)]}[cfg]
+    for policy, divisor in policies:
+        for limit in limits_mib:
+            w = configs.make(cfg, shrink)
+            try:
+                B.gpuvm_set_scratch_limit(w.h, (limit << 20) >> shrink)
+                if divisor is not None:
+                    B.gpuvm_set_inplace_divisor(w.h, divisor)
+                w.run(check=False)
+                runs = [w.run() for _ in range(3)]
+                res = min(runs, key=lambda r: r.seconds)
+                print(json.dumps({"sweep": "depth", "workload": w.name, "policy": policy,
+                                  "scratch_limit_bytes": (limit << 20) >> shrink,
+                                  "scratch_bytes": B.gpuvm_scratch_bytes(w.h), "pool_bytes": w.pool_bytes,
+                                  "seconds": res.seconds, "faults": res.stats["faults"], "pages": w.nbytes // w.page_bytes,
+                                  "bytes_in": res.stats["bytes_in"], "bytes_direct": res.stats["bytes_direct"],
+                                  "in_gbs": res.stats["bytes_in"] / res.seconds / 1e9,
+                                  "effective_gbs": res.effective_bytes / res.seconds / 1e9}), flush=True)
+            finally:
+                w.close()
 
 
 def sweep_link(gib: float):
