@@ -949,8 +949,14 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
 // page, exactly one page of columns, however the degrees are distributed; a long neighbour list
 // is shared by as many workers as it has chunks.  A warp draws a chunk ticket, walks the chunk's
 // vertices 32 at a time, and expands the part of each active vertex's list that lies in the chunk.  counters: [0] updates, [2] chunk ticket.
+#ifndef GPUVM_BCSR_BLOCKS
+#define GPUVM_BCSR_BLOCKS 2            /* 128 registers, no spills: 37 ms for the CC against 40 ms with four blocks at 64 */
+#endif
+#ifndef GPUVM_BCSR_CC_BACKWARD
+#define GPUVM_BCSR_CC_BACKWARD 1
+#endif
 template <class Mem, class Op>
-__global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
+__global__ void __launch_bounds__(256, GPUVM_BCSR_BLOCKS) bcsr_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
                                                          unsigned long long chunk_off, unsigned int nv,
                                                          unsigned long long n_edges, unsigned int chunk_edges,
                                                          unsigned int *__restrict__ counters, int sweep)
@@ -981,45 +987,95 @@ __global__ void __launch_bounds__(256, 2) bcsr_sweep_kernel(Mem m, Op op, unsign
             const bool a = vk <= v_last && vk < nv && op.active(vk);
             group_active |= (__any_sync(0xFFFFFFFFu, a) ? 1u : 0u) << k;
         }
-        for (unsigned int v0 = g0; group_active; v0 += 32, group_active >>= 1) {
-            if (!(group_active & 1u)) continue;
+        if (!group_active) continue;
+        // The row offsets of these 256 vertices and of the one after them: one pin when they lie in one unit (a
+        // chunk in a region of low degrees walks a thousand groups of 32 vertices; a pin per group was most of
+        // its time).  Nothing else is pinned meanwhile: one page at a time, no pool is too small.
+        long long lo8[8], lo_next;
+        const unsigned long long ob = off_off + 8ull * g0;
+        if ((unsigned long long)g0 + 256 <= nv && ob % m.unit() + 257 * 8 <= m.unit()) {
+            gpuvm_token tok_o;
+            const unsigned char *po = m.pin(ob, GPUVM_READ, tok_o);
+            if (!po) return;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) lo8[k] = Mem::load_i64(po + 8 * (32 * k + lane));
+            lo_next = Mem::load_i64(po + 8 * 256);
+            m.release(tok_o);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const unsigned long long vk = (unsigned long long)g0 + 32u * k + lane;
+                lo8[k] = m.template read<long long>(off_off, vk < nv ? vk : nv);
+            }
+            lo_next = m.template read<long long>(off_off, (unsigned long long)g0 + 256 < nv ? (unsigned long long)g0 + 256 : nv);
+        }
+        // the chunk's column page: pinned at the first group that has an edge in it, held to the end of the block
+        gpuvm_token tok;
+        const unsigned char *p = nullptr;
+#pragma unroll
+        for (int k8 = 0; k8 < 8; ++k8) {
+            if (!((group_active >> k8) & 1u)) continue;
+            const unsigned int v0 = g0 + 32u * k8;
             const unsigned long long v = (unsigned long long)v0 + lane;
             const bool active = v <= v_last && v < nv && op.active(v);
             if (!__any_sync(0xFFFFFFFFu, active)) continue;
-            long long lo, hi;                                    // one pin for the 33 row offsets when they lie in one unit
-            const unsigned long long ob = off_off + 8ull * v0;
-            if ((unsigned long long)v0 + 32 <= nv && ob % m.unit() + 33 * 8 <= m.unit()) {
-                gpuvm_token tok_o;
-                const unsigned char *po = m.pin(ob, GPUVM_READ, tok_o);
-                if (!po) return;
-                lo = Mem::load_i64(po + 8 * lane);
-                hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
-                if (lane == 31) hi = Mem::load_i64(po + 8 * 32);
-                m.release(tok_o);
-            } else {
-                lo = m.template read<long long>(off_off, v < nv ? v : nv);
-                hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
-                if (lane == 31) hi = m.template read<long long>(off_off, v + 1 < nv ? v + 1 : nv);
-            }
+            long long lo = lo8[k8];
+            long long hi = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
+            const long long first_of_next = k8 < 7 ? __shfl_sync(0xFFFFFFFFu, lo8[k8 < 7 ? k8 + 1 : 7], 0) : lo_next;
+            if (lane == 31) hi = first_of_next;
             if (lo < c_lo) lo = c_lo;
             if (hi > c_hi) hi = c_hi;
             unsigned int touch = __ballot_sync(0xFFFFFFFFu, active && hi > lo);
             if (!touch) continue;
             const int uval = active ? op.begin(v) : 0;
-            // the chunk's column page is held only while these 32 vertices are expanded, never
-            // while row offsets are read: one page at a time, no pool is too small
-            gpuvm_token tok;
-            const unsigned char *p = m.pin(col_off + 4ull * c_lo, GPUVM_READ, tok);
-            if (!p) return;
-            while (touch) {
-                const int L = __ffs(touch) - 1;
-                touch &= touch - 1;
-                const long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
-                found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), __shfl_sync(0xFFFFFFFFu, uval, L),
-                                                     blo, bhi, lane, 0u);
+            if (!p) {
+                p = m.pin(col_off + 4ull * c_lo, GPUVM_READ, tok);
+                if (!p) return;
             }
-            m.release(tok);
+            if (__popc(touch) >= 8) {
+                // Many of the 32 vertices have edges here: their lists lie one after the other in the chunk, so
+                // the lanes take the edges of the whole stretch, 32 x 4 at a time, and each looks up whose edge
+                // it has (the last vertex whose list starts at or before it: a binary search over the 32 clipped
+                // starts, five shuffles).  Every lane works whatever the degrees are; with one list at a time a
+                // list of sixteen edges leaves half the warp idle and every list costs its own round trips.
+                const long long e_begin = __shfl_sync(0xFFFFFFFFu, lo, 0);
+                long long e_end = __shfl_sync(0xFFFFFFFFu, hi, 31);
+                if (e_end < e_begin) e_end = e_begin;
+                constexpr int U = 4;
+                for (long long b = e_begin; b < e_end; b += 32 * U) {
+                    int c[U], own[U], seen[U];
+#pragma unroll
+                    for (int k = 0; k < U; ++k) {
+                        const long long e = b + 32 * k + lane;
+                        int j = 0;
+#pragma unroll
+                        for (int step = 16; step; step >>= 1) {
+                            const long long lo_t = __shfl_sync(0xFFFFFFFFu, lo, (j + step) & 31);
+                            if (lo_t <= e) j += step;                   // starts are sorted; j + step <= 31 here
+                        }
+                        const bool mine = e < e_end && ((touch >> j) & 1u);
+                        own[k] = mine ? j : -1;
+                        c[k] = mine ? Mem::load_i32(p + 4 * (e - c_lo)) : -1;
+                    }
+#pragma unroll
+                    for (int k = 0; k < U; ++k) seen[k] = c[k] >= 0 ? op.peek(c[k]) : 0;
+#pragma unroll
+                    for (int k = 0; k < U; ++k) {
+                        const int uv = __shfl_sync(0xFFFFFFFFu, uval, own[k] & 31);
+                        if (c[k] >= 0) found += op.edge(uv, (long long)(v0 + own[k]), c[k], 0, seen[k], 0u);
+                    }
+                }
+            } else {
+                while (touch) {
+                    const int L = __ffs(touch) - 1;
+                    touch &= touch - 1;
+                    const long long blo = __shfl_sync(0xFFFFFFFFu, lo, L), bhi = __shfl_sync(0xFFFFFFFFu, hi, L);
+                    found += visit_edges<Mem, Op, false>(op, p, nullptr, c_lo, (long long)(v0 + L), __shfl_sync(0xFFFFFFFFu, uval, L),
+                                                         blo, bhi, lane, 0u);
+                }
+            }
         }
+        if (p) m.release(tok);
         }
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
@@ -1659,7 +1715,7 @@ int run_bfs_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off,
     unsigned int found = 1;
     while (rc == GPUVM_OK && found > 0 && n_edges > 0) {
         cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
-        bcsr_sweep_kernel<Mem, BfsOp><<<sm_count() * 2, 256, 0, s>>>(m, BfsOp{d_level, depth}, off_off, col_off, chunk_off,
+        bcsr_sweep_kernel<Mem, BfsOp><<<sm_count() * GPUVM_BCSR_BLOCKS, 256, 0, s>>>(m, BfsOp{d_level, depth}, off_off, col_off, chunk_off,
                                                                      (unsigned int)nv, n_edges, (unsigned int)chunk_edges,
                                                                      counters, depth);
         rc = launched();
@@ -1687,8 +1743,8 @@ int run_cc_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off, 
     int rc = launched();
     if (rc == GPUVM_OK && n_edges > 0) {
         cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
-        bcsr_sweep_kernel<Mem, CcOp><<<sm_count() * 2, 256, 0, s>>>(m, CcOp{d_label}, off_off, col_off, chunk_off, (unsigned int)nv,
-                                                                    n_edges, (unsigned int)chunk_edges, counters, 0);
+        bcsr_sweep_kernel<Mem, CcOp><<<sm_count() * GPUVM_BCSR_BLOCKS, 256, 0, s>>>(m, CcOp{d_label}, off_off, col_off, chunk_off, (unsigned int)nv,
+                                                                    n_edges, (unsigned int)chunk_edges, counters, GPUVM_BCSR_CC_BACKWARD);
         rc = launched();
     }
     cc_finish_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
