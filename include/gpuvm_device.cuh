@@ -150,11 +150,7 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 __device__ __forceinline__ unsigned long long pin_acquire(unsigned long long *pte)
 {
     unsigned long long old;
-#ifdef GPUVM_EXP_RELAXED_PIN
-    asm volatile("atom.relaxed.gpu.global.add.u64 %0, [%1], 1;" : "=l"(old) : "l"(pte) : "memory");
-#else
     asm volatile("atom.acquire.gpu.global.add.u64 %0, [%1], 1;" : "=l"(old) : "l"(pte) : "memory");
-#endif
     return old;
 }
 
@@ -186,11 +182,7 @@ __device__ __forceinline__ void st_relaxed_u32(unsigned int *p, unsigned int v)
  * barrier before it, its group's) frame accesses happen before the drop */
 __device__ __forceinline__ void unpin(unsigned long long *pte)
 {
-#ifdef GPUVM_EXP_RELAXED_UNPIN
-    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(pte), "l"(~0ull) : "memory");
-#else
     asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(pte), "l"(~0ull) : "memory");
-#endif
 }
 
 __device__ __forceinline__ void stat_add(const gpuvm_dev_t &vm, int kind, unsigned long long v)

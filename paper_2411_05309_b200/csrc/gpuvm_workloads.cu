@@ -949,14 +949,12 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
 // page, exactly one page of columns, however the degrees are distributed; a long neighbour list
 // is shared by as many workers as it has chunks.  A warp draws a chunk ticket, walks the chunk's
 // vertices 32 at a time, and expands the part of each active vertex's list that lies in the chunk.  counters: [0] updates, [2] chunk ticket.
-#ifndef GPUVM_BCSR_BLOCKS
-#define GPUVM_BCSR_BLOCKS 2            /* 128 registers, no spills: 37 ms for the CC against 40 ms with four blocks at 64 */
-#endif
-#ifndef GPUVM_BCSR_CC_BACKWARD
-#define GPUVM_BCSR_CC_BACKWARD 1
-#endif
+constexpr int kBcsrBlocksPerSm = 2;    // 128 registers, no spills: 37 ms for the CC against 40 ms with four blocks at 64
+// The CC draws its chunks from the last one down: in an RMAT graph the chunks of the sparse end span tens of
+// thousands of vertices each and take longest, so they go first and the short ones fill the tail (33 against 37 ms).
+constexpr int kBcsrCcSweep = 1;
 template <class Mem, class Op>
-__global__ void __launch_bounds__(256, GPUVM_BCSR_BLOCKS) bcsr_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
+__global__ void __launch_bounds__(256, kBcsrBlocksPerSm) bcsr_sweep_kernel(Mem m, Op op, unsigned long long off_off, unsigned long long col_off,
                                                          unsigned long long chunk_off, unsigned int nv,
                                                          unsigned long long n_edges, unsigned int chunk_edges,
                                                          unsigned int *__restrict__ counters, int sweep)
@@ -1715,7 +1713,7 @@ int run_bfs_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off,
     unsigned int found = 1;
     while (rc == GPUVM_OK && found > 0 && n_edges > 0) {
         cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
-        bcsr_sweep_kernel<Mem, BfsOp><<<sm_count() * GPUVM_BCSR_BLOCKS, 256, 0, s>>>(m, BfsOp{d_level, depth}, off_off, col_off, chunk_off,
+        bcsr_sweep_kernel<Mem, BfsOp><<<sm_count() * kBcsrBlocksPerSm, 256, 0, s>>>(m, BfsOp{d_level, depth}, off_off, col_off, chunk_off,
                                                                      (unsigned int)nv, n_edges, (unsigned int)chunk_edges,
                                                                      counters, depth);
         rc = launched();
@@ -1743,8 +1741,8 @@ int run_cc_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off, 
     int rc = launched();
     if (rc == GPUVM_OK && n_edges > 0) {
         cudaMemsetAsync(counters, 0, 4 * sizeof(unsigned int), s);
-        bcsr_sweep_kernel<Mem, CcOp><<<sm_count() * GPUVM_BCSR_BLOCKS, 256, 0, s>>>(m, CcOp{d_label}, off_off, col_off, chunk_off, (unsigned int)nv,
-                                                                    n_edges, (unsigned int)chunk_edges, counters, GPUVM_BCSR_CC_BACKWARD);
+        bcsr_sweep_kernel<Mem, CcOp><<<sm_count() * kBcsrBlocksPerSm, 256, 0, s>>>(m, CcOp{d_label}, off_off, col_off, chunk_off, (unsigned int)nv,
+                                                                    n_edges, (unsigned int)chunk_edges, counters, kBcsrCcSweep);
         rc = launched();
     }
     cc_finish_kernel<<<sm_count() * 4, 256, 0, s>>>(d_label, (unsigned int)nv);
