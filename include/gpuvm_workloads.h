@@ -239,6 +239,12 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
  * t_off a multiple of the row size.  Any other layout (dims = 20 or 100, pages smaller than a
  * row) is served by the unbatched kernel, with the same result.  A row id whose row does not lie
  * inside the backing store entirely sets the sticky GPUVM_E_RANGE.
+ * Which pages are fetched (gpuvm_set_inplace_divisor, gpuvm_set_inplace_counted in gpuvm.h): by default a short
+ * kernel first counts the lookups per page (4 bytes of scratch per page); the rows of pages with fewer lookups than
+ * a quarter of the page holds are read in place from the backing store (counted as bytes_direct, no fault, the page
+ * table untouched), every other page is fetched at its first touch.  With the divisor 0 every first touch fetches
+ * its page, as in the paper.  The result is the same bit for bit; the table must not be written through the
+ * runtime while the call runs.
  * gpuvm_embag_f32_unbatched: one warp per bag, one row request at a time through
  * gpuvm_read; no scratch.
  */
