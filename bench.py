@@ -36,7 +36,7 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-DEFAULT_INPLACE_DIVISOR = 4          # the library's default (include/gpuvm.h, gpuvm_set_inplace_divisor)
+DEFAULT_INPLACE_DIVISOR = 0xFFFFFFFF  # GPUVM_INPLACE_AUTO, the library's default (include/gpuvm.h, gpuvm_set_inplace_divisor)
 METRIC = "effective_app_GBps"
 UNIT = "GB/s"
 
@@ -535,7 +535,7 @@ def run_config(torch, B, configs, cfg: int, args, steps: int, warmup: int, link:
             rec["roofline"]["compulsory_pages"] = pages
             rec["roofline"]["frac_compulsory"] = pages * w.page_bytes / kern_s / 1e9 / link["ce_h2d_gbs"]
         if cfg == 5:
-            rec["migration"]["inplace_divisor"] = args.inplace_divisor if args.inplace_divisor >= 0 else DEFAULT_INPLACE_DIVISOR
+            rec["migration"]["inplace_divisor"] = args.inplace_divisor if args.inplace_divisor >= 0 else "auto"
         if cfg == 5 and rank == 0:
             rec["roofline"].update(embag_policy_records(torch, B, w, args, link, kern_s, direct, rec))
         if cfg in (2, 5) and not args.scratch_limit_mib:

@@ -226,26 +226,33 @@ int gpuvm_set_clean_ahead(gpuvm_t h, unsigned int frames);
 int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes);
 size_t gpuvm_scratch_bytes(gpuvm_t h);
 
-/* Rent or buy (not in the paper, which fetches a page at its first fault).  The batched row workloads
- * (gpuvm_embag_f32) do not fetch a page for its first requests: while the requests served from a page since it
- * was last resident have read less than page_bytes / divisor over the link, the next one reads its row in place
- * from the backing store (pinned host memory is as reachable for a load as for a page copy) and the page stays
- * where it is; the request after that fetches it.  A page that is asked for a few times never costs a page of
- * traffic; one that turns out hot costs at most 1 / divisor more than if it had been fetched at once.  Counted in
- * gpuvm_stats as bytes_direct.  Only for reads, and only right for data that is not written through the
- * runtime while such a kernel runs.  divisor: default 4; 0 = off (every first touch fetches the page).
- * Why 4 and not 1 (the break-even point by bytes): a row read in place is a scattered link read, and over a
- * 64 GiB backing store those were measured at 24.5 GB/s however many were in flight (51.4 GB/s over 1 GiB, 33.4
- * over 8 GiB: address translation on the host side), while page copies run at 51.4 GB/s beside them; the two
- * streams finish together near a quarter (measured on the 64 GiB Zipf table: 70 / 61 / 77 ms for 2 / 4 / 8). */
+/* Reading rows in place instead of fetching their page (not in the paper, which fetches a page at its first
+ * fault).  The batched row workloads (gpuvm_embag_f32) do not fetch a page for a few rows: pinned host memory is as
+ * reachable for a load as for a page copy, so rows of pages with few lookups are read in place from the backing
+ * store and the page stays where it is.  A page is worth fetching when its lookups would otherwise move at least
+ * page_bytes / divisor over the link; limit = page_bytes / divisor / max(row_bytes, 128) lookups.  Rows read in
+ * place are counted in gpuvm_stats as bytes_direct.  Only for reads, and only right for data that is not written
+ * through the runtime while such a kernel runs.
+ * divisor: 0 = off (every first touch fetches the page, as in the paper); GPUVM_INPLACE_AUTO (default) = 1 when
+ * the rows read in place can be read page by page (see below), else 4.  Why: sequential reads over the link run
+ * at 51.4 GB/s, and so do rows read page by page, so the break-even point is the page's own size; rows read one
+ * lookup after the other are scattered over the table, and scattered reads over a 64 GiB pinned region were
+ * measured at 24.5 GB/s however many were in flight (51.4 over 1 GiB, 33.4 over 8 GiB: address translation on the
+ * host side), beside page copies at the full rate: the two streams finish together near a quarter of a page
+ * (measured on the 64 GiB Zipf table, scattered: 70 / 61 / 77 ms for the divisors 2 / 4 / 8). */
+#define GPUVM_INPLACE_AUTO 0xFFFFFFFFu
 int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor);
 
-/* How the batched row workloads decide which pages are worth fetching.  counted != 0 (default): a short kernel
+/* How the batched row workloads find the pages that are worth fetching.  counted != 0 (default): a short kernel
  * first counts, per page, the lookups of the whole list (the list is the kernel's input, so the demand is
- * known before the first access); rows of pages with fewer than page_bytes / divisor / row_bytes lookups are
- * read in place without the page table being touched, every other page is fetched at its first touch: no
- * row of a page that will be fetched anyway is read in place first.  counted == 0: the online form described
- * above, which needs no pass over the list. */
+ * known before the first access); rows of pages below the limit are read in place without the page table being
+ * touched, every other page is fetched at its first touch (it is handed to the migrator warps before the first
+ * lookup, unless such pages would fill more than half the pool): no row of a page that will be fetched anyway is
+ * read in place first.  When every lookup has a staging slot of its own (all bags in flight at once: the default
+ * without gpuvm_set_scratch_limit), the lookups of the pages that are not fetched are also bucketed by page and
+ * their rows read page by page, at the link's sequential rate.  counted == 0: the online form, which needs no
+ * pass over the list: the first `limit` requests that find a page absent read their rows in place (counted in the
+ * frame field of the invalid entry), the next one fetches the page. */
 int gpuvm_set_inplace_counted(gpuvm_t h, int counted);
 
 /* Largest number of simultaneously resident warps that can each hold

@@ -206,6 +206,9 @@ def gpuvm_check_on(h, stream, raise_on_error: bool = True) -> dict:
     return d
 
 
+INPLACE_AUTO = 0xFFFFFFFF
+
+
 def gpuvm_set_inplace_divisor(h, divisor: int):
     _check(lib().gpuvm_set_inplace_divisor(h, divisor), "gpuvm_set_inplace_divisor")
 

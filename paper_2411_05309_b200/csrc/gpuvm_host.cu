@@ -146,7 +146,7 @@ int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_byt
     memset(h, 0, sizeof(*h));
     cudaGetDevice(&h->device);
     h->sms = sm_count_of(h->device);
-    h->inplace_divisor = 4;
+    h->inplace_divisor = GPUVM_INPLACE_AUTO;
     h->inplace_counted = true;
     cudaError_t e;
 

@@ -14,7 +14,7 @@ struct gpuvm_handle;
 void *gpuvm_scratch_(struct gpuvm_handle *h, size_t bytes);
 /* bound set with gpuvm_set_scratch_limit, SIZE_MAX when there is none */
 size_t gpuvm_scratch_limit_(struct gpuvm_handle *h);
-/* divisor set with gpuvm_set_inplace_divisor (default 4; 0: requests are never served in place) and
+/* divisor set with gpuvm_set_inplace_divisor (default GPUVM_INPLACE_AUTO; 0: requests are never served in place) and
  * whether lookups are counted per page first (gpuvm_set_inplace_counted, default yes) */
 size_t gpuvm_inplace_divisor_(struct gpuvm_handle *h);
 int gpuvm_inplace_counted_(struct gpuvm_handle *h);

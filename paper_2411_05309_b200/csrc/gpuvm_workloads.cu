@@ -1221,6 +1221,10 @@ constexpr int kEmbagRequesters = 28;
 constexpr int kEmbagMigrators = 4;
 constexpr unsigned int kEmbagLookups = 32;                 // lookups of a bag per batch (table rows)
 constexpr unsigned int kEmbagChunk = 8192;                 // bytes per bulk copy of a migrator warp
+// Bulk copies a migrator warp keeps in flight.  Rows read in place keep thousands of 512-byte reads outstanding,
+// and the link serves its queue in order: a page copy with one 8 KiB chunk outstanding per warp gets a
+// correspondingly small share and the pages arrive after the rows.
+constexpr unsigned int kEmbagStages = 4;                    // 57 / 50 / 46 / 46 ms for 1 / 2 / 4 / 6 on the 64 GiB Zipf table
 constexpr unsigned int kEmbagMaxGroups = 8;                // groups of 32 bags a requester warp takes at a time
 
 // How many lookups of the whole list name each page, up to `limit` (all the batched kernel asks is whether a page
@@ -1247,17 +1251,110 @@ __global__ void embag_demand_kernel(const long long *__restrict__ rows, unsigned
     }
 }
 
+// Grouped reads in place.  Rows read in place one lookup after the other are scattered over the whole table, and
+// scattered reads over a large pinned region are slow on the host side (24.5 GB/s over 64 GiB against 51.4 for
+// sequential ones); the same rows read page by page go at 50 GB/s.  So the lookups of the pages that are not
+// fetched ("cold": fewer lookups than the limit) are bucketed by page first: bucket_off[p] becomes the start of page
+// p's bucket (an exclusive scan of the cold pages' counts; one block, 1024 pages per step), the fill kernel puts
+// every cold lookup's number into its page's bucket, and the main kernel reads the rows in bucket order.
+// counts[0] = number of cold lookups, counts[1] = number of pages that will be fetched.
+__global__ void __launch_bounds__(1024) embag_bucket_scan_kernel(const unsigned int *__restrict__ demand, unsigned int n_pages,
+                                                                  unsigned int limit, unsigned int *__restrict__ bucket_off,
+                                                                  unsigned int *__restrict__ counts)
+{
+    __shared__ unsigned int warp_sums[32];
+    __shared__ unsigned int carry_s, hot_s;
+    const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { carry_s = 0; hot_s = 0; }
+    __syncthreads();
+    unsigned int hot = 0;
+    for (unsigned int base = 0; base < n_pages; base += 1024) {
+        const unsigned int p = base + threadIdx.x;
+        const unsigned int d = p < n_pages ? demand[p] : 0u, v = d < limit ? d : 0u;
+        hot += p < n_pages && d >= limit;
+        unsigned int x = v;                                      // inclusive scan in the warp
+        for (int o = 1; o < 32; o <<= 1) { const unsigned int y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= (unsigned int)o) x += y; }
+        if (lane == 31) warp_sums[warp] = x;
+        __syncthreads();
+        if (warp == 0) {                                         // exclusive scan of the 32 warp totals
+            const unsigned int t = warp_sums[lane];
+            unsigned int e = t;
+            for (int o = 1; o < 32; o <<= 1) { const unsigned int y = __shfl_up_sync(0xFFFFFFFFu, e, o); if (lane >= (unsigned int)o) e += y; }
+            warp_sums[lane] = e - t;
+        }
+        __syncthreads();
+        const unsigned int carry = carry_s;
+        if (p < n_pages) bucket_off[p] = carry + warp_sums[warp] + x - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = carry + warp_sums[31] + x;
+        __syncthreads();
+    }
+    for (int o = 16; o; o >>= 1) hot += __shfl_down_sync(0xFFFFFFFFu, hot, o);
+    if (lane == 0 && hot) atomicAdd(&hot_s, hot);
+    __syncthreads();
+    if (threadIdx.x == 0) { counts[0] = carry_s; counts[1] = hot_s; }
+}
+
+// After this kernel bucket_off[p] is the END of page p's bucket (every cold lookup moved it on by one).
+__global__ void embag_bucket_fill_kernel(const long long *__restrict__ rows, unsigned long long n, unsigned long long t_off,
+                                         unsigned long long row_bytes, unsigned int page_shift, unsigned long long rows_inside,
+                                         const unsigned int *__restrict__ demand, unsigned int limit,
+                                         unsigned int *__restrict__ bucket_off, unsigned int *__restrict__ cold_idx)
+{
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n; i += stride) {
+        const unsigned long long r = (unsigned long long)rows[i];
+        if (r >= rows_inside) continue;
+        const unsigned int vpn = (unsigned int)((t_off + r * row_bytes) >> page_shift);
+        if (demand[vpn] < limit) cold_idx[atomicAdd(bucket_off + vpn, 1u)] = (unsigned int)i;
+    }
+}
+
+// Where the row of lookup i is staged when every requester warp has one item (one pass): the layout the main
+// kernel's tables use (request ((gi * bag + k) * 32 + b) of the warp that has bag g0 + 32 gi + b).
+__device__ __forceinline__ size_t embag_staged_row(unsigned long long i, unsigned int bag, unsigned int groups)
+{
+    const unsigned long long g = i / bag, per_item = 32ull * groups;
+    const unsigned int k = (unsigned int)(i - g * bag);
+    const unsigned long long t = g / per_item;
+    const unsigned int rr = (unsigned int)(g - t * per_item), gi = rr >> 5, b = rr & 31u;
+    return (size_t)t * ((size_t)groups * 32 * bag) + (size_t)((gi * bag + k) * 32 + b);
+}
+
+// The bags' sums as a kernel of their own (grouped mode: the rows of a bag are staged by many warps, so the sums
+// wait for the whole main kernel): one warp per bag, the rows added in list order.
+__global__ void embag_sum_kernel(const unsigned char *__restrict__ g_staging, unsigned int dims, unsigned long long n_bags,
+                                 unsigned int bag, unsigned int groups, float *__restrict__ out)
+{
+    const unsigned int lane = threadIdx.x & 31, q = dims >> 2;
+    const uint4 *staging = reinterpret_cast<const uint4 *>(g_staging);
+    for (unsigned long long g = warp_in_grid(); g < n_bags; g += warps_in_grid()) {
+        if (lane >= q) continue;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+        for (unsigned int k = 0; k < bag; ++k) {
+            const uint4 v = staging[embag_staged_row(g * bag + k, bag, groups) * q + lane];
+            acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
+            acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
+            acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
+            acc.w = __fadd_rn(acc.w, __uint_as_float(v.w));
+        }
+        reinterpret_cast<float4 *>(out + g * dims)[lane] = acc;
+    }
+}
+
 __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
                                                               const long long *__restrict__ rows, unsigned long long n_bags,
                                                               unsigned int bag, float *__restrict__ out, int requesters,
                                                               gpuvm_batch_entry *g_tables, unsigned char *g_staging,
                                                               unsigned int groups, bool one_pass,
                                                               gpuvm_shared_queue *shared_queue, unsigned int inplace_limit,
-                                                              const unsigned int *demand)
+                                                              const unsigned int *demand, const unsigned int *cold_idx,
+                                                              const unsigned int *cold_counts)
 {
     __shared__ gpuvm_fault_queue queue_s;
-    __shared__ __align__(128) unsigned char stage_s[kEmbagMigrators][kEmbagChunk];   // bulk-copy staging of the migrator warps
-    __shared__ __align__(8) unsigned long long mbar_s[kEmbagMigrators];
+    extern __shared__ __align__(128) unsigned char stage_s[];   // bulk-copy staging: kEmbagStages chunks per migrator warp
+    __shared__ __align__(8) unsigned long long mbar_s[kEmbagMigrators][kEmbagStages];
     gpuvm_fault_queue *queue = &queue_s;
     const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
@@ -1269,7 +1366,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
         const unsigned int mig = warp - requesters;
         const unsigned int chunk = (1ull << vm.page_shift) < kEmbagChunk ? (unsigned int)(1ull << vm.page_shift) : kEmbagChunk;
         if (mig < kEmbagMigrators && chunk >= 128)
-            gpuvm_migrator_loop(vm, queue, stage_s[mig], &mbar_s[mig], chunk, 1);
+            gpuvm_migrator_loop(vm, queue, stage_s + (size_t)mig * kEmbagStages * kEmbagChunk, mbar_s[mig], chunk, kEmbagStages);
         else
             gpuvm_migrator_loop(vm, queue);
         return;
@@ -1285,6 +1382,51 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
     const unsigned long long items = (n_bags + per_item - 1) / per_item;
     const unsigned long long stride = (unsigned long long)gridDim.x * requesters;
     const unsigned long long rows_inside = (vm.bytes - t_off) / row_bytes;   // rows that lie in the backing store entirely
+    const bool grouped = cold_idx != nullptr;                    // one pass, every lookup's staging slot is known (embag_staged_row)
+    if (grouped) {
+        // (1) The pages that will be fetched are asked for up front, so that the migrator warps move them while the
+        // requesters read the other pages' rows: a warp looks at its share of the page counts and hands every
+        // page at or above the limit that nobody has asked for yet to the fault ring.  Not when those pages
+        // would fill more than half the pool: then they are fetched as their lookups come up.
+        const unsigned int n_cold = cold_counts[0], n_hot = cold_counts[1];
+        if (2ull * n_hot <= vm.n_frames) {
+            for (unsigned long long p = slot * 32 + lane; p < vm.n_pages; p += stride * 32) {
+                if (demand[p] < inplace_limit) continue;
+                const unsigned long long w = gpuvm::ld_relaxed_u64(vm.pte + p);
+                if ((w & gpuvm::kStMask) != gpuvm::kInvalid) continue;
+                if (atomicCAS(vm.pte + p, w, (w & ~gpuvm::kFrameMask) | gpuvm::kBusy) != w) continue;
+                if (!gpuvm::fault_queue_push(queue, (unsigned int)p, gpuvm::kRead, &vm))
+                    atomicXor(vm.pte + p, gpuvm::kBusy);         // the ring is full: back to INVALID, its lookups will fetch it
+            }
+            __syncwarp();
+        }
+        // (2) The rows of the other pages, in bucket order (page by page), four in flight per warp; the warps of
+        // the grid take neighbouring entries, so at any moment the reads in flight fall into a few hundred pages.
+        unsigned int n_here = 0;
+        constexpr int Q = 4;
+        uint4 *const all_staging = reinterpret_cast<uint4 *>(g_staging);
+        for (unsigned long long j0 = slot * Q; j0 < n_cold; j0 += stride * Q) {
+            uint4 v[Q];
+            size_t where[Q];
+            int cnt = 0;
+#pragma unroll
+            for (int u = 0; u < Q; ++u) {
+                where[u] = 0;
+                if (j0 + u < n_cold) {
+                    const unsigned int i = cold_idx[j0 + u];
+                    const unsigned long long r = (unsigned long long)rows[i];
+                    where[u] = embag_staged_row(i, bag, groups) * q;
+                    if (lane < q) v[u] = gpuvm_load16(vm.host + t_off + r * row_bytes + 16u * lane);
+                    cnt = u + 1;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < Q; ++u)
+                if (u < cnt && lane < q) all_staging[where[u] + lane] = v[u];
+            n_here += cnt;
+        }
+        if (lane == 0 && n_here) gpuvm::stat_add(vm, gpuvm::kBytesDirect, (unsigned long long)n_here * row_bytes);
+    }
     for (unsigned long long t = slot; t < items; t += stride) {
         const unsigned long long g0 = per_item * t;
         for (unsigned int k0 = 0; k0 < bag; k0 += kEmbagLookups) {
@@ -1297,7 +1439,10 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                         // a row that ends past the backing store is refused like one that starts there
                         const unsigned long long r = (unsigned long long)rows[g * bag + k0 + k];
                         const bool inside = r < rows_inside;
-                        gpuvm_batch_set(vm, table, (gi * nk + k) * 32 + lane, inside ? t_off + r * row_bytes : ~0ull);
+                        if (grouped && inside && demand[(t_off + r * row_bytes) >> vm.page_shift] < inplace_limit)
+                            gpuvm_batch_skip(table, (gi * nk + k) * 32 + lane);          // its row is staged by step (2)
+                        else
+                            gpuvm_batch_set(vm, table, (gi * nk + k) * 32 + lane, inside ? t_off + r * row_bytes : ~0ull);
                     } else
                         gpuvm_batch_skip(table, (gi * nk + k) * 32 + lane);
                 }
@@ -1305,8 +1450,10 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
             // every served row is copied to its slot of the staging area by the whole warp (the engine does it
             // itself, four rows in flight: gpuvm_row_copy), from its frame or in place from the backing store
             gpuvm_batch_run<true>(vm, gpuvm_entry_table{table}, groups * nk * 32, GPUVM_READ, gpuvm_row_copy{staging, q},
-                                  queue, masks, 1u, one_pass, inplace_limit, (unsigned int)row_bytes, demand);
+                                  queue, masks, 1u, one_pass, grouped ? 0u : inplace_limit, (unsigned int)row_bytes,
+                                  grouped ? nullptr : demand);
             __syncwarp();
+            if (grouped) continue;                               // the sums follow in embag_sum_kernel
             // add the staged rows of each bag in list order
             for (unsigned int gb = 0; gb < 32 * groups && g0 + gb < n_bags; ++gb) {
                 if (lane < q) {
@@ -2065,34 +2212,67 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     const size_t slots = items < (size_t)grid * requesters ? items : (size_t)grid * requesters;   // warps that get work
     const size_t table_bytes = (slots * per_warp * sizeof(gpuvm_batch_entry) + 255) & ~size_t(255);
     const size_t staging_bytes = (slots * per_warp * 4 * dims + 255) & ~size_t(255);
+    const bool one_pass = items <= (size_t)grid * requesters && bag <= kEmbagLookups;
+    // Which pages are fetched.  A page is fetched when its lookups would move at least page_bytes / divisor in place
+    // (gpuvm_set_inplace_divisor); the rows of the others are read in place from the backing store.  The lookup
+    // list is at hand, so the lookups per page are counted before the first access (gpuvm_set_inplace_counted);
+    // when, in addition, every lookup's staging slot is known beforehand (one pass) the rows read in place are
+    // bucketed by page and read page by page ("grouped"), which the host link serves at its full rate, and
+    // the break-even point is the page's size (divisor 1); read one lookup after the other they are scattered
+    // over the table and served at half that rate or less, and a quarter of the page is where the two streams
+    // balance (divisor 4).  A row is a whole number of 128-byte link reads when it is a multiple of 128 bytes
+    // long; shorter rows are charged 128 bytes.
+    const size_t n_lookups = n_bags * bag;
+    const bool counted = gpuvm_inplace_counted_(h) != 0;
     const size_t demand_bytes = (m.vm.n_pages * sizeof(unsigned int) + 255) & ~size_t(255);
-    unsigned char *scratch = static_cast<unsigned char *>(
-        gpuvm_scratch_(h, table_bytes + staging_bytes + sizeof(gpuvm_shared_queue) + demand_bytes));
-    if (!scratch) return GPUVM_E_ALLOC;
-    gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, scratch + table_bytes + staging_bytes, static_cast<cudaStream_t>(stream));
-    // Rent or buy: a page is fetched only once its rows have been asked for often enough to have moved a stated
-    // fraction of its size over the link (gpuvm_set_inplace_divisor; a quarter of it by default); until then its rows
-    // are read in place from the backing store.  A row is a whole number of 128-byte link reads when it is a
-    // multiple of 128 bytes long; shorter rows are charged 128 bytes.
-    const size_t divisor = gpuvm_inplace_divisor_(h);
+    const size_t index_bytes = (n_lookups * sizeof(unsigned int) + 255) & ~size_t(255);
+    const size_t base_bytes = table_bytes + staging_bytes + sizeof(gpuvm_shared_queue) + demand_bytes;
+    const bool grouped = counted && one_pass && n_lookups < 0xFFFFFFFFull && m.vm.n_pages <= (1ull << 20) &&
+                         (gpuvm_scratch_limit_(h) == ~size_t(0) || base_bytes + demand_bytes + index_bytes + 256 <= gpuvm_scratch_limit_(h));
+    size_t divisor = gpuvm_inplace_divisor_(h);
+    if (divisor == GPUVM_INPLACE_AUTO) divisor = grouped ? 1 : 4;
     const size_t charged = row_bytes < 128 ? 128 : row_bytes;
     const unsigned int inplace_limit = divisor ? (unsigned int)(page_bytes / divisor / charged) : 0u;
-    // The lookup list is at hand, so the lookups per page can be counted before the first access: pages below the
-    // limit are then read in place throughout and the others fetched at once (gpuvm_set_inplace_counted).
-    unsigned int *demand = nullptr;
+    const bool use_grouped = grouped && inplace_limit != 0u;
+    unsigned char *scratch = static_cast<unsigned char *>(
+        gpuvm_scratch_(h, base_bytes + (use_grouped ? demand_bytes + index_bytes + 256 : 0)));
+    if (!scratch) return GPUVM_E_ALLOC;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, scratch + table_bytes + staging_bytes, s);
+    unsigned int *demand = nullptr, *bucket_off = nullptr, *cold_idx = nullptr, *cold_counts = nullptr;
     unsigned long long launches = 1;
-    if (inplace_limit != 0u && gpuvm_inplace_counted_(h)) {
+    const long long *rows_ll = reinterpret_cast<const long long *>(d_rows);
+    const unsigned long long rows_inside = (m.vm.bytes - t_off) / row_bytes;
+    if (inplace_limit != 0u && counted) {
         demand = reinterpret_cast<unsigned int *>(scratch + table_bytes + staging_bytes + sizeof(gpuvm_shared_queue));
-        if (cudaMemsetAsync(demand, 0, demand_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
-        embag_demand_kernel<<<sm_count() * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-            reinterpret_cast<const long long *>(d_rows), (unsigned long long)n_bags * bag, t_off, row_bytes, m.vm.page_shift,
-            (m.vm.bytes - t_off) / row_bytes, demand, inplace_limit);
+        if (cudaMemsetAsync(demand, 0, demand_bytes, s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+        embag_demand_kernel<<<sm_count() * 8, 256, 0, s>>>(rows_ll, n_lookups, t_off, row_bytes, m.vm.page_shift, rows_inside,
+                                                            demand, inplace_limit);
+        ++launches;
+        if (use_grouped) {
+            bucket_off = reinterpret_cast<unsigned int *>(scratch + base_bytes);
+            cold_idx = reinterpret_cast<unsigned int *>(scratch + base_bytes + demand_bytes);
+            cold_counts = reinterpret_cast<unsigned int *>(scratch + base_bytes + demand_bytes + index_bytes);
+            embag_bucket_scan_kernel<<<1, 1024, 0, s>>>(demand, (unsigned int)m.vm.n_pages, inplace_limit, bucket_off, cold_counts);
+            embag_bucket_fill_kernel<<<sm_count() * 8, 256, 0, s>>>(rows_ll, n_lookups, t_off, row_bytes, m.vm.page_shift,
+                                                                 rows_inside, demand, inplace_limit, bucket_off, cold_idx);
+            launches += 2;
+        }
+    }
+    const size_t stage_bytes = (size_t)kEmbagMigrators * kEmbagStages * kEmbagChunk;
+    if (stage_bytes > 40 * 1024 &&
+        cudaFuncSetAttribute(embag_batch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return GPUVM_E_CUDA;
+    }
+    embag_batch_kernel<<<grid, (requesters + migrators) * 32, stage_bytes, s>>>(
+        m.vm, t_off, (unsigned int)dims, rows_ll, n_bags, (unsigned int)bag, d_out,
+        requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes, groups, one_pass, shared_queue,
+        inplace_limit, demand, cold_idx, cold_counts);
+    if (use_grouped) {
+        embag_sum_kernel<<<sm_count() * 8, 256, 0, s>>>(scratch + table_bytes, (unsigned int)dims, n_bags, (unsigned int)bag, groups, d_out);
         ++launches;
     }
-    embag_batch_kernel<<<grid, (requesters + migrators) * 32, 0, static_cast<cudaStream_t>(stream)>>>(
-        m.vm, t_off, (unsigned int)dims, reinterpret_cast<const long long *>(d_rows), n_bags, (unsigned int)bag, d_out,
-        requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes, groups,
-        /* one_pass = */ items <= (size_t)grid * requesters && bag <= kEmbagLookups, shared_queue, inplace_limit, demand);
     return launched(launches);
 }
 

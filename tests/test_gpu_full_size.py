@@ -161,15 +161,16 @@ def test_cfg5_zipf_embedding_bag_64GiB():
             assert np.array_equal(ref.view(np.uint32), out[start:start + step].view(np.uint32)), start
         st = res.stats
         distinct = np.unique(rows >> 12).size                   # 4096 rows per 2 MiB page
-        # Pages with fewer than 1024 lookups (a quarter of their 4096 rows) are never fetched: their rows are read
-        # in place, every one of them; the others are fetched once, at their first touch (all requests are in
-        # flight together and 615 pages fit the pool)
+        # Pages with fewer lookups than they have rows (4096) are never fetched: their rows are read in place, page
+        # by page, every one of them; the others are fetched once (all requests are in flight together and 163
+        # pages fit the pool)
         per_page = np.bincount(rows >> 12, minlength=w.n_pages)
-        limit = (2 << 20) // 4 // 512
+        limit = (2 << 20) // 512
         assert st["faults"] == np.count_nonzero(per_page >= limit)
         assert st["bytes_direct"] == int(per_page[per_page < limit].sum()) * 512
         B = __import__("paper_2411_05309_b200.binding", fromlist=["x"])
-        # the online form (no count beforehand): a page is fetched after 1024 of its rows have been read in place
+        # the online form (no count beforehand): a page is fetched after 1024 of its rows (a quarter) have been read in place
+        limit = (2 << 20) // 4 // 512
         B.gpuvm_set_inplace_counted(w.h, False)
         res1 = w.run()
         st1 = res1.stats
