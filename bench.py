@@ -130,7 +130,7 @@ NCU_LINK_TRAFFIC = {
         "full size; sweep 1 of the four sweeps of a run, 95 % of its time"),
     4: (33554432 * 32 * 8 + (4 << 30), "vadd_kernel_cfg4_eighth_full_set.md", 33554432,
         "1/8 case x 8: 8 GiB in, plus the 4 GiB of c that go out"),
-    5: (76624608 * 32, "embag_batch_kernel_cfg5_counted_policy.md", 76624608,
+    5: (60863056 * 32, "embag_batch_kernel_cfg5_counted_policy.md", 60863056,
         "full size, default policy; one metric, one pass"),
     "5_always_migrate": (134217728 * 32 * 16, "embag_batch_kernel_cfg5_sixteenth_full_set.md", 134217728,
                          "1/16 case x 16, every first touch fetching its page"),
@@ -416,11 +416,12 @@ def e2e_step(torch, B, w, cfg: int):
 
 
 def embag_policy_records(torch, B, w, args, link: dict, kern_s: float, direct: float, rec: dict) -> dict:
-    """cfg 5 runs with the library's default: lookups are counted per page first, rows of pages with fewer lookups
-    than a quarter of their rows are read in place, the other pages are fetched at their first touch.  Reported
-    beside it: the ceiling of scattered row reads over this backing store, measured here, which bounds the rows
-    read in place; the online form of the policy (no count beforehand); and the same launch with the policy off
-    (the paper's way: every first touch fetches the page), each with its own link roofline."""
+    """cfg 5 runs with the library's default: lookups are counted per page first, the rows of pages with fewer
+    lookups than rows are read in place, page by page, the other pages are fetched once.  Reported beside it: the
+    ceiling of scattered row reads over this backing store, measured here; the same policy with the rows read as
+    their lookups come up (scattered: that ceiling bounds it); the online form (no count beforehand); and the same
+    launch with the policy off (the paper's way: every first touch fetches the page), each with its own link
+    roofline."""
     out = {}
     row_bytes = 4 * w.dims
     buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -428,9 +429,10 @@ def embag_policy_records(torch, B, w, args, link: dict, kern_s: float, direct: f
     del buf
     out["in_place"] = {
         "bytes": direct, "gbs": direct / kern_s / 1e9 if kern_s else 0.0, "scattered_read_peak_gbs": scattered,
-        "frac": direct / kern_s / 1e9 / scattered if kern_s and scattered else None,
-        "what": f"rows read in place from the backing store; the peak is {1 << 22} rows of {row_bytes} B at hashed "
-                f"positions of the same {w.nbytes >> 30} GiB region, four in flight per warp, measured in this run"}
+        "what": f"rows read in place from the backing store, page by page (bucketed by page first); "
+                f"scattered_read_peak_gbs is what {1 << 22} rows of {row_bytes} B at hashed positions of the same "
+                f"{w.nbytes >> 30} GiB region reach, four in flight per warp, measured in this run: the ceiling of "
+                f"reading them as their lookups come up (roofline.counted_scattered)"}
     if args.inplace_divisor < 0 and not args.scratch_limit_mib:
         def other_policy(what, setup, restore):
             setup()
@@ -448,10 +450,14 @@ def embag_policy_records(torch, B, w, args, link: dict, kern_s: float, direct: f
                     "bytes_direct": st.get("bytes_direct", 0), "in_gbs": st["bytes_in"] / secs / 1e9,
                     "invariants_status": rs[-1].check["status"], "roofline": roof}
 
+        out["counted_scattered"] = other_policy(
+            "gpuvm_set_inplace_counted(h, 1): lookups counted per page first, rows of pages with fewer lookups than a "
+            "quarter of their rows read in place as their lookups come up (scattered over the table)",
+            lambda: B.gpuvm_set_inplace_counted(w.h, 1), lambda: B.gpuvm_set_inplace_counted(w.h, 2))
         out["online"] = other_policy(
             "gpuvm_set_inplace_counted(h, 0): no count beforehand; the first requests that find a page absent read "
             "their rows in place, the one after them fetches the page",
-            lambda: B.gpuvm_set_inplace_counted(w.h, False), lambda: B.gpuvm_set_inplace_counted(w.h, True))
+            lambda: B.gpuvm_set_inplace_counted(w.h, 0), lambda: B.gpuvm_set_inplace_counted(w.h, 2))
         rec_am = other_policy(
             "gpuvm_set_inplace_divisor(h, 0): every first touch fetches the page, as in the paper",
             lambda: B.gpuvm_set_inplace_divisor(w.h, 0), lambda: B.gpuvm_set_inplace_divisor(w.h, DEFAULT_INPLACE_DIVISOR))

@@ -243,16 +243,19 @@ size_t gpuvm_scratch_bytes(gpuvm_t h);
 #define GPUVM_INPLACE_AUTO 0xFFFFFFFFu
 int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor);
 
-/* How the batched row workloads find the pages that are worth fetching.  counted != 0 (default): a short kernel
- * first counts, per page, the lookups of the whole list (the list is the kernel's input, so the demand is
- * known before the first access); rows of pages below the limit are read in place without the page table being
- * touched, every other page is fetched at its first touch (it is handed to the migrator warps before the first
- * lookup, unless such pages would fill more than half the pool): no row of a page that will be fetched anyway is
- * read in place first.  When every lookup has a staging slot of its own (all bags in flight at once: the default
- * without gpuvm_set_scratch_limit), the lookups of the pages that are not fetched are also bucketed by page and
- * their rows read page by page, at the link's sequential rate.  counted == 0: the online form, which needs no
- * pass over the list: the first `limit` requests that find a page absent read their rows in place (counted in the
- * frame field of the invalid entry), the next one fetches the page. */
+/* How the batched row workloads find the pages that are worth fetching.
+ * counted = 1: a short kernel first counts, per page, the lookups of the whole list (the list is the kernel's
+ * input, so the demand is known before the first access); rows of pages below the limit are read in place
+ * without the page table being touched, as their lookups come up, and every other page is fetched at its first
+ * touch: no row of a page that will be fetched anyway is read in place first.
+ * counted = 2 (default): the same, and when every lookup has a staging slot of its own (all bags in flight at once:
+ * the default without gpuvm_set_scratch_limit) the lookups of the pages that are not fetched are bucketed by page
+ * and their rows read page by page, at the link's sequential rate; the pages that are fetched are handed to the
+ * migrator warps before the first lookup (unless they would fill more than half the pool).  Where that is not
+ * possible it behaves like 1.
+ * counted = 0: the online form, which needs no pass over the list: the first `limit` requests that find a page
+ * absent read their rows in place (counted in the frame field of the invalid entry), the next one fetches the
+ * page.  Other values: GPUVM_E_ARG. */
 int gpuvm_set_inplace_counted(gpuvm_t h, int counted);
 
 /* Largest number of simultaneously resident warps that can each hold

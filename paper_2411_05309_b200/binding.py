@@ -213,8 +213,9 @@ def gpuvm_set_inplace_divisor(h, divisor: int):
     _check(lib().gpuvm_set_inplace_divisor(h, divisor), "gpuvm_set_inplace_divisor")
 
 
-def gpuvm_set_inplace_counted(h, counted: bool):
-    _check(lib().gpuvm_set_inplace_counted(h, int(bool(counted))), "gpuvm_set_inplace_counted")
+def gpuvm_set_inplace_counted(h, counted: int):
+    """0: online; 1: lookups counted per page first; 2 (default): counted, rows in place read page by page."""
+    _check(lib().gpuvm_set_inplace_counted(h, int(counted)), "gpuvm_set_inplace_counted")
 
 
 def gpuvm_set_clean_ahead(h, frames: int):

@@ -24,7 +24,7 @@ struct gpuvm_handle {
     size_t scratch_bytes;
     size_t scratch_limit;      /* 0: none */
     unsigned int inplace_divisor;
-    bool inplace_counted;   // the batched row workloads count the lookups per page first
+    int inplace_counted;    // 0: online; 1: lookups counted per page first; 2: counted, and rows in place read page by page
 };
 
 namespace {
@@ -147,7 +147,7 @@ int gpuvm_create(gpuvm_t *out, void *host_backing, size_t bytes, size_t page_byt
     cudaGetDevice(&h->device);
     h->sms = sm_count_of(h->device);
     h->inplace_divisor = GPUVM_INPLACE_AUTO;
-    h->inplace_counted = true;
+    h->inplace_counted = 2;
     cudaError_t e;
 
     // backing store: pinned and mapped (Section 4: the host region is registered before
@@ -340,7 +340,7 @@ int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes)
 size_t gpuvm_scratch_bytes(gpuvm_t h) { return h ? h->scratch_bytes : 0; }
 
 size_t gpuvm_inplace_divisor_(gpuvm_handle *h) { return h ? h->inplace_divisor : 0; }
-int gpuvm_inplace_counted_(gpuvm_handle *h) { return h && h->inplace_counted; }
+int gpuvm_inplace_counted_(gpuvm_handle *h) { return h ? h->inplace_counted : 0; }
 
 int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor)
 {
@@ -351,8 +351,8 @@ int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor)
 
 int gpuvm_set_inplace_counted(gpuvm_t h, int counted)
 {
-    if (!h) return GPUVM_E_ARG;
-    h->inplace_counted = counted != 0;
+    if (!h || counted < 0 || counted > 2) return GPUVM_E_ARG;
+    h->inplace_counted = counted;
     return GPUVM_OK;
 }
 

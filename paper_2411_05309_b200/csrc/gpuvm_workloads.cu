@@ -2223,11 +2223,11 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     // balance (divisor 4).  A row is a whole number of 128-byte link reads when it is a multiple of 128 bytes
     // long; shorter rows are charged 128 bytes.
     const size_t n_lookups = n_bags * bag;
-    const bool counted = gpuvm_inplace_counted_(h) != 0;
+    const bool counted = gpuvm_inplace_counted_(h) != 0, want_grouped = gpuvm_inplace_counted_(h) == 2;
     const size_t demand_bytes = (m.vm.n_pages * sizeof(unsigned int) + 255) & ~size_t(255);
     const size_t index_bytes = (n_lookups * sizeof(unsigned int) + 255) & ~size_t(255);
     const size_t base_bytes = table_bytes + staging_bytes + sizeof(gpuvm_shared_queue) + demand_bytes;
-    const bool grouped = counted && one_pass && n_lookups < 0xFFFFFFFFull && m.vm.n_pages <= (1ull << 20) &&
+    const bool grouped = want_grouped && one_pass && n_lookups < 0xFFFFFFFFull && m.vm.n_pages <= (1ull << 20) &&
                          (gpuvm_scratch_limit_(h) == ~size_t(0) || base_bytes + demand_bytes + index_bytes + 256 <= gpuvm_scratch_limit_(h));
     size_t divisor = gpuvm_inplace_divisor_(h);
     if (divisor == GPUVM_INPLACE_AUTO) divisor = grouped ? 1 : 4;

@@ -28,9 +28,9 @@ def _row(cfg: str, r: dict) -> str:
     frac = f"{roof['frac']:.3f}"
     if "frac_compulsory" in roof:
         frac += f" by faults, {roof['frac_compulsory']:.3f} of the compulsory floor"
-    if roof.get("in_place", {}).get("frac"):
-        frac += (f"; rows in place at {roof['in_place']['frac']:.2f} of the {roof['in_place']['scattered_read_peak_gbs']:.1f} GB/s "
-                 "scattered reads reach")
+    if roof.get("in_place"):
+        frac += (f" (rows in place page by page; scattered reads over this table reach "
+                 f"{roof['in_place']['scattered_read_peak_gbs']:.1f} GB/s)")
     cpu = r.get("cpu_baseline")
     cpu_s = "-"
     if cpu:
@@ -53,7 +53,9 @@ def policies(line: dict) -> str:
     recs = line.get("per_config") or {str(line["config"]["cfg"]): line}
     roof = recs.get("5", {}).get("roofline", {})
     out = []
-    for key, name in (("online", "online rent-or-buy (no count beforehand)"), ("always_migrate", "the paper's policy (every first touch fetches)")):
+    for key, name in (("counted_scattered", "the counted policy with rows read as their lookups come up"),
+                      ("online", "the online policy (no count beforehand)"),
+                      ("always_migrate", "the paper's policy (every first touch fetches)")):
         r = roof.get(key)
         if r:
             out.append(f"cfg 5 under {name}: {r['ms_per_step']:.1f} ms, {r['value']:.2f} GB/s, {r['faults']} faults, "

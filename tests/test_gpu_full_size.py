@@ -171,14 +171,14 @@ def test_cfg5_zipf_embedding_bag_64GiB():
         B = __import__("paper_2411_05309_b200.binding", fromlist=["x"])
         # the online form (no count beforehand): a page is fetched after 1024 of its rows (a quarter) have been read in place
         limit = (2 << 20) // 4 // 512
-        B.gpuvm_set_inplace_counted(w.h, False)
+        B.gpuvm_set_inplace_counted(w.h, 0)
         res1 = w.run()
         st1 = res1.stats
         assert np.count_nonzero(per_page > limit + 4096) <= st1["faults"] <= np.count_nonzero(per_page > limit) + 1
         in_place = st1["bytes_direct"] // 512
         assert int(per_page[per_page <= limit].sum()) <= in_place <= int(np.minimum(per_page, limit + 4096).sum())
         assert np.array_equal(w.d_out.cpu().numpy().reshape(w.n_bags, w.dims)[:4096].view(np.uint32), out[:4096].view(np.uint32))
-        B.gpuvm_set_inplace_counted(w.h, True)
+        B.gpuvm_set_inplace_counted(w.h, 2)
         # the paper's way (every first touch fetches the page): never fewer than one fault per page touched
         B.gpuvm_set_inplace_divisor(w.h, 0)
         res0 = w.run()

@@ -391,13 +391,13 @@ def test_embag(B, page, n_rows, n_bags, frames, dims, bag, batched):
         assert st["bytes_direct"] == 0 and st["faults"] >= touched
 
 
-@pytest.mark.parametrize("counted", [True, False])
+@pytest.mark.parametrize("counted", [2, 1, 0])
 @pytest.mark.parametrize("frames", [1, 4, 64])
 def test_embag_rent_or_buy(B, frames, counted):
     """The batched embedding bag does not fetch a page for a few rows.  Counted (default): the lookups per page are
-    counted first; rows of pages below the limit (page / divisor / row size; the divisor is 1 unless set otherwise,
-    because here the rows in place are read page by page) are read in place, all of them, and the other pages are
-    fetched once.  Online: the
+    counted first; rows of pages below the limit (page / divisor / row size) are read in place, all of them, and the
+    other pages are fetched once.  With counted = 2 (the default) the rows in place are read page by page and the
+    divisor is 1 unless set otherwise; with counted = 1 they are read as their lookups come up and it is 4.  Online: the
     first `limit` requests that find a page absent read their rows in place, the next one fetches it.  Divisor 0:
     every first touch fetches, as in the paper.  Results are exact either way."""
     import torch
@@ -417,7 +417,7 @@ def test_embag_rent_or_buy(B, frames, counted):
             with paged(ar.host, page, frames) as h:
                 B.gpuvm_set_inplace_counted(h, counted)
                 if divisor is None:
-                    divisor = 1 if counted else 4                              # the default: 1 when the rows in place are read page by page
+                    divisor = 1 if counted == 2 else 4                         # the default: 1 when the rows in place are read page by page
                 else:
                     B.gpuvm_set_inplace_divisor(h, divisor)
                 B.gpuvm_embag_f32(h, 0, dims, dev(rows), n_bags, bag, out)
