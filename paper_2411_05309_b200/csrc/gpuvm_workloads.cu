@@ -1257,7 +1257,8 @@ __global__ void embag_demand_kernel(const long long *__restrict__ rows, unsigned
 // fetched ("cold": fewer lookups than the limit) are bucketed by page first: bucket_off[p] becomes the start of page
 // p's bucket (an exclusive scan of the cold pages' counts; one block, 1024 pages per step), the fill kernel puts
 // every cold lookup's number into its page's bucket, and the main kernel reads the rows in bucket order.
-// counts[0] = number of cold lookups, counts[1] = number of pages that will be fetched.
+// counts[0] = number of cold lookups, counts[1] = number of pages that will be fetched, counts[2] = cold lookups
+// whose rows have been staged (counted up by the main kernel).
 __global__ void __launch_bounds__(1024) embag_bucket_scan_kernel(const unsigned int *__restrict__ demand, unsigned int n_pages,
                                                                   unsigned int limit, unsigned int *__restrict__ bucket_off,
                                                                   unsigned int *__restrict__ counts)
@@ -1292,7 +1293,7 @@ __global__ void __launch_bounds__(1024) embag_bucket_scan_kernel(const unsigned 
     for (int o = 16; o; o >>= 1) hot += __shfl_down_sync(0xFFFFFFFFu, hot, o);
     if (lane == 0 && hot) atomicAdd(&hot_s, hot);
     __syncthreads();
-    if (threadIdx.x == 0) { counts[0] = carry_s; counts[1] = hot_s; }
+    if (threadIdx.x == 0) { counts[0] = carry_s; counts[1] = hot_s; counts[2] = 0; }
 }
 
 // After this kernel bucket_off[p] is the END of page p's bucket (every cold lookup moved it on by one).
@@ -1319,28 +1320,6 @@ __device__ __forceinline__ size_t embag_staged_row(unsigned long long i, unsigne
     const unsigned long long t = g / per_item;
     const unsigned int rr = (unsigned int)(g - t * per_item), gi = rr >> 5, b = rr & 31u;
     return (size_t)t * ((size_t)groups * 32 * bag) + (size_t)((gi * bag + k) * 32 + b);
-}
-
-// The bags' sums as a kernel of their own (grouped mode: the rows of a bag are staged by many warps, so the sums
-// wait for the whole main kernel): one warp per bag, the rows added in list order.
-__global__ void embag_sum_kernel(const unsigned char *__restrict__ g_staging, unsigned int dims, unsigned long long n_bags,
-                                 unsigned int bag, unsigned int groups, float *__restrict__ out)
-{
-    const unsigned int lane = threadIdx.x & 31, q = dims >> 2;
-    const uint4 *staging = reinterpret_cast<const uint4 *>(g_staging);
-    for (unsigned long long g = warp_in_grid(); g < n_bags; g += warps_in_grid()) {
-        if (lane >= q) continue;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 8
-        for (unsigned int k = 0; k < bag; ++k) {
-            const uint4 v = staging[embag_staged_row(g * bag + k, bag, groups) * q + lane];
-            acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
-            acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
-            acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
-            acc.w = __fadd_rn(acc.w, __uint_as_float(v.w));
-        }
-        reinterpret_cast<float4 *>(out + g * dims)[lane] = acc;
-    }
 }
 
 __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
@@ -1426,6 +1405,10 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
             n_here += cnt;
         }
         if (lane == 0 && n_here) gpuvm::stat_add(vm, gpuvm::kBytesDirect, (unsigned long long)n_here * row_bytes);
+        // the rows are in their slots for everybody before they are counted as staged
+        __threadfence();
+        __syncwarp();
+        if (lane == 0 && n_here) atomicAdd(const_cast<unsigned int *>(cold_counts) + 2, n_here);
     }
     for (unsigned long long t = slot; t < items; t += stride) {
         const unsigned long long g0 = per_item * t;
@@ -1453,7 +1436,27 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                                   queue, masks, 1u, one_pass, grouped ? 0u : inplace_limit, (unsigned int)row_bytes,
                                   grouped ? nullptr : demand);
             __syncwarp();
-            if (grouped) continue;                               // the sums follow in embag_sum_kernel
+            if (grouped) {
+                // The rows of this warp's bags that were read in place were staged by whichever warps had their
+                // bucket entries: wait (bounded) until all of them are counted as staged.  Every warp stages its
+                // share before it comes here, so the wait is for the stragglers of the grid only.  (The shares
+                // are fixed, not drawn from a counter: warps get through theirs at different speeds, 20 to 40 ms,
+                // and the early ones run the engine and add up their bags while the others keep the link busy;
+                // with a counter all warps finish reading together and all that work comes after it, 5 ms later.)
+                const unsigned int n_cold = cold_counts[0];
+                const unsigned long long limit_ns = (unsigned long long)vm.spin_limit_us * 1000ull;
+                unsigned long long t0 = 0;
+                bool ok = true;
+                while (ld_volatile_u32(cold_counts + 2) < n_cold) {
+                    const unsigned long long now = gpuvm::now_ns();
+                    if (t0 == 0) t0 = now;
+                    if (now - t0 > limit_ns || gpuvm::has_error(vm)) { ok = false; break; }
+                    __nanosleep(256);
+                }
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) { if (lane == 0) gpuvm::set_error(vm, GPUVM_E_TIMEOUT, ~0ull); continue; }
+                __threadfence();
+            }
             // add the staged rows of each bag in list order
             for (unsigned int gb = 0; gb < 32 * groups && g0 + gb < n_bags; ++gb) {
                 if (lane < q) {
@@ -1462,7 +1465,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                     float4 acc = k0 == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *dst;
 #pragma unroll 8
                     for (unsigned int k = 0; k < nk; ++k) {
-                        const uint4 v = staging[(size_t)((gi * nk + k) * 32 + b) * q + lane];
+                        const uint4 v = __ldcg(staging + (size_t)((gi * nk + k) * 32 + b) * q + lane);   // some were staged by other warps
                         acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
                         acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
                         acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
@@ -2269,10 +2272,6 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
         m.vm, t_off, (unsigned int)dims, rows_ll, n_bags, (unsigned int)bag, d_out,
         requesters, reinterpret_cast<gpuvm_batch_entry *>(scratch), scratch + table_bytes, groups, one_pass, shared_queue,
         inplace_limit, demand, cold_idx, cold_counts);
-    if (use_grouped) {
-        embag_sum_kernel<<<sm_count() * 8, 256, 0, s>>>(scratch + table_bytes, (unsigned int)dims, n_bags, (unsigned int)bag, groups, d_out);
-        ++launches;
-    }
     return launched(launches);
 }
 
