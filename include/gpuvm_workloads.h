@@ -225,7 +225,9 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
  * Embedding-bag gather: d_out[g][d] = sum over the `bag` rows of bag g of
  * table[row][d], added in list order in fp32.  table: fp32 [rows][dims] at t_off,
  * dims a multiple of 4 with dims/4 <= 32 lanes (a lane owns 4 consecutive dims);
- * d_rows: n_bags * bag int64 row ids; d_out: n_bags * dims fp32.
+ * d_rows: n_bags * bag int64 row ids; d_out: n_bags * dims fp32 (device memory, or pinned mapped host memory:
+ * the sums are then written straight to the host; measured, that saves the copy afterwards and costs the kernel
+ * as much).
  *
  * gpuvm_embag_f32: a requester warp registers the rows of 32 to 256 bags (up to 32 lookups
  * each) at once (gpuvm_batch.cuh); rows that arrive are staged in device scratch and added

@@ -438,6 +438,24 @@ def test_embag_rent_or_buy(B, frames, counted):
                 assert limit * 512 <= st["bytes_direct"] <= (limit + 31) * 512 * st["faults"]
 
 
+def test_embag_writes_its_sums_to_pinned_host_memory(B):
+    """d_out may be pinned host memory: the kernel writes the bags' sums there itself, same bits."""
+    import torch
+    page, dims, bag, n_rows, n_bags = 4096, 128, 8, 2048, 300
+    t = inputs.fill_f32_pm1(np.empty(n_rows * dims, np.float32), n_rows * dims, inputs.config_seed(5))
+    rows = inputs.fill_zipf_rows(np.empty(n_bags * bag, np.int64), n_bags * bag, inputs.config_seed(5, 1), n_rows, 1.05)
+    ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
+    ar = Arena(page, {"t": t})
+    for counted in (2, 1, 0):
+        out = torch.zeros(n_bags * dims, dtype=torch.float32).pin_memory()
+        with paged(ar.host, page, 16) as h:
+            B.gpuvm_set_inplace_counted(h, counted)
+            B.gpuvm_embag_f32(h, 0, dims, dev(rows), n_bags, bag, out)
+            finish(h)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.numpy().view(np.uint32), ref.view(np.uint32)), counted
+
+
 def test_embag_rows_past_the_end_and_tables_off_the_row_grid(B):
     """A row id whose row does not lie inside the backing store sets the sticky range error (batched
     and unbatched); a table that starts off the row grid of its page is still summed correctly."""
