@@ -1322,6 +1322,30 @@ __device__ __forceinline__ size_t embag_staged_row(unsigned long long i, unsigne
     return (size_t)t * ((size_t)groups * 32 * bag) + (size_t)((gi * bag + k) * 32 + b);
 }
 
+// All 32 lanes: add the staged rows of the warp's bags g0 .. g0 + 32 groups - 1 in list order (lookups k of this
+// batch, nk of them; `first`: the batch starts the bag, otherwise it adds to what is in out).
+__device__ __forceinline__ void embag_add_bags(const uint4 *staging, float *__restrict__ out, unsigned int dims, unsigned int q,
+                                               unsigned long long g0, unsigned long long n_bags, unsigned int groups,
+                                               unsigned int nk, bool first, unsigned int lane)
+{
+    for (unsigned int gb = 0; gb < 32 * groups && g0 + gb < n_bags; ++gb) {
+        if (lane < q) {
+            const unsigned int gi = gb >> 5, b = gb & 31;
+            float4 *dst = reinterpret_cast<float4 *>(out + (g0 + gb) * dims) + lane;
+            float4 acc = first ? make_float4(0.f, 0.f, 0.f, 0.f) : *dst;
+#pragma unroll 8
+            for (unsigned int k = 0; k < nk; ++k) {
+                const uint4 v = __ldcg(staging + (size_t)((gi * nk + k) * 32 + b) * q + lane);   // some may have been staged by other warps
+                acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
+                acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
+                acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
+                acc.w = __fadd_rn(acc.w, __uint_as_float(v.w));
+            }
+            *dst = acc;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
                                                               const long long *__restrict__ rows, unsigned long long n_bags,
                                                               unsigned int bag, float *__restrict__ out, int requesters,
@@ -1381,34 +1405,86 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
         }
         // (2) The rows of the other pages, in bucket order (page by page), four in flight per warp; the warps of
         // the grid take neighbouring entries, so at any moment the reads in flight fall into a few hundred pages.
+        // A warp reads its whole share first and then runs the engine over its lookups of the fetched pages, which
+        // have arrived by then (running the engine after 30, 50 or 70 % of the share was measured: 52 / 49 / 49 ms
+        // against 44-45).
         unsigned int n_here = 0;
         constexpr int Q = 4;
         uint4 *const all_staging = reinterpret_cast<uint4 *>(g_staging);
-        for (unsigned long long j0 = slot * Q; j0 < n_cold; j0 += stride * Q) {
-            uint4 v[Q];
-            size_t where[Q];
-            int cnt = 0;
+        auto read_in_place = [&](unsigned long long j_begin, unsigned long long j_end) {
+            for (unsigned long long j0 = j_begin + slot * Q; j0 < j_end; j0 += stride * Q) {
+                uint4 v[Q];
+                size_t where[Q];
+                int cnt = 0;
 #pragma unroll
-            for (int u = 0; u < Q; ++u) {
-                where[u] = 0;
-                if (j0 + u < n_cold) {
-                    const unsigned int i = cold_idx[j0 + u];
-                    const unsigned long long r = (unsigned long long)rows[i];
-                    where[u] = embag_staged_row(i, bag, groups) * q;
-                    if (lane < q) v[u] = gpuvm_load16(vm.host + t_off + r * row_bytes + 16u * lane);
-                    cnt = u + 1;
+                for (int u = 0; u < Q; ++u) {
+                    where[u] = 0;
+                    if (j0 + u < j_end) {
+                        const unsigned int i = cold_idx[j0 + u];
+                        const unsigned long long r = (unsigned long long)rows[i];
+                        where[u] = embag_staged_row(i, bag, groups) * q;
+                        if (lane < q) v[u] = gpuvm_load16(vm.host + t_off + r * row_bytes + 16u * lane);
+                        cnt = u + 1;
+                    }
                 }
-            }
 #pragma unroll
-            for (int u = 0; u < Q; ++u)
-                if (u < cnt && lane < q) all_staging[where[u] + lane] = v[u];
-            n_here += cnt;
+                for (int u = 0; u < Q; ++u)
+                    if (u < cnt && lane < q) all_staging[where[u] + lane] = v[u];
+                n_here += cnt;
+            }
+        };
+        read_in_place(0, n_cold);
+        const unsigned long long t = slot, g0 = per_item * t;
+        const unsigned int nk = bag;                             // one pass: bag <= kEmbagLookups, one item per warp
+        if (t < items) {
+            for (unsigned int gi = 0; gi < groups; ++gi)
+                for (unsigned int k = 0; k < nk; ++k) {
+                    const unsigned long long g = g0 + 32ull * gi + lane;
+                    const unsigned int at = (gi * nk + k) * 32 + lane;
+                    if (g < n_bags) {
+                        const unsigned long long r = (unsigned long long)rows[g * bag + k];
+                        const bool inside = r < rows_inside;
+                        if (inside && demand[(t_off + r * row_bytes) >> vm.page_shift] < inplace_limit)
+                            gpuvm_batch_skip(table, at);                     // its row is staged by read_in_place
+                        else
+                            gpuvm_batch_set(vm, table, at, inside ? t_off + r * row_bytes : ~0ull);
+                    } else
+                        gpuvm_batch_skip(table, at);
+                }
+            __syncwarp();
+            gpuvm_batch_run<true>(vm, gpuvm_entry_table{table}, groups * nk * 32, GPUVM_READ, gpuvm_row_copy{staging, q},
+                                  queue, masks, 1u, true, 0u, (unsigned int)row_bytes, nullptr);
+            __syncwarp();
         }
         if (lane == 0 && n_here) gpuvm::stat_add(vm, gpuvm::kBytesDirect, (unsigned long long)n_here * row_bytes);
         // the rows are in their slots for everybody before they are counted as staged
         __threadfence();
         __syncwarp();
         if (lane == 0 && n_here) atomicAdd(const_cast<unsigned int *>(cold_counts) + 2, n_here);
+        // A bag's rows that were read in place were staged by whichever warps had their bucket entries: wait
+        // (bounded) until all of them are counted as staged.  Every warp stages its share before it comes here,
+        // so the wait is for the stragglers of the grid only.  (The shares are fixed, not drawn from a counter:
+        // warps get through theirs at different speeds, and the early ones add up their bags while the others
+        // keep the link busy; with a counter all warps finished reading together and all that came after it.)
+        if (t < items) {
+            const unsigned long long limit_ns = (unsigned long long)vm.spin_limit_us * 1000ull;
+            unsigned long long t0 = 0;
+            bool ok = true;
+            while (ld_volatile_u32(cold_counts + 2) < n_cold) {
+                const unsigned long long now = gpuvm::now_ns();
+                if (t0 == 0) t0 = now;
+                if (now - t0 > limit_ns || gpuvm::has_error(vm)) { ok = false; break; }
+                __nanosleep(256);
+            }
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) { if (lane == 0) gpuvm::set_error(vm, GPUVM_E_TIMEOUT, ~0ull); }
+            else {
+                __threadfence();
+                embag_add_bags(staging, out, dims, q, g0, n_bags, groups, nk, /* first = */ true, lane);
+            }
+        }
+        if (lane == 0) gpuvm_requester_done(queue);
+        return;
     }
     for (unsigned long long t = slot; t < items; t += stride) {
         const unsigned long long g0 = per_item * t;
@@ -1422,10 +1498,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                         // a row that ends past the backing store is refused like one that starts there
                         const unsigned long long r = (unsigned long long)rows[g * bag + k0 + k];
                         const bool inside = r < rows_inside;
-                        if (grouped && inside && demand[(t_off + r * row_bytes) >> vm.page_shift] < inplace_limit)
-                            gpuvm_batch_skip(table, (gi * nk + k) * 32 + lane);          // its row is staged by step (2)
-                        else
-                            gpuvm_batch_set(vm, table, (gi * nk + k) * 32 + lane, inside ? t_off + r * row_bytes : ~0ull);
+                        gpuvm_batch_set(vm, table, (gi * nk + k) * 32 + lane, inside ? t_off + r * row_bytes : ~0ull);
                     } else
                         gpuvm_batch_skip(table, (gi * nk + k) * 32 + lane);
                 }
@@ -1433,47 +1506,9 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
             // every served row is copied to its slot of the staging area by the whole warp (the engine does it
             // itself, four rows in flight: gpuvm_row_copy), from its frame or in place from the backing store
             gpuvm_batch_run<true>(vm, gpuvm_entry_table{table}, groups * nk * 32, GPUVM_READ, gpuvm_row_copy{staging, q},
-                                  queue, masks, 1u, one_pass, grouped ? 0u : inplace_limit, (unsigned int)row_bytes,
-                                  grouped ? nullptr : demand);
+                                  queue, masks, 1u, one_pass, inplace_limit, (unsigned int)row_bytes, demand);
             __syncwarp();
-            if (grouped) {
-                // The rows of this warp's bags that were read in place were staged by whichever warps had their
-                // bucket entries: wait (bounded) until all of them are counted as staged.  Every warp stages its
-                // share before it comes here, so the wait is for the stragglers of the grid only.  (The shares
-                // are fixed, not drawn from a counter: warps get through theirs at different speeds, 20 to 40 ms,
-                // and the early ones run the engine and add up their bags while the others keep the link busy;
-                // with a counter all warps finish reading together and all that work comes after it, 5 ms later.)
-                const unsigned int n_cold = cold_counts[0];
-                const unsigned long long limit_ns = (unsigned long long)vm.spin_limit_us * 1000ull;
-                unsigned long long t0 = 0;
-                bool ok = true;
-                while (ld_volatile_u32(cold_counts + 2) < n_cold) {
-                    const unsigned long long now = gpuvm::now_ns();
-                    if (t0 == 0) t0 = now;
-                    if (now - t0 > limit_ns || gpuvm::has_error(vm)) { ok = false; break; }
-                    __nanosleep(256);
-                }
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) { if (lane == 0) gpuvm::set_error(vm, GPUVM_E_TIMEOUT, ~0ull); continue; }
-                __threadfence();
-            }
-            // add the staged rows of each bag in list order
-            for (unsigned int gb = 0; gb < 32 * groups && g0 + gb < n_bags; ++gb) {
-                if (lane < q) {
-                    const unsigned int gi = gb >> 5, b = gb & 31;
-                    float4 *dst = reinterpret_cast<float4 *>(out + (g0 + gb) * dims) + lane;
-                    float4 acc = k0 == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *dst;
-#pragma unroll 8
-                    for (unsigned int k = 0; k < nk; ++k) {
-                        const uint4 v = __ldcg(staging + (size_t)((gi * nk + k) * 32 + b) * q + lane);   // some were staged by other warps
-                        acc.x = __fadd_rn(acc.x, __uint_as_float(v.x));
-                        acc.y = __fadd_rn(acc.y, __uint_as_float(v.y));
-                        acc.z = __fadd_rn(acc.z, __uint_as_float(v.z));
-                        acc.w = __fadd_rn(acc.w, __uint_as_float(v.w));
-                    }
-                    *dst = acc;
-                }
-            }
+            embag_add_bags(staging, out, dims, q, g0, n_bags, groups, nk, k0 == 0, lane);
             __syncwarp();
         }
     }
