@@ -114,3 +114,52 @@ def test_many_small_vector_adds_and_graphs(B):
             finish(h)
         assert np.array_equal(lvl.cpu().numpy(), oracle.bfs_levels_direct(off, col, src)), (case, scale, page, frames)
         assert np.array_equal(lab.cpu().numpy(), oracle.cc_labels_direct(off, col)), (case, scale, page, frames)
+
+
+def test_random_embedding_bags_under_every_page_policy(B):
+    """Embedding bags of random shape (row size, bag length, table size, skew) over pools from one frame to the
+    whole table, under the three forms of the in-place policy with random divisors (0 = every first touch
+    fetches), with and without a scratch bound (a bound takes the staging slots away from the lookups, so rows in
+    place are read as their lookups come up), every other case with frames poisoned on eviction.  The sums must
+    have the oracle's bits, the invariants must hold, and what the counters say must add up: every lookup's row
+    came from a fetched page or was read in place."""
+    import torch
+    rng = np.random.default_rng(20241106)
+    for case in range(48 * SOAK):
+        page = int(rng.choice([512, 4096, 65536]))
+        dims = int(rng.choice([4, 16, 32, 128]))
+        row_bytes = 4 * dims
+        if row_bytes > page:
+            continue
+        n_rows = int(rng.integers(1, 40)) * (page // row_bytes) + int(rng.integers(0, 3))
+        bag = int(rng.choice([1, 3, 8, 32, 40]))
+        n_bags = int(rng.integers(1, 400))
+        n_pages = (n_rows * row_bytes + page - 1) // page
+        frames = int(rng.choice([1, 2, max(1, n_pages // 4), n_pages, n_pages + 2]))
+        t = inputs.fill_f32_pm1(np.empty(n_rows * dims, np.float32), n_rows * dims, 3000 + case)
+        if rng.integers(0, 2):
+            rows = inputs.fill_zipf_rows(np.empty(n_bags * bag, np.int64), n_bags * bag, 4000 + case, n_rows, 1.05)
+        else:
+            rows = rng.integers(0, n_rows, n_bags * bag).astype(np.int64)
+        ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
+        ar = Arena(page, {"t": t})
+        out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
+        counted = int(rng.integers(0, 3))
+        divisor = int(rng.choice([0, 1, 2, 4, 16, B.INPLACE_AUTO]))
+        bound = int(rng.choice([0, 0, 1 << 16, 1 << 20]))
+        with paged(ar.host, page, frames, int(rng.integers(0, 2))) as h:
+            if case & 1:
+                B.gpuvm_set_debug(h, B.DEBUG_POISON)
+            B.gpuvm_set_inplace_counted(h, counted)
+            B.gpuvm_set_inplace_divisor(h, divisor)
+            if bound:
+                B.gpuvm_set_scratch_limit(h, bound)
+            for _ in range(2):                                          # the second call finds pages resident
+                out.zero_()
+                B.gpuvm_embag_f32(h, 0, dims, dev(rows), n_bags, bag, out)
+                st, ck = finish(h)
+                what = (case, page, dims, n_rows, bag, n_bags, frames, counted, divisor, bound)
+                assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32)), what
+                assert st["bytes_direct"] % row_bytes == 0, what
+                if divisor == 0:
+                    assert st["bytes_direct"] == 0, what
