@@ -426,13 +426,16 @@ def embag_policy_records(torch, B, w, args, link: dict, kern_s: float, direct: f
     row_bytes = 4 * w.dims
     buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     scattered = B.gpuvm_link_peak_scattered(B.gpuvm_host_ptr(w.h), w.nbytes, row_bytes, 1 << 22, buf.data_ptr(), buf.numel())
+    grouped = B.gpuvm_link_peak_scattered(B.gpuvm_host_ptr(w.h), w.nbytes, row_bytes, 1 << 22, buf.data_ptr(), buf.numel(), 2, 64)
     del buf
     out["in_place"] = {
         "bytes": direct, "gbs": direct / kern_s / 1e9 if kern_s else 0.0, "scattered_read_peak_gbs": scattered,
+        "grouped_read_peak_gbs": grouped,
         "what": f"rows read in place from the backing store, page by page (bucketed by page first); "
                 f"scattered_read_peak_gbs is what {1 << 22} rows of {row_bytes} B at hashed positions of the same "
                 f"{w.nbytes >> 30} GiB region reach, four in flight per warp, measured in this run: the ceiling of "
-                f"reading them as their lookups come up (roofline.counted_scattered)"}
+                f"reading them as their lookups come up (roofline.counted_scattered); grouped_read_peak_gbs is the same "
+                f"with 64 consecutive rows in the same 2 MiB of the region"}
     if args.inplace_divisor < 0 and not args.scratch_limit_mib:
         def other_policy(what, setup, restore):
             setup()

@@ -312,12 +312,15 @@ int gpuvm_link_peak(void *host_ptr, void *d_buf, size_t bytes, int reps, double 
  * The same link read as scattered rows: n_rows rows of row_bytes (a multiple of 16, at most 512) at hashed
  * positions of the pinned region [host_ptr, host_ptr + host_bytes) are loaded by warps, four rows in flight
  * each, and stored to the device buffer d_buf of d_bytes (reused round-robin).  out[0] = GB/s, best of `reps`.
- * This is the ceiling of rows read in place from the backing store; it falls with the size of the region
- * (measured on one host: 51.4 GB/s over 1 GiB, 33.4 over 8 GiB, 24.5 over 64 GiB, whatever the number of reads
- * in flight).  out: host pointer to 1 double.  Synchronises.
+ * run = 1: every row at a position of its own: the ceiling of rows read in place as their lookups come up; it
+ * falls with the size of the region (measured on one host: 51.4 GB/s over 1 GiB, 33.4 over 8 GiB, 24.5 over
+ * 64 GiB, whatever the number of reads in flight).  run > 1: `run` consecutive rows fall into the same 2 MiB
+ * of the region (a hashed 2 MiB block, hashed rows inside it): the pattern of rows bucketed by page, which the
+ * same host serves at the sequential rate from a few dozen rows per block on.
+ * out: host pointer to 1 double.  Synchronises.
  */
-int gpuvm_link_peak_scattered(void *host_ptr, size_t host_bytes, size_t row_bytes, size_t n_rows, void *d_buf,
-                              size_t d_bytes, int reps, double *out);
+int gpuvm_link_peak_scattered(void *host_ptr, size_t host_bytes, size_t row_bytes, size_t n_rows, size_t run,
+                              void *d_buf, size_t d_bytes, int reps, double *out);
 
 /* Number of kernels this library has launched in the calling process. */
 unsigned long long gpuvm_launch_count(void);

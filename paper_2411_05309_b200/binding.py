@@ -107,7 +107,7 @@ SYMBOLS = {
     "gpuvm_raw_vadd_f32": (_i, [_vp, _vp, _vp, _sz, _vp]),
     "gpuvm_raw_embag_f32": (_i, [_vp, _sz, _vp, _sz, _sz, _vp, _vp]),
     "gpuvm_link_peak": (_i, [_vp, _vp, _sz, _i, ctypes.POINTER(ctypes.c_double)]),
-    "gpuvm_link_peak_scattered": (_i, [_vp, _sz, _sz, _sz, _vp, _sz, _i, ctypes.POINTER(ctypes.c_double)]),
+    "gpuvm_link_peak_scattered": (_i, [_vp, _sz, _sz, _sz, _sz, _vp, _sz, _i, ctypes.POINTER(ctypes.c_double)]),
     "gpuvm_launch_count": (ctypes.c_ulonglong, []),
     "gpuvm_uvm_alloc": (_i, [ctypes.POINTER(_vp), _sz]),
     "gpuvm_uvm_free": (_i, [_vp]),
@@ -455,9 +455,10 @@ def gpuvm_link_peak(host_ptr, d_buf, nbytes: int, reps: int = 3):
     return {"h2d_gbs": out[0], "d2h_gbs": out[1], "duplex_gbs": out[2]}
 
 
-def gpuvm_link_peak_scattered(host_ptr, host_bytes: int, row_bytes: int, n_rows: int, d_buf, d_bytes: int, reps: int = 2) -> float:
+def gpuvm_link_peak_scattered(host_ptr, host_bytes: int, row_bytes: int, n_rows: int, d_buf, d_bytes: int, reps: int = 2,
+                              run: int = 1) -> float:
     out = (ctypes.c_double * 1)()
-    _check(lib().gpuvm_link_peak_scattered(_ptr(host_ptr), host_bytes, row_bytes, n_rows, _ptr(d_buf), d_bytes, reps, out),
+    _check(lib().gpuvm_link_peak_scattered(_ptr(host_ptr), host_bytes, row_bytes, n_rows, run, _ptr(d_buf), d_bytes, reps, out),
            "gpuvm_link_peak_scattered")
     return out[0]
 

@@ -1622,26 +1622,36 @@ __global__ void link_in_kernel(const uint4 *__restrict__ src, uint4 *__restrict_
     }
 }
 
-// Scattered rows over the link: row i of the launch is row hash(seed, i) of the host region; a warp has four
-// rows in flight (16 bytes per lane and row).  What a workload that reads rows in place can reach at most.
+// Scattered rows over the link: row i of the launch is a hashed row of the host region; a warp has four rows in
+// flight (16 bytes per lane and row).  What a workload that reads rows in place can reach at most.  With
+// run > 1, `run` consecutive rows of the launch fall into the same 2 MiB of the region (a hashed 2 MiB block, hashed
+// rows inside it): the access pattern of rows that have been bucketed by page.
+__device__ __forceinline__ unsigned long long splitmix64(unsigned long long z)
+{
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
 __global__ void link_scattered_kernel(const unsigned char *__restrict__ host, unsigned long long host_rows, unsigned int units16,
-                                      unsigned long long n_rows, unsigned long long seed, uint4 *__restrict__ dst,
+                                      unsigned long long n_rows, unsigned long long seed, unsigned int run, uint4 *__restrict__ dst,
                                       unsigned long long dst_rows)
 {
     const unsigned int lane = threadIdx.x & 31;
     const unsigned long long warp = (blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x) >> 5;
     const unsigned long long warps = ((unsigned long long)gridDim.x * blockDim.x) >> 5;
     const unsigned long long row_bytes = 16ull * units16;
+    const unsigned long long block_rows = (2ull << 20) / row_bytes, blocks = host_rows / block_rows;
     for (unsigned long long i = warp * 4; i < n_rows; i += warps * 4) {
         uint4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            unsigned long long z = seed + (i + u) * 0x9E3779B97F4A7C15ull;       // splitmix64 of the row's index
-            z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
-            z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-            z ^= z >> 31;
+            unsigned long long r = splitmix64(seed + (i + u) * 0x9E3779B97F4A7C15ull) % host_rows;
+            if (run > 1 && blocks > 0)
+                r = (splitmix64(seed ^ ((i + u) / run)) % blocks) * block_rows + splitmix64(seed + i + u) % block_rows;
             if (i + u < n_rows && lane < units16)
-                v[u] = gpuvm::ld_host16(reinterpret_cast<const uint4 *>(host + (z % host_rows) * row_bytes) + lane);
+                v[u] = gpuvm::ld_host16(reinterpret_cast<const uint4 *>(host + r * row_bytes) + lane);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u)
@@ -2490,11 +2500,11 @@ int gpuvm_link_peak(void *host_ptr, void *d_buf, size_t bytes, int reps, double 
     return GPUVM_OK;
 }
 
-int gpuvm_link_peak_scattered(void *host_ptr, size_t host_bytes, size_t row_bytes, size_t n_rows, void *d_buf, size_t d_bytes,
-                              int reps, double *out)
+int gpuvm_link_peak_scattered(void *host_ptr, size_t host_bytes, size_t row_bytes, size_t n_rows, size_t run, void *d_buf,
+                              size_t d_bytes, int reps, double *out)
 {
     if (!host_ptr || !d_buf || !out || row_bytes < 16 || row_bytes % 16 || row_bytes > 512 || host_bytes < row_bytes ||
-        d_bytes < row_bytes || n_rows == 0 || reps <= 0)
+        d_bytes < row_bytes || n_rows == 0 || reps <= 0 || run == 0 || run > 0xFFFFFFFFull)
         return GPUVM_E_ARG;
     void *dh = nullptr;
     if (cudaHostGetDevicePointer(&dh, host_ptr, 0) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_PIN; }
@@ -2505,7 +2515,7 @@ int gpuvm_link_peak_scattered(void *host_ptr, size_t host_bytes, size_t row_byte
     for (int r = 0; r <= reps; ++r) {
         cudaEventRecord(a);
         link_scattered_kernel<<<sm_count(), 1024>>>(static_cast<const unsigned char *>(dh), host_bytes / row_bytes,
-                                                    (unsigned int)(row_bytes / 16), n_rows, 0x5CA77E2ull + r,
+                                                    (unsigned int)(row_bytes / 16), n_rows, 0x5CA77E2ull + r, (unsigned int)run,
                                                     static_cast<uint4 *>(d_buf), d_bytes / row_bytes);
         gpuvm_note_launch_(1);
         cudaEventRecord(b);

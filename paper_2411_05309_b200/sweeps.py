@@ -209,6 +209,16 @@ def sweep_link(gib: float):
     sm = B.gpuvm_link_peak(host.data_ptr(), devb.data_ptr(), nbytes, 3)
     out.update({"sm_h2d_gbs": sm["h2d_gbs"], "sm_d2h_gbs": sm["d2h_gbs"], "sm_duplex_gbs": sm["duplex_gbs"]})
     print(json.dumps(out), flush=True)
+    # rows of 512 bytes at hashed positions of the first `span` bytes of the region: each at a position of its own
+    # (run 1) or `run` consecutive ones in the same 2 MiB of it
+    n_rows = 1 << 22
+    span = 1 << 30
+    while span <= nbytes:
+        for run in (1, 4, 16, 64, 256):
+            gbs = B.gpuvm_link_peak_scattered(host.data_ptr(), span, 512, n_rows, devb.data_ptr(), min(nbytes, 1 << 30), 2, run)
+            print(json.dumps({"sweep": "link", "rows_of_512_bytes": n_rows, "span_bytes": span, "rows_per_2MiB_run": run,
+                              "gbs": gbs}), flush=True)
+        span *= 8
 
 
 def sweep_writeback():

@@ -351,6 +351,10 @@ def test_scattered_link_peak_runs_and_checks_its_arguments(B):
     buf = torch.empty(8 << 20, dtype=torch.uint8, device="cuda")
     gbs = B.gpuvm_link_peak_scattered(host.data_ptr(), host.numel(), 512, 1 << 16, buf.data_ptr(), buf.numel(), 1)
     assert 0.5 < gbs < 200.0
+    gbs = B.gpuvm_link_peak_scattered(host.data_ptr(), host.numel(), 512, 1 << 16, buf.data_ptr(), buf.numel(), 1, run=64)
+    assert 0.5 < gbs < 200.0
+    with pytest.raises(B.GpuvmError):
+        B.gpuvm_link_peak_scattered(host.data_ptr(), host.numel(), 512, 16, buf.data_ptr(), buf.numel(), 1, run=0)
     for row_bytes, n_rows in ((24, 16), (1024, 16), (512, 0)):
         with pytest.raises(B.GpuvmError):
             B.gpuvm_link_peak_scattered(host.data_ptr(), host.numel(), row_bytes, n_rows, buf.data_ptr(), buf.numel(), 1)
