@@ -1434,6 +1434,11 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
             }
         };
         read_in_place(0, n_cold);
+        if (lane == 0 && n_here) gpuvm::stat_add(vm, gpuvm::kBytesDirect, (unsigned long long)n_here * row_bytes);
+        // the rows are in their slots for everybody before they are counted as staged
+        __threadfence();
+        __syncwarp();
+        if (lane == 0 && n_here) atomicAdd(const_cast<unsigned int *>(cold_counts) + 2, n_here);
         const unsigned long long t = slot, g0 = per_item * t;
         const unsigned int nk = bag;                             // one pass: bag <= kEmbagLookups, one item per warp
         if (t < items) {
@@ -1456,11 +1461,6 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
                                   queue, masks, 1u, true, 0u, (unsigned int)row_bytes, nullptr);
             __syncwarp();
         }
-        if (lane == 0 && n_here) gpuvm::stat_add(vm, gpuvm::kBytesDirect, (unsigned long long)n_here * row_bytes);
-        // the rows are in their slots for everybody before they are counted as staged
-        __threadfence();
-        __syncwarp();
-        if (lane == 0 && n_here) atomicAdd(const_cast<unsigned int *>(cold_counts) + 2, n_here);
         // A bag's rows that were read in place were staged by whichever warps had their bucket entries: wait
         // (bounded) until all of them are counted as staged.  Every warp stages its share before it comes here,
         // so the wait is for the stragglers of the grid only.  (The shares are fixed, not drawn from a counter:
