@@ -1409,7 +1409,7 @@ __global__ void __launch_bounds__(1024, 1) embag_batch_kernel(gpuvm_dev_t vm, un
         // have arrived by then (running the engine after 30, 50 or 70 % of the share was measured: 52 / 49 / 49 ms
         // against 44-45).
         unsigned int n_here = 0;
-        constexpr int Q = 4;
+        constexpr int Q = 4;                                     // (2, 4 and 8 rows in flight per warp: the same 44-46 ms)
         uint4 *const all_staging = reinterpret_cast<uint4 *>(g_staging);
         auto read_in_place = [&](unsigned long long j_begin, unsigned long long j_end) {
             for (unsigned long long j0 = j_begin + slot * Q; j0 < j_end; j0 += stride * Q) {
