@@ -1912,8 +1912,13 @@ int run_bfs_bcsr(const Mem &m, size_t off_off, size_t col_off, size_t chunk_off,
                                                                      (unsigned int)nv, n_edges, (unsigned int)chunk_edges,
                                                                      counters, depth);
         rc = launched();
+        const auto t0 = std::chrono::steady_clock::now();
         if (cudaMemcpyAsync(&found, counters, sizeof(found), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
             cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); rc = GPUVM_E_CUDA; break; }
+        static const bool trace = getenv("GPUVM_TRACE_SWEEPS") != nullptr;     // one line per level on stderr
+        if (trace)
+            fprintf(stderr, "level %d: %.3f ms (host clock, from launch to counters read), found %u\n", depth,
+                    std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count(), found);
         ++depth;
     }
     if (n_edges == 0) depth = 1;
