@@ -1010,7 +1010,9 @@ __global__ void __launch_bounds__(256, kBcsrBlocksPerSm) bcsr_sweep_kernel(Mem m
         // the chunk's column page: pinned at the first group that has an edge in it, held to the end of the block
         gpuvm_token tok;
         const unsigned char *p = nullptr;
-#pragma unroll
+        // (not unrolled: eight copies of the body below overflow the instruction cache, a quarter of all issue
+        // slots went to waiting for instructions; the eight offsets then live in local memory, two reads per group)
+#pragma unroll 1
         for (int k8 = 0; k8 < 8; ++k8) {
             if (!((group_active >> k8) & 1u)) continue;
             const unsigned int v0 = g0 + 32u * k8;
