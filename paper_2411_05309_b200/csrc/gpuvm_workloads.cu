@@ -644,16 +644,31 @@ __device__ __noinline__ int expand_behind(const Mem m, const Op op, unsigned lon
     bool have = u != kNoVertex && u < nv && op.active(u);
     long long lo = 0, hi = 0;
     unsigned long long direct = 0;                            // bytes read in place from the backing store
+    // The two row offsets of each vertex: from their frame when the page is resident, else in place from the
+    // backing store (no page is fetched for a vertex behind the sweep).
+    bool got = false;
     if (have) {
-        // the two row offsets: from their frame when the page is resident, else in place from the backing store
-        // (no page is fetched for a vertex behind the sweep)
-        gpuvm_token tok;
-        const unsigned char *p = m.pin_if_resident(off_off + 8ull * u, tok);
-        if (p) { lo = Mem::load_i64(p); m.release(tok); }
-        else { lo = Mem::load_i64(m.through(off_off + 8ull * u)); direct += 8; }
-        const unsigned char *q = m.pin_if_resident(off_off + 8ull * u + 8, tok);
-        if (q) { hi = Mem::load_i64(q); m.release(tok); }
-        else { hi = Mem::load_i64(m.through(off_off + 8ull * u + 8)); direct += 8; }
+        const unsigned long long ob = off_off + 8ull * u, unit_o = m.unit();
+        if (ob / unit_o == (ob + 8) / unit_o) {                // both in one page: one pin
+            gpuvm_token tok;
+            const unsigned char *p = m.pin_if_resident(ob, tok);
+            if (p) { lo = Mem::load_i64(p); hi = Mem::load_i64(p + 8); m.release(tok); got = true; }
+        }
+    }
+    // In place, two lanes per vertex, so that the pair's loads are one instruction and, the two offsets lying
+    // side by side, one request on the link (issued by one lane one after the other they were two): what these
+    // reads cost is requests.
+    const unsigned int in_place = __ballot_sync(0xFFFFFFFFu, have && !got);
+#pragma unroll
+    for (unsigned int r = 0; r < 2 && in_place; ++r) {
+        const unsigned int src = (lane >> 1) + 16u * r;
+        const unsigned int uu = __shfl_sync(0xFFFFFFFFu, u, src);
+        long long val = 0;
+        if ((in_place >> src) & 1u) val = Mem::load_i64(m.through(off_off + 8ull * ((unsigned long long)uu + (lane & 1u))));
+        const long long a = __shfl_sync(0xFFFFFFFFu, val, (lane & 15u) * 2u), b = __shfl_sync(0xFFFFFFFFu, val, (lane & 15u) * 2u + 1u);
+        if ((lane >> 4) == r && ((in_place >> lane) & 1u)) { lo = a; hi = b; direct += 16; }
+    }
+    if (have) {
         if (hi <= lo) { op.begin(u); have = false; }          // nothing to expand: just not dirty any more
         if (have && hi - lo >= kBigDegree) have = false;      // a hub: left dirty, the next sweep cuts it into pieces
     }
