@@ -226,6 +226,14 @@ int gpuvm_set_clean_ahead(gpuvm_t h, unsigned int frames);
 int gpuvm_set_scratch_limit(gpuvm_t h, size_t bytes);
 size_t gpuvm_scratch_bytes(gpuvm_t h);
 
+/* Advice: the pages that hold [byte_off, byte_off + bytes) are not to be evicted (keep != 0), or may be again
+ * (keep == 0).  A kept page is fetched when it is first touched, like any other, and then stays in its frame
+ * whatever the pressure on the pool; the evictor passes over it.  For small arrays that every part of a workload
+ * comes back to (the row offsets of a graph beside its edge arrays).  At most half the pool's frames may be kept
+ * (GPUVM_E_FRAMES beyond that; GPUVM_E_RANGE outside the backing store); the advice survives gpuvm_reset and is
+ * dropped with the handle.  Synchronises the device. */
+int gpuvm_advise_keep(gpuvm_t h, size_t byte_off, size_t bytes, int keep);
+
 /* Reading rows in place instead of fetching their page (not in the paper, which fetches a page at its first
  * fault).  The batched row workloads (gpuvm_embag_f32) do not fetch a page for a few rows: pinned host memory is as
  * reachable for a load as for a page copy, so rows of pages with few lookups are read in place from the backing

@@ -65,6 +65,7 @@ SYMBOLS = {
     "gpuvm_set_debug": (_i, [_vp, ctypes.c_uint]),
     "gpuvm_set_clean_ahead": (_i, [_vp, ctypes.c_uint]),
     "gpuvm_set_inplace_divisor": (_i, [_vp, ctypes.c_uint]),
+    "gpuvm_advise_keep": (_i, [_vp, _sz, _sz, _i]),
     "gpuvm_set_inplace_counted": (_i, [_vp, _i]),
     "gpuvm_bcsr_build": (_i, [_vp, _sz, _sz, _vp, _sz, ctypes.POINTER(_sz)]),
     "gpuvm_device_view": (_i, [_vp, ctypes.POINTER(DevView)]),
@@ -204,6 +205,10 @@ def gpuvm_check_on(h, stream, raise_on_error: bool = True) -> dict:
     d = c.as_dict()
     d["status"] = rc
     return d
+
+
+def gpuvm_advise_keep(h, byte_off: int, nbytes: int, keep: bool = True):
+    _check(lib().gpuvm_advise_keep(h, byte_off, nbytes, int(bool(keep))), "gpuvm_advise_keep")
 
 
 INPLACE_AUTO = 0xFFFFFFFF

@@ -24,6 +24,7 @@ struct gpuvm_handle {
     size_t scratch_bytes;
     size_t scratch_limit;      /* 0: none */
     unsigned int inplace_divisor;
+    unsigned long long kept_pages;   // pages with the keep advice (gpuvm_advise_keep)
     int inplace_counted;    // 0: online; 1: lookups counted per page first; 2: counted, and rows in place read page by page
 };
 
@@ -80,9 +81,9 @@ __global__ void check_kernel(gpuvm_dev_t vm, unsigned long long *out)
             unsigned long long f = (w & kFrameMask) >> kFrameShift;
             if (f >= vm.n_frames) c[5]++;
             else if (vm.frame_vpn[f] != (unsigned int)v) c[4]++;
-            if (w & ~(kStMask | kDirty | kRef | kFrameMask | kRcMask)) c[2]++;
+            if (w & ~(kStMask | kDirty | kRef | kKeep | kFrameMask | kRcMask)) c[2]++;
         } else if (st == kInvalid) {
-            if (w & ~(kRcMask | kFrameMask)) c[2]++;        // (the frame field counts in-place reads while INVALID)
+            if (w & ~(kRcMask | kFrameMask | kKeep)) c[2]++;   // (the frame field counts in-place reads while INVALID)
         } else {
             c[2]++;
         }
@@ -101,6 +102,26 @@ __global__ void check_kernel(gpuvm_dev_t vm, unsigned long long *out)
         for (int o = 16; o; o >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, o);
         if ((threadIdx.x & 31) == 0 && v) atomicAdd(out + k, v);
     }
+}
+
+__global__ void reset_keep_kernel(unsigned long long *pte, unsigned long long n_pages)
+{
+    for (unsigned long long v = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; v < n_pages;
+         v += (unsigned long long)gridDim.x * blockDim.x)
+        pte[v] &= kKeep;
+}
+
+// Sets or clears the keep bit of the pages [first, first + n); *changed counts the entries whose bit changed.
+__global__ void advise_keep_kernel(unsigned long long *pte, unsigned long long first, unsigned long long n, int keep,
+                                   unsigned long long *changed)
+{
+    unsigned long long c = 0;
+    for (unsigned long long v = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; v < n;
+         v += (unsigned long long)gridDim.x * blockDim.x) {
+        const unsigned long long old = keep ? atomicOr(pte + first + v, kKeep) : atomicAnd(pte + first + v, ~kKeep);
+        c += ((old & kKeep) != 0ull) != (keep != 0);
+    }
+    if (c) atomicAdd(changed, c);
 }
 
 // Number of SMs of the handle's device (grids are sized in multiples of it).
@@ -217,7 +238,14 @@ int gpuvm_reset_on(gpuvm_t h, void *stream)
     if (!h) return GPUVM_E_ARG;
     gpuvm_dev_t &d = h->dev;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemsetAsync(d.pte, 0, d.n_pages * sizeof(unsigned long long), s);
+    cudaError_t e = cudaSuccess;
+    if (h->kept_pages == 0) {
+        e = cudaMemsetAsync(d.pte, 0, d.n_pages * sizeof(unsigned long long), s);
+    } else {                                                  // advice survives a reset
+        reset_keep_kernel<<<h->sms * 4, 256, 0, s>>>(d.pte, d.n_pages);
+        gpuvm_note_launch_(1);
+        e = cudaGetLastError();
+    }
     if (e == cudaSuccess) e = cudaMemsetAsync(d.frame_vpn, 0xFF, d.n_frames * sizeof(unsigned int), s);
     if (e == cudaSuccess) e = cudaMemsetAsync(d.ctl, 0, kCtlWords * sizeof(unsigned long long), s);
     return e == cudaSuccess ? GPUVM_OK : fail(h, e, GPUVM_E_CUDA);
@@ -346,6 +374,29 @@ int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor)
 {
     if (!h) return GPUVM_E_ARG;
     h->inplace_divisor = divisor;
+    return GPUVM_OK;
+}
+
+int gpuvm_advise_keep(gpuvm_t h, size_t byte_off, size_t bytes, int keep)
+{
+    if (!h || bytes == 0) return GPUVM_E_ARG;
+    gpuvm_dev_t &d = h->dev;
+    if (byte_off >= d.bytes || bytes > d.bytes - byte_off) return GPUVM_E_RANGE;
+    const unsigned long long first = byte_off >> d.page_shift, last = (byte_off + bytes - 1) >> d.page_shift;
+    const unsigned long long n = last - first + 1;
+    // pages that may never be evicted must leave room for the others: at most half the pool
+    if (keep && h->kept_pages + n > d.n_frames / 2) return GPUVM_E_FRAMES;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
+    unsigned long long *changed = h->check_buf;               // (device scratch of the checker, free between calls)
+    e = cudaMemset(changed, 0, sizeof(unsigned long long));
+    if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
+    advise_keep_kernel<<<h->sms * 4, 256>>>(d.pte, first, n, keep, changed);
+    gpuvm_note_launch_(1);
+    unsigned long long c = 0;
+    e = cudaMemcpy(&c, changed, sizeof(c), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(h, e, GPUVM_E_CUDA);
+    if (keep) h->kept_pages += c; else h->kept_pages -= c < h->kept_pages ? c : h->kept_pages;
     return GPUVM_OK;
 }
 

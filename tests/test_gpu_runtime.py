@@ -358,3 +358,50 @@ def test_scattered_link_peak_runs_and_checks_its_arguments(B):
     for row_bytes, n_rows in ((24, 16), (1024, 16), (512, 0)):
         with pytest.raises(B.GpuvmError):
             B.gpuvm_link_peak_scattered(host.data_ptr(), host.numel(), row_bytes, n_rows, buf.data_ptr(), buf.numel(), 1)
+
+
+def test_advise_keep_pages_stay_resident_under_pressure(B):
+    """Pages advised to be kept are fetched at their first touch and never evicted afterwards, whatever streams
+    through the rest of the pool; the advice survives a reset, can be taken back, and is refused beyond half the
+    pool and outside the backing store."""
+    import torch
+    page, n_pages, frames = 4096, 64, 8
+    per_page = page // 4
+    n = n_pages * per_page
+    a = inputs.fill_i32_u20(np.empty(n, np.int32), n, 7)
+    ar = Arena(page, {"a": a})
+    out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    head = int(a[:4 * per_page].astype(np.int64).sum())
+
+    def touch_head_then_flood(h):
+        """Read pages 0..3, stream pages 8..63 through the pool, read pages 0..3 again; returns the faults of the
+        last read and the states of pages 0..3 before it."""
+        B.gpuvm_stream_sum_i32(h, 0, 4 * per_page, out)
+        assert int(out.item()) == head
+        B.gpuvm_stream_sum_i32(h, 8 * page, 56 * per_page, out)
+        before = finish(h)[0]["faults"]
+        states = [(B.gpuvm_debug_peek_pte(h, p) >> 60) & 3 for p in range(4)]
+        B.gpuvm_stream_sum_i32(h, 0, 4 * per_page, out)
+        assert int(out.item()) == head
+        return finish(h)[0]["faults"] - before, states
+
+    with paged(ar.host, page, frames) as h:
+        again, states = touch_head_then_flood(h)
+        assert again == 4 and states == [0, 0, 0, 0]                      # without advice: evicted, fetched again
+        B.gpuvm_reset(h)
+        B.gpuvm_advise_keep(h, 0, 4 * page)                              # pages 0..3
+        again, states = touch_head_then_flood(h)
+        assert again == 0 and states == [2, 2, 2, 2]                      # VALID throughout
+        B.gpuvm_reset(h)                                                  # the advice survives a reset
+        again, states = touch_head_then_flood(h)
+        assert again == 0 and states == [2, 2, 2, 2]
+        B.gpuvm_advise_keep(h, 0, 4 * page, False)                        # taken back: evictable again
+        B.gpuvm_reset(h)
+        again, states = touch_head_then_flood(h)
+        assert again == 4 and states == [0, 0, 0, 0]
+        with pytest.raises(B.GpuvmError) as e:
+            B.gpuvm_advise_keep(h, 0, 5 * page)                           # more than half of eight frames
+        assert e.value.status == B.E_FRAMES
+        with pytest.raises(B.GpuvmError) as e:
+            B.gpuvm_advise_keep(h, ar.host.nbytes, page)
+        assert e.value.status == B.E_RANGE
