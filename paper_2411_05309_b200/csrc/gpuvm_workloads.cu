@@ -504,6 +504,8 @@ struct LcOp {
     __device__ __forceinline__ void redirty(unsigned long long v) const { atomicOr(dist + v, 1); }
     __device__ __forceinline__ int value(unsigned long long u) const { return __ldcg(dist + u) >> 1; }
     __device__ __forceinline__ int peek(int c) const { return dist[c]; }
+    // could an edge of weight >= 0 from a vertex at distance du lower a vertex whose entry reads `seen`?
+    __device__ __forceinline__ bool could_lower(int du, int seen) const { return ((du << 1) | 1) < seen; }
     __device__ __forceinline__ unsigned int edge(int du, long long, int c, int w, int seen, unsigned int pos) const
     {
         const int nd = ((du + (WEIGHTED ? w : 1)) << 1) | 1;
@@ -526,10 +528,13 @@ struct LcOp {
 // Visit the edges [elo, ehi) of vertex u that lie inside the pinned unit starting at edge `first`,
 // four per lane at a time: the column (and weight) loads of the four are issued together, then
 // the peeks at their other ends, then the updates.
-template <class Mem, class Op, bool WEIGHTED>
+// LAZY_W (weights that would be read in place over the link): a weight is loaded only for an edge that could
+// lower its other end at all, i.e. with the weight 0; where no edge of a 128-byte line can, the line is not
+// requested.  Most edges of a vertex that is expanded again cannot, and what reads in place cost is requests.
+template <class Mem, class Op, bool WEIGHTED, bool LAZY_W = false>
 __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned char *col_unit, const unsigned char *w_unit,
                                                     long long first, long long u, int uval, long long elo, long long ehi,
-                                                    unsigned int lane, unsigned int pos)
+                                                    unsigned int lane, unsigned int pos, unsigned long long *lazy_bytes = nullptr)
 {
     constexpr int U = 4;
     unsigned int found = 0;
@@ -539,10 +544,17 @@ __device__ __forceinline__ unsigned int visit_edges(const Op &op, const unsigned
         for (int k = 0; k < U; ++k) {
             const long long e = e0 + 32 * k;
             c[k] = e < ehi ? Mem::load_i32(col_unit + 4 * (e - first)) : -1;
-            w[k] = (WEIGHTED && e < ehi) ? Mem::load_i32(w_unit + 4 * (e - first)) : 0;
+            w[k] = (WEIGHTED && !LAZY_W && e < ehi) ? Mem::load_i32(w_unit + 4 * (e - first)) : 0;
         }
 #pragma unroll
         for (int k = 0; k < U; ++k) seen[k] = c[k] >= 0 ? op.peek(c[k]) : 0;
+        if constexpr (WEIGHTED && LAZY_W) {
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                if (c[k] >= 0 && !op.could_lower(uval, seen[k])) c[k] = -1;
+                if (c[k] >= 0) { w[k] = Mem::load_i32(w_unit + 4 * (e0 + 32 * k - first)); if (lazy_bytes) *lazy_bytes += 4; }
+            }
+        }
 #pragma unroll
         for (int k = 0; k < U; ++k)
             if (c[k] >= 0) found += op.edge(uval, u, c[k], w[k], seen[k], pos);
@@ -698,9 +710,10 @@ __device__ __noinline__ int expand_behind(const Mem m, const Op op, unsigned lon
             if (WEIGHTED) {
                 pw = m.pin_if_resident(w_off + 4ull * first, tok_w);
                 held_w = pw != nullptr;
-                if (!held_w) { pw = m.through(w_off + 4ull * first); if (lane == 0) direct += 4ull * (unsigned long long)(last - first); }
+                if (!held_w) pw = m.through(w_off + 4ull * first);      // (its bytes are counted as they are loaded)
             }
-            found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, bu, uval, first, last, lane, pos);
+            if (WEIGHTED && !held_w) found += visit_edges<Mem, Op, WEIGHTED, true>(op, p, pw, first, bu, uval, first, last, lane, pos, &direct);
+            else found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, bu, uval, first, last, lane, pos);
             if (held_w) m.release(tok_w);
             if (held) m.release(tok);
             first = last;
@@ -789,6 +802,7 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
     const long long epoch = sweep + 1;
     unsigned int found = 0, my_done = 0, iter = 0, next_chunk = 0, last_chunk = 0;
     unsigned long long direct = 0;                           // bytes this lane read in place from the backing store
+    unsigned long long direct_w = 0;                         // weights this lane loaded in place, in bytes (all lanes count)
     for (;;) {
         // ---- a piece of a long neighbour list, if one is waiting (looked for before every kSpanPoll-th chunk)
         if ((iter++ & (kSpanPoll - 1)) == 0) {
@@ -943,8 +957,11 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
                     const int bval = __shfl_sync(0xFFFFFFFFu, uval, L);
                     if (blo < first) blo = first;
                     if (bhi > last) bhi = last;
-                    found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, (long long)(v0 + L), bval, blo, bhi, lane, pos);
-                    if (lane == 0) direct += 4ull * (unsigned long long)(bhi - blo) * ((held ? 0u : 1u) + (WEIGHTED && !held_w ? 1u : 0u));
+                    if (WEIGHTED && !held_w)
+                        found += visit_edges<Mem, Op, WEIGHTED, true>(op, p, pw, first, (long long)(v0 + L), bval, blo, bhi, lane, pos, &direct_w);
+                    else
+                        found += visit_edges<Mem, Op, WEIGHTED>(op, p, pw, first, (long long)(v0 + L), bval, blo, bhi, lane, pos);
+                    if (lane == 0 && !held) direct += 4ull * (unsigned long long)(bhi - blo);   // (weights: direct_w, as they are loaded)
                 }
                 if (held_w) m.release(tok_w);
                 if (held) m.release(tok);
@@ -955,7 +972,8 @@ __global__ void __launch_bounds__(256, 4) graph_sweep_kernel(Mem m, Op op, unsig
     }
     for (int o = 16; o; o >>= 1) found += __shfl_down_sync(0xFFFFFFFFu, found, o);
     if (lane == 0 && found) atomicAdd(counters + kCntUpdates, found);
-    if (lane == 0 && direct) m.note_direct(direct);
+    for (int o = 16; o; o >>= 1) direct_w += __shfl_down_sync(0xFFFFFFFFu, direct_w, o);
+    if (lane == 0 && direct + direct_w) m.note_direct(direct + direct_w);
 }
 
 // Balanced CSR (Section 5.2, Fig. 8): the edge array is cut into chunks of equal length and a
