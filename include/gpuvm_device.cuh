@@ -80,6 +80,7 @@ constexpr unsigned long long kFrameMask = 0xFFFFFFFFull << kFrameShift;
 constexpr unsigned long long kRef = 1ull << 56;
 constexpr unsigned long long kDirty = 1ull << 57;
 constexpr unsigned long long kKeep = 1ull << 58;    /* advice: not to be evicted (gpuvm_advise_keep); survives every state change */
+constexpr unsigned long long kHold = 1ull << 59;    /* not to be evicted while the running kernel reads it without a reference (set and cleared by that kernel) */
 constexpr unsigned long long kStMask = 3ull << 60;
 constexpr unsigned long long kInvalid = 0ull;
 constexpr unsigned long long kBusy = 1ull << 60;
@@ -496,7 +497,7 @@ __device__ __forceinline__ bool try_claim(const gpuvm_dev_t &vm, unsigned long l
         if ((w & kStMask) != kValid || (w & kRcMask) != 0ull ||
             (unsigned int)((w & kFrameMask) >> kFrameShift) != h)
             continue;                                       /* in use, or a stale ring read */
-        if (w & kKeep) continue;                            /* the caller asked for this page to stay */
+        if (w & (kKeep | kHold)) continue;                  /* the caller asked for this page to stay, or a kernel is reading it unpinned */
         if (vm.policy == GPUVM_POLICY_CLOCK && (w & kRef)) {
             atomicAnd(qpte, ~kRef);                         /* second chance */
             continue;

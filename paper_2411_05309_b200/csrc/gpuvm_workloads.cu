@@ -1328,21 +1328,26 @@ __global__ void __launch_bounds__(1024) embag_bucket_scan_kernel(const unsigned 
     for (int o = 16; o; o >>= 1) hot += __shfl_down_sync(0xFFFFFFFFu, hot, o);
     if (lane == 0 && hot) atomicAdd(&hot_s, hot);
     __syncthreads();
-    if (threadIdx.x == 0) { counts[0] = carry_s; counts[1] = hot_s; counts[2] = 0; }
+    if (threadIdx.x == 0) { counts[0] = carry_s; counts[1] = hot_s; counts[2] = 0; counts[4] = 0; counts[5] = 0; }
 }
 
 // After this kernel bucket_off[p] is the END of page p's bucket (every cold lookup moved it on by one).
 __global__ void embag_bucket_fill_kernel(const long long *__restrict__ rows, unsigned long long n, unsigned long long t_off,
                                          unsigned long long row_bytes, unsigned int page_shift, unsigned long long rows_inside,
                                          const unsigned int *__restrict__ demand, unsigned int limit,
-                                         unsigned int *__restrict__ bucket_off, unsigned int *__restrict__ cold_idx)
+                                         unsigned int *__restrict__ bucket_off, unsigned int *__restrict__ cold_idx,
+                                         unsigned int *__restrict__ where = nullptr)
 {
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n; i += stride) {
         const unsigned long long r = (unsigned long long)rows[i];
         if (r >= rows_inside) continue;
         const unsigned int vpn = (unsigned int)((t_off + r * row_bytes) >> page_shift);
-        if (demand[vpn] < limit) cold_idx[atomicAdd(bucket_off + vpn, 1u)] = (unsigned int)i;
+        if (demand[vpn] < limit) {
+            const unsigned int pos = atomicAdd(bucket_off + vpn, 1u);
+            cold_idx[pos] = (unsigned int)i;
+            if (where) where[i] = pos;                      // (where[] starts out as kNoSlot everywhere)
+        }
     }
 }
 
@@ -1355,6 +1360,185 @@ __device__ __forceinline__ size_t embag_staged_row(unsigned long long i, unsigne
     const unsigned long long t = g / per_item;
     const unsigned int rr = (unsigned int)(g - t * per_item), gi = rr >> 5, b = rr & 31u;
     return (size_t)t * ((size_t)groups * 32 * bag) + (size_t)((gi * bag + k) * 32 + b);
+}
+
+// The embedding bag when the pages that are worth fetching fit the pool twice over: no request tables, no copy of
+// the rows of fetched pages.  counts: [0] cold lookups, [1] pages to fetch, [2] cold rows staged, [4] warps past
+// step (1), [5] warps finished.
+//   (1) every page at or above the limit gets the hold bit (the evictor passes over it until this kernel clears
+//       the bit again) and, where it is not resident, is handed to the fault ring for the migrator warps;
+//   (2) the rows of the other pages are read in place, in bucket order, into a staging area that holds just them
+//       (cold_staging[j] for bucket entry j; where[i] = j for lookup i);
+//   (3) when all warps are past (1) and all cold rows are staged, a warp adds up its bags in list order: a cold row
+//       from the staging area, any other straight from its page's frame, without a reference (the hold bit
+//       protects the frame), waiting (bounded) for pages that are still on their way;
+//   (4) the last warp to finish clears the hold bits.
+constexpr unsigned int kNoSlot = 0xFFFFFFFFu;
+__global__ void __launch_bounds__(1024, 1) embag_direct_kernel(gpuvm_dev_t vm, unsigned long long t_off, unsigned int dims,
+                                                               const long long *__restrict__ rows, unsigned long long n_bags,
+                                                               unsigned int bag, float *__restrict__ out, int requesters,
+                                                               gpuvm_shared_queue *shared_queue, unsigned int limit,
+                                                               const unsigned int *__restrict__ demand,
+                                                               const unsigned int *__restrict__ cold_idx,
+                                                               const unsigned int *__restrict__ where, uint4 *cold_staging,
+                                                               unsigned int *counts)
+{
+    __shared__ gpuvm_fault_queue queue_s;
+    extern __shared__ __align__(128) unsigned char stage_s[];   // bulk-copy staging: kEmbagStages chunks per migrator warp
+    __shared__ __align__(8) unsigned long long mbar_s[kEmbagMigrators][kEmbagStages];
+    gpuvm_fault_queue *queue = &queue_s;
+    const unsigned int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (unsigned int k = threadIdx.x; k < sizeof(gpuvm_fault_queue) / 4; k += blockDim.x)
+        reinterpret_cast<unsigned int *>(queue)[k] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) { queue->requesters = (unsigned int)requesters; queue->shared = shared_queue; }
+    __syncthreads();
+    if ((int)warp >= requesters) {
+        const unsigned int mig = warp - requesters;
+        const unsigned int chunk = (1ull << vm.page_shift) < kEmbagChunk ? (unsigned int)(1ull << vm.page_shift) : kEmbagChunk;
+        if (mig < kEmbagMigrators && chunk >= 128)
+            gpuvm_migrator_loop(vm, queue, stage_s + (size_t)mig * kEmbagStages * kEmbagChunk, mbar_s[mig], chunk, kEmbagStages);
+        else
+            gpuvm_migrator_loop(vm, queue);
+        return;
+    }
+    const unsigned int q = dims >> 2;                            // 16-byte pieces per row
+    const unsigned long long row_bytes = 4ull * dims;
+    const unsigned long long slot = (unsigned long long)blockIdx.x * requesters + warp;
+    const unsigned long long stride = (unsigned long long)gridDim.x * requesters;
+    const unsigned long long rows_inside = (vm.bytes - t_off) / row_bytes;
+    const unsigned int n_cold = counts[0];
+    const unsigned long long limit_ns = (unsigned long long)vm.spin_limit_us * 1000ull;
+
+    // hand page p to the migrators: the caller has turned its entry BUSY
+    auto push = [&](unsigned long long p) {
+        unsigned long long t0 = 0;
+        while (!gpuvm::fault_queue_push(queue, (unsigned int)p, gpuvm::kRead, &vm)) {
+            const unsigned long long now = gpuvm::now_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > limit_ns || gpuvm::has_error(vm)) {
+                gpuvm::set_error(vm, GPUVM_E_TIMEOUT, p);
+                atomicXor(vm.pte + p, gpuvm::kBusy);             // back to INVALID
+                return;
+            }
+            __nanosleep(256);
+        }
+    };
+
+    // (1)
+    for (unsigned long long p = slot * 32 + lane; p < vm.n_pages; p += stride * 32) {
+        if (demand[p] < limit) continue;
+        const unsigned long long w = atomicOr(vm.pte + p, gpuvm::kHold) | gpuvm::kHold;
+        if ((w & gpuvm::kStMask) == gpuvm::kInvalid && atomicCAS(vm.pte + p, w, (w & ~gpuvm::kFrameMask) | gpuvm::kBusy) == w)
+            push(p);
+    }
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) atomicAdd(counts + 4, 1u);
+
+    // (2)
+    unsigned int n_here = 0;
+    constexpr int Q = 4;
+    for (unsigned long long j0 = slot * Q; j0 < n_cold; j0 += stride * Q) {
+        uint4 v[Q];
+        int cnt = 0;
+#pragma unroll
+        for (int u = 0; u < Q; ++u)
+            if (j0 + u < n_cold) {
+                const unsigned long long r = (unsigned long long)rows[cold_idx[j0 + u]];
+                if (lane < q) v[u] = gpuvm_load16(vm.host + t_off + r * row_bytes + 16u * lane);
+                cnt = u + 1;
+            }
+#pragma unroll
+        for (int u = 0; u < Q; ++u)
+            if (u < cnt && lane < q) cold_staging[(j0 + u) * q + lane] = v[u];
+        n_here += cnt;
+    }
+    if (lane == 0 && n_here) gpuvm::stat_add(vm, gpuvm::kBytesDirect, (unsigned long long)n_here * row_bytes);
+    __threadfence();
+    __syncwarp();
+    if (lane == 0 && n_here) atomicAdd(counts + 2, n_here);
+
+    // (3) wait for the stragglers of (1) and (2)
+    {
+        unsigned long long t0 = 0;
+        bool ok = true;
+        while (ld_volatile_u32(counts + 2) < n_cold || ld_volatile_u32(counts + 4) < (unsigned int)stride) {
+            const unsigned long long now = gpuvm::now_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > limit_ns || gpuvm::has_error(vm)) { ok = false; break; }
+            __nanosleep(256);
+        }
+        if (!__all_sync(0xFFFFFFFFu, ok) && lane == 0) gpuvm::set_error(vm, GPUVM_E_TIMEOUT, ~0ull);
+        __threadfence();
+    }
+    for (unsigned long long g = slot; g < n_bags && !gpuvm::has_error(vm); g += stride) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (unsigned int k0 = 0; k0 < bag; k0 += 32) {
+            const unsigned int nk = bag - k0 < 32u ? bag - k0 : 32u;
+            // lane k finds where the row of lookup k0 + k is
+            const unsigned char *src = nullptr;
+            if (lane < nk) {
+                const unsigned long long i = g * bag + k0 + lane;
+                const unsigned long long r = (unsigned long long)rows[i];
+                const unsigned int at = where[i];
+                if (at != kNoSlot) {
+                    src = reinterpret_cast<const unsigned char *>(cold_staging) + (size_t)at * row_bytes;
+                } else if (r >= rows_inside) {
+                    gpuvm::set_error(vm, GPUVM_E_RANGE, ~0ull);   // a row past the end of the table: nothing is added for it
+                } else {
+                    const unsigned long long byte_off = t_off + r * row_bytes, p = byte_off >> vm.page_shift;
+                    unsigned long long t0 = 0;
+                    for (;;) {
+                        const unsigned long long w = gpuvm::ld_acquire_u64(vm.pte + p);
+                        const unsigned long long st = w & gpuvm::kStMask;
+                        if (st == gpuvm::kValid) {
+                            src = vm.pool + (((w & gpuvm::kFrameMask) >> gpuvm::kFrameShift) << vm.page_shift) +
+                                  (byte_off & ((1ull << vm.page_shift) - 1ull));
+                            break;
+                        }
+                        // nobody has asked for it (it was being evicted when (1) looked): ask now
+                        if (st == gpuvm::kInvalid && atomicCAS(vm.pte + p, w, (w & ~gpuvm::kFrameMask) | gpuvm::kBusy) == w) push(p);
+                        const unsigned long long now = gpuvm::now_ns();
+                        if (t0 == 0) t0 = now;
+                        if (now - t0 > limit_ns || gpuvm::has_error(vm)) { gpuvm::set_error(vm, GPUVM_E_TIMEOUT, p); break; }
+                        __nanosleep(128);
+                    }
+                }
+            }
+            __syncwarp();
+            // the rows, in list order, eight loads in flight
+            for (unsigned int k = 0; k < nk; k += 8) {
+                uint4 v[8];
+#pragma unroll
+                for (unsigned int u = 0; u < 8; ++u) {
+                    const unsigned char *s = reinterpret_cast<const unsigned char *>(
+                        __shfl_sync(0xFFFFFFFFu, reinterpret_cast<unsigned long long>(src), (k + u) & 31u));
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (k + u < nk && s != nullptr && lane < q) v[u] = gpuvm_load16(s + 16u * lane);
+                }
+#pragma unroll
+                for (unsigned int u = 0; u < 8; ++u)
+                    if (k + u < nk) {
+                        acc.x = __fadd_rn(acc.x, __uint_as_float(v[u].x));
+                        acc.y = __fadd_rn(acc.y, __uint_as_float(v[u].y));
+                        acc.z = __fadd_rn(acc.z, __uint_as_float(v[u].z));
+                        acc.w = __fadd_rn(acc.w, __uint_as_float(v[u].w));
+                    }
+            }
+        }
+        if (lane < q) reinterpret_cast<float4 *>(out + g * dims)[lane] = acc;
+    }
+
+    // (4) the last warp to get here lets the pages go
+    __syncwarp();
+    unsigned int done = 0;
+    if (lane == 0) done = atomicAdd(counts + 5, 1u) + 1u;
+    done = __shfl_sync(0xFFFFFFFFu, done, 0);
+    if (done == (unsigned int)stride)
+        for (unsigned long long p = lane; p < vm.n_pages; p += 32)
+            if (demand[p] >= limit) atomicAnd(vm.pte + p, ~gpuvm::kHold);
+    if (lane == 0) gpuvm_requester_done(queue);
 }
 
 // All 32 lanes: add the staged rows of the warp's bags g0 .. g0 + 32 groups - 1 in list order (lookups k of this
@@ -2285,6 +2469,74 @@ int gpuvm_embag_f32(gpuvm_t h, size_t t_off, size_t dims, const int64_t *d_rows,
     if (page_bytes % row_bytes != 0 || t_off % row_bytes != 0)
         return run_embag(m, t_off, dims, d_rows, n_bags, bag, d_out, static_cast<cudaStream_t>(stream));
     const int requesters = kEmbagRequesters, migrators = kEmbagMigrators;
+    {
+        // The direct form (embag_direct_kernel): lookups counted per page, rows of the pages below the limit read in
+        // place page by page into a staging area of their own, every other row read straight from its page's
+        // frame.  It needs the pages at or above the limit to fit the pool twice over (they are held in their
+        // frames for the length of the launch) and their number to fit the fault rings; how many there are is
+        // read back after the count, which makes this call synchronous at that point.
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        const size_t n_lookups = n_bags * bag;
+        size_t divisor = gpuvm_inplace_divisor_(h);
+        if (divisor == GPUVM_INPLACE_AUTO) divisor = 1;
+        const size_t charged = row_bytes < 128 ? 128 : row_bytes;
+        const unsigned int limit = divisor ? (unsigned int)(page_bytes / divisor / charged) : 0u;
+        if (gpuvm_inplace_counted_(h) == 2 && limit != 0u && n_lookups < 0xFFFFFFFFull && m.vm.n_pages <= (1ull << 20)) {
+            const long long *rows_ll = reinterpret_cast<const long long *>(d_rows);
+            const unsigned long long rows_inside = (m.vm.bytes - t_off) / row_bytes;
+            const size_t pages_bytes = (m.vm.n_pages * sizeof(unsigned int) + 255) & ~size_t(255);
+            const size_t head_bytes = 2 * pages_bytes + 256 + sizeof(gpuvm_shared_queue);      // demand, bucket starts, counts, ring
+            const size_t where_bytes = (n_lookups * sizeof(unsigned int) + 255) & ~size_t(255);
+            unsigned int host_counts[2] = {0, 0};
+            unsigned char *scratch = nullptr;
+            unsigned int *demand = nullptr, *bucket_off = nullptr, *counts = nullptr;
+            size_t total = head_bytes;
+            bool fits = true;
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                scratch = static_cast<unsigned char *>(gpuvm_scratch_(h, total));
+                if (!scratch) return GPUVM_E_ALLOC;
+                demand = reinterpret_cast<unsigned int *>(scratch);
+                bucket_off = reinterpret_cast<unsigned int *>(scratch + pages_bytes);
+                counts = reinterpret_cast<unsigned int *>(scratch + 2 * pages_bytes);
+                if (cudaMemsetAsync(demand, 0, pages_bytes, s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+                embag_demand_kernel<<<sm_count() * 8, 256, 0, s>>>(rows_ll, n_lookups, t_off, row_bytes, m.vm.page_shift, rows_inside,
+                                                                    demand, limit);
+                embag_bucket_scan_kernel<<<1, 1024, 0, s>>>(demand, (unsigned int)m.vm.n_pages, limit, bucket_off, counts);
+                gpuvm_note_launch_(2);
+                if (cudaMemcpyAsync(host_counts, counts, sizeof(host_counts), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                    cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+                const size_t cold_bytes = ((size_t)host_counts[0] * sizeof(unsigned int) + 255) & ~size_t(255);
+                const size_t rows_bytes_total = ((size_t)host_counts[0] * row_bytes + 255) & ~size_t(255);
+                total = head_bytes + cold_bytes + where_bytes + rows_bytes_total;
+                fits = 2ull * host_counts[1] <= m.vm.n_frames && host_counts[1] <= 32768u &&
+                       (gpuvm_scratch_limit_(h) == ~size_t(0) || total <= gpuvm_scratch_limit_(h));
+                if (!fits || total <= gpuvm_scratch_bytes(h)) break;     // else: the scratch grows and the count is taken again in it
+            }
+            if (fits) {
+                const size_t cold_bytes = ((size_t)host_counts[0] * sizeof(unsigned int) + 255) & ~size_t(255);
+                unsigned int *cold_idx = reinterpret_cast<unsigned int *>(scratch + head_bytes);
+                unsigned int *where = reinterpret_cast<unsigned int *>(scratch + head_bytes + cold_bytes);
+                uint4 *cold_staging = reinterpret_cast<uint4 *>(scratch + head_bytes + cold_bytes + where_bytes);
+                gpuvm_shared_queue *shared_queue = shared_queue_at(m.vm, scratch + 2 * pages_bytes + 256, s);
+                if (cudaMemsetAsync(where, 0xFF, where_bytes, s) != cudaSuccess) { cudaGetLastError(); return GPUVM_E_CUDA; }
+                embag_bucket_fill_kernel<<<sm_count() * 8, 256, 0, s>>>(rows_ll, n_lookups, t_off, row_bytes, m.vm.page_shift,
+                                                                     rows_inside, demand, limit, bucket_off, cold_idx, where);
+                const size_t stage_bytes = (size_t)kEmbagMigrators * kEmbagStages * kEmbagChunk;
+                if (stage_bytes > 40 * 1024 &&
+                    cudaFuncSetAttribute(embag_direct_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes) != cudaSuccess) {
+                    cudaGetLastError();
+                    return GPUVM_E_CUDA;
+                }
+                const size_t warps_needed = n_bags > (size_t)host_counts[0] / 4 ? n_bags : (size_t)host_counts[0] / 4 + 1;
+                const size_t blocks_needed = (warps_needed + requesters - 1) / requesters;
+                const unsigned int grid = (unsigned int)(blocks_needed < (size_t)sm_count() ? blocks_needed : (size_t)sm_count());
+                embag_direct_kernel<<<grid, (requesters + migrators) * 32, stage_bytes, s>>>(
+                    m.vm, t_off, (unsigned int)dims, rows_ll, n_bags, (unsigned int)bag, d_out, requesters, shared_queue, limit,
+                    demand, cold_idx, where, cold_staging, counts);
+                return launched(2);
+            }
+        }
+    }
     // Groups of 32 bags per requester warp: enough for every bag to be in flight at once when
     // that takes at most kEmbagMaxGroups, within the scratch bound (table + staged rows).
     const size_t warps_all = (size_t)sm_count() * requesters;
