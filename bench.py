@@ -130,7 +130,7 @@ NCU_LINK_TRAFFIC = {
         "full size; sweep 1 of the four sweeps of a run, 95 % of its time"),
     4: (33554432 * 32 * 8 + (4 << 30), "vadd_kernel_cfg4_eighth_full_set.md", 33554432,
         "1/8 case x 8: 8 GiB in, plus the 4 GiB of c that go out"),
-    5: (60863056 * 32, "embag_batch_kernel_cfg5_counted_policy.md", 60863056,
+    5: (60863056 * 32, "embag_direct_kernel_cfg5_default_policy.md", 60863056,
         "full size, default policy; one metric, one pass"),
     "5_always_migrate": (134217728 * 32 * 16, "embag_batch_kernel_cfg5_sixteenth_full_set.md", 134217728,
                          "1/16 case x 16, every first touch fetching its page"),
