@@ -259,8 +259,11 @@ int gpuvm_set_inplace_divisor(gpuvm_t h, unsigned int divisor);
  * counted = 2 (default): the same, and when every lookup has a staging slot of its own (all bags in flight at once:
  * the default without gpuvm_set_scratch_limit) the lookups of the pages that are not fetched are bucketed by page
  * and their rows read page by page, at the link's sequential rate; the pages that are fetched are handed to the
- * migrator warps before the first lookup (unless they would fill more than half the pool).  Where that is not
- * possible it behaves like 1.
+ * migrator warps before the first lookup (unless they would fill more than half the pool).  When those pages
+ * fit the pool twice over they are also held in their frames for the length of the launch and their rows are
+ * added up straight from the frames: no request tables, and only the rows read in place are staged (the call then
+ * reads two counters back after its counting kernels, i.e. it synchronises with its stream once).  Where none of
+ * that is possible it behaves like 1.
  * counted = 0: the online form, which needs no pass over the list: the first `limit` requests that find a page
  * absent read their rows in place (counted in the frame field of the invalid entry), the next one fetches the
  * page.  Other values: GPUVM_E_ARG. */

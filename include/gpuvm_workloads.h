@@ -243,8 +243,10 @@ int gpuvm_vadd_f32(gpuvm_t h, size_t a_off, size_t b_off, size_t c_off, size_t n
  * inside the backing store entirely sets the sticky GPUVM_E_RANGE.
  * Which pages are fetched (gpuvm_set_inplace_divisor, gpuvm_set_inplace_counted in gpuvm.h): by default a short
  * kernel first counts the lookups per page (4 bytes of scratch per page); the rows of pages with fewer lookups than
- * a quarter of the page holds are read in place from the backing store (counted as bytes_direct, no fault, the page
- * table untouched), every other page is fetched at its first touch.  With the divisor 0 every first touch fetches
+ * the page holds rows are read in place from the backing store, page by page (counted as bytes_direct, no fault,
+ * the page table untouched), every other page is fetched once, and when those pages fit the pool twice over the
+ * rows are added up straight from their frames: the scratch is then 4 * dims + 4 bytes per row read in place and
+ * 4 bytes per lookup instead of the tables and staged rows described above.  With the divisor 0 every first touch fetches
  * its page, as in the paper.  The result is the same bit for bit; the table must not be written through the
  * runtime while the call runs.
  * gpuvm_embag_f32_unbatched: one warp per bag, one row request at a time through
