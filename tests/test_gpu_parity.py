@@ -438,6 +438,35 @@ def test_embag_rent_or_buy(B, frames, counted):
                 assert limit * 512 <= st["bytes_direct"] <= (limit + 31) * 512 * st["faults"]
 
 
+def test_embag_direct_form_stages_only_the_rows_read_in_place(B):
+    """When the pages that are fetched fit the pool twice over, the default policy holds them in their frames and
+    adds their rows up from there: the scratch is the rows read in place plus a few bytes per lookup, not a staged
+    copy of every row; with a pool too small for that the form with request tables runs and stages every row.
+    Either way the hold bits are gone afterwards (the checker would flag one) and the sums are the oracle's."""
+    import torch
+    page, dims, bag, n_rows, n_bags = 4096, 128, 8, 4096, 1500
+    t = inputs.fill_f32_pm1(np.empty(n_rows * dims, np.float32), n_rows * dims, inputs.config_seed(5))
+    rows = inputs.fill_zipf_rows(np.empty(n_bags * bag, np.int64), n_bags * bag, inputs.config_seed(5, 1), n_rows, 1.05)
+    ref = oracle.embag_f32_direct(t.reshape(n_rows, dims), rows, bag).reshape(-1)
+    per_page = np.bincount(rows // 8, minlength=n_rows // 8)
+    hot, cold_rows = int(np.count_nonzero(per_page >= 8)), int(per_page[per_page < 8].sum())
+    assert hot > 4 and cold_rows > 1000
+    ar = Arena(page, {"t": t})
+    every_row = n_bags * bag * dims * 4
+    for frames, direct in ((2 * hot, True), (2 * hot - 1, False)):
+        out = torch.zeros(n_bags * dims, dtype=torch.float32, device="cuda")
+        with paged(ar.host, page, frames) as h:
+            B.gpuvm_embag_f32(h, 0, dims, dev(rows), n_bags, bag, out)
+            st, ck = finish(h)
+            scratch = B.gpuvm_scratch_bytes(h)
+        assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32)), frames
+        assert ck["bad_state"] == 0 and st["bytes_direct"] == cold_rows * 512
+        if direct:
+            assert st["faults"] == hot and cold_rows * 512 <= scratch < cold_rows * 512 + every_row // 4 + (1 << 20)
+        else:
+            assert scratch >= every_row
+
+
 def test_embag_writes_its_sums_to_pinned_host_memory(B):
     """d_out may be pinned host memory: the kernel writes the bags' sums there itself, same bits."""
     import torch
