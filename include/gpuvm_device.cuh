@@ -70,7 +70,7 @@
 
 namespace gpuvm {
 
-/* ---- page-table entry: [state:2 @60][dirty @57][ref @56][frame:32 @24][refcount:24 @0]
+/* ---- page-table entry: [state:2 @60][hold @59][keep @58][dirty @57][ref @56][frame:32 @24][refcount:24 @0]
  *      (while the state is INVALID the frame field counts the requests served in place, see advance) */
 constexpr unsigned long long kRcMask = 0xFFFFFFull;
 constexpr unsigned long long kRcLimit = 1ull << 23;   /* a pin that would take the counter beyond this is refused */
